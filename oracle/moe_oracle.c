@@ -1,0 +1,292 @@
+/*
+ * moe_oracle.c -- TEST INFRASTRUCTURE, NOT THE PRODUCT.
+ *
+ * A plain, slow, host-only evaluation of the top-k gated SwiGLU Mixture-of-Experts
+ * layer forward pass, written out directly from its definition.  It exists only so
+ * that tests, the smoke check and the benchmark's CPU-baseline leg have something
+ * independent to compare the CUDA path against.  Nothing in the product may call it,
+ * and it shares no code, header, table or helper with the CUDA sources.
+ *
+ * What it follows (paper: "Kernel Analysis: FP8 MoE Kernel (Blackwell)", the Sec. 4.5
+ * description of the layer; Sec. 4.5 "Expert FFN computation" for the pipeline order):
+ *   - per token, k experts are chosen out of E candidates from the router scores;
+ *   - tokens are reordered so that each expert's tokens are contiguous
+ *     ("sort-scatter"), experts with no token are skipped;
+ *   - every chosen expert applies a gate and an up projection, combined through
+ *     SiLU, followed by a down projection;
+ *   - the k expert outputs of a token are summed with the routing weights.
+ * The paper leaves the scoring function open; the build's stated reading is
+ * softmax -> top-k -> renormalise with ties broken towards the lower expert index,
+ * w13 rows [0,I) = gate and [I,2I) = up, weights applied at the combine.
+ *
+ * Arithmetic type: every floating-point operation is done in REAL, which the build
+ * sets to float (liboracle_f32.so, the precision the layer is specified in) or to
+ * double (liboracle_f64.so, used to put an error bar on the float build).  bf16
+ * inputs are widened exactly.  No blocking, fusion or reordering: the loops below are
+ * the sums of the definition in index order.  OpenMP only distributes independent
+ * tokens over threads; it never splits a sum.
+ *
+ * Pins (tests/test_oracle_*.py): hand-computed closed forms, a NumPy float64
+ * brute-force evaluation of all E experts per token, library reductions
+ * (torch.softmax/topk, numpy stable argsort, torch matmul), and invariants
+ * (identical experts with k=E collapse to one dense MLP, weights sum to one,
+ * token-permutation equivariance, exact power-of-two scaling).
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#ifndef REAL
+#define REAL float
+#endif
+
+#define ORACLE_OK 0
+#define ORACLE_ERR_ARG (-1)
+#define ORACLE_ERR_MISSING_EXPERT (-2)
+#define ORACLE_ERR_NOMEM (-3)
+
+static inline REAL real_exp(REAL v) { return sizeof(REAL) == sizeof(float) ? (REAL)expf((float)v) : (REAL)exp((double)v); }
+
+/* bfloat16 is the upper half of an IEEE binary32: widening is exact. */
+static inline REAL bf16_to_real(uint16_t b) {
+    uint32_t u = (uint32_t)b << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (REAL)f;
+}
+
+int moe_oracle_real_bytes(void) { return (int)sizeof(REAL); }
+
+int moe_oracle_num_threads(void) {
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* Strict total order used for selection: expert a ranks before expert b when its
+ * logit is larger, or when the logits compare equal and a has the lower index.
+ * The comparison is on the raw fp32 logits (softmax is increasing, so this is the
+ * order of the probabilities, without depending on how exp rounds). */
+static inline int ranks_before(const float *l, int a, int b) {
+    return l[a] > l[b] || (l[a] == l[b] && a < b);
+}
+
+/* Router for one token: softmax over E logits, the k best experts in rank order,
+ * and their probabilities renormalised to sum to one.
+ *   logits [E] f32 -> ids [k] i32 (rank order), w [k] REAL.
+ * scratch p [E] REAL, taken [E] bytes. */
+static void route_token(const float *l, int E, int k, int32_t *ids, REAL *w, REAL *p, unsigned char *taken) {
+    /* softmax: p_e = exp(l_e - m) / sum_e' exp(l_e' - m), sums in ascending e */
+    float m = l[0];
+    for (int e = 1; e < E; ++e)
+        if (l[e] > m) m = l[e];
+    REAL S = 0;
+    for (int e = 0; e < E; ++e) {
+        p[e] = real_exp((REAL)l[e] - (REAL)m);
+        S += p[e];
+    }
+    for (int e = 0; e < E; ++e) p[e] = p[e] / S;
+    /* selection: k passes, each picking the best expert not yet taken */
+    memset(taken, 0, (size_t)E);
+    for (int j = 0; j < k; ++j) {
+        int best = -1;
+        for (int e = 0; e < E; ++e) {
+            if (taken[e]) continue;
+            if (best < 0 || ranks_before(l, e, best)) best = e;
+        }
+        taken[best] = 1;
+        ids[j] = best;
+    }
+    /* renormalise over the selected experts, ascending rank */
+    REAL D = 0;
+    for (int j = 0; j < k; ++j) D += p[ids[j]];
+    for (int j = 0; j < k; ++j) w[j] = p[ids[j]] / D;
+}
+
+/* Router for a batch.  router_logits [T,E] f32 -> topk_ids [T,k] i32, topk_w [T,k] REAL. */
+int moe_oracle_route(const float *router_logits, int T, int E, int k, int32_t *topk_ids, REAL *topk_w) {
+    if (T < 0 || E < 1 || k < 1 || k > E) return ORACLE_ERR_ARG;
+    REAL *p = (REAL *)malloc(sizeof(REAL) * (size_t)E);
+    unsigned char *taken = (unsigned char *)malloc((size_t)E);
+    if (!p || !taken) { free(p); free(taken); return ORACLE_ERR_NOMEM; }
+    for (int t = 0; t < T; ++t)
+        route_token(router_logits + (size_t)t * E, E, k, topk_ids + (size_t)t * k, topk_w + (size_t)t * k, p, taken);
+    free(p);
+    free(taken);
+    return ORACLE_OK;
+}
+
+/* Stable counting sort of the A = T*k assignments by expert ("sort-scatter").
+ * Flat assignment index a = t*k + j.
+ *   expert_offsets [E+1]: exclusive prefix sum of the per-expert counts
+ *   flat_to_sorted [A]  : position of assignment a in expert-contiguous order
+ *   sorted_to_flat [A]  : its inverse
+ * Within an expert, assignments keep their flat order. */
+int moe_oracle_permute(const int32_t *topk_ids, int T, int k, int E, int32_t *expert_offsets,
+                       int32_t *sorted_to_flat, int32_t *flat_to_sorted) {
+    if (T < 0 || E < 1 || k < 1) return ORACLE_ERR_ARG;
+    const long A = (long)T * k;
+    for (int e = 0; e <= E; ++e) expert_offsets[e] = 0;
+    for (long a = 0; a < A; ++a) {
+        if (topk_ids[a] < 0 || topk_ids[a] >= E) return ORACLE_ERR_ARG;
+        expert_offsets[topk_ids[a] + 1] += 1; /* counts, shifted by one */
+    }
+    for (int e = 0; e < E; ++e) expert_offsets[e + 1] += expert_offsets[e];
+    int32_t *next = (int32_t *)malloc(sizeof(int32_t) * (size_t)E);
+    if (!next) return ORACLE_ERR_NOMEM;
+    for (int e = 0; e < E; ++e) next[e] = expert_offsets[e];
+    for (long a = 0; a < A; ++a) {
+        int32_t pos = next[topk_ids[a]]++;
+        flat_to_sorted[a] = pos;
+        sorted_to_flat[pos] = (int32_t)a;
+    }
+    free(next);
+    return ORACLE_OK;
+}
+
+/* One expert applied to one token row (gate/up projections, SiLU, down projection):
+ *   g_i = sum_h x_h * w13[i,h],  u_i = sum_h x_h * w13[I+i,h],
+ *   s_i = g_i / (1 + exp(-g_i)) * u_i,
+ *   y_n = sum_i s_i * w2[n,i].
+ * x_row [H] bf16, w13_e [2I,H] bf16, w2_e [H,I] bf16 -> y [H] REAL; scratch s [I] REAL.
+ * Nothing is rounded to bf16 on the way. */
+static void expert_ffn_row(const uint16_t *x_row, const uint16_t *w13_e, const uint16_t *w2_e, int H, int I, REAL *y, REAL *s) {
+    for (int i = 0; i < I; ++i) {
+        const uint16_t *wg = w13_e + (size_t)i * H;
+        const uint16_t *wu = w13_e + (size_t)(I + i) * H;
+        REAL g = 0, u = 0;
+        for (int h = 0; h < H; ++h) {
+            REAL xv = bf16_to_real(x_row[h]);
+            g += xv * bf16_to_real(wg[h]);
+            u += xv * bf16_to_real(wu[h]);
+        }
+        s[i] = g / ((REAL)1 + real_exp(-g)) * u;
+    }
+    for (int n = 0; n < H; ++n) {
+        const uint16_t *wd = w2_e + (size_t)n * I;
+        REAL acc = 0;
+        for (int i = 0; i < I; ++i) acc += s[i] * bf16_to_real(wd[i]);
+        y[n] = acc;
+    }
+}
+
+int moe_oracle_expert_ffn(const uint16_t *x_row, const uint16_t *w13_e, const uint16_t *w2_e, int H, int I, REAL *y) {
+    if (H < 1 || I < 1) return ORACLE_ERR_ARG;
+    REAL *s = (REAL *)malloc(sizeof(REAL) * (size_t)I);
+    if (!s) return ORACLE_ERR_NOMEM;
+    expert_ffn_row(x_row, w13_e, w2_e, H, I, y, s);
+    free(s);
+    return ORACLE_OK;
+}
+
+/* The layer for a chosen list of tokens, with the experts given as a table of
+ * per-expert pointers (an entry may be NULL when no listed token routes to it, so a
+ * caller can keep only the needed experts in host memory).
+ *   x [T,H] bf16, router_logits [T,E] f32, w13_ptrs[e] -> [2I,H] bf16, w2_ptrs[e] -> [H,I] bf16,
+ *   tokens [n_tokens] (indices into [0,T)), out [n_tokens,H] REAL.
+ * out[i,:] = sum_{j ascending} topk_w[t,j] * expert_{ids[t,j]}(x[t,:]),  t = tokens[i]. */
+int moe_oracle_forward_sampled(const uint16_t *x, const float *router_logits, const uint16_t *const *w13_ptrs,
+                               const uint16_t *const *w2_ptrs, int T, int H, int I, int E, int k,
+                               const int32_t *tokens, int n_tokens, REAL *out) {
+    if (T < 0 || H < 1 || I < 1 || E < 1 || k < 1 || k > E || n_tokens < 0) return ORACLE_ERR_ARG;
+    int status = ORACLE_OK;
+#pragma omp parallel
+    {
+        REAL *p = (REAL *)malloc(sizeof(REAL) * (size_t)E);
+        unsigned char *taken = (unsigned char *)malloc((size_t)E);
+        int32_t *ids = (int32_t *)malloc(sizeof(int32_t) * (size_t)k);
+        REAL *w = (REAL *)malloc(sizeof(REAL) * (size_t)k);
+        REAL *s = (REAL *)malloc(sizeof(REAL) * (size_t)I);
+        REAL *y = (REAL *)malloc(sizeof(REAL) * (size_t)H);
+        if (!p || !taken || !ids || !w || !s || !y) {
+#pragma omp critical
+            status = ORACLE_ERR_NOMEM;
+        } else {
+#pragma omp for schedule(dynamic, 1)
+            for (int i = 0; i < n_tokens; ++i) {
+                const int t = tokens[i];
+                REAL *o = out + (size_t)i * H;
+                for (int n = 0; n < H; ++n) o[n] = 0;
+                if (t < 0 || t >= T) {
+#pragma omp critical
+                    status = ORACLE_ERR_ARG;
+                    continue;
+                }
+                route_token(router_logits + (size_t)t * E, E, k, ids, w, p, taken);
+                for (int j = 0; j < k; ++j) {
+                    const int e = ids[j];
+                    if (!w13_ptrs[e] || !w2_ptrs[e]) {
+#pragma omp critical
+                        status = ORACLE_ERR_MISSING_EXPERT;
+                        continue;
+                    }
+                    expert_ffn_row(x + (size_t)t * H, w13_ptrs[e], w2_ptrs[e], H, I, y, s);
+                    for (int n = 0; n < H; ++n) o[n] += w[j] * y[n];
+                }
+            }
+        }
+        free(p); free(taken); free(ids); free(w); free(s); free(y);
+    }
+    return status;
+}
+
+/* The whole layer on contiguous weights: w13 [E,2I,H] bf16, w2 [E,H,I] bf16 -> out [T,H] REAL. */
+int moe_oracle_forward(const uint16_t *x, const float *router_logits, const uint16_t *w13, const uint16_t *w2,
+                       int T, int H, int I, int E, int k, REAL *out) {
+    if (T < 0 || H < 1 || I < 1 || E < 1 || k < 1 || k > E) return ORACLE_ERR_ARG;
+    const uint16_t **p13 = (const uint16_t **)malloc(sizeof(void *) * (size_t)E);
+    const uint16_t **p2 = (const uint16_t **)malloc(sizeof(void *) * (size_t)E);
+    int32_t *tokens = (int32_t *)malloc(sizeof(int32_t) * (size_t)(T > 0 ? T : 1));
+    int status = ORACLE_ERR_NOMEM;
+    if (p13 && p2 && tokens) {
+        for (int e = 0; e < E; ++e) {
+            p13[e] = w13 + (size_t)e * 2 * I * H;
+            p2[e] = w2 + (size_t)e * H * I;
+        }
+        for (int t = 0; t < T; ++t) tokens[t] = t;
+        status = moe_oracle_forward_sampled(x, router_logits, p13, p2, T, H, I, E, k, tokens, T, out);
+    }
+    free(p13); free(p2); free(tokens);
+    return status;
+}
+
+/* The two halves of the layer around the sort-scatter, exposed so that tests can
+ * compare the CUDA path's intermediates in expert-contiguous order:
+ *   h [A,I]  = SiLU(gate) * up   per sorted assignment row,
+ *   y [A,H]  = down projection   per sorted assignment row.
+ * Row r of either belongs to flat assignment sorted_to_flat[r]. */
+int moe_oracle_sorted_intermediates(const uint16_t *x, const uint16_t *w13, const uint16_t *w2, const int32_t *topk_ids,
+                                    const int32_t *sorted_to_flat, int T, int H, int I, int E, int k, REAL *h, REAL *y) {
+    if (T < 0 || H < 1 || I < 1 || E < 1 || k < 1) return ORACLE_ERR_ARG;
+    const long A = (long)T * k;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (long r = 0; r < A; ++r) {
+        const int a = sorted_to_flat[r];
+        const int t = a / k, e = topk_ids[a];
+        const uint16_t *xr = x + (size_t)t * H;
+        const uint16_t *w13_e = w13 + (size_t)e * 2 * I * H;
+        const uint16_t *w2_e = w2 + (size_t)e * H * I;
+        REAL *hr = h + (size_t)r * I;
+        for (int i = 0; i < I; ++i) {
+            REAL g = 0, u = 0;
+            for (int c = 0; c < H; ++c) {
+                REAL xv = bf16_to_real(xr[c]);
+                g += xv * bf16_to_real(w13_e[(size_t)i * H + c]);
+                u += xv * bf16_to_real(w13_e[(size_t)(I + i) * H + c]);
+            }
+            hr[i] = g / ((REAL)1 + real_exp(-g)) * u;
+        }
+        for (int n = 0; n < H; ++n) {
+            REAL acc = 0;
+            for (int i = 0; i < I; ++i) acc += hr[i] * bf16_to_real(w2_e[(size_t)n * I + i]);
+            y[(size_t)r * H + n] = acc;
+        }
+    }
+    return ORACLE_OK;
+}

@@ -1,0 +1,162 @@
+"""ctypes loader for the CPU oracle (TEST INFRASTRUCTURE, not the product).
+
+Only tests, the smoke check and the benchmark's CPU-baseline / reference legs may import
+this module.  It compiles ``moe_oracle.c`` with gcc into two shared objects -- one with
+every floating-point operation in float (``f32``, the precision the layer is specified in)
+and one in double (``f64``, the error bar for the float build) -- and wraps their entry
+points with numpy-array marshalling.  It imports nothing from the CUDA package.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from pathlib import Path
+
+import numpy as np
+
+_HERE = Path(__file__).resolve().parent
+_SRC = _HERE / "moe_oracle.c"
+_BUILD = _HERE / "_build"
+
+_c_i32p = ctypes.POINTER(ctypes.c_int32)
+_c_f32p = ctypes.POINTER(ctypes.c_float)
+_c_u16p = ctypes.POINTER(ctypes.c_uint16)
+
+
+def build(force: bool = False) -> dict[str, Path]:
+    """Compile the oracle (gcc, OpenMP) for both arithmetic types; returns the .so paths."""
+    _BUILD.mkdir(exist_ok=True)
+    out = {}
+    for name, real in (("f32", "float"), ("f64", "double")):
+        so = _BUILD / f"liboracle_{name}.so"
+        if force or not so.exists() or so.stat().st_mtime < _SRC.stat().st_mtime:
+            tmp = so.with_suffix(f".{os.getpid()}.tmp")
+            cmd = ["gcc", "-std=c11", "-O2", "-fno-fast-math", "-ffp-contract=off", "-fopenmp", "-shared", "-fPIC",
+                   f"-DREAL={real}", str(_SRC), "-o", str(tmp), "-lm"]
+            subprocess.run(cmd, check=True)
+            os.replace(tmp, so)
+        out[name] = so
+    return out
+
+
+class Oracle:
+    """One precision build of the oracle.  Arrays in, arrays out; bf16 tensors travel as uint16."""
+
+    def __init__(self, precision: str = "f32"):
+        assert precision in ("f32", "f64")
+        self.precision = precision
+        self.real = np.float32 if precision == "f32" else np.float64
+        self.lib = ctypes.CDLL(str(build()[precision]))
+        assert self.lib.moe_oracle_real_bytes() == np.dtype(self.real).itemsize
+        for fn in ("moe_oracle_route", "moe_oracle_permute", "moe_oracle_expert_ffn", "moe_oracle_forward",
+                   "moe_oracle_forward_sampled", "moe_oracle_sorted_intermediates"):
+            getattr(self.lib, fn).restype = ctypes.c_int
+
+    # -- helpers ---------------------------------------------------------------------------
+    @staticmethod
+    def _ptr(a: np.ndarray):
+        return ctypes.c_void_p(a.ctypes.data)
+
+    @staticmethod
+    def _u16(a) -> np.ndarray:
+        a = np.ascontiguousarray(a)
+        assert a.dtype == np.uint16, "bf16 data must be passed as its uint16 bit pattern"
+        return a
+
+    @staticmethod
+    def _check(status: int, what: str):
+        if status != 0:
+            raise RuntimeError(f"{what} failed with oracle status {status}")
+
+    @property
+    def num_threads(self) -> int:
+        return int(self.lib.moe_oracle_num_threads())
+
+    # -- entry points ----------------------------------------------------------------------
+    def route(self, router_logits: np.ndarray, top_k: int):
+        l = np.ascontiguousarray(router_logits, dtype=np.float32)
+        T, E = l.shape
+        ids = np.empty((T, top_k), np.int32)
+        w = np.empty((T, top_k), self.real)
+        self._check(self.lib.moe_oracle_route(self._ptr(l), T, E, top_k, self._ptr(ids), self._ptr(w)), "route")
+        return ids, w
+
+    def permute(self, topk_ids: np.ndarray, E: int):
+        ids = np.ascontiguousarray(topk_ids, dtype=np.int32)
+        T, k = ids.shape
+        offsets = np.empty(E + 1, np.int32)
+        s2f = np.empty(T * k, np.int32)
+        f2s = np.empty(T * k, np.int32)
+        self._check(self.lib.moe_oracle_permute(self._ptr(ids), T, k, E, self._ptr(offsets), self._ptr(s2f),
+                                                self._ptr(f2s)), "permute")
+        return offsets, s2f, f2s
+
+    def expert_ffn(self, x_row, w13_e, w2_e):
+        x_row, w13_e, w2_e = self._u16(x_row), self._u16(w13_e), self._u16(w2_e)
+        H = x_row.shape[0]
+        I = w13_e.shape[0] // 2
+        assert w13_e.shape == (2 * I, H) and w2_e.shape == (H, I)
+        y = np.empty(H, self.real)
+        self._check(self.lib.moe_oracle_expert_ffn(self._ptr(x_row), self._ptr(w13_e), self._ptr(w2_e), H, I,
+                                                   self._ptr(y)), "expert_ffn")
+        return y
+
+    def forward(self, x, router_logits, w13, w2, top_k: int):
+        x, w13, w2 = self._u16(x), self._u16(w13), self._u16(w2)
+        l = np.ascontiguousarray(router_logits, dtype=np.float32)
+        T, H = x.shape
+        E, I2, _ = w13.shape
+        I = I2 // 2
+        assert w13.shape == (E, 2 * I, H) and w2.shape == (E, H, I) and l.shape == (T, E)
+        out = np.empty((T, H), self.real)
+        self._check(self.lib.moe_oracle_forward(self._ptr(x), self._ptr(l), self._ptr(w13), self._ptr(w2), T, H, I, E,
+                                                top_k, self._ptr(out)), "forward")
+        return out
+
+    def forward_sampled(self, x, router_logits, experts: dict, I: int, top_k: int, tokens):
+        """Layer output for the listed tokens.  ``experts`` maps expert id -> (w13_e, w2_e) uint16
+        arrays; only the experts those tokens route to need to be present."""
+        x = self._u16(x)
+        l = np.ascontiguousarray(router_logits, dtype=np.float32)
+        T, H = x.shape
+        E = l.shape[1]
+        tokens = np.ascontiguousarray(tokens, dtype=np.int32)
+        p13 = (ctypes.c_void_p * E)()
+        p2 = (ctypes.c_void_p * E)()
+        keep = []
+        for e, (a, b) in experts.items():
+            a, b = self._u16(a), self._u16(b)
+            assert a.shape == (2 * I, H) and b.shape == (H, I)
+            keep.append((a, b))
+            p13[e] = a.ctypes.data
+            p2[e] = b.ctypes.data
+        out = np.empty((len(tokens), H), self.real)
+        self._check(self.lib.moe_oracle_forward_sampled(self._ptr(x), self._ptr(l), p13, p2, T, H, I, E, top_k,
+                                                        self._ptr(tokens), len(tokens), self._ptr(out)),
+                    "forward_sampled")
+        return out
+
+    def sorted_intermediates(self, x, w13, w2, topk_ids, sorted_to_flat):
+        x, w13, w2 = self._u16(x), self._u16(w13), self._u16(w2)
+        ids = np.ascontiguousarray(topk_ids, dtype=np.int32)
+        s2f = np.ascontiguousarray(sorted_to_flat, dtype=np.int32)
+        T, H = x.shape
+        E, I2, _ = w13.shape
+        I = I2 // 2
+        k = ids.shape[1]
+        h = np.empty((T * k, I), self.real)
+        y = np.empty((T * k, H), self.real)
+        self._check(self.lib.moe_oracle_sorted_intermediates(self._ptr(x), self._ptr(w13), self._ptr(w2),
+                                                             self._ptr(ids), self._ptr(s2f), T, H, I, E, k,
+                                                             self._ptr(h), self._ptr(y)), "sorted_intermediates")
+        return h, y
+
+
+_cache: dict[str, Oracle] = {}
+
+
+def get(precision: str = "f32") -> Oracle:
+    if precision not in _cache:
+        _cache[precision] = Oracle(precision)
+    return _cache[precision]

@@ -1,0 +1,79 @@
+"""Seeded synthetic inputs for the MoE layer (shapes, dtypes and distributions of the
+benchmark workloads).  This module only draws random numbers and reshapes them: it holds
+none of the layer's arithmetic, and it is the one module that both the CUDA path's callers
+and the CPU oracle's callers share.
+
+Recipe (all draws from one ``torch.Generator`` seeded per workload, in the order
+x, router_logits, w13, w2):
+  x              [T,H]     N(0,1)            drawn in fp32, rounded to bf16
+  router_logits  [T,E]     N(0,1) fp32       (+ a per-expert bias for the skewed workload)
+  w13            [E,2I,H]  N(0,1/H)          std H**-0.5, drawn in fp32, rounded to bf16
+  w2             [E,H,I]   N(0,1/I)          std I**-0.5, drawn in fp32, rounded to bf16
+The skewed workload adds bias_e = 2*ln(1/(e+1)**1.1) = -2.2*ln(e+1) to every token's logit of
+expert e, so a few low-index experts receive most tokens and most experts receive none.
+The bytes produced are what both sides consume; a CPU generator and a CUDA generator give
+different streams, so a test draws once and hands the same tensors to both sides.
+"""
+from __future__ import annotations
+
+import math
+
+import numpy as np
+import torch
+
+CONFIGS = {
+    # name: T tokens, H hidden, I intermediate, E experts, top_k, zipf-biased router
+    "tiny": dict(T=16, H=256, I=512, E=8, top_k=2, skew=False),
+    "mixtral": dict(T=512, H=4096, I=14336, E=8, top_k=2, skew=False),
+    "dsv3_decode": dict(T=128, H=7168, I=2048, E=256, top_k=8, skew=False),
+    "dsv3_prefill": dict(T=8192, H=7168, I=2048, E=256, top_k=8, skew=False),
+    "skewed": dict(T=4096, H=4096, I=1536, E=128, top_k=8, skew=True),
+}
+
+
+def zipf_bias(E: int) -> torch.Tensor:
+    rank = torch.arange(1, E + 1, dtype=torch.float32)
+    return (-2.2 * torch.log(rank)).to(torch.float32)
+
+
+def _normal_bf16(shape, std: float, gen: torch.Generator, device, chunk_elems: int = 1 << 28) -> torch.Tensor:
+    """N(0, std^2) in bf16, drawn in fp32 slabs along dim 0 so the fp32 temporary stays small."""
+    out = torch.empty(shape, dtype=torch.bfloat16, device=device)
+    rows = shape[0]
+    per_row = int(np.prod(shape[1:])) if len(shape) > 1 else 1
+    step = max(1, chunk_elems // max(per_row, 1))
+    for r0 in range(0, rows, step):
+        r1 = min(rows, r0 + step)
+        slab = torch.randn((r1 - r0, *shape[1:]), generator=gen, device=device, dtype=torch.float32)
+        if std != 1.0:
+            slab.mul_(std)
+        out[r0:r1] = slab.to(torch.bfloat16)
+    return out
+
+
+def make_inputs(cfg, seed: int = 0, device="cpu") -> dict:
+    """Draw one workload.  ``cfg`` is a name in CONFIGS or a dict with T,H,I,E,top_k[,skew]."""
+    if isinstance(cfg, str):
+        cfg = CONFIGS[cfg]
+    T, H, I, E = cfg["T"], cfg["H"], cfg["I"], cfg["E"]
+    device = torch.device(device)
+    gen = torch.Generator(device=device)
+    gen.manual_seed(seed)
+    x = _normal_bf16((T, H), 1.0, gen, device)
+    logits = torch.randn((T, E), generator=gen, device=device, dtype=torch.float32)
+    if cfg.get("skew", False):
+        logits = logits + zipf_bias(E).to(device)
+    w13 = _normal_bf16((E, 2 * I, H), 1.0 / math.sqrt(H), gen, device)
+    w2 = _normal_bf16((E, H, I), 1.0 / math.sqrt(I), gen, device)
+    return dict(x=x, router_logits=logits.contiguous(), w13=w13, w2=w2, T=T, H=H, I=I, E=E, top_k=cfg["top_k"])
+
+
+def bf16_bits(t: torch.Tensor) -> np.ndarray:
+    """The uint16 bit pattern of a bf16 tensor, on the host, as a numpy array."""
+    assert t.dtype == torch.bfloat16
+    return t.detach().cpu().contiguous().view(torch.int16).numpy().view(np.uint16)
+
+
+def bits_to_f64(bits: np.ndarray) -> np.ndarray:
+    """Widen bf16 bit patterns exactly to float64."""
+    return (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
