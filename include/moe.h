@@ -1,0 +1,158 @@
+/*
+ * moe.h -- C ABI of the B200 (sm_100a) fused Mixture-of-Experts layer forward pass.
+ *
+ * The layer (K-Search paper, Sec. 4.5 "Kernel Analysis: FP8 MoE Kernel (Blackwell)"): for each
+ * token the top-k experts are chosen out of E from the router scores; tokens are reordered so
+ * that every expert's tokens are contiguous ("sort-scatter", Sec. 4.5 "Expert FFN computation");
+ * each chosen expert applies a gate and an up projection combined through SiLU, then a down
+ * projection; the k results of a token are summed with the routing weights.  This library
+ * computes it in bf16 with fp32 accumulation:
+ *
+ *   router   p = softmax(router_logits[t,:]); topk_ids[t,0..k) = the k largest logits, ties to the
+ *            lower expert index, listed from largest to smallest; topk_weights = p[ids] / sum p[ids]
+ *   permute  stable counting sort of the A = T*k assignments (flat index a = t*k + j) by expert:
+ *            expert_offsets[E+1] (exclusive prefix sum of per-expert counts),
+ *            flat_to_sorted[a] = position of a in expert-contiguous order, sorted_to_flat = inverse
+ *   gemm1    h[r,:] = SiLU(x[t(r),:] . w13[e, 0:I, :]^T) * (x[t(r),:] . w13[e, I:2I, :]^T)   (bf16)
+ *   gemm2    y[r,:] = h[r,:] . w2[e,:,:]^T                                                    (bf16)
+ *   combine  out[t,:] = sum_{j ascending} topk_weights[t,j] * y[flat_to_sorted[t*k+j],:]      (bf16)
+ *
+ * Conventions for every entry point
+ *   - All tensors are row-major with the last index contiguous.  bf16 data is passed as void*.
+ *   - Unless a parameter says HOST, every pointer is a DEVICE pointer owned by the caller and
+ *     valid on the current device.  The library allocates and frees no device memory, launches
+ *     only on the given stream (a cudaStream_t passed as void*, NULL = default stream) and does
+ *     not synchronise it, except where stated.
+ *   - Inputs are read-only and must not alias outputs or the workspace.
+ *   - The return value is a moe_status_t: 0 on success, negative on error.  Arguments are
+ *     checked on the host before anything is launched; on an error nothing has been launched.
+ *   - Supported envelope: 1 <= E <= 256, 1 <= top_k <= min(E, 32), H % 64 == 0, I % 64 == 0,
+ *     H % 128 == 0, T >= 0, T*top_k < 2^27.  T == 0 succeeds without a launch.
+ *     Pointers must be 16-byte aligned, the workspace 256-byte aligned.
+ *   - Device-side waits are bounded.  If one expires (which indicates a bug, not bad input) the
+ *     kernel records MOE_ERR_DEVICE_TIMEOUT in the workspace's status word and returns; read it
+ *     with moe_last_status().
+ *   - Results are deterministic: no floating-point atomics, no split accumulation; two calls on
+ *     the same inputs give bit-identical outputs.
+ */
+#ifndef MOE_B200_H_
+#define MOE_B200_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define MOE_API __attribute__((visibility("default")))
+#else
+#define MOE_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    MOE_OK = 0,
+    MOE_ERR_NULL = -1,           /* a required pointer is NULL */
+    MOE_ERR_SHAPE = -2,          /* a size is negative, zero where it must not be, or top_k > E */
+    MOE_ERR_UNSUPPORTED = -3,    /* outside the supported envelope (see above) */
+    MOE_ERR_ALIGN = -4,          /* a pointer is not aligned as required */
+    MOE_ERR_WORKSPACE = -5,      /* workspace_bytes is smaller than moe_*_workspace_bytes() */
+    MOE_ERR_CUDA = -6,           /* a CUDA runtime/driver call failed (launch, descriptor encoding) */
+    MOE_ERR_DEVICE_TIMEOUT = -7, /* a bounded device-side wait expired (reported by moe_last_status) */
+    MOE_ERR_ARCH = -8            /* the current device is not compute capability 10.x */
+} moe_status_t;
+
+/* Flags for moe_forward_ex. */
+#define MOE_FLAG_NONE 0u
+/* Run the two grouped GEMMs on plain CUDA-core kernels instead of the tcgen05 kernels.  Meant
+ * for validating the tensor-core path at sizes the CPU cannot check in full; about 100x slower. */
+#define MOE_FLAG_VALIDATION_GEMM 1u
+
+/* Byte offsets of the intermediates inside the workspace of moe_forward (so tests and tools can
+ * read them after the stream has been synchronised).  Filled by moe_workspace_layout(). */
+typedef struct {
+    size_t total_bytes;
+    size_t status;          /* int32[4]: status, site, aux0, aux1 */
+    size_t topk_ids;        /* int32 [T,k] */
+    size_t topk_weights;    /* f32   [T,k] */
+    size_t expert_offsets;  /* int32 [E+1] */
+    size_t sorted_to_flat;  /* int32 [A] */
+    size_t flat_to_sorted;  /* int32 [A] */
+    size_t route_scratch;   /* router/permute scratch (per-chunk histograms, tile schedule) */
+    size_t x_perm;          /* bf16 [A,H]: rows of x in expert-contiguous order */
+    size_t h;               /* bf16 [A,I] */
+    size_t y;               /* bf16 [A,H] */
+    size_t staging;         /* used only by moe_forward_host: device copies of x, logits, out */
+} moe_workspace_layout_t;
+
+/* Host-only, pure.  Size in bytes of the workspace moe_forward / moe_forward_host need for this
+ * problem; 0 if the problem is outside the supported envelope.  (Sec. 4.5: the intermediates are
+ * the sort-scatter's reordered tokens and the two projections' results.) */
+MOE_API size_t moe_workspace_bytes(int T, int H, int I, int E, int top_k);
+
+/* Host-only, pure.  Fills *layout for the same problem; MOE_ERR_UNSUPPORTED outside the envelope. */
+MOE_API int moe_workspace_layout(int T, int H, int I, int E, int top_k, moe_workspace_layout_t *layout);
+
+/* Host-only, pure.  Workspace bytes needed by moe_route alone; 0 if unsupported. */
+MOE_API size_t moe_route_workspace_bytes(int T, int E, int top_k);
+
+/* Router + sort-scatter (Sec. 4.5 "Routing" and step (2) of "Expert FFN computation").
+ *   router_logits  [T,E] f32, in
+ *   topk_ids       [T,k] int32, out: chosen experts in rank order
+ *   topk_weights   [T,k] f32,   out: renormalised softmax probabilities (sum to 1 per token)
+ *   expert_offsets [E+1] int32, out
+ *   sorted_to_flat [T*k] int32, out
+ *   flat_to_sorted [T*k] int32, out
+ *   workspace      scratch of at least moe_route_workspace_bytes(T,E,top_k) bytes; contents
+ *                  undefined afterwards.  Concurrent calls need distinct workspaces.
+ * Non-finite logits are outside the contract but the kernels still terminate and stay in bounds. */
+MOE_API int moe_route(const float *router_logits, int T, int E, int top_k, int32_t *topk_ids, float *topk_weights,
+              int32_t *expert_offsets, int32_t *sorted_to_flat, int32_t *flat_to_sorted, void *workspace,
+              size_t workspace_bytes, void *stream);
+
+/* The whole layer (Sec. 4.5: routing, sort-scatter, gate+up with SiLU, down projection; then the
+ * weighted combine).
+ *   x              [T,H]    bf16, in
+ *   router_logits  [T,E]    f32,  in
+ *   w13            [E,2I,H] bf16, in: rows [0,I) of an expert are the gate projection, [I,2I) the up projection
+ *   w2             [E,H,I]  bf16, in
+ *   out            [T,H]    bf16, out
+ *   workspace      at least moe_workspace_bytes(T,H,I,E,top_k) bytes, 256-byte aligned.  Holds the
+ *                  routing arrays and intermediates at the offsets moe_workspace_layout() reports;
+ *                  they stay valid until the next call that uses this workspace.
+ * Launches seven kernels on `stream` and returns without waiting for them. */
+MOE_API int moe_forward(const void *x, const float *router_logits, const void *w13, const void *w2, int T, int H, int I,
+                int E, int top_k, void *out, void *workspace, size_t workspace_bytes, void *stream);
+
+/* moe_forward with option flags (MOE_FLAG_*). */
+MOE_API int moe_forward_ex(const void *x, const float *router_logits, const void *w13, const void *w2, int T, int H, int I,
+                   int E, int top_k, void *out, void *workspace, size_t workspace_bytes, void *stream,
+                   unsigned flags);
+
+/* moe_forward for a caller whose activations live in HOST memory: x_host [T,H] bf16 and
+ * router_logits_host [T,E] f32 are HOST pointers (pinned memory makes the copies asynchronous),
+ * out_host [T,H] bf16 is a HOST pointer; the expert weights w13 / w2 stay DEVICE pointers
+ * (they are model parameters, resident across calls).  The call enqueues, on `stream`, the
+ * host-to-device copies into the workspace's staging area, the layer, and the device-to-host
+ * copy of the result, and returns without synchronising: out_host is valid once the stream
+ * has been synchronised. */
+MOE_API int moe_forward_host(const void *x_host, const float *router_logits_host, const void *w13, const void *w2, int T,
+                     int H, int I, int E, int top_k, void *out_host, void *workspace, size_t workspace_bytes,
+                     void *stream);
+
+/* Synchronises `stream`, then reads the status word the kernels of the last moe_forward /
+ * moe_route call left in `workspace`.  MOE_OK, MOE_ERR_DEVICE_TIMEOUT, or MOE_ERR_CUDA if the
+ * stream reports an error. */
+MOE_API int moe_last_status(const void *workspace, void *stream);
+
+/* Number of kernels moe_forward_ex launches for this problem with these flags (0 when T == 0). */
+MOE_API int moe_forward_launch_count(int T, unsigned flags);
+
+/* Static, NUL-terminated description of a status code. */
+MOE_API const char *moe_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MOE_B200_H_ */

@@ -1,0 +1,170 @@
+"""Thin ctypes binding over the C-ABI library (``include/moe.h``).
+
+Argument marshalling only: every step of the layer runs in the library's CUDA kernels.  There is
+no CPU path and no fallback -- if ``libmoe_b200.so`` is missing or a call fails, this raises.
+PyTorch is used for device memory and streams.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+
+import torch
+
+_LIB_PATH = Path(__file__).resolve().parent / "libmoe_b200.so"
+
+MOE_OK = 0
+MOE_FLAG_NONE = 0
+MOE_FLAG_VALIDATION_GEMM = 1
+
+EXPORTED = ["moe_workspace_bytes", "moe_workspace_layout", "moe_route_workspace_bytes", "moe_route", "moe_forward",
+            "moe_forward_ex", "moe_forward_host", "moe_last_status", "moe_forward_launch_count", "moe_status_string"]
+
+
+class MoeError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        super().__init__(f"{what}: status {status} ({moe_status_string(status)})")
+
+
+class WorkspaceLayout(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_size_t) for n in
+                ("total_bytes", "status", "topk_ids", "topk_weights", "expert_offsets", "sorted_to_flat",
+                 "flat_to_sorted", "route_scratch", "x_perm", "h", "y", "staging")]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded shared library.  Raises if it has not been built (python -m paper_2602_19128_b200.build)."""
+    global _lib
+    if _lib is None:
+        if not _LIB_PATH.exists():
+            raise FileNotFoundError(f"{_LIB_PATH} is missing: build it with `python -m paper_2602_19128_b200.build`; "
+                                    "there is no fallback path")
+        L = ctypes.CDLL(str(_LIB_PATH))
+        i, sz, vp = ctypes.c_int, ctypes.c_size_t, ctypes.c_void_p
+        L.moe_workspace_bytes.restype = sz
+        L.moe_workspace_bytes.argtypes = [i] * 5
+        L.moe_workspace_layout.restype = i
+        L.moe_workspace_layout.argtypes = [i] * 5 + [ctypes.POINTER(WorkspaceLayout)]
+        L.moe_route_workspace_bytes.restype = sz
+        L.moe_route_workspace_bytes.argtypes = [i] * 3
+        L.moe_route.restype = i
+        L.moe_route.argtypes = [vp, i, i, i, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.moe_forward.restype = i
+        L.moe_forward.argtypes = [vp, vp, vp, vp, i, i, i, i, i, vp, vp, sz, vp]
+        L.moe_forward_ex.restype = i
+        L.moe_forward_ex.argtypes = [vp, vp, vp, vp, i, i, i, i, i, vp, vp, sz, vp, ctypes.c_uint]
+        L.moe_forward_host.restype = i
+        L.moe_forward_host.argtypes = [vp, vp, vp, vp, i, i, i, i, i, vp, vp, sz, vp]
+        L.moe_last_status.restype = i
+        L.moe_last_status.argtypes = [vp, vp]
+        L.moe_forward_launch_count.restype = i
+        L.moe_forward_launch_count.argtypes = [i, ctypes.c_uint]
+        L.moe_status_string.restype = ctypes.c_char_p
+        L.moe_status_string.argtypes = [i]
+        _lib = L
+    return _lib
+
+
+def _ptr(t):
+    if t is None:
+        return None
+    assert t.is_contiguous(), "tensors must be contiguous"
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> ctypes.c_void_p:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def moe_status_string(status: int) -> str:
+    return lib().moe_status_string(int(status)).decode()
+
+
+def moe_workspace_bytes(T: int, H: int, I: int, E: int, top_k: int) -> int:
+    return int(lib().moe_workspace_bytes(T, H, I, E, top_k))
+
+
+def moe_route_workspace_bytes(T: int, E: int, top_k: int) -> int:
+    return int(lib().moe_route_workspace_bytes(T, E, top_k))
+
+
+def moe_workspace_layout(T: int, H: int, I: int, E: int, top_k: int) -> WorkspaceLayout:
+    L = WorkspaceLayout()
+    st = lib().moe_workspace_layout(T, H, I, E, top_k, ctypes.byref(L))
+    if st != MOE_OK:
+        raise MoeError(st, "moe_workspace_layout")
+    return L
+
+
+def moe_forward_launch_count(T: int, flags: int = 0) -> int:
+    return int(lib().moe_forward_launch_count(T, flags))
+
+
+def alloc_workspace(nbytes: int, device="cuda") -> torch.Tensor:
+    """A 256-byte aligned device buffer of at least ``nbytes`` (torch's allocator aligns to 512)."""
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+def moe_route(router_logits, top_k: int, topk_ids, topk_weights, expert_offsets, sorted_to_flat, flat_to_sorted,
+              workspace, stream=None, check: bool = True) -> int:
+    T, E = router_logits.shape
+    st = lib().moe_route(_ptr(router_logits), T, E, top_k, _ptr(topk_ids), _ptr(topk_weights), _ptr(expert_offsets),
+                         _ptr(sorted_to_flat), _ptr(flat_to_sorted), _ptr(workspace), workspace.numel(),
+                         _stream(stream))
+    if check and st != MOE_OK:
+        raise MoeError(st, "moe_route")
+    return st
+
+
+def moe_forward(x, router_logits, w13, w2, top_k: int, out, workspace, stream=None, flags: int = 0,
+                check: bool = True) -> int:
+    T, H = x.shape
+    E, I2, _ = w13.shape
+    st = lib().moe_forward_ex(_ptr(x), _ptr(router_logits), _ptr(w13), _ptr(w2), T, H, I2 // 2, E, top_k, _ptr(out),
+                              _ptr(workspace), workspace.numel(), _stream(stream), flags)
+    if check and st != MOE_OK:
+        raise MoeError(st, "moe_forward")
+    return st
+
+
+def moe_forward_host(x_host, router_logits_host, w13, w2, top_k: int, out_host, workspace, stream=None,
+                     check: bool = True) -> int:
+    """x_host / router_logits_host / out_host are CPU tensors (pinned for asynchronous copies)."""
+    T, H = x_host.shape
+    E, I2, _ = w13.shape
+    st = lib().moe_forward_host(_ptr(x_host), _ptr(router_logits_host), _ptr(w13), _ptr(w2), T, H, I2 // 2, E, top_k,
+                                _ptr(out_host), _ptr(workspace), workspace.numel(), _stream(stream))
+    if check and st != MOE_OK:
+        raise MoeError(st, "moe_forward_host")
+    return st
+
+
+def moe_last_status(workspace, stream=None) -> int:
+    return int(lib().moe_last_status(_ptr(workspace), _stream(stream)))
+
+
+def workspace_views(workspace: torch.Tensor, T: int, H: int, I: int, E: int, top_k: int) -> dict:
+    """Typed views of the routing arrays and intermediates a moe_forward call left in ``workspace``."""
+    L = moe_workspace_layout(T, H, I, E, top_k)
+    A = T * top_k
+
+    def view(off, nbytes, dtype, shape):
+        return workspace[off:off + nbytes].view(dtype).view(shape)
+
+    return dict(
+        status=view(L.status, 16, torch.int32, (4,)),
+        topk_ids=view(L.topk_ids, A * 4, torch.int32, (T, top_k)),
+        topk_weights=view(L.topk_weights, A * 4, torch.float32, (T, top_k)),
+        expert_offsets=view(L.expert_offsets, (E + 1) * 4, torch.int32, (E + 1,)),
+        sorted_to_flat=view(L.sorted_to_flat, A * 4, torch.int32, (A,)),
+        flat_to_sorted=view(L.flat_to_sorted, A * 4, torch.int32, (A,)),
+        x_perm=view(L.x_perm, A * H * 2, torch.bfloat16, (A, H)),
+        h=view(L.h, A * I * 2, torch.bfloat16, (A, I)),
+        y=view(L.y, A * H * 2, torch.bfloat16, (A, H)),
+    )

@@ -1,0 +1,220 @@
+// C ABI of the MoE library: argument checking, workspace layout, and the launch sequence
+//   router+histogram -> scan+schedule -> stable scatter -> gather rows -> gemm1 (SwiGLU) -> gemm2 -> combine
+// (paper, Sec. 4.5: routing, sort-scatter, gate+up with SiLU, down projection; then the weighted sum).
+#include "moe_internal.cuh"
+
+namespace {
+
+using namespace moe;
+
+bool envelope_ok(long long T, int H, int I, int E, int k) {
+    if (E < 1 || E > kMaxExperts || k < 1 || k > E || k > kMaxTopK) return false;
+    if (H < 128 || I < 64 || H % 128 != 0 || I % 64 != 0) return false;
+    if (T < 0 || T * k >= (1LL << 27)) return false;
+    return true;
+}
+
+bool route_envelope_ok(long long T, int E, int k) {
+    return !(E < 1 || E > kMaxExperts || k < 1 || k > E || k > kMaxTopK || T < 0 || T * k >= (1LL << 27));
+}
+
+bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+void fill_layout(int T, int H, int I, int E, int k, moe_workspace_layout_t *L) {
+    const size_t A = (size_t)T * k;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t at = off; off += align_up(bytes, 256); return at; };
+    L->status = take(kStatusInts * sizeof(int));
+    L->topk_ids = take(A * sizeof(int));
+    L->topk_weights = take(A * sizeof(float));
+    L->expert_offsets = take((size_t)(E + 1) * sizeof(int));
+    L->sorted_to_flat = take(A * sizeof(int));
+    L->flat_to_sorted = take(A * sizeof(int));
+    L->route_scratch = take(route_scratch_bytes(T, E));
+    L->x_perm = take(A * H * 2);
+    L->h = take(A * I * 2);
+    L->y = take(A * H * 2);
+    L->staging = take((size_t)T * H * 2) /* x */;
+    take((size_t)T * E * sizeof(float)) /* logits */;
+    take((size_t)T * H * 2) /* out */;
+    L->total_bytes = off;
+}
+
+int check_device() {
+    int dev = 0, major = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return MOE_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return MOE_ERR_CUDA;
+    return major == 10 ? MOE_OK : MOE_ERR_ARCH;
+}
+
+int forward_impl(const void *x, const float *logits, const void *w13, const void *w2, int T, int H, int I, int E, int k,
+                 void *out, void *workspace, size_t workspace_bytes, cudaStream_t stream, unsigned flags) {
+    if (T < 0 || H <= 0 || I <= 0 || E <= 0 || k <= 0 || k > E) return MOE_ERR_SHAPE;
+    if (!envelope_ok(T, H, I, E, k)) return MOE_ERR_UNSUPPORTED;
+    if (flags & ~MOE_FLAG_VALIDATION_GEMM) return MOE_ERR_UNSUPPORTED;
+    if (T == 0) return MOE_OK;
+    if (!x || !logits || !w13 || !w2 || !out || !workspace) return MOE_ERR_NULL;
+    if (!aligned(x, 16) || !aligned(logits, 16) || !aligned(w13, 16) || !aligned(w2, 16) || !aligned(out, 16) ||
+        !aligned(workspace, 256))
+        return MOE_ERR_ALIGN;
+    moe_workspace_layout_t L;
+    fill_layout(T, H, I, E, k, &L);
+    if (workspace_bytes < L.total_bytes) return MOE_ERR_WORKSPACE;
+    const int arch = check_device();
+    if (arch != MOE_OK) return arch;
+
+    char *ws = static_cast<char *>(workspace);
+    int *status = reinterpret_cast<int *>(ws + L.status);
+    int *ids = reinterpret_cast<int *>(ws + L.topk_ids);
+    float *wts = reinterpret_cast<float *>(ws + L.topk_weights);
+    int *offsets = reinterpret_cast<int *>(ws + L.expert_offsets);
+    int *s2f = reinterpret_cast<int *>(ws + L.sorted_to_flat);
+    int *f2s = reinterpret_cast<int *>(ws + L.flat_to_sorted);
+    RouteScratch rs = carve_route_scratch(ws + L.route_scratch, T, E);
+    __nv_bfloat16 *x_perm = reinterpret_cast<__nv_bfloat16 *>(ws + L.x_perm);
+    __nv_bfloat16 *h = reinterpret_cast<__nv_bfloat16 *>(ws + L.h);
+    __nv_bfloat16 *y = reinterpret_cast<__nv_bfloat16 *>(ws + L.y);
+    const int A = T * k;
+    const int nt_max = choose_nt_max(T, E, k);
+
+    if (launch_route(logits, T, E, k, nt_max, ids, wts, offsets, s2f, f2s, rs, status, stream) != cudaSuccess)
+        return MOE_ERR_CUDA;
+    if (launch_gather_rows(static_cast<const __nv_bfloat16 *>(x), s2f, A, k, H, x_perm, stream) != cudaSuccess)
+        return MOE_ERR_CUDA;
+
+    GroupedGemmArgs g1;
+    g1.act = x_perm; g1.w = static_cast<const __nv_bfloat16 *>(w13); g1.out = h;
+    g1.A = A; g1.K = H; g1.n_out = I; g1.E = E; g1.w_rows = 2 * I; g1.nt_max = nt_max;
+    g1.expert_offsets = offsets; g1.tile_prefix = rs.tile_prefix; g1.tile_rows = rs.tile_rows;
+    g1.status = status; g1.swiglu = true;
+    GroupedGemmArgs g2 = g1;
+    g2.act = h; g2.w = static_cast<const __nv_bfloat16 *>(w2); g2.out = y;
+    g2.K = I; g2.n_out = H; g2.w_rows = H; g2.swiglu = false;
+
+    if (flags & MOE_FLAG_VALIDATION_GEMM) {
+        if (launch_grouped_gemm_validation(g1, stream) != cudaSuccess) return MOE_ERR_CUDA;
+        if (launch_grouped_gemm_validation(g2, stream) != cudaSuccess) return MOE_ERR_CUDA;
+    } else {
+        int st = launch_grouped_gemm_tc(g1, stream);
+        if (st != MOE_OK) return st;
+        st = launch_grouped_gemm_tc(g2, stream);
+        if (st != MOE_OK) return st;
+    }
+    if (launch_combine(y, wts, f2s, T, k, H, static_cast<__nv_bfloat16 *>(out), stream) != cudaSuccess)
+        return MOE_ERR_CUDA;
+    return MOE_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t moe_workspace_bytes(int T, int H, int I, int E, int top_k) {
+    if (!envelope_ok(T, H, I, E, top_k)) return 0;
+    moe_workspace_layout_t L;
+    fill_layout(T, H, I, E, top_k, &L);
+    return L.total_bytes;
+}
+
+int moe_workspace_layout(int T, int H, int I, int E, int top_k, moe_workspace_layout_t *layout) {
+    if (!layout) return MOE_ERR_NULL;
+    if (!envelope_ok(T, H, I, E, top_k)) return MOE_ERR_UNSUPPORTED;
+    fill_layout(T, H, I, E, top_k, layout);
+    return MOE_OK;
+}
+
+size_t moe_route_workspace_bytes(int T, int E, int top_k) {
+    if (!route_envelope_ok(T, E, top_k)) return 0;
+    return 256 + route_scratch_bytes(T, E);
+}
+
+int moe_route(const float *router_logits, int T, int E, int top_k, int32_t *topk_ids, float *topk_weights,
+              int32_t *expert_offsets, int32_t *sorted_to_flat, int32_t *flat_to_sorted, void *workspace,
+              size_t workspace_bytes, void *stream) {
+    if (T < 0 || E <= 0 || top_k <= 0 || top_k > E) return MOE_ERR_SHAPE;
+    if (!route_envelope_ok(T, E, top_k)) return MOE_ERR_UNSUPPORTED;
+    if (!expert_offsets) return MOE_ERR_NULL;
+    if (T > 0 && (!router_logits || !topk_ids || !topk_weights || !sorted_to_flat || !flat_to_sorted)) return MOE_ERR_NULL;
+    if (!workspace) return MOE_ERR_NULL;
+    if (!aligned(workspace, 256) || !aligned(router_logits, 4) || !aligned(topk_ids, 4) || !aligned(topk_weights, 4) ||
+        !aligned(expert_offsets, 4) || !aligned(sorted_to_flat, 4) || !aligned(flat_to_sorted, 4))
+        return MOE_ERR_ALIGN;
+    if (workspace_bytes < moe_route_workspace_bytes(T, E, top_k)) return MOE_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (T == 0) {  // no assignments: every segment is empty
+        return cudaMemsetAsync(expert_offsets, 0, (size_t)(E + 1) * sizeof(int), s) == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+    }
+    char *ws = static_cast<char *>(workspace);
+    RouteScratch rs = carve_route_scratch(ws + 256, T, E);
+    const cudaError_t err = launch_route(router_logits, T, E, top_k, 256, topk_ids, topk_weights, expert_offsets,
+                                         sorted_to_flat, flat_to_sorted, rs, reinterpret_cast<int *>(ws), s);
+    return err == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
+
+int moe_forward(const void *x, const float *router_logits, const void *w13, const void *w2, int T, int H, int I, int E,
+                int top_k, void *out, void *workspace, size_t workspace_bytes, void *stream) {
+    return forward_impl(x, router_logits, w13, w2, T, H, I, E, top_k, out, workspace, workspace_bytes,
+                        static_cast<cudaStream_t>(stream), MOE_FLAG_NONE);
+}
+
+int moe_forward_ex(const void *x, const float *router_logits, const void *w13, const void *w2, int T, int H, int I,
+                   int E, int top_k, void *out, void *workspace, size_t workspace_bytes, void *stream, unsigned flags) {
+    return forward_impl(x, router_logits, w13, w2, T, H, I, E, top_k, out, workspace, workspace_bytes,
+                        static_cast<cudaStream_t>(stream), flags);
+}
+
+int moe_forward_host(const void *x_host, const float *router_logits_host, const void *w13, const void *w2, int T, int H,
+                     int I, int E, int top_k, void *out_host, void *workspace, size_t workspace_bytes, void *stream) {
+    if (T < 0 || H <= 0 || I <= 0 || E <= 0 || top_k <= 0 || top_k > E) return MOE_ERR_SHAPE;
+    if (!envelope_ok(T, H, I, E, top_k)) return MOE_ERR_UNSUPPORTED;
+    if (T == 0) return MOE_OK;
+    if (!x_host || !router_logits_host || !out_host || !workspace) return MOE_ERR_NULL;
+    if (!aligned(workspace, 256)) return MOE_ERR_ALIGN;
+    moe_workspace_layout_t L;
+    fill_layout(T, H, I, E, top_k, &L);
+    if (workspace_bytes < L.total_bytes) return MOE_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    char *ws = static_cast<char *>(workspace);
+    const size_t x_bytes = (size_t)T * H * 2, l_bytes = (size_t)T * E * sizeof(float);
+    char *x_dev = ws + L.staging;
+    char *l_dev = x_dev + align_up(x_bytes, 256);
+    char *out_dev = l_dev + align_up(l_bytes, 256);
+    if (cudaMemcpyAsync(x_dev, x_host, x_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return MOE_ERR_CUDA;
+    if (cudaMemcpyAsync(l_dev, router_logits_host, l_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return MOE_ERR_CUDA;
+    const int st = forward_impl(x_dev, reinterpret_cast<const float *>(l_dev), w13, w2, T, H, I, E, top_k, out_dev,
+                                workspace, workspace_bytes, s, MOE_FLAG_NONE);
+    if (st != MOE_OK) return st;
+    if (cudaMemcpyAsync(out_host, out_dev, x_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) return MOE_ERR_CUDA;
+    return MOE_OK;
+}
+
+int moe_last_status(const void *workspace, void *stream) {
+    if (!workspace) return MOE_ERR_NULL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (cudaStreamSynchronize(s) != cudaSuccess) return MOE_ERR_CUDA;
+    int status[moe::kStatusInts] = {0, 0, 0, 0};
+    if (cudaMemcpy(status, workspace, sizeof(status), cudaMemcpyDeviceToHost) != cudaSuccess) return MOE_ERR_CUDA;
+    return status[0];
+}
+
+int moe_forward_launch_count(int T, unsigned flags) {
+    (void)flags;
+    return T > 0 ? 7 : 0;
+}
+
+const char *moe_status_string(int status) {
+    switch (status) {
+        case MOE_OK: return "ok";
+        case MOE_ERR_NULL: return "a required pointer is NULL";
+        case MOE_ERR_SHAPE: return "invalid shape (negative size, zero dimension, or top_k > E)";
+        case MOE_ERR_UNSUPPORTED: return "outside the supported envelope (E<=256, top_k<=32, H%128==0, I%64==0)";
+        case MOE_ERR_ALIGN: return "pointer not sufficiently aligned";
+        case MOE_ERR_WORKSPACE: return "workspace too small";
+        case MOE_ERR_CUDA: return "a CUDA call failed";
+        case MOE_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired";
+        case MOE_ERR_ARCH: return "device is not compute capability 10.x";
+        default: return "unknown status";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,88 @@
+// Internal declarations shared by the CUDA translation units of the MoE library.
+// Nothing here is part of the public ABI (see include/moe.h).
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "moe.h"
+
+namespace moe {
+
+constexpr int kMaxExperts = 256;        // router keeps ceil(E/32) <= 8 logits per lane
+constexpr int kMaxTopK = 32;            // lane j of the token's warp owns rank j
+constexpr int kRouteTokensPerBlock = 32;  // tokens per router block = one histogram chunk
+constexpr int kStatusInts = 4;          // status word: {status, site, aux0, aux1}
+
+// Site ids recorded next to MOE_ERR_DEVICE_TIMEOUT.
+enum : int { kSiteProducerEmpty = 1, kSiteMmaFull = 2, kSiteMmaTmemEmpty = 3, kSiteEpilogueTmemFull = 4 };
+
+static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Scratch of the router / sort-scatter, all int32, carved out of the caller's workspace.
+struct RouteScratch {
+    int *chunk_counts;  // [n_chunks, E] per-chunk expert histogram, then per-chunk start positions
+    int *tile_prefix;   // [E+1] exclusive prefix sum of token tiles per expert
+    int *tile_rows;     // [E]   rows per token tile of this expert (multiple of 16; 0 if empty)
+    int n_chunks;
+};
+
+static inline int route_num_chunks(int T) { return (T + kRouteTokensPerBlock - 1) / kRouteTokensPerBlock; }
+
+static inline size_t route_scratch_bytes(int T, int E) {
+    size_t ints = (size_t)route_num_chunks(T) * E + (size_t)(E + 1) + (size_t)E;
+    return align_up(ints * sizeof(int), 256);
+}
+
+static inline RouteScratch carve_route_scratch(void *base, int T, int E) {
+    RouteScratch s;
+    s.n_chunks = route_num_chunks(T);
+    s.chunk_counts = reinterpret_cast<int *>(base);
+    s.tile_prefix = s.chunk_counts + (size_t)s.n_chunks * E;
+    s.tile_rows = s.tile_prefix + (E + 1);
+    return s;
+}
+
+// Router + histogram, exclusive scans + tile schedule, stable scatter.  `nt_max` is the largest
+// number of rows a GEMM token tile may have (multiple of 16).
+cudaError_t launch_route(const float *logits, int T, int E, int k, int nt_max, int *topk_ids, float *topk_w,
+                         int *expert_offsets, int *sorted_to_flat, int *flat_to_sorted, RouteScratch scratch,
+                         int *status, cudaStream_t stream);
+
+// x_perm[r,:] = x[sorted_to_flat[r] / k, :]
+cudaError_t launch_gather_rows(const __nv_bfloat16 *x, const int *sorted_to_flat, int A, int k, int H,
+                               __nv_bfloat16 *x_perm, cudaStream_t stream);
+
+// out[t,:] = sum_j topk_w[t,j] * y[flat_to_sorted[t*k+j],:]
+cudaError_t launch_combine(const __nv_bfloat16 *y, const float *topk_w, const int *flat_to_sorted, int T, int k,
+                           int H, __nv_bfloat16 *out, cudaStream_t stream);
+
+// Grouped GEMM over expert-contiguous rows, tcgen05 / TMEM / TMA.
+//   swiglu = true : act [A,K=H] x w [E,2I,H]  -> out [A,I]  = SiLU(gate) * up
+//   swiglu = false: act [A,K=I] x w [E,H,I]   -> out [A,H]
+// `n_out` is the number of output features per row (I resp. H).
+struct GroupedGemmArgs {
+    const __nv_bfloat16 *act;  // [A, K]
+    const __nv_bfloat16 *w;    // [E, w_rows, K]
+    __nv_bfloat16 *out;        // [A, n_out]
+    int A, K, n_out, E;
+    int w_rows;                // rows per expert in w (2I for gemm1, H for gemm2)
+    int nt_max;                // token-tile bound the schedule was built with
+    const int *expert_offsets; // [E+1]
+    const int *tile_prefix;    // [E+1]
+    const int *tile_rows;      // [E]
+    int *status;               // status word
+    bool swiglu;
+};
+int launch_grouped_gemm_tc(const GroupedGemmArgs &args, cudaStream_t stream);  // returns a moe_status_t
+
+// Same contract on plain CUDA cores (validation only).
+cudaError_t launch_grouped_gemm_validation(const GroupedGemmArgs &args, cudaStream_t stream);
+
+// Token-tile bound chosen from the average rows per expert.
+int choose_nt_max(int T, int E, int k);
+
+}  // namespace moe

@@ -1,0 +1,273 @@
+// Router (softmax -> top-k -> renormalise) and the stable sort-scatter by expert.
+//
+// Paper, Sec. 4.5 "Routing": each token gets scores for E experts and the top k are picked with
+// warp-level cooperation; "Expert FFN computation", step (2): tokens are reordered by expert into
+// contiguous memory.  Here one warp owns one token (E <= 256 logits fit in 8 registers per lane),
+// selection is k rounds of a warp arg-max under the strict order
+//     e before e'  <=>  logit[e] > logit[e']  or  (logit[e] == logit[e'] and e < e'),
+// and the sort-scatter is a counting sort made stable without ordered atomics:
+//   1. every router block histograms the assignments of its own 32 tokens (one "chunk");
+//   2. one block turns the [chunk, expert] histogram into start positions (scan over chunks per
+//      expert, scan over experts) and derives the GEMM token-tile schedule;
+//   3. one warp per chunk walks its assignments in flat order, 32 at a time, ranking equal
+//      experts inside a group with match_any and carrying per-expert counters between groups.
+// Integer results are therefore unique and reproducible.
+#include "moe_internal.cuh"
+
+#include <limits.h>
+
+namespace moe {
+namespace {
+
+constexpr unsigned kFullMask = 0xffffffffu;
+constexpr int kRouteThreads = 256;
+constexpr int kLogitsPerLane = kMaxExperts / 32;
+
+__global__ void __launch_bounds__(kRouteThreads)
+route_topk_kernel(const float *__restrict__ logits, int T, int E, int k, int *__restrict__ topk_ids,
+                  float *__restrict__ topk_w, int *__restrict__ chunk_counts) {
+    __shared__ int hist[kMaxExperts];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    for (int e = tid; e < E; e += kRouteThreads) hist[e] = 0;
+    __syncthreads();
+
+    const int t_base = blockIdx.x * kRouteTokensPerBlock;
+    for (int tt = warp; tt < kRouteTokensPerBlock; tt += kRouteThreads / 32) {
+        const int t = t_base + tt;
+        if (t >= T) break;  // uniform over the warp
+        const float *row = logits + (size_t)t * E;
+        float v[kLogitsPerLane], p[kLogitsPerLane];
+        float m = -INFINITY;
+#pragma unroll
+        for (int i = 0; i < kLogitsPerLane; ++i) {
+            const int e = i * 32 + lane;
+            v[i] = e < E ? row[e] : -INFINITY;
+            m = fmaxf(m, v[i]);
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(kFullMask, m, off));
+        float s = 0.f;
+#pragma unroll
+        for (int i = 0; i < kLogitsPerLane; ++i) {
+            const int e = i * 32 + lane;
+            p[i] = e < E ? expf(v[i] - m) : 0.f;
+            s += p[i];
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(kFullMask, s, off);
+#pragma unroll
+        for (int i = 0; i < kLogitsPerLane; ++i) p[i] = p[i] / s;
+
+        unsigned taken = 0;
+        int my_id = 0;
+        float my_p = 0.f;
+        for (int j = 0; j < k; ++j) {
+            // best candidate among this lane's experts that are still available
+            int ci = INT_MAX;
+            float cv = -INFINITY, cp = 0.f;
+#pragma unroll
+            for (int i = 0; i < kLogitsPerLane; ++i) {
+                const int e = i * 32 + lane;
+                if (e < E && !((taken >> i) & 1u) && (ci == INT_MAX || v[i] > cv)) {
+                    ci = e; cv = v[i]; cp = p[i];
+                }
+            }
+            // warp arg-max; INT_MAX marks "no candidate" and always loses
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) {
+                const float ov = __shfl_xor_sync(kFullMask, cv, off);
+                const int oi = __shfl_xor_sync(kFullMask, ci, off);
+                const float op = __shfl_xor_sync(kFullMask, cp, off);
+                const bool other = (ci == INT_MAX) ? (oi != INT_MAX)
+                                                   : (oi != INT_MAX && (ov > cv || (ov == cv && oi < ci)));
+                if (other) { cv = ov; ci = oi; cp = op; }
+            }
+            // with non-finite logits lanes could disagree; lane 0's answer is the warp's answer
+            ci = __shfl_sync(kFullMask, ci, 0);
+            cp = __shfl_sync(kFullMask, cp, 0);
+            if (ci == INT_MAX) ci = 0;  // unreachable for k <= E; keeps the index in range regardless
+            if ((ci & 31) == lane) taken |= 1u << (ci >> 5);
+            if (lane == j) { my_id = ci; my_p = cp; }
+        }
+        float denom = 0.f;  // ascending rank, the order the definition states
+        for (int j = 0; j < k; ++j) denom += __shfl_sync(kFullMask, my_p, j);
+        if (lane < k) {
+            topk_ids[(size_t)t * k + lane] = my_id;
+            topk_w[(size_t)t * k + lane] = my_p / denom;
+            atomicAdd(&hist[my_id], 1);
+        }
+    }
+    __syncthreads();
+    for (int e = tid; e < E; e += kRouteThreads) chunk_counts[(size_t)blockIdx.x * E + e] = hist[e];
+}
+
+// Exclusive scan over the 256 threads of the block; returns the exclusive prefix, total in *total.
+__device__ __forceinline__ int block_exclusive_scan_256(int value, int *warp_sums, int *total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int incl = value;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const int n = __shfl_up_sync(kFullMask, incl, off);
+        if (lane >= off) incl += n;
+    }
+    if (lane == 31) warp_sums[warp] = incl;
+    __syncthreads();
+    int base = 0, sum = 0;
+#pragma unroll
+    for (int wi = 0; wi < 8; ++wi) {
+        const int ws = warp_sums[wi];
+        if (wi < warp) base += ws;
+        sum += ws;
+    }
+    __syncthreads();
+    *total = sum;
+    return base + incl - value;
+}
+
+__global__ void __launch_bounds__(256)
+route_scan_kernel(int *__restrict__ chunk_counts, int n_chunks, int E, int nt_max, int *__restrict__ expert_offsets,
+                  int *__restrict__ tile_prefix, int *__restrict__ tile_rows) {
+    __shared__ int warp_sums[8];
+    const int e = threadIdx.x;
+    int count = 0;
+    if (e < E) {
+        for (int b = 0; b < n_chunks; ++b) {
+            const int c = chunk_counts[(size_t)b * E + e];
+            chunk_counts[(size_t)b * E + e] = count;
+            count += c;
+        }
+    }
+    // token tiles of this expert: as few as fit under nt_max, evenly sized, rounded up to 16 rows
+    int n_tiles = 0, rows = 0;
+    if (count > 0) {
+        n_tiles = (count + nt_max - 1) / nt_max;
+        rows = (((count + n_tiles - 1) / n_tiles) + 15) & ~15;
+    }
+    int total_rows, total_tiles;
+    const int row_start = block_exclusive_scan_256(count, warp_sums, &total_rows);
+    const int tile_start = block_exclusive_scan_256(n_tiles, warp_sums, &total_tiles);
+    if (e < E) {
+        expert_offsets[e] = row_start;
+        tile_prefix[e] = tile_start;
+        tile_rows[e] = rows;
+        for (int b = 0; b < n_chunks; ++b) chunk_counts[(size_t)b * E + e] += row_start;
+    }
+    if (e == 0) {
+        expert_offsets[E] = total_rows;
+        tile_prefix[E] = total_tiles;
+    }
+}
+
+__global__ void __launch_bounds__(32)
+route_scatter_kernel(const int *__restrict__ topk_ids, const int *__restrict__ chunk_starts, int A, int E, int k,
+                     int *__restrict__ sorted_to_flat, int *__restrict__ flat_to_sorted) {
+    __shared__ int next[kMaxExperts];
+    const int lane = threadIdx.x;
+    for (int e = lane; e < E; e += 32) next[e] = chunk_starts[(size_t)blockIdx.x * E + e];
+    __syncwarp();
+    const int a0 = blockIdx.x * kRouteTokensPerBlock * k;
+    const int a1 = min(A, a0 + kRouteTokensPerBlock * k);
+    for (int base = a0; base < a1; base += 32) {
+        const int a = base + lane;
+        const bool valid = a < a1;
+        const int e = valid ? topk_ids[a] : 0;
+        const int key = valid ? e : -1 - lane;  // lanes past the end never match anything
+        const unsigned same = __match_any_sync(kFullMask, key);
+        const int rank = __popc(same & ((1u << lane) - 1u));
+        const int pos = valid ? next[e] + rank : 0;
+        __syncwarp();
+        if (valid && rank == 0) next[e] += __popc(same);
+        __syncwarp();
+        if (valid) {
+            flat_to_sorted[a] = pos;
+            sorted_to_flat[pos] = a;
+        }
+    }
+}
+
+__global__ void __launch_bounds__(256)
+gather_rows_kernel(const uint4 *__restrict__ x, const int *__restrict__ sorted_to_flat, int A, int k, int vec_per_row,
+                   uint4 *__restrict__ x_perm) {
+    const int lane = threadIdx.x & 31;
+    const int r = blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (r >= A) return;
+    const int t = sorted_to_flat[r] / k;
+    const uint4 *src = x + (size_t)t * vec_per_row;
+    uint4 *dst = x_perm + (size_t)r * vec_per_row;
+    for (int i = lane; i < vec_per_row; i += 32) dst[i] = src[i];
+}
+
+__global__ void __launch_bounds__(256)
+combine_kernel(const uint4 *__restrict__ y, const float *__restrict__ topk_w, const int *__restrict__ flat_to_sorted,
+               int k, int vec_per_row, uint4 *__restrict__ out) {
+    __shared__ int rows[kMaxTopK];
+    __shared__ float weights[kMaxTopK];
+    const int t = blockIdx.x;
+    if (threadIdx.x < k) {
+        rows[threadIdx.x] = flat_to_sorted[(size_t)t * k + threadIdx.x];
+        weights[threadIdx.x] = topk_w[(size_t)t * k + threadIdx.x];
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < vec_per_row; i += 256) {
+        float acc[8];
+#pragma unroll
+        for (int c = 0; c < 8; ++c) acc[c] = 0.f;
+        for (int j = 0; j < k; ++j) {  // ascending rank: the summation order is fixed
+            const uint4 v = y[(size_t)rows[j] * vec_per_row + i];
+            const float wj = weights[j];
+            const __nv_bfloat162 *h2 = reinterpret_cast<const __nv_bfloat162 *>(&v);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const float2 f = __bfloat1622float2(h2[c]);
+                acc[2 * c] = fmaf(wj, f.x, acc[2 * c]);
+                acc[2 * c + 1] = fmaf(wj, f.y, acc[2 * c + 1]);
+            }
+        }
+        uint4 o;
+        __nv_bfloat162 *o2 = reinterpret_cast<__nv_bfloat162 *>(&o);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) o2[c] = __floats2bfloat162_rn(acc[2 * c], acc[2 * c + 1]);
+        out[(size_t)t * vec_per_row + i] = o;
+    }
+}
+
+}  // namespace
+
+int choose_nt_max(int T, int E, int k) {
+    const double avg = (double)T * k / E;
+    const int options[3] = {32, 64, 128};
+    for (int nt : options)
+        if (1.5 * avg <= nt) return nt;
+    return 256;
+}
+
+cudaError_t launch_route(const float *logits, int T, int E, int k, int nt_max, int *topk_ids, float *topk_w,
+                         int *expert_offsets, int *sorted_to_flat, int *flat_to_sorted, RouteScratch scratch,
+                         int *status, cudaStream_t stream) {
+    cudaError_t err = cudaMemsetAsync(status, 0, kStatusInts * sizeof(int), stream);
+    if (err != cudaSuccess) return err;
+    const int A = T * k;
+    route_topk_kernel<<<scratch.n_chunks, kRouteThreads, 0, stream>>>(logits, T, E, k, topk_ids, topk_w,
+                                                                       scratch.chunk_counts);
+    route_scan_kernel<<<1, 256, 0, stream>>>(scratch.chunk_counts, scratch.n_chunks, E, nt_max, expert_offsets,
+                                             scratch.tile_prefix, scratch.tile_rows);
+    route_scatter_kernel<<<scratch.n_chunks, 32, 0, stream>>>(topk_ids, scratch.chunk_counts, A, E, k,
+                                                              sorted_to_flat, flat_to_sorted);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_gather_rows(const __nv_bfloat16 *x, const int *sorted_to_flat, int A, int k, int H,
+                               __nv_bfloat16 *x_perm, cudaStream_t stream) {
+    gather_rows_kernel<<<(A + 7) / 8, 256, 0, stream>>>(reinterpret_cast<const uint4 *>(x), sorted_to_flat, A, k,
+                                                        H / 8, reinterpret_cast<uint4 *>(x_perm));
+    return cudaGetLastError();
+}
+
+cudaError_t launch_combine(const __nv_bfloat16 *y, const float *topk_w, const int *flat_to_sorted, int T, int k,
+                           int H, __nv_bfloat16 *out, cudaStream_t stream) {
+    combine_kernel<<<T, 256, 0, stream>>>(reinterpret_cast<const uint4 *>(y), topk_w, flat_to_sorted, k, H / 8,
+                                          reinterpret_cast<uint4 *>(out));
+    return cudaGetLastError();
+}
+
+}  // namespace moe
