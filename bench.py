@@ -1,0 +1,344 @@
+#!/usr/bin/env python
+"""Benchmark of the MoE layer forward pass (one step = one whole pass: router, sort-scatter, row
+gather, gate/up GEMM + SwiGLU, down GEMM, combine) on seeded synthetic inputs.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl ours|reference]
+
+Prints ONE JSON line.  With N > 1 (launched by torch.distributed.run, one rank per GPU) every rank
+runs an independent replica on its own tokens -- the layer has no exchange step on one node, so
+there is no data-path collective -- and the line reports the aggregate (weak scaling).
+`--impl reference` times the CPU oracle (test infrastructure under oracle/) on the host cores for
+the same workload and metric; it is a deliberately plain program, reported as a baseline.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+from pathlib import Path
+
+import numpy as np
+import torch
+
+ROOT = Path(__file__).resolve().parent
+sys.path.insert(0, str(ROOT))
+
+from paper_2602_19128_b200.inputs import CONFIGS, bf16_bits, make_inputs  # noqa: E402
+
+METRIC = "moe_layer_tokens_per_s"
+UNIT = "tokens/s"
+L2_BYTES = 126 * 1024 * 1024
+# Which roofline bounds the dominant kernel (gate/up GEMM) of each workload: weight bytes per useful
+# flop put mixtral / dsv3_decode (and tiny) below the ridge point and the prefill-sized ones above it.
+BOUND = {"tiny": "hbm", "mixtral": "hbm", "dsv3_decode": "hbm", "dsv3_prefill": "tensor", "skewed": "tensor"}
+# DRAM bytes (read + write) of one gate/up GEMM launch, from the ncu capture summarised under profiles/.
+NCU_TRAFFIC_BYTES = {}
+
+
+def load_peaks() -> dict:
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        d = json.loads(p.read_text())
+        return dict(hbm_gbs=float(d["hbm_gbs"]), tflops_burst=float(d["bf16_tflops"]),
+                    tflops_sustained=float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), source="measured")
+    return dict(hbm_gbs=6650.0, tflops_burst=1590.0, tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples nvidia-smi (clocks, power, throttle reasons) for one GPU while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device: int):
+        self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        try:
+            uuid = str(torch.cuda.get_device_properties(device).uuid)
+            ident = uuid if uuid.startswith("GPU-") else "GPU-" + uuid
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", ident, f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.tmp,
+                                         stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["unavailable"])
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.tmp.flush()
+        rows = [r.split(",") for r in Path(self.tmp.name).read_text().strip().splitlines() if r.count(",") >= 7]
+        os.unlink(self.tmp.name)
+        sm, smax, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            try:
+                sm.append(float(r[0])); smax.append(float(r[1])); power.append(float(r[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, r[4:8]):
+                if v.strip().lower() == "active":
+                    reasons.add(n)
+        if not sm:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["no_samples"])
+        return dict(sm_mhz=statistics.median(sm), sm_max_mhz=max(smax), power_w=round(statistics.median(power), 1),
+                    samples=len(sm), reasons=sorted(reasons))
+
+
+def dist_setup(n_gpus: int):
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        return dist, rank, world, local
+    if n_gpus != 1:
+        raise SystemExit("--gpus N > 1 must be launched with torch.distributed.run (one rank per GPU)")
+    torch.cuda.set_device(0)
+    return None, 0, 1, 0
+
+
+def flush_l2(buf: torch.Tensor):
+    buf.add_(1)
+
+
+def oracle_sample(cfg_name: str, inp: dict, n_tokens: int, seed: int = 0):
+    """Host-side arguments for the oracle on a bounded sample of tokens: only the experts those tokens
+    route to are copied to the host."""
+    from oracle import moe_oracle
+    o = moe_oracle.get("f32")
+    T, k, I = inp["T"], inp["top_k"], inp["I"]
+    rng = np.random.default_rng(seed)
+    tokens = np.sort(rng.choice(T, size=min(n_tokens, T), replace=False)).astype(np.int32)
+    logits = inp["router_logits"].cpu().numpy()
+    ids, _ = o.route(logits, k)
+    need = sorted({int(e) for t in tokens for e in ids[t]})
+    experts = {e: (bf16_bits(inp["w13"][e]), bf16_bits(inp["w2"][e])) for e in need}
+    return o, bf16_bits(inp["x"]), logits, experts, I, k, tokens
+
+
+def time_oracle(cfg_name: str, inp: dict, budget_s: float):
+    """Times the oracle, as it stands, on a token sample sized to take roughly budget_s seconds."""
+    from oracle import moe_oracle
+    cores = moe_oracle.get("f32").num_threads
+    o, x, logits, experts, I, k, tokens = oracle_sample(cfg_name, inp, cores)
+    t0 = time.perf_counter()
+    o.forward_sampled(x, logits, experts, I, k, tokens)
+    t_probe = time.perf_counter() - t0
+    rounds = max(1, min(64, int(budget_s / max(t_probe, 1e-3))))
+    n = min(inp["T"], cores * rounds)
+    if n > len(tokens):
+        o, x, logits, experts, I, k, tokens = oracle_sample(cfg_name, inp, n)
+        t0 = time.perf_counter()
+        o.forward_sampled(x, logits, experts, I, k, tokens)
+        t_probe = time.perf_counter() - t0
+    return dict(value=len(tokens) / t_probe, unit=UNIT, cores=cores, kind="oracle",
+                sample=f"{len(tokens)} of {inp['T']} tokens of '{cfg_name}' (all top-k experts of each), float oracle, "
+                       f"{t_probe:.2f} s wall")
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle on the host cores (rank 0 only)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    from oracle import moe_oracle
+    cfg = CONFIGS[args.config]
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    inp = make_inputs(args.config, seed=args.seed, device=dev)
+    cores = moe_oracle.get("f32").num_threads
+    o, x, logits, experts, I, k, tokens = oracle_sample(args.config, inp, cores)
+    del inp
+    t0 = time.perf_counter()
+    o.forward_sampled(x, logits, experts, I, k, tokens)
+    probe = time.perf_counter() - t0
+    # keep the whole run within a few minutes: shrink the per-step sample if K steps would not fit
+    total_steps = args.steps + args.warmup
+    n = len(tokens)
+    if probe * total_steps > 240.0:
+        n = max(1, int(n * 240.0 / (probe * total_steps)))
+        tokens = tokens[:n]
+    for _ in range(args.warmup):
+        o.forward_sampled(x, logits, experts, I, k, tokens)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        o.forward_sampled(x, logits, experts, I, k, tokens)
+    wall = time.perf_counter() - t0
+    value = n * args.steps / wall
+    sample = f"{n} tokens of '{args.config}' per step (all top-k experts of each), float oracle"
+    line = dict(impl="reference", metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps,
+                warmup=args.warmup, ms_per_step=1e3 * wall / args.steps, higher_is_better=True, scaling="weak",
+                vs_baseline=None, dtype="f32", data="synthetic",
+                config=dict(workload=args.config, **{k_: cfg[k_] for k_ in ("T", "H", "I", "E", "top_k")},
+                            tokens_per_step=n),
+                cpu_baseline=dict(value=value, unit=UNIT, cores=cores, kind="oracle", sample=sample),
+                e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0), gpu_launches=0)
+    print(json.dumps(line), flush=True)
+
+
+def run_ours(args):
+    import paper_2602_19128_b200 as moe
+    dist, rank, world, local = dist_setup(args.gpus)
+    dev = torch.device("cuda", local)
+    cfg = CONFIGS[args.config]
+    T, H, I, E, k = (cfg[n] for n in ("T", "H", "I", "E", "top_k"))
+    inp = make_inputs(args.config, seed=args.seed + rank, device=dev)
+    x, logits, w13, w2 = inp["x"], inp["router_logits"], inp["w13"], inp["w2"]
+    out = torch.empty((T, H), dtype=torch.bfloat16, device=dev)
+    ws = moe.alloc_workspace(moe.moe_workspace_bytes(T, H, I, E, k), dev)
+    weight_bytes = (w13.numel() + w2.numel()) * 2
+    need_flush = weight_bytes < 2 * L2_BYTES
+    flush_buf = torch.zeros(2 * L2_BYTES // 4, dtype=torch.float32, device=dev) if need_flush else None
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing ----------------------------------------------------------------
+    for _ in range(max(args.warmup, 3)):
+        moe.moe_forward(x, logits, w13, w2, k, out, ws)
+    status = moe.moe_last_status(ws)
+    if status != moe.MOE_OK:
+        raise SystemExit(f"device status {status}: {moe.moe_status_string(status)}")
+    stage_events = [moe.make_stage_events() for _ in range(args.steps)]
+    barrier()
+    sampler = ClockSampler(local) if rank == 0 else None
+    for s in range(args.steps):
+        if need_flush:
+            flush_l2(flush_buf)
+        moe.moe_forward_staged(x, logits, w13, w2, k, out, ws, stage_events[s])
+    barrier()
+    clocks = sampler.stop() if sampler else None
+    if need_flush:
+        step_ms = [ev[0].elapsed_time(ev[-1]) for ev in stage_events]
+        total_ms = sum(step_ms)
+    else:
+        total_ms = stage_events[0][0].elapsed_time(stage_events[-1][-1])
+    stage_ms = {name: statistics.fmean(ev[i].elapsed_time(ev[i + 1]) for ev in stage_events)
+                for i, name in enumerate(moe.STAGE_NAMES)}
+    if dist is not None:
+        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    status = moe.moe_last_status(ws)
+    if status != moe.MOE_OK:
+        raise SystemExit(f"device status {status}: {moe.moe_status_string(status)}")
+    views = moe.workspace_views(ws, T, H, I, E, k)
+    counts = torch.diff(views["expert_offsets"]).cpu().numpy()
+    n_active = int((counts > 0).sum())
+
+    # ---- end to end through the host-buffer entry point ---------------------------------------------
+    xh = x.cpu().pin_memory()
+    lh = logits.cpu().pin_memory()
+    oh = torch.empty((T, H), dtype=torch.bfloat16).pin_memory()
+    for _ in range(3):
+        moe.moe_forward_host(xh, lh, w13, w2, k, oh, ws)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e2e_ms = 0.0
+    if need_flush:
+        for _ in range(args.steps):
+            flush_l2(flush_buf)
+            e0.record()
+            moe.moe_forward_host(xh, lh, w13, w2, k, oh, ws)
+            e1.record()
+            e1.synchronize()
+            e2e_ms += e0.elapsed_time(e1)
+    else:
+        e0.record()
+        for _ in range(args.steps):
+            moe.moe_forward_host(xh, lh, w13, w2, k, oh, ws)
+        e1.record()
+        e1.synchronize()
+        e2e_ms = e0.elapsed_time(e1)
+    barrier()
+    if dist is not None:
+        t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    same = bool(torch.equal(oh.view(torch.int16), out.cpu().view(torch.int16)))
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel (gate/up GEMM + SwiGLU) -----------------------------------
+    peaks = load_peaks()
+    A = T * k
+    t_gemm1 = stage_ms["gemm1_swiglu"] * 1e-3
+    bound = BOUND[args.config]
+    if bound == "hbm":
+        algorithmic = n_active * 2 * I * H * 2  # bytes of the active experts' w13, read once
+        achieved = algorithmic / t_gemm1 / 1e9
+        peak, unit = peaks["hbm_gbs"], "GB/s"
+    else:
+        algorithmic = 4.0 * A * H * I  # useful flops of the gate and up projections
+        achieved = algorithmic / t_gemm1 / 1e12
+        peak, unit = peaks["tflops_sustained"], "TFLOP/s"
+    step_s = total_ms * 1e-3 / args.steps
+    active_weight_bytes = n_active * 3 * I * H * 2
+    roofline = dict(bound=bound, kernel="grouped_gemm_tc_kernel<swiglu> (gate/up GEMM)", achieved=achieved, peak=peak,
+                    unit=unit, frac=achieved / peak, peak_source=f"of {peaks['source']}",
+                    traffic=NCU_TRAFFIC_BYTES.get(args.config), algorithmic_per_launch=algorithmic,
+                    kernel_ms=stage_ms["gemm1_swiglu"])
+    layer = dict(stage_ms={n: round(v, 5) for n, v in stage_ms.items()}, n_active_experts=n_active,
+                 rows_per_expert_min=int(counts.min()), rows_per_expert_max=int(counts.max()),
+                 weight_gbs=active_weight_bytes / step_s / 1e9, weight_gbs_frac=active_weight_bytes / step_s / 1e9 / peaks["hbm_gbs"],
+                 useful_tflops=6.0 * A * H * I / step_s / 1e12,
+                 useful_tflops_frac_sustained=6.0 * A * H * I / step_s / 1e12 / peaks["tflops_sustained"],
+                 useful_tflops_frac_burst=6.0 * A * H * I / step_s / 1e12 / peaks["tflops_burst"])
+
+    cpu_baseline = None
+    if world == 1 and not args.no_cpu_baseline:
+        cpu_baseline = time_oracle(args.config, inp, budget_s=15.0)
+
+    line = dict(metric=METRIC, value=world * T * args.steps / (total_ms * 1e-3), unit=UNIT, n_gpus=world,
+                steps=args.steps, warmup=max(args.warmup, 3), ms_per_step=total_ms / args.steps, higher_is_better=True,
+                scaling="weak", vs_baseline=None, dtype="bf16", data="synthetic",
+                config=dict(workload=args.config, T=T, H=H, I=I, E=E, top_k=k, parallelism=f"replicas x{world}",
+                            l2="flushed between steps" if need_flush else "weights larger than L2, no flush",
+                            seed=args.seed),
+                clocks=clocks,
+                e2e=dict(value=world * T * args.steps / (e2e_ms * 1e-3), unit=UNIT,
+                         h2d_bytes_per_step=T * H * 2 + T * E * 4, d2h_bytes_per_step=T * H * 2,
+                         ms_per_step=e2e_ms / args.steps, matches_device_path=same),
+                gpu_launches=moe.moe_forward_launch_count(T) * args.steps,
+                roofline=roofline, layer=layer, cpu_baseline=cpu_baseline)
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--config", choices=list(CONFIGS), default="mixtral")
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -130,6 +130,17 @@ MOE_API int moe_forward_ex(const void *x, const float *router_logits, const void
                    int E, int top_k, void *out, void *workspace, size_t workspace_bytes, void *stream,
                    unsigned flags);
 
+/* moe_forward_ex that also records CUDA events between the stages, for per-kernel timing inside a
+ * whole step.  stage_events is a HOST array of MOE_NUM_STAGE_EVENTS cudaEvent_t handles (passed as
+ * void*, created by the caller with timing enabled).  Event 0 is recorded on `stream` before the
+ * first kernel, and event i+1 after stage i, where the stages are
+ *   0 router + sort-scatter (3 kernels), 1 row gather, 2 gate/up GEMM + SwiGLU, 3 down GEMM, 4 combine.
+ * With T == 0 nothing is launched and no event is recorded. */
+#define MOE_NUM_STAGE_EVENTS 6
+MOE_API int moe_forward_staged(const void *x, const float *router_logits, const void *w13, const void *w2, int T, int H,
+                               int I, int E, int top_k, void *out, void *workspace, size_t workspace_bytes,
+                               void *stream, unsigned flags, void *const *stage_events);
+
 /* moe_forward for a caller whose activations live in HOST memory: x_host [T,H] bf16 and
  * router_logits_host [T,E] f32 are HOST pointers (pinned memory makes the copies asynchronous),
  * out_host [T,H] bf16 is a HOST pointer; the expert weights w13 / w2 stay DEVICE pointers

@@ -18,7 +18,7 @@ MOE_FLAG_NONE = 0
 MOE_FLAG_VALIDATION_GEMM = 1
 
 EXPORTED = ["moe_workspace_bytes", "moe_workspace_layout", "moe_route_workspace_bytes", "moe_route", "moe_forward",
-            "moe_forward_ex", "moe_forward_host", "moe_last_status", "moe_forward_launch_count", "moe_status_string"]
+            "moe_forward_ex", "moe_forward_staged", "moe_forward_host", "moe_last_status", "moe_forward_launch_count", "moe_status_string"]
 
 
 class MoeError(RuntimeError):
@@ -57,6 +57,9 @@ def lib() -> ctypes.CDLL:
         L.moe_forward.argtypes = [vp, vp, vp, vp, i, i, i, i, i, vp, vp, sz, vp]
         L.moe_forward_ex.restype = i
         L.moe_forward_ex.argtypes = [vp, vp, vp, vp, i, i, i, i, i, vp, vp, sz, vp, ctypes.c_uint]
+        L.moe_forward_staged.restype = i
+        L.moe_forward_staged.argtypes = [vp, vp, vp, vp, i, i, i, i, i, vp, vp, sz, vp, ctypes.c_uint,
+                                         ctypes.POINTER(vp)]
         L.moe_forward_host.restype = i
         L.moe_forward_host.argtypes = [vp, vp, vp, vp, i, i, i, i, i, vp, vp, sz, vp]
         L.moe_last_status.restype = i
@@ -130,6 +133,32 @@ def moe_forward(x, router_logits, w13, w2, top_k: int, out, workspace, stream=No
                               _ptr(workspace), workspace.numel(), _stream(stream), flags)
     if check and st != MOE_OK:
         raise MoeError(st, "moe_forward")
+    return st
+
+
+STAGE_NAMES = ("route", "gather", "gemm1_swiglu", "gemm2", "combine")
+NUM_STAGE_EVENTS = len(STAGE_NAMES) + 1
+
+
+def make_stage_events() -> list:
+    """CUDA events for moe_forward_staged; each is recorded once so that its handle exists."""
+    events = [torch.cuda.Event(enable_timing=True) for _ in range(NUM_STAGE_EVENTS)]
+    for e in events:
+        e.record()
+    torch.cuda.synchronize()
+    return events
+
+
+def moe_forward_staged(x, router_logits, w13, w2, top_k: int, out, workspace, stage_events, stream=None,
+                       flags: int = 0, check: bool = True) -> int:
+    """moe_forward that records ``stage_events`` (from make_stage_events) around the five stages."""
+    T, H = x.shape
+    E, I2, _ = w13.shape
+    handles = (ctypes.c_void_p * NUM_STAGE_EVENTS)(*[e.cuda_event for e in stage_events])
+    st = lib().moe_forward_staged(_ptr(x), _ptr(router_logits), _ptr(w13), _ptr(w2), T, H, I2 // 2, E, top_k,
+                                  _ptr(out), _ptr(workspace), workspace.numel(), _stream(stream), flags, handles)
+    if check and st != MOE_OK:
+        raise MoeError(st, "moe_forward_staged")
     return st
 
 

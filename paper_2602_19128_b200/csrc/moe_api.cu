@@ -48,7 +48,8 @@ int check_device() {
 }
 
 int forward_impl(const void *x, const float *logits, const void *w13, const void *w2, int T, int H, int I, int E, int k,
-                 void *out, void *workspace, size_t workspace_bytes, cudaStream_t stream, unsigned flags) {
+                 void *out, void *workspace, size_t workspace_bytes, cudaStream_t stream, unsigned flags,
+                 void *const *stage_events = nullptr) {
     if (T < 0 || H <= 0 || I <= 0 || E <= 0 || k <= 0 || k > E) return MOE_ERR_SHAPE;
     if (!envelope_ok(T, H, I, E, k)) return MOE_ERR_UNSUPPORTED;
     if (flags & ~MOE_FLAG_VALIDATION_GEMM) return MOE_ERR_UNSUPPORTED;
@@ -77,10 +78,16 @@ int forward_impl(const void *x, const float *logits, const void *w13, const void
     const int A = T * k;
     const int nt_max = choose_nt_max(T, E, k);
 
+    auto mark = [&](int i) {
+        return !stage_events || cudaEventRecord(static_cast<cudaEvent_t>(stage_events[i]), stream) == cudaSuccess;
+    };
+    if (!mark(0)) return MOE_ERR_CUDA;
     if (launch_route(logits, T, E, k, nt_max, ids, wts, offsets, s2f, f2s, rs, status, stream) != cudaSuccess)
         return MOE_ERR_CUDA;
+    if (!mark(1)) return MOE_ERR_CUDA;
     if (launch_gather_rows(static_cast<const __nv_bfloat16 *>(x), s2f, A, k, H, x_perm, stream) != cudaSuccess)
         return MOE_ERR_CUDA;
+    if (!mark(2)) return MOE_ERR_CUDA;
 
     GroupedGemmArgs g1;
     g1.act = x_perm; g1.w = static_cast<const __nv_bfloat16 *>(w13); g1.out = h;
@@ -93,15 +100,19 @@ int forward_impl(const void *x, const float *logits, const void *w13, const void
 
     if (flags & MOE_FLAG_VALIDATION_GEMM) {
         if (launch_grouped_gemm_validation(g1, stream) != cudaSuccess) return MOE_ERR_CUDA;
+        if (!mark(3)) return MOE_ERR_CUDA;
         if (launch_grouped_gemm_validation(g2, stream) != cudaSuccess) return MOE_ERR_CUDA;
     } else {
         int st = launch_grouped_gemm_tc(g1, stream);
         if (st != MOE_OK) return st;
+        if (!mark(3)) return MOE_ERR_CUDA;
         st = launch_grouped_gemm_tc(g2, stream);
         if (st != MOE_OK) return st;
     }
+    if (!mark(4)) return MOE_ERR_CUDA;
     if (launch_combine(y, wts, f2s, T, k, H, static_cast<__nv_bfloat16 *>(out), stream) != cudaSuccess)
         return MOE_ERR_CUDA;
+    if (!mark(5)) return MOE_ERR_CUDA;
     return MOE_OK;
 }
 
@@ -161,6 +172,16 @@ int moe_forward_ex(const void *x, const float *router_logits, const void *w13, c
                    int E, int top_k, void *out, void *workspace, size_t workspace_bytes, void *stream, unsigned flags) {
     return forward_impl(x, router_logits, w13, w2, T, H, I, E, top_k, out, workspace, workspace_bytes,
                         static_cast<cudaStream_t>(stream), flags);
+}
+
+int moe_forward_staged(const void *x, const float *router_logits, const void *w13, const void *w2, int T, int H, int I,
+                       int E, int top_k, void *out, void *workspace, size_t workspace_bytes, void *stream, unsigned flags,
+                       void *const *stage_events) {
+    if (!stage_events) return MOE_ERR_NULL;
+    for (int i = 0; i < MOE_NUM_STAGE_EVENTS; ++i)
+        if (!stage_events[i]) return MOE_ERR_NULL;
+    return forward_impl(x, router_logits, w13, w2, T, H, I, E, top_k, out, workspace, workspace_bytes,
+                        static_cast<cudaStream_t>(stream), flags, stage_events);
 }
 
 int moe_forward_host(const void *x_host, const float *router_logits_host, const void *w13, const void *w2, int T, int H,

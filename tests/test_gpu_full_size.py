@@ -1,0 +1,62 @@
+"""GPU parity at the full workload sizes, in the launch configuration bench.py times.
+
+The CPU oracle cannot evaluate these layers in full, so each workload is checked three ways:
+routing and permutation bit-exactly on all tokens (cheap on the CPU); the layer output on a
+sample of tokens the oracle computes one by one; and every intermediate and output element
+against the CUDA-core validation kernels, which share no code with the tcgen05 path.
+"""
+import numpy as np
+import pytest
+import torch
+
+import paper_2602_19128_b200 as moe
+from oracle import moe_oracle
+from paper_2602_19128_b200.inputs import CONFIGS, bf16_bits
+from tests.gpu_common import OUT_TOL, assert_close_out, assert_routing_exact, bf16_to_f64, gpu_inputs, run_forward
+
+pytestmark = pytest.mark.gpu
+
+
+def close_on_device(a: torch.Tensor, b: torch.Tensor, what: str):
+    a, b = a.float(), b.float()
+    assert torch.isfinite(a).all(), what
+    bad = (a - b).abs() > OUT_TOL * (1 + b.abs())
+    assert not bad.any(), f"{what}: {int(bad.sum())} elements differ beyond tolerance"
+
+
+@pytest.mark.parametrize("name", ["mixtral", "dsv3_decode", "skewed", "dsv3_prefill"])
+def test_full_size_workload(name):
+    cfg = CONFIGS[name]
+    T, H, I, E, k = (cfg[n] for n in ("T", "H", "I", "E", "top_k"))
+    inp = gpu_inputs(name, seed=0)
+    out, views, ws = run_forward(inp)
+
+    # 1. routing and permutation, all tokens, bit-exact
+    o = moe_oracle.get("f32")
+    logits = inp["router_logits"].cpu().numpy()
+    ids, w = o.route(logits, k)
+    off, s2f, f2s = o.permute(ids, E)
+    assert_routing_exact(views, ids, w, off, s2f, f2s)
+    assert torch.equal(views["x_perm"].view(torch.int16),
+                       inp["x"][views["sorted_to_flat"].long() // k].view(torch.int16))
+
+    # 2. sampled tokens against the oracle (first, last, and a seeded draw; hot and cold experts)
+    rng = np.random.default_rng(0)
+    tokens = np.unique(np.concatenate([[0, T - 1], rng.choice(T, size=6, replace=False)])).astype(np.int32)
+    need = sorted({int(e) for t in tokens for e in ids[t]})
+    experts = {e: (bf16_bits(inp["w13"][e]), bf16_bits(inp["w2"][e])) for e in need}
+    ref = o.forward_sampled(bf16_bits(inp["x"]), logits, experts, I, k, tokens)
+    assert_close_out(bf16_to_f64(out[torch.from_numpy(tokens).long().cuda()]), ref, f"{name} sampled out")
+
+    # 3. run-to-run determinism
+    out_again, _, ws2 = run_forward(inp)
+    assert torch.equal(out.view(torch.int16), out_again.view(torch.int16))
+    del ws2, out_again
+
+    # 4. every element of h, y and out against the CUDA-core validation kernels
+    h, y = views["h"].clone(), views["y"].clone()
+    del ws, views
+    out_v, views_v, _ = run_forward(inp, flags=moe.MOE_FLAG_VALIDATION_GEMM)
+    close_on_device(h, views_v["h"], f"{name} h")
+    close_on_device(y, views_v["y"], f"{name} y")
+    close_on_device(out, out_v, f"{name} out")
