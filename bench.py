@@ -331,9 +331,15 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--config", choices=list(CONFIGS), default="mixtral")
+    ap.add_argument("--shape", default=None, help="custom T,H,I,E,top_k instead of a named workload (profiling)")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
+    if args.shape:
+        T, H, I, E, k = (int(v) for v in args.shape.split(","))
+        args.config = f"custom_{T}x{H}x{I}x{E}x{k}"
+        CONFIGS[args.config] = dict(T=T, H=H, I=I, E=E, top_k=k, skew=False)
+        BOUND[args.config] = "hbm"
     if args.impl == "reference":
         run_reference(args)
     else:
