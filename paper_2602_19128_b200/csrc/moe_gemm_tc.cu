@@ -23,79 +23,12 @@
 //    one tile overlaps the MMAs of the next).
 //  * Every wait is bounded: if one expires the CTA records MOE_ERR_DEVICE_TIMEOUT and the site in
 //    the status word, every role stops, TMEM is released and the kernel returns.
-#include "moe_internal.cuh"
-
-#include <mutex>
+#include "moe_tc_common.cuh"
 
 namespace moe {
 namespace {
 
-constexpr int kBlockK = 64;                        // K elements per ring slot = one 128-byte swizzle row
-constexpr int kTileM = 128;                        // weight rows per tile (MMA M)
-constexpr int kSlotABytes = kTileM * kBlockK * 2;  // 16 KiB
-constexpr int kRowBytes = kBlockK * 2;             // 128
-constexpr int kThreads = 192;
-constexpr int kEpilogueWarps = 4;
-constexpr long long kWaitLimitCycles = 4000000000LL;  // about two seconds at full clock
-
-struct KernelParams {
-    __nv_bfloat16 *out;
-    const int *expert_offsets, *tile_prefix, *tile_rows;
-    int *status;
-    int E, n_k_blocks, n_out, w_rows, n_feature_tiles, up_row_offset;
-};
-
-// ---- PTX wrappers -----------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t done;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(done)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return done != 0;
-}
-// Bounded wait.  Returns false if the CTA is aborting (this wait expired, or another role's did).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status,
-                                          int site) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const long long start = clock64();
-    while (true) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag) return false;
-        if (clock64() - start > kWaitLimitCycles) {
-            *abort_flag = 1;
-            if (atomicCAS(status, 0, (int)MOE_ERR_DEVICE_TIMEOUT) == 0) {
-                status[1] = site;
-                status[2] = blockIdx.x;
-            }
-            return false;
-        }
-    }
-}
-
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int c0, int c1, uint32_t bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar)
-        : "memory");
-}
-
-__device__ __forceinline__ void tcgen05_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tcgen05_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+using namespace tc;
 
 // D[tmem] (+)= A[smem] * B[smem]^T, bf16 inputs, fp32 accumulate, issued by one thread.
 __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
@@ -110,60 +43,6 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint
 // Arrive on an mbarrier once all MMAs issued so far by this thread have completed.
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-// 16 consecutive fp32 columns of this thread's TMEM lane.
-__device__ __forceinline__ void tmem_load_16(uint32_t taddr, float (&v)[16]) {
-    uint32_t r[16];
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-        : "r"(taddr));
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
-}
-
-// Shared-memory matrix descriptor for a K-major bf16 tile whose rows are 128 bytes with the 128-byte
-// swizzle TMA applies: start address, leading offset 1 (unused for swizzled K-major), stride between
-// 8-row groups 1024 bytes, descriptor version 1, layout type 2 (128-byte swizzle).
-__device__ __forceinline__ uint64_t smem_desc_k_major_sw128(uint32_t smem_addr) {
-    uint64_t d = 0;
-    d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
-    d |= (uint64_t)1 << 16;
-    d |= (uint64_t)(1024 >> 4) << 32;
-    d |= (uint64_t)1 << 46;
-    d |= (uint64_t)2 << 61;
-    return d;
-}
-// Instruction descriptor: fp32 accumulator, bf16 A and B, both K-major, M = 128, N = n.
-__device__ __forceinline__ uint32_t instr_desc_bf16_m128(int n) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
-}
-
-struct Tile {
-    int e, f, row0, n_valid, n_mma;
-};
-// Tile order: expert-major, then feature tile, then the expert's token tiles (fastest).
-__device__ __forceinline__ Tile decode_tile(int tile, const KernelParams &p) {
-    int lo = 0, hi = p.E;
-    while (hi - lo > 1) {
-        const int mid = (lo + hi) >> 1;
-        if (p.tile_prefix[mid] * p.n_feature_tiles <= tile) lo = mid; else hi = mid;
-    }
-    Tile t;
-    t.e = lo;
-    const int first = p.tile_prefix[lo], n_tok_tiles = p.tile_prefix[lo + 1] - first;
-    const int local = tile - first * p.n_feature_tiles;
-    t.f = local / n_tok_tiles;
-    const int j = local - t.f * n_tok_tiles;
-    const int rows = p.tile_rows[lo];
-    const int begin = p.expert_offsets[lo], count = p.expert_offsets[lo + 1] - begin;
-    t.row0 = begin + j * rows;
-    t.n_valid = min(rows, count - j * rows);
-    t.n_mma = (t.n_valid + 15) & ~15;
-    return t;
 }
 
 template <int NT_MAX, int STAGES>
@@ -180,8 +59,7 @@ struct SmemLayout {
 
 template <int NT_MAX, int STAGES, bool SWIGLU>
 __global__ void __launch_bounds__(kThreads, 1)
-grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_act64,
-                       const __grid_constant__ CUtensorMap map_act16, const KernelParams p) {
+grouped_gemm_tc_kernel(const __grid_constant__ TensorMaps maps, const KernelParams p) {
     using L = SmemLayout<NT_MAX, STAGES>;
     constexpr int kTmemCols = 2 * NT_MAX;
     extern __shared__ uint8_t smem_raw[];
@@ -226,8 +104,9 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_c
             bool ok = true;
             for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
                 const Tile t = decode_tile(tile, p);
-                const int w_row = t.e * p.w_rows + t.f * (SWIGLU ? kTileM / 2 : kTileM);
-                const uint32_t tx_bytes = kSlotABytes + t.n_mma * kRowBytes;
+                const int n_mma = (t.n_valid + 15) & ~15;
+                const int w_row = t.e * p.w_rows + t.f * kTileM;  // down projection: 128 rows of w2[e]
+                const uint32_t tx_bytes = kSlotABytes + n_mma * kRowBytes;
                 for (int kb = 0; kb < p.n_k_blocks; ++kb) {
                     ok = mbar_wait(bar_empty + stage * 8, phase ^ 1u, abort_flag, p.status, kSiteProducerEmpty);
                     if (!ok) break;
@@ -236,18 +115,13 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_c
                     const uint32_t sa = base + L::kA + stage * kSlotABytes;
                     const uint32_t sb = base + L::kB + stage * L::kSlotBBytes;
                     const int k0 = kb * kBlockK;
-                    if (SWIGLU) {
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            tma_load_2d(sa + q * 32 * kRowBytes, &map_w, k0, w_row + q * 16, full);
-                            tma_load_2d(sa + (q * 32 + 16) * kRowBytes, &map_w, k0, w_row + p.up_row_offset + q * 16, full);
-                        }
-                    } else {
-                        tma_load_2d(sa, &map_w, k0, w_row, full);
-                    }
-                    int r = 0;
-                    for (; r + 64 <= t.n_mma; r += 64) tma_load_2d(sb + r * kRowBytes, &map_act64, k0, t.row0 + r, full);
-                    for (; r < t.n_mma; r += 16) tma_load_2d(sb + r * kRowBytes, &map_act16, k0, t.row0 + r, full);
+                    if (SWIGLU)  // 64 features = groups 4f..4f+3 of 16, gate and up rows interleaved per group
+                        tma_load_5d(sa, &maps.w, k0, 0, 0, t.f * 4, t.e, full);
+                    else
+                        tma_load_2d(sa, &maps.w, k0, w_row, full);
+                    load_act_rows(maps, sb, k0, t.row0, n_mma, [&](uint32_t dst, const CUtensorMap *m, int c0, int c1) {
+                        tma_load_2d(dst, m, c0, c1, full);
+                    });
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -261,7 +135,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_c
             bool ok = true;
             for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
                 const Tile t = decode_tile(tile, p);
-                const uint32_t idesc = instr_desc_bf16_m128(t.n_mma);
+                const uint32_t idesc = instr_desc_bf16(kTileM, (t.n_valid + 15) & ~15);
                 ok = mbar_wait(bar_acc_empty + acc * 8, acc_phase ^ 1u, abort_flag, p.status, kSiteMmaTmemEmpty);
                 if (!ok) break;
                 tcgen05_fence_after();
@@ -292,6 +166,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_c
         bool ok = true;
         for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
             const Tile t = decode_tile(tile, p);
+            const int n_mma = (t.n_valid + 15) & ~15;
             ok = mbar_wait(bar_acc_full + acc * 8, acc_phase, abort_flag, p.status, kSiteEpilogueTmemFull);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
@@ -300,7 +175,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_c
             if (SWIGLU) {
                 const int hi = lane >> 4;
                 __nv_bfloat16 *dst = p.out + (size_t)t.row0 * p.n_out + t.f * (kTileM / 2) + q * 16 + (lane & 15);
-                for (int c0 = 0; c0 < t.n_mma; c0 += 16) {
+                for (int c0 = 0; c0 < n_mma; c0 += 16) {
                     float v[16];
                     tmem_load_16(taddr + c0, v);
 #pragma unroll
@@ -310,12 +185,12 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_c
                         const float u = hi ? v[8 + i] : other;
                         const int col = c0 + hi * 8 + i;
                         if (col < t.n_valid)
-                            dst[(size_t)col * p.n_out] = __float2bfloat16_rn(__fdividef(g, 1.f + __expf(-g)) * u);
+                            dst[(size_t)col * p.n_out] = __float2bfloat16_rn(swiglu(g, u));
                     }
                 }
             } else {
                 __nv_bfloat16 *dst = p.out + (size_t)t.row0 * p.n_out + t.f * kTileM + q * 32 + lane;
-                for (int c0 = 0; c0 < t.n_mma; c0 += 16) {
+                for (int c0 = 0; c0 < n_mma; c0 += 16) {
                     float v[16];
                     tmem_load_16(taddr + c0, v);
 #pragma unroll
@@ -343,70 +218,25 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_c
     }
 }
 
-// ---- host side ----------------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn get_encode_fn() {
-    static EncodeTiledFn fn = nullptr;
-    static std::once_flag once;
-    std::call_once(once, [] {
-        void *ptr = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(ptr);
-    });
-    return fn;
-}
-
-// 2-D bf16 tensor [rows, cols] row-major; box = box_rows x 64 columns, 128-byte swizzle, zero fill.
-bool encode_2d(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
-    EncodeTiledFn fn = get_encode_fn();
-    if (!fn) return false;
-    const cuuint64_t dims[2] = {cols, rows};
-    const cuuint64_t strides[1] = {cols * 2};
-    const cuuint32_t box[2] = {(cuuint32_t)kBlockK, box_rows};
-    const cuuint32_t elem_strides[2] = {1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, elem_strides,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
-int sm_count() {
-    static int cached[64] = {0};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 1;
-    if (cached[dev] == 0) {
-        int n = 0;
-        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-        cached[dev] = n > 0 ? n : 1;
-    }
-    return cached[dev];
-}
-
 template <int NT_MAX, int STAGES, bool SWIGLU>
-int launch_instance(const GroupedGemmArgs &a, const CUtensorMap &map_w, const CUtensorMap &m64, const CUtensorMap &m16,
-                    const KernelParams &p, int grid, cudaStream_t stream) {
+int launch_instance(const TensorMaps &maps, const KernelParams &p, int grid, cudaStream_t stream) {
     using L = SmemLayout<NT_MAX, STAGES>;
     static_assert(L::kDynamicBytes <= 232448, "ring does not fit in shared memory");
     auto kernel = grouped_gemm_tc_kernel<NT_MAX, STAGES, SWIGLU>;
     // per device and cheap, so set on every launch rather than cached per process
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) != cudaSuccess)
         return MOE_ERR_CUDA;
-    kernel<<<grid, kThreads, L::kDynamicBytes, stream>>>(map_w, m64, m16, p);
+    kernel<<<grid, kThreads, L::kDynamicBytes, stream>>>(maps, p);
     return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
 
 template <bool SWIGLU>
-int dispatch(const GroupedGemmArgs &a, const CUtensorMap &w, const CUtensorMap &m64, const CUtensorMap &m16,
-             const KernelParams &p, int grid, cudaStream_t s) {
-    switch (a.nt_max) {
-        case 32: return launch_instance<32, 10, SWIGLU>(a, w, m64, m16, p, grid, s);
-        case 64: return launch_instance<64, 8, SWIGLU>(a, w, m64, m16, p, grid, s);
-        case 128: return launch_instance<128, 6, SWIGLU>(a, w, m64, m16, p, grid, s);
-        case 256: return launch_instance<256, 4, SWIGLU>(a, w, m64, m16, p, grid, s);
+int dispatch(int nt_max, const TensorMaps &maps, const KernelParams &p, int grid, cudaStream_t s) {
+    switch (nt_max) {
+        case 32: return launch_instance<32, 10, SWIGLU>(maps, p, grid, s);
+        case 64: return launch_instance<64, 8, SWIGLU>(maps, p, grid, s);
+        case 128: return launch_instance<128, 6, SWIGLU>(maps, p, grid, s);
+        case 256: return launch_instance<256, 4, SWIGLU>(maps, p, grid, s);
         default: return MOE_ERR_UNSUPPORTED;
     }
 }
@@ -418,10 +248,10 @@ int launch_grouped_gemm_tc(const GroupedGemmArgs &a, cudaStream_t stream) {
     const int features_per_tile = a.swiglu ? kTileM / 2 : kTileM;
     if (a.n_out % features_per_tile != 0) return MOE_ERR_UNSUPPORTED;
 
-    CUtensorMap map_w, map_act64, map_act16;
-    if (!encode_2d(&map_w, a.w, (uint64_t)a.E * a.w_rows, a.K, a.swiglu ? 16 : kTileM)) return MOE_ERR_CUDA;
-    if (!encode_2d(&map_act64, a.act, a.A, a.K, 64)) return MOE_ERR_CUDA;
-    if (!encode_2d(&map_act16, a.act, a.A, a.K, 16)) return MOE_ERR_CUDA;
+    TensorMaps maps;
+    const bool ok_w = a.swiglu ? encode_weight_map_gate_up(&maps.w, a.w, a.E, a.n_out, a.K)
+                               : encode_weight_map_2d(&maps.w, a.w, (uint64_t)a.E * a.w_rows, a.K);
+    if (!ok_w || !encode_act_maps(maps.act, a.act, a.A, a.K)) return MOE_ERR_CUDA;
 
     KernelParams p;
     p.out = a.out;
@@ -434,15 +264,13 @@ int launch_grouped_gemm_tc(const GroupedGemmArgs &a, cudaStream_t stream) {
     p.n_out = a.n_out;
     p.w_rows = a.w_rows;
     p.n_feature_tiles = a.n_out / features_per_tile;
-    p.up_row_offset = a.swiglu ? a.n_out : 0;
 
     // The tile count is only known on the device; this is its upper bound.
     const long long max_token_tiles = (long long)(a.A < a.E ? a.A : a.E) + a.A / a.nt_max;
     const long long max_tiles = max_token_tiles * p.n_feature_tiles;
     const int sms = sm_count();
     const int grid = (int)(max_tiles < sms ? max_tiles : sms);
-    return a.swiglu ? dispatch<true>(a, map_w, map_act64, map_act16, p, grid, stream)
-                    : dispatch<false>(a, map_w, map_act64, map_act16, p, grid, stream);
+    return a.swiglu ? dispatch<true>(a.nt_max, maps, p, grid, stream) : dispatch<false>(a.nt_max, maps, p, grid, stream);
 }
 
 }  // namespace moe

@@ -1,0 +1,171 @@
+// Device-side PTX wrappers, descriptors and the tile schedule decoder shared by the two tcgen05
+// grouped-GEMM kernels (one CTA per tile, and CTA pairs), plus the host-side tensor-map encoders.
+#pragma once
+
+#include "moe_internal.cuh"
+
+namespace moe {
+namespace tc {
+
+constexpr int kBlockK = 64;                        // K elements per ring slot = one 128-byte swizzle row
+constexpr int kTileM = 128;                        // weight rows per CTA (MMA M per CTA)
+constexpr int kSlotABytes = kTileM * kBlockK * 2;  // 16 KiB
+constexpr int kRowBytes = kBlockK * 2;             // 128
+constexpr int kThreads = 192;                      // warp 0 TMA, warp 1 MMA, warps 2..5 epilogue
+constexpr int kEpilogueWarps = 4;
+constexpr long long kWaitLimitCycles = 4000000000LL;  // about two seconds at full clock
+constexpr int kNumActMaps = 4;                     // activation boxes of 128, 64, 32 and 16 rows
+
+// Tensor maps of one grouped GEMM.  `w` is either a 2-D map over [E*w_rows, K] with a 128-row box
+// (down projection) or a 5-D map over w13 viewed as [E][I/16][gate|up][16][H] whose
+// {64,16,2,4,1} box delivers 64 features as 4 x (16 gate rows, 16 up rows) in one copy.
+struct TensorMaps {
+    CUtensorMap w;
+    CUtensorMap act[kNumActMaps];  // box rows 128, 64, 32, 16
+};
+
+struct KernelParams {
+    __nv_bfloat16 *out;
+    const int *expert_offsets, *tile_prefix, *tile_rows;
+    int *status;
+    int E, n_k_blocks, n_out, w_rows, n_feature_tiles;
+};
+
+// ---- PTX wrappers -----------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return done != 0;
+}
+// Bounded wait.  Returns false if the CTA is aborting (this wait expired, or another role's did).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status,
+                                          int site) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long start = clock64();
+    while (true) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (clock64() - start > kWaitLimitCycles) {
+            *abort_flag = 1;
+            if (atomicCAS(status, 0, (int)MOE_ERR_DEVICE_TIMEOUT) == 0) {
+                status[1] = site;
+                status[2] = blockIdx.x;
+            }
+            return false;
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int c0, int c1, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap *map, int c0, int c1, int c2, int c3,
+                                            int c4, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(bar)
+        : "memory");
+}
+
+__device__ __forceinline__ void tcgen05_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tcgen05_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// 16 consecutive fp32 columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_load_16(uint32_t taddr, float (&v)[16]) {
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Shared-memory matrix descriptor for a K-major bf16 tile whose rows are 128 bytes with the 128-byte
+// swizzle TMA applies: start address, leading offset 1 (unused for swizzled K-major), stride between
+// 8-row groups 1024 bytes, descriptor version 1, layout type 2 (128-byte swizzle).
+__device__ __forceinline__ uint64_t smem_desc_k_major_sw128(uint32_t smem_addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)1 << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+// Instruction descriptor: fp32 accumulator, bf16 A and B, both K-major, M = m (128, or 256 for a CTA
+// pair), N = n.
+__device__ __forceinline__ uint32_t instr_desc_bf16(int m, int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+
+// Activation rows [row, row + n_rows) (n_rows a multiple of 16) of K block k0 into shared memory at
+// `dst`, as few boxes as the four maps allow.  LOAD(dst, map, k0, row) issues one copy.
+template <class Load>
+__device__ __forceinline__ void load_act_rows(const TensorMaps &maps, uint32_t dst, int k0, int row, int n_rows,
+                                              Load &&load) {
+    int r = 0;
+    for (; r + 128 <= n_rows; r += 128) load(dst + r * kRowBytes, &maps.act[0], k0, row + r);
+    if (r + 64 <= n_rows) { load(dst + r * kRowBytes, &maps.act[1], k0, row + r); r += 64; }
+    if (r + 32 <= n_rows) { load(dst + r * kRowBytes, &maps.act[2], k0, row + r); r += 32; }
+    if (r + 16 <= n_rows) { load(dst + r * kRowBytes, &maps.act[3], k0, row + r); r += 16; }
+}
+
+struct Tile {
+    int e, f, row0, n_valid;
+};
+// Tile order: expert-major, then weight slab, then the expert's token tiles (fastest), so tiles that
+// share a weight slab run at the same time on neighbouring CTAs.
+__device__ __forceinline__ Tile decode_tile(int tile, const KernelParams &p) {
+    int lo = 0, hi = p.E;
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (p.tile_prefix[mid] * p.n_feature_tiles <= tile) lo = mid; else hi = mid;
+    }
+    Tile t;
+    t.e = lo;
+    const int first = p.tile_prefix[lo], n_tok_tiles = p.tile_prefix[lo + 1] - first;
+    const int local = tile - first * p.n_feature_tiles;
+    t.f = local / n_tok_tiles;
+    const int j = local - t.f * n_tok_tiles;
+    const int rows = p.tile_rows[lo];
+    const int begin = p.expert_offsets[lo], count = p.expert_offsets[lo + 1] - begin;
+    t.row0 = begin + j * rows;
+    t.n_valid = min(rows, count - j * rows);
+    return t;
+}
+
+// SiLU(g) * u with the fast exponential; exp overflow gives g / inf = -0 for very negative g.
+__device__ __forceinline__ float swiglu(float g, float u) { return __fdividef(g, 1.f + __expf(-g)) * u; }
+
+// ---- host side ----------------------------------------------------------------------------------
+bool encode_weight_map_2d(CUtensorMap *map, const void *w, uint64_t rows, uint64_t K);
+bool encode_weight_map_gate_up(CUtensorMap *map, const void *w13, int E, int I, int H);
+bool encode_act_maps(CUtensorMap *maps, const void *act, uint64_t rows, uint64_t K);
+int sm_count();
+
+}  // namespace tc
+}  // namespace moe

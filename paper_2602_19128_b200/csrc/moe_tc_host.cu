@@ -1,0 +1,84 @@
+// Host-side helpers of the tcgen05 grouped GEMMs: TMA tensor-map encoding (through the driver entry
+// point, so the library links against no driver stub and loads on a machine without a GPU) and the
+// SM count.
+#include "moe_tc_common.cuh"
+
+#include <mutex>
+
+namespace moe {
+namespace tc {
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void *ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    });
+    return fn;
+}
+
+bool encode(CUtensorMap *map, const void *base, int rank, const cuuint64_t *dims, const cuuint64_t *strides,
+            const cuuint32_t *box) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    const cuuint32_t elem_strides[5] = {1, 1, 1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void *>(base), dims, strides, box, elem_strides,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// 2-D bf16 tensor [rows, cols] row-major; box = box_rows x 64 columns, 128-byte swizzle, zero fill.
+bool encode_2d(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {cols * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kBlockK, box_rows};
+    return encode(map, base, 2, dims, strides, box);
+}
+
+}  // namespace
+
+bool encode_weight_map_2d(CUtensorMap *map, const void *w, uint64_t rows, uint64_t K) {
+    return encode_2d(map, w, rows, K, kTileM);
+}
+
+// w13 [E, 2I, H] viewed as [E][I/16 groups][2 halves][16 rows][H]: coordinates (k, row, half, group,
+// expert).  The {64,16,2,4,1} box lands in shared memory as, for each of 4 consecutive groups, 16
+// gate rows followed by the 16 up rows of the same features: one copy per 128-row A slot.
+bool encode_weight_map_gate_up(CUtensorMap *map, const void *w13, int E, int I, int H) {
+    const cuuint64_t row_bytes = (cuuint64_t)H * 2;
+    const cuuint64_t dims[5] = {(cuuint64_t)H, 16, 2, (cuuint64_t)(I / 16), (cuuint64_t)E};
+    const cuuint64_t strides[4] = {row_bytes, (cuuint64_t)I * row_bytes, 16 * row_bytes, 2 * (cuuint64_t)I * row_bytes};
+    const cuuint32_t box[5] = {(cuuint32_t)kBlockK, 16, 2, 4, 1};
+    return encode(map, w13, 5, dims, strides, box);
+}
+
+bool encode_act_maps(CUtensorMap *maps, const void *act, uint64_t rows, uint64_t K) {
+    const uint32_t box_rows[kNumActMaps] = {128, 64, 32, 16};
+    for (int i = 0; i < kNumActMaps; ++i)
+        if (!encode_2d(&maps[i], act, rows, K, box_rows[i])) return false;
+    return true;
+}
+
+int sm_count() {
+    static int cached[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 1;
+    if (cached[dev] == 0) {
+        int n = 0;
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+        cached[dev] = n > 0 ? n : 1;
+    }
+    return cached[dev];
+}
+
+}  // namespace tc
+}  // namespace moe
