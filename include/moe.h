@@ -68,6 +68,9 @@ typedef enum {
 /* Run the two grouped GEMMs on plain CUDA-core kernels instead of the tcgen05 kernels.  Meant
  * for validating the tensor-core path at sizes the CPU cannot check in full; about 100x slower. */
 #define MOE_FLAG_VALIDATION_GEMM 1u
+/* Keep the tcgen05 GEMMs on the one-CTA-per-tile kernel even where the CTA-pair kernel would be
+ * chosen (token tiles of up to 128 / 256 rows).  For tests and A/B timing. */
+#define MOE_FLAG_SINGLE_CTA_GEMM 2u
 
 /* Byte offsets of the intermediates inside the workspace of moe_forward (so tests and tools can
  * read them after the stream has been synchronised).  Filled by moe_workspace_layout(). */

@@ -16,6 +16,7 @@ _LIB_PATH = Path(__file__).resolve().parent / "libmoe_b200.so"
 MOE_OK = 0
 MOE_FLAG_NONE = 0
 MOE_FLAG_VALIDATION_GEMM = 1
+MOE_FLAG_SINGLE_CTA_GEMM = 2
 
 EXPORTED = ["moe_workspace_bytes", "moe_workspace_layout", "moe_route_workspace_bytes", "moe_route", "moe_forward",
             "moe_forward_ex", "moe_forward_staged", "moe_forward_host", "moe_last_status", "moe_forward_launch_count", "moe_status_string"]

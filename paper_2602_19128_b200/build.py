@@ -13,7 +13,7 @@ PKG = Path(__file__).resolve().parent
 ROOT = PKG.parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libmoe_b200.so"
-SOURCES = ["moe_api.cu", "moe_route.cu", "moe_gemm_tc.cu", "moe_tc_host.cu", "moe_gemm_validation.cu"]
+SOURCES = ["moe_api.cu", "moe_route.cu", "moe_gemm_tc.cu", "moe_gemm_tc_pair.cu", "moe_tc_host.cu", "moe_gemm_validation.cu"]
 
 
 def _nvcc() -> str:
@@ -39,6 +39,7 @@ def build_library(force: bool = False, verbose: bool = False) -> Path:
            "-I", str(ROOT / "include"), "-I", str(CSRC)]
     if verbose:
         cmd += ["-Xptxas", "-v"]
+    cmd += os.environ.get("MOE_NVCC_FLAGS", "").split()  # extra flags for experiment builds
     cmd += [str(CSRC / s) for s in SOURCES] + ["-o", str(tmp)]
     subprocess.run(cmd, check=True)
     os.replace(tmp, LIB)

@@ -52,7 +52,7 @@ int forward_impl(const void *x, const float *logits, const void *w13, const void
                  void *const *stage_events = nullptr) {
     if (T < 0 || H <= 0 || I <= 0 || E <= 0 || k <= 0 || k > E) return MOE_ERR_SHAPE;
     if (!envelope_ok(T, H, I, E, k)) return MOE_ERR_UNSUPPORTED;
-    if (flags & ~MOE_FLAG_VALIDATION_GEMM) return MOE_ERR_UNSUPPORTED;
+    if (flags & ~(MOE_FLAG_VALIDATION_GEMM | MOE_FLAG_SINGLE_CTA_GEMM)) return MOE_ERR_UNSUPPORTED;
     if (T == 0) return MOE_OK;
     if (!x || !logits || !w13 || !w2 || !out || !workspace) return MOE_ERR_NULL;
     if (!aligned(x, 16) || !aligned(logits, 16) || !aligned(w13, 16) || !aligned(w2, 16) || !aligned(out, 16) ||
@@ -92,7 +92,7 @@ int forward_impl(const void *x, const float *logits, const void *w13, const void
     GroupedGemmArgs g1;
     g1.act = x_perm; g1.w = static_cast<const __nv_bfloat16 *>(w13); g1.out = h;
     g1.A = A; g1.K = H; g1.n_out = I; g1.E = E; g1.w_rows = 2 * I; g1.nt_max = nt_max;
-    g1.expert_offsets = offsets; g1.tile_prefix = rs.tile_prefix; g1.tile_rows = rs.tile_rows;
+    g1.expert_offsets = offsets; g1.tile_prefix = rs.tile_prefix; g1.tile_order = rs.tile_order; g1.tile_rows = rs.tile_rows;
     g1.status = status; g1.swiglu = true;
     GroupedGemmArgs g2 = g1;
     g2.act = h; g2.w = static_cast<const __nv_bfloat16 *>(w2); g2.out = y;
@@ -103,10 +103,14 @@ int forward_impl(const void *x, const float *logits, const void *w13, const void
         if (!mark(3)) return MOE_ERR_CUDA;
         if (launch_grouped_gemm_validation(g2, stream) != cudaSuccess) return MOE_ERR_CUDA;
     } else {
-        int st = launch_grouped_gemm_tc(g1, stream);
+        // CTA pairs where the token tiles are large enough for the halved token-tile traffic to matter
+        const bool single = (flags & MOE_FLAG_SINGLE_CTA_GEMM) != 0;
+        int st = (!single && grouped_gemm_tc_pair_supported(g1)) ? launch_grouped_gemm_tc_pair(g1, stream)
+                                                                 : launch_grouped_gemm_tc(g1, stream);
         if (st != MOE_OK) return st;
         if (!mark(3)) return MOE_ERR_CUDA;
-        st = launch_grouped_gemm_tc(g2, stream);
+        st = (!single && grouped_gemm_tc_pair_supported(g2)) ? launch_grouped_gemm_tc_pair(g2, stream)
+                                                             : launch_grouped_gemm_tc(g2, stream);
         if (st != MOE_OK) return st;
     }
     if (!mark(4)) return MOE_ERR_CUDA;

@@ -62,6 +62,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 grouped_gemm_tc_kernel(const __grid_constant__ TensorMaps maps, const KernelParams p) {
     using L = SmemLayout<NT_MAX, STAGES>;
     constexpr int kTmemCols = 2 * NT_MAX;
+    constexpr int kSiteOffset = SWIGLU ? 0 : 4;  // the down GEMM reports sites 5..8
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *base_ptr = smem_raw + (base - smem_u32(smem_raw));
@@ -102,16 +103,27 @@ grouped_gemm_tc_kernel(const __grid_constant__ TensorMaps maps, const KernelPara
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+            for (int round = 0; ok; ++round) {
+                const int tile = tile_of_round(round, blockIdx.x, gridDim.x);
+                if (tile >= total_tiles) break;
                 const Tile t = decode_tile(tile, p);
                 const int n_mma = (t.n_valid + 15) & ~15;
                 const int w_row = t.e * p.w_rows + t.f * kTileM;  // down projection: 128 rows of w2[e]
                 const uint32_t tx_bytes = kSlotABytes + n_mma * kRowBytes;
                 for (int kb = 0; kb < p.n_k_blocks; ++kb) {
-                    ok = mbar_wait(bar_empty + stage * 8, phase ^ 1u, abort_flag, p.status, kSiteProducerEmpty);
+                    ok = mbar_wait(bar_empty + stage * 8, phase ^ 1u, abort_flag, p.status, kSiteProducerEmpty + kSiteOffset);
                     if (!ok) break;
                     const uint32_t full = bar_full + stage * 8;
+#ifdef MOE_ABLATE_NO_TMA  // experiment builds only: time the MMA side alone
+                    mbar_arrive(full);
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                    continue;
+#endif
+#ifdef MOE_ABLATE_NO_B
+                    mbar_expect_tx(full, kSlotABytes);
+#else
                     mbar_expect_tx(full, tx_bytes);
+#endif
                     const uint32_t sa = base + L::kA + stage * kSlotABytes;
                     const uint32_t sb = base + L::kB + stage * L::kSlotBBytes;
                     const int k0 = kb * kBlockK;
@@ -119,9 +131,9 @@ grouped_gemm_tc_kernel(const __grid_constant__ TensorMaps maps, const KernelPara
                         tma_load_5d(sa, &maps.w, k0, 0, 0, t.f * 4, t.e, full);
                     else
                         tma_load_2d(sa, &maps.w, k0, w_row, full);
-                    load_act_rows(maps, sb, k0, t.row0, n_mma, [&](uint32_t dst, const CUtensorMap *m, int c0, int c1) {
-                        tma_load_2d(dst, m, c0, c1, full);
-                    });
+#ifndef MOE_ABLATE_NO_B
+                    tma_load_2d(sb, act_map(maps, n_mma), k0, t.row0, full);
+#endif
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -133,22 +145,26 @@ grouped_gemm_tc_kernel(const __grid_constant__ TensorMaps maps, const KernelPara
             int stage = 0, acc = 0;
             uint32_t phase = 0, acc_phase = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+            for (int round = 0; ok; ++round) {
+                const int tile = tile_of_round(round, blockIdx.x, gridDim.x);
+                if (tile >= total_tiles) break;
                 const Tile t = decode_tile(tile, p);
                 const uint32_t idesc = instr_desc_bf16(kTileM, (t.n_valid + 15) & ~15);
-                ok = mbar_wait(bar_acc_empty + acc * 8, acc_phase ^ 1u, abort_flag, p.status, kSiteMmaTmemEmpty);
+                ok = mbar_wait(bar_acc_empty + acc * 8, acc_phase ^ 1u, abort_flag, p.status, kSiteMmaTmemEmpty + kSiteOffset);
                 if (!ok) break;
                 tcgen05_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * NT_MAX;
                 for (int kb = 0; kb < p.n_k_blocks; ++kb) {
-                    ok = mbar_wait(bar_full + stage * 8, phase, abort_flag, p.status, kSiteMmaFull);
+                    ok = mbar_wait(bar_full + stage * 8, phase, abort_flag, p.status, kSiteMmaFull + kSiteOffset);
                     if (!ok) break;
                     tcgen05_fence_after();
                     const uint64_t a_desc = smem_desc_k_major_sw128(base + L::kA + stage * kSlotABytes);
                     const uint64_t b_desc = smem_desc_k_major_sw128(base + L::kB + stage * L::kSlotBBytes);
 #pragma unroll
+#ifndef MOE_ABLATE_NO_MMA  // (experiment builds may drop the MMAs to time the load side alone)
                     for (int kk = 0; kk < kBlockK / 16; ++kk)  // 16 K-elements = 32 bytes = 2 descriptor units
                         umma_bf16(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (kb | kk) != 0);
+#endif
                     umma_commit(bar_empty + stage * 8);
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
@@ -164,10 +180,12 @@ grouped_gemm_tc_kernel(const __grid_constant__ TensorMaps maps, const KernelPara
         int acc = 0;
         uint32_t acc_phase = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+        for (int round = 0; ok; ++round) {
+                const int tile = tile_of_round(round, blockIdx.x, gridDim.x);
+                if (tile >= total_tiles) break;
             const Tile t = decode_tile(tile, p);
             const int n_mma = (t.n_valid + 15) & ~15;
-            ok = mbar_wait(bar_acc_full + acc * 8, acc_phase, abort_flag, p.status, kSiteEpilogueTmemFull);
+            ok = mbar_wait(bar_acc_full + acc * 8, acc_phase, abort_flag, p.status, kSiteEpilogueTmemFull + kSiteOffset);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tcgen05_fence_after();
@@ -257,6 +275,7 @@ int launch_grouped_gemm_tc(const GroupedGemmArgs &a, cudaStream_t stream) {
     p.out = a.out;
     p.expert_offsets = a.expert_offsets;
     p.tile_prefix = a.tile_prefix;
+    p.tile_order = a.tile_order;
     p.tile_rows = a.tile_rows;
     p.status = a.status;
     p.E = a.E;

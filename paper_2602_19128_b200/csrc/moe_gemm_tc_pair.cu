@@ -1,0 +1,352 @@
+// Grouped expert GEMMs on CTA pairs: tcgen05.mma.cta_group::2, a 256 x N tile per pair.
+//
+// Same role split, ring and tile schedule as the one-CTA kernel (moe_gemm_tc.cu; paper Sec. 4.5
+// "Expert FFN computation" for what is computed), but two CTAs of a cluster work on one tile:
+// each CTA stages its own 128 weight rows and only HALF of the token tile (N/2 rows), and the
+// pair's MMA reads both halves.  Per useful flop the SMs pull (1/N + 1/256) bytes from L2 instead
+// of (1/N + 1/128), which is what bounds the prefill-sized workloads; no load is multicast, every
+// CTA fetches what it stages.
+//
+// Protocol (rank 0 = leader):
+//   full[s]      lives in the leader.  The leader's producer arms it with the bytes of BOTH CTAs;
+//                both producers' TMA copies (cta_group::2 form) complete on it.
+//   empty[s]     one per CTA.  The leader's MMA thread commits ring slots back with a commit that
+//                arrives on the barrier of both CTAs.
+//   acc_full[a]  one per CTA, same commit form; each CTA's epilogue warps drain their own TMEM
+//                (128 weight rows x N tokens) and arrive on the LEADER's acc_empty[a] (8 arrivals).
+// Before leaving, each producer waits until every ring slot has been handed back and the leader
+// waits for both accumulators to be released, so no arrival can reach a CTA that has exited; a
+// cluster barrier then precedes the TMEM release.  Every wait is bounded as in the one-CTA kernel.
+#include "moe_tc_common.cuh"
+
+namespace moe {
+namespace {
+
+using namespace tc;
+
+constexpr int kPairThreads = 224;  // warp 0 weight TMA, warp 1 MMA, warps 2..5 epilogue, warp 6 token TMA
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// Address of the same shared-memory location in CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void store_cluster_u32(uint32_t cluster_addr, uint32_t v) {
+    asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(cluster_addr), "r"(v) : "memory");
+}
+// TMA copies whose completion is signalled on a barrier that may live in the peer CTA.
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, int c0, int c1, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_5d_pair(uint32_t dst, const CUtensorMap *map, int c0, int c1, int c2, int c3,
+                                                 int c4, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.5d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(bar)
+        : "memory");
+}
+// D[tmem of both CTAs] (+)= A * B^T over the pair: M = 256 (128 rows per CTA), B halves from both CTAs.
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                               uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// Arrive, on the barrier at this offset in BOTH CTAs, once the MMAs issued so far have completed.
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+    const uint16_t both = 3;
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"(both)
+                 : "memory");
+}
+
+// Bounded wait that also raises the peer's abort flag when it expires.
+__device__ __forceinline__ bool pair_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, uint32_t peer_abort,
+                                          int *status, int site) {
+    const bool ok = mbar_wait(bar, parity, abort_flag, status, site);
+    if (!ok) store_cluster_u32(peer_abort, 1u);
+    return ok;
+}
+
+template <int NT_MAX, int STAGES>
+struct PairSmem {
+    static constexpr int kSlotBBytes = (NT_MAX / 2) * kRowBytes;
+    static constexpr int kA = 0;
+    static constexpr int kB = STAGES * kSlotABytes;
+    static constexpr int kBars = kB + STAGES * kSlotBBytes;  // full[S], empty[S], acc_full[2], acc_empty[2]
+    static constexpr int kTmemSlot = kBars + (2 * STAGES + 4) * 8;
+    static constexpr int kAbort = kTmemSlot + 4;
+    static constexpr int kBytes = kAbort + 4;
+    static constexpr int kDynamicBytes = kBytes + 1024;
+};
+
+template <int NT_MAX, int STAGES, bool SWIGLU>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
+grouped_gemm_tc_pair_kernel(const __grid_constant__ TensorMaps maps, const KernelParams p) {
+    using L = PairSmem<NT_MAX, STAGES>;
+    constexpr int kTmemCols = 2 * NT_MAX;
+    constexpr int kSiteOffset = SWIGLU ? 0 : 4;  // the down GEMM reports sites 5..8
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *base_ptr = smem_raw + (base - smem_u32(smem_raw));
+    const uint32_t bar_full = base + L::kBars, bar_empty = bar_full + STAGES * 8;
+    const uint32_t bar_acc_full = bar_empty + STAGES * 8, bar_acc_empty = bar_acc_full + 16;
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(base_ptr + L::kTmemSlot);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(base_ptr + L::kAbort);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();
+    const uint32_t peer_abort = map_to_cta(base + L::kAbort, rank ^ 1u);
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(bar_full + s * 8, 1);
+            mbar_init(bar_empty + s * 8, 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(bar_acc_full + a * 8, 1);
+            mbar_init(bar_acc_empty + a * 8, 2 * kEpilogueWarps);
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {  // collective over the same warp of both CTAs
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(base + L::kTmemSlot),
+                     "r"(kTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tcgen05_fence_before();
+    __syncthreads();
+    cluster_sync_all();  // the peer's barriers exist before anything can signal them
+    tcgen05_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const int total_tiles = p.tile_prefix[p.E] * p.n_feature_tiles;
+    const int n_pairs = gridDim.x >> 1, pair = blockIdx.x >> 1;
+
+    // ---------------- TMA producers (both CTAs) ----------------
+    // The weight slab and the token rows of a slot are issued by two different warps: a copy
+    // instruction occupies its issuing thread for a while, and two issuers keep the ring ahead.
+    auto producer_loop = [&](const bool load_w, const bool load_act) {
+        int stage = 0;
+        uint32_t phase = 0;
+        bool ok = true;
+        for (int round = 0; ok; ++round) {
+            const int tile = tile_of_round(round, pair, n_pairs);
+            if (tile >= total_tiles) break;
+            const Tile t = decode_tile(tile, p);
+            const int n_mma = (t.n_valid + 31) & ~31, half = n_mma >> 1;
+            const int w_row = t.e * p.w_rows + t.f * (2 * kTileM) + (int)rank * kTileM;  // down projection
+            for (int kb = 0; kb < p.n_k_blocks; ++kb) {
+                ok = pair_wait(bar_empty + stage * 8, phase ^ 1u, abort_flag, peer_abort, p.status, kSiteProducerEmpty + kSiteOffset);
+                if (!ok) break;
+                const uint32_t full = map_to_cta(bar_full + stage * 8, 0);
+                const int k0 = kb * kBlockK;
+                if (load_w) {
+#ifdef MOE_ABLATE_NO_TMA  // experiment builds only: time the MMA side alone
+                    if (rank == 0) mbar_arrive(bar_full + stage * 8);
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                    continue;
+#endif
+#ifdef MOE_ABLATE_NO_B
+                    if (rank == 0) mbar_expect_tx(bar_full + stage * 8, 2 * kSlotABytes);
+#else
+                    if (rank == 0) mbar_expect_tx(bar_full + stage * 8, 2 * kSlotABytes + n_mma * kRowBytes);
+#endif
+                    const uint32_t sa = base + L::kA + stage * kSlotABytes;
+                    if (SWIGLU)  // this CTA's 64 features = groups 8f + 4*rank .. +3 of 16
+                        tma_load_5d_pair(sa, &maps.w, k0, 0, 0, t.f * 8 + (int)rank * 4, t.e, full);
+                    else
+                        tma_load_2d_pair(sa, &maps.w, k0, w_row, full);
+                }
+#if !defined(MOE_ABLATE_NO_B) && !defined(MOE_ABLATE_NO_TMA)
+                if (load_act) {
+                    const uint32_t sb = base + L::kB + stage * L::kSlotBBytes;
+                    tma_load_2d_pair(sb, act_map(maps, half), k0, t.row0 + (int)rank * half, full);
+                }
+#endif
+                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+            }
+        }
+        // wait until every slot has been handed back: no commit may arrive here after exit
+        for (int s = 0; ok && s < STAGES; ++s) {
+            ok = pair_wait(bar_empty + stage * 8, phase ^ 1u, abort_flag, peer_abort, p.status, kSiteProducerEmpty + kSiteOffset);
+            if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+    };
+    if (warp == 0) {
+        if (lane == 0) producer_loop(true, false);
+        __syncwarp();
+    } else if (warp == kPairThreads / 32 - 1) {
+        if (lane == 0) producer_loop(false, true);
+        __syncwarp();
+    } else if (warp == 1) {
+        // ---------------- MMA issuer (leader CTA only) ----------------
+        if (lane == 0 && rank == 0) {
+            int stage = 0, acc = 0;
+            uint32_t phase = 0, acc_phase = 0;
+            bool ok = true;
+            for (int round = 0; ok; ++round) {
+            const int tile = tile_of_round(round, pair, n_pairs);
+            if (tile >= total_tiles) break;
+                const Tile t = decode_tile(tile, p);
+                const uint32_t idesc = instr_desc_bf16(2 * kTileM, (t.n_valid + 31) & ~31);
+                ok = pair_wait(bar_acc_empty + acc * 8, acc_phase ^ 1u, abort_flag, peer_abort, p.status, kSiteMmaTmemEmpty + kSiteOffset);
+                if (!ok) break;
+                tcgen05_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * NT_MAX;
+                for (int kb = 0; kb < p.n_k_blocks; ++kb) {
+                    ok = pair_wait(bar_full + stage * 8, phase, abort_flag, peer_abort, p.status, kSiteMmaFull + kSiteOffset);
+                    if (!ok) break;
+                    tcgen05_fence_after();
+                    const uint64_t a_desc = smem_desc_k_major_sw128(base + L::kA + stage * kSlotABytes);
+                    const uint64_t b_desc = smem_desc_k_major_sw128(base + L::kB + stage * L::kSlotBBytes);
+#ifndef MOE_ABLATE_NO_MMA  // (experiment builds may drop the MMAs to time the load side alone)
+#pragma unroll
+                    for (int kk = 0; kk < kBlockK / 16; ++kk)
+                        umma_bf16_pair(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (kb | kk) != 0);
+#endif
+                    umma_commit_pair(bar_empty + stage * 8);
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+                if (!ok) break;
+                umma_commit_pair(bar_acc_full + acc * 8);
+                if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+            }
+            // wait until both accumulators have been released by both CTAs' epilogues
+            for (int a = 0; ok && a < 2; ++a) {
+                ok = pair_wait(bar_acc_empty + acc * 8, acc_phase ^ 1u, abort_flag, peer_abort, p.status, kSiteMmaTmemEmpty + kSiteOffset);
+                if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+            }
+        }
+        __syncwarp();
+    } else {
+        // ---------------- epilogue (both CTAs): own 128 weight rows x all N tokens ----------------
+        const int q = warp & 3;
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        bool ok = true;
+        for (int round = 0; ok; ++round) {
+            const int tile = tile_of_round(round, pair, n_pairs);
+            if (tile >= total_tiles) break;
+            const Tile t = decode_tile(tile, p);
+            const int n_mma = (t.n_valid + 31) & ~31;
+            ok = pair_wait(bar_acc_full + acc * 8, acc_phase, abort_flag, peer_abort, p.status, kSiteEpilogueTmemFull + kSiteOffset);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tcgen05_fence_after();
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + acc * NT_MAX;
+            if (SWIGLU) {
+                const int hi = lane >> 4;
+                __nv_bfloat16 *dst = p.out + (size_t)t.row0 * p.n_out + t.f * kTileM + (int)rank * (kTileM / 2) + q * 16 + (lane & 15);
+                for (int c0 = 0; c0 < n_mma; c0 += 16) {
+                    float v[16];
+                    tmem_load_16(taddr + c0, v);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const float other = __shfl_xor_sync(0xffffffffu, hi ? v[i] : v[8 + i], 16);
+                        const float g = hi ? other : v[i];
+                        const float u = hi ? v[8 + i] : other;
+                        const int col = c0 + hi * 8 + i;
+                        if (col < t.n_valid) dst[(size_t)col * p.n_out] = __float2bfloat16_rn(swiglu(g, u));
+                    }
+                }
+            } else {
+                __nv_bfloat16 *dst = p.out + (size_t)t.row0 * p.n_out + t.f * (2 * kTileM) + (int)rank * kTileM + q * 32 + lane;
+                for (int c0 = 0; c0 < n_mma; c0 += 16) {
+                    float v[16];
+                    tmem_load_16(taddr + c0, v);
+#pragma unroll
+                    for (int i = 0; i < 16; ++i)
+                        if (c0 + i < t.n_valid) dst[(size_t)(c0 + i) * p.n_out] = __float2bfloat16_rn(v[i]);
+                }
+            }
+            tcgen05_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(map_to_cta(bar_acc_empty + acc * 8, 0));
+            if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        }
+    }
+
+    // ---------------- teardown ----------------
+    tcgen05_fence_before();
+    __syncthreads();
+    cluster_sync_all();
+    if (*abort_flag) {
+        for (int i = 0; i < 1000; ++i) __nanosleep(1000);
+    }
+    if (warp == 1) {
+        tcgen05_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    }
+}
+
+template <int NT_MAX, int STAGES, bool SWIGLU>
+int launch_pair_instance(const TensorMaps &maps, const KernelParams &p, int grid, cudaStream_t stream) {
+    using L = PairSmem<NT_MAX, STAGES>;
+    static_assert(L::kDynamicBytes <= 232448, "ring does not fit in shared memory");
+    auto kernel = grouped_gemm_tc_pair_kernel<NT_MAX, STAGES, SWIGLU>;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) != cudaSuccess)
+        return MOE_ERR_CUDA;
+    kernel<<<grid, kPairThreads, L::kDynamicBytes, stream>>>(maps, p);
+    return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
+
+}  // namespace
+
+bool grouped_gemm_tc_pair_supported(const GroupedGemmArgs &a) {
+    return (a.nt_max == 128 || a.nt_max == 256) && a.K % kBlockK == 0 && a.A > 0 &&
+           a.n_out % (a.swiglu ? kTileM : 2 * kTileM) == 0;
+}
+
+int launch_grouped_gemm_tc_pair(const GroupedGemmArgs &a, cudaStream_t stream) {
+    if (!grouped_gemm_tc_pair_supported(a)) return MOE_ERR_UNSUPPORTED;
+    TensorMaps maps;
+    const bool ok_w = a.swiglu ? encode_weight_map_gate_up(&maps.w, a.w, a.E, a.n_out, a.K)
+                               : encode_weight_map_2d(&maps.w, a.w, (uint64_t)a.E * a.w_rows, a.K);
+    if (!ok_w || !encode_act_maps(maps.act, a.act, a.A, a.K)) return MOE_ERR_CUDA;
+
+    KernelParams p;
+    p.out = a.out;
+    p.expert_offsets = a.expert_offsets;
+    p.tile_prefix = a.tile_prefix;
+    p.tile_order = a.tile_order;
+    p.tile_rows = a.tile_rows;
+    p.status = a.status;
+    p.E = a.E;
+    p.n_k_blocks = a.K / kBlockK;
+    p.n_out = a.n_out;
+    p.w_rows = a.w_rows;
+    p.n_feature_tiles = a.n_out / (a.swiglu ? kTileM : 2 * kTileM);
+
+    const long long max_token_tiles = (long long)(a.A < a.E ? a.A : a.E) + a.A / a.nt_max;
+    const long long max_tiles = max_token_tiles * p.n_feature_tiles;
+    const int pairs_on_device = sm_count() / 2;
+    const int n_pairs = (int)(max_tiles < pairs_on_device ? max_tiles : pairs_on_device);
+    const int grid = 2 * (n_pairs > 0 ? n_pairs : 1);
+    if (a.nt_max == 256)
+        return a.swiglu ? launch_pair_instance<256, 7, true>(maps, p, grid, stream)
+                        : launch_pair_instance<256, 7, false>(maps, p, grid, stream);
+    return a.swiglu ? launch_pair_instance<128, 9, true>(maps, p, grid, stream)
+                    : launch_pair_instance<128, 9, false>(maps, p, grid, stream);
+}
+
+}  // namespace moe

@@ -17,7 +17,7 @@ constexpr int kMaxTopK = 32;            // lane j of the token's warp owns rank 
 constexpr int kRouteTokensPerBlock = 32;  // tokens per router block = one histogram chunk
 constexpr int kStatusInts = 4;          // status word: {status, site, aux0, aux1}
 
-// Site ids recorded next to MOE_ERR_DEVICE_TIMEOUT.
+// Site ids recorded next to MOE_ERR_DEVICE_TIMEOUT (gate/up GEMM; the down GEMM adds 4).
 enum : int { kSiteProducerEmpty = 1, kSiteMmaFull = 2, kSiteMmaTmemEmpty = 3, kSiteEpilogueTmemFull = 4 };
 
 static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -25,7 +25,8 @@ static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; 
 // Scratch of the router / sort-scatter, all int32, carved out of the caller's workspace.
 struct RouteScratch {
     int *chunk_counts;  // [n_chunks, E] per-chunk expert histogram, then per-chunk start positions
-    int *tile_prefix;   // [E+1] exclusive prefix sum of token tiles per expert
+    int *tile_prefix;   // [E+1] exclusive prefix sum of token tiles over experts in schedule order
+    int *tile_order;    // [E]   expert at each schedule position: most rows first, ties to the lower index
     int *tile_rows;     // [E]   rows per token tile of this expert (multiple of 16; 0 if empty)
     int n_chunks;
 };
@@ -33,7 +34,7 @@ struct RouteScratch {
 static inline int route_num_chunks(int T) { return (T + kRouteTokensPerBlock - 1) / kRouteTokensPerBlock; }
 
 static inline size_t route_scratch_bytes(int T, int E) {
-    size_t ints = (size_t)route_num_chunks(T) * E + (size_t)(E + 1) + (size_t)E;
+    size_t ints = (size_t)route_num_chunks(T) * E + (size_t)(E + 1) + 2 * (size_t)E;
     return align_up(ints * sizeof(int), 256);
 }
 
@@ -42,7 +43,8 @@ static inline RouteScratch carve_route_scratch(void *base, int T, int E) {
     s.n_chunks = route_num_chunks(T);
     s.chunk_counts = reinterpret_cast<int *>(base);
     s.tile_prefix = s.chunk_counts + (size_t)s.n_chunks * E;
-    s.tile_rows = s.tile_prefix + (E + 1);
+    s.tile_order = s.tile_prefix + (E + 1);
+    s.tile_rows = s.tile_order + E;
     return s;
 }
 
@@ -72,12 +74,18 @@ struct GroupedGemmArgs {
     int w_rows;                // rows per expert in w (2I for gemm1, H for gemm2)
     int nt_max;                // token-tile bound the schedule was built with
     const int *expert_offsets; // [E+1]
-    const int *tile_prefix;    // [E+1]
+    const int *tile_prefix;    // [E+1] in schedule order
+    const int *tile_order;     // [E]
     const int *tile_rows;      // [E]
     int *status;               // status word
     bool swiglu;
 };
 int launch_grouped_gemm_tc(const GroupedGemmArgs &args, cudaStream_t stream);  // returns a moe_status_t
+
+// The same GEMM on CTA pairs (cta_group::2, 256 x N tiles); only for token-tile bounds of 128 / 256
+// and feature counts the 256-row pair tile divides.
+bool grouped_gemm_tc_pair_supported(const GroupedGemmArgs &args);
+int launch_grouped_gemm_tc_pair(const GroupedGemmArgs &args, cudaStream_t stream);
 
 // Same contract on plain CUDA cores (validation only).
 cudaError_t launch_grouped_gemm_validation(const GroupedGemmArgs &args, cudaStream_t stream);

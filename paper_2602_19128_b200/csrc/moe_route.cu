@@ -126,8 +126,9 @@ __device__ __forceinline__ int block_exclusive_scan_256(int value, int *warp_sum
 
 __global__ void __launch_bounds__(256)
 route_scan_kernel(int *__restrict__ chunk_counts, int n_chunks, int E, int nt_max, int *__restrict__ expert_offsets,
-                  int *__restrict__ tile_prefix, int *__restrict__ tile_rows) {
+                  int *__restrict__ tile_prefix, int *__restrict__ tile_order, int *__restrict__ tile_rows) {
     __shared__ int warp_sums[8];
+    __shared__ int counts[kMaxExperts], tiles_at[kMaxExperts];
     const int e = threadIdx.x;
     int count = 0;
     if (e < E) {
@@ -137,6 +138,8 @@ route_scan_kernel(int *__restrict__ chunk_counts, int n_chunks, int E, int nt_ma
             count += c;
         }
     }
+    counts[e] = e < E ? count : -1;
+    tiles_at[e] = 0;
     // token tiles of this expert: as few as fit under nt_max, evenly sized, rounded up to 16 rows
     int n_tiles = 0, rows = 0;
     if (count > 0) {
@@ -144,11 +147,20 @@ route_scan_kernel(int *__restrict__ chunk_counts, int n_chunks, int E, int nt_ma
         rows = (((count + n_tiles - 1) / n_tiles) + 15) & ~15;
     }
     int total_rows, total_tiles;
-    const int row_start = block_exclusive_scan_256(count, warp_sums, &total_rows);
-    const int tile_start = block_exclusive_scan_256(n_tiles, warp_sums, &total_tiles);
+    const int row_start = block_exclusive_scan_256(count, warp_sums, &total_rows);  // (syncs: counts[] is visible)
+    // Schedule order: experts with more rows first (ties to the lower index), so that tiles of similar
+    // cost are adjacent and the GEMMs' static tile assignment stays balanced; the small tiles come last.
+    int pos = 0;
+    if (e < E) {
+        for (int o = 0; o < E; ++o) pos += (counts[o] > count || (counts[o] == count && o < e)) ? 1 : 0;
+        tiles_at[pos] = n_tiles;
+        tile_order[pos] = e;
+    }
+    __syncthreads();
+    const int tile_start = block_exclusive_scan_256(tiles_at[e], warp_sums, &total_tiles);
     if (e < E) {
         expert_offsets[e] = row_start;
-        tile_prefix[e] = tile_start;
+        tile_prefix[e] = tile_start;  // indexed by schedule position
         tile_rows[e] = rows;
         for (int b = 0; b < n_chunks; ++b) chunk_counts[(size_t)b * E + e] += row_start;
     }
@@ -244,13 +256,13 @@ int choose_nt_max(int T, int E, int k) {
 cudaError_t launch_route(const float *logits, int T, int E, int k, int nt_max, int *topk_ids, float *topk_w,
                          int *expert_offsets, int *sorted_to_flat, int *flat_to_sorted, RouteScratch scratch,
                          int *status, cudaStream_t stream) {
-    cudaError_t err = cudaMemsetAsync(status, 0, kStatusInts * sizeof(int), stream);
+    cudaError_t err = cudaMemsetAsync(status, 0, 256, stream);  // the status word and its padding
     if (err != cudaSuccess) return err;
     const int A = T * k;
     route_topk_kernel<<<scratch.n_chunks, kRouteThreads, 0, stream>>>(logits, T, E, k, topk_ids, topk_w,
                                                                        scratch.chunk_counts);
     route_scan_kernel<<<1, 256, 0, stream>>>(scratch.chunk_counts, scratch.n_chunks, E, nt_max, expert_offsets,
-                                             scratch.tile_prefix, scratch.tile_rows);
+                                             scratch.tile_prefix, scratch.tile_order, scratch.tile_rows);
     route_scatter_kernel<<<scratch.n_chunks, 32, 0, stream>>>(topk_ids, scratch.chunk_counts, A, E, k,
                                                               sorted_to_flat, flat_to_sorted);
     return cudaGetLastError();

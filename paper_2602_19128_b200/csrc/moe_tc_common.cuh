@@ -14,19 +14,19 @@ constexpr int kRowBytes = kBlockK * 2;             // 128
 constexpr int kThreads = 192;                      // warp 0 TMA, warp 1 MMA, warps 2..5 epilogue
 constexpr int kEpilogueWarps = 4;
 constexpr long long kWaitLimitCycles = 4000000000LL;  // about two seconds at full clock
-constexpr int kNumActMaps = 4;                     // activation boxes of 128, 64, 32 and 16 rows
+constexpr int kNumActMaps = 16;                    // activation boxes of 16, 32, ..., 256 rows
 
 // Tensor maps of one grouped GEMM.  `w` is either a 2-D map over [E*w_rows, K] with a 128-row box
 // (down projection) or a 5-D map over w13 viewed as [E][I/16][gate|up][16][H] whose
 // {64,16,2,4,1} box delivers 64 features as 4 x (16 gate rows, 16 up rows) in one copy.
 struct TensorMaps {
     CUtensorMap w;
-    CUtensorMap act[kNumActMaps];  // box rows 128, 64, 32, 16
+    CUtensorMap act[kNumActMaps];  // act[i]: box of 16 * (i + 1) rows, so any token tile is ONE copy
 };
 
 struct KernelParams {
     __nv_bfloat16 *out;
-    const int *expert_offsets, *tile_prefix, *tile_rows;
+    const int *expert_offsets, *tile_prefix, *tile_order, *tile_rows;
     int *status;
     int E, n_k_blocks, n_out, w_rows, n_feature_tiles;
 };
@@ -60,7 +60,16 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     if (mbar_try_wait(bar, parity)) return true;
     const long long start = clock64();
     while (true) {
-        if (mbar_try_wait(bar, parity)) return true;
+        if (mbar_try_wait(bar, parity)) {
+#ifdef MOE_WAIT_STATS  // experiment builds only: cycles spent waiting, per site, after the status ints
+            if ((threadIdx.x & 31) == 0) {
+                unsigned long long *stats = reinterpret_cast<unsigned long long *>(status + 8);
+                atomicAdd(&stats[site], (unsigned long long)(clock64() - start));
+                atomicAdd(&stats[8 + site], 1ull);
+            }
+#endif
+            return true;
+        }
         if (*abort_flag) return false;
         if (clock64() - start > kWaitLimitCycles) {
             *abort_flag = 1;
@@ -122,23 +131,18 @@ __device__ __forceinline__ uint32_t instr_desc_bf16(int m, int n) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
-// Activation rows [row, row + n_rows) (n_rows a multiple of 16) of K block k0 into shared memory at
-// `dst`, as few boxes as the four maps allow.  LOAD(dst, map, k0, row) issues one copy.
-template <class Load>
-__device__ __forceinline__ void load_act_rows(const TensorMaps &maps, uint32_t dst, int k0, int row, int n_rows,
-                                              Load &&load) {
-    int r = 0;
-    for (; r + 128 <= n_rows; r += 128) load(dst + r * kRowBytes, &maps.act[0], k0, row + r);
-    if (r + 64 <= n_rows) { load(dst + r * kRowBytes, &maps.act[1], k0, row + r); r += 64; }
-    if (r + 32 <= n_rows) { load(dst + r * kRowBytes, &maps.act[2], k0, row + r); r += 32; }
-    if (r + 16 <= n_rows) { load(dst + r * kRowBytes, &maps.act[3], k0, row + r); r += 16; }
+// The map whose box holds exactly n_rows activation rows (n_rows a multiple of 16, at most 256).
+// One copy per ring slot and operand: every TMA copy has a fixed cost in the copy engine that is
+// comparable to moving several KiB, so a token tile is never assembled from smaller boxes.
+__device__ __forceinline__ const CUtensorMap *act_map(const TensorMaps &maps, int n_rows) {
+    return &maps.act[(n_rows >> 4) - 1];
 }
 
 struct Tile {
     int e, f, row0, n_valid;
 };
-// Tile order: expert-major, then weight slab, then the expert's token tiles (fastest), so tiles that
-// share a weight slab run at the same time on neighbouring CTAs.
+// Tile order: experts in schedule order (most rows first), then weight slab, then the expert's token
+// tiles (fastest), so tiles that share a weight slab run at the same time on neighbouring CTAs.
 __device__ __forceinline__ Tile decode_tile(int tile, const KernelParams &p) {
     int lo = 0, hi = p.E;
     while (hi - lo > 1) {
@@ -146,16 +150,23 @@ __device__ __forceinline__ Tile decode_tile(int tile, const KernelParams &p) {
         if (p.tile_prefix[mid] * p.n_feature_tiles <= tile) lo = mid; else hi = mid;
     }
     Tile t;
-    t.e = lo;
+    t.e = p.tile_order[lo];
     const int first = p.tile_prefix[lo], n_tok_tiles = p.tile_prefix[lo + 1] - first;
     const int local = tile - first * p.n_feature_tiles;
     t.f = local / n_tok_tiles;
     const int j = local - t.f * n_tok_tiles;
-    const int rows = p.tile_rows[lo];
-    const int begin = p.expert_offsets[lo], count = p.expert_offsets[lo + 1] - begin;
+    const int rows = p.tile_rows[t.e];
+    const int begin = p.expert_offsets[t.e], count = p.expert_offsets[t.e + 1] - begin;
     t.row0 = begin + j * rows;
     t.n_valid = min(rows, count - j * rows);
     return t;
+}
+
+// Static tile assignment: worker w of n_workers takes, in round i, tile i*n_workers + w on even rounds
+// and i*n_workers + (n_workers-1-w) on odd rounds.  With tiles ordered by decreasing cost this
+// back-and-forth deal keeps every worker's total within about 1 % of the mean, without atomics.
+__device__ __forceinline__ int tile_of_round(int round, int worker, int n_workers) {
+    return round * n_workers + ((round & 1) ? n_workers - 1 - worker : worker);
 }
 
 // SiLU(g) * u with the fast exponential; exp overflow gives g / inf = -0 for very negative g.

@@ -62,9 +62,8 @@ bool encode_weight_map_gate_up(CUtensorMap *map, const void *w13, int E, int I, 
 }
 
 bool encode_act_maps(CUtensorMap *maps, const void *act, uint64_t rows, uint64_t K) {
-    const uint32_t box_rows[kNumActMaps] = {128, 64, 32, 16};
     for (int i = 0; i < kNumActMaps; ++i)
-        if (!encode_2d(&maps[i], act, rows, K, box_rows[i])) return false;
+        if (!encode_2d(&maps[i], act, rows, K, 16u * (uint32_t)(i + 1))) return false;
     return true;
 }
 

@@ -21,6 +21,9 @@ SMALL = [
     (300, 128, 64, 64, 4, True),      # skewed: hot experts over 256 rows, most experts empty
     (128, 384, 128, 256, 8, False),   # decode-like: ~4 rows per expert, N = 16
     (96, 128, 256, 8, 8, False),      # k = E = 8: every expert sees every token
+    (700, 256, 256, 4, 2, False),     # CTA-pair kernel for both GEMMs, two token tiles per expert
+    (300, 512, 384, 2, 2, False),     # CTA-pair kernel, 300 rows per expert: two ragged tiles of N = 160
+    (130, 256, 128, 1, 1, False),     # one expert, 130 rows: pair tile with a nearly empty second half
 ]
 
 
@@ -34,7 +37,8 @@ def oracle_everything(case):
     return ids, w, off, s2f, f2s, h, y, out
 
 
-@pytest.mark.parametrize("flags", [moe.MOE_FLAG_VALIDATION_GEMM, moe.MOE_FLAG_NONE], ids=["cuda_core", "tcgen05"])
+@pytest.mark.parametrize("flags", [moe.MOE_FLAG_VALIDATION_GEMM, moe.MOE_FLAG_SINGLE_CTA_GEMM, moe.MOE_FLAG_NONE],
+                         ids=["cuda_core", "tcgen05_single", "tcgen05"])
 @pytest.mark.parametrize("T,H,I,E,k,skew", SMALL)
 def test_forward_matches_oracle(T, H, I, E, k, skew, flags):
     inp = gpu_inputs(dict(T=T, H=H, I=I, E=E, top_k=k, skew=skew), seed=0)
