@@ -37,7 +37,7 @@ L2_BYTES = 126 * 1024 * 1024
 # flop put mixtral / dsv3_decode (and tiny) below the ridge point and the prefill-sized ones above it.
 BOUND = {"tiny": "hbm", "mixtral": "hbm", "dsv3_decode": "hbm", "dsv3_prefill": "tensor", "skewed": "tensor"}
 # DRAM bytes (read + write) of one gate/up GEMM launch, from the ncu capture summarised under profiles/.
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {"mixtral": 1929712128}
 
 
 def load_peaks() -> dict:
