@@ -60,7 +60,8 @@ typedef enum {
     MOE_ERR_WORKSPACE = -5,      /* workspace_bytes is smaller than moe_*_workspace_bytes() */
     MOE_ERR_CUDA = -6,           /* a CUDA runtime/driver call failed (launch, descriptor encoding) */
     MOE_ERR_DEVICE_TIMEOUT = -7, /* a bounded device-side wait expired (reported by moe_last_status) */
-    MOE_ERR_ARCH = -8            /* the current device is not compute capability 10.x */
+    MOE_ERR_ARCH = -8,           /* the current device is not compute capability 10.x */
+    MOE_ERR_STATIC_LIMIT = -9    /* moe_route_static: the problem needs more than its built-in scratch */
 } moe_status_t;
 
 /* Flags for moe_forward_ex. */
@@ -113,6 +114,32 @@ MOE_API size_t moe_route_workspace_bytes(int T, int E, int top_k);
 MOE_API int moe_route(const float *router_logits, int T, int E, int top_k, int32_t *topk_ids, float *topk_weights,
               int32_t *expert_offsets, int32_t *sorted_to_flat, int32_t *flat_to_sorted, void *workspace,
               size_t workspace_bytes, void *stream);
+
+/* moe_route for callers that can neither allocate device memory nor hand the library a workspace.
+ * (The paper has no counterpart: this is a packaging variant of moe_route, not a step of the method.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a region where the framework
+ * forbids allocation (a real-time serving loop with a frozen memory plan, a plugin that is given
+ * tensors but no allocator handle), or where an allocation could synchronise the device or fragment a
+ * pool at a bad moment.  Such a caller passes only the inputs and outputs below; the scratch that
+ * moe_route takes as `workspace` lives instead in a 512 KiB array compiled into the library's device
+ * image.  Every GPU that loads the library holds those 512 KiB until the process exits.
+ *
+ * Same arguments and results as moe_route, without workspace / workspace_bytes.  Differences:
+ *   - Limit: 256 + 4 * (ceil(T/32) * E + 3 * E + 1) bytes (rounded up to 256) must fit in 512 KiB,
+ *     e.g. T <= 16256 tokens at E = 256, T <= 32640 at E = 128.  Larger problems return
+ *     MOE_ERR_STATIC_LIMIT and launch nothing; use moe_route with a workspace for those.
+ *   - The call performs no cudaMalloc / cudaFree and calls no allocating library routine.
+ *   - The first call on each device looks up the array's device address (a host-side query); make that
+ *     first call before starting any stream capture on that device.
+ *   - All calls on a device share the one array, and it keeps the previous call's contents: the call
+ *     clears or overwrites everything it later reads, so calls that run one after another (same
+ *     stream, or ordered by events) are independent, but two calls whose kernels may overlap on the
+ *     GPU (different streams without ordering) race on the array and give undefined results.
+ *   - moe_last_status() cannot be used (there is no workspace); these kernels contain no waits. */
+MOE_API int moe_route_static(const float *router_logits, int T, int E, int top_k, int32_t *topk_ids,
+                             float *topk_weights, int32_t *expert_offsets, int32_t *sorted_to_flat,
+                             int32_t *flat_to_sorted, void *stream);
 
 /* The whole layer (Sec. 4.5: routing, sort-scatter, gate+up with SiLU, down projection; then the
  * weighted combine).

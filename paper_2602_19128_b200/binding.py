@@ -18,7 +18,8 @@ MOE_FLAG_NONE = 0
 MOE_FLAG_VALIDATION_GEMM = 1
 MOE_FLAG_SINGLE_CTA_GEMM = 2
 
-EXPORTED = ["moe_workspace_bytes", "moe_workspace_layout", "moe_route_workspace_bytes", "moe_route", "moe_forward",
+EXPORTED = ["moe_workspace_bytes", "moe_workspace_layout", "moe_route_workspace_bytes", "moe_route", "moe_route_static",
+            "moe_forward",
             "moe_forward_ex", "moe_forward_staged", "moe_forward_host", "moe_last_status", "moe_forward_launch_count", "moe_status_string"]
 
 
@@ -54,6 +55,8 @@ def lib() -> ctypes.CDLL:
         L.moe_route_workspace_bytes.argtypes = [i] * 3
         L.moe_route.restype = i
         L.moe_route.argtypes = [vp, i, i, i, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.moe_route_static.restype = i
+        L.moe_route_static.argtypes = [vp, i, i, i, vp, vp, vp, vp, vp, vp]
         L.moe_forward.restype = i
         L.moe_forward.argtypes = [vp, vp, vp, vp, i, i, i, i, i, vp, vp, sz, vp]
         L.moe_forward_ex.restype = i
@@ -123,6 +126,18 @@ def moe_route(router_logits, top_k: int, topk_ids, topk_weights, expert_offsets,
                          _stream(stream))
     if check and st != MOE_OK:
         raise MoeError(st, "moe_route")
+    return st
+
+
+def moe_route_static(router_logits, top_k: int, topk_ids, topk_weights, expert_offsets, sorted_to_flat, flat_to_sorted,
+                     stream=None, check: bool = True) -> int:
+    """moe_route without a workspace: the scratch is a fixed array inside the library (no allocation
+    anywhere in the call).  Problems beyond its 512 KiB return MOE_ERR_STATIC_LIMIT (-9)."""
+    T, E = router_logits.shape
+    st = lib().moe_route_static(_ptr(router_logits), T, E, top_k, _ptr(topk_ids), _ptr(topk_weights),
+                                _ptr(expert_offsets), _ptr(sorted_to_flat), _ptr(flat_to_sorted), _stream(stream))
+    if check and st != MOE_OK:
+        raise MoeError(st, "moe_route_static")
     return st
 
 

@@ -238,6 +238,7 @@ const char *moe_status_string(int status) {
         case MOE_ERR_CUDA: return "a CUDA call failed";
         case MOE_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired";
         case MOE_ERR_ARCH: return "device is not compute capability 10.x";
+        case MOE_ERR_STATIC_LIMIT: return "problem exceeds the built-in scratch of moe_route_static (512 KiB)";
         default: return "unknown status";
     }
 }

@@ -16,6 +16,8 @@
 
 #include <limits.h>
 
+#include <mutex>
+
 namespace moe {
 namespace {
 
@@ -283,3 +285,63 @@ cudaError_t launch_combine(const __nv_bfloat16 *y, const float *topk_w, const in
 }
 
 }  // namespace moe
+
+// ---- moe_route_static: the router + sort-scatter for callers that cannot allocate --------------------
+//
+// The scratch (status word, per-chunk histograms, tile schedule) lives in a file-scope device array,
+// so the caller passes only inputs and outputs.  In host code the array's name is only a handle for
+// the runtime, not a device address: its address is looked up once per device with
+// cudaGetSymbolAddress (with that device current) and that pointer is what the kernels receive.
+namespace moe {
+namespace {
+
+constexpr size_t kStaticScratchBytes = 512 * 1024;
+static __device__ __align__(256) unsigned char g_route_static_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+void *g_static_scratch_ptr[kMaxDevices] = {nullptr};
+
+// Device address of the static scratch on the current device (looked up on the first call per device).
+cudaError_t static_scratch_address(void **out) {
+    int dev = 0;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) return err;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_scratch_ptr[dev]) {
+        void *ptr = nullptr;
+        err = cudaGetSymbolAddress(&ptr, g_route_static_scratch);
+        if (err != cudaSuccess) return err;
+        g_static_scratch_ptr[dev] = ptr;
+    }
+    *out = g_static_scratch_ptr[dev];
+    return cudaSuccess;
+}
+
+}  // namespace
+}  // namespace moe
+
+extern "C" int moe_route_static(const float *router_logits, int T, int E, int top_k, int32_t *topk_ids,
+                                float *topk_weights, int32_t *expert_offsets, int32_t *sorted_to_flat,
+                                int32_t *flat_to_sorted, void *stream) {
+    using namespace moe;
+    if (T < 0 || E <= 0 || top_k <= 0 || top_k > E) return MOE_ERR_SHAPE;
+    if (E > kMaxExperts || top_k > kMaxTopK || (long long)T * top_k >= (1LL << 27)) return MOE_ERR_UNSUPPORTED;
+    if (256 + route_scratch_bytes(T, E) > kStaticScratchBytes) return MOE_ERR_STATIC_LIMIT;
+    if (!expert_offsets) return MOE_ERR_NULL;
+    if (T > 0 && (!router_logits || !topk_ids || !topk_weights || !sorted_to_flat || !flat_to_sorted)) return MOE_ERR_NULL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (T == 0)
+        return cudaMemsetAsync(expert_offsets, 0, (size_t)(E + 1) * sizeof(int), s) == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+    void *scratch = nullptr;
+    if (static_scratch_address(&scratch) != cudaSuccess || !scratch) return MOE_ERR_CUDA;
+    char *base = static_cast<char *>(scratch);
+    // The array keeps the previous call's contents.  The status word is cleared by launch_route; the
+    // histogram and schedule regions are fully overwritten for this T and E before they are read.
+    RouteScratch rs = carve_route_scratch(base + 256, T, E);
+    const cudaError_t err = launch_route(router_logits, T, E, top_k, 256, topk_ids, topk_weights, expert_offsets,
+                                         sorted_to_flat, flat_to_sorted, rs, reinterpret_cast<int *>(base), s);
+    return err == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
+
