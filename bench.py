@@ -110,6 +110,20 @@ def dist_setup(n_gpus: int):
     return None, 0, 1, 0
 
 
+def max_over_ranks(dist, value: float, device) -> float:
+    """The slowest rank's time: the whole job is as slow as that rank."""
+    if dist is None:
+        return float(value)
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_tokens_per_s(world: int, tokens_per_rank_step: int, steps: int, total_ms: float) -> float:
+    """Whole-job throughput of `world` independent replicas (weak scaling): all tokens / slowest time."""
+    return world * tokens_per_rank_step * steps / (total_ms * 1e-3)
+
+
 def flush_l2(buf: torch.Tensor):
     buf.add_(1)
 
@@ -230,10 +244,7 @@ def run_ours(args):
         total_ms = stage_events[0][0].elapsed_time(stage_events[-1][-1])
     stage_ms = {name: statistics.fmean(ev[i].elapsed_time(ev[i + 1]) for ev in stage_events)
                 for i, name in enumerate(moe.STAGE_NAMES)}
-    if dist is not None:
-        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(dist, total_ms, dev)
     status = moe.moe_last_status(ws)
     if status != moe.MOE_OK:
         raise SystemExit(f"device status {status}: {moe.moe_status_string(status)}")
@@ -266,10 +277,7 @@ def run_ours(args):
         e1.synchronize()
         e2e_ms = e0.elapsed_time(e1)
     barrier()
-    if dist is not None:
-        t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = max_over_ranks(dist, e2e_ms, dev)
     same = bool(torch.equal(oh.view(torch.int16), out.cpu().view(torch.int16)))
 
     if rank != 0:
@@ -307,14 +315,14 @@ def run_ours(args):
     if world == 1 and not args.no_cpu_baseline:
         cpu_baseline = time_oracle(args.config, inp, budget_s=15.0)
 
-    line = dict(metric=METRIC, value=world * T * args.steps / (total_ms * 1e-3), unit=UNIT, n_gpus=world,
+    line = dict(metric=METRIC, value=aggregate_tokens_per_s(world, T, args.steps, total_ms), unit=UNIT, n_gpus=world,
                 steps=args.steps, warmup=max(args.warmup, 3), ms_per_step=total_ms / args.steps, higher_is_better=True,
                 scaling="weak", vs_baseline=None, dtype="bf16", data="synthetic",
                 config=dict(workload=args.config, T=T, H=H, I=I, E=E, top_k=k, parallelism=f"replicas x{world}",
                             l2="flushed between steps" if need_flush else "weights larger than L2, no flush",
                             seed=args.seed),
                 clocks=clocks,
-                e2e=dict(value=world * T * args.steps / (e2e_ms * 1e-3), unit=UNIT,
+                e2e=dict(value=aggregate_tokens_per_s(world, T, args.steps, e2e_ms), unit=UNIT,
                          h2d_bytes_per_step=T * H * 2 + T * E * 4, d2h_bytes_per_step=T * H * 2,
                          ms_per_step=e2e_ms / args.steps, matches_device_path=same),
                 gpu_launches=moe.moe_forward_launch_count(T) * args.steps,
