@@ -72,6 +72,9 @@ typedef enum {
 /* Keep the tcgen05 GEMMs on the one-CTA-per-tile kernel even where the CTA-pair kernel would be
  * chosen (token tiles of up to 128 / 256 rows).  For tests and A/B timing. */
 #define MOE_FLAG_SINGLE_CTA_GEMM 2u
+/* Let the CTA-pair kernel of the gate/up GEMM use two weight slabs per CTA (512 x N pair tiles) where
+ * the shape allows it.  Off by default (slower on the measured workloads); for tests and A/B timing. */
+#define MOE_FLAG_TWO_SLAB_GEMM 4u
 
 /* Byte offsets of the intermediates inside the workspace of moe_forward (so tests and tools can
  * read them after the stream has been synchronised).  Filled by moe_workspace_layout(). */

@@ -17,6 +17,7 @@ MOE_OK = 0
 MOE_FLAG_NONE = 0
 MOE_FLAG_VALIDATION_GEMM = 1
 MOE_FLAG_SINGLE_CTA_GEMM = 2
+MOE_FLAG_TWO_SLAB_GEMM = 4
 
 EXPORTED = ["moe_workspace_bytes", "moe_workspace_layout", "moe_route_workspace_bytes", "moe_route", "moe_route_static",
             "moe_forward",

@@ -52,7 +52,7 @@ int forward_impl(const void *x, const float *logits, const void *w13, const void
                  void *const *stage_events = nullptr) {
     if (T < 0 || H <= 0 || I <= 0 || E <= 0 || k <= 0 || k > E) return MOE_ERR_SHAPE;
     if (!envelope_ok(T, H, I, E, k)) return MOE_ERR_UNSUPPORTED;
-    if (flags & ~(MOE_FLAG_VALIDATION_GEMM | MOE_FLAG_SINGLE_CTA_GEMM)) return MOE_ERR_UNSUPPORTED;
+    if (flags & ~(MOE_FLAG_VALIDATION_GEMM | MOE_FLAG_SINGLE_CTA_GEMM | MOE_FLAG_TWO_SLAB_GEMM)) return MOE_ERR_UNSUPPORTED;
     if (T == 0) return MOE_OK;
     if (!x || !logits || !w13 || !w2 || !out || !workspace) return MOE_ERR_NULL;
     if (!aligned(x, 16) || !aligned(logits, 16) || !aligned(w13, 16) || !aligned(w2, 16) || !aligned(out, 16) ||
@@ -103,14 +103,26 @@ int forward_impl(const void *x, const float *logits, const void *w13, const void
         if (!mark(3)) return MOE_ERR_CUDA;
         if (launch_grouped_gemm_validation(g2, stream) != cudaSuccess) return MOE_ERR_CUDA;
     } else {
-        // CTA pairs where the token tiles are large enough for the halved token-tile traffic to matter
+        // CTA pairs where the token tiles are large enough for the halved token-tile traffic to matter.
+        // Two weight slabs per CTA (512 x N pair tiles) are opt-in: measured on the prefill-sized and
+        // skewed workloads they are 5 % resp. 25 % slower than one slab, because the accumulators then
+        // fill TMEM and the epilogue no longer overlaps the next tile's MMAs.
         const bool single = (flags & MOE_FLAG_SINGLE_CTA_GEMM) != 0;
-        int st = (!single && grouped_gemm_tc_pair_supported(g1)) ? launch_grouped_gemm_tc_pair(g1, stream)
-                                                                 : launch_grouped_gemm_tc(g1, stream);
+        const bool dense_tiles = (flags & MOE_FLAG_TWO_SLAB_GEMM) != 0;
+        auto run = [&](const GroupedGemmArgs &g, bool allow_two_slabs) {
+            int slabs = single ? 0 : grouped_gemm_tc_pair_slabs(g);
+            if (slabs == 2 && !(dense_tiles && allow_two_slabs)) slabs = grouped_gemm_tc_pair_slabs(g) >= 1 ? 1 : 0;
+            if (slabs == 2 || slabs == 1) {
+                // a one-slab launch needs its own divisibility (256 resp. 128 features)
+                const int st = launch_grouped_gemm_tc_pair(g, slabs, stream);
+                if (st != MOE_ERR_UNSUPPORTED) return st;
+            }
+            return launch_grouped_gemm_tc(g, stream);
+        };
+        int st = run(g1, true);
         if (st != MOE_OK) return st;
         if (!mark(3)) return MOE_ERR_CUDA;
-        st = (!single && grouped_gemm_tc_pair_supported(g2)) ? launch_grouped_gemm_tc_pair(g2, stream)
-                                                             : launch_grouped_gemm_tc(g2, stream);
+        st = run(g2, false);
         if (st != MOE_OK) return st;
     }
     if (!mark(4)) return MOE_ERR_CUDA;

@@ -98,27 +98,25 @@ grouped_gemm_tc_kernel(const __grid_constant__ TensorMaps maps, const KernelPara
     const int total_tiles = p.tile_prefix[p.E] * p.n_feature_tiles;
 
     if (warp == 0) {
-        // ---------------- TMA producer ----------------
-        if (lane == 0) {
-            int stage = 0;
-            uint32_t phase = 0;
-            bool ok = true;
-            for (int round = 0; ok; ++round) {
-                const int tile = tile_of_round(round, blockIdx.x, gridDim.x);
-                if (tile >= total_tiles) break;
-                const Tile t = decode_tile(tile, p);
-                const int n_mma = (t.n_valid + 15) & ~15;
-                const int w_row = t.e * p.w_rows + t.f * kTileM;  // down projection: 128 rows of w2[e]
-                const uint32_t tx_bytes = kSlotABytes + n_mma * kRowBytes;
-                for (int kb = 0; kb < p.n_k_blocks; ++kb) {
-                    ok = mbar_wait(bar_empty + stage * 8, phase ^ 1u, abort_flag, p.status, kSiteProducerEmpty + kSiteOffset);
-                    if (!ok) break;
+        // ---------------- TMA producer: the warp walks the ring, one elected lane issues ----------------
+        int stage = 0;
+        uint32_t phase = 0;
+        bool ok = true;
+        for (int round = 0; ok; ++round) {
+            const int tile = tile_of_round(round, blockIdx.x, gridDim.x);
+            if (tile >= total_tiles) break;
+            const Tile t = decode_tile(tile, p);
+            const int n_mma = (t.n_valid + 15) & ~15;
+            const int w_row = t.e * p.w_rows + t.f * kTileM;  // down projection: 128 rows of w2[e]
+            const uint32_t tx_bytes = kSlotABytes + n_mma * kRowBytes;
+            for (int kb = 0; kb < p.n_k_blocks; ++kb) {
+                ok = mbar_wait_warp(bar_empty + stage * 8, phase ^ 1u, abort_flag, p.status, kSiteProducerEmpty + kSiteOffset);
+                if (!ok) break;
+                if (elect_one()) {
                     const uint32_t full = bar_full + stage * 8;
-#ifdef MOE_ABLATE_NO_TMA  // experiment builds only: time the MMA side alone
+#if defined(MOE_ABLATE_NO_TMA)  // experiment builds only: time the MMA side alone
                     mbar_arrive(full);
-                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
-                    continue;
-#endif
+#else
 #ifdef MOE_ABLATE_NO_B
                     mbar_expect_tx(full, kSlotABytes);
 #else
@@ -132,48 +130,49 @@ grouped_gemm_tc_kernel(const __grid_constant__ TensorMaps maps, const KernelPara
                     else
                         tma_load_2d(sa, &maps.w, k0, w_row, full);
 #ifndef MOE_ABLATE_NO_B
-                    tma_load_2d(sb, act_map(maps, n_mma), k0, t.row0, full);
+                    tma_load_2d(sb, act_map<16>(maps, n_mma), k0, t.row0, full);
 #endif
-                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+#endif
                 }
+                __syncwarp();
+                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
             }
         }
-        __syncwarp();
     } else if (warp == 1) {
-        // ---------------- MMA issuer ----------------
-        if (lane == 0) {
-            int stage = 0, acc = 0;
-            uint32_t phase = 0, acc_phase = 0;
-            bool ok = true;
-            for (int round = 0; ok; ++round) {
-                const int tile = tile_of_round(round, blockIdx.x, gridDim.x);
-                if (tile >= total_tiles) break;
-                const Tile t = decode_tile(tile, p);
-                const uint32_t idesc = instr_desc_bf16(kTileM, (t.n_valid + 15) & ~15);
-                ok = mbar_wait(bar_acc_empty + acc * 8, acc_phase ^ 1u, abort_flag, p.status, kSiteMmaTmemEmpty + kSiteOffset);
+        // ---------------- MMA issuer: same structure; MMAs and their commits come from one lane ----------------
+        int stage = 0, acc = 0;
+        uint32_t phase = 0, acc_phase = 0;
+        bool ok = true;
+        for (int round = 0; ok; ++round) {
+            const int tile = tile_of_round(round, blockIdx.x, gridDim.x);
+            if (tile >= total_tiles) break;
+            const Tile t = decode_tile(tile, p);
+            const uint32_t idesc = instr_desc_bf16(kTileM, (t.n_valid + 15) & ~15);
+            ok = mbar_wait_warp(bar_acc_empty + acc * 8, acc_phase ^ 1u, abort_flag, p.status, kSiteMmaTmemEmpty + kSiteOffset);
+            if (!ok) break;
+            tcgen05_fence_after();
+            const uint32_t d_tmem = tmem_base + acc * NT_MAX;
+            for (int kb = 0; kb < p.n_k_blocks; ++kb) {
+                ok = mbar_wait_warp(bar_full + stage * 8, phase, abort_flag, p.status, kSiteMmaFull + kSiteOffset);
                 if (!ok) break;
                 tcgen05_fence_after();
-                const uint32_t d_tmem = tmem_base + acc * NT_MAX;
-                for (int kb = 0; kb < p.n_k_blocks; ++kb) {
-                    ok = mbar_wait(bar_full + stage * 8, phase, abort_flag, p.status, kSiteMmaFull + kSiteOffset);
-                    if (!ok) break;
-                    tcgen05_fence_after();
+                if (elect_one()) {
                     const uint64_t a_desc = smem_desc_k_major_sw128(base + L::kA + stage * kSlotABytes);
                     const uint64_t b_desc = smem_desc_k_major_sw128(base + L::kB + stage * L::kSlotBBytes);
-#pragma unroll
 #ifndef MOE_ABLATE_NO_MMA  // (experiment builds may drop the MMAs to time the load side alone)
+#pragma unroll
                     for (int kk = 0; kk < kBlockK / 16; ++kk)  // 16 K-elements = 32 bytes = 2 descriptor units
                         umma_bf16(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (kb | kk) != 0);
 #endif
                     umma_commit(bar_empty + stage * 8);
-                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                    if (kb == p.n_k_blocks - 1) umma_commit(bar_acc_full + acc * 8);
                 }
-                if (!ok) break;
-                umma_commit(bar_acc_full + acc * 8);
-                if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+                __syncwarp();
+                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
             }
+            if (!ok) break;
+            if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
         }
-        __syncwarp();
     } else {
         // ---------------- epilogue: TMEM -> registers -> global ----------------
         const int q = warp & 3;  // a warp may only read TMEM lanes 32*(warp%4) .. +31
@@ -269,7 +268,7 @@ int launch_grouped_gemm_tc(const GroupedGemmArgs &a, cudaStream_t stream) {
     TensorMaps maps;
     const bool ok_w = a.swiglu ? encode_weight_map_gate_up(&maps.w, a.w, a.E, a.n_out, a.K)
                                : encode_weight_map_2d(&maps.w, a.w, (uint64_t)a.E * a.w_rows, a.K);
-    if (!ok_w || !encode_act_maps(maps.act, a.act, a.A, a.K)) return MOE_ERR_CUDA;
+    if (!ok_w || !encode_act_maps(maps.act, a.act, a.A, a.K, 16)) return MOE_ERR_CUDA;
 
     KernelParams p;
     p.out = a.out;

@@ -1,4 +1,4 @@
-// Grouped expert GEMMs on CTA pairs: tcgen05.mma.cta_group::2, a 256 x N tile per pair.
+// Grouped expert GEMMs on CTA pairs: tcgen05.mma.cta_group::2, a 256 x N or 512 x N tile per pair.
 //
 // Same role split, ring and tile schedule as the one-CTA kernel (moe_gemm_tc.cu; paper Sec. 4.5
 // "Expert FFN computation" for what is computed), but two CTAs of a cluster work on one tile:
@@ -17,6 +17,13 @@
 // Before leaving, each producer waits until every ring slot has been handed back and the leader
 // waits for both accumulators to be released, so no arrival can reach a CTA that has exited; a
 // cluster barrier then precedes the TMEM release.  Every wait is bounded as in the one-CTA kernel.
+//
+// SLABS = 2 gives each CTA two 128-row weight slabs per ring slot that share one token tile (two MMAs
+// per K step, two accumulators): (1/N + 1/512) bytes per flop through the copy engine, which keeps
+// the tensor pipe busy for token tiles well below 256 rows.  The two accumulators fill TMEM
+// (2 x 256 columns), so the epilogue is not overlapped with the next tile's MMAs; measured slower than
+// one slab on every benchmark workload, it is opt-in (MOE_FLAG_TWO_SLAB_GEMM) and kept for shapes
+// with much longer K.
 #include "moe_tc_common.cuh"
 
 namespace moe {
@@ -86,11 +93,12 @@ __device__ __forceinline__ bool pair_wait(uint32_t bar, uint32_t parity, volatil
     return ok;
 }
 
-template <int NT_MAX, int STAGES>
+template <int NT_MAX, int STAGES, int SLABS>
 struct PairSmem {
+    static constexpr int kSlotABytesAll = SLABS * kSlotABytes;
     static constexpr int kSlotBBytes = (NT_MAX / 2) * kRowBytes;
     static constexpr int kA = 0;
-    static constexpr int kB = STAGES * kSlotABytes;
+    static constexpr int kB = STAGES * kSlotABytesAll;
     static constexpr int kBars = kB + STAGES * kSlotBBytes;  // full[S], empty[S], acc_full[2], acc_empty[2]
     static constexpr int kTmemSlot = kBars + (2 * STAGES + 4) * 8;
     static constexpr int kAbort = kTmemSlot + 4;
@@ -98,12 +106,48 @@ struct PairSmem {
     static constexpr int kDynamicBytes = kBytes + 1024;
 };
 
-template <int NT_MAX, int STAGES, bool SWIGLU>
+// Drain one accumulator (this warp's 32 TMEM lanes x n_mma columns) to global memory.
+//   SWIGLU: lanes 0..15 hold gate, lanes 16..31 up of the same 16 features; dst points at this lane's
+//           feature in row 0 of the tile.  Plain: one output feature per lane.
+template <bool SWIGLU>
+__device__ __forceinline__ void drain_accumulator(uint32_t taddr, int n_mma, int n_valid, __nv_bfloat16 *dst,
+                                                  size_t row_stride, int lane) {
+    if (SWIGLU) {
+        const int hi = lane >> 4;
+        for (int c0 = 0; c0 < n_mma; c0 += 16) {
+            float v[16];
+            tmem_load_16(taddr + c0, v);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const float other = __shfl_xor_sync(0xffffffffu, hi ? v[i] : v[8 + i], 16);
+                const float g = hi ? other : v[i];
+                const float u = hi ? v[8 + i] : other;
+                const int col = c0 + hi * 8 + i;
+                if (col < n_valid) dst[(size_t)col * row_stride] = __float2bfloat16_rn(swiglu(g, u));
+            }
+        }
+    } else {
+        for (int c0 = 0; c0 < n_mma; c0 += 16) {
+            float v[16];
+            tmem_load_16(taddr + c0, v);
+#pragma unroll
+            for (int i = 0; i < 16; ++i)
+                if (c0 + i < n_valid) dst[(size_t)(c0 + i) * row_stride] = __float2bfloat16_rn(v[i]);
+        }
+    }
+}
+
+template <int NT_MAX, int STAGES, int SLABS, bool SWIGLU>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
 grouped_gemm_tc_pair_kernel(const __grid_constant__ TensorMaps maps, const KernelParams p) {
-    using L = PairSmem<NT_MAX, STAGES>;
-    constexpr int kTmemCols = 2 * NT_MAX;
-    constexpr int kSiteOffset = SWIGLU ? 0 : 4;  // the down GEMM reports sites 5..8
+    using L = PairSmem<NT_MAX, STAGES, SLABS>;
+    constexpr int kAccBufs = SLABS == 1 ? 2 : 1;          // accumulator sets in TMEM
+    constexpr int kTmemCols = SLABS * kAccBufs * NT_MAX;  // = 2 * NT_MAX either way
+    constexpr int kSiteOffset = SWIGLU ? 0 : 4;           // the down GEMM reports sites 5..8
+    // weight rows (plain) resp. h features (SwiGLU) covered by one pair tile, one slab of it, one CTA of a slab
+    constexpr int kFeatPerCta = SWIGLU ? kTileM / 2 : kTileM;
+    constexpr int kFeatPerSlab = 2 * kFeatPerCta;
+    constexpr int kFeatPerTile = SLABS * kFeatPerSlab;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *base_ptr = smem_raw + (base - smem_u32(smem_raw));
@@ -143,9 +187,9 @@ grouped_gemm_tc_pair_kernel(const __grid_constant__ TensorMaps maps, const Kerne
     const int n_pairs = gridDim.x >> 1, pair = blockIdx.x >> 1;
 
     // ---------------- TMA producers (both CTAs) ----------------
-    // The weight slab and the token rows of a slot are issued by two different warps: a copy
+    // The weight slabs and the token rows of a slot are issued by two different warps: a copy
     // instruction occupies its issuing thread for a while, and two issuers keep the ring ahead.
-    auto producer_loop = [&](const bool load_w, const bool load_act) {
+    auto producer_loop = [&](const bool load_w, const bool load_act) {  // run by a whole warp
         int stage = 0;
         uint32_t phase = 0;
         bool ok = true;
@@ -153,94 +197,109 @@ grouped_gemm_tc_pair_kernel(const __grid_constant__ TensorMaps maps, const Kerne
             const int tile = tile_of_round(round, pair, n_pairs);
             if (tile >= total_tiles) break;
             const Tile t = decode_tile(tile, p);
-            const int n_mma = (t.n_valid + 31) & ~31, half = n_mma >> 1;
-            const int w_row = t.e * p.w_rows + t.f * (2 * kTileM) + (int)rank * kTileM;  // down projection
+            const int n_mma = (t.n_valid + 15) & ~15, half = n_mma >> 1;  // each CTA stages half: a multiple of 8 rows
+            const int feat0 = t.f * kFeatPerTile + (int)rank * kFeatPerCta;  // this CTA's part of slab 0
             for (int kb = 0; kb < p.n_k_blocks; ++kb) {
-                ok = pair_wait(bar_empty + stage * 8, phase ^ 1u, abort_flag, peer_abort, p.status, kSiteProducerEmpty + kSiteOffset);
+                ok = __all_sync(0xffffffffu, pair_wait(bar_empty + stage * 8, phase ^ 1u, abort_flag, peer_abort, p.status,
+                                                       kSiteProducerEmpty + kSiteOffset));
                 if (!ok) break;
-                const uint32_t full = map_to_cta(bar_full + stage * 8, 0);
-                const int k0 = kb * kBlockK;
-                if (load_w) {
-#ifdef MOE_ABLATE_NO_TMA  // experiment builds only: time the MMA side alone
-                    if (rank == 0) mbar_arrive(bar_full + stage * 8);
-                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
-                    continue;
-#endif
-#ifdef MOE_ABLATE_NO_B
-                    if (rank == 0) mbar_expect_tx(bar_full + stage * 8, 2 * kSlotABytes);
+                if (elect_one()) {
+                    const uint32_t full = map_to_cta(bar_full + stage * 8, 0);
+                    const int k0 = kb * kBlockK;
+                    if (load_w) {
+#if defined(MOE_ABLATE_NO_TMA)  // experiment builds only: time the MMA side alone
+                        if (rank == 0) mbar_arrive(bar_full + stage * 8);
 #else
-                    if (rank == 0) mbar_expect_tx(bar_full + stage * 8, 2 * kSlotABytes + n_mma * kRowBytes);
+#ifdef MOE_ABLATE_NO_B
+                        if (rank == 0) mbar_expect_tx(bar_full + stage * 8, 2 * L::kSlotABytesAll);
+#else
+                        if (rank == 0) mbar_expect_tx(bar_full + stage * 8, 2 * L::kSlotABytesAll + n_mma * kRowBytes);
 #endif
-                    const uint32_t sa = base + L::kA + stage * kSlotABytes;
-                    if (SWIGLU)  // this CTA's 64 features = groups 8f + 4*rank .. +3 of 16
-                        tma_load_5d_pair(sa, &maps.w, k0, 0, 0, t.f * 8 + (int)rank * 4, t.e, full);
-                    else
-                        tma_load_2d_pair(sa, &maps.w, k0, w_row, full);
-                }
+#pragma unroll
+                        for (int s = 0; s < SLABS; ++s) {
+                            const uint32_t sa = base + L::kA + stage * L::kSlotABytesAll + s * kSlotABytes;
+                            const int feat = feat0 + s * kFeatPerSlab;
+                            if (SWIGLU)  // 64 features = 4 groups of 16, gate and up rows interleaved per group
+                                tma_load_5d_pair(sa, &maps.w, k0, 0, 0, feat >> 4, t.e, full);
+                            else
+                                tma_load_2d_pair(sa, &maps.w, k0, t.e * p.w_rows + feat, full);
+                        }
+#endif
+                    }
 #if !defined(MOE_ABLATE_NO_B) && !defined(MOE_ABLATE_NO_TMA)
-                if (load_act) {
-                    const uint32_t sb = base + L::kB + stage * L::kSlotBBytes;
-                    tma_load_2d_pair(sb, act_map(maps, half), k0, t.row0 + (int)rank * half, full);
-                }
+                    if (load_act) {
+                        const uint32_t sb = base + L::kB + stage * L::kSlotBBytes;
+                        tma_load_2d_pair(sb, act_map<8>(maps, half), k0, t.row0 + (int)rank * half, full);
+                    }
 #endif
+                }
+                __syncwarp();
                 if (++stage == STAGES) { stage = 0; phase ^= 1u; }
             }
         }
         // wait until every slot has been handed back: no commit may arrive here after exit
         for (int s = 0; ok && s < STAGES; ++s) {
-            ok = pair_wait(bar_empty + stage * 8, phase ^ 1u, abort_flag, peer_abort, p.status, kSiteProducerEmpty + kSiteOffset);
+            ok = __all_sync(0xffffffffu, pair_wait(bar_empty + stage * 8, phase ^ 1u, abort_flag, peer_abort, p.status,
+                                                   kSiteProducerEmpty + kSiteOffset));
             if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
     };
     if (warp == 0) {
-        if (lane == 0) producer_loop(true, false);
-        __syncwarp();
+        producer_loop(true, false);
     } else if (warp == kPairThreads / 32 - 1) {
-        if (lane == 0) producer_loop(false, true);
-        __syncwarp();
+        producer_loop(false, true);
     } else if (warp == 1) {
-        // ---------------- MMA issuer (leader CTA only) ----------------
-        if (lane == 0 && rank == 0) {
+        // ---------------- MMA issuer (leader CTA only): the warp walks the ring, one elected lane issues ----------------
+        if (rank == 0) {
             int stage = 0, acc = 0;
             uint32_t phase = 0, acc_phase = 0;
             bool ok = true;
             for (int round = 0; ok; ++round) {
-            const int tile = tile_of_round(round, pair, n_pairs);
-            if (tile >= total_tiles) break;
+                const int tile = tile_of_round(round, pair, n_pairs);
+                if (tile >= total_tiles) break;
                 const Tile t = decode_tile(tile, p);
-                const uint32_t idesc = instr_desc_bf16(2 * kTileM, (t.n_valid + 31) & ~31);
-                ok = pair_wait(bar_acc_empty + acc * 8, acc_phase ^ 1u, abort_flag, peer_abort, p.status, kSiteMmaTmemEmpty + kSiteOffset);
+                const uint32_t idesc = instr_desc_bf16(2 * kTileM, (t.n_valid + 15) & ~15);
+                ok = __all_sync(0xffffffffu, pair_wait(bar_acc_empty + acc * 8, acc_phase ^ 1u, abort_flag, peer_abort,
+                                                       p.status, kSiteMmaTmemEmpty + kSiteOffset));
                 if (!ok) break;
                 tcgen05_fence_after();
-                const uint32_t d_tmem = tmem_base + acc * NT_MAX;
+                const uint32_t d_tmem = tmem_base + acc * SLABS * NT_MAX;
                 for (int kb = 0; kb < p.n_k_blocks; ++kb) {
-                    ok = pair_wait(bar_full + stage * 8, phase, abort_flag, peer_abort, p.status, kSiteMmaFull + kSiteOffset);
+                    ok = __all_sync(0xffffffffu, pair_wait(bar_full + stage * 8, phase, abort_flag, peer_abort, p.status,
+                                                           kSiteMmaFull + kSiteOffset));
                     if (!ok) break;
                     tcgen05_fence_after();
-                    const uint64_t a_desc = smem_desc_k_major_sw128(base + L::kA + stage * kSlotABytes);
-                    const uint64_t b_desc = smem_desc_k_major_sw128(base + L::kB + stage * L::kSlotBBytes);
+                    if (elect_one()) {
+                        const uint64_t b_desc = smem_desc_k_major_sw128(base + L::kB + stage * L::kSlotBBytes);
 #ifndef MOE_ABLATE_NO_MMA  // (experiment builds may drop the MMAs to time the load side alone)
 #pragma unroll
-                    for (int kk = 0; kk < kBlockK / 16; ++kk)
-                        umma_bf16_pair(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (kb | kk) != 0);
+                        for (int s = 0; s < SLABS; ++s) {
+                            const uint64_t a_desc =
+                                smem_desc_k_major_sw128(base + L::kA + stage * L::kSlotABytesAll + s * kSlotABytes);
+#pragma unroll
+                            for (int kk = 0; kk < kBlockK / 16; ++kk)  // 16 K-elements = 32 bytes = 2 descriptor units
+                                umma_bf16_pair(d_tmem + s * NT_MAX, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (kb | kk) != 0);
+                        }
 #endif
-                    umma_commit_pair(bar_empty + stage * 8);
+                        umma_commit_pair(bar_empty + stage * 8);
+                        if (kb == p.n_k_blocks - 1) umma_commit_pair(bar_acc_full + acc * 8);
+                    }
+                    __syncwarp();
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
                 if (!ok) break;
-                umma_commit_pair(bar_acc_full + acc * 8);
-                if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+                if (++acc == kAccBufs) { acc = 0; acc_phase ^= 1u; }
             }
-            // wait until both accumulators have been released by both CTAs' epilogues
-            for (int a = 0; ok && a < 2; ++a) {
-                ok = pair_wait(bar_acc_empty + acc * 8, acc_phase ^ 1u, abort_flag, peer_abort, p.status, kSiteMmaTmemEmpty + kSiteOffset);
-                if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+            // wait until every accumulator set has been released by both CTAs' epilogues
+            for (int a = 0; ok && a < kAccBufs; ++a) {
+                ok = __all_sync(0xffffffffu, pair_wait(bar_acc_empty + acc * 8, acc_phase ^ 1u, abort_flag, peer_abort,
+                                                       p.status, kSiteMmaTmemEmpty + kSiteOffset));
+                if (++acc == kAccBufs) { acc = 0; acc_phase ^= 1u; }
             }
         }
-        __syncwarp();
     } else {
-        // ---------------- epilogue (both CTAs): own 128 weight rows x all N tokens ----------------
-        const int q = warp & 3;
+        // ---------------- epilogue (both CTAs): own 128 weight rows per slab x all N tokens ----------------
+        const int q = warp & 3;  // a warp may only read TMEM lanes 32*(warp%4) .. +31
         int acc = 0;
         uint32_t acc_phase = 0;
         bool ok = true;
@@ -248,41 +307,23 @@ grouped_gemm_tc_pair_kernel(const __grid_constant__ TensorMaps maps, const Kerne
             const int tile = tile_of_round(round, pair, n_pairs);
             if (tile >= total_tiles) break;
             const Tile t = decode_tile(tile, p);
-            const int n_mma = (t.n_valid + 31) & ~31;
+            const int n_mma = (t.n_valid + 15) & ~15;
             ok = pair_wait(bar_acc_full + acc * 8, acc_phase, abort_flag, peer_abort, p.status, kSiteEpilogueTmemFull + kSiteOffset);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tcgen05_fence_after();
-            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + acc * NT_MAX;
-            if (SWIGLU) {
-                const int hi = lane >> 4;
-                __nv_bfloat16 *dst = p.out + (size_t)t.row0 * p.n_out + t.f * kTileM + (int)rank * (kTileM / 2) + q * 16 + (lane & 15);
-                for (int c0 = 0; c0 < n_mma; c0 += 16) {
-                    float v[16];
-                    tmem_load_16(taddr + c0, v);
+            const int lane_feat = SWIGLU ? q * 16 + (lane & 15) : q * 32 + lane;
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const float other = __shfl_xor_sync(0xffffffffu, hi ? v[i] : v[8 + i], 16);
-                        const float g = hi ? other : v[i];
-                        const float u = hi ? v[8 + i] : other;
-                        const int col = c0 + hi * 8 + i;
-                        if (col < t.n_valid) dst[(size_t)col * p.n_out] = __float2bfloat16_rn(swiglu(g, u));
-                    }
-                }
-            } else {
-                __nv_bfloat16 *dst = p.out + (size_t)t.row0 * p.n_out + t.f * (2 * kTileM) + (int)rank * kTileM + q * 32 + lane;
-                for (int c0 = 0; c0 < n_mma; c0 += 16) {
-                    float v[16];
-                    tmem_load_16(taddr + c0, v);
-#pragma unroll
-                    for (int i = 0; i < 16; ++i)
-                        if (c0 + i < t.n_valid) dst[(size_t)(c0 + i) * p.n_out] = __float2bfloat16_rn(v[i]);
-                }
+            for (int s = 0; s < SLABS; ++s) {
+                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (acc * SLABS + s) * NT_MAX;
+                __nv_bfloat16 *dst = p.out + (size_t)t.row0 * p.n_out + t.f * kFeatPerTile + s * kFeatPerSlab +
+                                     (int)rank * kFeatPerCta + lane_feat;
+                drain_accumulator<SWIGLU>(taddr, n_mma, t.n_valid, dst, (size_t)p.n_out, lane);
             }
             tcgen05_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(map_to_cta(bar_acc_empty + acc * 8, 0));
-            if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+            if (++acc == kAccBufs) { acc = 0; acc_phase ^= 1u; }
         }
     }
 
@@ -299,30 +340,35 @@ grouped_gemm_tc_pair_kernel(const __grid_constant__ TensorMaps maps, const Kerne
     }
 }
 
-template <int NT_MAX, int STAGES, bool SWIGLU>
+template <int NT_MAX, int STAGES, int SLABS, bool SWIGLU>
 int launch_pair_instance(const TensorMaps &maps, const KernelParams &p, int grid, cudaStream_t stream) {
-    using L = PairSmem<NT_MAX, STAGES>;
+    using L = PairSmem<NT_MAX, STAGES, SLABS>;
     static_assert(L::kDynamicBytes <= 232448, "ring does not fit in shared memory");
-    auto kernel = grouped_gemm_tc_pair_kernel<NT_MAX, STAGES, SWIGLU>;
+    auto kernel = grouped_gemm_tc_pair_kernel<NT_MAX, STAGES, SLABS, SWIGLU>;
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) != cudaSuccess)
         return MOE_ERR_CUDA;
     kernel<<<grid, kPairThreads, L::kDynamicBytes, stream>>>(maps, p);
     return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
 
+int features_per_pair_tile(const GroupedGemmArgs &a, int slabs) { return slabs * (a.swiglu ? kTileM : 2 * kTileM); }
+
 }  // namespace
 
-bool grouped_gemm_tc_pair_supported(const GroupedGemmArgs &a) {
-    return (a.nt_max == 128 || a.nt_max == 256) && a.K % kBlockK == 0 && a.A > 0 &&
-           a.n_out % (a.swiglu ? kTileM : 2 * kTileM) == 0;
+// Largest number of weight slabs per CTA (2, 1) the pair kernel supports for this GEMM, 0 if none.
+int grouped_gemm_tc_pair_slabs(const GroupedGemmArgs &a) {
+    if (!(a.nt_max == 128 || a.nt_max == 256) || a.K % kBlockK != 0 || a.A <= 0) return 0;
+    if (a.nt_max == 256 && a.n_out % features_per_pair_tile(a, 2) == 0) return 2;
+    return a.n_out % features_per_pair_tile(a, 1) == 0 ? 1 : 0;
 }
 
-int launch_grouped_gemm_tc_pair(const GroupedGemmArgs &a, cudaStream_t stream) {
-    if (!grouped_gemm_tc_pair_supported(a)) return MOE_ERR_UNSUPPORTED;
+int launch_grouped_gemm_tc_pair(const GroupedGemmArgs &a, int slabs, cudaStream_t stream) {
+    const int max_slabs = grouped_gemm_tc_pair_slabs(a);
+    if (slabs < 1 || slabs > max_slabs) return MOE_ERR_UNSUPPORTED;
     TensorMaps maps;
     const bool ok_w = a.swiglu ? encode_weight_map_gate_up(&maps.w, a.w, a.E, a.n_out, a.K)
                                : encode_weight_map_2d(&maps.w, a.w, (uint64_t)a.E * a.w_rows, a.K);
-    if (!ok_w || !encode_act_maps(maps.act, a.act, a.A, a.K)) return MOE_ERR_CUDA;
+    if (!ok_w || !encode_act_maps(maps.act, a.act, a.A, a.K, 8)) return MOE_ERR_CUDA;
 
     KernelParams p;
     p.out = a.out;
@@ -335,18 +381,21 @@ int launch_grouped_gemm_tc_pair(const GroupedGemmArgs &a, cudaStream_t stream) {
     p.n_k_blocks = a.K / kBlockK;
     p.n_out = a.n_out;
     p.w_rows = a.w_rows;
-    p.n_feature_tiles = a.n_out / (a.swiglu ? kTileM : 2 * kTileM);
+    p.n_feature_tiles = a.n_out / features_per_pair_tile(a, slabs);
 
     const long long max_token_tiles = (long long)(a.A < a.E ? a.A : a.E) + a.A / a.nt_max;
     const long long max_tiles = max_token_tiles * p.n_feature_tiles;
     const int pairs_on_device = sm_count() / 2;
     const int n_pairs = (int)(max_tiles < pairs_on_device ? max_tiles : pairs_on_device);
     const int grid = 2 * (n_pairs > 0 ? n_pairs : 1);
+    if (slabs == 2)
+        return a.swiglu ? launch_pair_instance<256, 4, 2, true>(maps, p, grid, stream)
+                        : launch_pair_instance<256, 4, 2, false>(maps, p, grid, stream);
     if (a.nt_max == 256)
-        return a.swiglu ? launch_pair_instance<256, 7, true>(maps, p, grid, stream)
-                        : launch_pair_instance<256, 7, false>(maps, p, grid, stream);
-    return a.swiglu ? launch_pair_instance<128, 9, true>(maps, p, grid, stream)
-                    : launch_pair_instance<128, 9, false>(maps, p, grid, stream);
+        return a.swiglu ? launch_pair_instance<256, 7, 1, true>(maps, p, grid, stream)
+                        : launch_pair_instance<256, 7, 1, false>(maps, p, grid, stream);
+    return a.swiglu ? launch_pair_instance<128, 9, 1, true>(maps, p, grid, stream)
+                    : launch_pair_instance<128, 9, 1, false>(maps, p, grid, stream);
 }
 
 }  // namespace moe

@@ -24,7 +24,7 @@ static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; 
 
 // Scratch of the router / sort-scatter, all int32, carved out of the caller's workspace.
 struct RouteScratch {
-    int *chunk_counts;  // [n_chunks, E] per-chunk expert histogram, then per-chunk start positions
+    int *chunk_counts;  // [n_chunks, E] per-chunk expert histogram, then rows of earlier chunks per expert
     int *tile_prefix;   // [E+1] exclusive prefix sum of token tiles over experts in schedule order
     int *tile_order;    // [E]   expert at each schedule position: most rows first, ties to the lower index
     int *tile_rows;     // [E]   rows per token tile of this expert (multiple of 16; 0 if empty)
@@ -82,10 +82,12 @@ struct GroupedGemmArgs {
 };
 int launch_grouped_gemm_tc(const GroupedGemmArgs &args, cudaStream_t stream);  // returns a moe_status_t
 
-// The same GEMM on CTA pairs (cta_group::2, 256 x N tiles); only for token-tile bounds of 128 / 256
-// and feature counts the 256-row pair tile divides.
-bool grouped_gemm_tc_pair_supported(const GroupedGemmArgs &args);
-int launch_grouped_gemm_tc_pair(const GroupedGemmArgs &args, cudaStream_t stream);
+// The same GEMM on CTA pairs (cta_group::2): 256 x N tiles (one weight slab per CTA) or 512 x N tiles
+// (two slabs per CTA sharing one token tile).  grouped_gemm_tc_pair_slabs gives the largest slab count
+// usable for this GEMM: 2, 1, or 0 when the pair kernel does not apply (token-tile bound below 128, or a
+// feature count the pair tile does not divide).
+int grouped_gemm_tc_pair_slabs(const GroupedGemmArgs &args);
+int launch_grouped_gemm_tc_pair(const GroupedGemmArgs &args, int slabs, cudaStream_t stream);
 
 // Same contract on plain CUDA cores (validation only).
 cudaError_t launch_grouped_gemm_validation(const GroupedGemmArgs &args, cudaStream_t stream);

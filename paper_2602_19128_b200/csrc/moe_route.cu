@@ -134,10 +134,17 @@ route_scan_kernel(int *__restrict__ chunk_counts, int n_chunks, int E, int nt_ma
     const int e = threadIdx.x;
     int count = 0;
     if (e < E) {
-        for (int b = 0; b < n_chunks; ++b) {
-            const int c = chunk_counts[(size_t)b * E + e];
-            chunk_counts[(size_t)b * E + e] = count;
-            count += c;
+        // running sum over chunks, 16 independent loads in flight at a time (the loop is latency-bound)
+        constexpr int kBatch = 16;
+        for (int b0 = 0; b0 < n_chunks; b0 += kBatch) {
+            int c[kBatch];
+#pragma unroll
+            for (int i = 0; i < kBatch; ++i) c[i] = b0 + i < n_chunks ? chunk_counts[(size_t)(b0 + i) * E + e] : 0;
+#pragma unroll
+            for (int i = 0; i < kBatch; ++i) {
+                if (b0 + i < n_chunks) chunk_counts[(size_t)(b0 + i) * E + e] = count;
+                count += c[i];
+            }
         }
     }
     counts[e] = e < E ? count : -1;
@@ -164,7 +171,6 @@ route_scan_kernel(int *__restrict__ chunk_counts, int n_chunks, int E, int nt_ma
         expert_offsets[e] = row_start;
         tile_prefix[e] = tile_start;  // indexed by schedule position
         tile_rows[e] = rows;
-        for (int b = 0; b < n_chunks; ++b) chunk_counts[(size_t)b * E + e] += row_start;
     }
     if (e == 0) {
         expert_offsets[E] = total_rows;
@@ -173,11 +179,13 @@ route_scan_kernel(int *__restrict__ chunk_counts, int n_chunks, int E, int nt_ma
 }
 
 __global__ void __launch_bounds__(32)
-route_scatter_kernel(const int *__restrict__ topk_ids, const int *__restrict__ chunk_starts, int A, int E, int k,
-                     int *__restrict__ sorted_to_flat, int *__restrict__ flat_to_sorted) {
+route_scatter_kernel(const int *__restrict__ topk_ids, const int *__restrict__ chunk_starts,
+                     const int *__restrict__ expert_offsets, int A, int E, int k, int *__restrict__ sorted_to_flat,
+                     int *__restrict__ flat_to_sorted) {
     __shared__ int next[kMaxExperts];
     const int lane = threadIdx.x;
-    for (int e = lane; e < E; e += 32) next[e] = chunk_starts[(size_t)blockIdx.x * E + e];
+    // first position of this chunk's assignments to expert e = segment start + rows of earlier chunks
+    for (int e = lane; e < E; e += 32) next[e] = expert_offsets[e] + chunk_starts[(size_t)blockIdx.x * E + e];
     __syncwarp();
     const int a0 = blockIdx.x * kRouteTokensPerBlock * k;
     const int a1 = min(A, a0 + kRouteTokensPerBlock * k);
@@ -208,7 +216,12 @@ gather_rows_kernel(const uint4 *__restrict__ x, const int *__restrict__ sorted_t
     const int t = sorted_to_flat[r] / k;
     const uint4 *src = x + (size_t)t * vec_per_row;
     uint4 *dst = x_perm + (size_t)r * vec_per_row;
-    for (int i = lane; i < vec_per_row; i += 32) dst[i] = src[i];
+    int i = lane;
+    for (; i + 96 < vec_per_row; i += 128) {  // four independent 16-byte loads in flight per lane
+        const uint4 a = src[i], b = src[i + 32], c = src[i + 64], d = src[i + 96];
+        dst[i] = a; dst[i + 32] = b; dst[i + 64] = c; dst[i + 96] = d;
+    }
+    for (; i < vec_per_row; i += 32) dst[i] = src[i];
 }
 
 __global__ void __launch_bounds__(256)
@@ -265,7 +278,7 @@ cudaError_t launch_route(const float *logits, int T, int E, int k, int nt_max, i
                                                                        scratch.chunk_counts);
     route_scan_kernel<<<1, 256, 0, stream>>>(scratch.chunk_counts, scratch.n_chunks, E, nt_max, expert_offsets,
                                              scratch.tile_prefix, scratch.tile_order, scratch.tile_rows);
-    route_scatter_kernel<<<scratch.n_chunks, 32, 0, stream>>>(topk_ids, scratch.chunk_counts, A, E, k,
+    route_scatter_kernel<<<scratch.n_chunks, 32, 0, stream>>>(topk_ids, scratch.chunk_counts, expert_offsets, A, E, k,
                                                               sorted_to_flat, flat_to_sorted);
     return cudaGetLastError();
 }

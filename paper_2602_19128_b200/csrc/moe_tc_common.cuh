@@ -14,14 +14,14 @@ constexpr int kRowBytes = kBlockK * 2;             // 128
 constexpr int kThreads = 192;                      // warp 0 TMA, warp 1 MMA, warps 2..5 epilogue
 constexpr int kEpilogueWarps = 4;
 constexpr long long kWaitLimitCycles = 4000000000LL;  // about two seconds at full clock
-constexpr int kNumActMaps = 16;                    // activation boxes of 16, 32, ..., 256 rows
+constexpr int kNumActMaps = 16;                    // activation boxes of q, 2q, ..., 16q rows (q = 16, or 8 for pairs)
 
 // Tensor maps of one grouped GEMM.  `w` is either a 2-D map over [E*w_rows, K] with a 128-row box
 // (down projection) or a 5-D map over w13 viewed as [E][I/16][gate|up][16][H] whose
 // {64,16,2,4,1} box delivers 64 features as 4 x (16 gate rows, 16 up rows) in one copy.
 struct TensorMaps {
     CUtensorMap w;
-    CUtensorMap act[kNumActMaps];  // act[i]: box of 16 * (i + 1) rows, so any token tile is ONE copy
+    CUtensorMap act[kNumActMaps];  // act[i]: box of q * (i + 1) rows, so any token tile is ONE copy
 };
 
 struct KernelParams {
@@ -82,6 +82,26 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
 }
 
+// True in exactly one lane of a converged warp, always the same lane.  The role loops are run by
+// whole warps and only the issuing instructions sit under this predicate: loop state then stays
+// warp-uniform and the descriptors of TMA / tcgen05 instructions (which take uniform-register
+// operands) need no per-instruction transfer.  Measured: with a single lane running the whole loop
+// under `lane == 0`, every TMA or MMA instruction cost about 150 cycles to issue.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "elect.sync _|p, 0xffffffff;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(pred));
+    return pred != 0;
+}
+// Bounded wait by a whole warp; the result is made uniform.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status,
+                                               int site) {
+    return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, status, site));
+}
+
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int c0, int c1, uint32_t bar) {
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
@@ -131,11 +151,13 @@ __device__ __forceinline__ uint32_t instr_desc_bf16(int m, int n) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
-// The map whose box holds exactly n_rows activation rows (n_rows a multiple of 16, at most 256).
+// The map whose box holds exactly n_rows activation rows (n_rows a multiple of the quantum the maps
+// were encoded with: 16 rows up to 256 for the one-CTA kernel, 8 rows up to 128 for each CTA of a pair).
 // One copy per ring slot and operand: every TMA copy has a fixed cost in the copy engine that is
 // comparable to moving several KiB, so a token tile is never assembled from smaller boxes.
+template <int kQuantum>
 __device__ __forceinline__ const CUtensorMap *act_map(const TensorMaps &maps, int n_rows) {
-    return &maps.act[(n_rows >> 4) - 1];
+    return &maps.act[n_rows / kQuantum - 1];
 }
 
 struct Tile {
@@ -175,7 +197,7 @@ __device__ __forceinline__ float swiglu(float g, float u) { return __fdividef(g,
 // ---- host side ----------------------------------------------------------------------------------
 bool encode_weight_map_2d(CUtensorMap *map, const void *w, uint64_t rows, uint64_t K);
 bool encode_weight_map_gate_up(CUtensorMap *map, const void *w13, int E, int I, int H);
-bool encode_act_maps(CUtensorMap *maps, const void *act, uint64_t rows, uint64_t K);
+bool encode_act_maps(CUtensorMap *maps, const void *act, uint64_t rows, uint64_t K, int row_quantum);
 int sm_count();
 
 }  // namespace tc

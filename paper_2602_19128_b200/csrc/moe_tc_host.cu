@@ -61,9 +61,9 @@ bool encode_weight_map_gate_up(CUtensorMap *map, const void *w13, int E, int I, 
     return encode(map, w13, 5, dims, strides, box);
 }
 
-bool encode_act_maps(CUtensorMap *maps, const void *act, uint64_t rows, uint64_t K) {
+bool encode_act_maps(CUtensorMap *maps, const void *act, uint64_t rows, uint64_t K, int row_quantum) {
     for (int i = 0; i < kNumActMaps; ++i)
-        if (!encode_2d(&maps[i], act, rows, K, 16u * (uint32_t)(i + 1))) return false;
+        if (!encode_2d(&maps[i], act, rows, K, (uint32_t)row_quantum * (uint32_t)(i + 1))) return false;
     return true;
 }
 

@@ -24,6 +24,8 @@ SMALL = [
     (700, 256, 256, 4, 2, False),     # CTA-pair kernel for both GEMMs, two token tiles per expert
     (300, 512, 384, 2, 2, False),     # CTA-pair kernel, 300 rows per expert: two ragged tiles of N = 160
     (130, 256, 128, 1, 1, False),     # one expert, 130 rows: pair tile with a nearly empty second half
+    (700, 256, 256, 2, 1, False),     # ~350 rows per expert: two weight slabs per CTA in the gate/up GEMM
+    (600, 512, 512, 2, 2, False),     # 600 rows per expert: three token tiles of 208, two 512-row pair tiles
 ]
 
 
@@ -37,8 +39,9 @@ def oracle_everything(case):
     return ids, w, off, s2f, f2s, h, y, out
 
 
-@pytest.mark.parametrize("flags", [moe.MOE_FLAG_VALIDATION_GEMM, moe.MOE_FLAG_SINGLE_CTA_GEMM, moe.MOE_FLAG_NONE],
-                         ids=["cuda_core", "tcgen05_single", "tcgen05"])
+@pytest.mark.parametrize("flags", [moe.MOE_FLAG_VALIDATION_GEMM, moe.MOE_FLAG_SINGLE_CTA_GEMM,
+                                   moe.MOE_FLAG_TWO_SLAB_GEMM, moe.MOE_FLAG_NONE],
+                         ids=["cuda_core", "tcgen05_single", "tcgen05_two_slab", "tcgen05"])
 @pytest.mark.parametrize("T,H,I,E,k,skew", SMALL)
 def test_forward_matches_oracle(T, H, I, E, k, skew, flags):
     inp = gpu_inputs(dict(T=T, H=H, I=I, E=E, top_k=k, skew=skew), seed=0)
