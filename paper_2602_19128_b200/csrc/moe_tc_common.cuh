@@ -14,6 +14,7 @@ constexpr int kRowBytes = kBlockK * 2;             // 128
 constexpr int kThreads = 192;                      // warp 0 TMA, warp 1 MMA, warps 2..5 epilogue
 constexpr int kEpilogueWarps = 4;
 constexpr long long kWaitLimitCycles = 4000000000LL;  // about two seconds at full clock
+constexpr uint32_t kWaitSuspendNs = 20000;            // upper bound of one hardware-suspended wait
 constexpr int kNumActMaps = 16;                    // activation boxes of q, 2q, ..., 16q rows (q = 16, or 8 for pairs)
 
 // Tensor maps of one grouped GEMM.  `w` is either a 2-D map over [E*w_rows, K] with a 128-row box
@@ -54,13 +55,26 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "memory");
     return done != 0;
 }
+// The same test, but the thread may be suspended by the hardware for up to `hint_ns` (it is woken
+// when the phase completes), so a long wait costs neither issue slots nor power.
+__device__ __forceinline__ bool mbar_try_wait_suspend(uint32_t bar, uint32_t parity, uint32_t hint_ns) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(bar), "r"(parity), "r"(hint_ns)
+        : "memory");
+    return done != 0;
+}
 // Bounded wait.  Returns false if the CTA is aborting (this wait expired, or another role's did).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status,
                                           int site) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long start = clock64();
     while (true) {
-        if (mbar_try_wait(bar, parity)) {
+        if (mbar_try_wait_suspend(bar, parity, kWaitSuspendNs)) {
 #ifdef MOE_WAIT_STATS  // experiment builds only: cycles spent waiting, per site, after the status ints
             if ((threadIdx.x & 31) == 0) {
                 unsigned long long *stats = reinterpret_cast<unsigned long long *>(status + 8);
