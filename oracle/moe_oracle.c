@@ -191,9 +191,9 @@ int moe_oracle_expert_ffn(const uint16_t *x_row, const uint16_t *w13_e, const ui
  *   x [T,H] bf16, router_logits [T,E] f32, w13_ptrs[e] -> [2I,H] bf16, w2_ptrs[e] -> [H,I] bf16,
  *   tokens [n_tokens] (indices into [0,T)), out [n_tokens,H] REAL.
  * out[i,:] = sum_{j ascending} topk_w[t,j] * expert_{ids[t,j]}(x[t,:]),  t = tokens[i]. */
-int moe_oracle_forward_sampled(const uint16_t *x, const float *router_logits, const uint16_t *const *w13_ptrs,
-                               const uint16_t *const *w2_ptrs, int T, int H, int I, int E, int k,
-                               const int32_t *tokens, int n_tokens, REAL *out) {
+static int forward_tokens(const uint16_t *x, const float *router_logits, const uint16_t *const *w13_ptrs,
+                          const uint16_t *const *w2_ptrs, int T, int H, int I, int E, int k, const int32_t *tokens,
+                          int n_tokens, int skip_missing, REAL *out) {
     if (T < 0 || H < 1 || I < 1 || E < 1 || k < 1 || k > E || n_tokens < 0) return ORACLE_ERR_ARG;
     int status = ORACLE_OK;
 #pragma omp parallel
@@ -222,6 +222,7 @@ int moe_oracle_forward_sampled(const uint16_t *x, const float *router_logits, co
                 for (int j = 0; j < k; ++j) {
                     const int e = ids[j];
                     if (!w13_ptrs[e] || !w2_ptrs[e]) {
+                        if (skip_missing) continue; /* expert not resident here: it contributes nothing */
 #pragma omp critical
                         status = ORACLE_ERR_MISSING_EXPERT;
                         continue;
@@ -234,6 +235,70 @@ int moe_oracle_forward_sampled(const uint16_t *x, const float *router_logits, co
         free(p); free(taken); free(ids); free(w); free(s); free(y);
     }
     return status;
+}
+
+int moe_oracle_forward_sampled(const uint16_t *x, const float *router_logits, const uint16_t *const *w13_ptrs,
+                               const uint16_t *const *w2_ptrs, int T, int H, int I, int E, int k,
+                               const int32_t *tokens, int n_tokens, REAL *out) {
+    return forward_tokens(x, router_logits, w13_ptrs, w2_ptrs, T, H, I, E, k, tokens, n_tokens, 0, out);
+}
+
+/* The layer restricted to the experts resident on one device (the paper's kernel computes "32 local
+ * experts" of 256, Sec. 4.5): routing is over all E experts, but only assignments whose expert lies in
+ * [local_offset, local_offset + n_local) are evaluated; the others contribute nothing, and the routing
+ * weights are NOT renormalised over the local ones, so the partial outputs of devices that partition
+ * the experts add up to the full layer.
+ *   w13_local [n_local,2I,H] bf16, w2_local [n_local,H,I] bf16 -> out [T,H] REAL. */
+int moe_oracle_forward_local(const uint16_t *x, const float *router_logits, const uint16_t *w13_local,
+                             const uint16_t *w2_local, int T, int H, int I, int E, int k, int local_offset, int n_local,
+                             REAL *out) {
+    if (T < 0 || H < 1 || I < 1 || E < 1 || k < 1 || k > E || local_offset < 0 || n_local < 0 || local_offset + n_local > E)
+        return ORACLE_ERR_ARG;
+    const uint16_t **p13 = (const uint16_t **)calloc((size_t)E, sizeof(void *));
+    const uint16_t **p2 = (const uint16_t **)calloc((size_t)E, sizeof(void *));
+    int32_t *tokens = (int32_t *)malloc(sizeof(int32_t) * (size_t)(T > 0 ? T : 1));
+    int status = ORACLE_ERR_NOMEM;
+    if (p13 && p2 && tokens) {
+        for (int l = 0; l < n_local; ++l) {
+            p13[local_offset + l] = w13_local + (size_t)l * 2 * I * H;
+            p2[local_offset + l] = w2_local + (size_t)l * H * I;
+        }
+        for (int t = 0; t < T; ++t) tokens[t] = t;
+        status = forward_tokens(x, router_logits, p13, p2, T, H, I, E, k, tokens, T, 1, out);
+    }
+    free(p13); free(p2); free(tokens);
+    return status;
+}
+
+/* Sort-scatter restricted to the local experts: a stable counting sort of the assignments whose
+ * expert is local, by local expert index; dropped assignments get flat_to_sorted = -1, and the tail
+ * of sorted_to_flat past expert_offsets[n_local] is -1. */
+int moe_oracle_permute_local(const int32_t *topk_ids, int T, int k, int local_offset, int n_local,
+                             int32_t *expert_offsets, int32_t *sorted_to_flat, int32_t *flat_to_sorted) {
+    if (T < 0 || k < 1 || n_local < 0 || local_offset < 0) return ORACLE_ERR_ARG;
+    const long A = (long)T * k;
+    for (int e = 0; e <= n_local; ++e) expert_offsets[e] = 0;
+    for (long a = 0; a < A; ++a) {
+        const int l = topk_ids[a] - local_offset;
+        if (l >= 0 && l < n_local) expert_offsets[l + 1] += 1;
+    }
+    for (int e = 0; e < n_local; ++e) expert_offsets[e + 1] += expert_offsets[e];
+    int32_t *next = (int32_t *)malloc(sizeof(int32_t) * (size_t)(n_local > 0 ? n_local : 1));
+    if (!next) return ORACLE_ERR_NOMEM;
+    for (int e = 0; e < n_local; ++e) next[e] = expert_offsets[e];
+    for (long a = 0; a < A; ++a) sorted_to_flat[a] = -1;
+    for (long a = 0; a < A; ++a) {
+        const int l = topk_ids[a] - local_offset;
+        if (l >= 0 && l < n_local) {
+            const int32_t pos = next[l]++;
+            flat_to_sorted[a] = pos;
+            sorted_to_flat[pos] = (int32_t)a;
+        } else {
+            flat_to_sorted[a] = -1;
+        }
+    }
+    free(next);
+    return ORACLE_OK;
 }
 
 /* The whole layer on contiguous weights: w13 [E,2I,H] bf16, w2 [E,H,I] bf16 -> out [T,H] REAL. */
@@ -250,7 +315,7 @@ int moe_oracle_forward(const uint16_t *x, const float *router_logits, const uint
             p2[e] = w2 + (size_t)e * H * I;
         }
         for (int t = 0; t < T; ++t) tokens[t] = t;
-        status = moe_oracle_forward_sampled(x, router_logits, p13, p2, T, H, I, E, k, tokens, T, out);
+        status = forward_tokens(x, router_logits, p13, p2, T, H, I, E, k, tokens, T, 0, out);
     }
     free(p13); free(p2); free(tokens);
     return status;

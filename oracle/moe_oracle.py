@@ -50,7 +50,8 @@ class Oracle:
         self.lib = ctypes.CDLL(str(build()[precision]))
         assert self.lib.moe_oracle_real_bytes() == np.dtype(self.real).itemsize
         for fn in ("moe_oracle_route", "moe_oracle_permute", "moe_oracle_expert_ffn", "moe_oracle_forward",
-                   "moe_oracle_forward_sampled", "moe_oracle_sorted_intermediates"):
+                   "moe_oracle_forward_sampled", "moe_oracle_sorted_intermediates", "moe_oracle_forward_local",
+                   "moe_oracle_permute_local"):
             getattr(self.lib, fn).restype = ctypes.c_int
 
     # -- helpers ---------------------------------------------------------------------------
@@ -136,6 +137,30 @@ class Oracle:
                                                         self._ptr(tokens), len(tokens), self._ptr(out)),
                     "forward_sampled")
         return out
+
+    def forward_local(self, x, router_logits, w13_local, w2_local, E: int, top_k: int, local_offset: int):
+        """Partial layer output of a device that holds experts [local_offset, local_offset + n_local)."""
+        x, w13_local, w2_local = self._u16(x), self._u16(w13_local), self._u16(w2_local)
+        l = np.ascontiguousarray(router_logits, dtype=np.float32)
+        T, H = x.shape
+        n_local, I2, _ = w13_local.shape
+        I = I2 // 2
+        assert l.shape == (T, E) and w2_local.shape == (n_local, H, I)
+        out = np.empty((T, H), self.real)
+        self._check(self.lib.moe_oracle_forward_local(self._ptr(x), self._ptr(l), self._ptr(w13_local),
+                                                      self._ptr(w2_local), T, H, I, E, top_k, local_offset, n_local,
+                                                      self._ptr(out)), "forward_local")
+        return out
+
+    def permute_local(self, topk_ids: np.ndarray, local_offset: int, n_local: int):
+        ids = np.ascontiguousarray(topk_ids, dtype=np.int32)
+        T, k = ids.shape
+        offsets = np.empty(n_local + 1, np.int32)
+        s2f = np.empty(T * k, np.int32)
+        f2s = np.empty(T * k, np.int32)
+        self._check(self.lib.moe_oracle_permute_local(self._ptr(ids), T, k, local_offset, n_local, self._ptr(offsets),
+                                                      self._ptr(s2f), self._ptr(f2s)), "permute_local")
+        return offsets, s2f, f2s
 
     def sorted_intermediates(self, x, w13, w2, topk_ids, sorted_to_flat):
         x, w13, w2 = self._u16(x), self._u16(w13), self._u16(w2)
