@@ -28,14 +28,17 @@ import torch
 ROOT = Path(__file__).resolve().parent
 sys.path.insert(0, str(ROOT))
 
-from paper_2602_19128_b200.inputs import CONFIGS, bf16_bits, make_inputs  # noqa: E402
+from paper_2602_19128_b200.inputs import CONFIGS, LOCAL_CONFIGS, bf16_bits, make_inputs  # noqa: E402
+
+CONFIGS = dict(CONFIGS, **LOCAL_CONFIGS)  # the five workloads plus the local-expert-subset shapes
 
 METRIC = "moe_layer_tokens_per_s"
 UNIT = "tokens/s"
 L2_BYTES = 126 * 1024 * 1024
 # Which roofline bounds the dominant kernel (gate/up GEMM) of each workload: weight bytes per useful
 # flop put mixtral / dsv3_decode (and tiny) below the ridge point and the prefill-sized ones above it.
-BOUND = {"tiny": "hbm", "mixtral": "hbm", "dsv3_decode": "hbm", "dsv3_prefill": "tensor", "skewed": "tensor"}
+BOUND = {"tiny": "hbm", "mixtral": "hbm", "dsv3_decode": "hbm", "dsv3_prefill": "tensor", "skewed": "tensor",
+         "dsv3_local32_prefill": "hbm", "dsv3_local32_decode": "hbm"}
 # DRAM bytes (read + write) of one gate/up GEMM launch, from the ncu capture summarised under profiles/.
 NCU_TRAFFIC_BYTES = {"mixtral": 1929712128}
 
@@ -209,6 +212,7 @@ def run_ours(args):
     T, H, I, E, k = (cfg[n] for n in ("T", "H", "I", "E", "top_k"))
     inp = make_inputs(args.config, seed=args.seed + rank, device=dev)
     x, logits, w13, w2 = inp["x"], inp["router_logits"], inp["w13"], inp["w2"]
+    local_offset, n_local = inp["local_offset"], inp["local"]
     out = torch.empty((T, H), dtype=torch.bfloat16, device=dev)
     ws = moe.alloc_workspace(moe.moe_workspace_bytes(T, H, I, E, k), dev)
     weight_bytes = (w13.numel() + w2.numel()) * 2
@@ -224,7 +228,7 @@ def run_ours(args):
 
     # ---- device-resident timing ----------------------------------------------------------------
     for _ in range(max(args.warmup, 3)):
-        moe.moe_forward(x, logits, w13, w2, k, out, ws)
+        moe.moe_forward_local(x, logits, w13, w2, k, local_offset, out, ws)
     status = moe.moe_last_status(ws)
     if status != moe.MOE_OK:
         raise SystemExit(f"device status {status}: {moe.moe_status_string(status)}")
@@ -234,7 +238,7 @@ def run_ours(args):
     for s in range(args.steps):
         if need_flush:
             flush_l2(flush_buf)
-        moe.moe_forward_staged(x, logits, w13, w2, k, out, ws, stage_events[s])
+        moe.moe_forward_staged(x, logits, w13, w2, k, out, ws, stage_events[s], local_expert_offset=local_offset)
     barrier()
     clocks = sampler.stop() if sampler else None
     if need_flush:
@@ -249,7 +253,8 @@ def run_ours(args):
     if status != moe.MOE_OK:
         raise SystemExit(f"device status {status}: {moe.moe_status_string(status)}")
     views = moe.workspace_views(ws, T, H, I, E, k)
-    counts = torch.diff(views["expert_offsets"]).cpu().numpy()
+    counts = torch.diff(views["expert_offsets"][:n_local + 1]).cpu().numpy()
+    rows_scheduled = int(counts.sum())  # = T*k unless only a subset of the experts is resident
     n_active = int((counts > 0).sum())
 
     # ---- end to end through the host-buffer entry point ---------------------------------------------
@@ -257,7 +262,7 @@ def run_ours(args):
     lh = logits.cpu().pin_memory()
     oh = torch.empty((T, H), dtype=torch.bfloat16).pin_memory()
     for _ in range(3):
-        moe.moe_forward_host(xh, lh, w13, w2, k, oh, ws)
+        moe.moe_forward_host(xh, lh, w13, w2, k, oh, ws, local_expert_offset=local_offset)
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e2e_ms = 0.0
@@ -265,14 +270,14 @@ def run_ours(args):
         for _ in range(args.steps):
             flush_l2(flush_buf)
             e0.record()
-            moe.moe_forward_host(xh, lh, w13, w2, k, oh, ws)
+            moe.moe_forward_host(xh, lh, w13, w2, k, oh, ws, local_expert_offset=local_offset)
             e1.record()
             e1.synchronize()
             e2e_ms += e0.elapsed_time(e1)
     else:
         e0.record()
         for _ in range(args.steps):
-            moe.moe_forward_host(xh, lh, w13, w2, k, oh, ws)
+            moe.moe_forward_host(xh, lh, w13, w2, k, oh, ws, local_expert_offset=local_offset)
         e1.record()
         e1.synchronize()
         e2e_ms = e0.elapsed_time(e1)
@@ -287,7 +292,7 @@ def run_ours(args):
 
     # ---- roofline of the dominant kernel (gate/up GEMM + SwiGLU) -----------------------------------
     peaks = load_peaks()
-    A = T * k
+    A = rows_scheduled
     t_gemm1 = stage_ms["gemm1_swiglu"] * 1e-3
     bound = BOUND[args.config]
     if bound == "hbm":
@@ -312,13 +317,14 @@ def run_ours(args):
                  useful_tflops_frac_burst=6.0 * A * H * I / step_s / 1e12 / peaks["tflops_burst"])
 
     cpu_baseline = None
-    if world == 1 and not args.no_cpu_baseline:
+    if world == 1 and not args.no_cpu_baseline and n_local == E:
         cpu_baseline = time_oracle(args.config, inp, budget_s=15.0)
 
     line = dict(metric=METRIC, value=aggregate_tokens_per_s(world, T, args.steps, total_ms), unit=UNIT, n_gpus=world,
                 steps=args.steps, warmup=max(args.warmup, 3), ms_per_step=total_ms / args.steps, higher_is_better=True,
                 scaling="weak", vs_baseline=None, dtype="bf16", data="synthetic",
-                config=dict(workload=args.config, T=T, H=H, I=I, E=E, top_k=k, parallelism=f"replicas x{world}",
+                config=dict(workload=args.config, T=T, H=H, I=I, E=E, top_k=k, resident_experts=n_local,
+                            parallelism=f"replicas x{world}",
                             l2="flushed between steps" if need_flush else "weights larger than L2, no flush",
                             seed=args.seed),
                 clocks=clocks,
@@ -349,6 +355,8 @@ def main():
         CONFIGS[args.config] = dict(T=T, H=H, I=I, E=E, top_k=k, skew=False)
         BOUND[args.config] = "hbm"
     if args.impl == "reference":
+        if args.config in LOCAL_CONFIGS:
+            raise SystemExit("the reference arm covers the five whole-layer workloads")
         run_reference(args)
     else:
         run_ours(args)

@@ -163,27 +163,44 @@ MOE_API int moe_forward_ex(const void *x, const float *router_logits, const void
                    int E, int top_k, void *out, void *workspace, size_t workspace_bytes, void *stream,
                    unsigned flags);
 
-/* moe_forward_ex that also records CUDA events between the stages, for per-kernel timing inside a
- * whole step.  stage_events is a HOST array of MOE_NUM_STAGE_EVENTS cudaEvent_t handles (passed as
- * void*, created by the caller with timing enabled).  Event 0 is recorded on `stream` before the
- * first kernel, and event i+1 after stage i, where the stages are
+/* The layer restricted to the experts resident on this device (the paper's kernel computes "32 local
+ * experts" out of 256, Sec. 4.5): the router still chooses among all E experts from router_logits
+ * [T,E], but only assignments to experts [local_expert_offset, local_expert_offset + num_local_experts)
+ * are computed; the others contribute nothing to `out`, and the routing weights are NOT renormalised
+ * over the local experts, so the outputs of devices that partition the experts add up to the full layer.
+ *   w13_local [num_local_experts, 2I, H] bf16, w2_local [num_local_experts, H, I] bf16: the resident experts,
+ *   local expert l being global expert local_expert_offset + l.
+ * Workspace as for moe_forward (same size); afterwards topk_ids / topk_weights hold the full routing,
+ * expert_offsets has num_local_experts + 1 entries, flat_to_sorted is -1 for dropped assignments and
+ * only the first expert_offsets[num_local_experts] entries of sorted_to_flat are defined.
+ * MOE_ERR_SHAPE if the local range is empty or not inside [0, E). */
+MOE_API int moe_forward_local(const void *x, const float *router_logits, const void *w13_local, const void *w2_local,
+                              int T, int H, int I, int E, int top_k, int local_expert_offset, int num_local_experts,
+                              void *out, void *workspace, size_t workspace_bytes, void *stream, unsigned flags);
+
+/* moe_forward_local (pass local_expert_offset = 0, num_local_experts = E for the whole layer) that also
+ * records CUDA events between the stages, for per-kernel timing inside a whole step.  stage_events is a
+ * HOST array of MOE_NUM_STAGE_EVENTS cudaEvent_t handles (passed as void*, created by the caller with
+ * timing enabled).  Event 0 is recorded on `stream` before the first kernel, and event i+1 after
+ * stage i, where the stages are
  *   0 router + sort-scatter (3 kernels), 1 row gather, 2 gate/up GEMM + SwiGLU, 3 down GEMM, 4 combine.
  * With T == 0 nothing is launched and no event is recorded. */
 #define MOE_NUM_STAGE_EVENTS 6
 MOE_API int moe_forward_staged(const void *x, const float *router_logits, const void *w13, const void *w2, int T, int H,
-                               int I, int E, int top_k, void *out, void *workspace, size_t workspace_bytes,
-                               void *stream, unsigned flags, void *const *stage_events);
+                               int I, int E, int top_k, int local_expert_offset, int num_local_experts, void *out,
+                               void *workspace, size_t workspace_bytes, void *stream, unsigned flags,
+                               void *const *stage_events);
 
-/* moe_forward for a caller whose activations live in HOST memory: x_host [T,H] bf16 and
- * router_logits_host [T,E] f32 are HOST pointers (pinned memory makes the copies asynchronous),
- * out_host [T,H] bf16 is a HOST pointer; the expert weights w13 / w2 stay DEVICE pointers
- * (they are model parameters, resident across calls).  The call enqueues, on `stream`, the
- * host-to-device copies into the workspace's staging area, the layer, and the device-to-host
- * copy of the result, and returns without synchronising: out_host is valid once the stream
- * has been synchronised. */
+/* moe_forward_local (local_expert_offset = 0, num_local_experts = E for the whole layer) for a caller
+ * whose activations live in HOST memory: x_host [T,H] bf16 and router_logits_host [T,E] f32 are HOST
+ * pointers (pinned memory makes the copies asynchronous), out_host [T,H] bf16 is a HOST pointer; the
+ * expert weights w13 / w2 stay DEVICE pointers (they are model parameters, resident across calls).
+ * The call enqueues, on `stream`, the host-to-device copies into the workspace's staging area, the
+ * layer, and the device-to-host copy of the result, and returns without synchronising: out_host is
+ * valid once the stream has been synchronised. */
 MOE_API int moe_forward_host(const void *x_host, const float *router_logits_host, const void *w13, const void *w2, int T,
-                     int H, int I, int E, int top_k, void *out_host, void *workspace, size_t workspace_bytes,
-                     void *stream);
+                             int H, int I, int E, int top_k, int local_expert_offset, int num_local_experts,
+                             void *out_host, void *workspace, size_t workspace_bytes, void *stream);
 
 /* Synchronises `stream`, then reads the status word the kernels of the last moe_forward /
  * moe_route call left in `workspace`.  MOE_OK, MOE_ERR_DEVICE_TIMEOUT, or MOE_ERR_CUDA if the

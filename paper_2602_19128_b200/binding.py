@@ -21,7 +21,7 @@ MOE_FLAG_TWO_SLAB_GEMM = 4
 
 EXPORTED = ["moe_workspace_bytes", "moe_workspace_layout", "moe_route_workspace_bytes", "moe_route", "moe_route_static",
             "moe_forward",
-            "moe_forward_ex", "moe_forward_staged", "moe_forward_host", "moe_last_status", "moe_forward_launch_count", "moe_status_string"]
+            "moe_forward_ex", "moe_forward_local", "moe_forward_staged", "moe_forward_host", "moe_last_status", "moe_forward_launch_count", "moe_status_string"]
 
 
 class MoeError(RuntimeError):
@@ -62,11 +62,13 @@ def lib() -> ctypes.CDLL:
         L.moe_forward.argtypes = [vp, vp, vp, vp, i, i, i, i, i, vp, vp, sz, vp]
         L.moe_forward_ex.restype = i
         L.moe_forward_ex.argtypes = [vp, vp, vp, vp, i, i, i, i, i, vp, vp, sz, vp, ctypes.c_uint]
+        L.moe_forward_local.restype = i
+        L.moe_forward_local.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, vp, vp, sz, vp, ctypes.c_uint]
         L.moe_forward_staged.restype = i
-        L.moe_forward_staged.argtypes = [vp, vp, vp, vp, i, i, i, i, i, vp, vp, sz, vp, ctypes.c_uint,
+        L.moe_forward_staged.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, vp, vp, sz, vp, ctypes.c_uint,
                                          ctypes.POINTER(vp)]
         L.moe_forward_host.restype = i
-        L.moe_forward_host.argtypes = [vp, vp, vp, vp, i, i, i, i, i, vp, vp, sz, vp]
+        L.moe_forward_host.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, vp, vp, sz, vp]
         L.moe_last_status.restype = i
         L.moe_last_status.argtypes = [vp, vp]
         L.moe_forward_launch_count.restype = i
@@ -153,6 +155,20 @@ def moe_forward(x, router_logits, w13, w2, top_k: int, out, workspace, stream=No
     return st
 
 
+def moe_forward_local(x, router_logits, w13_local, w2_local, top_k: int, local_expert_offset: int, out, workspace,
+                      stream=None, flags: int = 0, check: bool = True) -> int:
+    """The layer restricted to the resident experts [local_expert_offset, + w13_local.shape[0])."""
+    T, H = x.shape
+    E = router_logits.shape[1]
+    n_local, I2, _ = w13_local.shape
+    st = lib().moe_forward_local(_ptr(x), _ptr(router_logits), _ptr(w13_local), _ptr(w2_local), T, H, I2 // 2, E, top_k,
+                                 local_expert_offset, n_local, _ptr(out), _ptr(workspace), workspace.numel(),
+                                 _stream(stream), flags)
+    if check and st != MOE_OK:
+        raise MoeError(st, "moe_forward_local")
+    return st
+
+
 STAGE_NAMES = ("route", "gather", "gemm1_swiglu", "gemm2", "combine")
 NUM_STAGE_EVENTS = len(STAGE_NAMES) + 1
 
@@ -167,25 +183,31 @@ def make_stage_events() -> list:
 
 
 def moe_forward_staged(x, router_logits, w13, w2, top_k: int, out, workspace, stage_events, stream=None,
-                       flags: int = 0, check: bool = True) -> int:
-    """moe_forward that records ``stage_events`` (from make_stage_events) around the five stages."""
+                       flags: int = 0, local_expert_offset: int = 0, check: bool = True) -> int:
+    """moe_forward (or moe_forward_local when w13 holds fewer experts than the router has columns) that
+    records ``stage_events`` (from make_stage_events) around the five stages."""
     T, H = x.shape
-    E, I2, _ = w13.shape
+    E = router_logits.shape[1]
+    n_local, I2, _ = w13.shape
     handles = (ctypes.c_void_p * NUM_STAGE_EVENTS)(*[e.cuda_event for e in stage_events])
     st = lib().moe_forward_staged(_ptr(x), _ptr(router_logits), _ptr(w13), _ptr(w2), T, H, I2 // 2, E, top_k,
-                                  _ptr(out), _ptr(workspace), workspace.numel(), _stream(stream), flags, handles)
+                                  local_expert_offset, n_local, _ptr(out), _ptr(workspace), workspace.numel(),
+                                  _stream(stream), flags, handles)
     if check and st != MOE_OK:
         raise MoeError(st, "moe_forward_staged")
     return st
 
 
 def moe_forward_host(x_host, router_logits_host, w13, w2, top_k: int, out_host, workspace, stream=None,
-                     check: bool = True) -> int:
-    """x_host / router_logits_host / out_host are CPU tensors (pinned for asynchronous copies)."""
+                     local_expert_offset: int = 0, check: bool = True) -> int:
+    """x_host / router_logits_host / out_host are CPU tensors (pinned for asynchronous copies); w13 / w2 are
+    the resident experts on the device (all E of them, or a local subset starting at local_expert_offset)."""
     T, H = x_host.shape
-    E, I2, _ = w13.shape
+    E = router_logits_host.shape[1]
+    n_local, I2, _ = w13.shape
     st = lib().moe_forward_host(_ptr(x_host), _ptr(router_logits_host), _ptr(w13), _ptr(w2), T, H, I2 // 2, E, top_k,
-                                _ptr(out_host), _ptr(workspace), workspace.numel(), _stream(stream))
+                                local_expert_offset, n_local, _ptr(out_host), _ptr(workspace), workspace.numel(),
+                                _stream(stream))
     if check and st != MOE_OK:
         raise MoeError(st, "moe_forward_host")
     return st

@@ -49,9 +49,11 @@ int check_device() {
 
 int forward_impl(const void *x, const float *logits, const void *w13, const void *w2, int T, int H, int I, int E, int k,
                  void *out, void *workspace, size_t workspace_bytes, cudaStream_t stream, unsigned flags,
-                 void *const *stage_events = nullptr) {
+                 void *const *stage_events = nullptr, int local_offset = 0, int n_local = -1) {
+    if (n_local < 0) n_local = E;  // every expert is resident
     if (T < 0 || H <= 0 || I <= 0 || E <= 0 || k <= 0 || k > E) return MOE_ERR_SHAPE;
     if (!envelope_ok(T, H, I, E, k)) return MOE_ERR_UNSUPPORTED;
+    if (local_offset < 0 || n_local < 1 || (long long)local_offset + n_local > E) return MOE_ERR_SHAPE;
     if (flags & ~(MOE_FLAG_VALIDATION_GEMM | MOE_FLAG_SINGLE_CTA_GEMM | MOE_FLAG_TWO_SLAB_GEMM)) return MOE_ERR_UNSUPPORTED;
     if (T == 0) return MOE_OK;
     if (!x || !logits || !w13 || !w2 || !out || !workspace) return MOE_ERR_NULL;
@@ -71,7 +73,7 @@ int forward_impl(const void *x, const float *logits, const void *w13, const void
     int *offsets = reinterpret_cast<int *>(ws + L.expert_offsets);
     int *s2f = reinterpret_cast<int *>(ws + L.sorted_to_flat);
     int *f2s = reinterpret_cast<int *>(ws + L.flat_to_sorted);
-    RouteScratch rs = carve_route_scratch(ws + L.route_scratch, T, E);
+    RouteScratch rs = carve_route_scratch(ws + L.route_scratch, T, n_local);
     __nv_bfloat16 *x_perm = reinterpret_cast<__nv_bfloat16 *>(ws + L.x_perm);
     __nv_bfloat16 *h = reinterpret_cast<__nv_bfloat16 *>(ws + L.h);
     __nv_bfloat16 *y = reinterpret_cast<__nv_bfloat16 *>(ws + L.y);
@@ -82,16 +84,18 @@ int forward_impl(const void *x, const float *logits, const void *w13, const void
         return !stage_events || cudaEventRecord(static_cast<cudaEvent_t>(stage_events[i]), stream) == cudaSuccess;
     };
     if (!mark(0)) return MOE_ERR_CUDA;
-    if (launch_route(logits, T, E, k, nt_max, ids, wts, offsets, s2f, f2s, rs, status, stream) != cudaSuccess)
+    if (launch_route(logits, T, E, k, LocalExperts{local_offset, n_local}, nt_max, ids, wts, offsets, s2f, f2s, rs, status,
+                     stream) != cudaSuccess)
         return MOE_ERR_CUDA;
     if (!mark(1)) return MOE_ERR_CUDA;
-    if (launch_gather_rows(static_cast<const __nv_bfloat16 *>(x), s2f, A, k, H, x_perm, stream) != cudaSuccess)
+    if (launch_gather_rows(static_cast<const __nv_bfloat16 *>(x), s2f, offsets + n_local, A, k, H, x_perm, stream) !=
+        cudaSuccess)
         return MOE_ERR_CUDA;
     if (!mark(2)) return MOE_ERR_CUDA;
 
     GroupedGemmArgs g1;
     g1.act = x_perm; g1.w = static_cast<const __nv_bfloat16 *>(w13); g1.out = h;
-    g1.A = A; g1.K = H; g1.n_out = I; g1.E = E; g1.w_rows = 2 * I; g1.nt_max = nt_max;
+    g1.A = A; g1.K = H; g1.n_out = I; g1.E = n_local; g1.w_rows = 2 * I; g1.nt_max = nt_max;
     g1.expert_offsets = offsets; g1.tile_prefix = rs.tile_prefix; g1.tile_order = rs.tile_order; g1.tile_rows = rs.tile_rows;
     g1.status = status; g1.swiglu = true;
     GroupedGemmArgs g2 = g1;
@@ -173,8 +177,8 @@ int moe_route(const float *router_logits, int T, int E, int top_k, int32_t *topk
     }
     char *ws = static_cast<char *>(workspace);
     RouteScratch rs = carve_route_scratch(ws + 256, T, E);
-    const cudaError_t err = launch_route(router_logits, T, E, top_k, 256, topk_ids, topk_weights, expert_offsets,
-                                         sorted_to_flat, flat_to_sorted, rs, reinterpret_cast<int *>(ws), s);
+    const cudaError_t err = launch_route(router_logits, T, E, top_k, LocalExperts{0, E}, 256, topk_ids, topk_weights,
+                                         expert_offsets, sorted_to_flat, flat_to_sorted, rs, reinterpret_cast<int *>(ws), s);
     return err == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
 
@@ -190,19 +194,29 @@ int moe_forward_ex(const void *x, const float *router_logits, const void *w13, c
                         static_cast<cudaStream_t>(stream), flags);
 }
 
+int moe_forward_local(const void *x, const float *router_logits, const void *w13_local, const void *w2_local, int T, int H,
+                      int I, int E, int top_k, int local_expert_offset, int num_local_experts, void *out, void *workspace,
+                      size_t workspace_bytes, void *stream, unsigned flags) {
+    if (num_local_experts < 1) return MOE_ERR_SHAPE;
+    return forward_impl(x, router_logits, w13_local, w2_local, T, H, I, E, top_k, out, workspace, workspace_bytes,
+                        static_cast<cudaStream_t>(stream), flags, nullptr, local_expert_offset, num_local_experts);
+}
+
 int moe_forward_staged(const void *x, const float *router_logits, const void *w13, const void *w2, int T, int H, int I,
-                       int E, int top_k, void *out, void *workspace, size_t workspace_bytes, void *stream, unsigned flags,
-                       void *const *stage_events) {
+                       int E, int top_k, int local_expert_offset, int num_local_experts, void *out, void *workspace,
+                       size_t workspace_bytes, void *stream, unsigned flags, void *const *stage_events) {
     if (!stage_events) return MOE_ERR_NULL;
     for (int i = 0; i < MOE_NUM_STAGE_EVENTS; ++i)
         if (!stage_events[i]) return MOE_ERR_NULL;
+    if (num_local_experts < 1) return MOE_ERR_SHAPE;
     return forward_impl(x, router_logits, w13, w2, T, H, I, E, top_k, out, workspace, workspace_bytes,
-                        static_cast<cudaStream_t>(stream), flags, stage_events);
+                        static_cast<cudaStream_t>(stream), flags, stage_events, local_expert_offset, num_local_experts);
 }
 
 int moe_forward_host(const void *x_host, const float *router_logits_host, const void *w13, const void *w2, int T, int H,
-                     int I, int E, int top_k, void *out_host, void *workspace, size_t workspace_bytes, void *stream) {
-    if (T < 0 || H <= 0 || I <= 0 || E <= 0 || top_k <= 0 || top_k > E) return MOE_ERR_SHAPE;
+                     int I, int E, int top_k, int local_expert_offset, int num_local_experts, void *out_host,
+                     void *workspace, size_t workspace_bytes, void *stream) {
+    if (T < 0 || H <= 0 || I <= 0 || E <= 0 || top_k <= 0 || top_k > E || num_local_experts < 1) return MOE_ERR_SHAPE;
     if (!envelope_ok(T, H, I, E, top_k)) return MOE_ERR_UNSUPPORTED;
     if (T == 0) return MOE_OK;
     if (!x_host || !router_logits_host || !out_host || !workspace) return MOE_ERR_NULL;
@@ -219,7 +233,8 @@ int moe_forward_host(const void *x_host, const float *router_logits_host, const 
     if (cudaMemcpyAsync(x_dev, x_host, x_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return MOE_ERR_CUDA;
     if (cudaMemcpyAsync(l_dev, router_logits_host, l_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return MOE_ERR_CUDA;
     const int st = forward_impl(x_dev, reinterpret_cast<const float *>(l_dev), w13, w2, T, H, I, E, top_k, out_dev,
-                                workspace, workspace_bytes, s, MOE_FLAG_NONE);
+                                workspace, workspace_bytes, s, MOE_FLAG_NONE, nullptr, local_expert_offset,
+                                num_local_experts);
     if (st != MOE_OK) return st;
     if (cudaMemcpyAsync(out_host, out_dev, x_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) return MOE_ERR_CUDA;
     return MOE_OK;

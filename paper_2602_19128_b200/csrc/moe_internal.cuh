@@ -48,15 +48,22 @@ static inline RouteScratch carve_route_scratch(void *base, int T, int E) {
     return s;
 }
 
-// Router + histogram, exclusive scans + tile schedule, stable scatter.  `nt_max` is the largest
-// number of rows a GEMM token tile may have (multiple of 16).
-cudaError_t launch_route(const float *logits, int T, int E, int k, int nt_max, int *topk_ids, float *topk_w,
-                         int *expert_offsets, int *sorted_to_flat, int *flat_to_sorted, RouteScratch scratch,
-                         int *status, cudaStream_t stream);
+// The experts resident on this device: ids [offset, offset + count) of the E the router chooses from.
+// Assignments to other experts are dropped from the schedule (flat_to_sorted = -1).
+struct LocalExperts {
+    int offset, count;
+};
 
-// x_perm[r,:] = x[sorted_to_flat[r] / k, :]
-cudaError_t launch_gather_rows(const __nv_bfloat16 *x, const int *sorted_to_flat, int A, int k, int H,
-                               __nv_bfloat16 *x_perm, cudaStream_t stream);
+// Router + histogram, exclusive scans + tile schedule, stable scatter.  `nt_max` is the largest
+// number of rows a GEMM token tile may have (multiple of 16).  Scratch and expert_offsets are sized
+// by local.count.
+cudaError_t launch_route(const float *logits, int T, int E, int k, LocalExperts local, int nt_max, int *topk_ids,
+                         float *topk_w, int *expert_offsets, int *sorted_to_flat, int *flat_to_sorted,
+                         RouteScratch scratch, int *status, cudaStream_t stream);
+
+// x_perm[r,:] = x[sorted_to_flat[r] / k, :] for r < *n_rows (a device-side count, at most A)
+cudaError_t launch_gather_rows(const __nv_bfloat16 *x, const int *sorted_to_flat, const int *n_rows, int A, int k,
+                               int H, __nv_bfloat16 *x_perm, cudaStream_t stream);
 
 // out[t,:] = sum_j topk_w[t,j] * y[flat_to_sorted[t*k+j],:]
 cudaError_t launch_combine(const __nv_bfloat16 *y, const float *topk_w, const int *flat_to_sorted, int T, int k,

@@ -26,11 +26,11 @@ constexpr int kRouteThreads = 256;
 constexpr int kLogitsPerLane = kMaxExperts / 32;
 
 __global__ void __launch_bounds__(kRouteThreads)
-route_topk_kernel(const float *__restrict__ logits, int T, int E, int k, int *__restrict__ topk_ids,
-                  float *__restrict__ topk_w, int *__restrict__ chunk_counts) {
-    __shared__ int hist[kMaxExperts];
+route_topk_kernel(const float *__restrict__ logits, int T, int E, int k, int local_offset, int n_local,
+                  int *__restrict__ topk_ids, float *__restrict__ topk_w, int *__restrict__ chunk_counts) {
+    __shared__ int hist[kMaxExperts];  // indexed by local expert (expert id - local_offset)
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    for (int e = tid; e < E; e += kRouteThreads) hist[e] = 0;
+    for (int e = tid; e < n_local; e += kRouteThreads) hist[e] = 0;
     __syncthreads();
 
     const int t_base = blockIdx.x * kRouteTokensPerBlock;
@@ -96,11 +96,12 @@ route_topk_kernel(const float *__restrict__ logits, int T, int E, int k, int *__
         if (lane < k) {
             topk_ids[(size_t)t * k + lane] = my_id;
             topk_w[(size_t)t * k + lane] = my_p / denom;
-            atomicAdd(&hist[my_id], 1);
+            const int local = my_id - local_offset;  // only experts resident here are scheduled
+            if (local >= 0 && local < n_local) atomicAdd(&hist[local], 1);
         }
     }
     __syncthreads();
-    for (int e = tid; e < E; e += kRouteThreads) chunk_counts[(size_t)blockIdx.x * E + e] = hist[e];
+    for (int e = tid; e < n_local; e += kRouteThreads) chunk_counts[(size_t)blockIdx.x * n_local + e] = hist[e];
 }
 
 // Exclusive scan over the 256 threads of the block; returns the exclusive prefix, total in *total.
@@ -180,39 +181,38 @@ route_scan_kernel(int *__restrict__ chunk_counts, int n_chunks, int E, int nt_ma
 
 __global__ void __launch_bounds__(32)
 route_scatter_kernel(const int *__restrict__ topk_ids, const int *__restrict__ chunk_starts,
-                     const int *__restrict__ expert_offsets, int A, int E, int k, int *__restrict__ sorted_to_flat,
-                     int *__restrict__ flat_to_sorted) {
+                     const int *__restrict__ expert_offsets, int A, int n_local, int local_offset, int k,
+                     int *__restrict__ sorted_to_flat, int *__restrict__ flat_to_sorted) {
     __shared__ int next[kMaxExperts];
     const int lane = threadIdx.x;
     // first position of this chunk's assignments to expert e = segment start + rows of earlier chunks
-    for (int e = lane; e < E; e += 32) next[e] = expert_offsets[e] + chunk_starts[(size_t)blockIdx.x * E + e];
+    for (int e = lane; e < n_local; e += 32) next[e] = expert_offsets[e] + chunk_starts[(size_t)blockIdx.x * n_local + e];
     __syncwarp();
     const int a0 = blockIdx.x * kRouteTokensPerBlock * k;
     const int a1 = min(A, a0 + kRouteTokensPerBlock * k);
     for (int base = a0; base < a1; base += 32) {
         const int a = base + lane;
         const bool valid = a < a1;
-        const int e = valid ? topk_ids[a] : 0;
-        const int key = valid ? e : -1 - lane;  // lanes past the end never match anything
+        const int e = valid ? topk_ids[a] - local_offset : -1;
+        const bool kept = e >= 0 && e < n_local;       // assignments to experts that are not resident are dropped
+        const int key = kept ? e : -1 - lane;          // ... and never match anything
         const unsigned same = __match_any_sync(kFullMask, key);
         const int rank = __popc(same & ((1u << lane) - 1u));
-        const int pos = valid ? next[e] + rank : 0;
+        const int pos = kept ? next[e] + rank : -1;
         __syncwarp();
-        if (valid && rank == 0) next[e] += __popc(same);
+        if (kept && rank == 0) next[e] += __popc(same);
         __syncwarp();
-        if (valid) {
-            flat_to_sorted[a] = pos;
-            sorted_to_flat[pos] = a;
-        }
+        if (valid) flat_to_sorted[a] = pos;
+        if (kept) sorted_to_flat[pos] = a;
     }
 }
 
 __global__ void __launch_bounds__(256)
-gather_rows_kernel(const uint4 *__restrict__ x, const int *__restrict__ sorted_to_flat, int A, int k, int vec_per_row,
-                   uint4 *__restrict__ x_perm) {
+gather_rows_kernel(const uint4 *__restrict__ x, const int *__restrict__ sorted_to_flat,
+                   const int *__restrict__ n_rows, int k, int vec_per_row, uint4 *__restrict__ x_perm) {
     const int lane = threadIdx.x & 31;
     const int r = blockIdx.x * 8 + (threadIdx.x >> 5);
-    if (r >= A) return;
+    if (r >= *n_rows) return;  // rows actually scheduled: all A assignments, or fewer with a local-expert subset
     const int t = sorted_to_flat[r] / k;
     const uint4 *src = x + (size_t)t * vec_per_row;
     uint4 *dst = x_perm + (size_t)r * vec_per_row;
@@ -240,6 +240,7 @@ combine_kernel(const uint4 *__restrict__ y, const float *__restrict__ topk_w, co
 #pragma unroll
         for (int c = 0; c < 8; ++c) acc[c] = 0.f;
         for (int j = 0; j < k; ++j) {  // ascending rank: the summation order is fixed
+            if (rows[j] < 0) continue;   // expert not resident on this device: contributes nothing
             const uint4 v = y[(size_t)rows[j] * vec_per_row + i];
             const float wj = weights[j];
             const __nv_bfloat162 *h2 = reinterpret_cast<const __nv_bfloat162 *>(&v);
@@ -268,24 +269,25 @@ int choose_nt_max(int T, int E, int k) {
     return 256;
 }
 
-cudaError_t launch_route(const float *logits, int T, int E, int k, int nt_max, int *topk_ids, float *topk_w,
-                         int *expert_offsets, int *sorted_to_flat, int *flat_to_sorted, RouteScratch scratch,
-                         int *status, cudaStream_t stream) {
+cudaError_t launch_route(const float *logits, int T, int E, int k, LocalExperts local, int nt_max, int *topk_ids,
+                         float *topk_w, int *expert_offsets, int *sorted_to_flat, int *flat_to_sorted,
+                         RouteScratch scratch, int *status, cudaStream_t stream) {
     cudaError_t err = cudaMemsetAsync(status, 0, 256, stream);  // the status word and its padding
     if (err != cudaSuccess) return err;
     const int A = T * k;
-    route_topk_kernel<<<scratch.n_chunks, kRouteThreads, 0, stream>>>(logits, T, E, k, topk_ids, topk_w,
-                                                                       scratch.chunk_counts);
-    route_scan_kernel<<<1, 256, 0, stream>>>(scratch.chunk_counts, scratch.n_chunks, E, nt_max, expert_offsets,
+    route_topk_kernel<<<scratch.n_chunks, kRouteThreads, 0, stream>>>(logits, T, E, k, local.offset, local.count,
+                                                                       topk_ids, topk_w, scratch.chunk_counts);
+    route_scan_kernel<<<1, 256, 0, stream>>>(scratch.chunk_counts, scratch.n_chunks, local.count, nt_max, expert_offsets,
                                              scratch.tile_prefix, scratch.tile_order, scratch.tile_rows);
-    route_scatter_kernel<<<scratch.n_chunks, 32, 0, stream>>>(topk_ids, scratch.chunk_counts, expert_offsets, A, E, k,
-                                                              sorted_to_flat, flat_to_sorted);
+    route_scatter_kernel<<<scratch.n_chunks, 32, 0, stream>>>(topk_ids, scratch.chunk_counts, expert_offsets, A,
+                                                              local.count, local.offset, k, sorted_to_flat,
+                                                              flat_to_sorted);
     return cudaGetLastError();
 }
 
-cudaError_t launch_gather_rows(const __nv_bfloat16 *x, const int *sorted_to_flat, int A, int k, int H,
-                               __nv_bfloat16 *x_perm, cudaStream_t stream) {
-    gather_rows_kernel<<<(A + 7) / 8, 256, 0, stream>>>(reinterpret_cast<const uint4 *>(x), sorted_to_flat, A, k,
+cudaError_t launch_gather_rows(const __nv_bfloat16 *x, const int *sorted_to_flat, const int *n_rows, int A, int k,
+                               int H, __nv_bfloat16 *x_perm, cudaStream_t stream) {
+    gather_rows_kernel<<<(A + 7) / 8, 256, 0, stream>>>(reinterpret_cast<const uint4 *>(x), sorted_to_flat, n_rows, k,
                                                         H / 8, reinterpret_cast<uint4 *>(x_perm));
     return cudaGetLastError();
 }
@@ -353,8 +355,9 @@ extern "C" int moe_route_static(const float *router_logits, int T, int E, int to
     // The array keeps the previous call's contents.  The status word is cleared by launch_route; the
     // histogram and schedule regions are fully overwritten for this T and E before they are read.
     RouteScratch rs = carve_route_scratch(base + 256, T, E);
-    const cudaError_t err = launch_route(router_logits, T, E, top_k, 256, topk_ids, topk_weights, expert_offsets,
-                                         sorted_to_flat, flat_to_sorted, rs, reinterpret_cast<int *>(base), s);
+    const cudaError_t err = launch_route(router_logits, T, E, top_k, LocalExperts{0, E}, 256, topk_ids, topk_weights,
+                                         expert_offsets, sorted_to_flat, flat_to_sorted, rs,
+                                         reinterpret_cast<int *>(base), s);
     return err == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
 

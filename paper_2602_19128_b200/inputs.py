@@ -30,6 +30,13 @@ CONFIGS = {
     "skewed": dict(T=4096, H=4096, I=1536, E=128, top_k=8, skew=True),
 }
 
+# The paper's own deployment shape (Sec. 4.5: top-8 of 256 experts, 32 of them resident, hidden 7168), in
+# bf16: the router sees 256 experts, weights exist only for experts [local_offset, local_offset + local).
+LOCAL_CONFIGS = {
+    "dsv3_local32_prefill": dict(T=8192, H=7168, I=2048, E=256, top_k=8, skew=False, local_offset=64, local=32),
+    "dsv3_local32_decode": dict(T=128, H=7168, I=2048, E=256, top_k=8, skew=False, local_offset=64, local=32),
+}
+
 
 def zipf_bias(E: int) -> torch.Tensor:
     rank = torch.arange(1, E + 1, dtype=torch.float32)
@@ -54,7 +61,7 @@ def _normal_bf16(shape, std: float, gen: torch.Generator, device, chunk_elems: i
 def make_inputs(cfg, seed: int = 0, device="cpu") -> dict:
     """Draw one workload.  ``cfg`` is a name in CONFIGS or a dict with T,H,I,E,top_k[,skew]."""
     if isinstance(cfg, str):
-        cfg = CONFIGS[cfg]
+        cfg = CONFIGS[cfg] if cfg in CONFIGS else LOCAL_CONFIGS[cfg]
     T, H, I, E = cfg["T"], cfg["H"], cfg["I"], cfg["E"]
     device = torch.device(device)
     gen = torch.Generator(device=device)
@@ -63,9 +70,11 @@ def make_inputs(cfg, seed: int = 0, device="cpu") -> dict:
     logits = torch.randn((T, E), generator=gen, device=device, dtype=torch.float32)
     if cfg.get("skew", False):
         logits = logits + zipf_bias(E).to(device)
-    w13 = _normal_bf16((E, 2 * I, H), 1.0 / math.sqrt(H), gen, device)
-    w2 = _normal_bf16((E, H, I), 1.0 / math.sqrt(I), gen, device)
-    return dict(x=x, router_logits=logits.contiguous(), w13=w13, w2=w2, T=T, H=H, I=I, E=E, top_k=cfg["top_k"])
+    n_experts = cfg.get("local", E)  # weights are drawn only for the resident experts
+    w13 = _normal_bf16((n_experts, 2 * I, H), 1.0 / math.sqrt(H), gen, device)
+    w2 = _normal_bf16((n_experts, H, I), 1.0 / math.sqrt(I), gen, device)
+    return dict(x=x, router_logits=logits.contiguous(), w13=w13, w2=w2, T=T, H=H, I=I, E=E, top_k=cfg["top_k"],
+                local_offset=cfg.get("local_offset", 0), local=n_experts)
 
 
 def bf16_bits(t: torch.Tensor) -> np.ndarray:
