@@ -154,7 +154,8 @@ MOE_API int moe_route_static(const float *router_logits, int T, int E, int top_k
  *   workspace      at least moe_workspace_bytes(T,H,I,E,top_k) bytes, 256-byte aligned.  Holds the
  *                  routing arrays and intermediates at the offsets moe_workspace_layout() reports;
  *                  they stay valid until the next call that uses this workspace.
- * Launches seven kernels on `stream` and returns without waiting for them. */
+ * Launches five kernels (seven above 1024 tokens, where the router and sort-scatter take three) on
+ * `stream` and returns without waiting for them. */
 MOE_API int moe_forward(const void *x, const float *router_logits, const void *w13, const void *w2, int T, int H, int I,
                 int E, int top_k, void *out, void *workspace, size_t workspace_bytes, void *stream);
 
@@ -183,7 +184,7 @@ MOE_API int moe_forward_local(const void *x, const float *router_logits, const v
  * HOST array of MOE_NUM_STAGE_EVENTS cudaEvent_t handles (passed as void*, created by the caller with
  * timing enabled).  Event 0 is recorded on `stream` before the first kernel, and event i+1 after
  * stage i, where the stages are
- *   0 router + sort-scatter (3 kernels), 1 row gather, 2 gate/up GEMM + SwiGLU, 3 down GEMM, 4 combine.
+ *   0 router + sort-scatter (1 or 3 kernels), 1 row gather, 2 gate/up GEMM + SwiGLU, 3 down GEMM, 4 combine.
  * With T == 0 nothing is launched and no event is recorded. */
 #define MOE_NUM_STAGE_EVENTS 6
 MOE_API int moe_forward_staged(const void *x, const float *router_logits, const void *w13, const void *w2, int T, int H,

@@ -251,7 +251,9 @@ int moe_last_status(const void *workspace, void *stream) {
 
 int moe_forward_launch_count(int T, unsigned flags) {
     (void)flags;
-    return T > 0 ? 7 : 0;
+    if (T <= 0) return 0;
+    // router + sort-scatter: one fused kernel up to 1024 tokens, three kernels beyond; then gather, two GEMMs, combine
+    return (route_num_chunks(T) <= 32 ? 1 : 3) + 4;
 }
 
 const char *moe_status_string(int status) {

@@ -16,6 +16,7 @@ constexpr int kMaxExperts = 256;        // router keeps ceil(E/32) <= 8 logits p
 constexpr int kMaxTopK = 32;            // lane j of the token's warp owns rank j
 constexpr int kRouteTokensPerBlock = 32;  // tokens per router block = one histogram chunk
 constexpr int kStatusInts = 4;          // status word: {status, site, aux0, aux1}
+constexpr int kDoneCounterInt = 4;      // int index, in the status word's zeroed padding, of the fused router's block counter
 
 // Site ids recorded next to MOE_ERR_DEVICE_TIMEOUT (gate/up GEMM; the down GEMM adds 4).
 enum : int { kSiteProducerEmpty = 1, kSiteMmaFull = 2, kSiteMmaTmemEmpty = 3, kSiteEpilogueTmemFull = 4 };

@@ -25,86 +25,102 @@ constexpr unsigned kFullMask = 0xffffffffu;
 constexpr int kRouteThreads = 256;
 constexpr int kLogitsPerLane = kMaxExperts / 32;
 
-__global__ void __launch_bounds__(kRouteThreads)
-route_topk_kernel(const float *__restrict__ logits, int T, int E, int k, int local_offset, int n_local,
-                  int *__restrict__ topk_ids, float *__restrict__ topk_w, int *__restrict__ chunk_counts) {
-    __shared__ int hist[kMaxExperts];  // indexed by local expert (expert id - local_offset)
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    for (int e = tid; e < n_local; e += kRouteThreads) hist[e] = 0;
-    __syncthreads();
+// Router for one token by one warp: softmax over the E logits (8 per lane), k rounds of a warp arg-max
+// under the strict order, renormalisation.  Lane j < k returns rank j's expert and weight.
+__device__ __forceinline__ void route_one_token(const float *__restrict__ row, int E, int k, int lane, int &my_id,
+                                                float &my_w) {
+    float v[kLogitsPerLane], p[kLogitsPerLane];
+    float m = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < kLogitsPerLane; ++i) {
+        const int e = i * 32 + lane;
+        v[i] = e < E ? row[e] : -INFINITY;
+        m = fmaxf(m, v[i]);
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(kFullMask, m, off));
+    float s = 0.f;
+#pragma unroll
+    for (int i = 0; i < kLogitsPerLane; ++i) {
+        const int e = i * 32 + lane;
+        p[i] = e < E ? expf(v[i] - m) : 0.f;
+        s += p[i];
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(kFullMask, s, off);
+#pragma unroll
+    for (int i = 0; i < kLogitsPerLane; ++i) p[i] = p[i] / s;
 
+    unsigned taken = 0;
+    float my_p = 0.f;
+    my_id = 0;
+    for (int j = 0; j < k; ++j) {
+        // best candidate among this lane's experts that are still available
+        int ci = INT_MAX;
+        float cv = -INFINITY, cp = 0.f;
+#pragma unroll
+        for (int i = 0; i < kLogitsPerLane; ++i) {
+            const int e = i * 32 + lane;
+            if (e < E && !((taken >> i) & 1u) && (ci == INT_MAX || v[i] > cv)) {
+                ci = e; cv = v[i]; cp = p[i];
+            }
+        }
+        // warp arg-max; INT_MAX marks "no candidate" and always loses
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            const float ov = __shfl_xor_sync(kFullMask, cv, off);
+            const int oi = __shfl_xor_sync(kFullMask, ci, off);
+            const float op = __shfl_xor_sync(kFullMask, cp, off);
+            const bool other = (ci == INT_MAX) ? (oi != INT_MAX)
+                                               : (oi != INT_MAX && (ov > cv || (ov == cv && oi < ci)));
+            if (other) { cv = ov; ci = oi; cp = op; }
+        }
+        // with non-finite logits lanes could disagree; lane 0's answer is the warp's answer
+        ci = __shfl_sync(kFullMask, ci, 0);
+        cp = __shfl_sync(kFullMask, cp, 0);
+        if (ci == INT_MAX) ci = 0;  // unreachable for k <= E; keeps the index in range regardless
+        if ((ci & 31) == lane) taken |= 1u << (ci >> 5);
+        if (lane == j) { my_id = ci; my_p = cp; }
+    }
+    float denom = 0.f;  // ascending rank, the order the definition states
+    for (int j = 0; j < k; ++j) denom += __shfl_sync(kFullMask, my_p, j);
+    my_w = my_p / denom;
+}
+
+// Routes the block's 32 tokens (warp w takes tokens w, w + n_warps, ...), writes ids and weights, and
+// leaves the block's histogram over the resident experts in hist[].
+__device__ __forceinline__ void route_block_tokens(const float *__restrict__ logits, int T, int E, int k, int local_offset,
+                                                   int n_local, int *topk_ids, float *topk_w, int *hist) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, n_warps = blockDim.x >> 5;
+    for (int e = tid; e < n_local; e += blockDim.x) hist[e] = 0;
+    __syncthreads();
     const int t_base = blockIdx.x * kRouteTokensPerBlock;
-    for (int tt = warp; tt < kRouteTokensPerBlock; tt += kRouteThreads / 32) {
+    for (int tt = warp; tt < kRouteTokensPerBlock; tt += n_warps) {
         const int t = t_base + tt;
         if (t >= T) break;  // uniform over the warp
-        const float *row = logits + (size_t)t * E;
-        float v[kLogitsPerLane], p[kLogitsPerLane];
-        float m = -INFINITY;
-#pragma unroll
-        for (int i = 0; i < kLogitsPerLane; ++i) {
-            const int e = i * 32 + lane;
-            v[i] = e < E ? row[e] : -INFINITY;
-            m = fmaxf(m, v[i]);
-        }
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(kFullMask, m, off));
-        float s = 0.f;
-#pragma unroll
-        for (int i = 0; i < kLogitsPerLane; ++i) {
-            const int e = i * 32 + lane;
-            p[i] = e < E ? expf(v[i] - m) : 0.f;
-            s += p[i];
-        }
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(kFullMask, s, off);
-#pragma unroll
-        for (int i = 0; i < kLogitsPerLane; ++i) p[i] = p[i] / s;
-
-        unsigned taken = 0;
-        int my_id = 0;
-        float my_p = 0.f;
-        for (int j = 0; j < k; ++j) {
-            // best candidate among this lane's experts that are still available
-            int ci = INT_MAX;
-            float cv = -INFINITY, cp = 0.f;
-#pragma unroll
-            for (int i = 0; i < kLogitsPerLane; ++i) {
-                const int e = i * 32 + lane;
-                if (e < E && !((taken >> i) & 1u) && (ci == INT_MAX || v[i] > cv)) {
-                    ci = e; cv = v[i]; cp = p[i];
-                }
-            }
-            // warp arg-max; INT_MAX marks "no candidate" and always loses
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) {
-                const float ov = __shfl_xor_sync(kFullMask, cv, off);
-                const int oi = __shfl_xor_sync(kFullMask, ci, off);
-                const float op = __shfl_xor_sync(kFullMask, cp, off);
-                const bool other = (ci == INT_MAX) ? (oi != INT_MAX)
-                                                   : (oi != INT_MAX && (ov > cv || (ov == cv && oi < ci)));
-                if (other) { cv = ov; ci = oi; cp = op; }
-            }
-            // with non-finite logits lanes could disagree; lane 0's answer is the warp's answer
-            ci = __shfl_sync(kFullMask, ci, 0);
-            cp = __shfl_sync(kFullMask, cp, 0);
-            if (ci == INT_MAX) ci = 0;  // unreachable for k <= E; keeps the index in range regardless
-            if ((ci & 31) == lane) taken |= 1u << (ci >> 5);
-            if (lane == j) { my_id = ci; my_p = cp; }
-        }
-        float denom = 0.f;  // ascending rank, the order the definition states
-        for (int j = 0; j < k; ++j) denom += __shfl_sync(kFullMask, my_p, j);
+        int my_id;
+        float my_w;
+        route_one_token(logits + (size_t)t * E, E, k, lane, my_id, my_w);
         if (lane < k) {
             topk_ids[(size_t)t * k + lane] = my_id;
-            topk_w[(size_t)t * k + lane] = my_p / denom;
+            topk_w[(size_t)t * k + lane] = my_w;
             const int local = my_id - local_offset;  // only experts resident here are scheduled
             if (local >= 0 && local < n_local) atomicAdd(&hist[local], 1);
         }
     }
     __syncthreads();
-    for (int e = tid; e < n_local; e += kRouteThreads) chunk_counts[(size_t)blockIdx.x * n_local + e] = hist[e];
 }
 
-// Exclusive scan over the 256 threads of the block; returns the exclusive prefix, total in *total.
+__global__ void __launch_bounds__(kRouteThreads)
+route_topk_kernel(const float *__restrict__ logits, int T, int E, int k, int local_offset, int n_local,
+                  int *__restrict__ topk_ids, float *__restrict__ topk_w, int *__restrict__ chunk_counts) {
+    __shared__ int hist[kMaxExperts];  // indexed by local expert (expert id - local_offset)
+    route_block_tokens(logits, T, E, k, local_offset, n_local, topk_ids, topk_w, hist);
+    for (int e = threadIdx.x; e < n_local; e += kRouteThreads) chunk_counts[(size_t)blockIdx.x * n_local + e] = hist[e];
+}
+
+// Exclusive scan over threads 0..255 of the block (wider blocks may call it; their other threads pass 0
+// and ignore the result); returns the exclusive prefix, total in *total.
 __device__ __forceinline__ int block_exclusive_scan_256(int value, int *warp_sums, int *total) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     int incl = value;
@@ -113,7 +129,7 @@ __device__ __forceinline__ int block_exclusive_scan_256(int value, int *warp_sum
         const int n = __shfl_up_sync(kFullMask, incl, off);
         if (lane >= off) incl += n;
     }
-    if (lane == 31) warp_sums[warp] = incl;
+    if (lane == 31 && warp < 8) warp_sums[warp] = incl;
     __syncthreads();
     int base = 0, sum = 0;
 #pragma unroll
@@ -127,12 +143,15 @@ __device__ __forceinline__ int block_exclusive_scan_256(int value, int *warp_sum
     return base + incl - value;
 }
 
-__global__ void __launch_bounds__(256)
-route_scan_kernel(int *__restrict__ chunk_counts, int n_chunks, int E, int nt_max, int *__restrict__ expert_offsets,
-                  int *__restrict__ tile_prefix, int *__restrict__ tile_order, int *__restrict__ tile_rows) {
-    __shared__ int warp_sums[8];
-    __shared__ int counts[kMaxExperts], tiles_at[kMaxExperts];
+// Scan phase, run by one block (threads 0..255 carry one expert each; wider blocks idle the rest):
+// per-expert running sum over chunks, exclusive scan over experts, token-tile schedule.
+// (Pointers are deliberately not __restrict__ and cross-block data is read with __ldcg: in the fused
+// kernel these arrays were written by other blocks, or are written here and read again by the scatter.)
+__device__ __forceinline__ void scan_phase(int *chunk_counts, int n_chunks, int E, int nt_max, int *expert_offsets,
+                                           int *tile_prefix, int *tile_order, int *tile_rows, int *warp_sums,
+                                           int *counts, int *tiles_at) {
     const int e = threadIdx.x;
+    const bool lane_of_scan = e < kMaxExperts;
     int count = 0;
     if (e < E) {
         // running sum over chunks, 16 independent loads in flight at a time (the loop is latency-bound)
@@ -140,7 +159,7 @@ route_scan_kernel(int *__restrict__ chunk_counts, int n_chunks, int E, int nt_ma
         for (int b0 = 0; b0 < n_chunks; b0 += kBatch) {
             int c[kBatch];
 #pragma unroll
-            for (int i = 0; i < kBatch; ++i) c[i] = b0 + i < n_chunks ? chunk_counts[(size_t)(b0 + i) * E + e] : 0;
+            for (int i = 0; i < kBatch; ++i) c[i] = b0 + i < n_chunks ? __ldcg(&chunk_counts[(size_t)(b0 + i) * E + e]) : 0;
 #pragma unroll
             for (int i = 0; i < kBatch; ++i) {
                 if (b0 + i < n_chunks) chunk_counts[(size_t)(b0 + i) * E + e] = count;
@@ -148,8 +167,10 @@ route_scan_kernel(int *__restrict__ chunk_counts, int n_chunks, int E, int nt_ma
             }
         }
     }
-    counts[e] = e < E ? count : -1;
-    tiles_at[e] = 0;
+    if (lane_of_scan) {
+        counts[e] = e < E ? count : -1;
+        tiles_at[e] = 0;
+    }
     // token tiles of this expert: as few as fit under nt_max, evenly sized, rounded up to 16 rows
     int n_tiles = 0, rows = 0;
     if (count > 0) {
@@ -160,14 +181,14 @@ route_scan_kernel(int *__restrict__ chunk_counts, int n_chunks, int E, int nt_ma
     const int row_start = block_exclusive_scan_256(count, warp_sums, &total_rows);  // (syncs: counts[] is visible)
     // Schedule order: experts with more rows first (ties to the lower index), so that tiles of similar
     // cost are adjacent and the GEMMs' static tile assignment stays balanced; the small tiles come last.
-    int pos = 0;
     if (e < E) {
+        int pos = 0;
         for (int o = 0; o < E; ++o) pos += (counts[o] > count || (counts[o] == count && o < e)) ? 1 : 0;
         tiles_at[pos] = n_tiles;
         tile_order[pos] = e;
     }
     __syncthreads();
-    const int tile_start = block_exclusive_scan_256(tiles_at[e], warp_sums, &total_tiles);
+    const int tile_start = block_exclusive_scan_256(lane_of_scan ? tiles_at[e] : 0, warp_sums, &total_tiles);
     if (e < E) {
         expert_offsets[e] = row_start;
         tile_prefix[e] = tile_start;  // indexed by schedule position
@@ -179,21 +200,29 @@ route_scan_kernel(int *__restrict__ chunk_counts, int n_chunks, int E, int nt_ma
     }
 }
 
-__global__ void __launch_bounds__(32)
-route_scatter_kernel(const int *__restrict__ topk_ids, const int *__restrict__ chunk_starts,
-                     const int *__restrict__ expert_offsets, int A, int n_local, int local_offset, int k,
-                     int *__restrict__ sorted_to_flat, int *__restrict__ flat_to_sorted) {
-    __shared__ int next[kMaxExperts];
-    const int lane = threadIdx.x;
+__global__ void __launch_bounds__(256)
+route_scan_kernel(int *chunk_counts, int n_chunks, int E, int nt_max, int *expert_offsets, int *tile_prefix,
+                  int *tile_order, int *tile_rows) {
+    __shared__ int warp_sums[8];
+    __shared__ int counts[kMaxExperts], tiles_at[kMaxExperts];
+    scan_phase(chunk_counts, n_chunks, E, nt_max, expert_offsets, tile_prefix, tile_order, tile_rows, warp_sums, counts,
+               tiles_at);
+}
+
+// Stable scatter of one chunk (32 tokens) by one warp; next[] is that warp's per-expert cursor.
+__device__ __forceinline__ void scatter_chunk(int chunk, const int *topk_ids, const int *chunk_starts,
+                                              const int *expert_offsets, int A, int n_local, int local_offset, int k,
+                                              int *sorted_to_flat, int *flat_to_sorted, int *next, int lane) {
     // first position of this chunk's assignments to expert e = segment start + rows of earlier chunks
-    for (int e = lane; e < n_local; e += 32) next[e] = expert_offsets[e] + chunk_starts[(size_t)blockIdx.x * n_local + e];
+    for (int e = lane; e < n_local; e += 32)
+        next[e] = __ldcg(&expert_offsets[e]) + __ldcg(&chunk_starts[(size_t)chunk * n_local + e]);
     __syncwarp();
-    const int a0 = blockIdx.x * kRouteTokensPerBlock * k;
+    const int a0 = chunk * kRouteTokensPerBlock * k;
     const int a1 = min(A, a0 + kRouteTokensPerBlock * k);
     for (int base = a0; base < a1; base += 32) {
         const int a = base + lane;
         const bool valid = a < a1;
-        const int e = valid ? topk_ids[a] - local_offset : -1;
+        const int e = valid ? __ldcg(&topk_ids[a]) - local_offset : -1;
         const bool kept = e >= 0 && e < n_local;       // assignments to experts that are not resident are dropped
         const int key = kept ? e : -1 - lane;          // ... and never match anything
         const unsigned same = __match_any_sync(kFullMask, key);
@@ -205,6 +234,47 @@ route_scatter_kernel(const int *__restrict__ topk_ids, const int *__restrict__ c
         if (valid) flat_to_sorted[a] = pos;
         if (kept) sorted_to_flat[pos] = a;
     }
+}
+
+__global__ void __launch_bounds__(32)
+route_scatter_kernel(const int *topk_ids, const int *chunk_starts, const int *expert_offsets, int A, int n_local,
+                     int local_offset, int k, int *sorted_to_flat, int *flat_to_sorted) {
+    __shared__ int next[kMaxExperts];
+    scatter_chunk(blockIdx.x, topk_ids, chunk_starts, expert_offsets, A, n_local, local_offset, k, sorted_to_flat,
+                  flat_to_sorted, next, threadIdx.x);
+}
+
+// Small batches (at most kFusedMaxChunks chunks = 1024 tokens): the three phases in ONE launch.  Every
+// block routes its 32 tokens with one warp per token; the block that finishes last (a counter in the
+// status word's padding, zeroed by the caller's memset) then runs the scan phase and scatters every
+// chunk, one warp per chunk.  Which block is last does not affect any result.
+constexpr int kFusedThreads = 1024;
+constexpr int kFusedMaxChunks = kFusedThreads / 32;
+
+__global__ void __launch_bounds__(kFusedThreads)
+route_fused_kernel(const float *__restrict__ logits, int T, int E, int k, int local_offset, int n_local, int nt_max,
+                   int *topk_ids, float *topk_w, int *chunk_counts, int *expert_offsets, int *tile_prefix,
+                   int *tile_order, int *tile_rows, int *sorted_to_flat, int *flat_to_sorted, int *done_counter) {
+    __shared__ int hist[kMaxExperts], counts[kMaxExperts], tiles_at[kMaxExperts], warp_sums[8];
+    __shared__ int next[kFusedMaxChunks][kMaxExperts];
+    __shared__ int is_last;
+    const int tid = threadIdx.x;
+    route_block_tokens(logits, T, E, k, local_offset, n_local, topk_ids, topk_w, hist);
+    for (int e = tid; e < n_local; e += kFusedThreads) chunk_counts[(size_t)blockIdx.x * n_local + e] = hist[e];
+    __threadfence();  // this block's ids, weights and histogram are visible before it is counted as done
+    __syncthreads();
+    if (tid == 0) is_last = atomicAdd(done_counter, 1) == (int)gridDim.x - 1;
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    const int n_chunks = gridDim.x;
+    scan_phase(chunk_counts, n_chunks, n_local, nt_max, expert_offsets, tile_prefix, tile_order, tile_rows, warp_sums,
+               counts, tiles_at);
+    __syncthreads();  // expert_offsets and the chunk starts written above are read below (same block)
+    const int warp = tid >> 5;
+    if (warp < n_chunks)
+        scatter_chunk(warp, topk_ids, chunk_counts, expert_offsets, T * k, n_local, local_offset, k, sorted_to_flat,
+                      flat_to_sorted, next[warp], tid & 31);
 }
 
 __global__ void __launch_bounds__(256)
@@ -275,6 +345,13 @@ cudaError_t launch_route(const float *logits, int T, int E, int k, LocalExperts 
     cudaError_t err = cudaMemsetAsync(status, 0, 256, stream);  // the status word and its padding
     if (err != cudaSuccess) return err;
     const int A = T * k;
+    if (scratch.n_chunks <= kFusedMaxChunks) {
+        route_fused_kernel<<<scratch.n_chunks, kFusedThreads, 0, stream>>>(
+            logits, T, E, k, local.offset, local.count, nt_max, topk_ids, topk_w, scratch.chunk_counts, expert_offsets,
+            scratch.tile_prefix, scratch.tile_order, scratch.tile_rows, sorted_to_flat, flat_to_sorted,
+            status + kDoneCounterInt);
+        return cudaGetLastError();
+    }
     route_topk_kernel<<<scratch.n_chunks, kRouteThreads, 0, stream>>>(logits, T, E, k, local.offset, local.count,
                                                                        topk_ids, topk_w, scratch.chunk_counts);
     route_scan_kernel<<<1, 256, 0, stream>>>(scratch.chunk_counts, scratch.n_chunks, local.count, nt_max, expert_offsets,

@@ -48,4 +48,5 @@ def test_status_strings_and_launch_count():
     assert moe.moe_status_string(0) == "ok"
     assert "wait" in moe.moe_status_string(-7)
     assert moe.moe_status_string(-99) == "unknown status"
-    assert moe.moe_forward_launch_count(0) == 0 and moe.moe_forward_launch_count(16) == 7
+    assert moe.moe_forward_launch_count(0) == 0 and moe.moe_forward_launch_count(16) == 5
+    assert moe.moe_forward_launch_count(1024) == 5 and moe.moe_forward_launch_count(1025) == 7
