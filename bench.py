@@ -40,7 +40,7 @@ L2_BYTES = 126 * 1024 * 1024
 BOUND = {"tiny": "hbm", "mixtral": "hbm", "dsv3_decode": "hbm", "dsv3_prefill": "tensor", "skewed": "tensor",
          "dsv3_local32_prefill": "hbm", "dsv3_local32_decode": "hbm"}
 # DRAM bytes (read + write) of one gate/up GEMM launch, from the ncu capture summarised under profiles/.
-NCU_TRAFFIC_BYTES = {"mixtral": 1929712128}
+NCU_TRAFFIC_BYTES = {"mixtral": 1928438528}
 
 
 def load_peaks() -> dict:
@@ -173,7 +173,7 @@ def run_reference(args):
     from oracle import moe_oracle
     cfg = CONFIGS[args.config]
     dev = "cuda" if torch.cuda.is_available() else "cpu"
-    inp = make_inputs(args.config, seed=args.seed, device=dev)
+    inp = make_inputs(CONFIGS[args.config], seed=args.seed, device=dev)
     cores = moe_oracle.get("f32").num_threads
     o, x, logits, experts, I, k, tokens = oracle_sample(args.config, inp, cores)
     del inp
@@ -210,7 +210,7 @@ def run_ours(args):
     dev = torch.device("cuda", local)
     cfg = CONFIGS[args.config]
     T, H, I, E, k = (cfg[n] for n in ("T", "H", "I", "E", "top_k"))
-    inp = make_inputs(args.config, seed=args.seed + rank, device=dev)
+    inp = make_inputs(CONFIGS[args.config], seed=args.seed + rank, device=dev)
     x, logits, w13, w2 = inp["x"], inp["router_logits"], inp["w13"], inp["w2"]
     local_offset, n_local = inp["local_offset"], inp["local"]
     out = torch.empty((T, H), dtype=torch.bfloat16, device=dev)
