@@ -355,3 +355,83 @@ int moe_oracle_sorted_intermediates(const uint16_t *x, const uint16_t *w13, cons
     }
     return ORACLE_OK;
 }
+
+/* ---- FP8 block-scaled weights -------------------------------------------------------------------
+ * The paper's workload stores the expert weights in FP8 ("FP8 MoE", Table 2; Sec. 4.5), and its kernel
+ * feeds 16-bit tensor-core tiles, so the stored weights are converted and rescaled on the way in.  The
+ * build's reading of the storage format: OCP E4M3 codes (1 sign, 4 exponent bits with bias 7, 3 mantissa
+ * bits; no infinities, S.1111.111 is NaN) with one fp32 scale per 128 x 128 block of each expert's weight
+ * matrix; the weight a code stands for is  decode(code) * scale[row / 128][col / 128].  Activations stay
+ * bf16.  Everything else (router, sort-scatter, SwiGLU, combine) is unchanged. */
+static inline REAL e4m3_decode(uint8_t b) {
+    const int sign = b >> 7, e = (b >> 3) & 15, m = b & 7;
+    REAL v;
+    if (e == 15 && m == 7) v = (REAL)NAN;
+    else if (e == 0) v = (REAL)m / (REAL)8 * (REAL)0.015625;                 /* subnormal: m/8 * 2^-6 */
+    else v = ((REAL)1 + (REAL)m / (REAL)8) * (REAL)ldexp(1.0, e - 7);        /* (1 + m/8) * 2^(e-7) */
+    return sign ? -v : v;
+}
+
+float moe_oracle_e4m3_decode(uint8_t code) { return (float)e4m3_decode(code); }
+
+/* One expert with FP8 block-scaled weights applied to one token row.
+ *   w13q_e [2I,H] codes, w13s_e [2I/128, H/128] scales; w2q_e [H,I] codes, w2s_e [H/128, I/128] scales. */
+static void expert_ffn_row_fp8w(const uint16_t *x_row, const uint8_t *w13q_e, const float *w13s_e, const uint8_t *w2q_e,
+                                const float *w2s_e, int H, int I, REAL *y, REAL *s) {
+    const int hb = H / 128, ib = I / 128;
+    for (int i = 0; i < I; ++i) {
+        REAL g = 0, u = 0;
+        for (int h = 0; h < H; ++h) {
+            const REAL xv = bf16_to_real(x_row[h]);
+            const REAL wg = e4m3_decode(w13q_e[(size_t)i * H + h]) * (REAL)w13s_e[(size_t)(i / 128) * hb + h / 128];
+            const REAL wu = e4m3_decode(w13q_e[(size_t)(I + i) * H + h]) * (REAL)w13s_e[(size_t)((I + i) / 128) * hb + h / 128];
+            g += xv * wg;
+            u += xv * wu;
+        }
+        s[i] = g / ((REAL)1 + real_exp(-g)) * u;
+    }
+    for (int n = 0; n < H; ++n) {
+        REAL acc = 0;
+        for (int i = 0; i < I; ++i)
+            acc += s[i] * (e4m3_decode(w2q_e[(size_t)n * I + i]) * (REAL)w2s_e[(size_t)(n / 128) * ib + i / 128]);
+        y[n] = acc;
+    }
+}
+
+/* The whole layer with FP8 block-scaled weights: w13_q [E,2I,H] codes, w13_scale [E,2I/128,H/128] f32,
+ * w2_q [E,H,I] codes, w2_scale [E,H/128,I/128] f32 -> out [T,H] REAL.  H and I must be multiples of 128. */
+int moe_oracle_forward_fp8w(const uint16_t *x, const float *router_logits, const uint8_t *w13_q, const float *w13_scale,
+                            const uint8_t *w2_q, const float *w2_scale, int T, int H, int I, int E, int k, REAL *out) {
+    if (T < 0 || H < 128 || I < 128 || H % 128 || I % 128 || E < 1 || k < 1 || k > E) return ORACLE_ERR_ARG;
+    int status = ORACLE_OK;
+    const size_t n13 = (size_t)2 * I * H, n2 = (size_t)H * I;
+    const size_t s13 = (size_t)(2 * I / 128) * (H / 128), s2 = (size_t)(H / 128) * (I / 128);
+#pragma omp parallel
+    {
+        REAL *p = (REAL *)malloc(sizeof(REAL) * (size_t)E);
+        unsigned char *taken = (unsigned char *)malloc((size_t)E);
+        int32_t *ids = (int32_t *)malloc(sizeof(int32_t) * (size_t)k);
+        REAL *w = (REAL *)malloc(sizeof(REAL) * (size_t)k);
+        REAL *s = (REAL *)malloc(sizeof(REAL) * (size_t)I);
+        REAL *y = (REAL *)malloc(sizeof(REAL) * (size_t)H);
+        if (!p || !taken || !ids || !w || !s || !y) {
+#pragma omp critical
+            status = ORACLE_ERR_NOMEM;
+        } else {
+#pragma omp for schedule(dynamic, 1)
+            for (int t = 0; t < T; ++t) {
+                REAL *o = out + (size_t)t * H;
+                for (int n = 0; n < H; ++n) o[n] = 0;
+                route_token(router_logits + (size_t)t * E, E, k, ids, w, p, taken);
+                for (int j = 0; j < k; ++j) {
+                    const int e = ids[j];
+                    expert_ffn_row_fp8w(x + (size_t)t * H, w13_q + e * n13, w13_scale + e * s13, w2_q + e * n2,
+                                        w2_scale + e * s2, H, I, y, s);
+                    for (int n = 0; n < H; ++n) o[n] += w[j] * y[n];
+                }
+            }
+        }
+        free(p); free(taken); free(ids); free(w); free(s); free(y);
+    }
+    return status;
+}

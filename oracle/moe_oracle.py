@@ -51,8 +51,10 @@ class Oracle:
         assert self.lib.moe_oracle_real_bytes() == np.dtype(self.real).itemsize
         for fn in ("moe_oracle_route", "moe_oracle_permute", "moe_oracle_expert_ffn", "moe_oracle_forward",
                    "moe_oracle_forward_sampled", "moe_oracle_sorted_intermediates", "moe_oracle_forward_local",
-                   "moe_oracle_permute_local"):
+                   "moe_oracle_permute_local", "moe_oracle_forward_fp8w"):
             getattr(self.lib, fn).restype = ctypes.c_int
+        self.lib.moe_oracle_e4m3_decode.restype = ctypes.c_float
+        self.lib.moe_oracle_e4m3_decode.argtypes = [ctypes.c_uint8]
 
     # -- helpers ---------------------------------------------------------------------------
     @staticmethod
@@ -161,6 +163,28 @@ class Oracle:
         self._check(self.lib.moe_oracle_permute_local(self._ptr(ids), T, k, local_offset, n_local, self._ptr(offsets),
                                                       self._ptr(s2f), self._ptr(f2s)), "permute_local")
         return offsets, s2f, f2s
+
+    def e4m3_decode(self, code: int) -> float:
+        return float(self.lib.moe_oracle_e4m3_decode(int(code) & 0xFF))
+
+    def forward_fp8w(self, x, router_logits, w13_q, w13_scale, w2_q, w2_scale, top_k: int):
+        """The layer with FP8 (E4M3) weights and one fp32 scale per 128 x 128 block."""
+        x = self._u16(x)
+        l = np.ascontiguousarray(router_logits, dtype=np.float32)
+        w13_q = np.ascontiguousarray(w13_q, dtype=np.uint8)
+        w2_q = np.ascontiguousarray(w2_q, dtype=np.uint8)
+        w13_scale = np.ascontiguousarray(w13_scale, dtype=np.float32)
+        w2_scale = np.ascontiguousarray(w2_scale, dtype=np.float32)
+        T, H = x.shape
+        E, I2, _ = w13_q.shape
+        I = I2 // 2
+        assert w13_q.shape == (E, 2 * I, H) and w2_q.shape == (E, H, I) and l.shape == (T, E)
+        assert w13_scale.shape == (E, 2 * I // 128, H // 128) and w2_scale.shape == (E, H // 128, I // 128)
+        out = np.empty((T, H), self.real)
+        self._check(self.lib.moe_oracle_forward_fp8w(self._ptr(x), self._ptr(l), self._ptr(w13_q), self._ptr(w13_scale),
+                                                     self._ptr(w2_q), self._ptr(w2_scale), T, H, I, E, top_k,
+                                                     self._ptr(out)), "forward_fp8w")
+        return out
 
     def sorted_intermediates(self, x, w13, w2, topk_ids, sorted_to_flat):
         x, w13, w2 = self._u16(x), self._u16(w13), self._u16(w2)

@@ -77,6 +77,37 @@ def make_inputs(cfg, seed: int = 0, device="cpu") -> dict:
                 local_offset=cfg.get("local_offset", 0), local=n_experts)
 
 
+FP8_BLOCK = 128
+E4M3_MAX = 448.0
+
+
+def quantize_fp8_blocks(w: torch.Tensor):
+    """Offline weight quantisation for the FP8 workloads: every 128 x 128 block of each expert's matrix
+    [E, rows, cols] gets the fp32 scale amax / 448 (1 for an all-zero block) and its entries are rounded to
+    E4M3 after division by it (torch's float8_e4m3fn conversion).  Returns (codes uint8 [E,rows,cols],
+    scales f32 [E, rows/128, cols/128]).  This prepares inputs; the layer's own arithmetic starts from them."""
+    E, R, C = w.shape
+    assert R % FP8_BLOCK == 0 and C % FP8_BLOCK == 0
+    codes = torch.empty((E, R, C), dtype=torch.uint8, device=w.device)
+    scales = torch.empty((E, R // FP8_BLOCK, C // FP8_BLOCK), dtype=torch.float32, device=w.device)
+    for e in range(E):  # one expert at a time keeps the fp32 temporaries small
+        blocks = w[e].float().view(R // FP8_BLOCK, FP8_BLOCK, C // FP8_BLOCK, FP8_BLOCK)
+        amax = blocks.abs().amax(dim=(1, 3))
+        scale = torch.where(amax > 0, amax / E4M3_MAX, torch.ones_like(amax))
+        q = (blocks / scale[:, None, :, None]).to(torch.float8_e4m3fn)
+        codes[e] = q.view(torch.uint8).view(R, C)
+        scales[e] = scale
+    return codes, scales
+
+
+def make_fp8w_inputs(cfg, seed: int = 0, device="cpu") -> dict:
+    """make_inputs plus the FP8 block-scaled form of the expert weights (w13_q, w13_scale, w2_q, w2_scale)."""
+    inp = make_inputs(cfg, seed=seed, device=device)
+    inp["w13_q"], inp["w13_scale"] = quantize_fp8_blocks(inp["w13"])
+    inp["w2_q"], inp["w2_scale"] = quantize_fp8_blocks(inp["w2"])
+    return inp
+
+
 def bf16_bits(t: torch.Tensor) -> np.ndarray:
     """The uint16 bit pattern of a bf16 tensor, on the host, as a numpy array."""
     assert t.dtype == torch.bfloat16
