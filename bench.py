@@ -28,7 +28,8 @@ import torch
 ROOT = Path(__file__).resolve().parent
 sys.path.insert(0, str(ROOT))
 
-from paper_2602_19128_b200.inputs import CONFIGS, LOCAL_CONFIGS, bf16_bits, make_inputs  # noqa: E402
+from paper_2602_19128_b200.inputs import (CONFIGS, LOCAL_CONFIGS, bf16_bits, make_inputs,  # noqa: E402
+                                          quantize_fp8_blocks)
 
 CONFIGS = dict(CONFIGS, **LOCAL_CONFIGS)  # the five workloads plus the local-expert-subset shapes
 
@@ -215,8 +216,24 @@ def run_ours(args):
     local_offset, n_local = inp["local_offset"], inp["local"]
     out = torch.empty((T, H), dtype=torch.bfloat16, device=dev)
     ws = moe.alloc_workspace(moe.moe_workspace_bytes(T, H, I, E, k), dev)
-    weight_bytes = (w13.numel() + w2.numel()) * 2
+    fp8 = args.weights == "fp8"
+    if fp8:  # FP8 (E4M3) codes + one fp32 scale per 128 x 128 block; the bf16 originals are dropped
+        if n_local != E:
+            raise SystemExit("--weights fp8 covers the whole-layer workloads")
+        w13, w13_scale = quantize_fp8_blocks(w13)
+        w2, w2_scale = quantize_fp8_blocks(w2)
+        inp["w13"], inp["w2"] = None, None
+    bytes_per_weight = 1 if fp8 else 2
+    weight_bytes = (w13.numel() + w2.numel()) * bytes_per_weight
     need_flush = weight_bytes < 2 * L2_BYTES
+
+    def forward(events=None):
+        if fp8:
+            moe.moe_forward_fp8w(x, logits, w13, w13_scale, w2, w2_scale, k, out, ws, stage_events=events)
+        elif events is None:
+            moe.moe_forward_local(x, logits, w13, w2, k, local_offset, out, ws)
+        else:
+            moe.moe_forward_staged(x, logits, w13, w2, k, out, ws, events, local_expert_offset=local_offset)
     flush_buf = torch.zeros(2 * L2_BYTES // 4, dtype=torch.float32, device=dev) if need_flush else None
     stream = torch.cuda.current_stream()
 
@@ -228,7 +245,7 @@ def run_ours(args):
 
     # ---- device-resident timing ----------------------------------------------------------------
     for _ in range(max(args.warmup, 3)):
-        moe.moe_forward_local(x, logits, w13, w2, k, local_offset, out, ws)
+        forward()
     status = moe.moe_last_status(ws)
     if status != moe.MOE_OK:
         raise SystemExit(f"device status {status}: {moe.moe_status_string(status)}")
@@ -238,7 +255,7 @@ def run_ours(args):
     for s in range(args.steps):
         if need_flush:
             flush_l2(flush_buf)
-        moe.moe_forward_staged(x, logits, w13, w2, k, out, ws, stage_events[s], local_expert_offset=local_offset)
+        forward(stage_events[s])
     barrier()
     clocks = sampler.stop() if sampler else None
     if need_flush:
@@ -261,8 +278,19 @@ def run_ours(args):
     xh = x.cpu().pin_memory()
     lh = logits.cpu().pin_memory()
     oh = torch.empty((T, H), dtype=torch.bfloat16).pin_memory()
+    x_stage, l_stage = torch.empty_like(x), torch.empty_like(logits)
+
+    def host_step():
+        if fp8:  # no host-buffer entry point for FP8 weights: the same copies, issued here on the same stream
+            x_stage.copy_(xh, non_blocking=True)
+            l_stage.copy_(lh, non_blocking=True)
+            moe.moe_forward_fp8w(x_stage, l_stage, w13, w13_scale, w2, w2_scale, k, out, ws)
+            oh.copy_(out, non_blocking=True)
+        else:
+            moe.moe_forward_host(xh, lh, w13, w2, k, oh, ws, local_expert_offset=local_offset)
+
     for _ in range(3):
-        moe.moe_forward_host(xh, lh, w13, w2, k, oh, ws, local_expert_offset=local_offset)
+        host_step()
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e2e_ms = 0.0
@@ -270,14 +298,14 @@ def run_ours(args):
         for _ in range(args.steps):
             flush_l2(flush_buf)
             e0.record()
-            moe.moe_forward_host(xh, lh, w13, w2, k, oh, ws, local_expert_offset=local_offset)
+            host_step()
             e1.record()
             e1.synchronize()
             e2e_ms += e0.elapsed_time(e1)
     else:
         e0.record()
         for _ in range(args.steps):
-            moe.moe_forward_host(xh, lh, w13, w2, k, oh, ws, local_expert_offset=local_offset)
+            host_step()
         e1.record()
         e1.synchronize()
         e2e_ms = e0.elapsed_time(e1)
@@ -296,7 +324,7 @@ def run_ours(args):
     t_gemm1 = stage_ms["gemm1_swiglu"] * 1e-3
     bound = BOUND[args.config]
     if bound == "hbm":
-        algorithmic = n_active * 2 * I * H * 2  # bytes of the active experts' w13, read once
+        algorithmic = n_active * 2 * I * H * bytes_per_weight  # bytes of the active experts' w13, read once
         achieved = algorithmic / t_gemm1 / 1e9
         peak, unit = peaks["hbm_gbs"], "GB/s"
     else:
@@ -304,10 +332,10 @@ def run_ours(args):
         achieved = algorithmic / t_gemm1 / 1e12
         peak, unit = peaks["tflops_sustained"], "TFLOP/s"
     step_s = total_ms * 1e-3 / args.steps
-    active_weight_bytes = n_active * 3 * I * H * 2
-    roofline = dict(bound=bound, kernel="grouped_gemm_tc_kernel<swiglu> (gate/up GEMM)", achieved=achieved, peak=peak,
+    active_weight_bytes = n_active * 3 * I * H * bytes_per_weight
+    roofline = dict(bound=bound, kernel="gate/up GEMM (grouped_gemm_tc*_kernel<swiglu>)", achieved=achieved, peak=peak,
                     unit=unit, frac=achieved / peak, peak_source=f"of {peaks['source']}",
-                    traffic=NCU_TRAFFIC_BYTES.get(args.config), algorithmic_per_launch=algorithmic,
+                    traffic=None if fp8 else NCU_TRAFFIC_BYTES.get(args.config), algorithmic_per_launch=algorithmic,
                     kernel_ms=stage_ms["gemm1_swiglu"])
     layer = dict(stage_ms={n: round(v, 5) for n, v in stage_ms.items()}, n_active_experts=n_active,
                  rows_per_expert_min=int(counts.min()), rows_per_expert_max=int(counts.max()),
@@ -317,13 +345,14 @@ def run_ours(args):
                  useful_tflops_frac_burst=6.0 * A * H * I / step_s / 1e12 / peaks["tflops_burst"])
 
     cpu_baseline = None
-    if world == 1 and not args.no_cpu_baseline and n_local == E:
+    if world == 1 and not args.no_cpu_baseline and n_local == E and not fp8:
         cpu_baseline = time_oracle(args.config, inp, budget_s=15.0)
 
     line = dict(metric=METRIC, value=aggregate_tokens_per_s(world, T, args.steps, total_ms), unit=UNIT, n_gpus=world,
                 steps=args.steps, warmup=max(args.warmup, 3), ms_per_step=total_ms / args.steps, higher_is_better=True,
                 scaling="weak", vs_baseline=None, dtype="bf16", data="synthetic",
                 config=dict(workload=args.config, T=T, H=H, I=I, E=E, top_k=k, resident_experts=n_local,
+                            weights="fp8 e4m3 codes + fp32 scale per 128x128 block" if fp8 else "bf16",
                             parallelism=f"replicas x{world}",
                             l2="flushed between steps" if need_flush else "weights larger than L2, no flush",
                             seed=args.seed),
@@ -346,6 +375,8 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--config", choices=list(CONFIGS), default="mixtral")
     ap.add_argument("--shape", default=None, help="custom T,H,I,E,top_k instead of a named workload (profiling)")
+    ap.add_argument("--weights", choices=["bf16", "fp8"], default="bf16",
+                    help="fp8: expert weights as E4M3 codes with one fp32 scale per 128 x 128 block (moe_forward_fp8w)")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

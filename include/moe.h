@@ -179,6 +179,21 @@ MOE_API int moe_forward_local(const void *x, const float *router_logits, const v
                               int T, int H, int I, int E, int top_k, int local_expert_offset, int num_local_experts,
                               void *out, void *workspace, size_t workspace_bytes, void *stream, unsigned flags);
 
+/* The layer with FP8 block-scaled expert weights (the paper's workload is an "FP8 MoE", Table 2 and
+ * Sec. 4.5; its kernel converts the stored FP8 operands and multiplies 16-bit tensor-core tiles, which is
+ * what this entry point does on tcgen05): weights are OCP E4M3 codes, one byte each, with one fp32 scale
+ * per 128 x 128 block of every expert's matrix; a weight is decode(code) * scale[row/128][col/128].
+ * Activations, routing, intermediates and the result are as in moe_forward.
+ *   w13_q      [E,2I,H] uint8 E4M3 codes (rows [0,I) gate, [I,2I) up)   w13_scale [E, 2I/128, H/128] f32
+ *   w2_q       [E,H,I]  uint8 E4M3 codes                                w2_scale  [E, H/128,  I/128] f32
+ *   stage_events  NULL, or MOE_NUM_STAGE_EVENTS cudaEvent_t handles recorded as by moe_forward_staged.
+ * Needs I % 128 == 0 in addition to the usual envelope (MOE_ERR_UNSUPPORTED otherwise).  Codes are
+ * converted to bf16 and multiplied by the block scale rounded to bf16 (at most 2^-8 relative per weight);
+ * scales must be below 2^7 in magnitude; NaN codes are outside the contract. */
+MOE_API int moe_forward_fp8w(const void *x, const float *router_logits, const void *w13_q, const float *w13_scale,
+                             const void *w2_q, const float *w2_scale, int T, int H, int I, int E, int top_k, void *out,
+                             void *workspace, size_t workspace_bytes, void *stream, void *const *stage_events);
+
 /* moe_forward_local (pass local_expert_offset = 0, num_local_experts = E for the whole layer) that also
  * records CUDA events between the stages, for per-kernel timing inside a whole step.  stage_events is a
  * HOST array of MOE_NUM_STAGE_EVENTS cudaEvent_t handles (passed as void*, created by the caller with

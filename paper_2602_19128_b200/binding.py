@@ -21,7 +21,7 @@ MOE_FLAG_TWO_SLAB_GEMM = 4
 
 EXPORTED = ["moe_workspace_bytes", "moe_workspace_layout", "moe_route_workspace_bytes", "moe_route", "moe_route_static",
             "moe_forward",
-            "moe_forward_ex", "moe_forward_local", "moe_forward_staged", "moe_forward_host", "moe_last_status", "moe_forward_launch_count", "moe_status_string"]
+            "moe_forward_ex", "moe_forward_local", "moe_forward_fp8w", "moe_forward_staged", "moe_forward_host", "moe_last_status", "moe_forward_launch_count", "moe_status_string"]
 
 
 class MoeError(RuntimeError):
@@ -64,6 +64,8 @@ def lib() -> ctypes.CDLL:
         L.moe_forward_ex.argtypes = [vp, vp, vp, vp, i, i, i, i, i, vp, vp, sz, vp, ctypes.c_uint]
         L.moe_forward_local.restype = i
         L.moe_forward_local.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, vp, vp, sz, vp, ctypes.c_uint]
+        L.moe_forward_fp8w.restype = i
+        L.moe_forward_fp8w.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, vp, vp, sz, vp, ctypes.POINTER(vp)]
         L.moe_forward_staged.restype = i
         L.moe_forward_staged.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, vp, vp, sz, vp, ctypes.c_uint,
                                          ctypes.POINTER(vp)]
@@ -166,6 +168,22 @@ def moe_forward_local(x, router_logits, w13_local, w2_local, top_k: int, local_e
                                  _stream(stream), flags)
     if check and st != MOE_OK:
         raise MoeError(st, "moe_forward_local")
+    return st
+
+
+def moe_forward_fp8w(x, router_logits, w13_q, w13_scale, w2_q, w2_scale, top_k: int, out, workspace, stream=None,
+                     stage_events=None, check: bool = True) -> int:
+    """The layer with FP8 (E4M3, uint8 codes) weights and one fp32 scale per 128 x 128 block."""
+    T, H = x.shape
+    E, I2, _ = w13_q.shape
+    handles = None
+    if stage_events is not None:
+        handles = (ctypes.c_void_p * (len(STAGE_NAMES) + 1))(*[e.cuda_event for e in stage_events])
+    st = lib().moe_forward_fp8w(_ptr(x), _ptr(router_logits), _ptr(w13_q), _ptr(w13_scale), _ptr(w2_q), _ptr(w2_scale),
+                                T, H, I2 // 2, E, top_k, _ptr(out), _ptr(workspace), workspace.numel(), _stream(stream),
+                                handles)
+    if check and st != MOE_OK:
+        raise MoeError(st, "moe_forward_fp8w")
     return st
 
 

@@ -49,14 +49,17 @@ int check_device() {
 
 int forward_impl(const void *x, const float *logits, const void *w13, const void *w2, int T, int H, int I, int E, int k,
                  void *out, void *workspace, size_t workspace_bytes, cudaStream_t stream, unsigned flags,
-                 void *const *stage_events = nullptr, int local_offset = 0, int n_local = -1) {
+                 void *const *stage_events = nullptr, int local_offset = 0, int n_local = -1,
+                 const float *w13_scale = nullptr, const float *w2_scale = nullptr) {
     if (n_local < 0) n_local = E;  // every expert is resident
+    const bool fp8w = w13_scale != nullptr;  // w13 / w2 then hold E4M3 codes, one byte per weight
     if (T < 0 || H <= 0 || I <= 0 || E <= 0 || k <= 0 || k > E) return MOE_ERR_SHAPE;
     if (!envelope_ok(T, H, I, E, k)) return MOE_ERR_UNSUPPORTED;
     if (local_offset < 0 || n_local < 1 || (long long)local_offset + n_local > E) return MOE_ERR_SHAPE;
     if (flags & ~(MOE_FLAG_VALIDATION_GEMM | MOE_FLAG_SINGLE_CTA_GEMM | MOE_FLAG_TWO_SLAB_GEMM)) return MOE_ERR_UNSUPPORTED;
+    if (fp8w && (I % 128 != 0 || flags != MOE_FLAG_NONE)) return MOE_ERR_UNSUPPORTED;
     if (T == 0) return MOE_OK;
-    if (!x || !logits || !w13 || !w2 || !out || !workspace) return MOE_ERR_NULL;
+    if (!x || !logits || !w13 || !w2 || !out || !workspace || (fp8w && !w2_scale)) return MOE_ERR_NULL;
     if (!aligned(x, 16) || !aligned(logits, 16) || !aligned(w13, 16) || !aligned(w2, 16) || !aligned(out, 16) ||
         !aligned(workspace, 256))
         return MOE_ERR_ALIGN;
@@ -102,7 +105,15 @@ int forward_impl(const void *x, const float *logits, const void *w13, const void
     g2.act = h; g2.w = static_cast<const __nv_bfloat16 *>(w2); g2.out = y;
     g2.K = I; g2.n_out = H; g2.w_rows = H; g2.swiglu = false;
 
-    if (flags & MOE_FLAG_VALIDATION_GEMM) {
+    if (fp8w) {
+        g1.w_scale = w13_scale;
+        g2.w_scale = w2_scale;
+        int st = launch_grouped_gemm_tc_fp8w(g1, stream);
+        if (st != MOE_OK) return st;
+        if (!mark(3)) return MOE_ERR_CUDA;
+        st = launch_grouped_gemm_tc_fp8w(g2, stream);
+        if (st != MOE_OK) return st;
+    } else if (flags & MOE_FLAG_VALIDATION_GEMM) {
         if (launch_grouped_gemm_validation(g1, stream) != cudaSuccess) return MOE_ERR_CUDA;
         if (!mark(3)) return MOE_ERR_CUDA;
         if (launch_grouped_gemm_validation(g2, stream) != cudaSuccess) return MOE_ERR_CUDA;
@@ -200,6 +211,18 @@ int moe_forward_local(const void *x, const float *router_logits, const void *w13
     if (num_local_experts < 1) return MOE_ERR_SHAPE;
     return forward_impl(x, router_logits, w13_local, w2_local, T, H, I, E, top_k, out, workspace, workspace_bytes,
                         static_cast<cudaStream_t>(stream), flags, nullptr, local_expert_offset, num_local_experts);
+}
+
+int moe_forward_fp8w(const void *x, const float *router_logits, const void *w13_q, const float *w13_scale,
+                     const void *w2_q, const float *w2_scale, int T, int H, int I, int E, int top_k, void *out,
+                     void *workspace, size_t workspace_bytes, void *stream, void *const *stage_events) {
+    if (!w13_scale || !w2_scale) return MOE_ERR_NULL;
+    if (!aligned(w13_scale, 4) || !aligned(w2_scale, 4)) return MOE_ERR_ALIGN;
+    if (stage_events)
+        for (int i = 0; i < MOE_NUM_STAGE_EVENTS; ++i)
+            if (!stage_events[i]) return MOE_ERR_NULL;
+    return forward_impl(x, router_logits, w13_q, w2_q, T, H, I, E, top_k, out, workspace, workspace_bytes,
+                        static_cast<cudaStream_t>(stream), MOE_FLAG_NONE, stage_events, 0, -1, w13_scale, w2_scale);
 }
 
 int moe_forward_staged(const void *x, const float *router_logits, const void *w13, const void *w2, int T, int H, int I,

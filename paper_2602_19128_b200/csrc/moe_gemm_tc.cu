@@ -281,6 +281,7 @@ int launch_grouped_gemm_tc(const GroupedGemmArgs &a, cudaStream_t stream) {
     p.n_k_blocks = a.K / kBlockK;
     p.n_out = a.n_out;
     p.w_rows = a.w_rows;
+    p.w_scale = nullptr;
     p.n_feature_tiles = a.n_out / features_per_tile;
 
     // The tile count is only known on the device; this is its upper bound.

@@ -381,6 +381,7 @@ int launch_grouped_gemm_tc_pair(const GroupedGemmArgs &a, int slabs, cudaStream_
     p.n_k_blocks = a.K / kBlockK;
     p.n_out = a.n_out;
     p.w_rows = a.w_rows;
+    p.w_scale = nullptr;
     p.n_feature_tiles = a.n_out / features_per_pair_tile(a, slabs);
 
     const long long max_token_tiles = (long long)(a.A < a.E ? a.A : a.E) + a.A / a.nt_max;

@@ -87,6 +87,7 @@ struct GroupedGemmArgs {
     const int *tile_rows;      // [E]
     int *status;               // status word
     bool swiglu;
+    const float *w_scale = nullptr;  // FP8-weight GEMM: w points at E4M3 codes, this at [E, w_rows/128, K/128] scales
 };
 int launch_grouped_gemm_tc(const GroupedGemmArgs &args, cudaStream_t stream);  // returns a moe_status_t
 
@@ -96,6 +97,11 @@ int launch_grouped_gemm_tc(const GroupedGemmArgs &args, cudaStream_t stream);  /
 // feature count the pair tile does not divide).
 int grouped_gemm_tc_pair_slabs(const GroupedGemmArgs &args);
 int launch_grouped_gemm_tc_pair(const GroupedGemmArgs &args, int slabs, cudaStream_t stream);
+
+// The one-CTA kernel for FP8 (E4M3) block-scaled weights: args.w holds one code byte per weight and
+// args.w_scale one fp32 scale per 128 x 128 block; converter warps rebuild bf16 operand tiles in shared
+// memory and the bf16 tensor-core path does the rest.  Needs K % 128 == 0.
+int launch_grouped_gemm_tc_fp8w(const GroupedGemmArgs &args, cudaStream_t stream);
 
 // Same contract on plain CUDA cores (validation only).
 cudaError_t launch_grouped_gemm_validation(const GroupedGemmArgs &args, cudaStream_t stream);

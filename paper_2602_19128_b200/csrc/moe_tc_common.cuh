@@ -30,6 +30,7 @@ struct KernelParams {
     const int *expert_offsets, *tile_prefix, *tile_order, *tile_rows;
     int *status;
     int E, n_k_blocks, n_out, w_rows, n_feature_tiles;
+    const float *w_scale;  // FP8-weight kernels only: [E, w_rows/128, K/128] block scales
 };
 
 // ---- PTX wrappers -----------------------------------------------------------------------------
@@ -122,6 +123,12 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
         ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar)
         : "memory");
 }
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, int c0, int c1, int c2, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
+        : "memory");
+}
 __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap *map, int c0, int c1, int c2, int c3,
                                             int c4, uint32_t bar) {
     asm volatile(
@@ -211,6 +218,9 @@ __device__ __forceinline__ float swiglu(float g, float u) { return __fdividef(g,
 // ---- host side ----------------------------------------------------------------------------------
 bool encode_weight_map_2d(CUtensorMap *map, const void *w, uint64_t rows, uint64_t K);
 bool encode_weight_map_gate_up(CUtensorMap *map, const void *w13, int E, int I, int H);
+bool encode_weight_map_2d_fp8(CUtensorMap *map, const void *w, uint64_t rows, uint64_t K);
+bool encode_act_maps_k128(CUtensorMap *maps, const void *act, uint64_t rows, uint64_t K, int row_quantum);
+bool encode_weight_map_gate_up_fp8(CUtensorMap *map, const void *w13, int E, int I, int H);
 bool encode_act_maps(CUtensorMap *maps, const void *act, uint64_t rows, uint64_t K, int row_quantum);
 int sm_count();
 

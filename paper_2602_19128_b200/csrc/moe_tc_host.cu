@@ -27,12 +27,15 @@ EncodeTiledFn get_encode_fn() {
 }
 
 bool encode(CUtensorMap *map, const void *base, int rank, const cuuint64_t *dims, const cuuint64_t *strides,
-            const cuuint32_t *box) {
+            const cuuint32_t *box, bool fp8_codes = false) {
     EncodeTiledFn fn = get_encode_fn();
     if (!fn) return false;
     const cuuint32_t elem_strides[5] = {1, 1, 1, 1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void *>(base), dims, strides, box, elem_strides,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+    // bf16 operands land in the 128-byte-swizzled layout the MMA reads; FP8 codes are staged unswizzled
+    // (64-byte rows) for the converter warps
+    return fn(map, fp8_codes ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank,
+              const_cast<void *>(base), dims, strides, box, elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              fp8_codes ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -59,6 +62,36 @@ bool encode_weight_map_gate_up(CUtensorMap *map, const void *w13, int E, int I, 
     const cuuint64_t strides[4] = {row_bytes, (cuuint64_t)I * row_bytes, 16 * row_bytes, 2 * (cuuint64_t)I * row_bytes};
     const cuuint32_t box[5] = {(cuuint32_t)kBlockK, 16, 2, 4, 1};
     return encode(map, w13, 5, dims, strides, box);
+}
+
+// The same two weight maps over FP8 codes (one byte per element): [rows, K] with a 128-row x 64-byte box,
+// and the gate/up view [E][I/16][2][16][H] with the {64,16,2,4,1} box.
+// (FP8 slots are 128 K-elements wide: 128-byte rows of codes.)
+bool encode_weight_map_2d_fp8(CUtensorMap *map, const void *w, uint64_t rows, uint64_t K) {
+    const cuuint64_t dims[2] = {K, rows};
+    const cuuint64_t strides[1] = {K};
+    const cuuint32_t box[2] = {128, (cuuint32_t)kTileM};
+    return encode(map, w, 2, dims, strides, box, true);
+}
+
+bool encode_weight_map_gate_up_fp8(CUtensorMap *map, const void *w13, int E, int I, int H) {
+    const cuuint64_t row_bytes = (cuuint64_t)H;
+    const cuuint64_t dims[5] = {(cuuint64_t)H, 16, 2, (cuuint64_t)(I / 16), (cuuint64_t)E};
+    const cuuint64_t strides[4] = {row_bytes, (cuuint64_t)I * row_bytes, 16 * row_bytes, 2 * (cuuint64_t)I * row_bytes};
+    const cuuint32_t box[5] = {128, 16, 2, 4, 1};
+    return encode(map, w13, 5, dims, strides, box, true);
+}
+
+// Activation maps whose box spans 128 K-elements: the tensor [rows, K] viewed as [K/64][rows][64], box
+// {64, q*(i+1), 2}, so one copy delivers two consecutive 128-byte-swizzled tiles (K 0..63, then 64..127).
+bool encode_act_maps_k128(CUtensorMap *maps, const void *act, uint64_t rows, uint64_t K, int row_quantum) {
+    for (int i = 0; i < kNumActMaps; ++i) {
+        const cuuint64_t dims[3] = {(cuuint64_t)kBlockK, rows, K / kBlockK};
+        const cuuint64_t strides[2] = {K * 2, (cuuint64_t)kBlockK * 2};
+        const cuuint32_t box[3] = {(cuuint32_t)kBlockK, (cuuint32_t)row_quantum * (cuuint32_t)(i + 1), 2};
+        if (!encode(&maps[i], act, 3, dims, strides, box)) return false;
+    }
+    return true;
 }
 
 bool encode_act_maps(CUtensorMap *maps, const void *act, uint64_t rows, uint64_t K, int row_quantum) {

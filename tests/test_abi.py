@@ -12,7 +12,7 @@ ROOT = Path(__file__).resolve().parent.parent
 
 def declared_symbols():
     text = (ROOT / "include" / "moe.h").read_text()
-    return sorted(set(re.findall(r"MOE_API[^;(]*?\b(moe_[a-z_]+)\s*\(", text)))
+    return sorted(set(re.findall(r"MOE_API[^;(]*?\b(moe_[a-z0-9_]+)\s*\(", text)))
 
 
 def test_library_builds_loads_and_exports_every_declared_symbol():
