@@ -120,3 +120,11 @@ def test_forward_host_buffers_match_device_buffers():
     moe.moe_forward_host(xh, lh, inp["w13"], inp["w2"], 2, oh, ws)
     assert moe.moe_last_status(ws) == 0
     assert torch.equal(oh.view(torch.int16), ref.cpu().view(torch.int16))
+
+
+def test_forward_with_the_largest_top_k():
+    inp = gpu_inputs(dict(T=24, H=128, I=64, E=64, top_k=32), seed=8)
+    out, views, _ = run_forward(inp)
+    ids, w, off, s2f, f2s, h, y, ref = oracle_everything(to_host_case(inp))
+    assert_routing_exact(views, ids, w, off, s2f, f2s)
+    assert_close_out(bf16_to_f64(out), ref, "out")

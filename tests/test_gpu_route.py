@@ -96,3 +96,30 @@ def test_route_empty_batch_and_argument_errors():
     assert moe.moe_route(logits, k, ids, w, off, s, s.clone(), tiny_ws, check=False) == -5
     big = moe.alloc_workspace(1 << 16, dev)
     assert moe.moe_route(logits, E + 1, ids, w, off, s, s.clone(), big, check=False) == -2
+
+
+def test_route_large_batch_three_kernel_path_and_max_top_k():
+    g = torch.Generator().manual_seed(21)
+    check_against_oracle(torch.randn(100_000, 64, generator=g), 8)      # 800k assignments, 3125 chunks
+    check_against_oracle(torch.randn(2_000, 64, generator=g), 32)       # the largest supported top_k
+
+
+def test_route_non_finite_logits_terminate_with_in_range_distinct_ids():
+    """NaN / inf logits are outside the contract, but the kernels must finish and stay in bounds."""
+    g = torch.Generator().manual_seed(22)
+    T, E, k = 300, 96, 8
+    logits = torch.randn(T, E, generator=g)
+    logits[0] = float("nan")
+    logits[1, ::3] = float("inf")
+    logits[2, 5:50] = float("-inf")
+    logits[3, 7] = float("nan")
+    logits[4] = float("-inf")
+    ids, w, off, s2f, f2s = run_route(logits.cuda().contiguous(), k)
+    assert ((ids >= 0) & (ids < E)).all()
+    assert all(len(set(r.tolist())) == k for r in ids)
+    assert off[0] == 0 and off[-1] == T * k and (np.diff(off) >= 0).all()
+    assert np.array_equal(np.sort(s2f), np.arange(T * k)) and np.array_equal(s2f[f2s], np.arange(T * k))
+    # rows without non-finite values are unaffected by their neighbours
+    o = moe_oracle.get("f32")
+    rid, _ = o.route(logits[5:].numpy(), k)
+    assert np.array_equal(ids[5:], rid)
