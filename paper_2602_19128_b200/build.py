@@ -39,7 +39,6 @@ def build_library(force: bool = False, verbose: bool = False) -> Path:
            "-I", str(ROOT / "include"), "-I", str(CSRC)]
     if verbose:
         cmd += ["-Xptxas", "-v"]
-    cmd += os.environ.get("MOE_NVCC_FLAGS", "").split()  # extra flags for experiment builds
     cmd += [str(CSRC / s) for s in SOURCES] + ["-o", str(tmp)]
     subprocess.run(cmd, check=True)
     os.replace(tmp, LIB)

@@ -114,14 +114,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ TensorMaps maps, const KernelPara
                 if (!ok) break;
                 if (elect_one()) {
                     const uint32_t full = bar_full + stage * 8;
-#if defined(MOE_ABLATE_NO_TMA)  // experiment builds only: time the MMA side alone
-                    mbar_arrive(full);
-#else
-#ifdef MOE_ABLATE_NO_B
-                    mbar_expect_tx(full, kSlotABytes);
-#else
                     mbar_expect_tx(full, tx_bytes);
-#endif
                     const uint32_t sa = base + L::kA + stage * kSlotABytes;
                     const uint32_t sb = base + L::kB + stage * L::kSlotBBytes;
                     const int k0 = kb * kBlockK;
@@ -129,10 +122,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ TensorMaps maps, const KernelPara
                         tma_load_5d(sa, &maps.w, k0, 0, 0, t.f * 4, t.e, full);
                     else
                         tma_load_2d(sa, &maps.w, k0, w_row, full);
-#ifndef MOE_ABLATE_NO_B
                     tma_load_2d(sb, act_map<16>(maps, n_mma), k0, t.row0, full);
-#endif
-#endif
                 }
                 __syncwarp();
                 if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -159,11 +149,9 @@ grouped_gemm_tc_kernel(const __grid_constant__ TensorMaps maps, const KernelPara
                 if (elect_one()) {
                     const uint64_t a_desc = smem_desc_k_major_sw128(base + L::kA + stage * kSlotABytes);
                     const uint64_t b_desc = smem_desc_k_major_sw128(base + L::kB + stage * L::kSlotBBytes);
-#ifndef MOE_ABLATE_NO_MMA  // (experiment builds may drop the MMAs to time the load side alone)
 #pragma unroll
                     for (int kk = 0; kk < kBlockK / 16; ++kk)  // 16 K-elements = 32 bytes = 2 descriptor units
                         umma_bf16(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (kb | kk) != 0);
-#endif
                     umma_commit(bar_empty + stage * 8);
                     if (kb == p.n_k_blocks - 1) umma_commit(bar_acc_full + acc * 8);
                 }
@@ -180,8 +168,8 @@ grouped_gemm_tc_kernel(const __grid_constant__ TensorMaps maps, const KernelPara
         uint32_t acc_phase = 0;
         bool ok = true;
         for (int round = 0; ok; ++round) {
-                const int tile = tile_of_round(round, blockIdx.x, gridDim.x);
-                if (tile >= total_tiles) break;
+            const int tile = tile_of_round(round, blockIdx.x, gridDim.x);
+            if (tile >= total_tiles) break;
             const Tile t = decode_tile(tile, p);
             const int n_mma = (t.n_valid + 15) & ~15;
             ok = mbar_wait(bar_acc_full + acc * 8, acc_phase, abort_flag, p.status, kSiteEpilogueTmemFull + kSiteOffset);

@@ -207,14 +207,7 @@ grouped_gemm_tc_pair_kernel(const __grid_constant__ TensorMaps maps, const Kerne
                     const uint32_t full = map_to_cta(bar_full + stage * 8, 0);
                     const int k0 = kb * kBlockK;
                     if (load_w) {
-#if defined(MOE_ABLATE_NO_TMA)  // experiment builds only: time the MMA side alone
-                        if (rank == 0) mbar_arrive(bar_full + stage * 8);
-#else
-#ifdef MOE_ABLATE_NO_B
-                        if (rank == 0) mbar_expect_tx(bar_full + stage * 8, 2 * L::kSlotABytesAll);
-#else
                         if (rank == 0) mbar_expect_tx(bar_full + stage * 8, 2 * L::kSlotABytesAll + n_mma * kRowBytes);
-#endif
 #pragma unroll
                         for (int s = 0; s < SLABS; ++s) {
                             const uint32_t sa = base + L::kA + stage * L::kSlotABytesAll + s * kSlotABytes;
@@ -224,14 +217,11 @@ grouped_gemm_tc_pair_kernel(const __grid_constant__ TensorMaps maps, const Kerne
                             else
                                 tma_load_2d_pair(sa, &maps.w, k0, t.e * p.w_rows + feat, full);
                         }
-#endif
                     }
-#if !defined(MOE_ABLATE_NO_B) && !defined(MOE_ABLATE_NO_TMA)
                     if (load_act) {
                         const uint32_t sb = base + L::kB + stage * L::kSlotBBytes;
                         tma_load_2d_pair(sb, act_map<8>(maps, half), k0, t.row0 + (int)rank * half, full);
                     }
-#endif
                 }
                 __syncwarp();
                 if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -271,7 +261,6 @@ grouped_gemm_tc_pair_kernel(const __grid_constant__ TensorMaps maps, const Kerne
                     tcgen05_fence_after();
                     if (elect_one()) {
                         const uint64_t b_desc = smem_desc_k_major_sw128(base + L::kB + stage * L::kSlotBBytes);
-#ifndef MOE_ABLATE_NO_MMA  // (experiment builds may drop the MMAs to time the load side alone)
 #pragma unroll
                         for (int s = 0; s < SLABS; ++s) {
                             const uint64_t a_desc =
@@ -280,7 +269,6 @@ grouped_gemm_tc_pair_kernel(const __grid_constant__ TensorMaps maps, const Kerne
                             for (int kk = 0; kk < kBlockK / 16; ++kk)  // 16 K-elements = 32 bytes = 2 descriptor units
                                 umma_bf16_pair(d_tmem + s * NT_MAX, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (kb | kk) != 0);
                         }
-#endif
                         umma_commit_pair(bar_empty + stage * 8);
                         if (kb == p.n_k_blocks - 1) umma_commit_pair(bar_acc_full + acc * 8);
                     }

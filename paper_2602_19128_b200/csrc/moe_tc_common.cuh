@@ -76,13 +76,6 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     const long long start = clock64();
     while (true) {
         if (mbar_try_wait_suspend(bar, parity, kWaitSuspendNs)) {
-#ifdef MOE_WAIT_STATS  // experiment builds only: cycles spent waiting, per site, after the status ints
-            if ((threadIdx.x & 31) == 0) {
-                unsigned long long *stats = reinterpret_cast<unsigned long long *>(status + 8);
-                atomicAdd(&stats[site], (unsigned long long)(clock64() - start));
-                atomicAdd(&stats[8 + site], 1ull);
-            }
-#endif
             return true;
         }
         if (*abort_flag) return false;
