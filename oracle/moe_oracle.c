@@ -435,3 +435,157 @@ int moe_oracle_forward_fp8w(const uint16_t *x, const float *router_logits, const
     }
     return status;
 }
+
+/* ---- MX FP8: weights AND activations in 8 bits, one power-of-two scale per 32 elements ---------------
+ * The paper's MoE workload is an FP8 one ("FP8 MoE", Table 2; Sec. 4.5 names the cost of FP8 packing and
+ * scaling).  It does not fix the scaling granularity.  The build's reading for a path whose products run
+ * on the tensor cores in 8 bits is the OCP Microscaling format MXFP8: E4M3 element codes and, for every
+ * 32 consecutive elements along the contraction dimension, one E8M0 scale byte b standing for 2^(b-127)
+ * (b = 255 is NaN).  A stored value is decode(code) * 2^(b-127).
+ *
+ * Quantising 32 values v (MX specification, "conversion to MX formats"):
+ *     shared exponent  s = floor(log2(max|v|)) - 8     (8 = exponent of the largest E4M3 binade),
+ *     scale byte       b = clamp(s + 127, 0, 254),
+ *     code_i           = E4M3 of v_i / 2^(b-127), round to nearest even, values beyond +-448 saturate.
+ * An all-zero block gets b = 0; a block holding an infinity or a NaN gets b = 255 and NaN codes.
+ *
+ * The layer: the expert weights arrive quantised (inputs); the token rows x are quantised along H before
+ * the gate/up projections, and h = SiLU(gate) * up is quantised along I before the down projection, both
+ * with the rule above; every dot product is the plain sum, in index order, of products of stored values. */
+static inline REAL e8m0_decode(uint8_t b) { return b == 255 ? (REAL)NAN : (REAL)ldexp(1.0, (int)b - 127); }
+
+/* E4M3 code of v: round to nearest, ties to the even code, finite values beyond the largest magnitude
+ * (448) saturate to it, NaN gives the NaN code. */
+static uint8_t e4m3_encode(double v) {
+    const uint8_t sign = signbit(v) ? 0x80 : 0;
+    const double a = fabs(v);
+    if (isnan(a)) return (uint8_t)(sign | 0x7F);
+    if (a >= 448.0) return (uint8_t)(sign | 0x7E);
+    if (a < 0.015625) return (uint8_t)(sign | (uint8_t)rint(a * 512.0)); /* multiples of 2^-9; 8 is the first normal */
+    int ex;
+    const double m = frexp(a, &ex);                  /* a = m * 2^ex, m in [0.5, 1) */
+    int E = ex - 1;                                  /* a = (2m) * 2^E, 2m in [1, 2) */
+    int mant = (int)rint((2.0 * m - 1.0) * 8.0);     /* eighths above one, nearest even */
+    if (mant == 8) { mant = 0; E += 1; }
+    return (uint8_t)(sign | ((E + 7) << 3) | mant);
+}
+
+uint8_t moe_oracle_e4m3_encode(float v) { return e4m3_encode((double)v); }
+
+/* Quantise one block of n values (n = 32 in the layer) to codes and one scale byte. */
+static void mx_quantize_block(const REAL *v, int n, uint8_t *codes, uint8_t *scale_byte) {
+    double amax = 0;
+    int nonfinite = 0;
+    for (int i = 0; i < n; ++i) {
+        const double a = fabs((double)v[i]);
+        if (!isfinite(a)) nonfinite = 1;
+        else if (a > amax) amax = a;
+    }
+    if (nonfinite) {
+        *scale_byte = 255;
+        for (int i = 0; i < n; ++i) codes[i] = 0x7F;
+        return;
+    }
+    int b = 0;
+    if (amax > 0) {
+        int ex;
+        (void)frexp(amax, &ex);       /* floor(log2(amax)) = ex - 1 */
+        b = (ex - 1) - 8 + 127;
+        if (b < 0) b = 0;
+        if (b > 254) b = 254;
+    }
+    *scale_byte = (uint8_t)b;
+    for (int i = 0; i < n; ++i) codes[i] = e4m3_encode(ldexp((double)v[i], 127 - b)); /* division by 2^(b-127) is exact */
+}
+
+/* Rows of fp32 values [R, K] -> codes [R, K] and scale bytes [R, K/32]; K a multiple of 32. */
+int moe_oracle_mx_quantize(const float *v, int R, int K, uint8_t *codes, uint8_t *scales) {
+    if (R < 0 || K < 32 || K % 32) return ORACLE_ERR_ARG;
+    REAL tmp[32];
+    for (long r = 0; r < R; ++r)
+        for (int b = 0; b < K / 32; ++b) {
+            for (int i = 0; i < 32; ++i) tmp[i] = (REAL)v[(size_t)r * K + 32 * b + i];
+            mx_quantize_block(tmp, 32, codes + (size_t)r * K + 32 * b, scales + (size_t)r * (K / 32) + b);
+        }
+    return ORACLE_OK;
+}
+
+static inline REAL mx_value(const uint8_t *codes, const uint8_t *scales, int i) {
+    return e4m3_decode(codes[i]) * e8m0_decode(scales[i / 32]);
+}
+
+/* One expert with MX weights applied to one quantised token row.
+ *   xq [H] codes, xs [H/32]; w13q_e [2I,H], w13s_e [2I,H/32]; w2q_e [H,I], w2s_e [H,I/32]
+ *   -> y [H] REAL; s [I] REAL receives h before quantisation, hq [I] / hs [I/32] its quantised form. */
+static void expert_ffn_row_mx(const uint8_t *xq, const uint8_t *xs, const uint8_t *w13q_e, const uint8_t *w13s_e,
+                              const uint8_t *w2q_e, const uint8_t *w2s_e, int H, int I, REAL *y, REAL *s, uint8_t *hq,
+                              uint8_t *hs) {
+    for (int i = 0; i < I; ++i) {
+        const uint8_t *gq = w13q_e + (size_t)i * H, *gs = w13s_e + (size_t)i * (H / 32);
+        const uint8_t *uq = w13q_e + (size_t)(I + i) * H, *us = w13s_e + (size_t)(I + i) * (H / 32);
+        REAL g = 0, u = 0;
+        for (int c = 0; c < H; ++c) {
+            const REAL xv = mx_value(xq, xs, c);
+            g += xv * mx_value(gq, gs, c);
+            u += xv * mx_value(uq, us, c);
+        }
+        s[i] = g / ((REAL)1 + real_exp(-g)) * u;
+    }
+    for (int b = 0; b < I / 32; ++b) mx_quantize_block(s + 32 * b, 32, hq + 32 * b, hs + b);
+    for (int n = 0; n < H; ++n) {
+        const uint8_t *dq = w2q_e + (size_t)n * I, *ds = w2s_e + (size_t)n * (I / 32);
+        REAL acc = 0;
+        for (int i = 0; i < I; ++i) acc += mx_value(hq, hs, i) * mx_value(dq, ds, i);
+        y[n] = acc;
+    }
+}
+
+/* The whole layer in MX FP8.  x [T,H] bf16, router_logits [T,E] f32, w13_q [E,2I,H] codes, w13_s [E,2I,H/32]
+ * scale bytes, w2_q [E,H,I], w2_s [E,H,I/32] -> out [T,H] REAL.  Optional (may be NULL), per flat assignment
+ * a = t*k + j:  h_pre [A,I] REAL = h before quantisation, h_q [A,I] codes, h_s [A,I/32] scale bytes.
+ * H and I must be multiples of 32. */
+int moe_oracle_forward_mxfp8(const uint16_t *x, const float *router_logits, const uint8_t *w13_q, const uint8_t *w13_s,
+                             const uint8_t *w2_q, const uint8_t *w2_s, int T, int H, int I, int E, int k, REAL *out,
+                             REAL *h_pre, uint8_t *h_q, uint8_t *h_s) {
+    if (T < 0 || H < 32 || I < 32 || H % 32 || I % 32 || E < 1 || k < 1 || k > E) return ORACLE_ERR_ARG;
+    int status = ORACLE_OK;
+    const size_t n13 = (size_t)2 * I * H, n2 = (size_t)H * I;
+    const size_t s13 = (size_t)2 * I * (H / 32), s2 = (size_t)H * (I / 32);
+#pragma omp parallel
+    {
+        REAL *p = (REAL *)malloc(sizeof(REAL) * (size_t)E);
+        unsigned char *taken = (unsigned char *)malloc((size_t)E);
+        int32_t *ids = (int32_t *)malloc(sizeof(int32_t) * (size_t)k);
+        REAL *w = (REAL *)malloc(sizeof(REAL) * (size_t)k);
+        REAL *s = (REAL *)malloc(sizeof(REAL) * (size_t)I);
+        REAL *y = (REAL *)malloc(sizeof(REAL) * (size_t)H);
+        REAL *xr = (REAL *)malloc(sizeof(REAL) * (size_t)H);
+        uint8_t *xq = (uint8_t *)malloc((size_t)H), *xs = (uint8_t *)malloc((size_t)(H / 32));
+        uint8_t *hq = (uint8_t *)malloc((size_t)I), *hs = (uint8_t *)malloc((size_t)(I / 32));
+        if (!p || !taken || !ids || !w || !s || !y || !xr || !xq || !xs || !hq || !hs) {
+#pragma omp critical
+            status = ORACLE_ERR_NOMEM;
+        } else {
+#pragma omp for schedule(dynamic, 1)
+            for (int t = 0; t < T; ++t) {
+                REAL *o = out + (size_t)t * H;
+                for (int n = 0; n < H; ++n) o[n] = 0;
+                route_token(router_logits + (size_t)t * E, E, k, ids, w, p, taken);
+                for (int c = 0; c < H; ++c) xr[c] = bf16_to_real(x[(size_t)t * H + c]);
+                for (int b = 0; b < H / 32; ++b) mx_quantize_block(xr + 32 * b, 32, xq + 32 * b, xs + b);
+                for (int j = 0; j < k; ++j) {
+                    const int e = ids[j];
+                    expert_ffn_row_mx(xq, xs, w13_q + e * n13, w13_s + e * s13, w2_q + e * n2, w2_s + e * s2, H, I, y, s,
+                                      hq, hs);
+                    const size_t a = (size_t)t * k + j;
+                    if (h_pre) memcpy(h_pre + a * I, s, sizeof(REAL) * (size_t)I);
+                    if (h_q) memcpy(h_q + a * I, hq, (size_t)I);
+                    if (h_s) memcpy(h_s + a * (I / 32), hs, (size_t)(I / 32));
+                    for (int n = 0; n < H; ++n) o[n] += w[j] * y[n];
+                }
+            }
+        }
+        free(p); free(taken); free(ids); free(w); free(s); free(y); free(xr); free(xq); free(xs); free(hq); free(hs);
+    }
+    return status;
+}

@@ -51,10 +51,13 @@ class Oracle:
         assert self.lib.moe_oracle_real_bytes() == np.dtype(self.real).itemsize
         for fn in ("moe_oracle_route", "moe_oracle_permute", "moe_oracle_expert_ffn", "moe_oracle_forward",
                    "moe_oracle_forward_sampled", "moe_oracle_sorted_intermediates", "moe_oracle_forward_local",
-                   "moe_oracle_permute_local", "moe_oracle_forward_fp8w"):
+                   "moe_oracle_permute_local", "moe_oracle_forward_fp8w", "moe_oracle_mx_quantize",
+                   "moe_oracle_forward_mxfp8"):
             getattr(self.lib, fn).restype = ctypes.c_int
         self.lib.moe_oracle_e4m3_decode.restype = ctypes.c_float
         self.lib.moe_oracle_e4m3_decode.argtypes = [ctypes.c_uint8]
+        self.lib.moe_oracle_e4m3_encode.restype = ctypes.c_uint8
+        self.lib.moe_oracle_e4m3_encode.argtypes = [ctypes.c_float]
 
     # -- helpers ---------------------------------------------------------------------------
     @staticmethod
@@ -185,6 +188,42 @@ class Oracle:
                                                      self._ptr(w2_q), self._ptr(w2_scale), T, H, I, E, top_k,
                                                      self._ptr(out)), "forward_fp8w")
         return out
+
+    def e4m3_encode(self, value: float) -> int:
+        return int(self.lib.moe_oracle_e4m3_encode(ctypes.c_float(value)))
+
+    def mx_quantize(self, values: np.ndarray):
+        """Rows of fp32 values [R,K] -> (E4M3 codes [R,K], E8M0 scale bytes [R,K/32]), blocks of 32 along K."""
+        v = np.ascontiguousarray(values, dtype=np.float32)
+        R, K = v.shape
+        codes = np.empty((R, K), np.uint8)
+        scales = np.empty((R, K // 32), np.uint8)
+        self._check(self.lib.moe_oracle_mx_quantize(self._ptr(v), R, K, self._ptr(codes), self._ptr(scales)), "mx_quantize")
+        return codes, scales
+
+    def forward_mxfp8(self, x, router_logits, w13_q, w13_s, w2_q, w2_s, top_k: int, intermediates: bool = False):
+        """The layer in MX FP8 (E4M3 codes, one E8M0 scale byte per 32 elements along the contraction).
+        With ``intermediates`` also returns, per flat assignment t*k+j, h before quantisation [A,I] and its
+        quantised codes [A,I] and scale bytes [A,I/32]."""
+        x = self._u16(x)
+        l = np.ascontiguousarray(router_logits, dtype=np.float32)
+        w13_q, w13_s = np.ascontiguousarray(w13_q, dtype=np.uint8), np.ascontiguousarray(w13_s, dtype=np.uint8)
+        w2_q, w2_s = np.ascontiguousarray(w2_q, dtype=np.uint8), np.ascontiguousarray(w2_s, dtype=np.uint8)
+        T, H = x.shape
+        E, I2, _ = w13_q.shape
+        I = I2 // 2
+        assert w13_q.shape == (E, 2 * I, H) and w2_q.shape == (E, H, I) and l.shape == (T, E)
+        assert w13_s.shape == (E, 2 * I, H // 32) and w2_s.shape == (E, H, I // 32)
+        out = np.empty((T, H), self.real)
+        A = T * top_k
+        h_pre = np.empty((A, I), self.real) if intermediates else None
+        h_q = np.empty((A, I), np.uint8) if intermediates else None
+        h_s = np.empty((A, I // 32), np.uint8) if intermediates else None
+        opt = lambda a: self._ptr(a) if a is not None else None
+        self._check(self.lib.moe_oracle_forward_mxfp8(self._ptr(x), self._ptr(l), self._ptr(w13_q), self._ptr(w13_s),
+                                                      self._ptr(w2_q), self._ptr(w2_s), T, H, I, E, top_k,
+                                                      self._ptr(out), opt(h_pre), opt(h_q), opt(h_s)), "forward_mxfp8")
+        return (out, h_pre, h_q, h_s) if intermediates else out
 
     def sorted_intermediates(self, x, w13, w2, topk_ids, sorted_to_flat):
         x, w13, w2 = self._u16(x), self._u16(w13), self._u16(w2)
