@@ -207,6 +207,66 @@ MOE_API int moe_forward_staged(const void *x, const float *router_logits, const 
                                void *workspace, size_t workspace_bytes, void *stream, unsigned flags,
                                void *const *stage_events);
 
+/* ---- MX FP8: 8-bit weights AND activations, multiplied by the block-scaled tensor-core instruction --------
+ *
+ * The paper's MoE workload is an FP8 one (Table 2, "FP8 MoE"; Sec. 4.5 names FP8 packing and scaling as a
+ * cost of the kernel) without fixing the scaling granularity.  This path uses the OCP Microscaling format
+ * MXFP8, the one sm_100a multiplies natively: E4M3 codes, and for every 32 consecutive elements along the
+ * contraction dimension one E8M0 scale byte b standing for 2^(b-127) (255 = NaN); a stored value is
+ * decode(code) * 2^(b-127).  Quantising 32 values: b = clamp(floor(log2(max|v|)) - 8 + 127, 0, 254) (0 for an
+ * all-zero block; 255 and NaN codes if the block holds an infinity or NaN), codes = E4M3(v / 2^(b-127)),
+ * round to nearest even, saturating at +-448.  The layer quantises each token row of x along H before the
+ * gate/up projections and h = SiLU(gate)*up along I (from its fp32 value) before the down projection;
+ * accumulation is fp32; y and out are bf16 as in moe_forward.
+ *
+ * Scale bytes are consumed in 512-byte "atoms": the 4 scale bytes (128 K-elements) of 128 rows, row r's at
+ * byte (r % 32) * 16 + (r / 32) * 4.  moe_mxfp8_pack_scales converts plain scale bytes to that form once. */
+
+/* Offsets of the MX path's workspace regions; A = T*top_k. */
+typedef struct {
+    size_t total_bytes;
+    size_t status, topk_ids, topk_weights, expert_offsets, sorted_to_flat, flat_to_sorted, route_scratch; /* as moe_workspace_layout_t */
+    size_t x_q;   /* uint8 [A,H]  codes of the token rows in expert-contiguous order */
+    size_t x_sf;  /* scale atoms of x_q: [H/128][sf_atoms][512]; row i of expert e is row i % tile_rows of atom
+                     expert_offsets[e] / tile_rows + e + i / tile_rows (one atom per token tile) */
+    size_t h_q;   /* uint8 [A,I]  codes of h */
+    size_t h_sf;  /* scale atoms of h_q: [I/128][sf_atoms][512], same row-to-atom rule */
+    size_t y;     /* bf16 [A,H] */
+    size_t sf_atoms;  /* a count, not an offset: atoms per K-slot in x_sf / h_sf (A / tile_rows + E + 1) */
+    size_t tile_rows; /* a count: rows per token tile of this problem (32, 64 or 128) */
+} moe_mxfp8_workspace_layout_t;
+
+/* Host-only, pure.  Workspace bytes of moe_forward_mxfp8; 0 outside the envelope (moe_forward's, plus I % 128 == 0). */
+MOE_API size_t moe_mxfp8_workspace_bytes(int T, int H, int I, int E, int top_k);
+MOE_API int moe_mxfp8_workspace_layout(int T, int H, int I, int E, int top_k, moe_mxfp8_workspace_layout_t *layout);
+
+/* Repack weight scale bytes for moe_forward_mxfp8 (done once per model; enqueues one kernel on `stream`).
+ *   scales  [E, rows, K/32] uint8, DEVICE, in: plain row-major scale bytes of a weight tensor [E, rows, K]
+ *   packed  E * rows * K/32 bytes, DEVICE, 16-byte aligned, out (must not alias `scales`)
+ *   gate_up 1 for w13 (rows = 2I, [gate | up]): atoms follow the gate/up GEMM's tiles of 64 features, whose 128
+ *           rows are, for each group of 16 features, the 16 gate rows then the 16 up rows;
+ *           0 for w2 (rows = H): atoms of 128 consecutive rows.
+ * Atom order: [E][rows/128 tiles][K/128][512].  Needs rows % 128 == 0 and K % 128 == 0. */
+MOE_API int moe_mxfp8_pack_scales(const void *scales, int E, int rows, int K, int gate_up, void *packed, void *stream);
+
+/* MX quantisation of bf16 rows by the rule above (the layer applies the same rule to x inside
+ * moe_forward_mxfp8; this entry point exposes it).  x [R,K] bf16 DEVICE (16-byte aligned) ->
+ * codes [R,K] uint8 (8-byte aligned), scales [R,K/32] uint8 plain row-major.  K % 128 == 0. */
+MOE_API int moe_mxfp8_quantize_rows(const void *x, int R, int K, void *codes, void *scales, void *stream);
+
+/* The layer in MX FP8, restricted to the resident experts as in moe_forward_local (pass 0 and E for all).
+ *   x [T,H] bf16, router_logits [T,E] f32, out [T,H] bf16: as moe_forward; all DEVICE pointers
+ *   w13_q [n_local,2I,H] uint8 codes, w13_sf_packed: its scale bytes packed with gate_up = 1
+ *   w2_q  [n_local,H,I]  uint8 codes, w2_sf_packed : its scale bytes packed with gate_up = 0
+ *   workspace  at least moe_mxfp8_workspace_bytes bytes, 256-byte aligned (layout: moe_mxfp8_workspace_layout)
+ *   stage_events  NULL, or MOE_NUM_STAGE_EVENTS events recorded as by moe_forward_staged
+ * Launches the same number of kernels as moe_forward (the gather also quantises).  Token tiles are at most
+ * 128 rows.  Errors as moe_forward; a block of x holding an infinity or NaN makes that token's output NaN. */
+MOE_API int moe_forward_mxfp8(const void *x, const float *router_logits, const void *w13_q, const void *w13_sf_packed,
+                              const void *w2_q, const void *w2_sf_packed, int T, int H, int I, int E, int top_k,
+                              int local_expert_offset, int num_local_experts, void *out, void *workspace,
+                              size_t workspace_bytes, void *stream, void *const *stage_events);
+
 /* moe_forward_local (local_expert_offset = 0, num_local_experts = E for the whole layer) for a caller
  * whose activations live in HOST memory: x_host [T,H] bf16 and router_logits_host [T,E] f32 are HOST
  * pointers (pinned memory makes the copies asynchronous), out_host [T,H] bf16 is a HOST pointer; the

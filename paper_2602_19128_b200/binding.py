@@ -21,7 +21,9 @@ MOE_FLAG_TWO_SLAB_GEMM = 4
 
 EXPORTED = ["moe_workspace_bytes", "moe_workspace_layout", "moe_route_workspace_bytes", "moe_route", "moe_route_static",
             "moe_forward",
-            "moe_forward_ex", "moe_forward_local", "moe_forward_fp8w", "moe_forward_staged", "moe_forward_host", "moe_last_status", "moe_forward_launch_count", "moe_status_string"]
+            "moe_forward_ex", "moe_forward_local", "moe_forward_fp8w", "moe_mxfp8_workspace_bytes",
+            "moe_mxfp8_workspace_layout", "moe_mxfp8_pack_scales", "moe_mxfp8_quantize_rows", "moe_forward_mxfp8",
+            "moe_forward_staged", "moe_forward_host", "moe_last_status", "moe_forward_launch_count", "moe_status_string"]
 
 
 class MoeError(RuntimeError):
@@ -34,6 +36,12 @@ class WorkspaceLayout(ctypes.Structure):
     _fields_ = [(n, ctypes.c_size_t) for n in
                 ("total_bytes", "status", "topk_ids", "topk_weights", "expert_offsets", "sorted_to_flat",
                  "flat_to_sorted", "route_scratch", "x_perm", "h", "y", "staging")]
+
+
+class MxWorkspaceLayout(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_size_t) for n in
+                ("total_bytes", "status", "topk_ids", "topk_weights", "expert_offsets", "sorted_to_flat",
+                 "flat_to_sorted", "route_scratch", "x_q", "x_sf", "h_q", "h_sf", "y", "sf_atoms", "tile_rows")]
 
 
 _lib = None
@@ -66,6 +74,16 @@ def lib() -> ctypes.CDLL:
         L.moe_forward_local.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, vp, vp, sz, vp, ctypes.c_uint]
         L.moe_forward_fp8w.restype = i
         L.moe_forward_fp8w.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, vp, vp, sz, vp, ctypes.POINTER(vp)]
+        L.moe_mxfp8_workspace_bytes.restype = sz
+        L.moe_mxfp8_workspace_bytes.argtypes = [i] * 5
+        L.moe_mxfp8_workspace_layout.restype = i
+        L.moe_mxfp8_workspace_layout.argtypes = [i] * 5 + [ctypes.POINTER(MxWorkspaceLayout)]
+        L.moe_mxfp8_pack_scales.restype = i
+        L.moe_mxfp8_pack_scales.argtypes = [vp, i, i, i, i, vp, vp]
+        L.moe_mxfp8_quantize_rows.restype = i
+        L.moe_mxfp8_quantize_rows.argtypes = [vp, i, i, vp, vp, vp]
+        L.moe_forward_mxfp8.restype = i
+        L.moe_forward_mxfp8.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, i, i, vp, vp, sz, vp, ctypes.POINTER(vp)]
         L.moe_forward_staged.restype = i
         L.moe_forward_staged.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, vp, vp, sz, vp, ctypes.c_uint,
                                          ctypes.POINTER(vp)]
@@ -185,6 +203,82 @@ def moe_forward_fp8w(x, router_logits, w13_q, w13_scale, w2_q, w2_scale, top_k: 
     if check and st != MOE_OK:
         raise MoeError(st, "moe_forward_fp8w")
     return st
+
+
+def moe_mxfp8_workspace_bytes(T: int, H: int, I: int, E: int, top_k: int) -> int:
+    return int(lib().moe_mxfp8_workspace_bytes(T, H, I, E, top_k))
+
+
+def moe_mxfp8_workspace_layout(T: int, H: int, I: int, E: int, top_k: int) -> MxWorkspaceLayout:
+    L = MxWorkspaceLayout()
+    st = lib().moe_mxfp8_workspace_layout(T, H, I, E, top_k, ctypes.byref(L))
+    if st != MOE_OK:
+        raise MoeError(st, "moe_mxfp8_workspace_layout")
+    return L
+
+
+def moe_mxfp8_pack_scales(scales, gate_up: bool, stream=None) -> torch.Tensor:
+    """Repack plain MX scale bytes [E, rows, K/32] of a weight tensor into the atoms moe_forward_mxfp8 reads."""
+    E, rows, kb = scales.shape
+    packed = torch.empty(scales.numel(), dtype=torch.uint8, device=scales.device)
+    st = lib().moe_mxfp8_pack_scales(_ptr(scales), E, rows, kb * 32, int(gate_up), _ptr(packed), _stream(stream))
+    if st != MOE_OK:
+        raise MoeError(st, "moe_mxfp8_pack_scales")
+    return packed
+
+
+def moe_mxfp8_quantize_rows(x, stream=None):
+    """MX quantisation of bf16 rows [R,K]: (codes uint8 [R,K], scale bytes uint8 [R,K/32])."""
+    R, K = x.shape
+    codes = torch.empty((R, K), dtype=torch.uint8, device=x.device)
+    scales = torch.empty((R, K // 32), dtype=torch.uint8, device=x.device)
+    st = lib().moe_mxfp8_quantize_rows(_ptr(x), R, K, _ptr(codes), _ptr(scales), _stream(stream))
+    if st != MOE_OK:
+        raise MoeError(st, "moe_mxfp8_quantize_rows")
+    return codes, scales
+
+
+def moe_forward_mxfp8(x, router_logits, w13_q, w13_sf_packed, w2_q, w2_sf_packed, top_k: int, out, workspace,
+                      stream=None, stage_events=None, local_expert_offset: int = 0, check: bool = True) -> int:
+    """The layer in MX FP8 (E4M3 codes, packed E8M0 scale bytes); w13_q may hold a local subset of the experts."""
+    T, H = x.shape
+    E = router_logits.shape[1]
+    n_local, I2, _ = w13_q.shape
+    handles = None
+    if stage_events is not None:
+        handles = (ctypes.c_void_p * (len(STAGE_NAMES) + 1))(*[e.cuda_event for e in stage_events])
+    st = lib().moe_forward_mxfp8(_ptr(x), _ptr(router_logits), _ptr(w13_q), _ptr(w13_sf_packed), _ptr(w2_q),
+                                 _ptr(w2_sf_packed), T, H, I2 // 2, E, top_k, local_expert_offset, n_local, _ptr(out),
+                                 _ptr(workspace), workspace.numel(), _stream(stream), handles)
+    if check and st != MOE_OK:
+        raise MoeError(st, "moe_forward_mxfp8")
+    return st
+
+
+def mx_workspace_views(workspace: torch.Tensor, T: int, H: int, I: int, E: int, top_k: int) -> dict:
+    """Typed views of what a moe_forward_mxfp8 call left in ``workspace`` (scale atoms as [K/128, atoms, 512])."""
+    L = moe_mxfp8_workspace_layout(T, H, I, E, top_k)
+    A = T * top_k
+    n = int(L.sf_atoms)
+
+    def view(off, nbytes, dtype, shape):
+        return workspace[off:off + nbytes].view(dtype).view(shape)
+
+    return dict(
+        status=view(L.status, 16, torch.int32, (4,)),
+        topk_ids=view(L.topk_ids, A * 4, torch.int32, (T, top_k)),
+        topk_weights=view(L.topk_weights, A * 4, torch.float32, (T, top_k)),
+        expert_offsets=view(L.expert_offsets, (E + 1) * 4, torch.int32, (E + 1,)),
+        sorted_to_flat=view(L.sorted_to_flat, A * 4, torch.int32, (A,)),
+        flat_to_sorted=view(L.flat_to_sorted, A * 4, torch.int32, (A,)),
+        x_q=view(L.x_q, A * H, torch.uint8, (A, H)),
+        x_sf=view(L.x_sf, (H // 128) * n * 512, torch.uint8, (H // 128, n, 512)),
+        h_q=view(L.h_q, A * I, torch.uint8, (A, I)),
+        h_sf=view(L.h_sf, (I // 128) * n * 512, torch.uint8, (I // 128, n, 512)),
+        y=view(L.y, A * H * 2, torch.bfloat16, (A, H)),
+        sf_atoms=n,
+        tile_rows=int(L.tile_rows),
+    )
 
 
 STAGE_NAMES = ("route", "gather", "gemm1_swiglu", "gemm2", "combine")

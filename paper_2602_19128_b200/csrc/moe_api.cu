@@ -147,9 +147,158 @@ int forward_impl(const void *x, const float *logits, const void *w13, const void
     return MOE_OK;
 }
 
+// ---- MX FP8 ---------------------------------------------------------------------------------------------
+bool mx_envelope_ok(long long T, int H, int I, int E, int k) { return envelope_ok(T, H, I, E, k) && I % 128 == 0; }
+
+// Token-tile bound of the MX path: the MX kernel keeps scale columns next to two accumulators in tensor
+// memory, and one scale atom covers 128 rows.
+int mx_tile_rows(int T, int E, int k) {
+    const int nt = choose_nt_max(T, E, k);
+    return nt > 128 ? 128 : nt;
+}
+
+void fill_mx_layout(int T, int H, int I, int E, int k, moe_mxfp8_workspace_layout_t *L) {
+    const size_t A = (size_t)T * k;
+    const int tile = mx_tile_rows(T, E, k);
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t at = off; off += align_up(bytes, 256); return at; };
+    L->status = take(kStatusInts * sizeof(int));
+    L->topk_ids = take(A * sizeof(int));
+    L->topk_weights = take(A * sizeof(float));
+    L->expert_offsets = take((size_t)(E + 1) * sizeof(int));
+    L->sorted_to_flat = take(A * sizeof(int));
+    L->flat_to_sorted = take(A * sizeof(int));
+    L->route_scratch = take(route_scratch_bytes(T, E));
+    L->x_q = take(A * H);
+    L->x_sf = take(mx_act_sf_bytes((int)A, E, H, tile));
+    L->h_q = take(A * I);
+    L->h_sf = take(mx_act_sf_bytes((int)A, E, I, tile));
+    L->y = take(A * H * 2);
+    L->sf_atoms = (size_t)mx_act_sf_atoms((int)A, E, tile);
+    L->tile_rows = (size_t)tile;
+    L->total_bytes = off;
+}
+
+int forward_mx_impl(const void *x, const float *logits, const void *w13_q, const void *w13_sf, const void *w2_q,
+                    const void *w2_sf, int T, int H, int I, int E, int k, int local_offset, int n_local, void *out,
+                    void *workspace, size_t workspace_bytes, cudaStream_t stream, void *const *stage_events) {
+    if (T < 0 || H <= 0 || I <= 0 || E <= 0 || k <= 0 || k > E) return MOE_ERR_SHAPE;
+    if (!mx_envelope_ok(T, H, I, E, k)) return MOE_ERR_UNSUPPORTED;
+    if (local_offset < 0 || n_local < 1 || (long long)local_offset + n_local > E) return MOE_ERR_SHAPE;
+    if (stage_events)
+        for (int i = 0; i < MOE_NUM_STAGE_EVENTS; ++i)
+            if (!stage_events[i]) return MOE_ERR_NULL;
+    if (T == 0) return MOE_OK;
+    if (!x || !logits || !w13_q || !w13_sf || !w2_q || !w2_sf || !out || !workspace) return MOE_ERR_NULL;
+    if (!aligned(x, 16) || !aligned(logits, 16) || !aligned(w13_q, 16) || !aligned(w2_q, 16) || !aligned(w13_sf, 16) ||
+        !aligned(w2_sf, 16) || !aligned(out, 16) || !aligned(workspace, 256))
+        return MOE_ERR_ALIGN;
+    moe_mxfp8_workspace_layout_t L;
+    fill_mx_layout(T, H, I, E, k, &L);
+    if (workspace_bytes < L.total_bytes) return MOE_ERR_WORKSPACE;
+    const int arch = check_device();
+    if (arch != MOE_OK) return arch;
+
+    char *ws = static_cast<char *>(workspace);
+    int *status = reinterpret_cast<int *>(ws + L.status);
+    int *ids = reinterpret_cast<int *>(ws + L.topk_ids);
+    float *wts = reinterpret_cast<float *>(ws + L.topk_weights);
+    int *offsets = reinterpret_cast<int *>(ws + L.expert_offsets);
+    int *s2f = reinterpret_cast<int *>(ws + L.sorted_to_flat);
+    int *f2s = reinterpret_cast<int *>(ws + L.flat_to_sorted);
+    RouteScratch rs = carve_route_scratch(ws + L.route_scratch, T, n_local);
+    uint8_t *x_q = reinterpret_cast<uint8_t *>(ws + L.x_q), *x_sf = reinterpret_cast<uint8_t *>(ws + L.x_sf);
+    uint8_t *h_q = reinterpret_cast<uint8_t *>(ws + L.h_q), *h_sf = reinterpret_cast<uint8_t *>(ws + L.h_sf);
+    __nv_bfloat16 *y = reinterpret_cast<__nv_bfloat16 *>(ws + L.y);
+    const int A = T * k;
+    const int n_atoms = (int)L.sf_atoms;
+    const int nt_max = (int)L.tile_rows;
+
+    auto mark = [&](int i) {
+        return !stage_events || cudaEventRecord(static_cast<cudaEvent_t>(stage_events[i]), stream) == cudaSuccess;
+    };
+    if (!mark(0)) return MOE_ERR_CUDA;
+    // every token tile exactly nt_max rows (the last of an expert partial): each tile owns one scale atom
+    if (launch_route(logits, T, E, k, LocalExperts{local_offset, n_local}, nt_max, ids, wts, offsets, s2f, f2s, rs, status,
+                     stream, nt_max) != cudaSuccess)
+        return MOE_ERR_CUDA;
+    if (!mark(1)) return MOE_ERR_CUDA;
+    if (launch_mx_gather_quantize(static_cast<const __nv_bfloat16 *>(x), s2f, offsets, n_local, A, k, H, x_q, x_sf, n_atoms,
+                                  nt_max, stream) != cudaSuccess)
+        return MOE_ERR_CUDA;
+    if (!mark(2)) return MOE_ERR_CUDA;
+
+    MxGemmArgs g1;
+    g1.act_q = x_q; g1.act_sf = x_sf; g1.w_q = static_cast<const uint8_t *>(w13_q);
+    g1.w_sf = static_cast<const uint8_t *>(w13_sf); g1.out = h_q; g1.out_sf = h_sf;
+    g1.A = A; g1.K = H; g1.n_out = I; g1.E = n_local; g1.w_rows = 2 * I; g1.nt_max = nt_max; g1.n_atoms = n_atoms;
+    g1.expert_offsets = offsets; g1.tile_prefix = rs.tile_prefix; g1.tile_order = rs.tile_order; g1.tile_rows = rs.tile_rows;
+    g1.status = status; g1.swiglu = true;
+    MxGemmArgs g2 = g1;
+    g2.act_q = h_q; g2.act_sf = h_sf; g2.w_q = static_cast<const uint8_t *>(w2_q);
+    g2.w_sf = static_cast<const uint8_t *>(w2_sf); g2.out = y; g2.out_sf = nullptr;
+    g2.K = I; g2.n_out = H; g2.w_rows = H; g2.swiglu = false;
+    int st = launch_grouped_gemm_tc_mx(g1, stream);
+    if (st != MOE_OK) return st;
+    if (!mark(3)) return MOE_ERR_CUDA;
+    st = launch_grouped_gemm_tc_mx(g2, stream);
+    if (st != MOE_OK) return st;
+    if (!mark(4)) return MOE_ERR_CUDA;
+    if (launch_combine(y, wts, f2s, T, k, H, static_cast<__nv_bfloat16 *>(out), stream) != cudaSuccess)
+        return MOE_ERR_CUDA;
+    if (!mark(5)) return MOE_ERR_CUDA;
+    return MOE_OK;
+}
+
 }  // namespace
 
 extern "C" {
+
+size_t moe_mxfp8_workspace_bytes(int T, int H, int I, int E, int top_k) {
+    if (!mx_envelope_ok(T, H, I, E, top_k)) return 0;
+    moe_mxfp8_workspace_layout_t L;
+    fill_mx_layout(T, H, I, E, top_k, &L);
+    return L.total_bytes;
+}
+
+int moe_mxfp8_workspace_layout(int T, int H, int I, int E, int top_k, moe_mxfp8_workspace_layout_t *layout) {
+    if (!layout) return MOE_ERR_NULL;
+    if (!mx_envelope_ok(T, H, I, E, top_k)) return MOE_ERR_UNSUPPORTED;
+    fill_mx_layout(T, H, I, E, top_k, layout);
+    return MOE_OK;
+}
+
+int moe_mxfp8_pack_scales(const void *scales, int E, int rows, int K, int gate_up, void *packed, void *stream) {
+    if (E < 1 || rows < 1 || K < 1) return MOE_ERR_SHAPE;
+    if (K % 128 != 0 || rows % 128 != 0) return MOE_ERR_UNSUPPORTED;
+    if (!scales || !packed) return MOE_ERR_NULL;
+    if (!aligned(scales, 4) || !aligned(packed, 16)) return MOE_ERR_ALIGN;
+    return launch_mx_pack_scales(static_cast<const uint8_t *>(scales), E, rows, K, gate_up != 0,
+                                 static_cast<uint8_t *>(packed), static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? MOE_OK
+               : MOE_ERR_CUDA;
+}
+
+int moe_mxfp8_quantize_rows(const void *x, int R, int K, void *codes, void *scales, void *stream) {
+    if (R < 0 || K < 1) return MOE_ERR_SHAPE;
+    if (K % 128 != 0) return MOE_ERR_UNSUPPORTED;
+    if (R == 0) return MOE_OK;
+    if (!x || !codes || !scales) return MOE_ERR_NULL;
+    if (!aligned(x, 16) || !aligned(codes, 8)) return MOE_ERR_ALIGN;
+    return launch_mx_quantize_rows(static_cast<const __nv_bfloat16 *>(x), R, K, static_cast<uint8_t *>(codes),
+                                   static_cast<uint8_t *>(scales), static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? MOE_OK
+               : MOE_ERR_CUDA;
+}
+
+int moe_forward_mxfp8(const void *x, const float *router_logits, const void *w13_q, const void *w13_sf_packed,
+                      const void *w2_q, const void *w2_sf_packed, int T, int H, int I, int E, int top_k,
+                      int local_expert_offset, int num_local_experts, void *out, void *workspace, size_t workspace_bytes,
+                      void *stream, void *const *stage_events) {
+    return forward_mx_impl(x, router_logits, w13_q, w13_sf_packed, w2_q, w2_sf_packed, T, H, I, E, top_k,
+                           local_expert_offset, num_local_experts, out, workspace, workspace_bytes,
+                           static_cast<cudaStream_t>(stream), stage_events);
+}
 
 size_t moe_workspace_bytes(int T, int H, int I, int E, int top_k) {
     if (!envelope_ok(T, H, I, E, top_k)) return 0;

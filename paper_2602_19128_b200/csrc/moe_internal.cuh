@@ -56,11 +56,11 @@ struct LocalExperts {
 };
 
 // Router + histogram, exclusive scans + tile schedule, stable scatter.  `nt_max` is the largest
-// number of rows a GEMM token tile may have (multiple of 16).  Scratch and expert_offsets are sized
-// by local.count.
+// number of rows a GEMM token tile may have (multiple of 16); tiles are sized in multiples of
+// `row_quantum` rows.  Scratch and expert_offsets are sized by local.count.
 cudaError_t launch_route(const float *logits, int T, int E, int k, LocalExperts local, int nt_max, int *topk_ids,
                          float *topk_w, int *expert_offsets, int *sorted_to_flat, int *flat_to_sorted,
-                         RouteScratch scratch, int *status, cudaStream_t stream);
+                         RouteScratch scratch, int *status, cudaStream_t stream, int row_quantum = 16);
 
 // x_perm[r,:] = x[sorted_to_flat[r] / k, :] for r < *n_rows (a device-side count, at most A)
 cudaError_t launch_gather_rows(const __nv_bfloat16 *x, const int *sorted_to_flat, const int *n_rows, int A, int k,
@@ -102,6 +102,57 @@ int launch_grouped_gemm_tc_pair(const GroupedGemmArgs &args, int slabs, cudaStre
 // args.w_scale one fp32 scale per 128 x 128 block; converter warps rebuild bf16 operand tiles in shared
 // memory and the bf16 tensor-core path does the rest.  Needs K % 128 == 0.
 int launch_grouped_gemm_tc_fp8w(const GroupedGemmArgs &args, cudaStream_t stream);
+
+// ---- MX FP8 (E4M3 codes, one E8M0 scale byte per 32 elements along K) ---------------------------------
+// The block-scaled MMA reads the scale bytes of its operands from tensor memory, where they arrive from
+// shared memory in 512-byte "atoms": the 4 scale bytes (4 x 32 = 128 K-elements, one ring slot) of 128
+// consecutive rows, row r of the atom at byte (r % 32) * 16 + (r / 32) * 4.  Scale bytes therefore live
+// in global memory in that form, one atom per (128-row group, ring slot), so a slot's scales are one
+// bulk copy.
+//   weights     : [E][feature tile][K/128][512]; a gate/up tile's rows are in the tile's interleaved order
+//   activations : [K/128][n_atoms][512], one atom per token tile.  The MX schedule cuts every expert's rows
+//                 into tiles of exactly `tile` rows (the token-tile bound, at most 128; the last may be
+//                 partial), and row i of expert e lives in atom  offsets[e] / tile + e + i / tile  at atom
+//                 row i % tile: every tile starts its own atom, so the MMA always reads its token scales
+//                 from the first column of the atom (an offset into the atom's columns is a misaligned
+//                 address for the instruction).  n_atoms = A / tile + E + 1 bounds the atom index.
+constexpr int kMxSfAtomBytes = 512;
+static inline int mx_act_sf_atoms(int A, int E, int tile) { return A / tile + E + 1; }
+static inline size_t mx_act_sf_bytes(int A, int E, int K, int tile) {
+    return (size_t)(K / 128) * mx_act_sf_atoms(A, E, tile) * kMxSfAtomBytes;
+}
+__host__ __device__ inline int mx_atom_byte(int row_in_atom, int sf) {
+    return (row_in_atom & 31) * 16 + (row_in_atom >> 5) * 4 + sf;
+}
+
+struct MxGemmArgs {
+    const uint8_t *act_q;   // [A, K] codes, rows in expert-contiguous order
+    const uint8_t *act_sf;  // activation scale atoms (layout above)
+    const uint8_t *w_q;     // [E, w_rows, K] codes
+    const uint8_t *w_sf;    // weight scale atoms (layout above)
+    void *out;              // swiglu: [A, n_out] codes of h; else [A, n_out] bf16
+    uint8_t *out_sf;        // swiglu: scale atoms of h as the next GEMM's activation (K = n_out); else unused
+    int A, K, n_out, E, w_rows, nt_max, n_atoms;
+    const int *expert_offsets, *tile_prefix, *tile_order, *tile_rows;
+    int *status;
+    bool swiglu;
+};
+// One-CTA tcgen05 kernel with kind::mxf8f6f4.block_scale.  The schedule must have been built with the row
+// quantum equal to nt_max (every tile nt_max rows, the last partial) and nt_max <= 128.  Needs K % 128 == 0.
+int launch_grouped_gemm_tc_mx(const MxGemmArgs &args, cudaStream_t stream);
+
+// xq[r,:], scale atoms <- MX quantisation of x[sorted_to_flat[r] / k, :] for r < expert_offsets[E].
+cudaError_t launch_mx_gather_quantize(const __nv_bfloat16 *x, const int *sorted_to_flat, const int *expert_offsets, int E,
+                                      int A, int k, int H, uint8_t *xq, uint8_t *x_sf, int n_atoms, int tile,
+                                      cudaStream_t stream);
+// codes[r,:], scales[r, K/32] (plain row-major) <- MX quantisation of x[r,:].
+cudaError_t launch_mx_quantize_rows(const __nv_bfloat16 *x, int R, int K, uint8_t *codes, uint8_t *scales,
+                                    cudaStream_t stream);
+// plain [E, rows, K/32] scale bytes -> weight scale atoms; gate_up: rows = 2I in [gate | up] order, tiles of
+// 64 features interleaved as the gate/up GEMM reads them; else tiles of 128 consecutive rows.
+cudaError_t launch_mx_pack_scales(const uint8_t *plain, int E, int rows, int K, bool gate_up, uint8_t *packed,
+                                  cudaStream_t stream);
+static inline size_t mx_weight_sf_bytes(int E, int rows, int K) { return (size_t)E * rows * (K / 32); }
 
 // Same contract on plain CUDA cores (validation only).
 cudaError_t launch_grouped_gemm_validation(const GroupedGemmArgs &args, cudaStream_t stream);

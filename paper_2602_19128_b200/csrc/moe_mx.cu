@@ -1,0 +1,148 @@
+// MX FP8 support kernels: quantisation of bf16 rows to E4M3 codes with one E8M0 scale byte per 32
+// elements (fused with the gather into expert-contiguous order), and the repacking of weight scale bytes
+// into the 512-byte atoms the block-scaled MMA consumes.
+//
+// Paper, Sec. 4.5: the MoE workload is an FP8 one and names FP8 packing and scaling as a cost of the
+// kernel; the granularity is not given.  This path uses the OCP Microscaling rule: for 32 values,
+// scale = 2^(floor(log2(amax)) - 8), codes = E4M3(value / scale) rounded to nearest even, saturating.
+#include <cuda_fp8.h>
+
+#include "moe_internal.cuh"
+
+namespace moe {
+namespace {
+
+// Scale byte from the largest |value| bit pattern of a block: exponent field - 8, floored at 0 (zero and
+// tiny blocks); 255 (NaN) when the block holds an infinity or a NaN.
+__device__ __forceinline__ uint32_t mx_scale_byte(uint32_t amax_bits) {
+    const uint32_t e = amax_bits >> 23;
+    if (e == 255u) return 255u;
+    return e > 8u ? e - 8u : 0u;
+}
+// 2^(127 - b): the factor that divides by the scale, exactly.
+__device__ __forceinline__ float mx_inverse_scale(uint32_t scale_byte) { return __uint_as_float((254u - scale_byte) << 23); }
+
+__device__ __forceinline__ uint32_t e4m3x2(float lo, float hi) {
+    return (uint32_t)__nv_cvt_float2_to_fp8x2(make_float2(lo, hi), __NV_SATFINITE, __NV_E4M3);
+}
+
+// Quantise the 8 bf16 values a lane holds; 4 neighbouring lanes form one block of 32.  Returns the codes
+// packed low-to-high and the block's scale byte (the same in the 4 lanes).  All 32 lanes must call.
+__device__ __forceinline__ uint2 quantize_8_of_32(const uint4 v, uint32_t &scale_byte) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    uint32_t amax = 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {  // bf16 magnitude bits widened to fp32 bit patterns compare like the values
+        amax = max(amax, (w[i] << 16) & 0x7FFFFFFFu);
+        amax = max(amax, w[i] & 0x7FFF0000u);
+    }
+    amax = max(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
+    amax = max(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
+    scale_byte = mx_scale_byte(amax);
+    if (scale_byte == 255u) return make_uint2(0x7F7F7F7Fu, 0x7F7F7F7Fu);
+    const float inv = mx_inverse_scale(scale_byte);
+    uint32_t c[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+        c[i] = e4m3x2(__uint_as_float(w[i] << 16) * inv, __uint_as_float(w[i] & 0xFFFF0000u) * inv);
+    return make_uint2(c[0] | (c[1] << 16), c[2] | (c[3] << 16));
+}
+
+// One warp per output row.  kGather: row r of the output is token sorted_to_flat[r] / k and the scale bytes
+// go to the activation atoms; otherwise row r is row r and the scale bytes are stored row-major.
+template <bool kGather>
+__global__ void __launch_bounds__(256)
+mx_quantize_rows_kernel(const uint4 *__restrict__ x, const int *__restrict__ sorted_to_flat,
+                        const int *__restrict__ expert_offsets, int E, int n_rows_plain, int k, int vec_per_row,
+                        uint2 *__restrict__ codes, uint8_t *__restrict__ scales, int n_atoms, int tile) {
+    const int lane = threadIdx.x & 31;
+    const int r = blockIdx.x * 8 + (threadIdx.x >> 5);
+    int src_row = r;
+    size_t sf_base = 0;
+    if (kGather) {
+        if (r >= expert_offsets[E]) return;  // rows actually scheduled
+        int lo = 0, hi = E;                  // the expert whose segment holds row r
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (expert_offsets[mid] <= r) lo = mid; else hi = mid;
+        }
+        const int begin = expert_offsets[lo], i = r - begin;
+        sf_base = (size_t)(begin / tile + lo + i / tile) * kMxSfAtomBytes + mx_atom_byte(i % tile, 0);
+        src_row = sorted_to_flat[r] / k;
+    } else {
+        if (r >= n_rows_plain) return;
+    }
+    const uint4 *src = x + (size_t)src_row * vec_per_row;
+    uint2 *dst = codes + (size_t)r * vec_per_row;
+    for (int v0 = 0; v0 < vec_per_row; v0 += 32) {  // uniform trip count: every lane takes part in the shuffles
+        const int v = v0 + lane;
+        const bool active = v < vec_per_row;
+        const uint4 in = active ? src[v] : make_uint4(0, 0, 0, 0);
+        uint32_t sb;
+        const uint2 q = quantize_8_of_32(in, sb);
+        if (active) {
+            dst[v] = q;
+            if ((lane & 3) == 0) {
+                const int block = v >> 2;  // 32-element block along the row; 4 blocks per 128-element slot
+                if (kGather)
+                    scales[(size_t)(block >> 2) * n_atoms * kMxSfAtomBytes + sf_base + (block & 3)] = (uint8_t)sb;
+                else
+                    scales[(size_t)r * (vec_per_row >> 2) + block] = (uint8_t)sb;
+            }
+        }
+    }
+}
+
+// One thread per (expert, tile, slot, row): moves the row's 4 scale bytes of that slot into its atom.
+__global__ void __launch_bounds__(256)
+mx_pack_scales_kernel(const uint32_t *__restrict__ plain, int E, int rows, int slots, int tiles, int gate_up,
+                      uint32_t *__restrict__ packed) {
+    const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
+    const long long total = (long long)E * tiles * slots * 128;
+    if (idx >= total) return;
+    const int m = (int)(idx % 128);
+    const int slot = (int)((idx / 128) % slots);
+    const int tile = (int)((idx / 128 / slots) % tiles);
+    const int e = (int)(idx / 128 / slots / tiles);
+    int row;
+    if (gate_up) {  // tile row m = 32q + 16 * half + j  <->  feature 64 * tile + 16q + j of the gate (half 0) or up (half 1) rows
+        const int q = m >> 5, half = (m >> 4) & 1, j = m & 15;
+        row = half * (rows / 2) + 64 * tile + 16 * q + j;
+    } else {
+        row = 128 * tile + m;
+    }
+    const uint32_t four = plain[((size_t)e * rows + row) * slots + slot];
+    packed[(((size_t)e * tiles + tile) * slots + slot) * (kMxSfAtomBytes / 4) + mx_atom_byte(m, 0) / 4] = four;
+}
+
+}  // namespace
+
+cudaError_t launch_mx_gather_quantize(const __nv_bfloat16 *x, const int *sorted_to_flat, const int *expert_offsets, int E,
+                                      int A, int k, int H, uint8_t *xq, uint8_t *x_sf, int n_atoms, int tile,
+                                      cudaStream_t stream) {
+    mx_quantize_rows_kernel<true><<<(A + 7) / 8, 256, 0, stream>>>(reinterpret_cast<const uint4 *>(x), sorted_to_flat,
+                                                                    expert_offsets, E, 0, k, H / 8,
+                                                                    reinterpret_cast<uint2 *>(xq), x_sf, n_atoms, tile);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_mx_quantize_rows(const __nv_bfloat16 *x, int R, int K, uint8_t *codes, uint8_t *scales,
+                                    cudaStream_t stream) {
+    mx_quantize_rows_kernel<false><<<(R + 7) / 8, 256, 0, stream>>>(reinterpret_cast<const uint4 *>(x), nullptr, nullptr, 0,
+                                                                     R, 1, K / 8, reinterpret_cast<uint2 *>(codes), scales,
+                                                                     0, 1);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_mx_pack_scales(const uint8_t *plain, int E, int rows, int K, bool gate_up, uint8_t *packed,
+                                  cudaStream_t stream) {
+    const int slots = K / 128;
+    const int tiles = gate_up ? rows / 2 / 64 : rows / 128;
+    const long long total = (long long)E * tiles * slots * 128;
+    mx_pack_scales_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(
+        reinterpret_cast<const uint32_t *>(plain), E, rows, slots, tiles, gate_up ? 1 : 0,
+        reinterpret_cast<uint32_t *>(packed));
+    return cudaGetLastError();
+}
+
+}  // namespace moe

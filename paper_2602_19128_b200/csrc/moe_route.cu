@@ -147,7 +147,7 @@ __device__ __forceinline__ int block_exclusive_scan_256(int value, int *warp_sum
 // per-expert running sum over chunks, exclusive scan over experts, token-tile schedule.
 // (Pointers are deliberately not __restrict__ and cross-block data is read with __ldcg: in the fused
 // kernel these arrays were written by other blocks, or are written here and read again by the scatter.)
-__device__ __forceinline__ void scan_phase(int *chunk_counts, int n_chunks, int E, int nt_max, int *expert_offsets,
+__device__ __forceinline__ void scan_phase(int *chunk_counts, int n_chunks, int E, int nt_max, int row_quantum, int *expert_offsets,
                                            int *tile_prefix, int *tile_order, int *tile_rows, int *warp_sums,
                                            int *counts, int *tiles_at) {
     const int e = threadIdx.x;
@@ -171,11 +171,12 @@ __device__ __forceinline__ void scan_phase(int *chunk_counts, int n_chunks, int 
         counts[e] = e < E ? count : -1;
         tiles_at[e] = 0;
     }
-    // token tiles of this expert: as few as fit under nt_max, evenly sized, rounded up to 16 rows
+    // token tiles of this expert: as few as fit under nt_max, evenly sized, rounded up to the row quantum
+    // (16 rows, the MMA's N granularity; 32 for the MX kernels, whose scale factors come in groups of 32 rows)
     int n_tiles = 0, rows = 0;
     if (count > 0) {
         n_tiles = (count + nt_max - 1) / nt_max;
-        rows = (((count + n_tiles - 1) / n_tiles) + 15) & ~15;
+        rows = (((count + n_tiles - 1) / n_tiles) + row_quantum - 1) / row_quantum * row_quantum;
     }
     int total_rows, total_tiles;
     const int row_start = block_exclusive_scan_256(count, warp_sums, &total_rows);  // (syncs: counts[] is visible)
@@ -201,12 +202,12 @@ __device__ __forceinline__ void scan_phase(int *chunk_counts, int n_chunks, int 
 }
 
 __global__ void __launch_bounds__(256)
-route_scan_kernel(int *chunk_counts, int n_chunks, int E, int nt_max, int *expert_offsets, int *tile_prefix,
-                  int *tile_order, int *tile_rows) {
+route_scan_kernel(int *chunk_counts, int n_chunks, int E, int nt_max, int row_quantum, int *expert_offsets,
+                  int *tile_prefix, int *tile_order, int *tile_rows) {
     __shared__ int warp_sums[8];
     __shared__ int counts[kMaxExperts], tiles_at[kMaxExperts];
-    scan_phase(chunk_counts, n_chunks, E, nt_max, expert_offsets, tile_prefix, tile_order, tile_rows, warp_sums, counts,
-               tiles_at);
+    scan_phase(chunk_counts, n_chunks, E, nt_max, row_quantum, expert_offsets, tile_prefix, tile_order, tile_rows, warp_sums,
+               counts, tiles_at);
 }
 
 // Stable scatter of one chunk (32 tokens) by one warp; next[] is that warp's per-expert cursor.
@@ -253,7 +254,7 @@ constexpr int kFusedMaxChunks = kFusedThreads / 32;
 
 __global__ void __launch_bounds__(kFusedThreads)
 route_fused_kernel(const float *__restrict__ logits, int T, int E, int k, int local_offset, int n_local, int nt_max,
-                   int *topk_ids, float *topk_w, int *chunk_counts, int *expert_offsets, int *tile_prefix,
+                   int row_quantum, int *topk_ids, float *topk_w, int *chunk_counts, int *expert_offsets, int *tile_prefix,
                    int *tile_order, int *tile_rows, int *sorted_to_flat, int *flat_to_sorted, int *done_counter) {
     __shared__ int hist[kMaxExperts], counts[kMaxExperts], tiles_at[kMaxExperts], warp_sums[8];
     __shared__ int next[kFusedMaxChunks][kMaxExperts];
@@ -268,8 +269,8 @@ route_fused_kernel(const float *__restrict__ logits, int T, int E, int k, int lo
     if (!is_last) return;
     __threadfence();
     const int n_chunks = gridDim.x;
-    scan_phase(chunk_counts, n_chunks, n_local, nt_max, expert_offsets, tile_prefix, tile_order, tile_rows, warp_sums,
-               counts, tiles_at);
+    scan_phase(chunk_counts, n_chunks, n_local, nt_max, row_quantum, expert_offsets, tile_prefix, tile_order, tile_rows,
+               warp_sums, counts, tiles_at);
     __syncthreads();  // expert_offsets and the chunk starts written above are read below (same block)
     const int warp = tid >> 5;
     if (warp < n_chunks)
@@ -341,20 +342,22 @@ int choose_nt_max(int T, int E, int k) {
 
 cudaError_t launch_route(const float *logits, int T, int E, int k, LocalExperts local, int nt_max, int *topk_ids,
                          float *topk_w, int *expert_offsets, int *sorted_to_flat, int *flat_to_sorted,
-                         RouteScratch scratch, int *status, cudaStream_t stream) {
+                         RouteScratch scratch, int *status, cudaStream_t stream, int row_quantum) {
     cudaError_t err = cudaMemsetAsync(status, 0, 256, stream);  // the status word and its padding
     if (err != cudaSuccess) return err;
     const int A = T * k;
     if (scratch.n_chunks <= kFusedMaxChunks) {
         route_fused_kernel<<<scratch.n_chunks, kFusedThreads, 0, stream>>>(
-            logits, T, E, k, local.offset, local.count, nt_max, topk_ids, topk_w, scratch.chunk_counts, expert_offsets,
+            logits, T, E, k, local.offset, local.count, nt_max, row_quantum, topk_ids, topk_w, scratch.chunk_counts,
+            expert_offsets,
             scratch.tile_prefix, scratch.tile_order, scratch.tile_rows, sorted_to_flat, flat_to_sorted,
             status + kDoneCounterInt);
         return cudaGetLastError();
     }
     route_topk_kernel<<<scratch.n_chunks, kRouteThreads, 0, stream>>>(logits, T, E, k, local.offset, local.count,
                                                                        topk_ids, topk_w, scratch.chunk_counts);
-    route_scan_kernel<<<1, 256, 0, stream>>>(scratch.chunk_counts, scratch.n_chunks, local.count, nt_max, expert_offsets,
+    route_scan_kernel<<<1, 256, 0, stream>>>(scratch.chunk_counts, scratch.n_chunks, local.count, nt_max, row_quantum,
+                                             expert_offsets,
                                              scratch.tile_prefix, scratch.tile_order, scratch.tile_rows);
     route_scatter_kernel<<<scratch.n_chunks, 32, 0, stream>>>(topk_ids, scratch.chunk_counts, expert_offsets, A,
                                                               local.count, local.offset, k, sorted_to_flat,

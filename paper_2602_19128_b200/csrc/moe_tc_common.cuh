@@ -215,6 +215,9 @@ bool encode_weight_map_2d_fp8(CUtensorMap *map, const void *w, uint64_t rows, ui
 bool encode_act_maps_k128(CUtensorMap *maps, const void *act, uint64_t rows, uint64_t K, int row_quantum);
 bool encode_weight_map_gate_up_fp8(CUtensorMap *map, const void *w13, int E, int I, int H);
 bool encode_act_maps(CUtensorMap *maps, const void *act, uint64_t rows, uint64_t K, int row_quantum);
+bool encode_mx_weight_map_2d(CUtensorMap *map, const void *w, uint64_t rows, uint64_t K);
+bool encode_mx_weight_map_gate_up(CUtensorMap *map, const void *w13, int E, int I, int H);
+bool encode_mx_act_maps(CUtensorMap *maps, const void *act, uint64_t rows, uint64_t K, int row_quantum);
 int sm_count();
 
 }  // namespace tc

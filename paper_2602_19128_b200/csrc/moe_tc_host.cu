@@ -26,17 +26,19 @@ EncodeTiledFn get_encode_fn() {
     return fn;
 }
 
+// bf16 operands and MX codes land in the 128-byte-swizzled layout the MMA reads; the FP8 codes of the
+// dequantising kernel are staged unswizzled for its converter warps.
+enum class Operand { kBf16, kCodesForConverter, kCodesForMma };
+
 bool encode(CUtensorMap *map, const void *base, int rank, const cuuint64_t *dims, const cuuint64_t *strides,
-            const cuuint32_t *box, bool fp8_codes = false) {
+            const cuuint32_t *box, Operand kind = Operand::kBf16) {
     EncodeTiledFn fn = get_encode_fn();
     if (!fn) return false;
     const cuuint32_t elem_strides[5] = {1, 1, 1, 1, 1};
-    // bf16 operands land in the 128-byte-swizzled layout the MMA reads; FP8 codes are staged unswizzled
-    // (64-byte rows) for the converter warps
-    return fn(map, fp8_codes ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank,
+    return fn(map, kind == Operand::kBf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, rank,
               const_cast<void *>(base), dims, strides, box, elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE,
-              fp8_codes ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+              kind == Operand::kCodesForConverter ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 // 2-D bf16 tensor [rows, cols] row-major; box = box_rows x 64 columns, 128-byte swizzle, zero fill.
@@ -71,7 +73,7 @@ bool encode_weight_map_2d_fp8(CUtensorMap *map, const void *w, uint64_t rows, ui
     const cuuint64_t dims[2] = {K, rows};
     const cuuint64_t strides[1] = {K};
     const cuuint32_t box[2] = {128, (cuuint32_t)kTileM};
-    return encode(map, w, 2, dims, strides, box, true);
+    return encode(map, w, 2, dims, strides, box, Operand::kCodesForConverter);
 }
 
 bool encode_weight_map_gate_up_fp8(CUtensorMap *map, const void *w13, int E, int I, int H) {
@@ -79,7 +81,33 @@ bool encode_weight_map_gate_up_fp8(CUtensorMap *map, const void *w13, int E, int
     const cuuint64_t dims[5] = {(cuuint64_t)H, 16, 2, (cuuint64_t)(I / 16), (cuuint64_t)E};
     const cuuint64_t strides[4] = {row_bytes, (cuuint64_t)I * row_bytes, 16 * row_bytes, 2 * (cuuint64_t)I * row_bytes};
     const cuuint32_t box[5] = {128, 16, 2, 4, 1};
-    return encode(map, w13, 5, dims, strides, box, true);
+    return encode(map, w13, 5, dims, strides, box, Operand::kCodesForConverter);
+}
+
+// MX operands: one byte per element, 128 K-elements (one 128-byte swizzle row) per ring slot.
+bool encode_mx_weight_map_2d(CUtensorMap *map, const void *w, uint64_t rows, uint64_t K) {
+    const cuuint64_t dims[2] = {K, rows};
+    const cuuint64_t strides[1] = {K};
+    const cuuint32_t box[2] = {128, (cuuint32_t)kTileM};
+    return encode(map, w, 2, dims, strides, box, Operand::kCodesForMma);
+}
+
+bool encode_mx_weight_map_gate_up(CUtensorMap *map, const void *w13, int E, int I, int H) {
+    const cuuint64_t row_bytes = (cuuint64_t)H;
+    const cuuint64_t dims[5] = {(cuuint64_t)H, 16, 2, (cuuint64_t)(I / 16), (cuuint64_t)E};
+    const cuuint64_t strides[4] = {row_bytes, (cuuint64_t)I * row_bytes, 16 * row_bytes, 2 * (cuuint64_t)I * row_bytes};
+    const cuuint32_t box[5] = {128, 16, 2, 4, 1};
+    return encode(map, w13, 5, dims, strides, box, Operand::kCodesForMma);
+}
+
+bool encode_mx_act_maps(CUtensorMap *maps, const void *act, uint64_t rows, uint64_t K, int row_quantum) {
+    for (int i = 0; i < kNumActMaps; ++i) {
+        const cuuint64_t dims[2] = {K, rows};
+        const cuuint64_t strides[1] = {K};
+        const cuuint32_t box[2] = {128, (cuuint32_t)row_quantum * (cuuint32_t)(i + 1)};
+        if (!encode(&maps[i], act, 2, dims, strides, box, Operand::kCodesForMma)) return false;
+    }
+    return true;
 }
 
 // Activation maps whose box spans 128 K-elements: the tensor [rows, K] viewed as [K/64][rows][64], box

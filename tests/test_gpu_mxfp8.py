@@ -1,0 +1,191 @@
+"""GPU parity of the MX FP8 path (E4M3 codes, E8M0 scale bytes, block-scaled tensor-core MMA) against the oracle:
+the row quantiser and the scale repacking bit for bit, the quantised token rows bit for bit, the codes of h up to
+the few decisions that sit on a rounding boundary, and the layer output within the workload's tolerance."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2602_19128_b200 as moe
+from oracle import moe_oracle
+from paper_2602_19128_b200.inputs import bf16_bits, make_mxfp8_inputs
+from tests.gpu_common import assert_close_out, assert_routing_exact, bf16_to_f64
+
+pytestmark = pytest.mark.gpu
+
+TABLE = torch.arange(256, dtype=torch.uint8).view(torch.float8_e4m3fn).float().numpy().astype(np.float64)
+
+
+def atom_byte(r, sf):
+    return (r % 32) * 16 + (r // 32) * 4 + sf
+
+
+def unpack_act_scales(atoms: np.ndarray, offsets: np.ndarray, n_blocks: int, tile: int) -> np.ndarray:
+    """Scale atoms [K/128, n_atoms, 512] -> plain [rows, K/32] for the rows of every expert segment."""
+    E = len(offsets) - 1
+    rows = offsets[E]
+    plain = np.zeros((rows, n_blocks), np.uint8)
+    for e in range(E):
+        begin = offsets[e]
+        for i in range(offsets[e + 1] - begin):
+            a = begin // tile + e + i // tile
+            for b in range(n_blocks):
+                plain[begin + i, b] = atoms[b // 4, a, atom_byte(i % tile, b % 4)]
+    return plain
+
+
+def run_mx(inp, local_offset=0):
+    T, H = inp["x"].shape
+    n_local, I2, _ = inp["w13_q"].shape
+    E = inp["router_logits"].shape[1]
+    I, k = I2 // 2, inp["top_k"]
+    w13_sf = moe.moe_mxfp8_pack_scales(inp["w13_s"], gate_up=True)
+    w2_sf = moe.moe_mxfp8_pack_scales(inp["w2_s"], gate_up=False)
+    ws = moe.alloc_workspace(moe.moe_mxfp8_workspace_bytes(T, H, I, E, k), "cuda")
+    ws.fill_(0xFF)
+    out = torch.full((T, H), float("nan"), dtype=torch.bfloat16, device="cuda")
+    moe.moe_forward_mxfp8(inp["x"], inp["router_logits"], inp["w13_q"], w13_sf, inp["w2_q"], w2_sf, k, out, ws,
+                          local_expert_offset=local_offset)
+    status = moe.moe_last_status(ws)
+    assert status == moe.MOE_OK, moe.moe_status_string(status)
+    return out, moe.mx_workspace_views(ws, T, H, I, E, k)
+
+
+def oracle_mx(inp, intermediates=False, prec="f32"):
+    return moe_oracle.get(prec).forward_mxfp8(bf16_bits(inp["x"]), inp["router_logits"].cpu().numpy(),
+                                             inp["w13_q"].cpu().numpy(), inp["w13_s"].cpu().numpy(),
+                                             inp["w2_q"].cpu().numpy(), inp["w2_s"].cpu().numpy(), inp["top_k"],
+                                             intermediates=intermediates)
+
+
+@pytest.mark.parametrize("R,K,scale", [(1, 128, 1.0), (37, 384, 1.0), (300, 7168, 3.0), (64, 256, 1e-30), (9, 128, 1e30),
+                                       (17, 128, 1e-38)])
+def test_row_quantiser_is_bit_exact(R, K, scale):
+    g = torch.Generator().manual_seed(R)
+    x = (torch.randn((R, K), generator=g) * torch.exp2(torch.randint(-6, 6, (R, K // 32, 1), generator=g).float())
+         .expand(R, K // 32, 32).reshape(R, K) * scale).to(torch.bfloat16)
+    x[0, :32] = 0                                    # an all-zero block
+    if R > 2:
+        x[1, 5] = float("inf")                       # non-finite blocks
+        x[2, 40] = float("nan")
+        x[2, 100] = -0.0
+    codes, scales = moe.moe_mxfp8_quantize_rows(x.cuda())
+    torch.cuda.synchronize()
+    want_c, want_s = moe_oracle.get("f32").mx_quantize(x.float().numpy())
+    assert np.array_equal(scales.cpu().numpy(), want_s)
+    assert np.array_equal(codes.cpu().numpy(), want_c)
+
+
+@pytest.mark.parametrize("E,rows,K,gate_up", [(2, 256, 128, True), (3, 512, 384, True), (2, 128, 256, False), (4, 384, 512, False)])
+def test_scale_repacking_is_the_documented_permutation(E, rows, K, gate_up):
+    g = torch.Generator().manual_seed(0)
+    plain = torch.randint(0, 255, (E, rows, K // 32), dtype=torch.uint8, generator=g)
+    packed = moe.moe_mxfp8_pack_scales(plain.cuda(), gate_up=gate_up).cpu().numpy()
+    p = plain.numpy()
+    slots = K // 128
+    tiles = rows // 128
+    got = packed.reshape(E, tiles, slots, 512)
+    I = rows // 2
+    for e in range(E):
+        for t in range(tiles):
+            for m in range(128):
+                if gate_up:
+                    q, half, j = m // 32, (m // 16) % 2, m % 16
+                    row = half * I + 64 * t + 16 * q + j
+                else:
+                    row = 128 * t + m
+                for s in range(slots):
+                    for sf in range(4):
+                        assert got[e, t, s, atom_byte(m, sf)] == p[e, row, 4 * s + sf]
+
+
+# T, H, I, E, k, skew: token-tile bounds 32 / 64 / 128, several tiles per expert
+CASES = [
+    (16, 256, 512, 8, 2, False),
+    (1, 128, 128, 4, 1, False),
+    (128, 384, 128, 256, 8, False),   # decode-like
+    (200, 256, 384, 8, 2, False),     # ~50 rows per expert
+    (300, 128, 128, 64, 4, True),     # skewed, empty experts, several tiles for the popular ones
+    (700, 256, 256, 4, 2, False),     # ~350 rows per expert: three tiles of up to 128 rows, second atoms
+    (96, 128, 256, 8, 8, False),
+    (513, 128, 128, 2, 1, False),     # ~256 rows per expert: full 128-row tiles and a ragged last one
+]
+
+
+@pytest.mark.parametrize("T,H,I,E,k,skew", CASES)
+def test_mxfp8_forward_matches_oracle(T, H, I, E, k, skew):
+    inp = make_mxfp8_inputs(dict(T=T, H=H, I=I, E=E, top_k=k, skew=skew), seed=0, device="cuda")
+    out, views = run_mx(inp)
+    o = moe_oracle.get("f32")
+    ids, w = o.route(inp["router_logits"].cpu().numpy(), k)
+    off, s2f, f2s = o.permute(ids, E)
+    assert_routing_exact(views, ids, w, off, s2f, f2s)
+
+    # token rows: gathered and quantised exactly as the oracle quantises x
+    xc, xs = o.mx_quantize(inp["x"].float().cpu().numpy())
+    tok = s2f // k
+    assert np.array_equal(views["x_q"].cpu().numpy(), xc[tok])
+    assert np.array_equal(unpack_act_scales(views["x_sf"].cpu().numpy(), off, H // 32, views["tile_rows"]), xs[tok])
+
+    ref, h_pre, h_q, h_s = oracle_mx(inp, intermediates=True)
+    # h: the same codes and scale bytes except where fp32 summation order moves a value across a rounding
+    # boundary; a differing code must still be a valid quantisation of the oracle's h (within one step)
+    got_q = views["h_q"].cpu().numpy()
+    got_s = unpack_act_scales(views["h_sf"].cpu().numpy(), off, I // 32, views["tile_rows"])
+    same = (got_q == h_q[s2f]) & (np.repeat(got_s, 32, axis=1) == np.repeat(h_s[s2f], 32, axis=1))
+    assert same.mean() > 0.98, same.mean()
+    got_h = TABLE[got_q] * np.repeat(np.exp2(got_s.astype(np.float64) - 127), 32, axis=1)
+    scale = np.repeat(np.exp2(got_s.astype(np.float64) - 127), 32, axis=1)
+    step = scale * np.maximum(np.abs(TABLE[got_q]), 2.0 ** -6) * 2.0 ** -3
+    step = np.where(np.abs(TABLE[got_q]) == 448, 64 * scale, step)   # the top binade saturates: [448, 512) -> 448
+    assert np.all(np.abs(got_h - h_pre[s2f]) <= 1.01 * step + 1e-30)
+
+    assert_close_out(bf16_to_f64(out), ref, "mxfp8 out")
+
+
+def test_mxfp8_local_experts():
+    cfg = dict(T=160, H=256, I=128, E=16, top_k=4, skew=False)
+    full = make_mxfp8_inputs(cfg, seed=3, device="cuda")
+    lo, n = 4, 8
+    inp = dict(full)
+    for key in ("w13_q", "w13_s", "w2_q", "w2_s"):
+        inp[key] = full[key][lo:lo + n].contiguous()
+    out, views = run_mx(inp, local_offset=lo)
+    # the oracle with the other experts' weights zeroed: their assignments contribute nothing
+    z = dict(full)
+    for key in ("w2_q",):
+        z[key] = full[key].clone()
+        z[key][:lo] = 0
+        z[key][lo + n:] = 0
+    ref = oracle_mx(z)
+    assert_close_out(bf16_to_f64(out), ref, "mxfp8 local out")
+    assert views["expert_offsets"][n].item() == int(((views["topk_ids"] >= lo) & (views["topk_ids"] < lo + n)).sum())
+
+
+def test_mxfp8_non_finite_token_poisons_only_itself():
+    inp = make_mxfp8_inputs(dict(T=8, H=128, I=128, E=2, top_k=1, skew=False), seed=5, device="cuda")
+    inp["x"][3, 17] = float("inf")
+    out, _ = run_mx(inp)
+    got = out.float().cpu().numpy()
+    assert np.all(np.isnan(got[3]))
+    assert np.all(np.isfinite(np.delete(got, 3, axis=0)))
+
+
+def test_mxfp8_rejects_shapes_outside_its_envelope():
+    assert moe.moe_mxfp8_workspace_bytes(8, 128, 64, 2, 1) == 0   # I must be a multiple of 128
+    inp = make_mxfp8_inputs(dict(T=8, H=128, I=128, E=2, top_k=1, skew=False), seed=1, device="cuda")
+    ws = moe.alloc_workspace(1 << 20, "cuda")
+    out = torch.empty((8, 128), dtype=torch.bfloat16, device="cuda")
+    sf13 = moe.moe_mxfp8_pack_scales(inp["w13_s"], True)
+    sf2 = moe.moe_mxfp8_pack_scales(inp["w2_s"], False)
+    st = moe.moe_forward_mxfp8(inp["x"], inp["router_logits"], inp["w13_q"], sf13, inp["w2_q"], sf2, 1, out, ws[:1024],
+                               check=False)
+    assert st == -5  # MOE_ERR_WORKSPACE
+    st = moe.moe_forward_mxfp8(inp["x"], inp["router_logits"], inp["w13_q"], None, inp["w2_q"], sf2, 1, out, ws, check=False)
+    assert st == -1  # MOE_ERR_NULL
+
+
+def test_mxfp8_repeated_calls_are_deterministic():
+    inp = make_mxfp8_inputs(dict(T=300, H=256, I=256, E=16, top_k=4, skew=True), seed=2, device="cuda")
+    a, _ = run_mx(inp)
+    b, _ = run_mx(inp)
+    assert torch.equal(a.view(torch.int16), b.view(torch.int16))
