@@ -29,7 +29,7 @@ ROOT = Path(__file__).resolve().parent
 sys.path.insert(0, str(ROOT))
 
 from paper_2602_19128_b200.inputs import (CONFIGS, LOCAL_CONFIGS, bf16_bits, make_inputs,  # noqa: E402
-                                          quantize_fp8_blocks)
+                                          quantize_fp8_blocks, quantize_mxfp8)
 
 CONFIGS = dict(CONFIGS, **LOCAL_CONFIGS)  # the five workloads plus the local-expert-subset shapes
 
@@ -217,18 +217,30 @@ def run_ours(args):
     out = torch.empty((T, H), dtype=torch.bfloat16, device=dev)
     ws = moe.alloc_workspace(moe.moe_workspace_bytes(T, H, I, E, k), dev)
     fp8 = args.weights == "fp8"
+    mx = args.weights == "mxfp8"
+    if mx:  # MX FP8: E4M3 codes + one E8M0 scale byte per 32 elements, scale bytes repacked once; bf16 originals dropped
+        ws = moe.alloc_workspace(moe.moe_mxfp8_workspace_bytes(T, H, I, E, k), dev)
+        w13, s13 = quantize_mxfp8(w13)
+        w2, s2 = quantize_mxfp8(w2)
+        inp["w13"], inp["w2"] = None, None
+        w13_sf, w2_sf = moe.moe_mxfp8_pack_scales(s13, gate_up=True), moe.moe_mxfp8_pack_scales(s2, gate_up=False)
+        torch.cuda.synchronize()
+        del s13, s2
     if fp8:  # FP8 (E4M3) codes + one fp32 scale per 128 x 128 block; the bf16 originals are dropped
         if n_local != E:
             raise SystemExit("--weights fp8 covers the whole-layer workloads")
         w13, w13_scale = quantize_fp8_blocks(w13)
         w2, w2_scale = quantize_fp8_blocks(w2)
         inp["w13"], inp["w2"] = None, None
-    bytes_per_weight = 1 if fp8 else 2
-    weight_bytes = (w13.numel() + w2.numel()) * bytes_per_weight
+    bytes_per_weight = 1 if fp8 else (1 + 1 / 32) if mx else 2
+    weight_bytes = int((w13.numel() + w2.numel()) * bytes_per_weight)
     need_flush = weight_bytes < 2 * L2_BYTES
 
     def forward(events=None):
-        if fp8:
+        if mx:
+            moe.moe_forward_mxfp8(x, logits, w13, w13_sf, w2, w2_sf, k, out, ws, stage_events=events,
+                                  local_expert_offset=local_offset)
+        elif fp8:
             moe.moe_forward_fp8w(x, logits, w13, w13_scale, w2, w2_scale, k, out, ws, stage_events=events)
         elif events is None:
             moe.moe_forward_local(x, logits, w13, w2, k, local_offset, out, ws)
@@ -269,7 +281,7 @@ def run_ours(args):
     status = moe.moe_last_status(ws)
     if status != moe.MOE_OK:
         raise SystemExit(f"device status {status}: {moe.moe_status_string(status)}")
-    views = moe.workspace_views(ws, T, H, I, E, k)
+    views = moe.mx_workspace_views(ws, T, H, I, E, k) if mx else moe.workspace_views(ws, T, H, I, E, k)
     counts = torch.diff(views["expert_offsets"][:n_local + 1]).cpu().numpy()
     rows_scheduled = int(counts.sum())  # = T*k unless only a subset of the experts is resident
     n_active = int((counts > 0).sum())
@@ -281,7 +293,12 @@ def run_ours(args):
     x_stage, l_stage = torch.empty_like(x), torch.empty_like(logits)
 
     def host_step():
-        if fp8:  # no host-buffer entry point for FP8 weights: the same copies, issued here on the same stream
+        if mx:  # no host-buffer entry point for the FP8 variants: the same copies, issued here on the same stream
+            x_stage.copy_(xh, non_blocking=True)
+            l_stage.copy_(lh, non_blocking=True)
+            moe.moe_forward_mxfp8(x_stage, l_stage, w13, w13_sf, w2, w2_sf, k, out, ws, local_expert_offset=local_offset)
+            oh.copy_(out, non_blocking=True)
+        elif fp8:
             x_stage.copy_(xh, non_blocking=True)
             l_stage.copy_(lh, non_blocking=True)
             moe.moe_forward_fp8w(x_stage, l_stage, w13, w13_scale, w2, w2_scale, k, out, ws)
@@ -324,18 +341,20 @@ def run_ours(args):
     t_gemm1 = stage_ms["gemm1_swiglu"] * 1e-3
     bound = BOUND[args.config]
     if bound == "hbm":
-        algorithmic = n_active * 2 * I * H * bytes_per_weight  # bytes of the active experts' w13, read once
+        algorithmic = int(n_active * 2 * I * H * bytes_per_weight)  # bytes of the active experts' w13, read once
         achieved = algorithmic / t_gemm1 / 1e9
         peak, unit = peaks["hbm_gbs"], "GB/s"
     else:
         algorithmic = 4.0 * A * H * I  # useful flops of the gate and up projections
         achieved = algorithmic / t_gemm1 / 1e12
         peak, unit = peaks["tflops_sustained"], "TFLOP/s"
+        if mx:  # 8-bit operands: the measured bf16 peak times the nominal fp8 / bf16 ratio
+            peak *= 2
     step_s = total_ms * 1e-3 / args.steps
-    active_weight_bytes = n_active * 3 * I * H * bytes_per_weight
+    active_weight_bytes = int(n_active * 3 * I * H * bytes_per_weight)
     roofline = dict(bound=bound, kernel="gate/up GEMM (grouped_gemm_tc*_kernel<swiglu>)", achieved=achieved, peak=peak,
                     unit=unit, frac=achieved / peak, peak_source=f"of {peaks['source']}",
-                    traffic=None if fp8 else NCU_TRAFFIC_BYTES.get(args.config), algorithmic_per_launch=algorithmic,
+                    traffic=None if (fp8 or mx) else NCU_TRAFFIC_BYTES.get(args.config), algorithmic_per_launch=algorithmic,
                     kernel_ms=stage_ms["gemm1_swiglu"])
     layer = dict(stage_ms={n: round(v, 5) for n, v in stage_ms.items()}, n_active_experts=n_active,
                  rows_per_expert_min=int(counts.min()), rows_per_expert_max=int(counts.max()),
@@ -345,14 +364,15 @@ def run_ours(args):
                  useful_tflops_frac_burst=6.0 * A * H * I / step_s / 1e12 / peaks["tflops_burst"])
 
     cpu_baseline = None
-    if world == 1 and not args.no_cpu_baseline and n_local == E and not fp8:
+    if world == 1 and not args.no_cpu_baseline and n_local == E and not fp8 and not mx:
         cpu_baseline = time_oracle(args.config, inp, budget_s=15.0)
 
     line = dict(metric=METRIC, value=aggregate_tokens_per_s(world, T, args.steps, total_ms), unit=UNIT, n_gpus=world,
                 steps=args.steps, warmup=max(args.warmup, 3), ms_per_step=total_ms / args.steps, higher_is_better=True,
-                scaling="weak", vs_baseline=None, dtype="bf16", data="synthetic",
+                scaling="weak", vs_baseline=None, dtype="mxfp8" if mx else "bf16", data="synthetic",
                 config=dict(workload=args.config, T=T, H=H, I=I, E=E, top_k=k, resident_experts=n_local,
-                            weights="fp8 e4m3 codes + fp32 scale per 128x128 block" if fp8 else "bf16",
+                            weights="fp8 e4m3 codes + fp32 scale per 128x128 block" if fp8 else
+                            "mxfp8: e4m3 codes + e8m0 scale per 32 elements, activations quantised on the fly" if mx else "bf16",
                             parallelism=f"replicas x{world}",
                             l2="flushed between steps" if need_flush else "weights larger than L2, no flush",
                             seed=args.seed),
@@ -375,8 +395,9 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--config", choices=list(CONFIGS), default="mixtral")
     ap.add_argument("--shape", default=None, help="custom T,H,I,E,top_k instead of a named workload (profiling)")
-    ap.add_argument("--weights", choices=["bf16", "fp8"], default="bf16",
-                    help="fp8: expert weights as E4M3 codes with one fp32 scale per 128 x 128 block (moe_forward_fp8w)")
+    ap.add_argument("--weights", choices=["bf16", "fp8", "mxfp8"], default="bf16",
+                    help="fp8: expert weights as E4M3 codes with one fp32 scale per 128 x 128 block (moe_forward_fp8w); "
+                         "mxfp8: weights and activations in MX FP8 on the block-scaled MMA (moe_forward_mxfp8)")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -227,13 +227,15 @@ typedef struct {
     size_t total_bytes;
     size_t status, topk_ids, topk_weights, expert_offsets, sorted_to_flat, flat_to_sorted, route_scratch; /* as moe_workspace_layout_t */
     size_t x_q;   /* uint8 [A,H]  codes of the token rows in expert-contiguous order */
-    size_t x_sf;  /* scale atoms of x_q: [H/128][sf_atoms][512]; row i of expert e is row i % tile_rows of atom
-                     expert_offsets[e] / tile_rows + e + i / tile_rows (one atom per token tile) */
+    size_t x_sf;  /* scale atoms of x_q: [H/128][sf_atoms][512].  Row i of expert e belongs to token tile
+                     n = expert_offsets[e] / tile_rows + e + i / tile_rows, as its row r = i % tile_rows; a tile owns
+                     ceil(tile_rows / 128) atoms, and the row's scales are in atom n * ceil(tile_rows / 128) + r / 128
+                     at atom row r % 128 */
     size_t h_q;   /* uint8 [A,I]  codes of h */
     size_t h_sf;  /* scale atoms of h_q: [I/128][sf_atoms][512], same row-to-atom rule */
     size_t y;     /* bf16 [A,H] */
-    size_t sf_atoms;  /* a count, not an offset: atoms per K-slot in x_sf / h_sf (A / tile_rows + E + 1) */
-    size_t tile_rows; /* a count: rows per token tile of this problem (32, 64 or 128) */
+    size_t sf_atoms;  /* a count, not an offset: atoms per K-slot in x_sf / h_sf */
+    size_t tile_rows; /* a count: rows per token tile of this problem (32, 64, 128 or 240) */
 } moe_mxfp8_workspace_layout_t;
 
 /* Host-only, pure.  Workspace bytes of moe_forward_mxfp8; 0 outside the envelope (moe_forward's, plus I % 128 == 0). */
@@ -261,7 +263,7 @@ MOE_API int moe_mxfp8_quantize_rows(const void *x, int R, int K, void *codes, vo
  *   workspace  at least moe_mxfp8_workspace_bytes bytes, 256-byte aligned (layout: moe_mxfp8_workspace_layout)
  *   stage_events  NULL, or MOE_NUM_STAGE_EVENTS events recorded as by moe_forward_staged
  * Launches the same number of kernels as moe_forward (the gather also quantises).  Token tiles are at most
- * 128 rows.  Errors as moe_forward; a block of x holding an infinity or NaN makes that token's output NaN. */
+ * 240 rows (128 when H is not a multiple of 256).  Errors as moe_forward; a block of x holding an infinity or NaN makes that token's output NaN. */
 MOE_API int moe_forward_mxfp8(const void *x, const float *router_logits, const void *w13_q, const void *w13_sf_packed,
                               const void *w2_q, const void *w2_sf_packed, int T, int H, int I, int E, int top_k,
                               int local_expert_offset, int num_local_experts, void *out, void *workspace,

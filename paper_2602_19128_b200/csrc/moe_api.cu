@@ -150,16 +150,18 @@ int forward_impl(const void *x, const float *logits, const void *w13, const void
 // ---- MX FP8 ---------------------------------------------------------------------------------------------
 bool mx_envelope_ok(long long T, int H, int I, int E, int k) { return envelope_ok(T, H, I, E, k) && I % 128 == 0; }
 
-// Token-tile bound of the MX path: the MX kernel keeps scale columns next to two accumulators in tensor
-// memory, and one scale atom covers 128 rows.
-int mx_tile_rows(int T, int E, int k) {
+// Token-tile rows of the MX path.  Scale columns sit next to the two accumulators in tensor memory, so the
+// largest tile is 240 rows (2 * 240 + 32 columns); only the CTA-pair kernel has that instance, and its down
+// projection needs H to be a multiple of its 256-row tile.
+int mx_tile_rows(int T, int H, int E, int k) {
     const int nt = choose_nt_max(T, E, k);
-    return nt > 128 ? 128 : nt;
+    if (nt <= 128) return nt;
+    return H % 256 == 0 ? 240 : 128;
 }
 
 void fill_mx_layout(int T, int H, int I, int E, int k, moe_mxfp8_workspace_layout_t *L) {
     const size_t A = (size_t)T * k;
-    const int tile = mx_tile_rows(T, E, k);
+    const int tile = mx_tile_rows(T, H, E, k);
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t at = off; off += align_up(bytes, 256); return at; };
     L->status = take(kStatusInts * sizeof(int));
@@ -238,10 +240,13 @@ int forward_mx_impl(const void *x, const float *logits, const void *w13_q, const
     g2.act_q = h_q; g2.act_sf = h_sf; g2.w_q = static_cast<const uint8_t *>(w2_q);
     g2.w_sf = static_cast<const uint8_t *>(w2_sf); g2.out = y; g2.out_sf = nullptr;
     g2.K = I; g2.n_out = H; g2.w_rows = H; g2.swiglu = false;
-    int st = launch_grouped_gemm_tc_mx(g1, stream);
+    auto run = [&](const MxGemmArgs &g) {
+        return grouped_gemm_tc_mx_pair_applies(g) ? launch_grouped_gemm_tc_mx_pair(g, stream) : launch_grouped_gemm_tc_mx(g, stream);
+    };
+    int st = run(g1);
     if (st != MOE_OK) return st;
     if (!mark(3)) return MOE_ERR_CUDA;
-    st = launch_grouped_gemm_tc_mx(g2, stream);
+    st = run(g2);
     if (st != MOE_OK) return st;
     if (!mark(4)) return MOE_ERR_CUDA;
     if (launch_combine(y, wts, f2s, T, k, H, static_cast<__nv_bfloat16 *>(out), stream) != cudaSuccess)

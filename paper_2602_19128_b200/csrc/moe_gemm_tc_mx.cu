@@ -22,77 +22,23 @@
 //    the largest magnitude over a block of 32 features comes from a 16-lane shuffle reduction and one
 //    exchange with the neighbouring warp through shared memory, then each lane scales and encodes its
 //    values and the scale byte goes straight into the atom layout the down GEMM loads.
-#include <cuda_fp8.h>
-
-#include "moe_tc_common.cuh"
+#include "moe_mx_tc.cuh"
 
 namespace moe {
 namespace {
 
 using namespace tc;
+using namespace mxtc;
 
-constexpr int kMxSlotK = 128;                          // K elements = bytes per operand row per ring slot
-constexpr int kMxSlotABytes = kTileM * kMxSlotK;       // 16 KiB
 constexpr int kMxSfBBytes = kMxSfAtomBytes;            // one atom per token tile (at most 128 rows)
-constexpr int kTmemColsMx = 512;
-
-struct MxParams {
-    void *out;
-    uint8_t *out_sf;
-    const uint8_t *w_sf, *act_sf;
-    const int *expert_offsets, *tile_prefix, *tile_order, *tile_rows;
-    int *status;
-    int E, n_k_blocks, n_out, w_rows, n_feature_tiles, n_atoms, tile_stride;
-};
-
-struct MxTile {
-    int e, f, row0, n_valid;
-    int atom;    // the tile's activation scale atom
-};
-
-__device__ __forceinline__ MxTile decode_mx_tile(int tile, const MxParams &p) {
-    int lo = 0, hi = p.E;
-    while (hi - lo > 1) {
-        const int mid = (lo + hi) >> 1;
-        if (p.tile_prefix[mid] * p.n_feature_tiles <= tile) lo = mid; else hi = mid;
-    }
-    MxTile t;
-    t.e = p.tile_order[lo];
-    const int first = p.tile_prefix[lo], n_tok_tiles = p.tile_prefix[lo + 1] - first;
-    const int local = tile - first * p.n_feature_tiles;
-    t.f = local / n_tok_tiles;
-    const int j = local - t.f * n_tok_tiles;
-    const int rows = p.tile_rows[t.e];
-    const int begin = p.expert_offsets[t.e], count = p.expert_offsets[t.e + 1] - begin;
-    t.row0 = begin + j * rows;  // rows == p.tile_stride for every expert of an MX schedule
-    t.n_valid = min(rows, count - j * rows);
-    t.atom = begin / p.tile_stride + t.e + j;
-    return t;
-}
 
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
                  : "memory");
 }
-
-// Shared-memory descriptor of one scale atom: 32 rows of 16 bytes, no swizzle, 8-row groups 128 bytes apart.
-__device__ __forceinline__ uint64_t smem_desc_sf_atom(uint32_t smem_addr) {
-    uint64_t d = 0;
-    d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
-    d |= (uint64_t)1 << 16;
-    d |= (uint64_t)(128 >> 4) << 32;
-    d |= (uint64_t)1 << 46;
-    return d;
-}
 __device__ __forceinline__ void tmem_copy_sf_atom(uint32_t taddr, uint64_t desc) {
     asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(desc) : "memory");
-}
-// Block-scaled instruction descriptor: E4M3 A and B (format 0), both K-major, E8M0 scales, M = 128, N = n,
-// scale byte `sf` of each row (the K-block within the slot) for both operands.
-__device__ __forceinline__ uint32_t instr_desc_mx(int n, int sf) {
-    return ((uint32_t)sf << 4) | ((uint32_t)(n >> 3) << 17) | (1u << 23) | ((uint32_t)(kTileM >> 4) << 24) |
-           ((uint32_t)sf << 29);
 }
 __device__ __forceinline__ void umma_mx(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                         uint32_t accumulate, uint32_t sfa_tmem, uint32_t sfb_tmem) {
@@ -105,30 +51,6 @@ __device__ __forceinline__ void umma_mx(uint32_t d_tmem, uint64_t a_desc, uint64
 }
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-
-// OR of `flag` over the 128 epilogue threads (named barrier 1), so that they leave their loop together.
-__device__ __forceinline__ bool epilogue_any(bool flag) {
-    uint32_t r;
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t"
-        "setp.ne.u32 q, %1, 0;\n\t"
-        "bar.red.or.pred p, 1, 128, q;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(r)
-        : "r"((uint32_t)flag)
-        : "memory");
-    return r != 0;
-}
-// Barrier of the two epilogue warps (64 threads) that share a block of 32 features.
-__device__ __forceinline__ void pair_sync(int pair) {
-    asm volatile("bar.sync %0, 64;" ::"r"(2 + pair) : "memory");
-}
-
-__device__ __forceinline__ uint32_t mx_scale_byte(uint32_t amax_bits) {
-    const uint32_t e = amax_bits >> 23;
-    if (e == 255u) return 255u;
-    return e > 8u ? e - 8u : 0u;
 }
 
 template <int NT_MAX, int STAGES>
@@ -251,7 +173,7 @@ grouped_gemm_tc_mx_kernel(const __grid_constant__ TensorMaps maps, const MxParam
                     const uint64_t b_desc = smem_desc_k_major_sw128(base + L::kB + stage * L::kSlotBBytes);
 #pragma unroll
                     for (int kk = 0; kk < kMxSlotK / 32; ++kk)  // 32 K-elements = 32 bytes = 2 descriptor units
-                        umma_mx(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, instr_desc_mx(n_mma, kk), (kb | kk) != 0,
+                        umma_mx(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, instr_desc_mx(kTileM, n_mma, kk), (kb | kk) != 0,
                                 sfa_tmem, sfb_tmem);
                     umma_commit(bar_empty + stage * 8);
                     if (kb == p.n_k_blocks - 1) umma_commit(bar_acc_full + acc * 8);
@@ -280,49 +202,11 @@ grouped_gemm_tc_mx_kernel(const __grid_constant__ TensorMaps maps, const MxParam
             tcgen05_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + acc * NT_MAX;
             if (SWIGLU) {
-                const int hi = lane >> 4, j = lane & 15;
-                uint8_t *dst = static_cast<uint8_t *>(p.out) + (size_t)t.row0 * p.n_out + t.f * (kTileM / 2) + q * 16 + j;
-                // scale bytes of h: K-slot f/2 of the down GEMM, block (f%2)*2 + q/2 within the slot
-                uint8_t *sf_dst = p.out_sf + (size_t)(t.f >> 1) * p.n_atoms * kMxSfAtomBytes + ((t.f & 1) * 2 + (q >> 1));
-                for (int c0 = 0; c0 < n_mma; c0 += 16) {
-                    float v[16];
-                    tmem_load_16(taddr + c0, v);
-                    float hv[8];
-                    uint32_t mag[8];
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const float other = __shfl_xor_sync(0xffffffffu, hi ? v[i] : v[8 + i], 16);
-                        const float g = hi ? other : v[i];
-                        const float u = hi ? v[8 + i] : other;
-                        hv[i] = swiglu(g, u);
-                        mag[i] = __float_as_uint(hv[i]) & 0x7FFFFFFFu;  // magnitudes compare as integers; NaN and inf on top
-                    }
-#pragma unroll
-                    for (int off = 8; off >= 1; off >>= 1)
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) mag[i] = max(mag[i], __shfl_xor_sync(0xffffffffu, mag[i], off));
-                    buf ^= 1;
-                    if (j == 0) {
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) amax_s[(buf * 4 + q) * 16 + hi * 8 + i] = mag[i];
-                    }
-                    pair_sync(q >> 1);
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const uint32_t block_mag = max(mag[i], amax_s[(buf * 4 + (q ^ 1)) * 16 + hi * 8 + i]);
-                        const uint32_t sb = mx_scale_byte(block_mag);
-                        const int col = c0 + hi * 8 + i;
-                        if (col < t.n_valid) {
-                            uint8_t code = 0x7F;
-                            if (sb != 255u)
-                                code = (uint8_t)__nv_cvt_float_to_fp8(hv[i] * __uint_as_float((254u - sb) << 23), __NV_SATFINITE,
-                                                                      __NV_E4M3);
-                            dst[(size_t)col * p.n_out] = code;
-                            if ((q & 1) == 0 && j == 0)
-                                sf_dst[(size_t)t.atom * kMxSfAtomBytes + mx_atom_byte(col, 0)] = (uint8_t)sb;
-                        }
-                    }
-                }
+                uint8_t *dst = static_cast<uint8_t *>(p.out) + (size_t)t.row0 * p.n_out + t.f * (kTileM / 2) + q * 16 + (lane & 15);
+                // scale bytes of h: features 64f + 16q.. lie in block 2f + q/2 = K-slot block/4 of the down GEMM
+                const int block = 2 * t.f + (q >> 1);
+                uint8_t *sf_dst = p.out_sf + ((size_t)(block >> 2) * p.n_atoms + t.atom) * kMxSfAtomBytes + (block & 3);
+                drain_swiglu_mx(taddr, n_mma, t.n_valid, dst, (size_t)p.n_out, sf_dst, amax_s, buf, q, lane);
             } else {
                 __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(p.out) + (size_t)t.row0 * p.n_out + t.f * kTileM + q * 32 + lane;
                 for (int c0 = 0; c0 < n_mma; c0 += 16) {
@@ -403,6 +287,7 @@ int launch_grouped_gemm_tc_mx(const MxGemmArgs &a, cudaStream_t stream) {
     p.n_feature_tiles = a.n_out / features_per_tile;
     p.n_atoms = a.n_atoms;
     p.tile_stride = a.nt_max;
+    p.atoms_per_tile = 1;
 
     const long long max_token_tiles = (long long)(a.A < a.E ? a.A : a.E) + a.A / a.nt_max;
     const long long max_tiles = max_token_tiles * p.n_feature_tiles;

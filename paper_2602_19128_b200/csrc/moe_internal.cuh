@@ -110,14 +110,15 @@ int launch_grouped_gemm_tc_fp8w(const GroupedGemmArgs &args, cudaStream_t stream
 // in global memory in that form, one atom per (128-row group, ring slot), so a slot's scales are one
 // bulk copy.
 //   weights     : [E][feature tile][K/128][512]; a gate/up tile's rows are in the tile's interleaved order
-//   activations : [K/128][n_atoms][512], one atom per token tile.  The MX schedule cuts every expert's rows
-//                 into tiles of exactly `tile` rows (the token-tile bound, at most 128; the last may be
-//                 partial), and row i of expert e lives in atom  offsets[e] / tile + e + i / tile  at atom
-//                 row i % tile: every tile starts its own atom, so the MMA always reads its token scales
-//                 from the first column of the atom (an offset into the atom's columns is a misaligned
-//                 address for the instruction).  n_atoms = A / tile + E + 1 bounds the atom index.
+//   activations : [K/128][n_atoms][512], whole atoms per token tile.  The MX schedule cuts every expert's
+//                 rows into tiles of exactly `tile` rows (the token-tile bound: 32, 64, 128 or 240; the last
+//                 may be partial).  Token tile j of expert e is tile number  offsets[e] / tile + e + j  and
+//                 owns ceil(tile / 128) consecutive atoms; its row r sits in atom r / 128 of those, at atom
+//                 row r % 128.  Every tile thus starts a fresh atom, and the MMA reads its token scales from
+//                 the first column of the atom (an odd column offset is a misaligned address for the
+//                 instruction).  n_atoms = (A / tile + E + 1) * ceil(tile / 128) bounds the atom index.
 constexpr int kMxSfAtomBytes = 512;
-static inline int mx_act_sf_atoms(int A, int E, int tile) { return A / tile + E + 1; }
+static inline int mx_act_sf_atoms(int A, int E, int tile) { return (A / tile + E + 1) * ((tile + 127) / 128); }
 static inline size_t mx_act_sf_bytes(int A, int E, int K, int tile) {
     return (size_t)(K / 128) * mx_act_sf_atoms(A, E, tile) * kMxSfAtomBytes;
 }
@@ -140,6 +141,10 @@ struct MxGemmArgs {
 // One-CTA tcgen05 kernel with kind::mxf8f6f4.block_scale.  The schedule must have been built with the row
 // quantum equal to nt_max (every tile nt_max rows, the last partial) and nt_max <= 128.  Needs K % 128 == 0.
 int launch_grouped_gemm_tc_mx(const MxGemmArgs &args, cudaStream_t stream);
+// The same GEMM on CTA pairs (cta_group::2, 256 x N tiles): nt_max 128 or 240, and n_out a multiple of the
+// pair tile (128 features of h, 256 output rows of the down projection).
+bool grouped_gemm_tc_mx_pair_applies(const MxGemmArgs &args);
+int launch_grouped_gemm_tc_mx_pair(const MxGemmArgs &args, cudaStream_t stream);
 
 // xq[r,:], scale atoms <- MX quantisation of x[sorted_to_flat[r] / k, :] for r < expert_offsets[E].
 cudaError_t launch_mx_gather_quantize(const __nv_bfloat16 *x, const int *sorted_to_flat, const int *expert_offsets, int E,

@@ -67,7 +67,8 @@ mx_quantize_rows_kernel(const uint4 *__restrict__ x, const int *__restrict__ sor
             if (expert_offsets[mid] <= r) lo = mid; else hi = mid;
         }
         const int begin = expert_offsets[lo], i = r - begin;
-        sf_base = (size_t)(begin / tile + lo + i / tile) * kMxSfAtomBytes + mx_atom_byte(i % tile, 0);
+        const int atoms_per_tile = (tile + 127) / 128, tr = i % tile;  // row tr of token tile i / tile of this expert
+        sf_base = (size_t)((begin / tile + lo + i / tile) * atoms_per_tile + tr / 128) * kMxSfAtomBytes + mx_atom_byte(tr % 128, 0);
         src_row = sorted_to_flat[r] / k;
     } else {
         if (r >= n_rows_plain) return;

@@ -1,7 +1,7 @@
 // Host-side helpers of the tcgen05 grouped GEMMs: TMA tensor-map encoding (through the driver entry
 // point, so the library links against no driver stub and loads on a machine without a GPU) and the
 // SM count.
-#include "moe_tc_common.cuh"
+#include "moe_mx_tc.cuh"
 
 #include <mutex>
 
@@ -128,6 +128,19 @@ bool encode_act_maps(CUtensorMap *maps, const void *act, uint64_t rows, uint64_t
     return true;
 }
 
+// Scale atoms as a 2-D tensor of 32-bit words: [n_atoms][128 words], box = atoms_per_box whole atoms, unswizzled.
+bool encode_scale_atoms(CUtensorMap *map, const void *atoms, uint64_t n_atoms, uint32_t atoms_per_box) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {kMxSfAtomBytes / 4, n_atoms};
+    const cuuint64_t strides[1] = {kMxSfAtomBytes};
+    const cuuint32_t box[2] = {kMxSfAtomBytes / 4, atoms_per_box};
+    const cuuint32_t elem_strides[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void *>(atoms), dims, strides, box, elem_strides,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 int sm_count() {
     static int cached[64] = {0};
     int dev = 0;
@@ -141,4 +154,10 @@ int sm_count() {
 }
 
 }  // namespace tc
+
+namespace mxtc {
+bool encode_mx_scale_map(CUtensorMap *map, const void *atoms, uint64_t n_atoms, uint32_t atoms_per_box) {
+    return tc::encode_scale_atoms(map, atoms, n_atoms, atoms_per_box);
+}
+}  // namespace mxtc
 }  // namespace moe

@@ -27,9 +27,10 @@ def unpack_act_scales(atoms: np.ndarray, offsets: np.ndarray, n_blocks: int, til
     for e in range(E):
         begin = offsets[e]
         for i in range(offsets[e + 1] - begin):
-            a = begin // tile + e + i // tile
+            apt, r = (tile + 127) // 128, i % tile
+            a = (begin // tile + e + i // tile) * apt + r // 128
             for b in range(n_blocks):
-                plain[begin + i, b] = atoms[b // 4, a, atom_byte(i % tile, b % 4)]
+                plain[begin + i, b] = atoms[b // 4, a, atom_byte(r % 128, b % 4)]
     return plain
 
 
@@ -107,7 +108,11 @@ CASES = [
     (300, 128, 128, 64, 4, True),     # skewed, empty experts, several tiles for the popular ones
     (700, 256, 256, 4, 2, False),     # ~350 rows per expert: three tiles of up to 128 rows, second atoms
     (96, 128, 256, 8, 8, False),
-    (513, 128, 128, 2, 1, False),     # ~256 rows per expert: full 128-row tiles and a ragged last one
+    (513, 128, 128, 2, 1, False),     # ~256 rows per expert; H not a multiple of 256: one-CTA kernel, 128-row tiles
+    (513, 256, 128, 2, 1, False),     # the same on CTA pairs: 240-row tiles (two scale atoms) and a ragged one
+    (1000, 512, 384, 4, 2, False),    # ~500 rows per expert: three pair tiles each, several feature tiles
+    (130, 256, 256, 4, 2, False),     # 128-row pair tiles (one atom each)
+    (300, 256, 128, 16, 4, True),     # the same, skewed: popular experts spill into a second tile
 ]
 
 
