@@ -48,50 +48,72 @@ __device__ __forceinline__ uint2 quantize_8_of_32(const uint4 v, uint32_t &scale
     return make_uint2(c[0] | (c[1] << 16), c[2] | (c[3] << 16));
 }
 
-// One warp per output row.  kGather: row r of the output is token sorted_to_flat[r] / k and the scale bytes
-// go to the activation atoms; otherwise row r is row r and the scale bytes are stored row-major.
+// A row is cut into 256-element segments (32 lanes x 8 elements = 8 blocks of 32) and shared by
+// `warps_per_row` warps, warp s taking segments s, s + warps_per_row, ...: small batches spread one row
+// over many warps so the device is not left idle, large ones keep one warp per row.  kGather: row r of
+// the output is token sorted_to_flat[r] / k and the scale bytes go to the activation atoms; otherwise
+// row r is row r and the scale bytes are stored row-major.
 template <bool kGather>
 __global__ void __launch_bounds__(256)
 mx_quantize_rows_kernel(const uint4 *__restrict__ x, const int *__restrict__ sorted_to_flat,
                         const int *__restrict__ expert_offsets, int E, int n_rows_plain, int k, int vec_per_row,
-                        uint2 *__restrict__ codes, uint8_t *__restrict__ scales, int n_atoms, int tile) {
+                        int warps_per_row, uint2 *__restrict__ codes, uint8_t *__restrict__ scales, int n_atoms, int tile) {
     const int lane = threadIdx.x & 31;
-    const int r = blockIdx.x * 8 + (threadIdx.x >> 5);
+    const long long w = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int r = (int)(w / warps_per_row), first_seg = (int)(w % warps_per_row);
     int src_row = r;
     size_t sf_base = 0;
     if (kGather) {
         if (r >= expert_offsets[E]) return;  // rows actually scheduled
-        int lo = 0, hi = E;                  // the expert whose segment holds row r
-        while (hi - lo > 1) {
-            const int mid = (lo + hi) >> 1;
-            if (expert_offsets[mid] <= r) lo = mid; else hi = mid;
-        }
-        const int begin = expert_offsets[lo], i = r - begin;
+        // the expert whose segment holds row r = last e with offsets[e] <= r: a 32-way search in two steps
+        // (offsets are non-decreasing, so the lanes that satisfy the test form a prefix)
+        const int stride = (E + 31) / 32;
+        const int coarse = __popc(__ballot_sync(0xffffffffu, lane * stride < E && expert_offsets[lane * stride] <= r)) - 1;
+        const int cand = coarse * stride + lane;
+        const int e = coarse * stride + __popc(__ballot_sync(0xffffffffu, lane < stride && cand < E && expert_offsets[cand] <= r)) - 1;
+        const int begin = expert_offsets[e], i = r - begin;
         const int atoms_per_tile = (tile + 127) / 128, tr = i % tile;  // row tr of token tile i / tile of this expert
-        sf_base = (size_t)((begin / tile + lo + i / tile) * atoms_per_tile + tr / 128) * kMxSfAtomBytes + mx_atom_byte(tr % 128, 0);
+        sf_base = (size_t)((begin / tile + e + i / tile) * atoms_per_tile + tr / 128) * kMxSfAtomBytes + mx_atom_byte(tr % 128, 0);
         src_row = sorted_to_flat[r] / k;
     } else {
         if (r >= n_rows_plain) return;
     }
     const uint4 *src = x + (size_t)src_row * vec_per_row;
-    uint2 *dst = codes + (size_t)r * vec_per_row;
-    for (int v0 = 0; v0 < vec_per_row; v0 += 32) {  // uniform trip count: every lane takes part in the shuffles
-        const int v = v0 + lane;
-        const bool active = v < vec_per_row;
-        const uint4 in = active ? src[v] : make_uint4(0, 0, 0, 0);
-        uint32_t sb;
-        const uint2 q = quantize_8_of_32(in, sb);
-        if (active) {
-            dst[v] = q;
-            if ((lane & 3) == 0) {
-                const int block = v >> 2;  // 32-element block along the row; 4 blocks per 128-element slot
-                if (kGather)
-                    scales[(size_t)(block >> 2) * n_atoms * kMxSfAtomBytes + sf_base + (block & 3)] = (uint8_t)sb;
-                else
-                    scales[(size_t)r * (vec_per_row >> 2) + block] = (uint8_t)sb;
+    constexpr int kInFlight = 4;  // independent 16-byte loads per lane before the first is used
+    const int n_segs = (vec_per_row + 31) / 32;
+    for (int s0 = first_seg; s0 < n_segs; s0 += kInFlight * warps_per_row) {  // uniform over the warp
+        uint4 in[kInFlight];
+#pragma unroll
+        for (int u = 0; u < kInFlight; ++u) {
+            const int v = (s0 + u * warps_per_row) * 32 + lane;
+            in[u] = (s0 + u * warps_per_row < n_segs && v < vec_per_row) ? src[v] : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int u = 0; u < kInFlight; ++u) {
+            if (s0 + u * warps_per_row >= n_segs) break;  // uniform
+            const int v = (s0 + u * warps_per_row) * 32 + lane;
+            uint32_t sb;
+            const uint2 q = quantize_8_of_32(in[u], sb);  // every lane takes part in the shuffles
+            if (v < vec_per_row) {
+                codes[(size_t)r * vec_per_row + v] = q;
+                if ((lane & 3) == 0) {
+                    const int block = v >> 2;  // 32-element block along the row; 4 blocks per 128-element slot
+                    if (kGather)
+                        scales[(size_t)(block >> 2) * n_atoms * kMxSfAtomBytes + sf_base + (block & 3)] = (uint8_t)sb;
+                    else
+                        scales[(size_t)r * (vec_per_row >> 2) + block] = (uint8_t)sb;
+                }
             }
         }
     }
+}
+
+// Warps per row: enough warps to fill the device (about 16 per SM slot) when there are few rows.
+int mx_quantize_warps_per_row(long long rows, int n_segs) {
+    const long long target = 32768;
+    long long per_row = rows > 0 ? (target + rows - 1) / rows : 1;
+    if (per_row > n_segs) per_row = n_segs;
+    return per_row < 1 ? 1 : (int)per_row;
 }
 
 // One thread per (expert, tile, slot, row): moves the row's 4 scale bytes of that slot into its atom.
@@ -121,17 +143,21 @@ mx_pack_scales_kernel(const uint32_t *__restrict__ plain, int E, int rows, int s
 cudaError_t launch_mx_gather_quantize(const __nv_bfloat16 *x, const int *sorted_to_flat, const int *expert_offsets, int E,
                                       int A, int k, int H, uint8_t *xq, uint8_t *x_sf, int n_atoms, int tile,
                                       cudaStream_t stream) {
-    mx_quantize_rows_kernel<true><<<(A + 7) / 8, 256, 0, stream>>>(reinterpret_cast<const uint4 *>(x), sorted_to_flat,
-                                                                    expert_offsets, E, 0, k, H / 8,
-                                                                    reinterpret_cast<uint2 *>(xq), x_sf, n_atoms, tile);
+    const int segs = mx_quantize_warps_per_row(A, (H / 8 + 31) / 32);
+    const long long warps = (long long)A * segs;
+    mx_quantize_rows_kernel<true><<<(unsigned)((warps + 7) / 8), 256, 0, stream>>>(
+        reinterpret_cast<const uint4 *>(x), sorted_to_flat, expert_offsets, E, 0, k, H / 8, segs,
+        reinterpret_cast<uint2 *>(xq), x_sf, n_atoms, tile);
     return cudaGetLastError();
 }
 
 cudaError_t launch_mx_quantize_rows(const __nv_bfloat16 *x, int R, int K, uint8_t *codes, uint8_t *scales,
                                     cudaStream_t stream) {
-    mx_quantize_rows_kernel<false><<<(R + 7) / 8, 256, 0, stream>>>(reinterpret_cast<const uint4 *>(x), nullptr, nullptr, 0,
-                                                                     R, 1, K / 8, reinterpret_cast<uint2 *>(codes), scales,
-                                                                     0, 1);
+    const int segs = mx_quantize_warps_per_row(R, (K / 8 + 31) / 32);
+    const long long warps = (long long)R * segs;
+    mx_quantize_rows_kernel<false><<<(unsigned)((warps + 7) / 8), 256, 0, stream>>>(
+        reinterpret_cast<const uint4 *>(x), nullptr, nullptr, 0, R, 1, K / 8, segs, reinterpret_cast<uint2 *>(codes), scales,
+        0, 1);
     return cudaGetLastError();
 }
 
