@@ -167,6 +167,30 @@ def time_oracle(cfg_name: str, inp: dict, budget_s: float):
                        f"{t_probe:.2f} s wall")
 
 
+def time_oracle_mx(cfg_name: str, x, logits, w13_q, s13, w2_q, s2, k: int, budget_s: float):
+    """Times the oracle's MX FP8 layer, as it stands, on the first tokens of the workload (all weights on the host)."""
+    from oracle import moe_oracle
+    o = moe_oracle.get("f32")
+    cores = o.num_threads
+    host = [t.cpu().numpy() for t in (w13_q, s13, w2_q, s2)]
+    xb, lg = bf16_bits(x), logits.cpu().numpy()
+
+    def run(n):
+        t0 = time.perf_counter()
+        o.forward_mxfp8(xb[:n], lg[:n], *host, k)
+        return time.perf_counter() - t0
+
+    n = min(x.shape[0], cores)
+    t = run(n)
+    rounds = max(1, min(64, int(budget_s / max(t, 1e-3))))
+    if min(x.shape[0], cores * rounds) > n:
+        n = min(x.shape[0], cores * rounds)
+        t = run(n)
+    return dict(value=n / t, unit=UNIT, cores=cores, kind="oracle",
+                sample=f"first {n} of {x.shape[0]} tokens of '{cfg_name}' (all top-k experts of each), float oracle, "
+                       f"MX FP8 layer, {t:.2f} s wall")
+
+
 def run_reference(args):
     """The reference arm: the CPU oracle on the host cores (rank 0 only)."""
     if int(os.environ.get("RANK", "0")) != 0:
@@ -225,6 +249,7 @@ def run_ours(args):
         inp["w13"], inp["w2"] = None, None
         w13_sf, w2_sf = moe.moe_mxfp8_pack_scales(s13, gate_up=True), moe.moe_mxfp8_pack_scales(s2, gate_up=False)
         torch.cuda.synchronize()
+        mx_plain_scales = (s13, s2) if (w13.numel() + w2.numel()) <= (4 << 30) else None  # for the CPU baseline leg
         del s13, s2
     if fp8:  # FP8 (E4M3) codes + one fp32 scale per 128 x 128 block; the bf16 originals are dropped
         if n_local != E:
@@ -366,6 +391,8 @@ def run_ours(args):
     cpu_baseline = None
     if world == 1 and not args.no_cpu_baseline and n_local == E and not fp8 and not mx:
         cpu_baseline = time_oracle(args.config, inp, budget_s=15.0)
+    if world == 1 and not args.no_cpu_baseline and n_local == E and mx and mx_plain_scales is not None:
+        cpu_baseline = time_oracle_mx(args.config, x, logits, w13, mx_plain_scales[0], w2, mx_plain_scales[1], k, 15.0)
 
     line = dict(metric=METRIC, value=aggregate_tokens_per_s(world, T, args.steps, total_ms), unit=UNIT, n_gpus=world,
                 steps=args.steps, warmup=max(args.warmup, 3), ms_per_step=total_ms / args.steps, higher_is_better=True,

@@ -19,6 +19,7 @@
 //     per token atom.  2 * 240 + 32 = 512 is why the largest tile is 240 rows and not 256.
 // Every wait is bounded; on expiry both CTAs are told, every role stops and tensor memory is released.
 #include "moe_mx_tc.cuh"
+#include "moe_tc_pair.cuh"
 
 namespace moe {
 namespace {
@@ -33,38 +34,6 @@ struct MxPairMaps {
     CUtensorMap w_sf, act_sf;  // scale atoms
 };
 
-__device__ __forceinline__ uint32_t cluster_ctarank() {
-    uint32_t r;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-    return r;
-}
-__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
-    uint32_t r;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
-    return r;
-}
-__device__ __forceinline__ void cluster_sync_all() {
-    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
-__device__ __forceinline__ void store_cluster_u32(uint32_t cluster_addr, uint32_t v) {
-    asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(cluster_addr), "r"(v) : "memory");
-}
-__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, int c0, int c1, uint32_t bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar)
-        : "memory");
-}
-__device__ __forceinline__ void tma_load_5d_pair(uint32_t dst, const CUtensorMap *map, int c0, int c1, int c2, int c3,
-                                                 int c4, uint32_t bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.5d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
-        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(bar)
-        : "memory");
-}
 // In both CTAs of the pair: one scale atom from that CTA's shared memory to its tensor memory.
 __device__ __forceinline__ void tmem_copy_sf_atom_pair(uint32_t taddr, uint64_t desc) {
     asm volatile("tcgen05.cp.cta_group::2.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(desc) : "memory");
@@ -78,19 +47,6 @@ __device__ __forceinline__ void umma_mx_pair(uint32_t d_tmem, uint64_t a_desc, u
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem)
         : "memory");
 }
-__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
-    const uint16_t both = 3;
-    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-                 ::"r"(bar), "h"(both)
-                 : "memory");
-}
-__device__ __forceinline__ bool pair_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, uint32_t peer_abort,
-                                          int *status, int site) {
-    const bool ok = mbar_wait(bar, parity, abort_flag, status, site);
-    if (!ok) store_cluster_u32(peer_abort, 1u);
-    return ok;
-}
-
 template <int NT_MAX, int STAGES>
 struct MxPairSmem {
     static constexpr int kAtomsB = (NT_MAX + 127) / 128;

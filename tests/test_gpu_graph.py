@@ -1,0 +1,65 @@
+"""The layer captured into a CUDA graph: the library never synchronises, allocates or reads device memory on the
+host, so its launch sequence can be recorded once and replayed; a replay on new inputs must equal a plain call."""
+import pytest
+import torch
+
+import paper_2602_19128_b200 as moe
+from paper_2602_19128_b200.inputs import make_inputs, make_mxfp8_inputs
+
+pytestmark = pytest.mark.gpu
+
+
+def _capture(call):
+    """Runs `call(stream)` once eagerly on a side stream, then records it into a graph on that stream."""
+    g = torch.cuda.CUDAGraph()
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        call(s)
+        s.synchronize()
+        with torch.cuda.graph(g, stream=s):
+            call(torch.cuda.current_stream())
+    torch.cuda.synchronize()
+    return g
+
+
+@pytest.mark.parametrize("cfg", [dict(T=16, H=256, I=512, E=8, top_k=2, skew=False),
+                                 dict(T=1500, H=256, I=128, E=32, top_k=4, skew=True)])  # fused and three-kernel router
+def test_bf16_layer_replays_from_a_graph(cfg):
+    a, b = make_inputs(cfg, seed=1, device="cuda"), make_inputs(cfg, seed=2, device="cuda")
+    T, H, I, E, k = cfg["T"], cfg["H"], cfg["I"], cfg["E"], cfg["top_k"]
+    x, logits = a["x"].clone(), a["router_logits"].clone()
+    out = torch.empty((T, H), dtype=torch.bfloat16, device="cuda")
+    ws = moe.alloc_workspace(moe.moe_workspace_bytes(T, H, I, E, k), "cuda")
+    g = _capture(lambda s: moe.moe_forward(x, logits, a["w13"], a["w2"], k, out, ws, stream=s))
+    for inp in (b, a):  # the graph reads whatever the captured buffers hold at replay time
+        x.copy_(inp["x"])
+        logits.copy_(inp["router_logits"])
+        g.replay()
+        torch.cuda.synchronize()
+        assert moe.moe_last_status(ws) == moe.MOE_OK
+        ref = torch.empty_like(out)
+        ws2 = moe.alloc_workspace(moe.moe_workspace_bytes(T, H, I, E, k), "cuda")
+        moe.moe_forward(inp["x"], inp["router_logits"], a["w13"], a["w2"], k, ref, ws2)
+        torch.cuda.synchronize()
+        assert torch.equal(out.view(torch.int16), ref.view(torch.int16))
+
+
+def test_mxfp8_layer_replays_from_a_graph():
+    cfg = dict(T=300, H=256, I=256, E=16, top_k=4, skew=True)
+    a, b = make_mxfp8_inputs(cfg, seed=1, device="cuda"), make_inputs(cfg, seed=2, device="cuda")
+    T, H, I, E, k = cfg["T"], cfg["H"], cfg["I"], cfg["E"], cfg["top_k"]
+    sf13, sf2 = moe.moe_mxfp8_pack_scales(a["w13_s"], True), moe.moe_mxfp8_pack_scales(a["w2_s"], False)
+    x, logits = a["x"].clone(), a["router_logits"].clone()
+    out = torch.empty((T, H), dtype=torch.bfloat16, device="cuda")
+    ws = moe.alloc_workspace(moe.moe_mxfp8_workspace_bytes(T, H, I, E, k), "cuda")
+    g = _capture(lambda s: moe.moe_forward_mxfp8(x, logits, a["w13_q"], sf13, a["w2_q"], sf2, k, out, ws, stream=s))
+    x.copy_(b["x"])
+    logits.copy_(b["router_logits"])
+    g.replay()
+    torch.cuda.synchronize()
+    assert moe.moe_last_status(ws) == moe.MOE_OK
+    ref = torch.empty_like(out)
+    ws2 = moe.alloc_workspace(moe.moe_mxfp8_workspace_bytes(T, H, I, E, k), "cuda")
+    moe.moe_forward_mxfp8(b["x"], b["router_logits"], a["w13_q"], sf13, a["w2_q"], sf2, k, ref, ws2)
+    torch.cuda.synchronize()
+    assert torch.equal(out.view(torch.int16), ref.view(torch.int16))
