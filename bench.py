@@ -318,12 +318,9 @@ def run_ours(args):
     x_stage, l_stage = torch.empty_like(x), torch.empty_like(logits)
 
     def host_step():
-        if mx:  # no host-buffer entry point for the FP8 variants: the same copies, issued here on the same stream
-            x_stage.copy_(xh, non_blocking=True)
-            l_stage.copy_(lh, non_blocking=True)
-            moe.moe_forward_mxfp8(x_stage, l_stage, w13, w13_sf, w2, w2_sf, k, out, ws, local_expert_offset=local_offset)
-            oh.copy_(out, non_blocking=True)
-        elif fp8:
+        if mx:
+            moe.moe_forward_mxfp8_host(xh, lh, w13, w13_sf, w2, w2_sf, k, oh, ws, local_expert_offset=local_offset)
+        elif fp8:  # no host-buffer entry point for this variant: the same copies, issued here on the same stream
             x_stage.copy_(xh, non_blocking=True)
             l_stage.copy_(lh, non_blocking=True)
             moe.moe_forward_fp8w(x_stage, l_stage, w13, w13_scale, w2, w2_scale, k, out, ws)

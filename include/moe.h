@@ -234,6 +234,7 @@ typedef struct {
     size_t h_q;   /* uint8 [A,I]  codes of h */
     size_t h_sf;  /* scale atoms of h_q: [I/128][sf_atoms][512], same row-to-atom rule */
     size_t y;     /* bf16 [A,H] */
+    size_t staging; /* used only by moe_forward_mxfp8_host: device copies of x, logits, out */
     size_t sf_atoms;  /* a count, not an offset: atoms per K-slot in x_sf / h_sf */
     size_t tile_rows; /* a count: rows per token tile of this problem (32, 64, 128 or 240) */
 } moe_mxfp8_workspace_layout_t;
@@ -268,6 +269,15 @@ MOE_API int moe_forward_mxfp8(const void *x, const float *router_logits, const v
                               const void *w2_q, const void *w2_sf_packed, int T, int H, int I, int E, int top_k,
                               int local_expert_offset, int num_local_experts, void *out, void *workspace,
                               size_t workspace_bytes, void *stream, void *const *stage_events);
+
+/* moe_forward_mxfp8 for a caller whose activations live in HOST memory, as moe_forward_host: x_host [T,H] bf16,
+ * router_logits_host [T,E] f32 and out_host [T,H] bf16 are HOST pointers (pinned memory makes the copies
+ * asynchronous); the weight codes and packed scales stay DEVICE pointers.  Enqueues the two host-to-device
+ * copies, the layer and the device-to-host copy on `stream` and returns without synchronising. */
+MOE_API int moe_forward_mxfp8_host(const void *x_host, const float *router_logits_host, const void *w13_q,
+                                   const void *w13_sf_packed, const void *w2_q, const void *w2_sf_packed, int T, int H,
+                                   int I, int E, int top_k, int local_expert_offset, int num_local_experts,
+                                   void *out_host, void *workspace, size_t workspace_bytes, void *stream);
 
 /* moe_forward_local (local_expert_offset = 0, num_local_experts = E for the whole layer) for a caller
  * whose activations live in HOST memory: x_host [T,H] bf16 and router_logits_host [T,E] f32 are HOST

@@ -540,17 +540,14 @@ static void expert_ffn_row_mx(const uint8_t *xq, const uint8_t *xs, const uint8_
     }
 }
 
-/* The whole layer in MX FP8.  x [T,H] bf16, router_logits [T,E] f32, w13_q [E,2I,H] codes, w13_s [E,2I,H/32]
- * scale bytes, w2_q [E,H,I], w2_s [E,H,I/32] -> out [T,H] REAL.  Optional (may be NULL), per flat assignment
- * a = t*k + j:  h_pre [A,I] REAL = h before quantisation, h_q [A,I] codes, h_s [A,I/32] scale bytes.
- * H and I must be multiples of 32. */
-int moe_oracle_forward_mxfp8(const uint16_t *x, const float *router_logits, const uint8_t *w13_q, const uint8_t *w13_s,
-                             const uint8_t *w2_q, const uint8_t *w2_s, int T, int H, int I, int E, int k, REAL *out,
-                             REAL *h_pre, uint8_t *h_q, uint8_t *h_s) {
-    if (T < 0 || H < 32 || I < 32 || H % 32 || I % 32 || E < 1 || k < 1 || k > E) return ORACLE_ERR_ARG;
+/* The MX FP8 layer for a chosen list of tokens, with the experts given as tables of per-expert pointers
+ * (an entry may be NULL when no listed token routes to it).  out [n_tokens,H] REAL; the optional
+ * intermediates are indexed by (position in `tokens`) * k + j. */
+static int forward_tokens_mx(const uint16_t *x, const float *router_logits, const uint8_t *const *w13q, const uint8_t *const *w13s,
+                             const uint8_t *const *w2q, const uint8_t *const *w2s, int T, int H, int I, int E, int k,
+                             const int32_t *tokens, int n_tokens, REAL *out, REAL *h_pre, uint8_t *h_q, uint8_t *h_s) {
+    if (T < 0 || H < 32 || I < 32 || H % 32 || I % 32 || E < 1 || k < 1 || k > E || n_tokens < 0) return ORACLE_ERR_ARG;
     int status = ORACLE_OK;
-    const size_t n13 = (size_t)2 * I * H, n2 = (size_t)H * I;
-    const size_t s13 = (size_t)2 * I * (H / 32), s2 = (size_t)H * (I / 32);
 #pragma omp parallel
     {
         REAL *p = (REAL *)malloc(sizeof(REAL) * (size_t)E);
@@ -567,17 +564,27 @@ int moe_oracle_forward_mxfp8(const uint16_t *x, const float *router_logits, cons
             status = ORACLE_ERR_NOMEM;
         } else {
 #pragma omp for schedule(dynamic, 1)
-            for (int t = 0; t < T; ++t) {
-                REAL *o = out + (size_t)t * H;
+            for (int n_i = 0; n_i < n_tokens; ++n_i) {
+                const int t = tokens[n_i];
+                REAL *o = out + (size_t)n_i * H;
                 for (int n = 0; n < H; ++n) o[n] = 0;
+                if (t < 0 || t >= T) {
+#pragma omp critical
+                    status = ORACLE_ERR_ARG;
+                    continue;
+                }
                 route_token(router_logits + (size_t)t * E, E, k, ids, w, p, taken);
                 for (int c = 0; c < H; ++c) xr[c] = bf16_to_real(x[(size_t)t * H + c]);
                 for (int b = 0; b < H / 32; ++b) mx_quantize_block(xr + 32 * b, 32, xq + 32 * b, xs + b);
                 for (int j = 0; j < k; ++j) {
                     const int e = ids[j];
-                    expert_ffn_row_mx(xq, xs, w13_q + e * n13, w13_s + e * s13, w2_q + e * n2, w2_s + e * s2, H, I, y, s,
-                                      hq, hs);
-                    const size_t a = (size_t)t * k + j;
+                    if (!w13q[e] || !w13s[e] || !w2q[e] || !w2s[e]) {
+#pragma omp critical
+                        status = ORACLE_ERR_MISSING_EXPERT;
+                        continue;
+                    }
+                    expert_ffn_row_mx(xq, xs, w13q[e], w13s[e], w2q[e], w2s[e], H, I, y, s, hq, hs);
+                    const size_t a = (size_t)n_i * k + j;
                     if (h_pre) memcpy(h_pre + a * I, s, sizeof(REAL) * (size_t)I);
                     if (h_q) memcpy(h_q + a * I, hq, (size_t)I);
                     if (h_s) memcpy(h_s + a * (I / 32), hs, (size_t)(I / 32));
@@ -587,5 +594,39 @@ int moe_oracle_forward_mxfp8(const uint16_t *x, const float *router_logits, cons
         }
         free(p); free(taken); free(ids); free(w); free(s); free(y); free(xr); free(xq); free(xs); free(hq); free(hs);
     }
+    return status;
+}
+
+int moe_oracle_forward_mxfp8_sampled(const uint16_t *x, const float *router_logits, const uint8_t *const *w13q,
+                                     const uint8_t *const *w13s, const uint8_t *const *w2q, const uint8_t *const *w2s, int T,
+                                     int H, int I, int E, int k, const int32_t *tokens, int n_tokens, REAL *out) {
+    return forward_tokens_mx(x, router_logits, w13q, w13s, w2q, w2s, T, H, I, E, k, tokens, n_tokens, out, NULL, NULL, NULL);
+}
+
+/* The whole layer in MX FP8.  x [T,H] bf16, router_logits [T,E] f32, w13_q [E,2I,H] codes, w13_s [E,2I,H/32]
+ * scale bytes, w2_q [E,H,I], w2_s [E,H,I/32] -> out [T,H] REAL.  Optional (may be NULL), per flat assignment
+ * a = t*k + j:  h_pre [A,I] REAL = h before quantisation, h_q [A,I] codes, h_s [A,I/32] scale bytes.
+ * H and I must be multiples of 32. */
+int moe_oracle_forward_mxfp8(const uint16_t *x, const float *router_logits, const uint8_t *w13_q, const uint8_t *w13_s,
+                             const uint8_t *w2_q, const uint8_t *w2_s, int T, int H, int I, int E, int k, REAL *out,
+                             REAL *h_pre, uint8_t *h_q, uint8_t *h_s) {
+    if (T < 0 || H < 32 || I < 32 || H % 32 || I % 32 || E < 1 || k < 1 || k > E) return ORACLE_ERR_ARG;
+    const size_t n13 = (size_t)2 * I * H, n2 = (size_t)H * I;
+    const size_t s13 = (size_t)2 * I * (H / 32), s2 = (size_t)H * (I / 32);
+    const uint8_t **tab = (const uint8_t **)malloc(sizeof(void *) * 4 * (size_t)E);
+    int32_t *tokens = (int32_t *)malloc(sizeof(int32_t) * (size_t)(T > 0 ? T : 1));
+    int status = ORACLE_ERR_NOMEM;
+    if (tab && tokens) {
+        for (int e = 0; e < E; ++e) {
+            tab[e] = w13_q + e * n13;
+            tab[E + e] = w13_s + e * s13;
+            tab[2 * E + e] = w2_q + e * n2;
+            tab[3 * E + e] = w2_s + e * s2;
+        }
+        for (int t = 0; t < T; ++t) tokens[t] = t;
+        status = forward_tokens_mx(x, router_logits, tab, tab + E, tab + 2 * E, tab + 3 * E, T, H, I, E, k, tokens, T, out,
+                                   h_pre, h_q, h_s);
+    }
+    free(tab); free(tokens);
     return status;
 }

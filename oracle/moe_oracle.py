@@ -52,7 +52,7 @@ class Oracle:
         for fn in ("moe_oracle_route", "moe_oracle_permute", "moe_oracle_expert_ffn", "moe_oracle_forward",
                    "moe_oracle_forward_sampled", "moe_oracle_sorted_intermediates", "moe_oracle_forward_local",
                    "moe_oracle_permute_local", "moe_oracle_forward_fp8w", "moe_oracle_mx_quantize",
-                   "moe_oracle_forward_mxfp8"):
+                   "moe_oracle_forward_mxfp8", "moe_oracle_forward_mxfp8_sampled"):
             getattr(self.lib, fn).restype = ctypes.c_int
         self.lib.moe_oracle_e4m3_decode.restype = ctypes.c_float
         self.lib.moe_oracle_e4m3_decode.argtypes = [ctypes.c_uint8]
@@ -224,6 +224,29 @@ class Oracle:
                                                       self._ptr(w2_q), self._ptr(w2_s), T, H, I, E, top_k,
                                                       self._ptr(out), opt(h_pre), opt(h_q), opt(h_s)), "forward_mxfp8")
         return (out, h_pre, h_q, h_s) if intermediates else out
+
+    def forward_mxfp8_sampled(self, x, router_logits, experts: dict, I: int, top_k: int, tokens):
+        """The MX FP8 layer for the listed tokens.  ``experts`` maps expert id -> (w13_q [2I,H], w13_s [2I,H/32],
+        w2_q [H,I], w2_s [H,I/32]) uint8 arrays; only the experts those tokens route to need to be present."""
+        x = self._u16(x)
+        l = np.ascontiguousarray(router_logits, dtype=np.float32)
+        T, H = x.shape
+        E = l.shape[1]
+        tokens = np.ascontiguousarray(tokens, dtype=np.int32)
+        tabs = [(ctypes.c_void_p * E)() for _ in range(4)]
+        keep = []
+        for e, arrays in experts.items():
+            arrays = [np.ascontiguousarray(a, dtype=np.uint8) for a in arrays]
+            assert arrays[0].shape == (2 * I, H) and arrays[1].shape == (2 * I, H // 32)
+            assert arrays[2].shape == (H, I) and arrays[3].shape == (H, I // 32)
+            keep.append(arrays)
+            for tab, a in zip(tabs, arrays):
+                tab[e] = a.ctypes.data
+        out = np.empty((len(tokens), H), self.real)
+        self._check(self.lib.moe_oracle_forward_mxfp8_sampled(self._ptr(x), self._ptr(l), *tabs, T, H, I, E, top_k,
+                                                              self._ptr(tokens), len(tokens), self._ptr(out)),
+                    "forward_mxfp8_sampled")
+        return out
 
     def sorted_intermediates(self, x, w13, w2, topk_ids, sorted_to_flat):
         x, w13, w2 = self._u16(x), self._u16(w13), self._u16(w2)

@@ -22,7 +22,7 @@ MOE_FLAG_TWO_SLAB_GEMM = 4
 EXPORTED = ["moe_workspace_bytes", "moe_workspace_layout", "moe_route_workspace_bytes", "moe_route", "moe_route_static",
             "moe_forward",
             "moe_forward_ex", "moe_forward_local", "moe_forward_fp8w", "moe_mxfp8_workspace_bytes",
-            "moe_mxfp8_workspace_layout", "moe_mxfp8_pack_scales", "moe_mxfp8_quantize_rows", "moe_forward_mxfp8",
+            "moe_mxfp8_workspace_layout", "moe_mxfp8_pack_scales", "moe_mxfp8_quantize_rows", "moe_forward_mxfp8", "moe_forward_mxfp8_host",
             "moe_forward_staged", "moe_forward_host", "moe_last_status", "moe_forward_launch_count", "moe_status_string"]
 
 
@@ -41,7 +41,7 @@ class WorkspaceLayout(ctypes.Structure):
 class MxWorkspaceLayout(ctypes.Structure):
     _fields_ = [(n, ctypes.c_size_t) for n in
                 ("total_bytes", "status", "topk_ids", "topk_weights", "expert_offsets", "sorted_to_flat",
-                 "flat_to_sorted", "route_scratch", "x_q", "x_sf", "h_q", "h_sf", "y", "sf_atoms", "tile_rows")]
+                 "flat_to_sorted", "route_scratch", "x_q", "x_sf", "h_q", "h_sf", "y", "staging", "sf_atoms", "tile_rows")]
 
 
 _lib = None
@@ -84,6 +84,8 @@ def lib() -> ctypes.CDLL:
         L.moe_mxfp8_quantize_rows.argtypes = [vp, i, i, vp, vp, vp]
         L.moe_forward_mxfp8.restype = i
         L.moe_forward_mxfp8.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, i, i, vp, vp, sz, vp, ctypes.POINTER(vp)]
+        L.moe_forward_mxfp8_host.restype = i
+        L.moe_forward_mxfp8_host.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, i, i, vp, vp, sz, vp]
         L.moe_forward_staged.restype = i
         L.moe_forward_staged.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, vp, vp, sz, vp, ctypes.c_uint,
                                          ctypes.POINTER(vp)]
@@ -252,6 +254,20 @@ def moe_forward_mxfp8(x, router_logits, w13_q, w13_sf_packed, w2_q, w2_sf_packed
                                  _ptr(workspace), workspace.numel(), _stream(stream), handles)
     if check and st != MOE_OK:
         raise MoeError(st, "moe_forward_mxfp8")
+    return st
+
+
+def moe_forward_mxfp8_host(x_host, router_logits_host, w13_q, w13_sf_packed, w2_q, w2_sf_packed, top_k: int, out_host,
+                           workspace, stream=None, local_expert_offset: int = 0, check: bool = True) -> int:
+    """moe_forward_mxfp8 with CPU tensors for x, the router logits and the result (pinned for asynchronous copies)."""
+    T, H = x_host.shape
+    E = router_logits_host.shape[1]
+    n_local, I2, _ = w13_q.shape
+    st = lib().moe_forward_mxfp8_host(_ptr(x_host), _ptr(router_logits_host), _ptr(w13_q), _ptr(w13_sf_packed), _ptr(w2_q),
+                                      _ptr(w2_sf_packed), T, H, I2 // 2, E, top_k, local_expert_offset, n_local,
+                                      _ptr(out_host), _ptr(workspace), workspace.numel(), _stream(stream))
+    if check and st != MOE_OK:
+        raise MoeError(st, "moe_forward_mxfp8_host")
     return st
 
 

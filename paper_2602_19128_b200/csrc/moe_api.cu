@@ -176,6 +176,9 @@ void fill_mx_layout(int T, int H, int I, int E, int k, moe_mxfp8_workspace_layou
     L->h_q = take(A * I);
     L->h_sf = take(mx_act_sf_bytes((int)A, E, I, tile));
     L->y = take(A * H * 2);
+    L->staging = take((size_t)T * H * 2) /* x */;
+    take((size_t)T * E * sizeof(float)) /* logits */;
+    take((size_t)T * H * 2) /* out */;
     L->sf_atoms = (size_t)mx_act_sf_atoms((int)A, E, tile);
     L->tile_rows = (size_t)tile;
     L->total_bytes = off;
@@ -294,6 +297,34 @@ int moe_mxfp8_quantize_rows(const void *x, int R, int K, void *codes, void *scal
                                    static_cast<uint8_t *>(scales), static_cast<cudaStream_t>(stream)) == cudaSuccess
                ? MOE_OK
                : MOE_ERR_CUDA;
+}
+
+int moe_forward_mxfp8_host(const void *x_host, const float *router_logits_host, const void *w13_q,
+                           const void *w13_sf_packed, const void *w2_q, const void *w2_sf_packed, int T, int H, int I, int E,
+                           int top_k, int local_expert_offset, int num_local_experts, void *out_host, void *workspace,
+                           size_t workspace_bytes, void *stream) {
+    if (T < 0 || H <= 0 || I <= 0 || E <= 0 || top_k <= 0 || top_k > E || num_local_experts < 1) return MOE_ERR_SHAPE;
+    if (!mx_envelope_ok(T, H, I, E, top_k)) return MOE_ERR_UNSUPPORTED;
+    if (T == 0) return MOE_OK;
+    if (!x_host || !router_logits_host || !out_host || !workspace) return MOE_ERR_NULL;
+    if (!aligned(workspace, 256)) return MOE_ERR_ALIGN;
+    moe_mxfp8_workspace_layout_t L;
+    fill_mx_layout(T, H, I, E, top_k, &L);
+    if (workspace_bytes < L.total_bytes) return MOE_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    char *ws = static_cast<char *>(workspace);
+    const size_t x_bytes = (size_t)T * H * 2, l_bytes = (size_t)T * E * sizeof(float);
+    char *x_dev = ws + L.staging;
+    char *l_dev = x_dev + align_up(x_bytes, 256);
+    char *out_dev = l_dev + align_up(l_bytes, 256);
+    if (cudaMemcpyAsync(x_dev, x_host, x_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return MOE_ERR_CUDA;
+    if (cudaMemcpyAsync(l_dev, router_logits_host, l_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return MOE_ERR_CUDA;
+    const int st = forward_mx_impl(x_dev, reinterpret_cast<const float *>(l_dev), w13_q, w13_sf_packed, w2_q, w2_sf_packed, T,
+                                   H, I, E, top_k, local_expert_offset, num_local_experts, out_dev, workspace,
+                                   workspace_bytes, s, nullptr);
+    if (st != MOE_OK) return st;
+    if (cudaMemcpyAsync(out_host, out_dev, x_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) return MOE_ERR_CUDA;
+    return MOE_OK;
 }
 
 int moe_forward_mxfp8(const void *x, const float *router_logits, const void *w13_q, const void *w13_sf_packed,

@@ -11,7 +11,7 @@ import torch
 
 import paper_2602_19128_b200 as moe
 from oracle import moe_oracle
-from paper_2602_19128_b200.inputs import CONFIGS, bf16_bits
+from paper_2602_19128_b200.inputs import CONFIGS, bf16_bits, quantize_mxfp8
 from tests.gpu_common import OUT_TOL, assert_close_out, assert_routing_exact, bf16_to_f64, gpu_inputs, run_forward
 
 pytestmark = pytest.mark.gpu
@@ -60,3 +60,50 @@ def test_full_size_workload(name):
     close_on_device(h, views_v["h"], f"{name} h")
     close_on_device(y, views_v["y"], f"{name} y")
     close_on_device(out, out_v, f"{name} out")
+
+
+@pytest.mark.parametrize("name", ["mixtral", "dsv3_decode", "skewed", "dsv3_prefill"])
+def test_full_size_workload_mxfp8(name):
+    """The MX FP8 layer at full size (CTA-pair kernel with 240-row tiles for the large batches, one-CTA kernel
+    for the decode-sized one): routing bit-exact on all tokens, quantised token rows bit-exact on a sample,
+    the output of sampled tokens against the oracle, and run-to-run determinism."""
+    cfg = CONFIGS[name]
+    T, H, I, E, k = (cfg[n] for n in ("T", "H", "I", "E", "top_k"))
+    inp = gpu_inputs(name, seed=0)
+    w13_q, w13_s = quantize_mxfp8(inp["w13"])
+    inp["w13"] = None
+    w2_q, w2_s = quantize_mxfp8(inp["w2"])
+    inp["w2"] = None
+    sf13, sf2 = moe.moe_mxfp8_pack_scales(w13_s, True), moe.moe_mxfp8_pack_scales(w2_s, False)
+
+    def run():
+        ws = moe.alloc_workspace(moe.moe_mxfp8_workspace_bytes(T, H, I, E, k), "cuda")
+        out = torch.full((T, H), float("nan"), dtype=torch.bfloat16, device="cuda")
+        moe.moe_forward_mxfp8(inp["x"], inp["router_logits"], w13_q, sf13, w2_q, sf2, k, out, ws)
+        assert moe.moe_last_status(ws) == moe.MOE_OK
+        return out, ws
+
+    out, ws = run()
+    views = moe.mx_workspace_views(ws, T, H, I, E, k)
+    o = moe_oracle.get("f32")
+    logits = inp["router_logits"].cpu().numpy()
+    ids, w = o.route(logits, k)
+    off, s2f, f2s = o.permute(ids, E)
+    assert_routing_exact(views, ids, w, off, s2f, f2s)
+
+    rng = np.random.default_rng(0)
+    tokens = np.unique(np.concatenate([[0, T - 1], rng.choice(T, size=6, replace=False)])).astype(np.int32)
+    xc, _ = o.mx_quantize(inp["x"][torch.from_numpy(tokens).long().cuda()].float().cpu().numpy())
+    for n_i, t in enumerate(tokens):  # every sorted row of a sampled token holds that token's codes
+        rows = f2s[t * k:(t + 1) * k]
+        got = views["x_q"][torch.from_numpy(rows).long().cuda()].cpu().numpy()
+        assert np.array_equal(got, np.broadcast_to(xc[n_i], got.shape))
+
+    need = sorted({int(e) for t in tokens for e in ids[t]})
+    experts = {e: (w13_q[e].cpu().numpy(), w13_s[e].cpu().numpy(), w2_q[e].cpu().numpy(), w2_s[e].cpu().numpy()) for e in need}
+    ref = o.forward_mxfp8_sampled(bf16_bits(inp["x"]), logits, experts, I, k, tokens)
+    assert_close_out(bf16_to_f64(out[torch.from_numpy(tokens).long().cuda()]), ref, f"{name} mxfp8 sampled out")
+
+    del views, ws
+    out_again, _ = run()
+    assert torch.equal(out.view(torch.int16), out_again.view(torch.int16))

@@ -194,3 +194,17 @@ def test_mxfp8_repeated_calls_are_deterministic():
     a, _ = run_mx(inp)
     b, _ = run_mx(inp)
     assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+
+
+def test_mxfp8_host_entry_point_equals_the_device_one():
+    inp = make_mxfp8_inputs(dict(T=200, H=256, I=128, E=8, top_k=2, skew=False), seed=4, device="cuda")
+    out, _ = run_mx(inp)
+    T, H = inp["x"].shape
+    ws = moe.alloc_workspace(moe.moe_mxfp8_workspace_bytes(T, H, 128, 8, 2), "cuda")
+    xh, lh = inp["x"].cpu().pin_memory(), inp["router_logits"].cpu().pin_memory()
+    oh = torch.empty((T, H), dtype=torch.bfloat16).pin_memory()
+    moe.moe_forward_mxfp8_host(xh, lh, inp["w13_q"], moe.moe_mxfp8_pack_scales(inp["w13_s"], True), inp["w2_q"],
+                               moe.moe_mxfp8_pack_scales(inp["w2_s"], False), 2, oh, ws)
+    torch.cuda.synchronize()
+    assert moe.moe_last_status(ws) == moe.MOE_OK
+    assert torch.equal(oh.view(torch.int16), out.cpu().view(torch.int16))

@@ -196,3 +196,20 @@ def test_non_finite_token_poisons_only_itself():
     out = moe_oracle.get("f32").forward_mxfp8(bf16_bits(x), inp["router_logits"].numpy(), inp["w13_q"].numpy(),
                                               inp["w13_s"].numpy(), inp["w2_q"].numpy(), inp["w2_s"].numpy(), 1)
     assert np.all(np.isnan(out[2])) and np.all(np.isfinite(out[[0, 1, 3]]))
+
+
+def test_sampled_form_equals_the_whole_layer_on_those_tokens():
+    inp = make_mxfp8_inputs(dict(T=12, H=64, I=64, E=6, top_k=2, skew=False), seed=13)
+    o = moe_oracle.get("f32")
+    args = (bf16_bits(inp["x"]), inp["router_logits"].numpy())
+    w = [inp[n].numpy() for n in ("w13_q", "w13_s", "w2_q", "w2_s")]
+    full = o.forward_mxfp8(*args, *w, 2)
+    tokens = np.array([11, 0, 5], dtype=np.int32)
+    ids, _ = o.route(args[1], 2)
+    need = {int(e) for t in tokens for e in ids[t]}
+    experts = {e: tuple(a[e] for a in w) for e in need}
+    got = o.forward_mxfp8_sampled(*args, experts, 64, 2, tokens)
+    assert np.array_equal(got, full[tokens])
+    missing = {e: v for e, v in experts.items() if e != int(ids[11][0])}
+    with pytest.raises(RuntimeError):
+        o.forward_mxfp8_sampled(*args, missing, 64, 2, tokens)
