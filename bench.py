@@ -147,6 +147,30 @@ def oracle_sample(cfg_name: str, inp: dict, n_tokens: int, seed: int = 0):
     return o, bf16_bits(inp["x"]), logits, experts, I, k, tokens
 
 
+def token_tile_bound(T: int, E: int, k: int) -> int:
+    """The library's token-tile bound for the bf16 layer: the smallest of 32, 64, 128 holding 1.5 x the mean rows
+    per expert, else 256 (reporting only; mirrors the rule stated in the design notes)."""
+    avg = T * k / E
+    for nt in (32, 64, 128):
+        if 1.5 * avg <= nt:
+            return nt
+    return 256
+
+
+def computed_rows(counts, tile_bound: int, even: bool) -> int:
+    """Rows the GEMMs multiply (MMA N summed over token tiles): an expert's rows are cut into as few tiles as fit
+    under the bound, evenly sized (bf16) or of exactly the bound (MX), and each tile is rounded up to 16 rows."""
+    total = 0
+    for c in (int(v) for v in counts):
+        if c == 0:
+            continue
+        n_tiles = -(-c // tile_bound)
+        rows = -(-(-(-c // n_tiles)) // 16) * 16 if even else tile_bound
+        for j in range(n_tiles):
+            total += -(-min(rows, c - j * rows) // 16) * 16
+    return total
+
+
 def time_oracle(cfg_name: str, inp: dict, budget_s: float):
     """Times the oracle, as it stands, on a token sample sized to take roughly budget_s seconds."""
     from oracle import moe_oracle
@@ -378,7 +402,13 @@ def run_ours(args):
                     unit=unit, frac=achieved / peak, peak_source=f"of {peaks['source']}",
                     traffic=None if (fp8 or mx) else NCU_TRAFFIC_BYTES.get(args.config), algorithmic_per_launch=algorithmic,
                     kernel_ms=stage_ms["gemm1_swiglu"])
+    per_step_ms = sorted(ev[0].elapsed_time(ev[-1]) for ev in stage_events)
+    tile_bound = int(views["tile_rows"]) if mx else token_tile_bound(T, E, k)
     layer = dict(stage_ms={n: round(v, 5) for n, v in stage_ms.items()}, n_active_experts=n_active,
+                 latency_ms_median=statistics.median(per_step_ms), latency_ms_min=per_step_ms[0],
+                 padding_efficiency=rows_scheduled / max(1, computed_rows(counts, tile_bound, even=not mx)),
+                 weight_gbs_frac_nominal=active_weight_bytes / step_s / 1e9 / 8000.0,
+                 useful_tflops_frac_nominal=6.0 * A * H * I / step_s / 1e12 / (4500.0 if mx else 2250.0),
                  rows_per_expert_min=int(counts.min()), rows_per_expert_max=int(counts.max()),
                  weight_gbs=active_weight_bytes / step_s / 1e9, weight_gbs_frac=active_weight_bytes / step_s / 1e9 / peaks["hbm_gbs"],
                  useful_tflops=6.0 * A * H * I / step_s / 1e12,

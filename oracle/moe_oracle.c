@@ -122,6 +122,114 @@ int moe_oracle_route(const float *router_logits, int T, int E, int k, int32_t *t
     return ORACLE_OK;
 }
 
+/* ---- Grouped sigmoid router ("DeepSeek-V3 style, top-8 routing", Sec. 4.5) -------------------------------
+ * The paper names the style without its formula; the build's reading is the routing published with
+ * DeepSeek-V3, restated here with every constant as a parameter:
+ *   score_e  = sigmoid(logit_e)                                    (the weight an expert gets if chosen)
+ *   choice_e = score_e + bias_e                                    (used for selection only)
+ *   the E experts form n_group contiguous groups of G = E / n_group; a group's score is the sum of its two
+ *   largest choice values (the single value when G = 1); the topk_group best groups stay eligible;
+ *   the k eligible experts with the largest choice values are selected, in rank order;
+ *   w_j = score_{id_j} / (sum over the selected, in rank order) * route_scale.
+ * Ties (groups and experts) go to the lower index.
+ * Selection is an integer decision taken from floating-point values, so it is defined in ONE arithmetic,
+ * binary32, for both builds of this file and for the CUDA kernel (which restates it on its own): every
+ * operation below is a single correctly rounded IEEE operation (fmaf counts as one), exp included, which is
+ * evaluated by the fixed recipe of exp_fixed.  Only the final division and scaling use REAL. */
+typedef struct {
+    int n_group, topk_group;
+    const float *bias; /* [E] or NULL */
+    float scale;
+} GroupedRouter;
+
+/* e^x in binary32 by a fixed sequence of correctly rounded operations (within 2 ulp of the true value):
+ * x is clamped to [-87, 88]; n = nearest integer (ties to even) of x * log2(e); r = x - n * ln 2 with ln 2 in
+ * two parts; e^r by the degree-7 Taylor polynomial in Horner form; the result is that times 2^n. */
+static float exp_fixed(float x) {
+    if (x < -87.0f) x = -87.0f;
+    if (x > 88.0f) x = 88.0f;
+    const float n = rintf(x * 1.44269502f);
+    float r = fmaf(n, -0.693145752f, x);
+    r = fmaf(n, -1.42860677e-06f, r);
+    float p = 1.98412701e-04f;            /* 1/5040 */
+    p = fmaf(p, r, 1.38888892e-03f);      /* 1/720 */
+    p = fmaf(p, r, 8.33333377e-03f);      /* 1/120 */
+    p = fmaf(p, r, 4.16666679e-02f);      /* 1/24 */
+    p = fmaf(p, r, 1.66666672e-01f);      /* 1/6 */
+    p = fmaf(p, r, 0.5f);
+    p = fmaf(p, r, 1.0f);
+    p = fmaf(p, r, 1.0f);
+    return p * ldexpf(1.0f, (int)n);      /* 2^n is exact for n in [-126, 127] */
+}
+
+static float sigmoid_fixed(float l) { return 1.0f / (1.0f + exp_fixed(-l)); }
+
+float moe_oracle_exp_fixed(float x) { return exp_fixed(x); }
+float moe_oracle_sigmoid_fixed(float l) { return sigmoid_fixed(l); }
+
+/* scratch: score [E], choice [E] floats; eligible [n_group], taken [E] bytes */
+static void route_token_grouped(const float *l, int E, int k, const GroupedRouter *g, int32_t *ids, REAL *w, float *score,
+                                float *choice, unsigned char *eligible, unsigned char *taken) {
+    const int G = E / g->n_group;
+    for (int e = 0; e < E; ++e) {
+        score[e] = sigmoid_fixed(l[e]);
+        choice[e] = g->bias ? score[e] + g->bias[e] : score[e];
+    }
+    /* group scores, then topk_group passes each picking the best group not yet eligible */
+    float gscore[256];
+    for (int q = 0; q < g->n_group; ++q) {
+        float t1 = -INFINITY, t2 = -INFINITY; /* the two largest choice values of the group */
+        for (int e = q * G; e < (q + 1) * G; ++e) {
+            if (choice[e] > t1) { t2 = t1; t1 = choice[e]; }
+            else if (choice[e] > t2) t2 = choice[e];
+        }
+        gscore[q] = G >= 2 ? t1 + t2 : t1;
+        eligible[q] = 0;
+    }
+    for (int j = 0; j < g->topk_group; ++j) {
+        int best = -1;
+        for (int q = 0; q < g->n_group; ++q) {
+            if (eligible[q]) continue;
+            if (best < 0 || gscore[q] > gscore[best]) best = q; /* strict >: ties keep the lower index */
+        }
+        eligible[best] = 1;
+    }
+    memset(taken, 0, (size_t)E);
+    for (int j = 0; j < k; ++j) {
+        int best = -1;
+        for (int e = 0; e < E; ++e) {
+            if (taken[e] || !eligible[e / G]) continue;
+            if (best < 0 || choice[e] > choice[best]) best = e;
+        }
+        taken[best] = 1;
+        ids[j] = best;
+    }
+    float D = 0;
+    for (int j = 0; j < k; ++j) D = D + score[ids[j]];
+    for (int j = 0; j < k; ++j) w[j] = (REAL)score[ids[j]] / (REAL)D * (REAL)g->scale;
+}
+
+static int grouped_router_ok(int E, int k, int n_group, int topk_group) {
+    return n_group >= 1 && n_group <= 256 && E % n_group == 0 && topk_group >= 1 && topk_group <= n_group &&
+           (long)topk_group * (E / n_group) >= k;
+}
+
+/* Grouped router for a batch: router_logits [T,E] f32, bias [E] f32 or NULL -> topk_ids [T,k], topk_w [T,k] REAL. */
+int moe_oracle_route_grouped(const float *router_logits, const float *bias, int T, int E, int k, int n_group, int topk_group,
+                             float scale, int32_t *topk_ids, REAL *topk_w) {
+    if (T < 0 || E < 1 || k < 1 || k > E || !grouped_router_ok(E, k, n_group, topk_group)) return ORACLE_ERR_ARG;
+    float *score = (float *)malloc(sizeof(float) * 2 * (size_t)E);
+    unsigned char *flags = (unsigned char *)malloc((size_t)E + 256);
+    if (!score || !flags) { free(score); free(flags); return ORACLE_ERR_NOMEM; }
+    const GroupedRouter g = {n_group, topk_group, bias, scale};
+    for (int t = 0; t < T; ++t)
+        route_token_grouped(router_logits + (size_t)t * E, E, k, &g, topk_ids + (size_t)t * k, topk_w + (size_t)t * k, score,
+                            score + E, flags + E, flags);
+    free(score);
+    free(flags);
+    return ORACLE_OK;
+}
+
 /* Stable counting sort of the A = T*k assignments by expert ("sort-scatter").
  * Flat assignment index a = t*k + j.
  *   expert_offsets [E+1]: exclusive prefix sum of the per-expert counts
@@ -193,8 +301,9 @@ int moe_oracle_expert_ffn(const uint16_t *x_row, const uint16_t *w13_e, const ui
  * out[i,:] = sum_{j ascending} topk_w[t,j] * expert_{ids[t,j]}(x[t,:]),  t = tokens[i]. */
 static int forward_tokens(const uint16_t *x, const float *router_logits, const uint16_t *const *w13_ptrs,
                           const uint16_t *const *w2_ptrs, int T, int H, int I, int E, int k, const int32_t *tokens,
-                          int n_tokens, int skip_missing, REAL *out) {
+                          int n_tokens, int skip_missing, const GroupedRouter *grouped, REAL *out) {
     if (T < 0 || H < 1 || I < 1 || E < 1 || k < 1 || k > E || n_tokens < 0) return ORACLE_ERR_ARG;
+    if (grouped && !grouped_router_ok(E, k, grouped->n_group, grouped->topk_group)) return ORACLE_ERR_ARG;
     int status = ORACLE_OK;
 #pragma omp parallel
     {
@@ -204,7 +313,9 @@ static int forward_tokens(const uint16_t *x, const float *router_logits, const u
         REAL *w = (REAL *)malloc(sizeof(REAL) * (size_t)k);
         REAL *s = (REAL *)malloc(sizeof(REAL) * (size_t)I);
         REAL *y = (REAL *)malloc(sizeof(REAL) * (size_t)H);
-        if (!p || !taken || !ids || !w || !s || !y) {
+        float *gs = (float *)malloc(sizeof(float) * 2 * (size_t)E);      /* grouped router: score, choice */
+        unsigned char *elig = (unsigned char *)malloc(256);             /* grouped router: eligible groups */
+        if (!p || !taken || !ids || !w || !s || !y || !gs || !elig) {
 #pragma omp critical
             status = ORACLE_ERR_NOMEM;
         } else {
@@ -218,7 +329,10 @@ static int forward_tokens(const uint16_t *x, const float *router_logits, const u
                     status = ORACLE_ERR_ARG;
                     continue;
                 }
-                route_token(router_logits + (size_t)t * E, E, k, ids, w, p, taken);
+                if (grouped)
+                    route_token_grouped(router_logits + (size_t)t * E, E, k, grouped, ids, w, gs, gs + E, elig, taken);
+                else
+                    route_token(router_logits + (size_t)t * E, E, k, ids, w, p, taken);
                 for (int j = 0; j < k; ++j) {
                     const int e = ids[j];
                     if (!w13_ptrs[e] || !w2_ptrs[e]) {
@@ -232,7 +346,7 @@ static int forward_tokens(const uint16_t *x, const float *router_logits, const u
                 }
             }
         }
-        free(p); free(taken); free(ids); free(w); free(s); free(y);
+        free(p); free(taken); free(ids); free(w); free(s); free(y); free(gs); free(elig);
     }
     return status;
 }
@@ -240,7 +354,16 @@ static int forward_tokens(const uint16_t *x, const float *router_logits, const u
 int moe_oracle_forward_sampled(const uint16_t *x, const float *router_logits, const uint16_t *const *w13_ptrs,
                                const uint16_t *const *w2_ptrs, int T, int H, int I, int E, int k,
                                const int32_t *tokens, int n_tokens, REAL *out) {
-    return forward_tokens(x, router_logits, w13_ptrs, w2_ptrs, T, H, I, E, k, tokens, n_tokens, 0, out);
+    return forward_tokens(x, router_logits, w13_ptrs, w2_ptrs, T, H, I, E, k, tokens, n_tokens, 0, NULL, out);
+}
+
+/* The same with the grouped sigmoid router (bias [E] f32 or NULL). */
+int moe_oracle_forward_sampled_grouped(const uint16_t *x, const float *router_logits, const float *bias, int n_group,
+                                       int topk_group, float scale, const uint16_t *const *w13_ptrs,
+                                       const uint16_t *const *w2_ptrs, int T, int H, int I, int E, int k,
+                                       const int32_t *tokens, int n_tokens, REAL *out) {
+    const GroupedRouter g = {n_group, topk_group, bias, scale};
+    return forward_tokens(x, router_logits, w13_ptrs, w2_ptrs, T, H, I, E, k, tokens, n_tokens, 0, &g, out);
 }
 
 /* The layer restricted to the experts resident on one device (the paper's kernel computes "32 local
@@ -264,7 +387,7 @@ int moe_oracle_forward_local(const uint16_t *x, const float *router_logits, cons
             p2[local_offset + l] = w2_local + (size_t)l * H * I;
         }
         for (int t = 0; t < T; ++t) tokens[t] = t;
-        status = forward_tokens(x, router_logits, p13, p2, T, H, I, E, k, tokens, T, 1, out);
+        status = forward_tokens(x, router_logits, p13, p2, T, H, I, E, k, tokens, T, 1, NULL, out);
     }
     free(p13); free(p2); free(tokens);
     return status;
@@ -315,7 +438,7 @@ int moe_oracle_forward(const uint16_t *x, const float *router_logits, const uint
             p2[e] = w2 + (size_t)e * H * I;
         }
         for (int t = 0; t < T; ++t) tokens[t] = t;
-        status = forward_tokens(x, router_logits, p13, p2, T, H, I, E, k, tokens, T, 0, out);
+        status = forward_tokens(x, router_logits, p13, p2, T, H, I, E, k, tokens, T, 0, NULL, out);
     }
     free(p13); free(p2); free(tokens);
     return status;

@@ -52,10 +52,17 @@ class Oracle:
         for fn in ("moe_oracle_route", "moe_oracle_permute", "moe_oracle_expert_ffn", "moe_oracle_forward",
                    "moe_oracle_forward_sampled", "moe_oracle_sorted_intermediates", "moe_oracle_forward_local",
                    "moe_oracle_permute_local", "moe_oracle_forward_fp8w", "moe_oracle_mx_quantize",
-                   "moe_oracle_forward_mxfp8", "moe_oracle_forward_mxfp8_sampled"):
+                   "moe_oracle_forward_mxfp8", "moe_oracle_forward_mxfp8_sampled", "moe_oracle_route_grouped",
+                   "moe_oracle_forward_sampled_grouped"):
             getattr(self.lib, fn).restype = ctypes.c_int
         self.lib.moe_oracle_e4m3_decode.restype = ctypes.c_float
         self.lib.moe_oracle_e4m3_decode.argtypes = [ctypes.c_uint8]
+        for fn in ("moe_oracle_exp_fixed", "moe_oracle_sigmoid_fixed"):
+            getattr(self.lib, fn).restype = ctypes.c_float
+            getattr(self.lib, fn).argtypes = [ctypes.c_float]
+        self.lib.moe_oracle_route_grouped.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int,
+                                                      ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_float,
+                                                      ctypes.c_void_p, ctypes.c_void_p]
         self.lib.moe_oracle_e4m3_encode.restype = ctypes.c_uint8
         self.lib.moe_oracle_e4m3_encode.argtypes = [ctypes.c_float]
 
@@ -87,6 +94,50 @@ class Oracle:
         w = np.empty((T, top_k), self.real)
         self._check(self.lib.moe_oracle_route(self._ptr(l), T, E, top_k, self._ptr(ids), self._ptr(w)), "route")
         return ids, w
+
+    def exp_fixed(self, x: float) -> float:
+        return float(self.lib.moe_oracle_exp_fixed(ctypes.c_float(x)))
+
+    def sigmoid_fixed(self, x: float) -> float:
+        return float(self.lib.moe_oracle_sigmoid_fixed(ctypes.c_float(x)))
+
+    def route_grouped(self, router_logits: np.ndarray, top_k: int, n_group: int, topk_group: int, bias=None,
+                      scale: float = 1.0):
+        """Grouped sigmoid router: (ids [T,k] in rank order, weights [T,k])."""
+        l = np.ascontiguousarray(router_logits, dtype=np.float32)
+        T, E = l.shape
+        b = None if bias is None else np.ascontiguousarray(bias, dtype=np.float32)
+        assert b is None or b.shape == (E,)
+        ids = np.empty((T, top_k), np.int32)
+        w = np.empty((T, top_k), self.real)
+        self._check(self.lib.moe_oracle_route_grouped(self._ptr(l), None if b is None else self._ptr(b), T, E, top_k,
+                                                      n_group, topk_group, ctypes.c_float(scale), self._ptr(ids),
+                                                      self._ptr(w)), "route_grouped")
+        return ids, w
+
+    def forward_sampled_grouped(self, x, router_logits, experts: dict, I: int, top_k: int, tokens, n_group: int,
+                                topk_group: int, bias=None, scale: float = 1.0):
+        """forward_sampled with the grouped sigmoid router."""
+        x = self._u16(x)
+        l = np.ascontiguousarray(router_logits, dtype=np.float32)
+        T, H = x.shape
+        E = l.shape[1]
+        tokens = np.ascontiguousarray(tokens, dtype=np.int32)
+        b = None if bias is None else np.ascontiguousarray(bias, dtype=np.float32)
+        p13 = (ctypes.c_void_p * E)()
+        p2 = (ctypes.c_void_p * E)()
+        keep = []
+        for e, (a, c) in experts.items():
+            a, c = self._u16(a), self._u16(c)
+            assert a.shape == (2 * I, H) and c.shape == (H, I)
+            keep.append((a, c))
+            p13[e] = a.ctypes.data
+            p2[e] = c.ctypes.data
+        out = np.empty((len(tokens), H), self.real)
+        self._check(self.lib.moe_oracle_forward_sampled_grouped(
+            self._ptr(x), self._ptr(l), None if b is None else self._ptr(b), n_group, topk_group, ctypes.c_float(scale),
+            p13, p2, T, H, I, E, top_k, self._ptr(tokens), len(tokens), self._ptr(out)), "forward_sampled_grouped")
+        return out
 
     def permute(self, topk_ids: np.ndarray, E: int):
         ids = np.ascontiguousarray(topk_ids, dtype=np.int32)
