@@ -207,6 +207,38 @@ MOE_API int moe_forward_staged(const void *x, const float *router_logits, const 
                                void *workspace, size_t workspace_bytes, void *stream, unsigned flags,
                                void *const *stage_events);
 
+/* ---- Grouped sigmoid router ("DeepSeek-V3 style, top-8 routing", paper Sec. 4.5) -------------------------
+ * The paper names the style without its formula; this is the routing published with DeepSeek-V3, with every
+ * constant a parameter:
+ *   score_e  = sigmoid(logit_e)                          the weight an expert gets if chosen
+ *   choice_e = score_e + selection_bias[e]               used for selection only
+ *   the E experts form n_group contiguous groups of E / n_group; a group's score is the sum of its two largest
+ *   choice values (the single value for groups of one); the topk_group best groups stay eligible; the top_k
+ *   eligible experts with the largest choice values are selected, in rank order; ties go to the lower index;
+ *   weight_j = score_{id_j} / (sum of the selected scores, in rank order) * route_scale.
+ * All of it is evaluated in binary32 with one correctly rounded operation per step, e^x by a fixed recipe
+ * (clamp to [-87, 88]; n = nearest integer of x * log2 e; r = x - n * ln 2 in two fused steps; degree-7 Taylor
+ * polynomial in Horner form; times 2^n), so the selected ids are reproducible bit for bit.
+ * Requirements: n_group >= 1 divides E, E / n_group is a power of two, 1 <= topk_group <= n_group,
+ * topk_group * (E / n_group) >= top_k (MOE_ERR_UNSUPPORTED otherwise). */
+typedef struct {
+    int n_group;
+    int topk_group;
+    const float *selection_bias; /* DEVICE, [E] f32, or NULL for no bias */
+    float route_scale;
+} moe_grouped_router_t;
+
+/* moe_route with the grouped router (same outputs, workspace and errors). */
+MOE_API int moe_route_grouped(const float *router_logits, int T, int E, int top_k, const moe_grouped_router_t *router,
+                              int32_t *topk_ids, float *topk_weights, int32_t *expert_offsets, int32_t *sorted_to_flat,
+                              int32_t *flat_to_sorted, void *workspace, size_t workspace_bytes, void *stream);
+
+/* moe_forward_local with the grouped router (pass local_expert_offset = 0, num_local_experts = E for all). */
+MOE_API int moe_forward_grouped(const void *x, const float *router_logits, const void *w13, const void *w2, int T, int H,
+                                int I, int E, int top_k, const moe_grouped_router_t *router, int local_expert_offset,
+                                int num_local_experts, void *out, void *workspace, size_t workspace_bytes, void *stream,
+                                unsigned flags);
+
 /* ---- MX FP8: 8-bit weights AND activations, multiplied by the block-scaled tensor-core instruction --------
  *
  * The paper's MoE workload is an FP8 one (Table 2, "FP8 MoE"; Sec. 4.5 names FP8 packing and scaling as a

@@ -21,7 +21,7 @@ MOE_FLAG_TWO_SLAB_GEMM = 4
 
 EXPORTED = ["moe_workspace_bytes", "moe_workspace_layout", "moe_route_workspace_bytes", "moe_route", "moe_route_static",
             "moe_forward",
-            "moe_forward_ex", "moe_forward_local", "moe_forward_fp8w", "moe_mxfp8_workspace_bytes",
+            "moe_forward_ex", "moe_forward_local", "moe_route_grouped", "moe_forward_grouped", "moe_forward_fp8w", "moe_mxfp8_workspace_bytes",
             "moe_mxfp8_workspace_layout", "moe_mxfp8_pack_scales", "moe_mxfp8_quantize_rows", "moe_forward_mxfp8", "moe_forward_mxfp8_host",
             "moe_forward_staged", "moe_forward_host", "moe_last_status", "moe_forward_launch_count", "moe_status_string"]
 
@@ -36,6 +36,17 @@ class WorkspaceLayout(ctypes.Structure):
     _fields_ = [(n, ctypes.c_size_t) for n in
                 ("total_bytes", "status", "topk_ids", "topk_weights", "expert_offsets", "sorted_to_flat",
                  "flat_to_sorted", "route_scratch", "x_perm", "h", "y", "staging")]
+
+
+class GroupedRouter(ctypes.Structure):
+    _fields_ = [("n_group", ctypes.c_int), ("topk_group", ctypes.c_int), ("selection_bias", ctypes.c_void_p),
+                ("route_scale", ctypes.c_float)]
+
+
+def grouped_router(n_group: int, topk_group: int, selection_bias=None, route_scale: float = 1.0) -> GroupedRouter:
+    """Description of the grouped sigmoid router; ``selection_bias`` is a device f32 tensor [E] or None (the
+    caller keeps it alive)."""
+    return GroupedRouter(n_group, topk_group, None if selection_bias is None else selection_bias.data_ptr(), route_scale)
 
 
 class MxWorkspaceLayout(ctypes.Structure):
@@ -72,6 +83,11 @@ def lib() -> ctypes.CDLL:
         L.moe_forward_ex.argtypes = [vp, vp, vp, vp, i, i, i, i, i, vp, vp, sz, vp, ctypes.c_uint]
         L.moe_forward_local.restype = i
         L.moe_forward_local.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, vp, vp, sz, vp, ctypes.c_uint]
+        L.moe_route_grouped.restype = i
+        L.moe_route_grouped.argtypes = [vp, i, i, i, ctypes.POINTER(GroupedRouter), vp, vp, vp, vp, vp, vp, sz, vp]
+        L.moe_forward_grouped.restype = i
+        L.moe_forward_grouped.argtypes = [vp, vp, vp, vp, i, i, i, i, i, ctypes.POINTER(GroupedRouter), i, i, vp, vp, sz, vp,
+                                          ctypes.c_uint]
         L.moe_forward_fp8w.restype = i
         L.moe_forward_fp8w.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, vp, vp, sz, vp, ctypes.POINTER(vp)]
         L.moe_mxfp8_workspace_bytes.restype = sz
@@ -188,6 +204,31 @@ def moe_forward_local(x, router_logits, w13_local, w2_local, top_k: int, local_e
                                  _stream(stream), flags)
     if check and st != MOE_OK:
         raise MoeError(st, "moe_forward_local")
+    return st
+
+
+def moe_route_grouped(router_logits, top_k: int, router: GroupedRouter, topk_ids, topk_weights, expert_offsets,
+                      sorted_to_flat, flat_to_sorted, workspace, stream=None, check: bool = True) -> int:
+    T, E = router_logits.shape
+    st = lib().moe_route_grouped(_ptr(router_logits), T, E, top_k, ctypes.byref(router), _ptr(topk_ids), _ptr(topk_weights),
+                                 _ptr(expert_offsets), _ptr(sorted_to_flat), _ptr(flat_to_sorted), _ptr(workspace),
+                                 workspace.numel(), _stream(stream))
+    if check and st != MOE_OK:
+        raise MoeError(st, "moe_route_grouped")
+    return st
+
+
+def moe_forward_grouped(x, router_logits, w13, w2, top_k: int, router: GroupedRouter, out, workspace, stream=None,
+                        flags: int = 0, local_expert_offset: int = 0, check: bool = True) -> int:
+    """The layer with the grouped sigmoid router; w13 may hold a local subset of the experts."""
+    T, H = x.shape
+    E = router_logits.shape[1]
+    n_local, I2, _ = w13.shape
+    st = lib().moe_forward_grouped(_ptr(x), _ptr(router_logits), _ptr(w13), _ptr(w2), T, H, I2 // 2, E, top_k,
+                                   ctypes.byref(router), local_expert_offset, n_local, _ptr(out), _ptr(workspace),
+                                   workspace.numel(), _stream(stream), flags)
+    if check and st != MOE_OK:
+        raise MoeError(st, "moe_forward_grouped")
     return st
 
 

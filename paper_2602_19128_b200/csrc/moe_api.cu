@@ -18,6 +18,22 @@ bool route_envelope_ok(long long T, int E, int k) {
     return !(E < 1 || E > kMaxExperts || k < 1 || k > E || k > kMaxTopK || T < 0 || T * k >= (1LL << 27));
 }
 
+// Checks a grouped-router description against the kernel's envelope and converts it.
+int make_router(const moe_grouped_router_t *r, int E, int k, RouterParams *out) {
+    if (!r) return MOE_ERR_NULL;
+    if (r->n_group < 1 || r->topk_group < 1) return MOE_ERR_SHAPE;
+    if (E % r->n_group != 0 || r->topk_group > r->n_group) return MOE_ERR_UNSUPPORTED;
+    const int G = E / r->n_group;
+    if ((G & (G - 1)) != 0 || (long long)r->topk_group * G < k) return MOE_ERR_UNSUPPORTED;
+    if (reinterpret_cast<uintptr_t>(r->selection_bias) % 4 != 0) return MOE_ERR_ALIGN;
+    out->grouped = 1;
+    out->n_group = r->n_group;
+    out->topk_group = r->topk_group;
+    out->bias = r->selection_bias;
+    out->scale = r->route_scale;
+    return MOE_OK;
+}
+
 bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
 void fill_layout(int T, int H, int I, int E, int k, moe_workspace_layout_t *L) {
@@ -50,7 +66,7 @@ int check_device() {
 int forward_impl(const void *x, const float *logits, const void *w13, const void *w2, int T, int H, int I, int E, int k,
                  void *out, void *workspace, size_t workspace_bytes, cudaStream_t stream, unsigned flags,
                  void *const *stage_events = nullptr, int local_offset = 0, int n_local = -1,
-                 const float *w13_scale = nullptr, const float *w2_scale = nullptr) {
+                 const float *w13_scale = nullptr, const float *w2_scale = nullptr, RouterParams router = RouterParams()) {
     if (n_local < 0) n_local = E;  // every expert is resident
     const bool fp8w = w13_scale != nullptr;  // w13 / w2 then hold E4M3 codes, one byte per weight
     if (T < 0 || H <= 0 || I <= 0 || E <= 0 || k <= 0 || k > E) return MOE_ERR_SHAPE;
@@ -88,7 +104,7 @@ int forward_impl(const void *x, const float *logits, const void *w13, const void
     };
     if (!mark(0)) return MOE_ERR_CUDA;
     if (launch_route(logits, T, E, k, LocalExperts{local_offset, n_local}, nt_max, ids, wts, offsets, s2f, f2s, rs, status,
-                     stream) != cudaSuccess)
+                     stream, 16, router) != cudaSuccess)
         return MOE_ERR_CUDA;
     if (!mark(1)) return MOE_ERR_CUDA;
     if (launch_gather_rows(static_cast<const __nv_bfloat16 *>(x), s2f, offsets + n_local, A, k, H, x_perm, stream) !=
@@ -376,6 +392,45 @@ int moe_route(const float *router_logits, int T, int E, int top_k, int32_t *topk
     const cudaError_t err = launch_route(router_logits, T, E, top_k, LocalExperts{0, E}, 256, topk_ids, topk_weights,
                                          expert_offsets, sorted_to_flat, flat_to_sorted, rs, reinterpret_cast<int *>(ws), s);
     return err == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
+
+int moe_route_grouped(const float *router_logits, int T, int E, int top_k, const moe_grouped_router_t *router,
+                      int32_t *topk_ids, float *topk_weights, int32_t *expert_offsets, int32_t *sorted_to_flat,
+                      int32_t *flat_to_sorted, void *workspace, size_t workspace_bytes, void *stream) {
+    if (T < 0 || E <= 0 || top_k <= 0 || top_k > E) return MOE_ERR_SHAPE;
+    if (!route_envelope_ok(T, E, top_k)) return MOE_ERR_UNSUPPORTED;
+    RouterParams rp;
+    const int rs_status = make_router(router, E, top_k, &rp);
+    if (rs_status != MOE_OK) return rs_status;
+    if (!expert_offsets) return MOE_ERR_NULL;
+    if (T > 0 && (!router_logits || !topk_ids || !topk_weights || !sorted_to_flat || !flat_to_sorted)) return MOE_ERR_NULL;
+    if (!workspace) return MOE_ERR_NULL;
+    if (!aligned(workspace, 256) || !aligned(router_logits, 4) || !aligned(topk_ids, 4) || !aligned(topk_weights, 4) ||
+        !aligned(expert_offsets, 4) || !aligned(sorted_to_flat, 4) || !aligned(flat_to_sorted, 4))
+        return MOE_ERR_ALIGN;
+    if (workspace_bytes < moe_route_workspace_bytes(T, E, top_k)) return MOE_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (T == 0)
+        return cudaMemsetAsync(expert_offsets, 0, (size_t)(E + 1) * sizeof(int), s) == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+    char *ws = static_cast<char *>(workspace);
+    RouteScratch rs = carve_route_scratch(ws + 256, T, E);
+    const cudaError_t err = launch_route(router_logits, T, E, top_k, LocalExperts{0, E}, 256, topk_ids, topk_weights,
+                                         expert_offsets, sorted_to_flat, flat_to_sorted, rs, reinterpret_cast<int *>(ws), s,
+                                         16, rp);
+    return err == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
+
+int moe_forward_grouped(const void *x, const float *router_logits, const void *w13, const void *w2, int T, int H, int I,
+                        int E, int top_k, const moe_grouped_router_t *router, int local_expert_offset,
+                        int num_local_experts, void *out, void *workspace, size_t workspace_bytes, void *stream,
+                        unsigned flags) {
+    if (num_local_experts < 1 || E <= 0 || top_k <= 0 || top_k > E) return MOE_ERR_SHAPE;
+    RouterParams rp;
+    const int rs_status = make_router(router, E, top_k, &rp);
+    if (rs_status != MOE_OK) return rs_status;
+    return forward_impl(x, router_logits, w13, w2, T, H, I, E, top_k, out, workspace, workspace_bytes,
+                        static_cast<cudaStream_t>(stream), flags, nullptr, local_expert_offset, num_local_experts, nullptr,
+                        nullptr, rp);
 }
 
 int moe_forward(const void *x, const float *router_logits, const void *w13, const void *w2, int T, int H, int I, int E,

@@ -49,6 +49,18 @@ static inline RouteScratch carve_route_scratch(void *base, int T, int E) {
     return s;
 }
 
+// How a token's experts and weights are derived from its logits.
+//   softmax : softmax -> top-k -> renormalise (the five workloads)
+//   grouped : sigmoid scores, a per-expert bias added for selection only, experts in n_group contiguous
+//             groups of which the topk_group best (by the sum of their two largest biased scores) stay
+//             eligible, top-k among those, weights = unbiased scores normalised and multiplied by `scale`.
+struct RouterParams {
+    int grouped = 0;
+    int n_group = 1, topk_group = 1;
+    const float *bias = nullptr;  // [E] or nullptr
+    float scale = 1.f;
+};
+
 // The experts resident on this device: ids [offset, offset + count) of the E the router chooses from.
 // Assignments to other experts are dropped from the schedule (flat_to_sorted = -1).
 struct LocalExperts {
@@ -60,7 +72,8 @@ struct LocalExperts {
 // `row_quantum` rows.  Scratch and expert_offsets are sized by local.count.
 cudaError_t launch_route(const float *logits, int T, int E, int k, LocalExperts local, int nt_max, int *topk_ids,
                          float *topk_w, int *expert_offsets, int *sorted_to_flat, int *flat_to_sorted,
-                         RouteScratch scratch, int *status, cudaStream_t stream, int row_quantum = 16);
+                         RouteScratch scratch, int *status, cudaStream_t stream, int row_quantum = 16,
+                         RouterParams router = RouterParams());
 
 // x_perm[r,:] = x[sorted_to_flat[r] / k, :] for r < *n_rows (a device-side count, at most A)
 cudaError_t launch_gather_rows(const __nv_bfloat16 *x, const int *sorted_to_flat, const int *n_rows, int A, int k,

@@ -87,10 +87,133 @@ __device__ __forceinline__ void route_one_token(const float *__restrict__ row, i
     my_w = my_p / denom;
 }
 
+// ---- grouped sigmoid router ("DeepSeek-V3 style" routing, Sec. 4.5) ---------------------------------------
+// Selection is an integer decision taken from floating-point values, so every operation that feeds it is one
+// correctly rounded binary32 operation in a fixed order (the _rn intrinsics keep the compiler from fusing or
+// reassociating them); e^x follows a fixed recipe: clamp to [-87, 88], n = nearest integer of x * log2(e),
+// r = x - n * ln 2 (ln 2 in two parts, fused multiply-adds), degree-7 Taylor polynomial in Horner form, times 2^n.
+__device__ __forceinline__ float exp_fixed(float x) {
+    x = fminf(fmaxf(x, -87.0f), 88.0f);
+    const float n = rintf(__fmul_rn(x, 1.44269502f));
+    float r = __fmaf_rn(n, -0.693145752f, x);
+    r = __fmaf_rn(n, -1.42860677e-06f, r);
+    float p = 1.98412701e-04f;
+    p = __fmaf_rn(p, r, 1.38888892e-03f);
+    p = __fmaf_rn(p, r, 8.33333377e-03f);
+    p = __fmaf_rn(p, r, 4.16666679e-02f);
+    p = __fmaf_rn(p, r, 1.66666672e-01f);
+    p = __fmaf_rn(p, r, 0.5f);
+    p = __fmaf_rn(p, r, 1.0f);
+    p = __fmaf_rn(p, r, 1.0f);
+    return __fmul_rn(p, __int_as_float(((int)n + 127) << 23));
+}
+__device__ __forceinline__ float sigmoid_fixed(float l) { return __fdiv_rn(1.0f, __fadd_rn(1.0f, exp_fixed(-l))); }
+
+// Merge two (largest, second largest) pairs.
+__device__ __forceinline__ void top2_merge(float &t1, float &t2, float o1, float o2) {
+    const float lo = fminf(t1, o1);
+    t1 = fmaxf(t1, o1);
+    t2 = fmaxf(lo, fmaxf(t2, o2));
+}
+
+// One token by one warp.  Expert e = 32 i + lane lives in register i of its lane; a group is G = E / n_group
+// consecutive experts, G a power of two: either a segment of G lanes within one register index (G <= 32) or all
+// lanes of G / 32 consecutive register indices.
+__device__ __forceinline__ void route_one_token_grouped(const float *__restrict__ row, int E, int k, int lane,
+                                                        const RouterParams &rp, int &my_id, float &my_w) {
+    const int G = E / rp.n_group;
+    float s[kLogitsPerLane], c[kLogitsPerLane], t1[kLogitsPerLane], t2[kLogitsPerLane];
+#pragma unroll
+    for (int i = 0; i < kLogitsPerLane; ++i) {
+        const int e = i * 32 + lane;
+        s[i] = e < E ? sigmoid_fixed(row[e]) : 0.f;
+        c[i] = e < E ? (rp.bias ? __fadd_rn(s[i], rp.bias[e]) : s[i]) : -INFINITY;
+        t1[i] = c[i];
+        t2[i] = -INFINITY;
+    }
+    // the two largest biased scores of every group
+    if (G > 32) {  // registers of the same group first
+        const int m = G >> 5;
+#pragma unroll
+        for (int i = 0; i < kLogitsPerLane; ++i) {
+            const int first = i & ~(m - 1);
+            float a1 = -INFINITY, a2 = -INFINITY;
+#pragma unroll
+            for (int j = 0; j < kLogitsPerLane; ++j)
+                if (j >= first && j < first + m) top2_merge(a1, a2, c[j], -INFINITY);
+            t1[i] = a1;
+            t2[i] = a2;
+        }
+    }
+    for (int off = (G < 32 ? G : 32) >> 1; off > 0; off >>= 1) {
+#pragma unroll
+        for (int i = 0; i < kLogitsPerLane; ++i) {
+            const float o1 = __shfl_xor_sync(kFullMask, t1[i], off), o2 = __shfl_xor_sync(kFullMask, t2[i], off);
+            top2_merge(t1[i], t2[i], o1, o2);
+        }
+    }
+    float gs[kLogitsPerLane];  // score of the group that holds this register's expert
+#pragma unroll
+    for (int i = 0; i < kLogitsPerLane; ++i) gs[i] = G >= 2 ? __fadd_rn(t1[i], t2[i]) : t1[i];
+    // rank of that group among all groups (ties to the lower group index); eligible if below topk_group
+    int rank[kLogitsPerLane];
+#pragma unroll
+    for (int i = 0; i < kLogitsPerLane; ++i) rank[i] = 0;
+    for (int g = 0; g < rp.n_group; ++g) {
+        const int e0 = g * G, ip = e0 >> 5;
+        float pick = gs[0];
+#pragma unroll
+        for (int i = 1; i < kLogitsPerLane; ++i) pick = ip == i ? gs[i] : pick;
+        const float val = __shfl_sync(kFullMask, pick, e0 & 31);
+#pragma unroll
+        for (int i = 0; i < kLogitsPerLane; ++i) {
+            const int gid = (i * 32 + lane) / G;
+            rank[i] += (val > gs[i] || (val == gs[i] && g < gid)) ? 1 : 0;
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < kLogitsPerLane; ++i)
+        if (rank[i] >= rp.topk_group) c[i] = -INFINITY;
+
+    // k rounds of a warp arg-max over the eligible biased scores; the payload is the unbiased score
+    unsigned taken = 0;
+    float my_s = 0.f;
+    my_id = 0;
+    for (int j = 0; j < k; ++j) {
+        int ci = INT_MAX;
+        float cv = -INFINITY, cp = 0.f;
+#pragma unroll
+        for (int i = 0; i < kLogitsPerLane; ++i) {
+            const int e = i * 32 + lane;
+            if (e < E && !((taken >> i) & 1u) && (ci == INT_MAX || c[i] > cv)) {
+                ci = e; cv = c[i]; cp = s[i];
+            }
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            const float ov = __shfl_xor_sync(kFullMask, cv, off);
+            const int oi = __shfl_xor_sync(kFullMask, ci, off);
+            const float op = __shfl_xor_sync(kFullMask, cp, off);
+            const bool other = (ci == INT_MAX) ? (oi != INT_MAX)
+                                               : (oi != INT_MAX && (ov > cv || (ov == cv && oi < ci)));
+            if (other) { cv = ov; ci = oi; cp = op; }
+        }
+        ci = __shfl_sync(kFullMask, ci, 0);
+        cp = __shfl_sync(kFullMask, cp, 0);
+        if (ci == INT_MAX) ci = 0;
+        if ((ci & 31) == lane) taken |= 1u << (ci >> 5);
+        if (lane == j) { my_id = ci; my_s = cp; }
+    }
+    float denom = 0.f;  // ascending rank
+    for (int j = 0; j < k; ++j) denom = __fadd_rn(denom, __shfl_sync(kFullMask, my_s, j));
+    my_w = __fmul_rn(__fdiv_rn(my_s, denom), rp.scale);
+}
+
 // Routes the block's 32 tokens (warp w takes tokens w, w + n_warps, ...), writes ids and weights, and
 // leaves the block's histogram over the resident experts in hist[].
 __device__ __forceinline__ void route_block_tokens(const float *__restrict__ logits, int T, int E, int k, int local_offset,
-                                                   int n_local, int *topk_ids, float *topk_w, int *hist) {
+                                                   int n_local, const RouterParams &rp, int *topk_ids, float *topk_w,
+                                                   int *hist) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, n_warps = blockDim.x >> 5;
     for (int e = tid; e < n_local; e += blockDim.x) hist[e] = 0;
     __syncthreads();
@@ -100,7 +223,10 @@ __device__ __forceinline__ void route_block_tokens(const float *__restrict__ log
         if (t >= T) break;  // uniform over the warp
         int my_id;
         float my_w;
-        route_one_token(logits + (size_t)t * E, E, k, lane, my_id, my_w);
+        if (rp.grouped)
+            route_one_token_grouped(logits + (size_t)t * E, E, k, lane, rp, my_id, my_w);
+        else
+            route_one_token(logits + (size_t)t * E, E, k, lane, my_id, my_w);
         if (lane < k) {
             topk_ids[(size_t)t * k + lane] = my_id;
             topk_w[(size_t)t * k + lane] = my_w;
@@ -113,9 +239,10 @@ __device__ __forceinline__ void route_block_tokens(const float *__restrict__ log
 
 __global__ void __launch_bounds__(kRouteThreads)
 route_topk_kernel(const float *__restrict__ logits, int T, int E, int k, int local_offset, int n_local,
-                  int *__restrict__ topk_ids, float *__restrict__ topk_w, int *__restrict__ chunk_counts) {
+                  const RouterParams rp, int *__restrict__ topk_ids, float *__restrict__ topk_w,
+                  int *__restrict__ chunk_counts) {
     __shared__ int hist[kMaxExperts];  // indexed by local expert (expert id - local_offset)
-    route_block_tokens(logits, T, E, k, local_offset, n_local, topk_ids, topk_w, hist);
+    route_block_tokens(logits, T, E, k, local_offset, n_local, rp, topk_ids, topk_w, hist);
     for (int e = threadIdx.x; e < n_local; e += kRouteThreads) chunk_counts[(size_t)blockIdx.x * n_local + e] = hist[e];
 }
 
@@ -254,13 +381,13 @@ constexpr int kFusedMaxChunks = kFusedThreads / 32;
 
 __global__ void __launch_bounds__(kFusedThreads)
 route_fused_kernel(const float *__restrict__ logits, int T, int E, int k, int local_offset, int n_local, int nt_max,
-                   int row_quantum, int *topk_ids, float *topk_w, int *chunk_counts, int *expert_offsets, int *tile_prefix,
+                   int row_quantum, const RouterParams rp, int *topk_ids, float *topk_w, int *chunk_counts, int *expert_offsets, int *tile_prefix,
                    int *tile_order, int *tile_rows, int *sorted_to_flat, int *flat_to_sorted, int *done_counter) {
     __shared__ int hist[kMaxExperts], counts[kMaxExperts], tiles_at[kMaxExperts], warp_sums[8];
     __shared__ int next[kFusedMaxChunks][kMaxExperts];
     __shared__ int is_last;
     const int tid = threadIdx.x;
-    route_block_tokens(logits, T, E, k, local_offset, n_local, topk_ids, topk_w, hist);
+    route_block_tokens(logits, T, E, k, local_offset, n_local, rp, topk_ids, topk_w, hist);
     for (int e = tid; e < n_local; e += kFusedThreads) chunk_counts[(size_t)blockIdx.x * n_local + e] = hist[e];
     __threadfence();  // this block's ids, weights and histogram are visible before it is counted as done
     __syncthreads();
@@ -342,19 +469,19 @@ int choose_nt_max(int T, int E, int k) {
 
 cudaError_t launch_route(const float *logits, int T, int E, int k, LocalExperts local, int nt_max, int *topk_ids,
                          float *topk_w, int *expert_offsets, int *sorted_to_flat, int *flat_to_sorted,
-                         RouteScratch scratch, int *status, cudaStream_t stream, int row_quantum) {
+                         RouteScratch scratch, int *status, cudaStream_t stream, int row_quantum, RouterParams router) {
     cudaError_t err = cudaMemsetAsync(status, 0, 256, stream);  // the status word and its padding
     if (err != cudaSuccess) return err;
     const int A = T * k;
     if (scratch.n_chunks <= kFusedMaxChunks) {
         route_fused_kernel<<<scratch.n_chunks, kFusedThreads, 0, stream>>>(
-            logits, T, E, k, local.offset, local.count, nt_max, row_quantum, topk_ids, topk_w, scratch.chunk_counts,
+            logits, T, E, k, local.offset, local.count, nt_max, row_quantum, router, topk_ids, topk_w, scratch.chunk_counts,
             expert_offsets,
             scratch.tile_prefix, scratch.tile_order, scratch.tile_rows, sorted_to_flat, flat_to_sorted,
             status + kDoneCounterInt);
         return cudaGetLastError();
     }
-    route_topk_kernel<<<scratch.n_chunks, kRouteThreads, 0, stream>>>(logits, T, E, k, local.offset, local.count,
+    route_topk_kernel<<<scratch.n_chunks, kRouteThreads, 0, stream>>>(logits, T, E, k, local.offset, local.count, router,
                                                                        topk_ids, topk_w, scratch.chunk_counts);
     route_scan_kernel<<<1, 256, 0, stream>>>(scratch.chunk_counts, scratch.n_chunks, local.count, nt_max, row_quantum,
                                              expert_offsets,
