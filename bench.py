@@ -285,10 +285,19 @@ def run_ours(args):
     weight_bytes = int((w13.numel() + w2.numel()) * bytes_per_weight)
     need_flush = weight_bytes < 2 * L2_BYTES
 
+    grouped = None
+    if args.router == "grouped":  # the published DeepSeek-V3 setting: 8 groups, 4 eligible, weights scaled by 2.5
+        if not mx or E % 8 != 0 or (E // 8) & (E // 8 - 1) or 4 * (E // 8) < k:
+            raise SystemExit("--router grouped is wired for --weights mxfp8 and E = 8 groups of a power of two")
+        gen = torch.Generator(device=dev)
+        gen.manual_seed(args.seed + 1000 + rank)
+        router_bias = torch.randn(E, generator=gen, device=dev) * 0.1
+        grouped = moe.grouped_router(8, 4, router_bias, 2.5)
+
     def forward(events=None):
         if mx:
             moe.moe_forward_mxfp8(x, logits, w13, w13_sf, w2, w2_sf, k, out, ws, stage_events=events,
-                                  local_expert_offset=local_offset)
+                                  local_expert_offset=local_offset, router=grouped)
         elif fp8:
             moe.moe_forward_fp8w(x, logits, w13, w13_scale, w2, w2_scale, k, out, ws, stage_events=events)
         elif events is None:
@@ -343,7 +352,8 @@ def run_ours(args):
 
     def host_step():
         if mx:
-            moe.moe_forward_mxfp8_host(xh, lh, w13, w13_sf, w2, w2_sf, k, oh, ws, local_expert_offset=local_offset)
+            moe.moe_forward_mxfp8_host(xh, lh, w13, w13_sf, w2, w2_sf, k, oh, ws, local_expert_offset=local_offset,
+                                       router=grouped)
         elif fp8:  # no host-buffer entry point for this variant: the same copies, issued here on the same stream
             x_stage.copy_(xh, non_blocking=True)
             l_stage.copy_(lh, non_blocking=True)
@@ -427,7 +437,7 @@ def run_ours(args):
                 config=dict(workload=args.config, T=T, H=H, I=I, E=E, top_k=k, resident_experts=n_local,
                             weights="fp8 e4m3 codes + fp32 scale per 128x128 block" if fp8 else
                             "mxfp8: e4m3 codes + e8m0 scale per 32 elements, activations quantised on the fly" if mx else "bf16",
-                            parallelism=f"replicas x{world}",
+                            router=args.router, parallelism=f"replicas x{world}",
                             l2="flushed between steps" if need_flush else "weights larger than L2, no flush",
                             seed=args.seed),
                 clocks=clocks,
@@ -452,6 +462,8 @@ def main():
     ap.add_argument("--weights", choices=["bf16", "fp8", "mxfp8"], default="bf16",
                     help="fp8: expert weights as E4M3 codes with one fp32 scale per 128 x 128 block (moe_forward_fp8w); "
                          "mxfp8: weights and activations in MX FP8 on the block-scaled MMA (moe_forward_mxfp8)")
+    ap.add_argument("--router", choices=["softmax", "grouped"], default="softmax",
+                    help="grouped: sigmoid scores, selection bias, 8 groups of which 4 eligible, weights x 2.5 (with --weights mxfp8)")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -290,7 +290,10 @@ MOE_API int moe_mxfp8_pack_scales(const void *scales, int E, int rows, int K, in
 MOE_API int moe_mxfp8_quantize_rows(const void *x, int R, int K, void *codes, void *scales, void *stream);
 
 /* The layer in MX FP8, restricted to the resident experts as in moe_forward_local (pass 0 and E for all).
+ * With the grouped router and 32 resident experts of 256 this is the configuration the paper's kernel serves
+ * (Sec. 4.5: FP8, "DeepSeek-V3 style, top-8 routing", 32 local experts).
  *   x [T,H] bf16, router_logits [T,E] f32, out [T,H] bf16: as moe_forward; all DEVICE pointers
+ *   router  NULL for softmax -> top-k -> renormalise, else the grouped sigmoid router (moe_grouped_router_t)
  *   w13_q [n_local,2I,H] uint8 codes, w13_sf_packed: its scale bytes packed with gate_up = 1
  *   w2_q  [n_local,H,I]  uint8 codes, w2_sf_packed : its scale bytes packed with gate_up = 0
  *   workspace  at least moe_mxfp8_workspace_bytes bytes, 256-byte aligned (layout: moe_mxfp8_workspace_layout)
@@ -299,8 +302,9 @@ MOE_API int moe_mxfp8_quantize_rows(const void *x, int R, int K, void *codes, vo
  * 240 rows (128 when H is not a multiple of 256).  Errors as moe_forward; a block of x holding an infinity or NaN makes that token's output NaN. */
 MOE_API int moe_forward_mxfp8(const void *x, const float *router_logits, const void *w13_q, const void *w13_sf_packed,
                               const void *w2_q, const void *w2_sf_packed, int T, int H, int I, int E, int top_k,
-                              int local_expert_offset, int num_local_experts, void *out, void *workspace,
-                              size_t workspace_bytes, void *stream, void *const *stage_events);
+                              const moe_grouped_router_t *router, int local_expert_offset, int num_local_experts,
+                              void *out, void *workspace, size_t workspace_bytes, void *stream,
+                              void *const *stage_events);
 
 /* moe_forward_mxfp8 for a caller whose activations live in HOST memory, as moe_forward_host: x_host [T,H] bf16,
  * router_logits_host [T,E] f32 and out_host [T,H] bf16 are HOST pointers (pinned memory makes the copies
@@ -308,8 +312,9 @@ MOE_API int moe_forward_mxfp8(const void *x, const float *router_logits, const v
  * copies, the layer and the device-to-host copy on `stream` and returns without synchronising. */
 MOE_API int moe_forward_mxfp8_host(const void *x_host, const float *router_logits_host, const void *w13_q,
                                    const void *w13_sf_packed, const void *w2_q, const void *w2_sf_packed, int T, int H,
-                                   int I, int E, int top_k, int local_expert_offset, int num_local_experts,
-                                   void *out_host, void *workspace, size_t workspace_bytes, void *stream);
+                                   int I, int E, int top_k, const moe_grouped_router_t *router, int local_expert_offset,
+                                   int num_local_experts, void *out_host, void *workspace, size_t workspace_bytes,
+                                   void *stream);
 
 /* moe_forward_local (local_expert_offset = 0, num_local_experts = E for the whole layer) for a caller
  * whose activations live in HOST memory: x_host [T,H] bf16 and router_logits_host [T,E] f32 are HOST

@@ -99,9 +99,11 @@ def lib() -> ctypes.CDLL:
         L.moe_mxfp8_quantize_rows.restype = i
         L.moe_mxfp8_quantize_rows.argtypes = [vp, i, i, vp, vp, vp]
         L.moe_forward_mxfp8.restype = i
-        L.moe_forward_mxfp8.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, i, i, vp, vp, sz, vp, ctypes.POINTER(vp)]
+        L.moe_forward_mxfp8.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, ctypes.POINTER(GroupedRouter), i, i, vp, vp, sz,
+                                        vp, ctypes.POINTER(vp)]
         L.moe_forward_mxfp8_host.restype = i
-        L.moe_forward_mxfp8_host.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, i, i, vp, vp, sz, vp]
+        L.moe_forward_mxfp8_host.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, ctypes.POINTER(GroupedRouter), i, i, vp, vp,
+                                             sz, vp]
         L.moe_forward_staged.restype = i
         L.moe_forward_staged.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, vp, vp, sz, vp, ctypes.c_uint,
                                          ctypes.POINTER(vp)]
@@ -282,8 +284,10 @@ def moe_mxfp8_quantize_rows(x, stream=None):
 
 
 def moe_forward_mxfp8(x, router_logits, w13_q, w13_sf_packed, w2_q, w2_sf_packed, top_k: int, out, workspace,
-                      stream=None, stage_events=None, local_expert_offset: int = 0, check: bool = True) -> int:
-    """The layer in MX FP8 (E4M3 codes, packed E8M0 scale bytes); w13_q may hold a local subset of the experts."""
+                      stream=None, stage_events=None, local_expert_offset: int = 0, router: GroupedRouter = None,
+                      check: bool = True) -> int:
+    """The layer in MX FP8 (E4M3 codes, packed E8M0 scale bytes); w13_q may hold a local subset of the experts;
+    ``router`` = None for the softmax router, else a grouped_router(...)."""
     T, H = x.shape
     E = router_logits.shape[1]
     n_local, I2, _ = w13_q.shape
@@ -291,21 +295,24 @@ def moe_forward_mxfp8(x, router_logits, w13_q, w13_sf_packed, w2_q, w2_sf_packed
     if stage_events is not None:
         handles = (ctypes.c_void_p * (len(STAGE_NAMES) + 1))(*[e.cuda_event for e in stage_events])
     st = lib().moe_forward_mxfp8(_ptr(x), _ptr(router_logits), _ptr(w13_q), _ptr(w13_sf_packed), _ptr(w2_q),
-                                 _ptr(w2_sf_packed), T, H, I2 // 2, E, top_k, local_expert_offset, n_local, _ptr(out),
-                                 _ptr(workspace), workspace.numel(), _stream(stream), handles)
+                                 _ptr(w2_sf_packed), T, H, I2 // 2, E, top_k, None if router is None else ctypes.byref(router),
+                                 local_expert_offset, n_local, _ptr(out), _ptr(workspace), workspace.numel(),
+                                 _stream(stream), handles)
     if check and st != MOE_OK:
         raise MoeError(st, "moe_forward_mxfp8")
     return st
 
 
 def moe_forward_mxfp8_host(x_host, router_logits_host, w13_q, w13_sf_packed, w2_q, w2_sf_packed, top_k: int, out_host,
-                           workspace, stream=None, local_expert_offset: int = 0, check: bool = True) -> int:
+                           workspace, stream=None, local_expert_offset: int = 0, router: GroupedRouter = None,
+                           check: bool = True) -> int:
     """moe_forward_mxfp8 with CPU tensors for x, the router logits and the result (pinned for asynchronous copies)."""
     T, H = x_host.shape
     E = router_logits_host.shape[1]
     n_local, I2, _ = w13_q.shape
     st = lib().moe_forward_mxfp8_host(_ptr(x_host), _ptr(router_logits_host), _ptr(w13_q), _ptr(w13_sf_packed), _ptr(w2_q),
-                                      _ptr(w2_sf_packed), T, H, I2 // 2, E, top_k, local_expert_offset, n_local,
+                                      _ptr(w2_sf_packed), T, H, I2 // 2, E, top_k,
+                                      None if router is None else ctypes.byref(router), local_expert_offset, n_local,
                                       _ptr(out_host), _ptr(workspace), workspace.numel(), _stream(stream))
     if check and st != MOE_OK:
         raise MoeError(st, "moe_forward_mxfp8_host")

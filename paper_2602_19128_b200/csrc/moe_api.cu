@@ -202,10 +202,16 @@ void fill_mx_layout(int T, int H, int I, int E, int k, moe_mxfp8_workspace_layou
 
 int forward_mx_impl(const void *x, const float *logits, const void *w13_q, const void *w13_sf, const void *w2_q,
                     const void *w2_sf, int T, int H, int I, int E, int k, int local_offset, int n_local, void *out,
-                    void *workspace, size_t workspace_bytes, cudaStream_t stream, void *const *stage_events) {
+                    void *workspace, size_t workspace_bytes, cudaStream_t stream, void *const *stage_events,
+                    const moe_grouped_router_t *grouped) {
     if (T < 0 || H <= 0 || I <= 0 || E <= 0 || k <= 0 || k > E) return MOE_ERR_SHAPE;
     if (!mx_envelope_ok(T, H, I, E, k)) return MOE_ERR_UNSUPPORTED;
     if (local_offset < 0 || n_local < 1 || (long long)local_offset + n_local > E) return MOE_ERR_SHAPE;
+    RouterParams router;
+    if (grouped) {
+        const int rs_status = make_router(grouped, E, k, &router);
+        if (rs_status != MOE_OK) return rs_status;
+    }
     if (stage_events)
         for (int i = 0; i < MOE_NUM_STAGE_EVENTS; ++i)
             if (!stage_events[i]) return MOE_ERR_NULL;
@@ -241,7 +247,7 @@ int forward_mx_impl(const void *x, const float *logits, const void *w13_q, const
     if (!mark(0)) return MOE_ERR_CUDA;
     // every token tile exactly nt_max rows (the last of an expert partial): each tile owns one scale atom
     if (launch_route(logits, T, E, k, LocalExperts{local_offset, n_local}, nt_max, ids, wts, offsets, s2f, f2s, rs, status,
-                     stream, nt_max) != cudaSuccess)
+                     stream, nt_max, router) != cudaSuccess)
         return MOE_ERR_CUDA;
     if (!mark(1)) return MOE_ERR_CUDA;
     if (launch_mx_gather_quantize(static_cast<const __nv_bfloat16 *>(x), s2f, offsets, n_local, A, k, H, x_q, x_sf, n_atoms,
@@ -317,8 +323,8 @@ int moe_mxfp8_quantize_rows(const void *x, int R, int K, void *codes, void *scal
 
 int moe_forward_mxfp8_host(const void *x_host, const float *router_logits_host, const void *w13_q,
                            const void *w13_sf_packed, const void *w2_q, const void *w2_sf_packed, int T, int H, int I, int E,
-                           int top_k, int local_expert_offset, int num_local_experts, void *out_host, void *workspace,
-                           size_t workspace_bytes, void *stream) {
+                           int top_k, const moe_grouped_router_t *router, int local_expert_offset, int num_local_experts,
+                           void *out_host, void *workspace, size_t workspace_bytes, void *stream) {
     if (T < 0 || H <= 0 || I <= 0 || E <= 0 || top_k <= 0 || top_k > E || num_local_experts < 1) return MOE_ERR_SHAPE;
     if (!mx_envelope_ok(T, H, I, E, top_k)) return MOE_ERR_UNSUPPORTED;
     if (T == 0) return MOE_OK;
@@ -337,7 +343,7 @@ int moe_forward_mxfp8_host(const void *x_host, const float *router_logits_host, 
     if (cudaMemcpyAsync(l_dev, router_logits_host, l_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return MOE_ERR_CUDA;
     const int st = forward_mx_impl(x_dev, reinterpret_cast<const float *>(l_dev), w13_q, w13_sf_packed, w2_q, w2_sf_packed, T,
                                    H, I, E, top_k, local_expert_offset, num_local_experts, out_dev, workspace,
-                                   workspace_bytes, s, nullptr);
+                                   workspace_bytes, s, nullptr, router);
     if (st != MOE_OK) return st;
     if (cudaMemcpyAsync(out_host, out_dev, x_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) return MOE_ERR_CUDA;
     return MOE_OK;
@@ -345,11 +351,11 @@ int moe_forward_mxfp8_host(const void *x_host, const float *router_logits_host, 
 
 int moe_forward_mxfp8(const void *x, const float *router_logits, const void *w13_q, const void *w13_sf_packed,
                       const void *w2_q, const void *w2_sf_packed, int T, int H, int I, int E, int top_k,
-                      int local_expert_offset, int num_local_experts, void *out, void *workspace, size_t workspace_bytes,
-                      void *stream, void *const *stage_events) {
+                      const moe_grouped_router_t *router, int local_expert_offset, int num_local_experts, void *out,
+                      void *workspace, size_t workspace_bytes, void *stream, void *const *stage_events) {
     return forward_mx_impl(x, router_logits, w13_q, w13_sf_packed, w2_q, w2_sf_packed, T, H, I, E, top_k,
                            local_expert_offset, num_local_experts, out, workspace, workspace_bytes,
-                           static_cast<cudaStream_t>(stream), stage_events);
+                           static_cast<cudaStream_t>(stream), stage_events, router);
 }
 
 size_t moe_workspace_bytes(int T, int H, int I, int E, int top_k) {

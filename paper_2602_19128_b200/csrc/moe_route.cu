@@ -3,7 +3,8 @@
 // Paper, Sec. 4.5 "Routing": each token gets scores for E experts and the top k are picked with
 // warp-level cooperation; "Expert FFN computation", step (2): tokens are reordered by expert into
 // contiguous memory.  Here one warp owns one token (E <= 256 logits fit in 8 registers per lane),
-// selection is k rounds of a warp arg-max under the strict order
+// selection is k rounds of a warp arg-max (two warp reductions per round: the largest order-preserving
+// key, then the lowest index holding it) under the strict order
 //     e before e'  <=>  logit[e] > logit[e']  or  (logit[e] == logit[e'] and e < e'),
 // and the sort-scatter is a counting sort made stable without ordered atomics:
 //   1. every router block histograms the assignments of its own 32 tokens (one "chunk");
@@ -22,66 +23,65 @@ namespace moe {
 namespace {
 
 constexpr unsigned kFullMask = 0xffffffffu;
-constexpr int kRouteThreads = 256;
+constexpr int kRouteThreads = 1024;  // one warp per token of the block's 32-token chunk
 constexpr int kLogitsPerLane = kMaxExperts / 32;
 
-// Router for one token by one warp: softmax over the E logits (8 per lane), k rounds of a warp arg-max
-// under the strict order, renormalisation.  Lane j < k returns rank j's expert and weight.
-__device__ __forceinline__ void route_one_token(const float *__restrict__ row, int E, int k, int lane, int &my_id,
-                                                float &my_w) {
-    float v[kLogitsPerLane], p[kLogitsPerLane];
-    float m = -INFINITY;
-#pragma unroll
-    for (int i = 0; i < kLogitsPerLane; ++i) {
-        const int e = i * 32 + lane;
-        v[i] = e < E ? row[e] : -INFINITY;
-        m = fmaxf(m, v[i]);
-    }
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(kFullMask, m, off));
-    float s = 0.f;
-#pragma unroll
-    for (int i = 0; i < kLogitsPerLane; ++i) {
-        const int e = i * 32 + lane;
-        p[i] = e < E ? expf(v[i] - m) : 0.f;
-        s += p[i];
-    }
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(kFullMask, s, off);
-#pragma unroll
-    for (int i = 0; i < kLogitsPerLane; ++i) p[i] = p[i] / s;
+// Order-preserving map from float to unsigned: a > b  <=>  ordered_key(a) > ordered_key(b) (for non-NaN values;
+// -0 is first folded into +0 so that the two compare equal, as the floats do).
+__device__ __forceinline__ unsigned ordered_key(float f) {
+    const unsigned u = __float_as_uint(f + 0.0f);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
 
+// k rounds of a warp arg-max under the strict order (larger key first, ties to the lower expert index).  Expert
+// e = 32 i + lane has key[i] in its lane; entries with e >= E must hold key 0 and are never selected while a real
+// candidate is left.  Each round: every lane finds its best remaining entry, one warp reduction gives the largest
+// key, a second one the lowest expert index among the lanes that hold it.  Lane j < k returns rank j's expert.
+__device__ __forceinline__ int select_top_k(const unsigned (&key)[kLogitsPerLane], int E, int k, int lane) {
     unsigned taken = 0;
-    float my_p = 0.f;
-    my_id = 0;
+    int my_id = 0;
     for (int j = 0; j < k; ++j) {
-        // best candidate among this lane's experts that are still available
-        int ci = INT_MAX;
-        float cv = -INFINITY, cp = 0.f;
+        unsigned best = 0;
+        int best_e = INT_MAX;  // no candidate
 #pragma unroll
         for (int i = 0; i < kLogitsPerLane; ++i) {
             const int e = i * 32 + lane;
-            if (e < E && !((taken >> i) & 1u) && (ci == INT_MAX || v[i] > cv)) {
-                ci = e; cv = v[i]; cp = p[i];
-            }
+            const bool free_slot = e < E && !((taken >> i) & 1u);
+            if (free_slot && (best_e == INT_MAX || key[i] > best)) { best = key[i]; best_e = e; }
         }
-        // warp arg-max; INT_MAX marks "no candidate" and always loses
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) {
-            const float ov = __shfl_xor_sync(kFullMask, cv, off);
-            const int oi = __shfl_xor_sync(kFullMask, ci, off);
-            const float op = __shfl_xor_sync(kFullMask, cp, off);
-            const bool other = (ci == INT_MAX) ? (oi != INT_MAX)
-                                               : (oi != INT_MAX && (ov > cv || (ov == cv && oi < ci)));
-            if (other) { cv = ov; ci = oi; cp = op; }
-        }
-        // with non-finite logits lanes could disagree; lane 0's answer is the warp's answer
-        ci = __shfl_sync(kFullMask, ci, 0);
-        cp = __shfl_sync(kFullMask, cp, 0);
-        if (ci == INT_MAX) ci = 0;  // unreachable for k <= E; keeps the index in range regardless
-        if ((ci & 31) == lane) taken |= 1u << (ci >> 5);
-        if (lane == j) { my_id = ci; my_p = cp; }
+        const unsigned top = __reduce_max_sync(kFullMask, best_e == INT_MAX ? 0u : best);
+        int winner = (int)__reduce_min_sync(kFullMask, (best_e != INT_MAX && best == top) ? (unsigned)best_e : 0xffffffffu);
+        if (winner < 0 || winner >= E) winner = 0;  // unreachable for k <= E; keeps the index in range regardless
+        if ((winner & 31) == lane) taken |= 1u << (winner >> 5);
+        if (lane == j) my_id = winner;
     }
+    return my_id;
+}
+
+// Router for one token by one warp: top-k of the E logits (8 per lane) under the strict order, then the
+// renormalised softmax weights.  Softmax's normaliser cancels in the renormalisation, so only the k selected
+// logits are exponentiated: w_j = exp(l_j - l_0) / sum_j' exp(l_j' - l_0), the sum in rank order.
+// Lane j < k returns rank j's expert and weight.
+__device__ __forceinline__ void route_one_token(const float *__restrict__ row, int E, int k, int lane, int &my_id,
+                                                float &my_w) {
+    float v[kLogitsPerLane];
+    unsigned key[kLogitsPerLane];
+#pragma unroll
+    for (int i = 0; i < kLogitsPerLane; ++i) {
+        const int e = i * 32 + lane;
+        v[i] = e < E ? row[e] : 0.f;
+        key[i] = e < E ? ordered_key(v[i]) : 0u;
+    }
+    my_id = select_top_k(key, E, k, lane);
+    // the selected logit lives in lane my_id % 32, register my_id / 32
+    float my_l = 0.f;
+#pragma unroll
+    for (int i = 0; i < kLogitsPerLane; ++i) {
+        const float got = __shfl_sync(kFullMask, v[i], my_id & 31);
+        if ((my_id >> 5) == i) my_l = got;
+    }
+    const float top_l = __shfl_sync(kFullMask, my_l, 0);  // rank 0 holds the largest logit
+    const float my_p = lane < k ? expf(my_l - top_l) : 0.f;
     float denom = 0.f;  // ascending rank, the order the definition states
     for (int j = 0; j < k; ++j) denom += __shfl_sync(kFullMask, my_p, j);
     my_w = my_p / denom;
@@ -155,55 +155,59 @@ __device__ __forceinline__ void route_one_token_grouped(const float *__restrict_
     float gs[kLogitsPerLane];  // score of the group that holds this register's expert
 #pragma unroll
     for (int i = 0; i < kLogitsPerLane; ++i) gs[i] = G >= 2 ? __fadd_rn(t1[i], t2[i]) : t1[i];
-    // rank of that group among all groups (ties to the lower group index); eligible if below topk_group
-    int rank[kLogitsPerLane];
-#pragma unroll
-    for (int i = 0; i < kLogitsPerLane; ++i) rank[i] = 0;
-    for (int g = 0; g < rp.n_group; ++g) {
-        const int e0 = g * G, ip = e0 >> 5;
-        float pick = gs[0];
-#pragma unroll
-        for (int i = 1; i < kLogitsPerLane; ++i) pick = ip == i ? gs[i] : pick;
-        const float val = __shfl_sync(kFullMask, pick, e0 & 31);
+    // a group is eligible if fewer than topk_group groups rank before it (ties to the lower group index)
+    if (rp.n_group <= 32) {
+        // lane g fetches group g's score from the lane and register that hold the group's first expert ...
+        const int first = lane < rp.n_group ? lane * G : 0;
+        float mine = 0.f;
 #pragma unroll
         for (int i = 0; i < kLogitsPerLane; ++i) {
-            const int gid = (i * 32 + lane) / G;
-            rank[i] += (val > gs[i] || (val == gs[i] && g < gid)) ? 1 : 0;
+            const float got = __shfl_sync(kFullMask, gs[i], first & 31);
+            if ((first >> 5) == i) mine = got;
         }
-    }
+        // ... ranks it against the others, and the eligible groups become a bit mask
+        int rank = 0;
+        for (int g = 0; g < rp.n_group; ++g) {
+            const float val = __shfl_sync(kFullMask, mine, g);
+            rank += (val > mine || (val == mine && g < lane)) ? 1 : 0;
+        }
+        const unsigned eligible = __ballot_sync(kFullMask, lane < rp.n_group && rank < rp.topk_group);
 #pragma unroll
-    for (int i = 0; i < kLogitsPerLane; ++i)
-        if (rank[i] >= rp.topk_group) c[i] = -INFINITY;
-
-    // k rounds of a warp arg-max over the eligible biased scores; the payload is the unbiased score
-    unsigned taken = 0;
-    float my_s = 0.f;
-    my_id = 0;
-    for (int j = 0; j < k; ++j) {
-        int ci = INT_MAX;
-        float cv = -INFINITY, cp = 0.f;
+        for (int i = 0; i < kLogitsPerLane; ++i)
+            if (!((eligible >> ((i * 32 + lane) / G)) & 1u)) c[i] = -INFINITY;
+    } else {  // more groups than lanes (groups of at most 4 experts): every register ranks its own group
+        int rank[kLogitsPerLane];
 #pragma unroll
-        for (int i = 0; i < kLogitsPerLane; ++i) {
-            const int e = i * 32 + lane;
-            if (e < E && !((taken >> i) & 1u) && (ci == INT_MAX || c[i] > cv)) {
-                ci = e; cv = c[i]; cp = s[i];
+        for (int i = 0; i < kLogitsPerLane; ++i) rank[i] = 0;
+        for (int g = 0; g < rp.n_group; ++g) {
+            const int e0 = g * G, ip = e0 >> 5;
+            float pick = gs[0];
+#pragma unroll
+            for (int i = 1; i < kLogitsPerLane; ++i) pick = ip == i ? gs[i] : pick;
+            const float val = __shfl_sync(kFullMask, pick, e0 & 31);
+#pragma unroll
+            for (int i = 0; i < kLogitsPerLane; ++i) {
+                const int gid = (i * 32 + lane) / G;
+                rank[i] += (val > gs[i] || (val == gs[i] && g < gid)) ? 1 : 0;
             }
         }
 #pragma unroll
-        for (int off = 16; off > 0; off >>= 1) {
-            const float ov = __shfl_xor_sync(kFullMask, cv, off);
-            const int oi = __shfl_xor_sync(kFullMask, ci, off);
-            const float op = __shfl_xor_sync(kFullMask, cp, off);
-            const bool other = (ci == INT_MAX) ? (oi != INT_MAX)
-                                               : (oi != INT_MAX && (ov > cv || (ov == cv && oi < ci)));
-            if (other) { cv = ov; ci = oi; cp = op; }
-        }
-        ci = __shfl_sync(kFullMask, ci, 0);
-        cp = __shfl_sync(kFullMask, cp, 0);
-        if (ci == INT_MAX) ci = 0;
-        if ((ci & 31) == lane) taken |= 1u << (ci >> 5);
-        if (lane == j) { my_id = ci; my_s = cp; }
+        for (int i = 0; i < kLogitsPerLane; ++i)
+            if (rank[i] >= rp.topk_group) c[i] = -INFINITY;
     }
+
+    // top-k of the eligible biased scores; the weight uses the unbiased score of the selected expert
+    unsigned key[kLogitsPerLane];
+#pragma unroll
+    for (int i = 0; i < kLogitsPerLane; ++i) key[i] = i * 32 + lane < E ? ordered_key(c[i]) : 0u;
+    my_id = select_top_k(key, E, k, lane);
+    float my_s = 0.f;
+#pragma unroll
+    for (int i = 0; i < kLogitsPerLane; ++i) {
+        const float got = __shfl_sync(kFullMask, s[i], my_id & 31);
+        if ((my_id >> 5) == i) my_s = got;
+    }
+    if (lane >= k) my_s = 0.f;
     float denom = 0.f;  // ascending rank
     for (int j = 0; j < k; ++j) denom = __fadd_rn(denom, __shfl_sync(kFullMask, my_s, j));
     my_w = __fmul_rn(__fdiv_rn(my_s, denom), rp.scale);
@@ -270,36 +274,64 @@ __device__ __forceinline__ int block_exclusive_scan_256(int value, int *warp_sum
     return base + incl - value;
 }
 
-// Scan phase, run by one block (threads 0..255 carry one expert each; wider blocks idle the rest):
+constexpr int kScanThreads = 1024;
+
+// Scan phase, run by one block of a multiple of 256 threads (threads 0..255 carry one expert each for the schedule):
 // per-expert running sum over chunks, exclusive scan over experts, token-tile schedule.
 // (Pointers are deliberately not __restrict__ and cross-block data is read with __ldcg: in the fused
 // kernel these arrays were written by other blocks, or are written here and read again by the scatter.)
 __device__ __forceinline__ void scan_phase(int *chunk_counts, int n_chunks, int E, int nt_max, int row_quantum, int *expert_offsets,
                                            int *tile_prefix, int *tile_order, int *tile_rows, int *warp_sums,
-                                           int *counts, int *tiles_at) {
+                                           int *counts, int *tiles_at, int *part_sums) {
     const int e = threadIdx.x;
     const bool lane_of_scan = e < kMaxExperts;
+    // Running sum over chunks per expert.  The block's threads form blockDim.x / 256 parts; part p of expert e
+    // first totals its share of the chunks, then, knowing the totals of the parts before it, replaces each of its
+    // chunk counts by the rows of all earlier chunks.  (16 independent loads in flight at a time: latency-bound.)
     int count = 0;
-    if (e < E) {
-        // running sum over chunks, 16 independent loads in flight at a time (the loop is latency-bound)
+    {
         constexpr int kBatch = 16;
-        for (int b0 = 0; b0 < n_chunks; b0 += kBatch) {
-            int c[kBatch];
+        const int pe = threadIdx.x % kMaxExperts, part = threadIdx.x / kMaxExperts, n_parts = blockDim.x / kMaxExperts;
+        const int per = (n_chunks + n_parts - 1) / n_parts;
+        const int b_begin = min(n_chunks, part * per), b_end = min(n_chunks, b_begin + per);
+        int sum = 0;
+        if (pe < E) {
+            for (int b0 = b_begin; b0 < b_end; b0 += kBatch) {
+                int c[kBatch];
 #pragma unroll
-            for (int i = 0; i < kBatch; ++i) c[i] = b0 + i < n_chunks ? __ldcg(&chunk_counts[(size_t)(b0 + i) * E + e]) : 0;
+                for (int i = 0; i < kBatch; ++i) c[i] = b0 + i < b_end ? __ldcg(&chunk_counts[(size_t)(b0 + i) * E + pe]) : 0;
 #pragma unroll
-            for (int i = 0; i < kBatch; ++i) {
-                if (b0 + i < n_chunks) chunk_counts[(size_t)(b0 + i) * E + e] = count;
-                count += c[i];
+                for (int i = 0; i < kBatch; ++i) sum += c[i];
             }
         }
+        part_sums[part * kMaxExperts + pe] = sum;
+        __syncthreads();
+        int run = 0;
+        for (int p = 0; p < n_parts; ++p) {
+            const int v = part_sums[p * kMaxExperts + pe];
+            if (p < part) run += v;
+            count += v;
+        }
+        if (pe < E) {
+            for (int b0 = b_begin; b0 < b_end; b0 += kBatch) {
+                int c[kBatch];
+#pragma unroll
+                for (int i = 0; i < kBatch; ++i) c[i] = b0 + i < b_end ? __ldcg(&chunk_counts[(size_t)(b0 + i) * E + pe]) : 0;
+#pragma unroll
+                for (int i = 0; i < kBatch; ++i) {
+                    if (b0 + i < b_end) chunk_counts[(size_t)(b0 + i) * E + pe] = run;
+                    run += c[i];
+                }
+            }
+        }
+        if (!lane_of_scan || e >= E) count = 0;  // the schedule below is built by threads 0..E-1
     }
     if (lane_of_scan) {
         counts[e] = e < E ? count : -1;
         tiles_at[e] = 0;
     }
     // token tiles of this expert: as few as fit under nt_max, evenly sized, rounded up to the row quantum
-    // (16 rows, the MMA's N granularity; 32 for the MX kernels, whose scale factors come in groups of 32 rows)
+    // (16 rows, the MMA's N granularity; the MX path passes its tile size, so that every tile is exactly that many rows)
     int n_tiles = 0, rows = 0;
     if (count > 0) {
         n_tiles = (count + nt_max - 1) / nt_max;
@@ -311,6 +343,7 @@ __device__ __forceinline__ void scan_phase(int *chunk_counts, int n_chunks, int 
     // cost are adjacent and the GEMMs' static tile assignment stays balanced; the small tiles come last.
     if (e < E) {
         int pos = 0;
+#pragma unroll 8
         for (int o = 0; o < E; ++o) pos += (counts[o] > count || (counts[o] == count && o < e)) ? 1 : 0;
         tiles_at[pos] = n_tiles;
         tile_order[pos] = e;
@@ -328,13 +361,13 @@ __device__ __forceinline__ void scan_phase(int *chunk_counts, int n_chunks, int 
     }
 }
 
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(kScanThreads)
 route_scan_kernel(int *chunk_counts, int n_chunks, int E, int nt_max, int row_quantum, int *expert_offsets,
                   int *tile_prefix, int *tile_order, int *tile_rows) {
     __shared__ int warp_sums[8];
-    __shared__ int counts[kMaxExperts], tiles_at[kMaxExperts];
+    __shared__ int counts[kMaxExperts], tiles_at[kMaxExperts], part_sums[kScanThreads];
     scan_phase(chunk_counts, n_chunks, E, nt_max, row_quantum, expert_offsets, tile_prefix, tile_order, tile_rows, warp_sums,
-               counts, tiles_at);
+               counts, tiles_at, part_sums);
 }
 
 // Stable scatter of one chunk (32 tokens) by one warp; next[] is that warp's per-expert cursor.
@@ -342,25 +375,46 @@ __device__ __forceinline__ void scatter_chunk(int chunk, const int *topk_ids, co
                                               const int *expert_offsets, int A, int n_local, int local_offset, int k,
                                               int *sorted_to_flat, int *flat_to_sorted, int *next, int lane) {
     // first position of this chunk's assignments to expert e = segment start + rows of earlier chunks
-    for (int e = lane; e < n_local; e += 32)
-        next[e] = __ldcg(&expert_offsets[e]) + __ldcg(&chunk_starts[(size_t)chunk * n_local + e]);
+    // (all loads issued before the first use: the loop is a chain of L2 round trips otherwise)
+    {
+        int start[kMaxExperts / 32];
+#pragma unroll
+        for (int i = 0; i < kMaxExperts / 32; ++i) {
+            const int e = i * 32 + lane;
+            start[i] = e < n_local ? __ldcg(&expert_offsets[e]) + __ldcg(&chunk_starts[(size_t)chunk * n_local + e]) : 0;
+        }
+#pragma unroll
+        for (int i = 0; i < kMaxExperts / 32; ++i)
+            if (i * 32 + lane < n_local) next[i * 32 + lane] = start[i];
+    }
     __syncwarp();
     const int a0 = chunk * kRouteTokensPerBlock * k;
     const int a1 = min(A, a0 + kRouteTokensPerBlock * k);
-    for (int base = a0; base < a1; base += 32) {
-        const int a = base + lane;
-        const bool valid = a < a1;
-        const int e = valid ? __ldcg(&topk_ids[a]) - local_offset : -1;
-        const bool kept = e >= 0 && e < n_local;       // assignments to experts that are not resident are dropped
-        const int key = kept ? e : -1 - lane;          // ... and never match anything
-        const unsigned same = __match_any_sync(kFullMask, key);
-        const int rank = __popc(same & ((1u << lane) - 1u));
-        const int pos = kept ? next[e] + rank : -1;
-        __syncwarp();
-        if (kept && rank == 0) next[e] += __popc(same);
-        __syncwarp();
-        if (valid) flat_to_sorted[a] = pos;
-        if (kept) sorted_to_flat[pos] = a;
+    constexpr int kAhead = 4;  // groups of 32 assignments whose ids are fetched together
+    for (int base0 = a0; base0 < a1; base0 += 32 * kAhead) {
+        int ids[kAhead];
+#pragma unroll
+        for (int u = 0; u < kAhead; ++u) {
+            const int a = base0 + u * 32 + lane;
+            ids[u] = a < a1 ? __ldcg(&topk_ids[a]) - local_offset : -1;
+        }
+#pragma unroll
+        for (int u = 0; u < kAhead; ++u) {
+            const int a = base0 + u * 32 + lane;
+            if (base0 + u * 32 >= a1) break;  // uniform over the warp
+            const bool valid = a < a1;
+            const int e = ids[u];
+            const bool kept = valid && e >= 0 && e < n_local;  // assignments to experts that are not resident are dropped
+            const int key = kept ? e : -1 - lane;             // ... and never match anything
+            const unsigned same = __match_any_sync(kFullMask, key);
+            const int rank = __popc(same & ((1u << lane) - 1u));
+            const int pos = kept ? next[e] + rank : -1;
+            __syncwarp();
+            if (kept && rank == 0) next[e] += __popc(same);
+            __syncwarp();
+            if (valid) flat_to_sorted[a] = pos;
+            if (kept) sorted_to_flat[pos] = a;
+        }
     }
 }
 
@@ -383,7 +437,7 @@ __global__ void __launch_bounds__(kFusedThreads)
 route_fused_kernel(const float *__restrict__ logits, int T, int E, int k, int local_offset, int n_local, int nt_max,
                    int row_quantum, const RouterParams rp, int *topk_ids, float *topk_w, int *chunk_counts, int *expert_offsets, int *tile_prefix,
                    int *tile_order, int *tile_rows, int *sorted_to_flat, int *flat_to_sorted, int *done_counter) {
-    __shared__ int hist[kMaxExperts], counts[kMaxExperts], tiles_at[kMaxExperts], warp_sums[8];
+    __shared__ int hist[kMaxExperts], counts[kMaxExperts], tiles_at[kMaxExperts], warp_sums[8], part_sums[kFusedThreads];
     __shared__ int next[kFusedMaxChunks][kMaxExperts];
     __shared__ int is_last;
     const int tid = threadIdx.x;
@@ -397,7 +451,7 @@ route_fused_kernel(const float *__restrict__ logits, int T, int E, int k, int lo
     __threadfence();
     const int n_chunks = gridDim.x;
     scan_phase(chunk_counts, n_chunks, n_local, nt_max, row_quantum, expert_offsets, tile_prefix, tile_order, tile_rows,
-               warp_sums, counts, tiles_at);
+               warp_sums, counts, tiles_at, part_sums);
     __syncthreads();  // expert_offsets and the chunk starts written above are read below (same block)
     const int warp = tid >> 5;
     if (warp < n_chunks)
@@ -483,7 +537,7 @@ cudaError_t launch_route(const float *logits, int T, int E, int k, LocalExperts 
     }
     route_topk_kernel<<<scratch.n_chunks, kRouteThreads, 0, stream>>>(logits, T, E, k, local.offset, local.count, router,
                                                                        topk_ids, topk_w, scratch.chunk_counts);
-    route_scan_kernel<<<1, 256, 0, stream>>>(scratch.chunk_counts, scratch.n_chunks, local.count, nt_max, row_quantum,
+    route_scan_kernel<<<1, kScanThreads, 0, stream>>>(scratch.chunk_counts, scratch.n_chunks, local.count, nt_max, row_quantum,
                                              expert_offsets,
                                              scratch.tile_prefix, scratch.tile_order, scratch.tile_rows);
     route_scatter_kernel<<<scratch.n_chunks, 32, 0, stream>>>(topk_ids, scratch.chunk_counts, expert_offsets, A,

@@ -208,3 +208,46 @@ def test_mxfp8_host_entry_point_equals_the_device_one():
     torch.cuda.synchronize()
     assert moe.moe_last_status(ws) == moe.MOE_OK
     assert torch.equal(oh.view(torch.int16), out.cpu().view(torch.int16))
+
+
+def test_mxfp8_with_grouped_router_and_local_experts():
+    """The configuration the paper's kernel serves, scaled down: FP8 operands, grouped sigmoid routing, a resident
+    subset of the experts."""
+    cfg = dict(T=180, H=256, I=128, E=32, top_k=4, skew=False)
+    full = make_mxfp8_inputs(cfg, seed=8, device="cuda")
+    lo, n = 8, 16
+    inp = dict(full)
+    for key in ("w13_q", "w13_s", "w2_q", "w2_s"):
+        inp[key] = full[key][lo:lo + n].contiguous()
+    bias = torch.linspace(-0.2, 0.2, 32).cuda()
+    T, H, I, E, k = 180, 256, 128, 32, 4
+    ws = moe.alloc_workspace(moe.moe_mxfp8_workspace_bytes(T, H, I, E, k), "cuda")
+    ws.fill_(0xFF)
+    out = torch.full((T, H), float("nan"), dtype=torch.bfloat16, device="cuda")
+    moe.moe_forward_mxfp8(inp["x"], inp["router_logits"], inp["w13_q"], moe.moe_mxfp8_pack_scales(inp["w13_s"], True),
+                          inp["w2_q"], moe.moe_mxfp8_pack_scales(inp["w2_s"], False), k, out, ws, local_expert_offset=lo,
+                          router=moe.grouped_router(4, 2, bias, 2.5))
+    assert moe.moe_last_status(ws) == moe.MOE_OK
+    o = moe_oracle.get("f32")
+    logits = full["router_logits"].cpu().numpy()
+    ids, w = o.route_grouped(logits, k, 4, 2, bias=bias.cpu().numpy(), scale=2.5)
+    views = moe.mx_workspace_views(ws, T, H, I, E, k)
+    assert np.array_equal(views["topk_ids"].cpu().numpy(), ids)
+    assert np.array_equal(views["topk_weights"].cpu().numpy(), w)
+    # reference: every expert applied to its tokens by the oracle's sampled MX form, combined with the grouped
+    # weights here, assignments to experts that are not resident dropped
+    tokens = np.arange(T, dtype=np.int32)
+    ref = np.zeros((T, H))
+    host = {key: full[key].cpu().numpy() for key in ("w13_q", "w13_s", "w2_q", "w2_s")}
+    xb = bf16_bits(full["x"])
+    for e in range(lo, lo + n):
+        sel = np.nonzero((ids == e).any(axis=1))[0].astype(np.int32)
+        if len(sel) == 0:
+            continue
+        # a one-expert layer (k = 1, every logit column but e irrelevant): its output is expert e applied to the token
+        one = o.forward_mxfp8(xb[sel], np.zeros((len(sel), 1), np.float32), host["w13_q"][e:e + 1], host["w13_s"][e:e + 1],
+                              host["w2_q"][e:e + 1], host["w2_s"][e:e + 1], 1)
+        wsel = np.array([w[t][list(ids[t]).index(e)] for t in sel])
+        ref[sel] += wsel[:, None] * one
+    err = np.abs(bf16_to_f64(out) - ref)
+    assert np.all(err <= 2e-2 * (2.5 + np.abs(ref)))
