@@ -41,6 +41,9 @@ CASES = [
     (1500, 256, 8, 8, 4),     # three-kernel router
     (77, 48, 5, 3, 2),        # E not a multiple of 32, G = 16
     (1, 8, 2, 4, 2),
+    (90, 64, 5, 64, 9),       # more groups than lanes (groups of one): the per-register ranking path
+    (60, 256, 8, 128, 6),     # 128 groups of two
+    (40, 256, 32, 8, 4),      # top_k = 32
 ]
 
 

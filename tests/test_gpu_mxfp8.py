@@ -113,6 +113,10 @@ CASES = [
     (1000, 512, 384, 4, 2, False),    # ~500 rows per expert: three pair tiles each, several feature tiles
     (130, 256, 256, 4, 2, False),     # 128-row pair tiles (one atom each)
     (300, 256, 128, 16, 4, True),     # the same, skewed: popular experts spill into a second tile
+    (64, 128, 128, 64, 32, False),    # top_k = 32
+    (2000, 128, 128, 1, 1, False),    # one expert, sixteen 128-row tiles: gate/up on pairs, down (H % 256 != 0) on one CTA
+    (2000, 256, 128, 1, 1, False),    # one expert, nine 240-row tiles on pairs
+    (33, 640, 384, 5, 3, False),      # H, I multiples of 128 only; E not a power of two
 ]
 
 
