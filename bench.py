@@ -319,20 +319,35 @@ def run_ours(args):
     status = moe.moe_last_status(ws)
     if status != moe.MOE_OK:
         raise SystemExit(f"device status {status}: {moe.moe_status_string(status)}")
-    stage_events = [moe.make_stage_events() for _ in range(args.steps)]
+    # The K timed steps run as a user's would: no event between the kernels of a step (an event record between two
+    # launches costs several microseconds of launch pipelining).  With an L2 flush between steps each step gets its
+    # own pair of events; otherwise one pair brackets all K.
+    step_events = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                   for _ in range(args.steps if need_flush else 1)]
     barrier()
     sampler = ClockSampler(local) if rank == 0 else None
+    if not need_flush:
+        step_events[0][0].record()
     for s in range(args.steps):
+        if need_flush:
+            flush_l2(flush_buf)
+            step_events[s][0].record()
+        forward()
+        if need_flush:
+            step_events[s][1].record()
+    if not need_flush:
+        step_events[0][1].record()
+    barrier()
+    clocks = sampler.stop() if sampler else None
+    total_ms = sum(a.elapsed_time(b) for a, b in step_events)
+    # Per-kernel times: the same steps again, instrumented with an event between the stages.
+    n_staged = min(args.steps, 100)
+    stage_events = [moe.make_stage_events() for _ in range(n_staged)]
+    for s in range(n_staged):
         if need_flush:
             flush_l2(flush_buf)
         forward(stage_events[s])
     barrier()
-    clocks = sampler.stop() if sampler else None
-    if need_flush:
-        step_ms = [ev[0].elapsed_time(ev[-1]) for ev in stage_events]
-        total_ms = sum(step_ms)
-    else:
-        total_ms = stage_events[0][0].elapsed_time(stage_events[-1][-1])
     stage_ms = {name: statistics.fmean(ev[i].elapsed_time(ev[i + 1]) for ev in stage_events)
                 for i, name in enumerate(moe.STAGE_NAMES)}
     total_ms = max_over_ranks(dist, total_ms, dev)
@@ -412,10 +427,14 @@ def run_ours(args):
                     unit=unit, frac=achieved / peak, peak_source=f"of {peaks['source']}",
                     traffic=None if (fp8 or mx) else NCU_TRAFFIC_BYTES.get(args.config), algorithmic_per_launch=algorithmic,
                     kernel_ms=stage_ms["gemm1_swiglu"])
-    per_step_ms = sorted(ev[0].elapsed_time(ev[-1]) for ev in stage_events)
+    # per-step latencies: from the timed steps when each has its own events, else from the instrumented pass
+    per_step_ms = sorted(a.elapsed_time(b) for a, b in step_events) if need_flush else \
+        sorted(ev[0].elapsed_time(ev[-1]) for ev in stage_events)
     tile_bound = int(views["tile_rows"]) if mx else token_tile_bound(T, E, k)
     layer = dict(stage_ms={n: round(v, 5) for n, v in stage_ms.items()}, n_active_experts=n_active,
                  latency_ms_median=statistics.median(per_step_ms), latency_ms_min=per_step_ms[0],
+                 latency_source="timed steps" if need_flush else "instrumented pass (events between the stages)",
+                 stage_ms_source=f"instrumented pass of {n_staged} steps after the timed ones",
                  padding_efficiency=rows_scheduled / max(1, computed_rows(counts, tile_bound, even=not mx)),
                  weight_gbs_frac_nominal=active_weight_bytes / step_s / 1e9 / 8000.0,
                  useful_tflops_frac_nominal=6.0 * A * H * I / step_s / 1e12 / (4500.0 if mx else 2250.0),

@@ -87,6 +87,7 @@ grouped_gemm_tc_fp8w_kernel(const __grid_constant__ TensorMaps maps, const Kerne
     using L = Fp8Smem<NT_MAX, STAGES, CONV>;
     constexpr int kTmemCols = 2 * NT_MAX;
     constexpr int kSiteOffset = SWIGLU ? 0 : 4;
+    chain_release();  // the next kernel of the forward call may be scheduled; it waits for this grid to finish
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *base_ptr = smem_raw + (base - smem_u32(smem_raw));
@@ -124,6 +125,7 @@ grouped_gemm_tc_fp8w_kernel(const __grid_constant__ TensorMaps maps, const Kerne
     __syncthreads();
     tcgen05_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    chain_wait();  // everything above overlapped the previous kernel; its results are read from here on
     const int total_tiles = p.tile_prefix[p.E] * p.n_feature_tiles;
 
     if (warp == 0) {
@@ -323,8 +325,7 @@ int launch_fp8_instance(const TensorMaps &maps, const KernelParams &p, int grid,
     auto kernel = grouped_gemm_tc_fp8w_kernel<NT_MAX, STAGES, CONV, SWIGLU>;
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) != cudaSuccess)
         return MOE_ERR_CUDA;
-    kernel<<<grid, kFp8Threads, L::kDynamicBytes, stream>>>(maps, p);
-    return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+    return launch_chained(kernel, grid, kFp8Threads, L::kDynamicBytes, stream, maps, p) == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
 
 template <bool SWIGLU>

@@ -75,6 +75,7 @@ grouped_gemm_tc_mx_kernel(const __grid_constant__ TensorMaps maps, const MxParam
     static_assert(2 * NT_MAX + 32 <= kTmemColsMx, "accumulators and scale columns exceed tensor memory");
     constexpr int kSiteOffset = SWIGLU ? 0 : 4;
     constexpr uint32_t kSfACol = 2 * NT_MAX, kSfBCol = 2 * NT_MAX + 16;
+    chain_release();  // the next kernel of the forward call may be scheduled; it waits for this grid to finish
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *base_ptr = smem_raw + (base - smem_u32(smem_raw));
@@ -107,6 +108,7 @@ grouped_gemm_tc_mx_kernel(const __grid_constant__ TensorMaps maps, const MxParam
     __syncthreads();
     tcgen05_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    chain_wait();  // everything above overlapped the previous kernel; its results are read from here on
     const int total_tiles = p.tile_prefix[p.E] * p.n_feature_tiles;
 
     if (warp == 0) {
@@ -243,8 +245,7 @@ int launch_instance(const TensorMaps &maps, const MxParams &p, int grid, cudaStr
     auto kernel = grouped_gemm_tc_mx_kernel<NT_MAX, STAGES, SWIGLU>;
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) != cudaSuccess)
         return MOE_ERR_CUDA;
-    kernel<<<grid, kThreads, L::kDynamicBytes, stream>>>(maps, p);
-    return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+    return launch_chained(kernel, grid, kThreads, L::kDynamicBytes, stream, maps, p) == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
 
 template <bool SWIGLU>

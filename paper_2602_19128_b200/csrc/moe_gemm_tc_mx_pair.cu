@@ -73,6 +73,7 @@ grouped_gemm_tc_mx_pair_kernel(const __grid_constant__ MxPairMaps maps, const Mx
     constexpr int kSiteOffset = SWIGLU ? 0 : 4;
     constexpr uint32_t kSfACol = 2 * NT_MAX, kSfBCol = 2 * NT_MAX + 16;
     constexpr int kFeatPerCta = SWIGLU ? kTileM / 2 : kTileM;  // h features resp. output rows per CTA of a pair tile
+    chain_release();  // the next kernel of the forward call may be scheduled; it waits for this grid to finish
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *base_ptr = smem_raw + (base - smem_u32(smem_raw));
@@ -108,6 +109,7 @@ grouped_gemm_tc_mx_pair_kernel(const __grid_constant__ MxPairMaps maps, const Mx
     cluster_sync_all();  // the peer's barriers exist before anything can signal them
     tcgen05_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    chain_wait();  // everything above overlapped the previous kernel; its results are read from here on
     const int total_tiles = p.tile_prefix[p.E] * p.n_feature_tiles;
     const int n_pairs = gridDim.x >> 1, pair = blockIdx.x >> 1;
     const int w_tiles_per_expert = p.n_out / kFeatPerCta;  // weight scale atoms are stored per 128-row CTA tile
@@ -273,8 +275,7 @@ int launch_pair_instance(const MxPairMaps &maps, const MxParams &p, int grid, cu
     auto kernel = grouped_gemm_tc_mx_pair_kernel<NT_MAX, STAGES, SWIGLU>;
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) != cudaSuccess)
         return MOE_ERR_CUDA;
-    kernel<<<grid, kPairThreads, L::kDynamicBytes, stream>>>(maps, p);
-    return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+    return launch_chained(kernel, grid, kPairThreads, L::kDynamicBytes, stream, maps, p) == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
 
 }  // namespace

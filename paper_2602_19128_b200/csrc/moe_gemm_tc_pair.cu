@@ -98,6 +98,7 @@ grouped_gemm_tc_pair_kernel(const __grid_constant__ TensorMaps maps, const Kerne
     constexpr int kFeatPerCta = SWIGLU ? kTileM / 2 : kTileM;
     constexpr int kFeatPerSlab = 2 * kFeatPerCta;
     constexpr int kFeatPerTile = SLABS * kFeatPerSlab;
+    chain_release();  // the next kernel of the forward call may be scheduled; it waits for this grid to finish
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *base_ptr = smem_raw + (base - smem_u32(smem_raw));
@@ -133,6 +134,7 @@ grouped_gemm_tc_pair_kernel(const __grid_constant__ TensorMaps maps, const Kerne
     cluster_sync_all();  // the peer's barriers exist before anything can signal them
     tcgen05_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    chain_wait();  // everything above overlapped the previous kernel; its results are read from here on
     const int total_tiles = p.tile_prefix[p.E] * p.n_feature_tiles;
     const int n_pairs = gridDim.x >> 1, pair = blockIdx.x >> 1;
 
@@ -285,8 +287,7 @@ int launch_pair_instance(const TensorMaps &maps, const KernelParams &p, int grid
     auto kernel = grouped_gemm_tc_pair_kernel<NT_MAX, STAGES, SLABS, SWIGLU>;
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) != cudaSuccess)
         return MOE_ERR_CUDA;
-    kernel<<<grid, kPairThreads, L::kDynamicBytes, stream>>>(maps, p);
-    return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+    return launch_chained(kernel, grid, kPairThreads, L::kDynamicBytes, stream, maps, p) == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
 
 int features_per_pair_tile(const GroupedGemmArgs &a, int slabs) { return slabs * (a.swiglu ? kTileM : 2 * kTileM); }

@@ -23,6 +23,34 @@ enum : int { kSiteProducerEmpty = 1, kSiteMmaFull = 2, kSiteMmaTmemEmpty = 3, kS
 
 static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// ---- chained launches (programmatic dependent launch) ----------------------------------------------------
+// The kernels of one forward call form a chain in which each reads what its predecessors wrote.  Every kernel
+// is launched with programmatic stream serialisation allowed, announces at its very start that its dependents
+// may be scheduled (chain_release), and waits for the completion of everything before it in the stream
+// (chain_wait) before it touches memory a predecessor writes.  A kernel's launch latency and prologue (barrier
+// set-up, tensor-memory allocation) then overlap the tail of the kernel before it.  Because EVERY block of
+// every kernel waits, completion is transitive: when a kernel's predecessor is complete, so is everything
+// earlier in the chain.
+#ifdef __CUDACC__
+__device__ __forceinline__ void chain_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void chain_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args &&...args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
+
 // Scratch of the router / sort-scatter, all int32, carved out of the caller's workspace.
 struct RouteScratch {
     int *chunk_counts;  // [n_chunks, E] per-chunk expert histogram, then rows of earlier chunks per expert

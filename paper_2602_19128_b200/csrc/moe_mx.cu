@@ -58,6 +58,8 @@ __global__ void __launch_bounds__(256)
 mx_quantize_rows_kernel(const uint4 *__restrict__ x, const int *__restrict__ sorted_to_flat,
                         const int *__restrict__ expert_offsets, int E, int n_rows_plain, int k, int vec_per_row,
                         int warps_per_row, uint2 *__restrict__ codes, uint8_t *__restrict__ scales, int n_atoms, int tile) {
+    chain_release();
+    chain_wait();
     const int lane = threadIdx.x & 31;
     const long long w = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
     const int r = (int)(w / warps_per_row), first_seg = (int)(w % warps_per_row);
@@ -145,10 +147,9 @@ cudaError_t launch_mx_gather_quantize(const __nv_bfloat16 *x, const int *sorted_
                                       cudaStream_t stream) {
     const int segs = mx_quantize_warps_per_row(A, (H / 8 + 31) / 32);
     const long long warps = (long long)A * segs;
-    mx_quantize_rows_kernel<true><<<(unsigned)((warps + 7) / 8), 256, 0, stream>>>(
-        reinterpret_cast<const uint4 *>(x), sorted_to_flat, expert_offsets, E, 0, k, H / 8, segs,
-        reinterpret_cast<uint2 *>(xq), x_sf, n_atoms, tile);
-    return cudaGetLastError();
+    return launch_chained(mx_quantize_rows_kernel<true>, (unsigned)((warps + 7) / 8), 256, 0, stream,
+                          reinterpret_cast<const uint4 *>(x), sorted_to_flat, expert_offsets, E, 0, k, H / 8, segs,
+                          reinterpret_cast<uint2 *>(xq), x_sf, n_atoms, tile);
 }
 
 cudaError_t launch_mx_quantize_rows(const __nv_bfloat16 *x, int R, int K, uint8_t *codes, uint8_t *scales,

@@ -246,6 +246,8 @@ route_topk_kernel(const float *__restrict__ logits, int T, int E, int k, int loc
                   const RouterParams rp, int *__restrict__ topk_ids, float *__restrict__ topk_w,
                   int *__restrict__ chunk_counts) {
     __shared__ int hist[kMaxExperts];  // indexed by local expert (expert id - local_offset)
+    chain_release();
+    chain_wait();
     route_block_tokens(logits, T, E, k, local_offset, n_local, rp, topk_ids, topk_w, hist);
     for (int e = threadIdx.x; e < n_local; e += kRouteThreads) chunk_counts[(size_t)blockIdx.x * n_local + e] = hist[e];
 }
@@ -366,6 +368,8 @@ route_scan_kernel(int *chunk_counts, int n_chunks, int E, int nt_max, int row_qu
                   int *tile_prefix, int *tile_order, int *tile_rows) {
     __shared__ int warp_sums[8];
     __shared__ int counts[kMaxExperts], tiles_at[kMaxExperts], part_sums[kScanThreads];
+    chain_release();
+    chain_wait();
     scan_phase(chunk_counts, n_chunks, E, nt_max, row_quantum, expert_offsets, tile_prefix, tile_order, tile_rows, warp_sums,
                counts, tiles_at, part_sums);
 }
@@ -422,6 +426,8 @@ __global__ void __launch_bounds__(32)
 route_scatter_kernel(const int *topk_ids, const int *chunk_starts, const int *expert_offsets, int A, int n_local,
                      int local_offset, int k, int *sorted_to_flat, int *flat_to_sorted) {
     __shared__ int next[kMaxExperts];
+    chain_release();
+    chain_wait();
     scatter_chunk(blockIdx.x, topk_ids, chunk_starts, expert_offsets, A, n_local, local_offset, k, sorted_to_flat,
                   flat_to_sorted, next, threadIdx.x);
 }
@@ -441,6 +447,8 @@ route_fused_kernel(const float *__restrict__ logits, int T, int E, int k, int lo
     __shared__ int next[kFusedMaxChunks][kMaxExperts];
     __shared__ int is_last;
     const int tid = threadIdx.x;
+    chain_release();
+    chain_wait();
     route_block_tokens(logits, T, E, k, local_offset, n_local, rp, topk_ids, topk_w, hist);
     for (int e = tid; e < n_local; e += kFusedThreads) chunk_counts[(size_t)blockIdx.x * n_local + e] = hist[e];
     __threadfence();  // this block's ids, weights and histogram are visible before it is counted as done
@@ -462,6 +470,8 @@ route_fused_kernel(const float *__restrict__ logits, int T, int E, int k, int lo
 __global__ void __launch_bounds__(256)
 gather_rows_kernel(const uint4 *__restrict__ x, const int *__restrict__ sorted_to_flat,
                    const int *__restrict__ n_rows, int k, int vec_per_row, uint4 *__restrict__ x_perm) {
+    chain_release();
+    chain_wait();
     const int lane = threadIdx.x & 31;
     const int r = blockIdx.x * 8 + (threadIdx.x >> 5);
     if (r >= *n_rows) return;  // rows actually scheduled: all A assignments, or fewer with a local-expert subset
@@ -481,6 +491,8 @@ combine_kernel(const uint4 *__restrict__ y, const float *__restrict__ topk_w, co
                int k, int vec_per_row, uint4 *__restrict__ out) {
     __shared__ int rows[kMaxTopK];
     __shared__ float weights[kMaxTopK];
+    chain_release();
+    chain_wait();
     const int t = blockIdx.x;
     if (threadIdx.x < k) {
         rows[threadIdx.x] = flat_to_sorted[(size_t)t * k + threadIdx.x];
@@ -528,36 +540,31 @@ cudaError_t launch_route(const float *logits, int T, int E, int k, LocalExperts 
     if (err != cudaSuccess) return err;
     const int A = T * k;
     if (scratch.n_chunks <= kFusedMaxChunks) {
-        route_fused_kernel<<<scratch.n_chunks, kFusedThreads, 0, stream>>>(
-            logits, T, E, k, local.offset, local.count, nt_max, row_quantum, router, topk_ids, topk_w, scratch.chunk_counts,
-            expert_offsets,
-            scratch.tile_prefix, scratch.tile_order, scratch.tile_rows, sorted_to_flat, flat_to_sorted,
-            status + kDoneCounterInt);
-        return cudaGetLastError();
+        return launch_chained(route_fused_kernel, scratch.n_chunks, kFusedThreads, 0, stream, logits, T, E, k, local.offset,
+                              local.count, nt_max, row_quantum, router, topk_ids, topk_w, scratch.chunk_counts, expert_offsets,
+                              scratch.tile_prefix, scratch.tile_order, scratch.tile_rows, sorted_to_flat, flat_to_sorted,
+                              status + kDoneCounterInt);
     }
-    route_topk_kernel<<<scratch.n_chunks, kRouteThreads, 0, stream>>>(logits, T, E, k, local.offset, local.count, router,
-                                                                       topk_ids, topk_w, scratch.chunk_counts);
-    route_scan_kernel<<<1, kScanThreads, 0, stream>>>(scratch.chunk_counts, scratch.n_chunks, local.count, nt_max, row_quantum,
-                                             expert_offsets,
-                                             scratch.tile_prefix, scratch.tile_order, scratch.tile_rows);
-    route_scatter_kernel<<<scratch.n_chunks, 32, 0, stream>>>(topk_ids, scratch.chunk_counts, expert_offsets, A,
-                                                              local.count, local.offset, k, sorted_to_flat,
-                                                              flat_to_sorted);
-    return cudaGetLastError();
+    err = launch_chained(route_topk_kernel, scratch.n_chunks, kRouteThreads, 0, stream, logits, T, E, k, local.offset,
+                         local.count, router, topk_ids, topk_w, scratch.chunk_counts);
+    if (err != cudaSuccess) return err;
+    err = launch_chained(route_scan_kernel, 1, kScanThreads, 0, stream, scratch.chunk_counts, scratch.n_chunks, local.count,
+                         nt_max, row_quantum, expert_offsets, scratch.tile_prefix, scratch.tile_order, scratch.tile_rows);
+    if (err != cudaSuccess) return err;
+    return launch_chained(route_scatter_kernel, scratch.n_chunks, 32, 0, stream, topk_ids, scratch.chunk_counts,
+                          expert_offsets, A, local.count, local.offset, k, sorted_to_flat, flat_to_sorted);
 }
 
 cudaError_t launch_gather_rows(const __nv_bfloat16 *x, const int *sorted_to_flat, const int *n_rows, int A, int k,
                                int H, __nv_bfloat16 *x_perm, cudaStream_t stream) {
-    gather_rows_kernel<<<(A + 7) / 8, 256, 0, stream>>>(reinterpret_cast<const uint4 *>(x), sorted_to_flat, n_rows, k,
-                                                        H / 8, reinterpret_cast<uint4 *>(x_perm));
-    return cudaGetLastError();
+    return launch_chained(gather_rows_kernel, (A + 7) / 8, 256, 0, stream, reinterpret_cast<const uint4 *>(x), sorted_to_flat,
+                          n_rows, k, H / 8, reinterpret_cast<uint4 *>(x_perm));
 }
 
 cudaError_t launch_combine(const __nv_bfloat16 *y, const float *topk_w, const int *flat_to_sorted, int T, int k,
                            int H, __nv_bfloat16 *out, cudaStream_t stream) {
-    combine_kernel<<<T, 256, 0, stream>>>(reinterpret_cast<const uint4 *>(y), topk_w, flat_to_sorted, k, H / 8,
-                                          reinterpret_cast<uint4 *>(out));
-    return cudaGetLastError();
+    return launch_chained(combine_kernel, T, 256, 0, stream, reinterpret_cast<const uint4 *>(y), topk_w, flat_to_sorted, k,
+                          H / 8, reinterpret_cast<uint4 *>(out));
 }
 
 }  // namespace moe
