@@ -120,7 +120,22 @@ CASES = [
 ]
 
 
-@pytest.mark.parametrize("T,H,I,E,k,skew", CASES)
+def draw_shapes(n, seed):
+    """Seeded random shapes inside the MX envelope, small enough for the oracle."""
+    rng = np.random.default_rng(seed)
+    shapes = []
+    while len(shapes) < n:
+        E = int(rng.choice([1, 2, 3, 6, 8, 16, 32, 128]))
+        k = int(rng.integers(1, min(E, 6) + 1))
+        H, I = 128 * int(rng.integers(1, 5)), 128 * int(rng.integers(1, 4))
+        T = int(rng.choice([1, 5, 32, 70, 150, 400, 1030]))
+        if T * k * H * I > 120_000_000:
+            continue
+        shapes.append((T, H, I, E, k, bool(rng.integers(0, 2))))
+    return shapes
+
+
+@pytest.mark.parametrize("T,H,I,E,k,skew", CASES + draw_shapes(16, seed=77))
 def test_mxfp8_forward_matches_oracle(T, H, I, E, k, skew):
     inp = make_mxfp8_inputs(dict(T=T, H=H, I=I, E=E, top_k=k, skew=skew), seed=0, device="cuda")
     out, views = run_mx(inp)
