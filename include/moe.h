@@ -34,6 +34,14 @@
  *     with moe_last_status().
  *   - Results are deterministic: no floating-point atomics, no split accumulation; two calls on
  *     the same inputs give bit-identical outputs.
+ *   - The kernels of one call are launched with programmatic stream serialisation (each waits for its
+ *     predecessor before reading its results), so a call can be captured into a CUDA graph and replayed.
+ *
+ * Variants of the layer, each with the same conventions: moe_forward_local (only the experts resident on
+ * this device), moe_route_grouped / moe_forward_grouped (sigmoid scores, selection bias, group-limited
+ * top-k, scaled weights), moe_forward_fp8w (FP8 weights with a scale per 128 x 128 block, dequantised on the
+ * way to 16-bit MMAs), moe_forward_mxfp8 (weights and activations in MX FP8, multiplied by the block-scaled
+ * MMA), the *_host forms for activations in host memory, moe_forward_staged for per-stage timing.
  */
 #ifndef MOE_B200_H_
 #define MOE_B200_H_

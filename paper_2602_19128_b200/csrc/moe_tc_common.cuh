@@ -1,5 +1,6 @@
-// Device-side PTX wrappers, descriptors and the tile schedule decoder shared by the two tcgen05
-// grouped-GEMM kernels (one CTA per tile, and CTA pairs), plus the host-side tensor-map encoders.
+// Device-side PTX wrappers, descriptors and the tile schedule decoder shared by the tcgen05 grouped-GEMM
+// kernels (bf16, FP8-dequantising and MX FP8; one CTA per tile and CTA pairs), plus the host-side tensor-map
+// encoders.
 #pragma once
 
 #include "moe_internal.cuh"
