@@ -296,6 +296,10 @@ __device__ __forceinline__ void scan_phase(int *chunk_counts, int n_chunks, int 
         const int pe = threadIdx.x % kMaxExperts, part = threadIdx.x / kMaxExperts, n_parts = blockDim.x / kMaxExperts;
         const int per = (n_chunks + n_parts - 1) / n_parts;
         const int b_begin = min(n_chunks, part * per), b_end = min(n_chunks, b_begin + per);
+        const bool one_batch = b_end - b_begin <= kBatch;  // then the counts stay in registers between the passes
+        int first[kBatch];
+#pragma unroll
+        for (int i = 0; i < kBatch; ++i) first[i] = 0;
         int sum = 0;
         if (pe < E) {
             for (int b0 = b_begin; b0 < b_end; b0 += kBatch) {
@@ -304,6 +308,10 @@ __device__ __forceinline__ void scan_phase(int *chunk_counts, int n_chunks, int 
                 for (int i = 0; i < kBatch; ++i) c[i] = b0 + i < b_end ? __ldcg(&chunk_counts[(size_t)(b0 + i) * E + pe]) : 0;
 #pragma unroll
                 for (int i = 0; i < kBatch; ++i) sum += c[i];
+                if (b0 == b_begin) {
+#pragma unroll
+                    for (int i = 0; i < kBatch; ++i) first[i] = c[i];
+                }
             }
         }
         part_sums[part * kMaxExperts + pe] = sum;
@@ -318,7 +326,8 @@ __device__ __forceinline__ void scan_phase(int *chunk_counts, int n_chunks, int 
             for (int b0 = b_begin; b0 < b_end; b0 += kBatch) {
                 int c[kBatch];
 #pragma unroll
-                for (int i = 0; i < kBatch; ++i) c[i] = b0 + i < b_end ? __ldcg(&chunk_counts[(size_t)(b0 + i) * E + pe]) : 0;
+                for (int i = 0; i < kBatch; ++i)
+                    c[i] = one_batch ? first[i] : (b0 + i < b_end ? __ldcg(&chunk_counts[(size_t)(b0 + i) * E + pe]) : 0);
 #pragma unroll
                 for (int i = 0; i < kBatch; ++i) {
                     if (b0 + i < b_end) chunk_counts[(size_t)(b0 + i) * E + pe] = run;
@@ -343,12 +352,25 @@ __device__ __forceinline__ void scan_phase(int *chunk_counts, int n_chunks, int 
     const int row_start = block_exclusive_scan_256(count, warp_sums, &total_rows);  // (syncs: counts[] is visible)
     // Schedule order: experts with more rows first (ties to the lower index), so that tiles of similar
     // cost are adjacent and the GEMMs' static tile assignment stays balanced; the small tiles come last.
-    if (e < E) {
-        int pos = 0;
-#pragma unroll 8
-        for (int o = 0; o < E; ++o) pos += (counts[o] > count || (counts[o] == count && o < e)) ? 1 : 0;
-        tiles_at[pos] = n_tiles;
-        tile_order[pos] = e;
+    // (all-pairs ranking, E^2 comparisons: every part of the block takes a share of the opponents)
+    {
+        const int pe = threadIdx.x % kMaxExperts, part = threadIdx.x / kMaxExperts, n_parts = blockDim.x / kMaxExperts;
+        part_sums[threadIdx.x] = 0;
+        if (pe < E) {
+            const int mine = counts[pe];
+            const int per = (E + n_parts - 1) / n_parts, o_end = min(E, (part + 1) * per);
+            int before = 0;
+#pragma unroll 4
+            for (int o = part * per; o < o_end; ++o) before += (counts[o] > mine || (counts[o] == mine && o < pe)) ? 1 : 0;
+            part_sums[threadIdx.x] = before;
+        }
+        __syncthreads();
+        if (e < E) {
+            int pos = 0;
+            for (int p = 0; p < n_parts; ++p) pos += part_sums[p * kMaxExperts + e];
+            tiles_at[pos] = n_tiles;
+            tile_order[pos] = e;
+        }
     }
     __syncthreads();
     const int tile_start = block_exclusive_scan_256(lane_of_scan ? tiles_at[e] : 0, warp_sums, &total_tiles);
