@@ -276,7 +276,7 @@ typedef struct {
     size_t y;     /* bf16 [A,H] */
     size_t staging; /* used only by moe_forward_mxfp8_host: device copies of x, logits, out */
     size_t sf_atoms;  /* a count, not an offset: atoms per K-slot in x_sf / h_sf */
-    size_t tile_rows; /* a count: rows per token tile of this problem (32, 64, 128 or 240) */
+    size_t tile_rows; /* a count: rows per token tile of this problem (32, 64, 128, 160 or 240) */
 } moe_mxfp8_workspace_layout_t;
 
 /* Host-only, pure.  Workspace bytes of moe_forward_mxfp8; 0 outside the envelope (moe_forward's, plus I % 128 == 0). */

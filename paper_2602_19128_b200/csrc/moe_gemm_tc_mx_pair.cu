@@ -281,7 +281,7 @@ int launch_pair_instance(const MxPairMaps &maps, const MxParams &p, int grid, cu
 }  // namespace
 
 bool grouped_gemm_tc_mx_pair_applies(const MxGemmArgs &a) {
-    if (!(a.nt_max == 128 || a.nt_max == 240) || a.K % kMxSlotK != 0 || a.A <= 0) return false;
+    if (!(a.nt_max == 128 || a.nt_max == 160 || a.nt_max == 240) || a.K % kMxSlotK != 0 || a.A <= 0) return false;
     return a.n_out % (a.swiglu ? kTileM : 2 * kTileM) == 0;
 }
 
@@ -326,6 +326,9 @@ int launch_grouped_gemm_tc_mx_pair(const MxGemmArgs &a, cudaStream_t stream) {
     if (a.nt_max == 240)
         return a.swiglu ? launch_pair_instance<240, 6, true>(maps, p, grid, stream)
                         : launch_pair_instance<240, 6, false>(maps, p, grid, stream);
+    if (a.nt_max == 160)  // a smaller token slot buys two more ring slots: more weight bytes in flight per SM
+        return a.swiglu ? launch_pair_instance<160, 8, true>(maps, p, grid, stream)
+                        : launch_pair_instance<160, 8, false>(maps, p, grid, stream);
     return a.swiglu ? launch_pair_instance<128, 8, true>(maps, p, grid, stream)
                     : launch_pair_instance<128, 8, false>(maps, p, grid, stream);
 }

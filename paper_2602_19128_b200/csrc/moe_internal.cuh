@@ -152,7 +152,7 @@ int launch_grouped_gemm_tc_fp8w(const GroupedGemmArgs &args, cudaStream_t stream
 // bulk copy.
 //   weights     : [E][feature tile][K/128][512]; a gate/up tile's rows are in the tile's interleaved order
 //   activations : [K/128][n_atoms][512], whole atoms per token tile.  The MX schedule cuts every expert's
-//                 rows into tiles of exactly `tile` rows (the token-tile bound: 32, 64, 128 or 240; the last
+//                 rows into tiles of exactly `tile` rows (the token-tile bound: 32, 64, 128, 160 or 240; the last
 //                 may be partial).  Token tile j of expert e is tile number  offsets[e] / tile + e + j  and
 //                 owns ceil(tile / 128) consecutive atoms; its row r sits in atom r / 128 of those, at atom
 //                 row r % 128.  Every tile thus starts a fresh atom, and the MMA reads its token scales from
@@ -182,7 +182,7 @@ struct MxGemmArgs {
 // One-CTA tcgen05 kernel with kind::mxf8f6f4.block_scale.  The schedule must have been built with the row
 // quantum equal to nt_max (every tile nt_max rows, the last partial) and nt_max <= 128.  Needs K % 128 == 0.
 int launch_grouped_gemm_tc_mx(const MxGemmArgs &args, cudaStream_t stream);
-// The same GEMM on CTA pairs (cta_group::2, 256 x N tiles): nt_max 128 or 240, and n_out a multiple of the
+// The same GEMM on CTA pairs (cta_group::2, 256 x N tiles): nt_max 128, 160 or 240, and n_out a multiple of the
 // pair tile (128 features of h, 256 output rows of the down projection).
 bool grouped_gemm_tc_mx_pair_applies(const MxGemmArgs &args);
 int launch_grouped_gemm_tc_mx_pair(const MxGemmArgs &args, cudaStream_t stream);
