@@ -63,3 +63,30 @@ def test_mxfp8_layer_replays_from_a_graph():
     moe.moe_forward_mxfp8(b["x"], b["router_logits"], a["w13_q"], sf13, a["w2_q"], sf2, k, ref, ws2)
     torch.cuda.synchronize()
     assert torch.equal(out.view(torch.int16), ref.view(torch.int16))
+
+
+def test_two_streams_with_their_own_workspaces_do_not_interfere():
+    """The library keeps no state between calls except what lives in the caller's workspace, so calls on different
+    streams with different workspaces may run concurrently."""
+    cfg = dict(T=700, H=256, I=256, E=16, top_k=4, skew=True)
+    a, b = make_inputs(cfg, seed=11, device="cuda"), make_inputs(cfg, seed=12, device="cuda")
+    T, H, I, E, k = cfg["T"], cfg["H"], cfg["I"], cfg["E"], cfg["top_k"]
+    refs = []
+    for inp in (a, b):
+        ws = moe.alloc_workspace(moe.moe_workspace_bytes(T, H, I, E, k), "cuda")
+        ref = torch.empty((T, H), dtype=torch.bfloat16, device="cuda")
+        moe.moe_forward(inp["x"], inp["router_logits"], inp["w13"], inp["w2"], k, ref, ws)
+        torch.cuda.synchronize()
+        refs.append(ref)
+    lanes = []
+    for inp in (a, b):
+        lanes.append((torch.cuda.Stream(), inp, moe.alloc_workspace(moe.moe_workspace_bytes(T, H, I, E, k), "cuda"),
+                      torch.empty((T, H), dtype=torch.bfloat16, device="cuda")))
+    torch.cuda.synchronize()
+    for _ in range(20):  # interleave the two lanes' launches
+        for st, inp, ws, out in lanes:
+            moe.moe_forward(inp["x"], inp["router_logits"], inp["w13"], inp["w2"], k, out, ws, stream=st)
+    torch.cuda.synchronize()
+    for (st, inp, ws, out), ref in zip(lanes, refs):
+        assert moe.moe_last_status(ws, stream=st) == moe.MOE_OK
+        assert torch.equal(out.view(torch.int16), ref.view(torch.int16))
