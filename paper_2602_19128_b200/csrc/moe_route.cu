@@ -501,11 +501,13 @@ gather_rows_kernel(const uint4 *__restrict__ x, const int *__restrict__ sorted_t
     const uint4 *src = x + (size_t)t * vec_per_row;
     uint4 *dst = x_perm + (size_t)r * vec_per_row;
     int i = lane;
+    // streaming stores: the copy is read by the GEMM from memory anyway, and keeping it out of L2 leaves the token
+    // rows (each read top_k times here) resident
     for (; i + 96 < vec_per_row; i += 128) {  // four independent 16-byte loads in flight per lane
         const uint4 a = src[i], b = src[i + 32], c = src[i + 64], d = src[i + 96];
-        dst[i] = a; dst[i + 32] = b; dst[i + 64] = c; dst[i + 96] = d;
+        __stcs(dst + i, a); __stcs(dst + i + 32, b); __stcs(dst + i + 64, c); __stcs(dst + i + 96, d);
     }
-    for (; i < vec_per_row; i += 32) dst[i] = src[i];
+    for (; i < vec_per_row; i += 32) __stcs(dst + i, src[i]);
 }
 
 __global__ void __launch_bounds__(256)
