@@ -97,7 +97,7 @@ mx_quantize_rows_kernel(const uint4 *__restrict__ x, const int *__restrict__ sor
             uint32_t sb;
             const uint2 q = quantize_8_of_32(in[u], sb);  // every lane takes part in the shuffles
             if (v < vec_per_row) {
-                codes[(size_t)r * vec_per_row + v] = q;
+                __stcs(codes + (size_t)r * vec_per_row + v, q);  // streaming: read next from memory by the GEMM, keep x in L2
                 if ((lane & 3) == 0) {
                     const int block = v >> 2;  // 32-element block along the row; 4 blocks per 128-element slot
                     if (kGather)
