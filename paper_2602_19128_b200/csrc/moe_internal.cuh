@@ -191,6 +191,10 @@ int launch_grouped_gemm_tc_mx_pair(const MxGemmArgs &args, cudaStream_t stream);
 cudaError_t launch_mx_gather_quantize(const __nv_bfloat16 *x, const int *sorted_to_flat, const int *expert_offsets, int E,
                                       int A, int k, int H, uint8_t *xq, uint8_t *x_sf, int n_atoms, int tile,
                                       cudaStream_t stream);
+// The same result from rows quantised once per token (tok_codes [T,H], tok_scales [T,H/32]): a copy per sorted row.
+cudaError_t launch_mx_gather_codes(const uint8_t *tok_codes, const uint8_t *tok_scales, const int *sorted_to_flat,
+                                   const int *expert_offsets, int E, int A, int k, int H, uint8_t *xq, uint8_t *x_sf,
+                                   int n_atoms, int tile, cudaStream_t stream);
 // codes[r,:], scales[r, K/32] (plain row-major) <- MX quantisation of x[r,:].
 cudaError_t launch_mx_quantize_rows(const __nv_bfloat16 *x, int R, int K, uint8_t *codes, uint8_t *scales,
                                     cudaStream_t stream);

@@ -270,3 +270,36 @@ def test_mxfp8_with_grouped_router_and_local_experts():
         ref[sel] += wsel[:, None] * one
     err = np.abs(bf16_to_f64(out) - ref)
     assert np.all(err <= 2e-2 * (2.5 + np.abs(ref)))
+
+
+def test_mxfp8_large_batch_quantises_per_token_then_copies():
+    """From T*top_k*H = 64 Mi on, x is quantised once per token and the codes are copied per assignment: the
+    gathered codes and every scale byte must equal the oracle's, and sampled outputs its layer."""
+    cfg = dict(T=2048, H=4096, I=128, E=16, top_k=8, skew=False)
+    inp = make_mxfp8_inputs(cfg, seed=21, device="cuda")
+    out, views = run_mx(inp)
+    T, H, I, E, k = (cfg[n] for n in ("T", "H", "I", "E", "top_k"))
+    o = moe_oracle.get("f32")
+    logits = inp["router_logits"].cpu().numpy()
+    ids, w = o.route(logits, k)
+    off, s2f, f2s = o.permute(ids, E)
+    assert_routing_exact(views, ids, w, off, s2f, f2s)
+    xc, xs = o.mx_quantize(inp["x"].float().cpu().numpy())
+    tok = s2f // k
+    assert np.array_equal(views["x_q"].cpu().numpy(), xc[tok])
+    # scale bytes: vectorised form of unpack_act_scales
+    tile = views["tile_rows"]
+    apt = (tile + 127) // 128
+    e_of_row = np.searchsorted(off, np.arange(off[E]), side="right") - 1
+    i = np.arange(off[E]) - off[e_of_row]
+    r = i % tile
+    atom = (off[e_of_row] // tile + e_of_row + i // tile) * apt + r // 128
+    base = (r % 128 % 32) * 16 + (r % 128 // 32) * 4
+    atoms = views["x_sf"].cpu().numpy()
+    got = np.stack([atoms[b // 4, atom, base + b % 4] for b in range(H // 32)], axis=1)
+    assert np.array_equal(got, xs[tok])
+    tokens = np.array([0, 1, 777, T - 1], dtype=np.int32)
+    need = sorted({int(e) for t in tokens for e in ids[t]})
+    experts = {e: tuple(inp[n][e].cpu().numpy() for n in ("w13_q", "w13_s", "w2_q", "w2_s")) for e in need}
+    ref = o.forward_mxfp8_sampled(bf16_bits(inp["x"]), logits, experts, I, k, tokens)
+    assert_close_out(bf16_to_f64(out[torch.from_numpy(tokens).long().cuda()]), ref, "two-step sampled out")
