@@ -527,16 +527,26 @@ combine_kernel(const uint4 *__restrict__ y, const float *__restrict__ topk_w, co
         float acc[8];
 #pragma unroll
         for (int c = 0; c < 8; ++c) acc[c] = 0.f;
-        for (int j = 0; j < k; ++j) {  // ascending rank: the summation order is fixed
-            if (rows[j] < 0) continue;   // expert not resident on this device: contributes nothing
-            const uint4 v = y[(size_t)rows[j] * vec_per_row + i];
-            const float wj = weights[j];
-            const __nv_bfloat162 *h2 = reinterpret_cast<const __nv_bfloat162 *>(&v);
+        // ascending rank: the summation order is fixed.  Four rows are fetched before the first is used (the
+        // loop is a chain of memory round trips otherwise); the additions still happen one rank after the other.
+        for (int j0 = 0; j0 < k; j0 += 4) {
+            uint4 v[4];
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                const float2 f = __bfloat1622float2(h2[c]);
-                acc[2 * c] = fmaf(wj, f.x, acc[2 * c]);
-                acc[2 * c + 1] = fmaf(wj, f.y, acc[2 * c + 1]);
+            for (int u = 0; u < 4; ++u) {
+                const bool live = j0 + u < k && rows[j0 + u] >= 0;  // rank exists and its expert is resident here
+                v[u] = live ? __ldcs(&y[(size_t)rows[j0 + u] * vec_per_row + i]) : make_uint4(0, 0, 0, 0);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (j0 + u >= k || rows[j0 + u] < 0) continue;  // contributes nothing (not even a signed zero)
+                const float wj = weights[j0 + u];
+                const __nv_bfloat162 *h2 = reinterpret_cast<const __nv_bfloat162 *>(&v[u]);
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const float2 f = __bfloat1622float2(h2[c]);
+                    acc[2 * c] = fmaf(wj, f.x, acc[2 * c]);
+                    acc[2 * c + 1] = fmaf(wj, f.y, acc[2 * c + 1]);
+                }
             }
         }
         uint4 o;
