@@ -202,7 +202,6 @@ cudaError_t launch_mx_quantize_rows(const __nv_bfloat16 *x, int R, int K, uint8_
 // 64 features interleaved as the gate/up GEMM reads them; else tiles of 128 consecutive rows.
 cudaError_t launch_mx_pack_scales(const uint8_t *plain, int E, int rows, int K, bool gate_up, uint8_t *packed,
                                   cudaStream_t stream);
-static inline size_t mx_weight_sf_bytes(int E, int rows, int K) { return (size_t)E * rows * (K / 32); }
 
 // Same contract on plain CUDA cores (validation only).
 cudaError_t launch_grouped_gemm_validation(const GroupedGemmArgs &args, cudaStream_t stream);
