@@ -50,3 +50,47 @@ def test_status_strings_and_launch_count():
     assert moe.moe_status_string(-99) == "unknown status"
     assert moe.moe_forward_launch_count(0) == 0 and moe.moe_forward_launch_count(16) == 5
     assert moe.moe_forward_launch_count(1024) == 5 and moe.moe_forward_launch_count(1025) == 7
+
+
+def test_mx_layout_and_launch_count():
+    for cfg in [(16, 256, 512, 8, 2), (512, 4096, 14336, 8, 2), (128, 7168, 2048, 256, 8), (8192, 7168, 2048, 256, 8)]:
+        n = moe.moe_mxfp8_workspace_bytes(*cfg)
+        L = moe.moe_mxfp8_workspace_layout(*cfg)
+        T, H, I, E, k = cfg
+        A = T * k
+        assert n == L.total_bytes > 0
+        offs = [L.status, L.topk_ids, L.topk_weights, L.expert_offsets, L.sorted_to_flat, L.flat_to_sorted,
+                L.route_scratch, L.x_q, L.x_sf, L.h_q, L.h_sf, L.y, L.x_q_tok, L.x_sf_tok, L.staging]
+        assert offs == sorted(offs) and all(o % 256 == 0 for o in offs) and offs[-1] < n
+        assert L.tile_rows in (32, 64, 128, 160, 240)
+        atoms_per_tile = (L.tile_rows + 127) // 128
+        assert L.sf_atoms == (A // L.tile_rows + E + 1) * atoms_per_tile
+        assert L.x_sf - L.x_q >= A * H and L.h_q - L.x_sf >= (H // 128) * L.sf_atoms * 512
+        assert L.y - L.h_sf >= (I // 128) * L.sf_atoms * 512
+    assert moe.moe_mxfp8_workspace_layout(512, 4096, 14336, 8, 2).tile_rows == 160     # 128 rows per expert on average
+    assert moe.moe_mxfp8_workspace_layout(8192, 7168, 2048, 256, 8).tile_rows == 240   # 256 on average
+    assert moe.moe_mxfp8_workspace_layout(8192, 7040, 2048, 256, 8).tile_rows == 128   # H not a multiple of 256
+    assert moe.moe_mxfp8_workspace_bytes(16, 256, 192, 8, 2) == 0                      # I must be a multiple of 128
+    assert moe.moe_mxfp8_launch_count(0, 256, 8, 2, 8) == 0
+    assert moe.moe_mxfp8_launch_count(512, 4096, 8, 2, 8) == 5
+    assert moe.moe_mxfp8_launch_count(8192, 7168, 256, 8, 256) == 8     # three router kernels, quantise + copy
+    assert moe.moe_mxfp8_launch_count(8192, 7168, 256, 8, 32) == 7      # a local subset gathers and quantises in one
+
+
+def test_argument_errors_are_reported_before_any_launch():
+    """Host-side validation needs no GPU: nothing is launched for an empty batch or a rejected argument."""
+    L = moe.lib()
+    null = None
+    assert L.moe_forward(null, null, null, null, 0, 256, 512, 8, 2, null, null, 0, null) == 0          # T == 0
+    assert L.moe_forward(null, null, null, null, -1, 256, 512, 8, 2, null, null, 0, null) == -2        # shape
+    assert L.moe_forward(null, null, null, null, 4, 200, 512, 8, 2, null, null, 0, null) == -3         # envelope
+    assert L.moe_forward(null, null, null, null, 4, 256, 512, 8, 2, null, null, 0, null) == -1         # NULL
+    assert L.moe_forward_mxfp8(null, null, null, null, null, null, 0, 256, 128, 8, 2, null, 0, 8, null, null, 0, null, null) == 0
+    assert L.moe_forward_mxfp8(null, null, null, null, null, null, 4, 256, 192, 8, 2, null, 0, 8, null, null, 0, null, null) == -3
+    assert L.moe_forward_mxfp8(null, null, null, null, null, null, 4, 256, 128, 8, 2, null, 6, 4, null, null, 0, null, null) == -2
+    router = binding.grouped_router(3, 1)   # 8 experts do not split into 3 groups
+    import ctypes
+    assert L.moe_forward_grouped(null, null, null, null, 4, 256, 512, 8, 2, ctypes.byref(router), 0, 8, null, null, 0, null, 0) == -3
+    assert L.moe_forward_grouped(null, null, null, null, 4, 256, 512, 8, 2, None, 0, 8, null, null, 0, null, 0) == -1
+    router = binding.grouped_router(4, 1)   # one eligible group of two experts cannot supply top_k = 3
+    assert L.moe_route_grouped(null, 4, 8, 3, ctypes.byref(router), null, null, null, null, null, null, 0, null) == -3
