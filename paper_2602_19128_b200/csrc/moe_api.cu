@@ -42,7 +42,7 @@ void fill_layout(int T, int H, int I, int E, int k, moe_workspace_layout_t *L) {
     const size_t A = (size_t)T * k;
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t at = off; off += align_up(bytes, 256); return at; };
-    L->status = take(kStatusInts * sizeof(int));
+    L->status = take(kStatusBytesForward);
     L->topk_ids = take(A * sizeof(int));
     L->topk_weights = take(A * sizeof(float));
     L->expert_offsets = take((size_t)(E + 1) * sizeof(int));
@@ -106,7 +106,7 @@ int forward_impl(const void *x, const float *logits, const void *w13, const void
     };
     if (!mark(0)) return MOE_ERR_CUDA;
     if (launch_route(logits, T, E, k, LocalExperts{local_offset, n_local}, nt_max, ids, wts, offsets, s2f, f2s, rs, status,
-                     stream, 16, router) != cudaSuccess)
+                     stream, 16, router, kStatusBytesForward) != cudaSuccess)
         return MOE_ERR_CUDA;
     if (!mark(1)) return MOE_ERR_CUDA;
     if (launch_gather_rows(static_cast<const __nv_bfloat16 *>(x), s2f, offsets + n_local, A, k, H, x_perm, stream) !=
@@ -142,6 +142,14 @@ int forward_impl(const void *x, const float *logits, const void *w13, const void
         // fill TMEM and the epilogue no longer overlaps the next tile's MMAs.
         const bool single = (flags & MOE_FLAG_SINGLE_CTA_GEMM) != 0;
         const bool dense_tiles = (flags & MOE_FLAG_TWO_SLAB_GEMM) != 0;
+        // Hand-over: the down GEMM starts expert by expert as the gate/up GEMM finishes them (not with the opt-in
+        // two-slab tiles, whose epilogue counts differently).
+        if (!dense_tiles) {
+            g1.handover_role = 1;
+            g2.handover_role = 2;
+            g1.handover = g2.handover = status;
+            g2.handover_per_token_tile = handover_counts_per_token_tile(I);
+        }
         auto run = [&](const GroupedGemmArgs &g, bool allow_two_slabs) {
             int slabs = single ? 0 : grouped_gemm_tc_pair_slabs(g);
             if (slabs == 2 && !(dense_tiles && allow_two_slabs)) slabs = grouped_gemm_tc_pair_slabs(g) >= 1 ? 1 : 0;
@@ -190,7 +198,7 @@ void fill_mx_layout(int T, int H, int I, int E, int k, moe_mxfp8_workspace_layou
     const int tile = mx_tile_rows(T, H, E, k);
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t at = off; off += align_up(bytes, 256); return at; };
-    L->status = take(kStatusInts * sizeof(int));
+    L->status = take(kStatusBytesForward);
     L->topk_ids = take(A * sizeof(int));
     L->topk_weights = take(A * sizeof(float));
     L->expert_offsets = take((size_t)(E + 1) * sizeof(int));
@@ -259,7 +267,7 @@ int forward_mx_impl(const void *x, const float *logits, const void *w13_q, const
     if (!mark(0)) return MOE_ERR_CUDA;
     // every token tile exactly nt_max rows (the last of an expert partial): each tile owns one scale atom
     if (launch_route(logits, T, E, k, LocalExperts{local_offset, n_local}, nt_max, ids, wts, offsets, s2f, f2s, rs, status,
-                     stream, nt_max, router) != cudaSuccess)
+                     stream, nt_max, router, kStatusBytesForward) != cudaSuccess)
         return MOE_ERR_CUDA;
     if (!mark(1)) return MOE_ERR_CUDA;
     // Large batches with every expert resident: quantise each token once, then copy codes per assignment (the
@@ -287,6 +295,10 @@ int forward_mx_impl(const void *x, const float *logits, const void *w13_q, const
     g2.act_q = h_q; g2.act_sf = h_sf; g2.w_q = static_cast<const uint8_t *>(w2_q);
     g2.w_sf = static_cast<const uint8_t *>(w2_sf); g2.out = y; g2.out_sf = nullptr;
     g2.K = I; g2.n_out = H; g2.w_rows = H; g2.swiglu = false;
+    g1.handover_role = 1;
+    g2.handover_role = 2;
+    g1.handover = g2.handover = status;
+    g2.handover_per_token_tile = handover_counts_per_token_tile(I);
     auto run = [&](const MxGemmArgs &g) {
         return grouped_gemm_tc_mx_pair_applies(g) ? launch_grouped_gemm_tc_mx_pair(g, stream) : launch_grouped_gemm_tc_mx(g, stream);
     };

@@ -96,14 +96,15 @@ grouped_gemm_tc_kernel(const __grid_constant__ TensorMaps maps, const KernelPara
     __syncthreads();
     tcgen05_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    chain_wait();  // everything above overlapped the previous kernel; its results are read from here on
-    const int total_tiles = p.tile_prefix[p.E] * p.n_feature_tiles;
+    // everything above overlapped the previous kernel; its results are read from here on
+    const bool started = gemm_chain_start(p.handover_role, p.handover, abort_flag, p.status);
+    const int total_tiles = started ? p.tile_prefix[p.E] * p.n_feature_tiles : 0;
 
     if (warp == 0) {
         // ---------------- TMA producer: the warp walks the ring, one elected lane issues ----------------
         int stage = 0;
         uint32_t phase = 0;
-        bool ok = true;
+        bool ok = true, gate_up_done = false;
         for (int round = 0; ok; ++round) {
             const int tile = tile_of_round(round, blockIdx.x, gridDim.x);
             if (tile >= total_tiles) break;
@@ -111,6 +112,9 @@ grouped_gemm_tc_kernel(const __grid_constant__ TensorMaps maps, const KernelPara
             const int n_mma = (t.n_valid + 15) & ~15;
             const int w_row = t.e * p.w_rows + t.f * kTileM;  // down projection: 128 rows of w2[e]
             const uint32_t tx_bytes = kSlotABytes + n_mma * kRowBytes;
+            ok = handover_wait_expert(p.handover_role, p.handover, t.e, t.n_tok_tiles, p.handover_per_token_tile,
+                                      p.tile_prefix[p.E], gate_up_done, abort_flag, p.status, lane);
+            if (!ok) break;
             for (int kb = 0; kb < p.n_k_blocks; ++kb) {
                 ok = mbar_wait_warp(bar_empty + stage * 8, phase ^ 1u, abort_flag, p.status, kSiteProducerEmpty + kSiteOffset);
                 if (!ok) break;
@@ -208,6 +212,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ TensorMaps maps, const KernelPara
             tcgen05_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_acc_empty + acc * 8);
+            handover_count_tile(p.handover_role, p.handover, t.e, lane);  // (after the accumulator is handed back)
             if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
         }
     }
@@ -271,6 +276,9 @@ int launch_grouped_gemm_tc(const GroupedGemmArgs &a, cudaStream_t stream) {
     p.n_out = a.n_out;
     p.w_rows = a.w_rows;
     p.w_scale = nullptr;
+    p.handover_role = a.handover_role;
+    p.handover = a.handover;
+    p.handover_per_token_tile = a.handover_per_token_tile;
     p.n_feature_tiles = a.n_out / features_per_tile;
 
     // The tile count is only known on the device; this is its upper bound.

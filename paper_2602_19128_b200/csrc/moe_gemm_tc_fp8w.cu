@@ -364,6 +364,9 @@ int launch_grouped_gemm_tc_fp8w(const GroupedGemmArgs &a, cudaStream_t stream) {
     p.w_rows = a.w_rows;
     p.n_feature_tiles = a.n_out / features_per_tile;
     p.w_scale = a.w_scale;
+    p.handover_role = 0;
+    p.handover = nullptr;
+    p.handover_per_token_tile = 0;
 
     const long long max_token_tiles = (long long)(a.A < a.E ? a.A : a.E) + a.A / a.nt_max;
     const long long max_tiles = max_token_tiles * p.n_feature_tiles;

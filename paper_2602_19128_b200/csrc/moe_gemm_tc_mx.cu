@@ -108,14 +108,15 @@ grouped_gemm_tc_mx_kernel(const __grid_constant__ TensorMaps maps, const MxParam
     __syncthreads();
     tcgen05_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    chain_wait();  // everything above overlapped the previous kernel; its results are read from here on
-    const int total_tiles = p.tile_prefix[p.E] * p.n_feature_tiles;
+    // everything above overlapped the previous kernel; its results are read from here on
+    const bool started = gemm_chain_start(p.handover_role, p.handover, abort_flag, p.status);
+    const int total_tiles = started ? p.tile_prefix[p.E] * p.n_feature_tiles : 0;
 
     if (warp == 0) {
         // ---------------- producer: codes by TMA, scale atoms by bulk copies ----------------
         int stage = 0;
         uint32_t phase = 0;
-        bool ok = true;
+        bool ok = true, gate_up_done = false;
         for (int round = 0; ok; ++round) {
             const int tile = tile_of_round(round, blockIdx.x, gridDim.x);
             if (tile >= total_tiles) break;
@@ -125,6 +126,9 @@ grouped_gemm_tc_mx_kernel(const __grid_constant__ TensorMaps maps, const MxParam
             const uint32_t tx_bytes = kMxSlotABytes + n_mma * kMxSlotK + kMxSfAtomBytes + kMxSfBBytes;
             const uint8_t *w_sf = p.w_sf + ((size_t)t.e * p.n_feature_tiles + t.f) * p.n_k_blocks * kMxSfAtomBytes;
             const uint8_t *a_sf = p.act_sf + (size_t)t.atom * kMxSfAtomBytes;
+            ok = handover_wait_expert(p.handover_role, p.handover, t.e, t.n_tok_tiles, p.handover_per_token_tile,
+                                      p.tile_prefix[p.E], gate_up_done, abort_flag, p.status, lane);
+            if (!ok) break;
             for (int kb = 0; kb < p.n_k_blocks; ++kb) {
                 ok = mbar_wait_warp(bar_empty + stage * 8, phase ^ 1u, abort_flag, p.status, kSiteProducerEmpty + kSiteOffset);
                 if (!ok) break;
@@ -222,6 +226,7 @@ grouped_gemm_tc_mx_kernel(const __grid_constant__ TensorMaps maps, const MxParam
             tcgen05_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_acc_empty + acc * 8);
+            handover_count_tile(p.handover_role, p.handover, t.e, lane);  // (after the accumulator is handed back)
             if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
         }
     }
@@ -289,6 +294,9 @@ int launch_grouped_gemm_tc_mx(const MxGemmArgs &a, cudaStream_t stream) {
     p.n_atoms = a.n_atoms;
     p.tile_stride = a.nt_max;
     p.atoms_per_tile = 1;
+    p.handover_role = a.handover_role;
+    p.handover = a.handover;
+    p.handover_per_token_tile = a.handover_per_token_tile;
 
     const long long max_token_tiles = (long long)(a.A < a.E ? a.A : a.E) + a.A / a.nt_max;
     const long long max_tiles = max_token_tiles * p.n_feature_tiles;

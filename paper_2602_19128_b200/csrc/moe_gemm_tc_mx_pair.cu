@@ -109,8 +109,9 @@ grouped_gemm_tc_mx_pair_kernel(const __grid_constant__ MxPairMaps maps, const Mx
     cluster_sync_all();  // the peer's barriers exist before anything can signal them
     tcgen05_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    chain_wait();  // everything above overlapped the previous kernel; its results are read from here on
-    const int total_tiles = p.tile_prefix[p.E] * p.n_feature_tiles;
+    // everything above overlapped the previous kernel; its results are read from here on
+    const bool started = gemm_chain_start(p.handover_role, p.handover, abort_flag, p.status);
+    const int total_tiles = started ? p.tile_prefix[p.E] * p.n_feature_tiles : 0;
     const int n_pairs = gridDim.x >> 1, pair = blockIdx.x >> 1;
     const int w_tiles_per_expert = p.n_out / kFeatPerCta;  // weight scale atoms are stored per 128-row CTA tile
 
@@ -118,7 +119,7 @@ grouped_gemm_tc_mx_pair_kernel(const __grid_constant__ MxPairMaps maps, const Mx
     auto producer_loop = [&](const bool load_w, const bool load_act) {
         int stage = 0;
         uint32_t phase = 0;
-        bool ok = true;
+        bool ok = true, gate_up_done = false;
         for (int round = 0; ok; ++round) {
             const int tile = tile_of_round(round, pair, n_pairs);
             if (tile >= total_tiles) break;
@@ -126,6 +127,11 @@ grouped_gemm_tc_mx_pair_kernel(const __grid_constant__ MxPairMaps maps, const Mx
             const int n_mma = (t.n_valid + 15) & ~15, half = n_mma >> 1;
             const int cta_tile = 2 * t.f + (int)rank;  // this CTA's 128 weight rows
             const int w_sf_row = (t.e * w_tiles_per_expert + cta_tile) * p.n_k_blocks;
+            if (load_act) {  // the token rows of a down GEMM are the gate/up GEMM's output for this expert
+                ok = handover_wait_expert(p.handover_role, p.handover, t.e, t.n_tok_tiles, p.handover_per_token_tile,
+                                          p.tile_prefix[p.E], gate_up_done, abort_flag, p.status, lane);
+                if (!ok) { store_cluster_u32(peer_abort, 1u); break; }
+            }
             for (int kb = 0; kb < p.n_k_blocks; ++kb) {
                 ok = __all_sync(0xffffffffu, pair_wait(bar_empty + stage * 8, phase ^ 1u, abort_flag, peer_abort, p.status,
                                                        kSiteProducerEmpty + kSiteOffset));
@@ -251,6 +257,7 @@ grouped_gemm_tc_mx_pair_kernel(const __grid_constant__ MxPairMaps maps, const Mx
             tcgen05_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(map_to_cta(bar_acc_empty + acc * 8, 0));
+            handover_count_tile(p.handover_role, p.handover, t.e, lane);  // (after the accumulator is handed back)
             if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
         }
     }
@@ -317,6 +324,9 @@ int launch_grouped_gemm_tc_mx_pair(const MxGemmArgs &a, cudaStream_t stream) {
     p.n_atoms = a.n_atoms;
     p.tile_stride = a.nt_max;
     p.atoms_per_tile = atoms_per_tile;
+    p.handover_role = a.handover_role;
+    p.handover = a.handover;
+    p.handover_per_token_tile = a.handover_per_token_tile;
 
     const long long max_token_tiles = (long long)(a.A < a.E ? a.A : a.E) + a.A / a.nt_max;
     const long long max_tiles = max_token_tiles * p.n_feature_tiles;

@@ -134,8 +134,9 @@ grouped_gemm_tc_pair_kernel(const __grid_constant__ TensorMaps maps, const Kerne
     cluster_sync_all();  // the peer's barriers exist before anything can signal them
     tcgen05_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    chain_wait();  // everything above overlapped the previous kernel; its results are read from here on
-    const int total_tiles = p.tile_prefix[p.E] * p.n_feature_tiles;
+    // everything above overlapped the previous kernel; its results are read from here on
+    const bool started = gemm_chain_start(p.handover_role, p.handover, abort_flag, p.status);
+    const int total_tiles = started ? p.tile_prefix[p.E] * p.n_feature_tiles : 0;
     const int n_pairs = gridDim.x >> 1, pair = blockIdx.x >> 1;
 
     // ---------------- TMA producers (both CTAs) ----------------
@@ -144,13 +145,18 @@ grouped_gemm_tc_pair_kernel(const __grid_constant__ TensorMaps maps, const Kerne
     auto producer_loop = [&](const bool load_w, const bool load_act) {  // run by a whole warp
         int stage = 0;
         uint32_t phase = 0;
-        bool ok = true;
+        bool ok = true, gate_up_done = false;
         for (int round = 0; ok; ++round) {
             const int tile = tile_of_round(round, pair, n_pairs);
             if (tile >= total_tiles) break;
             const Tile t = decode_tile(tile, p);
             const int n_mma = (t.n_valid + 15) & ~15, half = n_mma >> 1;  // each CTA stages half: a multiple of 8 rows
             const int feat0 = t.f * kFeatPerTile + (int)rank * kFeatPerCta;  // this CTA's part of slab 0
+            if (load_act) {  // the token rows of a down GEMM are the gate/up GEMM's output for this expert
+                ok = handover_wait_expert(p.handover_role, p.handover, t.e, t.n_tok_tiles, p.handover_per_token_tile,
+                                          p.tile_prefix[p.E], gate_up_done, abort_flag, p.status, lane);
+                if (!ok) { store_cluster_u32(peer_abort, 1u); break; }
+            }
             for (int kb = 0; kb < p.n_k_blocks; ++kb) {
                 ok = __all_sync(0xffffffffu, pair_wait(bar_empty + stage * 8, phase ^ 1u, abort_flag, peer_abort, p.status,
                                                        kSiteProducerEmpty + kSiteOffset));
@@ -263,6 +269,7 @@ grouped_gemm_tc_pair_kernel(const __grid_constant__ TensorMaps maps, const Kerne
             tcgen05_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(map_to_cta(bar_acc_empty + acc * 8, 0));
+            handover_count_tile(p.handover_role, p.handover, t.e, lane);  // (after the accumulator is handed back)
             if (++acc == kAccBufs) { acc = 0; acc_phase ^= 1u; }
         }
     }
@@ -321,6 +328,9 @@ int launch_grouped_gemm_tc_pair(const GroupedGemmArgs &a, int slabs, cudaStream_
     p.n_out = a.n_out;
     p.w_rows = a.w_rows;
     p.w_scale = nullptr;
+    p.handover_role = slabs == 1 ? a.handover_role : 0;  // (the two-slab tile counts differently; the caller does not combine them)
+    p.handover = a.handover;
+    p.handover_per_token_tile = a.handover_per_token_tile;
     p.n_feature_tiles = a.n_out / features_per_pair_tile(a, slabs);
 
     const long long max_token_tiles = (long long)(a.A < a.E ? a.A : a.E) + a.A / a.nt_max;

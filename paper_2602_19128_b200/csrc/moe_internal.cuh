@@ -17,9 +17,22 @@ constexpr int kMaxTopK = 32;            // lane j of the token's warp owns rank 
 constexpr int kRouteTokensPerBlock = 32;  // tokens per router block = one histogram chunk
 constexpr int kStatusInts = 4;          // status word: {status, site, aux0, aux1}
 constexpr int kDoneCounterInt = 4;      // int index, in the status word's zeroed padding, of the fused router's block counter
+// A forward call's status region is larger and also holds the hand-over between its two GEMMs (all zeroed by the
+// memset that opens the call): a flag the gate/up GEMM raises once it has waited for its predecessors (the tile
+// schedule is then complete), and per expert a count of finished gate/up epilogue passes.  With them the down GEMM
+// starts on the SMs the gate/up GEMM has already left, expert by expert, instead of waiting for its whole grid.
+constexpr int kStatusBytesRoute = 256;
+constexpr int kStatusBytesForward = 2048;
+constexpr int kHandoverFlagInt = 8;
+constexpr int kReadyTotalInt = 9;       // all experts' counts together
+constexpr int kReadyCounterInt = 64;    // [kMaxExperts] ints from here
+// What one gate/up tile adds to its expert's counter: each of the 4 epilogue warps of each CTA counts once, and a
+// token tile is covered by I / 64 CTA-tiles of 64 features whichever kernel runs it.
+static inline int handover_counts_per_token_tile(int I) { return (I / 64) * 4; }
 
 // Site ids recorded next to MOE_ERR_DEVICE_TIMEOUT (gate/up GEMM; the down GEMM adds 4).
-enum : int { kSiteProducerEmpty = 1, kSiteMmaFull = 2, kSiteMmaTmemEmpty = 3, kSiteEpilogueTmemFull = 4 };
+enum : int { kSiteProducerEmpty = 1, kSiteMmaFull = 2, kSiteMmaTmemEmpty = 3, kSiteEpilogueTmemFull = 4,
+              kSiteHandoverFlag = 9, kSiteHandoverCount = 10 };
 
 static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
@@ -101,7 +114,7 @@ struct LocalExperts {
 cudaError_t launch_route(const float *logits, int T, int E, int k, LocalExperts local, int nt_max, int *topk_ids,
                          float *topk_w, int *expert_offsets, int *sorted_to_flat, int *flat_to_sorted,
                          RouteScratch scratch, int *status, cudaStream_t stream, int row_quantum = 16,
-                         RouterParams router = RouterParams());
+                         RouterParams router = RouterParams(), size_t status_bytes = kStatusBytesRoute);
 
 // x_perm[r,:] = x[sorted_to_flat[r] / k, :] for r < *n_rows (a device-side count, at most A)
 cudaError_t launch_gather_rows(const __nv_bfloat16 *x, const int *sorted_to_flat, const int *n_rows, int A, int k,
@@ -129,6 +142,11 @@ struct GroupedGemmArgs {
     int *status;               // status word
     bool swiglu;
     const float *w_scale = nullptr;  // FP8-weight GEMM: w points at E4M3 codes, this at [E, w_rows/128, K/128] scales
+    // hand-over between the two GEMMs of a call: 0 none; 1 this GEMM raises the flag and counts finished tiles per
+    // expert; 2 this GEMM waits for the flag instead of the previous grid, and per tile for its expert's count
+    int handover_role = 0;
+    int *handover = nullptr;            // the call's status region (flag and counters at the offsets above)
+    int handover_per_token_tile = 0;    // role 2: counts that complete one token tile of an expert
 };
 int launch_grouped_gemm_tc(const GroupedGemmArgs &args, cudaStream_t stream);  // returns a moe_status_t
 
@@ -178,6 +196,9 @@ struct MxGemmArgs {
     const int *expert_offsets, *tile_prefix, *tile_order, *tile_rows;
     int *status;
     bool swiglu;
+    int handover_role = 0;  // as in GroupedGemmArgs
+    int *handover = nullptr;
+    int handover_per_token_tile = 0;
 };
 // One-CTA tcgen05 kernel with kind::mxf8f6f4.block_scale.  The schedule must have been built with the row
 // quantum equal to nt_max (every tile nt_max rows, the last partial) and nt_max <= 128.  Needs K % 128 == 0.

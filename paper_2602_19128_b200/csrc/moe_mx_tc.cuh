@@ -25,11 +25,15 @@ struct MxParams {
     int E, n_k_blocks, n_out, w_rows, n_feature_tiles, n_atoms;
     int tile_stride;     // rows of every token tile of the MX schedule (the last of an expert may be partial)
     int atoms_per_tile;  // ceil(tile_stride / 128)
+    int handover_role;   // hand-over between the two GEMMs of a call (moe_internal.cuh)
+    int *handover;
+    int handover_per_token_tile;
 };
 
 struct MxTile {
     int e, f, row0, n_valid;
-    int atom;  // first activation scale atom of the tile
+    int atom;         // first activation scale atom of the tile
+    int n_tok_tiles;  // token tiles of this tile's expert
 };
 
 __device__ __forceinline__ MxTile decode_mx_tile(int tile, const MxParams &p) {
@@ -49,6 +53,7 @@ __device__ __forceinline__ MxTile decode_mx_tile(int tile, const MxParams &p) {
     t.row0 = begin + j * rows;
     t.n_valid = min(rows, count - j * rows);
     t.atom = (begin / p.tile_stride + t.e + j) * p.atoms_per_tile;
+    t.n_tok_tiles = n_tok_tiles;
     return t;
 }
 

@@ -569,8 +569,9 @@ int choose_nt_max(int T, int E, int k) {
 
 cudaError_t launch_route(const float *logits, int T, int E, int k, LocalExperts local, int nt_max, int *topk_ids,
                          float *topk_w, int *expert_offsets, int *sorted_to_flat, int *flat_to_sorted,
-                         RouteScratch scratch, int *status, cudaStream_t stream, int row_quantum, RouterParams router) {
-    cudaError_t err = cudaMemsetAsync(status, 0, 256, stream);  // the status word and its padding
+                         RouteScratch scratch, int *status, cudaStream_t stream, int row_quantum, RouterParams router,
+                         size_t status_bytes) {
+    cudaError_t err = cudaMemsetAsync(status, 0, status_bytes, stream);  // the status word and what shares its region
     if (err != cudaSuccess) return err;
     const int A = T * k;
     if (scratch.n_chunks <= kFusedMaxChunks) {

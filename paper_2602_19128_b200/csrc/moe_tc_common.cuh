@@ -32,6 +32,9 @@ struct KernelParams {
     int *status;
     int E, n_k_blocks, n_out, w_rows, n_feature_tiles;
     const float *w_scale;  // FP8-weight kernels only: [E, w_rows/128, K/128] block scales
+    int handover_role;     // hand-over between the two GEMMs of a call (moe_internal.cuh)
+    int *handover;
+    int handover_per_token_tile;
 };
 
 // ---- PTX wrappers -----------------------------------------------------------------------------
@@ -177,6 +180,7 @@ __device__ __forceinline__ const CUtensorMap *act_map(const TensorMaps &maps, in
 
 struct Tile {
     int e, f, row0, n_valid;
+    int n_tok_tiles;  // token tiles of this tile's expert
 };
 // Tile order: experts in schedule order (most rows first), then weight slab, then the expert's token
 // tiles (fastest), so tiles that share a weight slab run at the same time on neighbouring CTAs.
@@ -196,7 +200,80 @@ __device__ __forceinline__ Tile decode_tile(int tile, const KernelParams &p) {
     const int begin = p.expert_offsets[t.e], count = p.expert_offsets[t.e + 1] - begin;
     t.row0 = begin + j * rows;
     t.n_valid = min(rows, count - j * rows);
+    t.n_tok_tiles = n_tok_tiles;
     return t;
+}
+
+// ---- hand-over between the gate/up and the down GEMM of one call -------------------------------------------
+// Bounded poll of an int in global memory until it reaches `target` (acquire); on expiry the CTA aborts as for an
+// expired barrier wait.
+__device__ __forceinline__ bool poll_at_least(const int *addr, int target, volatile int *abort_flag, int *status, int site) {
+    const long long start = clock64();
+    while (true) {
+        int v;
+        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(addr) : "memory");
+        if (v >= target) return true;
+        if (*abort_flag) return false;
+        if (clock64() - start > kWaitLimitCycles) {
+            *abort_flag = 1;
+            if (atomicCAS(status, 0, (int)MOE_ERR_DEVICE_TIMEOUT) == 0) {
+                status[1] = site;
+                status[2] = blockIdx.x;
+            }
+            return false;
+        }
+        __nanosleep(200);
+    }
+}
+// Start of a GEMM kernel's work, after its prologue.  Role 2 (down GEMM with hand-over) does not wait for the
+// whole gate/up grid: it waits until that grid has raised the flag, i.e. has itself waited for the router and the
+// gather, so the tile schedule is complete.  Every other kernel waits for its predecessors; role 1 then raises the flag.
+__device__ __forceinline__ bool gemm_chain_start(int role, int *handover, volatile int *abort_flag, int *status) {
+    if (role == 2) {
+        bool ok = true;
+        if (threadIdx.x == 0) ok = poll_at_least(handover + kHandoverFlagInt, 1, abort_flag, status, kSiteHandoverFlag);
+        __syncthreads();
+        return !*abort_flag && ok;
+    }
+    chain_wait();
+    if (role == 1 && threadIdx.x == 0) {
+        asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(handover + kHandoverFlagInt), "r"(1) : "memory");
+    }
+    return true;
+}
+// Role 1, called by every epilogue warp after it has stored its part of a tile: the stores of all its lanes are
+// made visible, then the expert's count goes up by one.
+__device__ __forceinline__ void handover_count_tile(int role, int *handover, int expert, int lane) {
+    if (role != 1) return;
+    __threadfence();
+    __syncwarp();
+    if (lane == 0) {
+        atomicAdd(handover + kReadyCounterInt + expert, 1);
+        atomicAdd(handover + kReadyTotalInt, 1);
+    }
+}
+// Role 2, called by the token-side producer warp before the first load of a tile: all gate/up tiles of the expert
+// must have been counted; then generic-proxy writes become visible to the TMA loads that follow.
+// Once the total over all experts has been seen complete (`all_done`, kept by the caller across tiles) nothing is
+// read any more: a load from global memory in front of every tile would starve the ring of a memory-bound GEMM.
+// (whole warp: lane 0 reads, every lane fences, the result is uniform)
+__device__ __forceinline__ bool handover_wait_expert(int role, int *handover, int expert, int n_tok_tiles, int per_token_tile,
+                                                     int total_token_tiles, bool &all_done, volatile int *abort_flag,
+                                                     int *status, int lane) {
+    if (role != 2 || all_done) return true;
+    bool ok = true, done = false;
+    if (lane == 0) {
+        int total;
+        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(total) : "l"(handover + kReadyTotalInt) : "memory");
+        done = total >= total_token_tiles * per_token_tile;
+        if (!done)
+            ok = poll_at_least(handover + kReadyCounterInt + expert, n_tok_tiles * per_token_tile, abort_flag, status,
+                               kSiteHandoverCount);
+    }
+    ok = __all_sync(0xffffffffu, ok);
+    all_done = __any_sync(0xffffffffu, done);
+    asm volatile("fence.proxy.async;" ::: "memory");
+    return ok;
 }
 
 // Static tile assignment: worker w of n_workers takes, in round i, tile i*n_workers + w on even rounds
