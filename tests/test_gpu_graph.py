@@ -90,3 +90,35 @@ def test_two_streams_with_their_own_workspaces_do_not_interfere():
     for (st, inp, ws, out), ref in zip(lanes, refs):
         assert moe.moe_last_status(ws, stream=st) == moe.MOE_OK
         assert torch.equal(out.view(torch.int16), ref.view(torch.int16))
+
+
+def test_alternating_problems_on_one_workspace_stay_bit_identical():
+    """The hand-over between the two GEMMs lives in the workspace's status region and is reset by every call:
+    back-to-back calls of different problems on the same workspace must not see each other's counters."""
+    cfgs = [dict(T=600, H=256, I=256, E=8, top_k=2, skew=False), dict(T=90, H=256, I=128, E=64, top_k=6, skew=True),
+            dict(T=1300, H=128, I=64, E=16, top_k=4, skew=False)]
+    inps = [make_inputs(c, seed=30 + i, device="cuda") for i, c in enumerate(cfgs)]
+    need = max(moe.moe_workspace_bytes(c["T"], c["H"], c["I"], c["E"], c["top_k"]) for c in cfgs)
+    ws = moe.alloc_workspace(need, "cuda")
+    ws.fill_(0xFF)
+    outs = [torch.empty((c["T"], c["H"]), dtype=torch.bfloat16, device="cuda") for c in cfgs]
+    refs = None
+    for it in range(40):
+        for inp, c, out in zip(inps, cfgs, outs):
+            moe.moe_forward(inp["x"], inp["router_logits"], inp["w13"], inp["w2"], c["top_k"], out, ws)
+        if it == 0:
+            torch.cuda.synchronize()
+            assert moe.moe_last_status(ws) == moe.MOE_OK
+            refs = []
+            for inp, c in zip(inps, cfgs):  # the reference: each problem alone, on a fresh workspace
+                w2 = moe.alloc_workspace(need, "cuda")
+                r = torch.empty((c["T"], c["H"]), dtype=torch.bfloat16, device="cuda")
+                moe.moe_forward(inp["x"], inp["router_logits"], inp["w13"], inp["w2"], c["top_k"], r, w2)
+                torch.cuda.synchronize()
+                refs.append(r)
+            for out, r in zip(outs, refs):
+                assert torch.equal(out.view(torch.int16), r.view(torch.int16))
+    torch.cuda.synchronize()
+    assert moe.moe_last_status(ws) == moe.MOE_OK
+    for out, r in zip(outs, refs):
+        assert torch.equal(out.view(torch.int16), r.view(torch.int16))
