@@ -500,7 +500,7 @@ def run_ours(args):
                              value=aggregate_tokens_per_s(world, T, args.steps, e2e_overlapped_ms), unit=UNIT,
                              ms_per_step=e2e_overlapped_ms / args.steps,
                              how="two streams with their own workspaces alternate, so copies overlap kernels")),
-                gpu_launches=(moe.moe_mxfp8_launch_count(T, H, E, k, n_local) if mx else moe.moe_forward_launch_count(T)) * args.steps,
+                gpu_launches=moe.moe_forward_launch_count(T) * args.steps,
                 roofline=roofline, layer=layer, cpu_baseline=cpu_baseline)
     print(json.dumps(line), flush=True)
     if dist is not None:

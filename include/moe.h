@@ -274,8 +274,6 @@ typedef struct {
     size_t h_q;   /* uint8 [A,I]  codes of h */
     size_t h_sf;  /* scale atoms of h_q: [I/128][sf_atoms][512], same row-to-atom rule */
     size_t y;     /* bf16 [A,H] */
-    size_t x_q_tok;  /* uint8 [T,H]: codes of x per token (large batches quantise once per token, then copy) */
-    size_t x_sf_tok; /* uint8 [T,H/32]: their scale bytes, row-major */
     size_t staging; /* used only by moe_forward_mxfp8_host: device copies of x, logits, out */
     size_t sf_atoms;  /* a count, not an offset: atoms per K-slot in x_sf / h_sf */
     size_t tile_rows; /* a count: rows per token tile of this problem (32, 64, 128, 160 or 240) */
@@ -308,17 +306,14 @@ MOE_API int moe_mxfp8_quantize_rows(const void *x, int R, int K, void *codes, vo
  *   w2_q  [n_local,H,I]  uint8 codes, w2_sf_packed : its scale bytes packed with gate_up = 0
  *   workspace  at least moe_mxfp8_workspace_bytes bytes, 256-byte aligned (layout: moe_mxfp8_workspace_layout)
  *   stage_events  NULL, or MOE_NUM_STAGE_EVENTS events recorded as by moe_forward_staged
- * Launches the same number of kernels as moe_forward (the gather also quantises), one more for large batches
- * (T*top_k*H >= 64 Mi with every expert resident), which quantise x once per token and then copy codes.  Token tiles are at most
+ * Launches the same number of kernels as moe_forward (the scatter into expert-contiguous order also quantises:
+ * each token row is read and quantised once and stored to its top_k destinations).  Token tiles are at most
  * 240 rows (128 when H is not a multiple of 256).  Errors as moe_forward; a block of x holding an infinity or NaN makes that token's output NaN. */
 MOE_API int moe_forward_mxfp8(const void *x, const float *router_logits, const void *w13_q, const void *w13_sf_packed,
                               const void *w2_q, const void *w2_sf_packed, int T, int H, int I, int E, int top_k,
                               const moe_grouped_router_t *router, int local_expert_offset, int num_local_experts,
                               void *out, void *workspace, size_t workspace_bytes, void *stream,
                               void *const *stage_events);
-
-/* Host-only, pure.  Kernels one moe_forward_mxfp8 call launches for this problem (0 for T <= 0). */
-MOE_API int moe_mxfp8_launch_count(int T, int H, int E, int top_k, int num_local_experts);
 
 /* moe_forward_mxfp8 for a caller whose activations live in HOST memory, as moe_forward_host: x_host [T,H] bf16,
  * router_logits_host [T,E] f32 and out_host [T,H] bf16 are HOST pointers (pinned memory makes the copies

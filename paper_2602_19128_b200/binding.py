@@ -22,7 +22,7 @@ MOE_FLAG_TWO_SLAB_GEMM = 4
 EXPORTED = ["moe_workspace_bytes", "moe_workspace_layout", "moe_route_workspace_bytes", "moe_route", "moe_route_static",
             "moe_forward",
             "moe_forward_ex", "moe_forward_local", "moe_route_grouped", "moe_forward_grouped", "moe_forward_fp8w", "moe_mxfp8_workspace_bytes",
-            "moe_mxfp8_workspace_layout", "moe_mxfp8_pack_scales", "moe_mxfp8_quantize_rows", "moe_forward_mxfp8", "moe_forward_mxfp8_host", "moe_mxfp8_launch_count",
+            "moe_mxfp8_workspace_layout", "moe_mxfp8_pack_scales", "moe_mxfp8_quantize_rows", "moe_forward_mxfp8", "moe_forward_mxfp8_host",
             "moe_forward_staged", "moe_forward_host", "moe_last_status", "moe_forward_launch_count", "moe_status_string"]
 
 
@@ -52,8 +52,7 @@ def grouped_router(n_group: int, topk_group: int, selection_bias=None, route_sca
 class MxWorkspaceLayout(ctypes.Structure):
     _fields_ = [(n, ctypes.c_size_t) for n in
                 ("total_bytes", "status", "topk_ids", "topk_weights", "expert_offsets", "sorted_to_flat",
-                 "flat_to_sorted", "route_scratch", "x_q", "x_sf", "h_q", "h_sf", "y", "x_q_tok", "x_sf_tok", "staging", "sf_atoms",
-                 "tile_rows")]
+                 "flat_to_sorted", "route_scratch", "x_q", "x_sf", "h_q", "h_sf", "y", "staging", "sf_atoms", "tile_rows")]
 
 
 _lib = None
@@ -105,8 +104,6 @@ def lib() -> ctypes.CDLL:
         L.moe_forward_mxfp8_host.restype = i
         L.moe_forward_mxfp8_host.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, ctypes.POINTER(GroupedRouter), i, i, vp, vp,
                                              sz, vp]
-        L.moe_mxfp8_launch_count.restype = i
-        L.moe_mxfp8_launch_count.argtypes = [i] * 5
         L.moe_forward_staged.restype = i
         L.moe_forward_staged.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, vp, vp, sz, vp, ctypes.c_uint,
                                          ctypes.POINTER(vp)]
@@ -320,10 +317,6 @@ def moe_forward_mxfp8_host(x_host, router_logits_host, w13_q, w13_sf_packed, w2_
     if check and st != MOE_OK:
         raise MoeError(st, "moe_forward_mxfp8_host")
     return st
-
-
-def moe_mxfp8_launch_count(T: int, H: int, E: int, top_k: int, num_local_experts: int) -> int:
-    return int(lib().moe_mxfp8_launch_count(T, H, E, top_k, num_local_experts))
 
 
 def mx_workspace_views(workspace: torch.Tensor, T: int, H: int, I: int, E: int, top_k: int) -> dict:

@@ -109,8 +109,7 @@ int forward_impl(const void *x, const float *logits, const void *w13, const void
                      stream, 16, router, kStatusBytesForward) != cudaSuccess)
         return MOE_ERR_CUDA;
     if (!mark(1)) return MOE_ERR_CUDA;
-    if (launch_gather_rows(static_cast<const __nv_bfloat16 *>(x), s2f, offsets + n_local, A, k, H, x_perm, stream) !=
-        cudaSuccess)
+    if (launch_scatter_rows(static_cast<const __nv_bfloat16 *>(x), f2s, T, k, H, x_perm, stream) != cudaSuccess)
         return MOE_ERR_CUDA;
     if (!mark(2)) return MOE_ERR_CUDA;
 
@@ -188,11 +187,6 @@ int mx_tile_rows(int T, int H, int E, int k) {
     return mean + 2.5 * sqrt(mean) <= 160.0 ? 160 : 240;
 }
 
-// Large batches with every expert resident quantise x once per token and then copy codes per assignment.
-bool mx_two_step(long long T, int H, int E, int k, int n_local) {
-    return n_local == E && k >= 2 && (size_t)T * k * H >= ((size_t)64 << 20);
-}
-
 void fill_mx_layout(int T, int H, int I, int E, int k, moe_mxfp8_workspace_layout_t *L) {
     const size_t A = (size_t)T * k;
     const int tile = mx_tile_rows(T, H, E, k);
@@ -210,8 +204,6 @@ void fill_mx_layout(int T, int H, int I, int E, int k, moe_mxfp8_workspace_layou
     L->h_q = take(A * I);
     L->h_sf = take(mx_act_sf_bytes((int)A, E, I, tile));
     L->y = take(A * H * 2);
-    L->x_q_tok = take((size_t)T * H);
-    L->x_sf_tok = take((size_t)T * (H / 32));
     L->staging = take((size_t)T * H * 2) /* x */;
     take((size_t)T * E * sizeof(float)) /* logits */;
     take((size_t)T * H * 2) /* out */;
@@ -270,19 +262,9 @@ int forward_mx_impl(const void *x, const float *logits, const void *w13_q, const
                      stream, nt_max, router, kStatusBytesForward) != cudaSuccess)
         return MOE_ERR_CUDA;
     if (!mark(1)) return MOE_ERR_CUDA;
-    // Large batches with every expert resident: quantise each token once, then copy codes per assignment (the
-    // per-token codes stay in L2); otherwise gather and quantise in one kernel.
-    const bool two_step = mx_two_step(T, H, E, k, n_local);
-    if (two_step) {
-        uint8_t *tok_q = reinterpret_cast<uint8_t *>(ws + L.x_q_tok), *tok_sf = reinterpret_cast<uint8_t *>(ws + L.x_sf_tok);
-        if (launch_mx_quantize_rows(static_cast<const __nv_bfloat16 *>(x), T, H, tok_q, tok_sf, stream) != cudaSuccess ||
-            launch_mx_gather_codes(tok_q, tok_sf, s2f, offsets, n_local, A, k, H, x_q, x_sf, n_atoms, nt_max, stream) !=
-                cudaSuccess)
-            return MOE_ERR_CUDA;
-    } else if (launch_mx_gather_quantize(static_cast<const __nv_bfloat16 *>(x), s2f, offsets, n_local, A, k, H, x_q, x_sf,
-                                         n_atoms, nt_max, stream) != cudaSuccess) {
+    if (launch_mx_scatter_quantize(static_cast<const __nv_bfloat16 *>(x), f2s, ids, offsets, LocalExperts{local_offset, n_local},
+                                   T, k, H, x_q, x_sf, n_atoms, nt_max, stream) != cudaSuccess)
         return MOE_ERR_CUDA;
-    }
     if (!mark(2)) return MOE_ERR_CUDA;
 
     MxGemmArgs g1;
@@ -557,11 +539,6 @@ int moe_forward_launch_count(int T, unsigned flags) {
     if (T <= 0) return 0;
     // router + sort-scatter: one fused kernel up to 1024 tokens, three kernels beyond; then gather, two GEMMs, combine
     return (route_num_chunks(T) <= 32 ? 1 : 3) + 4;
-}
-
-int moe_mxfp8_launch_count(int T, int H, int E, int top_k, int num_local_experts) {
-    if (T <= 0) return 0;
-    return (route_num_chunks(T) <= 32 ? 1 : 3) + 4 + (mx_two_step(T, H, E, top_k, num_local_experts) ? 1 : 0);
 }
 
 const char *moe_status_string(int status) {

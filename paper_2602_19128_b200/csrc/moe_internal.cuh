@@ -116,9 +116,9 @@ cudaError_t launch_route(const float *logits, int T, int E, int k, LocalExperts 
                          RouteScratch scratch, int *status, cudaStream_t stream, int row_quantum = 16,
                          RouterParams router = RouterParams(), size_t status_bytes = kStatusBytesRoute);
 
-// x_perm[r,:] = x[sorted_to_flat[r] / k, :] for r < *n_rows (a device-side count, at most A)
-cudaError_t launch_gather_rows(const __nv_bfloat16 *x, const int *sorted_to_flat, const int *n_rows, int A, int k,
-                               int H, __nv_bfloat16 *x_perm, cudaStream_t stream);
+// x_perm[flat_to_sorted[t*k+j], :] = x[t, :] for every assignment with flat_to_sorted >= 0
+cudaError_t launch_scatter_rows(const __nv_bfloat16 *x, const int *flat_to_sorted, int T, int k, int H, __nv_bfloat16 *x_perm,
+                                cudaStream_t stream);
 
 // out[t,:] = sum_j topk_w[t,j] * y[flat_to_sorted[t*k+j],:]
 cudaError_t launch_combine(const __nv_bfloat16 *y, const float *topk_w, const int *flat_to_sorted, int T, int k,
@@ -208,14 +208,11 @@ int launch_grouped_gemm_tc_mx(const MxGemmArgs &args, cudaStream_t stream);
 bool grouped_gemm_tc_mx_pair_applies(const MxGemmArgs &args);
 int launch_grouped_gemm_tc_mx_pair(const MxGemmArgs &args, cudaStream_t stream);
 
-// xq[r,:], scale atoms <- MX quantisation of x[sorted_to_flat[r] / k, :] for r < expert_offsets[E].
-cudaError_t launch_mx_gather_quantize(const __nv_bfloat16 *x, const int *sorted_to_flat, const int *expert_offsets, int E,
-                                      int A, int k, int H, uint8_t *xq, uint8_t *x_sf, int n_atoms, int tile,
-                                      cudaStream_t stream);
-// The same result from rows quantised once per token (tok_codes [T,H], tok_scales [T,H/32]): a copy per sorted row.
-cudaError_t launch_mx_gather_codes(const uint8_t *tok_codes, const uint8_t *tok_scales, const int *sorted_to_flat,
-                                   const int *expert_offsets, int E, int A, int k, int H, uint8_t *xq, uint8_t *x_sf,
-                                   int n_atoms, int tile, cudaStream_t stream);
+// xq[flat_to_sorted[t*k+j], :] and that row's scale atoms <- MX quantisation of x[t,:], for every assignment with
+// flat_to_sorted >= 0 (token-major: each row is read and quantised once).
+cudaError_t launch_mx_scatter_quantize(const __nv_bfloat16 *x, const int *flat_to_sorted, const int *topk_ids,
+                                       const int *expert_offsets, LocalExperts local, int T, int k, int H, uint8_t *xq,
+                                       uint8_t *x_sf, int n_atoms, int tile, cudaStream_t stream);
 // codes[r,:], scales[r, K/32] (plain row-major) <- MX quantisation of x[r,:].
 cudaError_t launch_mx_quantize_rows(const __nv_bfloat16 *x, int R, int K, uint8_t *codes, uint8_t *scales,
                                     cudaStream_t stream);

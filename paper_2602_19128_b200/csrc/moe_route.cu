@@ -489,25 +489,36 @@ route_fused_kernel(const float *__restrict__ logits, int T, int E, int k, int lo
                       flat_to_sorted, next[warp], tid & 31);
 }
 
+// Token rows into expert-contiguous order, token-major: a warp reads (a share of) token t's row once and stores
+// it to the up to top_k rows flat_to_sorted[t*k + j] >= 0.  Reading each row once instead of once per assignment
+// halves the traffic of a top-8 layer; the copies are streamed past L2 (the GEMM reads them from memory anyway).
 __global__ void __launch_bounds__(256)
-gather_rows_kernel(const uint4 *__restrict__ x, const int *__restrict__ sorted_to_flat,
-                   const int *__restrict__ n_rows, int k, int vec_per_row, uint4 *__restrict__ x_perm) {
+scatter_rows_kernel(const uint4 *__restrict__ x, const int *__restrict__ flat_to_sorted, int T, int k, int vec_per_row,
+                    int warps_per_token, uint4 *__restrict__ x_perm) {
     chain_release();
     chain_wait();
     const int lane = threadIdx.x & 31;
-    const int r = blockIdx.x * 8 + (threadIdx.x >> 5);
-    if (r >= *n_rows) return;  // rows actually scheduled: all A assignments, or fewer with a local-expert subset
-    const int t = sorted_to_flat[r] / k;
+    const long long w = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int t = (int)(w / warps_per_token), part = (int)(w % warps_per_token);
+    if (t >= T) return;
+    const int my_row = lane < k ? flat_to_sorted[(size_t)t * k + lane] : -1;  // lane j holds rank j's destination
     const uint4 *src = x + (size_t)t * vec_per_row;
-    uint4 *dst = x_perm + (size_t)r * vec_per_row;
-    int i = lane;
-    // streaming stores: the copy is read by the GEMM from memory anyway, and keeping it out of L2 leaves the token
-    // rows (each read top_k times here) resident
-    for (; i + 96 < vec_per_row; i += 128) {  // four independent 16-byte loads in flight per lane
-        const uint4 a = src[i], b = src[i + 32], c = src[i + 64], d = src[i + 96];
-        __stcs(dst + i, a); __stcs(dst + i + 32, b); __stcs(dst + i + 64, c); __stcs(dst + i + 96, d);
+    constexpr int kInFlight = 4;  // independent 16-byte loads per lane before the first is used
+    const int stride = 32 * warps_per_token;
+    for (int i0 = part * 32 + lane; i0 < vec_per_row + lane; i0 += kInFlight * stride) {  // (i0 - lane) uniform
+        uint4 v[kInFlight];
+#pragma unroll
+        for (int u = 0; u < kInFlight; ++u)
+            if (i0 + u * stride < vec_per_row) v[u] = src[i0 + u * stride];
+        for (int j = 0; j < k; ++j) {
+            const int row = __shfl_sync(kFullMask, my_row, j);
+            if (row < 0) continue;  // assignment to an expert that is not resident here
+            uint4 *dst = x_perm + (size_t)row * vec_per_row;
+#pragma unroll
+            for (int u = 0; u < kInFlight; ++u)
+                if (i0 + u * stride < vec_per_row) __stcs(dst + i0 + u * stride, v[u]);
+        }
     }
-    for (; i < vec_per_row; i += 32) __stcs(dst + i, src[i]);
 }
 
 __global__ void __launch_bounds__(256)
@@ -590,10 +601,21 @@ cudaError_t launch_route(const float *logits, int T, int E, int k, LocalExperts 
                           expert_offsets, A, local.count, local.offset, k, sorted_to_flat, flat_to_sorted);
 }
 
-cudaError_t launch_gather_rows(const __nv_bfloat16 *x, const int *sorted_to_flat, const int *n_rows, int A, int k,
-                               int H, __nv_bfloat16 *x_perm, cudaStream_t stream) {
-    return launch_chained(gather_rows_kernel, (A + 7) / 8, 256, 0, stream, reinterpret_cast<const uint4 *>(x), sorted_to_flat,
-                          n_rows, k, H / 8, reinterpret_cast<uint4 *>(x_perm));
+// Warps per token: enough warps to fill the device when there are few tokens, at most one per 32 vectors.
+static int scatter_warps_per_token(long long tokens, int vec_per_row) {
+    const long long target = 32768;
+    long long per = tokens > 0 ? (target + tokens - 1) / tokens : 1;
+    const int most = (vec_per_row + 31) / 32;
+    if (per > most) per = most;
+    return per < 1 ? 1 : (int)per;
+}
+
+cudaError_t launch_scatter_rows(const __nv_bfloat16 *x, const int *flat_to_sorted, int T, int k, int H, __nv_bfloat16 *x_perm,
+                                cudaStream_t stream) {
+    const int wpt = scatter_warps_per_token(T, H / 8);
+    const long long warps = (long long)T * wpt;
+    return launch_chained(scatter_rows_kernel, (unsigned)((warps + 7) / 8), 256, 0, stream,
+                          reinterpret_cast<const uint4 *>(x), flat_to_sorted, T, k, H / 8, wpt, reinterpret_cast<uint4 *>(x_perm));
 }
 
 cudaError_t launch_combine(const __nv_bfloat16 *y, const float *topk_w, const int *flat_to_sorted, int T, int k,

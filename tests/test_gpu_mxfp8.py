@@ -272,9 +272,9 @@ def test_mxfp8_with_grouped_router_and_local_experts():
     assert np.all(err <= 2e-2 * (2.5 + np.abs(ref)))
 
 
-def test_mxfp8_large_batch_quantises_per_token_then_copies():
-    """From T*top_k*H = 64 Mi on, x is quantised once per token and the codes are copied per assignment: the
-    gathered codes and every scale byte must equal the oracle's, and sampled outputs its layer."""
+def test_mxfp8_large_batch_codes_and_scale_bytes():
+    """A batch of 16384 assignments: the scattered codes and every scale byte must equal the oracle's, and sampled
+    outputs its layer."""
     cfg = dict(T=2048, H=4096, I=128, E=16, top_k=8, skew=False)
     inp = make_mxfp8_inputs(cfg, seed=21, device="cuda")
     out, views = run_mx(inp)
