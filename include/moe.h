@@ -207,7 +207,8 @@ MOE_API int moe_forward_fp8w(const void *x, const float *router_logits, const vo
  * HOST array of MOE_NUM_STAGE_EVENTS cudaEvent_t handles (passed as void*, created by the caller with
  * timing enabled).  Event 0 is recorded on `stream` before the first kernel, and event i+1 after
  * stage i, where the stages are
- *   0 router + sort-scatter (1 or 3 kernels), 1 row gather, 2 gate/up GEMM + SwiGLU, 3 down GEMM, 4 combine.
+ *   0 router + sort-scatter (1 or 3 kernels), 1 token rows into expert-contiguous order, 2 gate/up GEMM + SwiGLU,
+ *   3 down GEMM, 4 combine.
  * With T == 0 nothing is launched and no event is recorded. */
 #define MOE_NUM_STAGE_EVENTS 6
 MOE_API int moe_forward_staged(const void *x, const float *router_logits, const void *w13, const void *w2, int T, int H,
