@@ -74,7 +74,7 @@ class ClockSampler:
     def stop(self) -> dict:
         if self.proc is None:
             return dict(sm_mhz=None, sm_max_mhz=None, reasons=["unavailable"])
-        time.sleep(0.15)
+        time.sleep(0.03)  # let the last sample under load be written
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
@@ -96,7 +96,7 @@ class ClockSampler:
         if not sm:
             return dict(sm_mhz=None, sm_max_mhz=None, reasons=["no_samples"])
         return dict(sm_mhz=statistics.median(sm), sm_max_mhz=max(smax), power_w=round(statistics.median(power), 1),
-                    samples=len(sm), reasons=sorted(reasons))
+                    samples=len(sm), reasons=sorted(reasons), window="timed steps and the instrumented pass after them")
 
 
 def dist_setup(n_gpus: int):
@@ -338,16 +338,19 @@ def run_ours(args):
     if not need_flush:
         step_events[0][1].record()
     barrier()
-    clocks = sampler.stop() if sampler else None
     total_ms = sum(a.elapsed_time(b) for a, b in step_events)
     # Per-kernel times: the same steps again, instrumented with an event between the stages.
-    n_staged = min(args.steps, 100)
+    # (at least 0.1 s of it, so that the clock sampler sees the load even when K is small)
+    n_staged = min(max(min(args.steps, 100), int(100.0 * args.steps / max(total_ms, 1e-3)) + 1), 2000)
     stage_events = [moe.make_stage_events() for _ in range(n_staged)]
     for s in range(n_staged):
         if need_flush:
             flush_l2(flush_buf)
         forward(stage_events[s])
     barrier()
+    # the clock samples cover the timed steps and the instrumented pass over the same steps (the same load), so that
+    # a short run still yields samples under load
+    clocks = sampler.stop() if sampler else None
     stage_ms = {name: statistics.fmean(ev[i].elapsed_time(ev[i + 1]) for ev in stage_events)
                 for i, name in enumerate(moe.STAGE_NAMES)}
     total_ms = max_over_ranks(dist, total_ms, dev)
