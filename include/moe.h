@@ -342,6 +342,13 @@ MOE_API int moe_forward_host(const void *x_host, const float *router_logits_host
  * stream reports an error. */
 MOE_API int moe_last_status(const void *workspace, void *stream);
 
+/* Self-test of the device-side error path.  Every wait inside the kernels is bounded; when one expires the kernel
+ * records MOE_ERR_DEVICE_TIMEOUT in the workspace's status word, stops and returns.  This call enqueues one small
+ * kernel that waits, with a bound of about 0.1 s, for a flag that nothing raises; afterwards moe_last_status() on
+ * the same workspace must report MOE_ERR_DEVICE_TIMEOUT and the device must be usable as before.  workspace: at
+ * least 2048 bytes, 256-byte aligned (its first 2048 bytes are overwritten). */
+MOE_API int moe_selftest_wait_timeout(void *workspace, size_t workspace_bytes, void *stream);
+
 /* Number of kernels moe_forward_ex launches for this problem with these flags (0 when T == 0). */
 MOE_API int moe_forward_launch_count(int T, unsigned flags);
 

@@ -23,7 +23,7 @@ EXPORTED = ["moe_workspace_bytes", "moe_workspace_layout", "moe_route_workspace_
             "moe_forward",
             "moe_forward_ex", "moe_forward_local", "moe_route_grouped", "moe_forward_grouped", "moe_forward_fp8w", "moe_mxfp8_workspace_bytes",
             "moe_mxfp8_workspace_layout", "moe_mxfp8_pack_scales", "moe_mxfp8_quantize_rows", "moe_forward_mxfp8", "moe_forward_mxfp8_host",
-            "moe_forward_staged", "moe_forward_host", "moe_last_status", "moe_forward_launch_count", "moe_status_string"]
+            "moe_forward_staged", "moe_forward_host", "moe_last_status", "moe_selftest_wait_timeout", "moe_forward_launch_count", "moe_status_string"]
 
 
 class MoeError(RuntimeError):
@@ -109,6 +109,8 @@ def lib() -> ctypes.CDLL:
                                          ctypes.POINTER(vp)]
         L.moe_forward_host.restype = i
         L.moe_forward_host.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, vp, vp, sz, vp]
+        L.moe_selftest_wait_timeout.restype = i
+        L.moe_selftest_wait_timeout.argtypes = [vp, sz, vp]
         L.moe_last_status.restype = i
         L.moe_last_status.argtypes = [vp, vp]
         L.moe_forward_launch_count.restype = i
@@ -386,6 +388,14 @@ def moe_forward_host(x_host, router_logits_host, w13, w2, top_k: int, out_host, 
                                 _stream(stream))
     if check and st != MOE_OK:
         raise MoeError(st, "moe_forward_host")
+    return st
+
+
+def moe_selftest_wait_timeout(workspace, stream=None) -> int:
+    """Enqueues the bounded-wait self-test; moe_last_status(workspace) must then report MOE_ERR_DEVICE_TIMEOUT (-7)."""
+    st = lib().moe_selftest_wait_timeout(_ptr(workspace), workspace.numel(), _stream(stream))
+    if st != MOE_OK:
+        raise MoeError(st, "moe_selftest_wait_timeout")
     return st
 
 

@@ -541,6 +541,17 @@ int moe_forward_launch_count(int T, unsigned flags) {
     return (route_num_chunks(T) <= 32 ? 1 : 3) + 4;
 }
 
+int moe_selftest_wait_timeout(void *workspace, size_t workspace_bytes, void *stream) {
+    if (!workspace) return MOE_ERR_NULL;
+    if (!aligned(workspace, 256)) return MOE_ERR_ALIGN;
+    if (workspace_bytes < (size_t)kStatusBytesForward) return MOE_ERR_WORKSPACE;
+    const int arch = check_device();
+    if (arch != MOE_OK) return arch;
+    return launch_wait_timeout_selftest(static_cast<int *>(workspace), static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? MOE_OK
+               : MOE_ERR_CUDA;
+}
+
 const char *moe_status_string(int status) {
     switch (status) {
         case MOE_OK: return "ok";

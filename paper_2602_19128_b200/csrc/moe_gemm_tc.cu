@@ -252,7 +252,23 @@ int dispatch(int nt_max, const TensorMaps &maps, const KernelParams &p, int grid
     }
 }
 
+__global__ void __launch_bounds__(32)
+wait_timeout_selftest_kernel(int *status) {
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) abort_flag = 0;
+    __syncwarp();
+    // the flag was zeroed by the caller's memset and nobody sets it: the poll must give up after its limit
+    if (threadIdx.x == 0) poll_at_least(status + kHandoverFlagInt, 1, &abort_flag, status, kSiteSelfTest, 200000000LL);
+}
+
 }  // namespace
+
+cudaError_t launch_wait_timeout_selftest(int *status, cudaStream_t stream) {
+    cudaError_t err = cudaMemsetAsync(status, 0, kStatusBytesForward, stream);
+    if (err != cudaSuccess) return err;
+    wait_timeout_selftest_kernel<<<1, 32, 0, stream>>>(status);
+    return cudaGetLastError();
+}
 
 int launch_grouped_gemm_tc(const GroupedGemmArgs &a, cudaStream_t stream) {
     if (a.K % kBlockK != 0 || a.A <= 0) return MOE_ERR_UNSUPPORTED;

@@ -32,7 +32,7 @@ static inline int handover_counts_per_token_tile(int I) { return (I / 64) * 4; }
 
 // Site ids recorded next to MOE_ERR_DEVICE_TIMEOUT (gate/up GEMM; the down GEMM adds 4).
 enum : int { kSiteProducerEmpty = 1, kSiteMmaFull = 2, kSiteMmaTmemEmpty = 3, kSiteEpilogueTmemFull = 4,
-              kSiteHandoverFlag = 9, kSiteHandoverCount = 10 };
+              kSiteHandoverFlag = 9, kSiteHandoverCount = 10, kSiteSelfTest = 11 };
 
 static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
@@ -220,6 +220,10 @@ cudaError_t launch_mx_quantize_rows(const __nv_bfloat16 *x, int R, int K, uint8_
 // 64 features interleaved as the gate/up GEMM reads them; else tiles of 128 consecutive rows.
 cudaError_t launch_mx_pack_scales(const uint8_t *plain, int E, int rows, int K, bool gate_up, uint8_t *packed,
                                   cudaStream_t stream);
+
+// One block waits, with a short bound, for a hand-over flag that nothing raises, and must come back with
+// MOE_ERR_DEVICE_TIMEOUT in the status word: the error path of the bounded waits, exercised without a hang.
+cudaError_t launch_wait_timeout_selftest(int *status, cudaStream_t stream);
 
 // Same contract on plain CUDA cores (validation only).
 cudaError_t launch_grouped_gemm_validation(const GroupedGemmArgs &args, cudaStream_t stream);

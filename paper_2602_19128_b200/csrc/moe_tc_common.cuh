@@ -207,14 +207,15 @@ __device__ __forceinline__ Tile decode_tile(int tile, const KernelParams &p) {
 // ---- hand-over between the gate/up and the down GEMM of one call -------------------------------------------
 // Bounded poll of an int in global memory until it reaches `target` (acquire); on expiry the CTA aborts as for an
 // expired barrier wait.
-__device__ __forceinline__ bool poll_at_least(const int *addr, int target, volatile int *abort_flag, int *status, int site) {
+__device__ __forceinline__ bool poll_at_least(const int *addr, int target, volatile int *abort_flag, int *status, int site,
+                                              long long limit_cycles = kWaitLimitCycles) {
     const long long start = clock64();
     while (true) {
         int v;
         asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(addr) : "memory");
         if (v >= target) return true;
         if (*abort_flag) return false;
-        if (clock64() - start > kWaitLimitCycles) {
+        if (clock64() - start > limit_cycles) {
             *abort_flag = 1;
             if (atomicCAS(status, 0, (int)MOE_ERR_DEVICE_TIMEOUT) == 0) {
                 status[1] = site;

@@ -122,3 +122,19 @@ def test_alternating_problems_on_one_workspace_stay_bit_identical():
     assert moe.moe_last_status(ws) == moe.MOE_OK
     for out, r in zip(outs, refs):
         assert torch.equal(out.view(torch.int16), r.view(torch.int16))
+
+
+def test_an_expired_device_wait_is_reported_and_leaves_the_device_usable():
+    """Every device-side wait is bounded.  The self-test kernel waits about 0.1 s for a flag nothing raises: it must
+    return with MOE_ERR_DEVICE_TIMEOUT in the status word, and the next call on the same workspace must work."""
+    cfg = dict(T=64, H=256, I=128, E=8, top_k=2, skew=False)
+    inp = make_inputs(cfg, seed=40, device="cuda")
+    ws = moe.alloc_workspace(moe.moe_workspace_bytes(64, 256, 128, 8, 2), "cuda")
+    moe.moe_selftest_wait_timeout(ws)
+    assert moe.moe_last_status(ws) == -7
+    views = moe.workspace_views(ws, 64, 256, 128, 8, 2)
+    assert views["status"][1].item() == 11          # the site recorded next to the status
+    out = torch.empty((64, 256), dtype=torch.bfloat16, device="cuda")
+    moe.moe_forward(inp["x"], inp["router_logits"], inp["w13"], inp["w2"], 2, out, ws)
+    assert moe.moe_last_status(ws) == moe.MOE_OK
+    assert torch.isfinite(out.float()).all()
