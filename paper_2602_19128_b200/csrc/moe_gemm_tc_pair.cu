@@ -92,7 +92,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
 grouped_gemm_tc_pair_kernel(const __grid_constant__ TensorMaps maps, const KernelParams p) {
     using L = PairSmem<NT_MAX, STAGES, SLABS>;
     constexpr int kAccBufs = SLABS == 1 ? 2 : 1;          // accumulator sets in TMEM
-    constexpr int kTmemCols = SLABS * kAccBufs * NT_MAX;  // = 2 * NT_MAX either way
+    // accumulator columns (2 * NT_MAX either way), rounded up to the power of two an allocation must be
+    constexpr int kAccCols = SLABS * kAccBufs * NT_MAX;
+    constexpr int kTmemCols = kAccCols <= 32 ? 32 : kAccCols <= 64 ? 64 : kAccCols <= 128 ? 128 : kAccCols <= 256 ? 256 : 512;
+    static_assert(kAccCols <= 512, "accumulators exceed tensor memory");
     constexpr int kSiteOffset = SWIGLU ? 0 : 4;           // the down GEMM reports sites 5..8
     // weight rows (plain) resp. h features (SwiGLU) covered by one pair tile, one slab of it, one CTA of a slab
     constexpr int kFeatPerCta = SWIGLU ? kTileM / 2 : kTileM;
