@@ -62,6 +62,8 @@ __global__ void __launch_bounds__(kThreads, 1)
 grouped_gemm_tc_kernel(const __grid_constant__ TensorMaps maps, const KernelParams p) {
     using L = SmemLayout<NT_MAX, STAGES>;
     constexpr int kTmemCols = 2 * NT_MAX;
+    static_assert(kTmemCols >= 32 && kTmemCols <= 512 && (kTmemCols & (kTmemCols - 1)) == 0,
+                  "a tensor-memory allocation must be a power of two between 32 and 512 columns");
     constexpr int kSiteOffset = SWIGLU ? 0 : 4;  // the down GEMM reports sites 5..8
     chain_release();  // the next kernel of the forward call may be scheduled; it waits for this grid to finish
     extern __shared__ uint8_t smem_raw[];

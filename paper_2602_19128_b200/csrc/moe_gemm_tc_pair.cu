@@ -96,6 +96,7 @@ grouped_gemm_tc_pair_kernel(const __grid_constant__ TensorMaps maps, const Kerne
     constexpr int kAccCols = SLABS * kAccBufs * NT_MAX;
     constexpr int kTmemCols = kAccCols <= 32 ? 32 : kAccCols <= 64 ? 64 : kAccCols <= 128 ? 128 : kAccCols <= 256 ? 256 : 512;
     static_assert(kAccCols <= 512, "accumulators exceed tensor memory");
+    static_assert((kTmemCols & (kTmemCols - 1)) == 0, "a tensor-memory allocation must be a power of two");
     constexpr int kSiteOffset = SWIGLU ? 0 : 4;           // the down GEMM reports sites 5..8
     // weight rows (plain) resp. h features (SwiGLU) covered by one pair tile, one slab of it, one CTA of a slab
     constexpr int kFeatPerCta = SWIGLU ? kTileM / 2 : kTileM;
