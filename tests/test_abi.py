@@ -1,7 +1,10 @@
 """CPU-only checks of the C-ABI library: it loads without a GPU, exports every symbol the header
 declares, and its host-only entry points behave."""
 import re
+import subprocess
 from pathlib import Path
+
+import pytest
 
 import paper_2602_19128_b200 as moe
 from paper_2602_19128_b200 import binding
@@ -23,6 +26,20 @@ def test_library_builds_loads_and_exports_every_declared_symbol():
     assert sorted(names) == sorted(binding.EXPORTED)
     for n in names:
         assert hasattr(L, n), n
+
+
+@pytest.mark.parametrize("compiler,std,suffix", [("gcc", "-std=c99", ".c"), ("g++", "-std=c++11", ".cpp")])
+def test_header_stands_alone_in_c_and_cxx(tmp_path, compiler, std, suffix):
+    """The boundary is a C ABI: the header must compile by itself, as strict C and as C++, with no CUDA or
+    torch header on the include path, and a caller must be able to take the address of every entry point."""
+    src = tmp_path / ("use_header" + suffix)
+    body = "".join(f"    p[{i}] = (const void *)&{n};\n" for i, n in enumerate(declared_symbols()))
+    src.write_text('#include "moe.h"\n#include "moe.h"\n'  # twice: the include guard holds
+                   f"const void *p[{len(declared_symbols())}];\n"
+                   "void take_addresses(void) {\n" + body + "}\n")
+    r = subprocess.run([compiler, std, "-Wall", "-Wextra", "-Werror", "-I", str(ROOT / "include"),
+                        "-c", str(src), "-o", str(tmp_path / "use_header.o")], capture_output=True, text=True)
+    assert r.returncode == 0, r.stderr
 
 
 def test_workspace_size_and_layout_are_consistent():
