@@ -107,3 +107,25 @@ def test_argument_errors_are_reported_before_any_launch():
     assert L.moe_forward_grouped(null, null, null, null, 4, 256, 512, 8, 2, None, 0, 8, null, null, 0, null, 0) == -1
     router = binding.grouped_router(4, 1)   # one eligible group of two experts cannot supply top_k = 3
     assert L.moe_route_grouped(null, 4, 8, 3, ctypes.byref(router), null, null, null, null, null, null, 0, null) == -3
+
+
+def test_missing_library_fails_loudly(monkeypatch, tmp_path):
+    """No fallback: with the shared library absent, the binding raises instead of computing anything elsewhere."""
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(binding, "_LIB_PATH", tmp_path / "libmoe_b200.so")
+    with pytest.raises(FileNotFoundError, match="no fallback"):
+        moe.moe_workspace_bytes(16, 256, 512, 8, 2)
+
+
+def test_product_sources_never_reach_the_oracle():
+    """The oracle is test infrastructure: nothing in the package (Python or CUDA) imports, includes or names it."""
+    pkg = ROOT / "paper_2602_19128_b200"
+    for f in sorted(pkg.rglob("*")):
+        if f.suffix in (".py", ".cu", ".cuh", ".h"):
+            text = f.read_text()
+            assert not re.search(r"^\s*(from|import)\s+oracle\b", text, re.M), f
+            assert "moe_oracle" not in text and "oracle/" not in text, f
+    for f in sorted((ROOT / "oracle").rglob("*")):  # and the oracle reaches nothing of the product but the input recipe
+        if f.suffix in (".py", ".c", ".h"):
+            text = f.read_text()
+            assert "csrc" not in text and "binding" not in text and "libmoe_b200" not in text, f
