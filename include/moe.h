@@ -26,9 +26,12 @@
  *   - Inputs are read-only and must not alias outputs or the workspace.
  *   - The return value is a moe_status_t: 0 on success, negative on error.  Arguments are
  *     checked on the host before anything is launched; on an error nothing has been launched.
- *   - Supported envelope: 1 <= E <= 256, 1 <= top_k <= min(E, 32), H % 64 == 0, I % 64 == 0,
- *     H % 128 == 0, T >= 0, T*top_k < 2^27.  T == 0 succeeds without a launch.
- *     Pointers must be 16-byte aligned, the workspace 256-byte aligned.
+ *   - Supported envelope: 1 <= E <= 256, 1 <= top_k <= min(E, 32), H % 128 == 0, I % 64 == 0,
+ *     T >= 0, T*top_k < 2^27.  T == 0 succeeds without a launch.
+ *     Pointers of the layer's tensors must be 16-byte aligned (the router-only entry points need
+ *     4 bytes for their arrays), the workspace 256-byte aligned.
+ *   - The current device must be compute capability 10.x (MOE_ERR_ARCH otherwise; checked after the
+ *     arguments, before the first launch).
  *   - Device-side waits are bounded.  If one expires (which indicates a bug, not bad input) the
  *     kernel records MOE_ERR_DEVICE_TIMEOUT in the workspace's status word and returns; read it
  *     with moe_last_status().
@@ -142,7 +145,10 @@ MOE_API int moe_route(const float *router_logits, int T, int E, int top_k, int32
  *     MOE_ERR_STATIC_LIMIT and launch nothing; use moe_route with a workspace for those.
  *   - The call performs no cudaMalloc / cudaFree and calls no allocating library routine.
  *   - The first call on each device looks up the array's device address (a host-side query); make that
- *     first call before starting any stream capture on that device.
+ *     first call before starting any stream capture on that device.  The address is cached per device
+ *     for the life of the process: after cudaDeviceReset() the cached address is stale and this entry
+ *     point must not be called again in that process.
+ *   - Arguments are checked as for moe_route (NULL, 4-byte alignment of every array, architecture).
  *   - All calls on a device share the one array, and it keeps the previous call's contents: the call
  *     clears or overwrites everything it later reads, so calls that run one after another (same
  *     stream, or ordered by events) are independent, but two calls whose kernels may overlap on the

@@ -5,6 +5,29 @@
 
 #include <math.h>
 
+namespace moe {
+
+int check_device() {
+    int dev = 0, major = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return MOE_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return MOE_ERR_CUDA;
+    return major == 10 ? MOE_OK : MOE_ERR_ARCH;
+}
+
+int check_route_args(const float *logits, int T, int E, int k, const int32_t *ids, const float *w, const int32_t *offsets,
+                     const int32_t *s2f, const int32_t *f2s) {
+    if (T < 0 || E <= 0 || k <= 0 || k > E) return MOE_ERR_SHAPE;
+    if (E > kMaxExperts || k > kMaxTopK || (long long)T * k >= (1LL << 27)) return MOE_ERR_UNSUPPORTED;
+    if (!offsets) return MOE_ERR_NULL;
+    if (T > 0 && (!logits || !ids || !w || !s2f || !f2s)) return MOE_ERR_NULL;
+    auto misaligned = [](const void *p) { return (reinterpret_cast<uintptr_t>(p) % 4) != 0; };
+    if (misaligned(logits) || misaligned(ids) || misaligned(w) || misaligned(offsets) || misaligned(s2f) || misaligned(f2s))
+        return MOE_ERR_ALIGN;
+    return MOE_OK;
+}
+
+}  // namespace moe
+
 namespace {
 
 using namespace moe;
@@ -56,13 +79,6 @@ void fill_layout(int T, int H, int I, int E, int k, moe_workspace_layout_t *L) {
     take((size_t)T * E * sizeof(float)) /* logits */;
     take((size_t)T * H * 2) /* out */;
     L->total_bytes = off;
-}
-
-int check_device() {
-    int dev = 0, major = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return MOE_ERR_CUDA;
-    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return MOE_ERR_CUDA;
-    return major == 10 ? MOE_OK : MOE_ERR_ARCH;
 }
 
 int forward_impl(const void *x, const float *logits, const void *w13, const void *w2, int T, int H, int I, int E, int k,
@@ -396,15 +412,14 @@ size_t moe_route_workspace_bytes(int T, int E, int top_k) {
 int moe_route(const float *router_logits, int T, int E, int top_k, int32_t *topk_ids, float *topk_weights,
               int32_t *expert_offsets, int32_t *sorted_to_flat, int32_t *flat_to_sorted, void *workspace,
               size_t workspace_bytes, void *stream) {
-    if (T < 0 || E <= 0 || top_k <= 0 || top_k > E) return MOE_ERR_SHAPE;
-    if (!route_envelope_ok(T, E, top_k)) return MOE_ERR_UNSUPPORTED;
-    if (!expert_offsets) return MOE_ERR_NULL;
-    if (T > 0 && (!router_logits || !topk_ids || !topk_weights || !sorted_to_flat || !flat_to_sorted)) return MOE_ERR_NULL;
+    const int args = check_route_args(router_logits, T, E, top_k, topk_ids, topk_weights, expert_offsets, sorted_to_flat,
+                                      flat_to_sorted);
+    if (args != MOE_OK) return args;
     if (!workspace) return MOE_ERR_NULL;
-    if (!aligned(workspace, 256) || !aligned(router_logits, 4) || !aligned(topk_ids, 4) || !aligned(topk_weights, 4) ||
-        !aligned(expert_offsets, 4) || !aligned(sorted_to_flat, 4) || !aligned(flat_to_sorted, 4))
-        return MOE_ERR_ALIGN;
+    if (!aligned(workspace, 256)) return MOE_ERR_ALIGN;
     if (workspace_bytes < moe_route_workspace_bytes(T, E, top_k)) return MOE_ERR_WORKSPACE;
+    const int arch = check_device();
+    if (arch != MOE_OK) return arch;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (T == 0) {  // no assignments: every segment is empty
         return cudaMemsetAsync(expert_offsets, 0, (size_t)(E + 1) * sizeof(int), s) == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
@@ -424,13 +439,14 @@ int moe_route_grouped(const float *router_logits, int T, int E, int top_k, const
     RouterParams rp;
     const int rs_status = make_router(router, E, top_k, &rp);
     if (rs_status != MOE_OK) return rs_status;
-    if (!expert_offsets) return MOE_ERR_NULL;
-    if (T > 0 && (!router_logits || !topk_ids || !topk_weights || !sorted_to_flat || !flat_to_sorted)) return MOE_ERR_NULL;
+    const int args = check_route_args(router_logits, T, E, top_k, topk_ids, topk_weights, expert_offsets, sorted_to_flat,
+                                      flat_to_sorted);
+    if (args != MOE_OK) return args;
     if (!workspace) return MOE_ERR_NULL;
-    if (!aligned(workspace, 256) || !aligned(router_logits, 4) || !aligned(topk_ids, 4) || !aligned(topk_weights, 4) ||
-        !aligned(expert_offsets, 4) || !aligned(sorted_to_flat, 4) || !aligned(flat_to_sorted, 4))
-        return MOE_ERR_ALIGN;
+    if (!aligned(workspace, 256)) return MOE_ERR_ALIGN;
     if (workspace_bytes < moe_route_workspace_bytes(T, E, top_k)) return MOE_ERR_WORKSPACE;
+    const int arch = check_device();
+    if (arch != MOE_OK) return arch;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (T == 0)
         return cudaMemsetAsync(expert_offsets, 0, (size_t)(E + 1) * sizeof(int), s) == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
@@ -557,7 +573,7 @@ const char *moe_status_string(int status) {
         case MOE_OK: return "ok";
         case MOE_ERR_NULL: return "a required pointer is NULL";
         case MOE_ERR_SHAPE: return "invalid shape (negative size, zero dimension, or top_k > E)";
-        case MOE_ERR_UNSUPPORTED: return "outside the supported envelope (E<=256, top_k<=32, H%128==0, I%64==0)";
+        case MOE_ERR_UNSUPPORTED: return "outside the supported envelope (E<=256, top_k<=32, H%128==0, I%64==0, T*top_k<2^27)";
         case MOE_ERR_ALIGN: return "pointer not sufficiently aligned";
         case MOE_ERR_WORKSPACE: return "workspace too small";
         case MOE_ERR_CUDA: return "a CUDA call failed";

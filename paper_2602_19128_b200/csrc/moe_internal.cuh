@@ -36,6 +36,15 @@ enum : int { kSiteProducerEmpty = 1, kSiteMmaFull = 2, kSiteMmaTmemEmpty = 3, kS
 
 static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// Host-side checks shared by the entry points (defined in moe_api.cu).
+//   check_device    : MOE_OK when the current device is compute capability 10.x, MOE_ERR_ARCH when it is not,
+//                     MOE_ERR_CUDA when it cannot be queried.
+//   check_route_args: what moe_route, moe_route_grouped and moe_route_static all require of their arguments, in the
+//                     order shape, envelope, NULL, 4-byte alignment of every array.
+int check_device();
+int check_route_args(const float *logits, int T, int E, int k, const int32_t *ids, const float *w, const int32_t *offsets,
+                     const int32_t *s2f, const int32_t *f2s);
+
 // ---- chained launches (programmatic dependent launch) ----------------------------------------------------
 // The kernels of one forward call form a chain in which each reads what its predecessors wrote.  Every kernel
 // is launched with programmatic stream serialisation allowed, announces at its very start that its dependents

@@ -666,11 +666,13 @@ extern "C" int moe_route_static(const float *router_logits, int T, int E, int to
                                 float *topk_weights, int32_t *expert_offsets, int32_t *sorted_to_flat,
                                 int32_t *flat_to_sorted, void *stream) {
     using namespace moe;
-    if (T < 0 || E <= 0 || top_k <= 0 || top_k > E) return MOE_ERR_SHAPE;
-    if (E > kMaxExperts || top_k > kMaxTopK || (long long)T * top_k >= (1LL << 27)) return MOE_ERR_UNSUPPORTED;
+    const int args = check_route_args(router_logits, T, E, top_k, topk_ids, topk_weights, expert_offsets, sorted_to_flat,
+                                      flat_to_sorted);
+    if (args == MOE_ERR_SHAPE || args == MOE_ERR_UNSUPPORTED) return args;
     if (256 + route_scratch_bytes(T, E) > kStaticScratchBytes) return MOE_ERR_STATIC_LIMIT;
-    if (!expert_offsets) return MOE_ERR_NULL;
-    if (T > 0 && (!router_logits || !topk_ids || !topk_weights || !sorted_to_flat || !flat_to_sorted)) return MOE_ERR_NULL;
+    if (args != MOE_OK) return args;
+    const int arch = check_device();
+    if (arch != MOE_OK) return arch;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (T == 0)
         return cudaMemsetAsync(expert_offsets, 0, (size_t)(E + 1) * sizeof(int), s) == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;

@@ -109,6 +109,30 @@ def test_argument_errors_are_reported_before_any_launch():
     assert L.moe_route_grouped(null, 4, 8, 3, ctypes.byref(router), null, null, null, null, null, null, 0, null) == -3
 
 
+def test_router_entry_points_share_one_argument_check():
+    """moe_route, moe_route_grouped and moe_route_static validate their arrays the same way, on the host, before
+    anything touches the device: a NULL array is -1, an array that is not 4-byte aligned is -4 (fake addresses are
+    enough: a rejected call never dereferences them), and the static variant reports its size limit first."""
+    import ctypes
+    L = moe.lib()
+    ok, odd = 0x10000, 0x10002
+    router = binding.grouped_router(1, 1)
+    for bad_slot in range(6):   # logits, ids, weights, offsets, sorted_to_flat, flat_to_sorted
+        arrays = [odd if i == bad_slot else ok for i in range(6)]
+        assert L.moe_route(arrays[0], 4, 8, 2, *arrays[1:], ok, 1 << 20, None) == -4
+        assert L.moe_route_static(arrays[0], 4, 8, 2, *arrays[1:], None) == -4
+        assert L.moe_route_grouped(arrays[0], 4, 8, 2, ctypes.byref(router), *arrays[1:], ok, 1 << 20, None) == -4
+        arrays = [None if i == bad_slot else ok for i in range(6)]
+        assert L.moe_route(arrays[0], 4, 8, 2, *arrays[1:], ok, 1 << 20, None) == -1
+        assert L.moe_route_static(arrays[0], 4, 8, 2, *arrays[1:], None) == -1
+    assert L.moe_route_static(ok, 4, 8, 9, ok, ok, ok, ok, ok, None) == -2            # top_k > E
+    assert L.moe_route_static(ok, 4, 300, 2, ok, ok, ok, ok, ok, None) == -3           # E > 256
+    assert L.moe_route_static(odd, 16288, 256, 8, odd, ok, ok, ok, ok, None) == -9     # the size limit comes first
+    assert L.moe_route(ok, 4, 8, 2, ok, ok, ok, ok, ok, ok + 64, 1 << 20, None) == -4  # workspace: 256-byte aligned
+    assert L.moe_route(ok, 4, 8, 2, ok, ok, ok, ok, ok, ok, 16, None) == -5            # workspace too small
+    assert "2^27" in moe.moe_status_string(-3)
+
+
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     """No fallback: with the shared library absent, the binding raises instead of computing anything elsewhere."""
     monkeypatch.setattr(binding, "_lib", None)

@@ -59,3 +59,29 @@ def test_reference_arm_runs_on_rank_zero_only_and_prints_one_json_line():
 
 def test_every_workload_has_a_roofline_bound():
     assert set(bench.BOUND) >= set(bench.CONFIGS)
+
+
+def test_headline_is_the_largest_workload_and_the_sweep_covers_the_other_four():
+    weights = {n: 3 * c["H"] * c["I"] * c["E"] for n, c in bench.CONFIGS.items() if n not in bench.LOCAL_CONFIGS}
+    flops = {n: 6 * c["T"] * c["top_k"] * c["H"] * c["I"] for n, c in bench.CONFIGS.items() if n not in bench.LOCAL_CONFIGS}
+    assert bench.HEADLINE == max(flops, key=flops.get) and weights[bench.HEADLINE] == max(weights.values())
+    assert set(bench.SWEEP) | {bench.HEADLINE} == set(weights)
+
+
+def test_fraction_at_clock_and_the_three_tensor_denominators():
+    peaks = dict(hbm_gbs=6544.3, tflops_burst=1644.9, tflops_sustained=1350.0, source="measured")
+    # a kernel that does exactly what 148 SMs x 8192 flop/clk deliver in 1 ms at 1000 MHz
+    flops = 148 * 8192 * 1000e6 * 1e-3
+    assert abs(bench.fraction_at_clock(flops, 1e-3, 1000.0) - 1.0) < 1e-12
+    assert bench.fraction_at_clock(flops, 1e-3, None) is None
+    f = bench.tensor_fractions(flops, 1e-3, peaks, 1000.0)
+    assert abs(f["achieved"] - 1212.416) < 1e-3 and abs(f["frac_sustained"] - 1212.416 / 1350.0) < 1e-9
+    assert abs(f["frac_burst"] - 1212.416 / 1644.9) < 1e-9 and abs(f["frac_nominal"] - 1212.416 / 2250.0) < 1e-9
+    h = bench.hbm_fractions(8e9, 1e-3, peaks)
+    assert abs(h["frac_nominal"] - 1.0) < 1e-12 and abs(h["frac_measured_copy"] - 8000 / 6544.3) < 1e-9
+
+
+def test_recorded_ncu_traffic_names_its_kernel_instance_and_commit():
+    for entry in bench.NCU_TRAFFIC.values():
+        assert entry["kernel"] and entry["commit"] and entry["source"].startswith("profiles/") and entry["scale"] >= 1
+        assert (ROOT / entry["source"]).exists()

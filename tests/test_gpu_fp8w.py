@@ -5,7 +5,8 @@ import torch
 
 import paper_2602_19128_b200 as moe
 from oracle import moe_oracle
-from paper_2602_19128_b200.inputs import bf16_bits, make_fp8w_inputs
+from paper_2602_19128_b200.inputs import bf16_bits
+from tests.weight_quantizers import make_fp8w_inputs
 from tests.gpu_common import assert_close_out, assert_routing_exact, bf16_to_f64
 
 pytestmark = pytest.mark.gpu

@@ -11,7 +11,8 @@ import torch
 
 import paper_2602_19128_b200 as moe
 from oracle import moe_oracle
-from paper_2602_19128_b200.inputs import CONFIGS, bf16_bits, quantize_mxfp8
+from paper_2602_19128_b200.inputs import CONFIGS, bf16_bits
+from tests.weight_quantizers import quantize_mxfp8
 from tests.gpu_common import OUT_TOL, assert_close_out, assert_routing_exact, bf16_to_f64, gpu_inputs, run_forward
 
 pytestmark = pytest.mark.gpu

@@ -4,7 +4,8 @@ import pytest
 import torch
 
 import paper_2602_19128_b200 as moe
-from paper_2602_19128_b200.inputs import make_inputs, make_mxfp8_inputs
+from paper_2602_19128_b200.inputs import make_inputs
+from tests.weight_quantizers import make_mxfp8_inputs
 
 pytestmark = pytest.mark.gpu
 

@@ -4,7 +4,8 @@ import pytest
 import torch
 
 from oracle import moe_oracle
-from paper_2602_19128_b200.inputs import bf16_bits, make_fp8w_inputs
+from paper_2602_19128_b200.inputs import bf16_bits
+from tests.weight_quantizers import make_fp8w_inputs
 from tests.helpers import bits_to_f64, f32_to_bf16_bits
 
 PRECISIONS = ["f32", "f64"]

@@ -7,7 +7,8 @@ import pytest
 import torch
 
 from oracle import moe_oracle
-from paper_2602_19128_b200.inputs import bf16_bits, make_mxfp8_inputs, quantize_mxfp8
+from paper_2602_19128_b200.inputs import bf16_bits
+from tests.weight_quantizers import make_mxfp8_inputs, quantize_mxfp8
 from tests.helpers import bits_to_f64
 
 # every E4M3 code's value, from torch's own float8 type (independent of the oracle's decoder)
