@@ -220,6 +220,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ TensorMaps maps, const KernelPara
     }
 
     // ---------------- teardown ----------------
+    gemm_chain_finish(p.handover_role);
     tcgen05_fence_before();
     __syncthreads();
     if (*abort_flag) {

@@ -263,6 +263,7 @@ grouped_gemm_tc_mx_pair_kernel(const __grid_constant__ MxPairMaps maps, const Mx
     }
 
     // ---------------- teardown ----------------
+    gemm_chain_finish(p.handover_role);
     tcgen05_fence_before();
     __syncthreads();
     cluster_sync_all();

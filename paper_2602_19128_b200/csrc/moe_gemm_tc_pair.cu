@@ -279,6 +279,7 @@ grouped_gemm_tc_pair_kernel(const __grid_constant__ TensorMaps maps, const Kerne
     }
 
     // ---------------- teardown ----------------
+    gemm_chain_finish(p.handover_role);
     tcgen05_fence_before();
     __syncthreads();
     cluster_sync_all();

@@ -52,7 +52,8 @@ int check_route_args(const float *logits, int T, int E, int k, const int32_t *id
 // (chain_wait) before it touches memory a predecessor writes.  A kernel's launch latency and prologue (barrier
 // set-up, tensor-memory allocation) then overlap the tail of the kernel before it.  Because EVERY block of
 // every kernel waits, completion is transitive: when a kernel's predecessor is complete, so is everything
-// earlier in the chain.
+// earlier in the chain.  (The down GEMM of a hand-over pair starts on flags instead of this wait, so its blocks
+// make the wait at their end, before teardown: gemm_chain_finish.)
 #ifdef __CUDACC__
 __device__ __forceinline__ void chain_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void chain_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }

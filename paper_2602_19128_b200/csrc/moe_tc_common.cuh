@@ -242,6 +242,12 @@ __device__ __forceinline__ bool gemm_chain_start(int role, int *handover, volati
     }
     return true;
 }
+// End of a GEMM kernel's work, before its teardown.  A role-2 grid never waited for the grid before it, only for that
+// grid's flag and counts; it waits here (the gate/up grid is finished or finishing by now, so this costs nothing), so
+// that "this grid is complete" again implies "everything before it in the stream is complete" for whatever follows.
+__device__ __forceinline__ void gemm_chain_finish(int role) {
+    if (role == 2) chain_wait();
+}
 // Role 1, called by every epilogue warp after it has stored its part of a tile: the stores of all its lanes are
 // made visible, then the expert's count goes up by one.
 __device__ __forceinline__ void handover_count_tile(int role, int *handover, int expert, int lane) {

@@ -3,6 +3,8 @@
 // SM count.
 #include "moe_mx_tc.cuh"
 
+#include <string.h>
+
 #include <mutex>
 
 namespace moe {
@@ -26,19 +28,80 @@ EncodeTiledFn get_encode_fn() {
     return fn;
 }
 
+// ---- tensor-map cache ------------------------------------------------------------------------------------
+// A forward call needs 34 tensor maps (one weight map and sixteen activation maps per GEMM); encoding them through
+// the driver costs more host time than everything else in a call.  An encoded map is a pure function of the
+// arguments of the encode call (address, element type, rank, extents, strides, box, swizzle): it does not depend on
+// the memory's contents, so an entry can never go stale -- a buffer freed and allocated again at the same address
+// with the same shape has the same map.  The cache is a fixed table of kCacheSlots entries keyed by ALL those
+// arguments, direct-mapped with a short probe, overwritten in place when full, and guarded by one mutex (look-ups
+// copy the 128-byte map out under the lock), so concurrent callers on different streams are safe.
+struct EncodeKey {
+    const void *base;
+    uint32_t rank, dtype, swizzle, pad;
+    uint64_t dims[5], strides[4];
+    uint32_t box[5], pad2;
+};
+struct CacheSlot {
+    EncodeKey key;
+    CUtensorMap map;
+    bool used;
+};
+constexpr int kCacheSlots = 1024, kCacheProbe = 8;
+std::mutex g_cache_mutex;
+CacheSlot *g_cache = nullptr;  // allocated on first use (host memory), never freed
+
+uint64_t key_hash(const EncodeKey &k) {
+    const unsigned char *b = reinterpret_cast<const unsigned char *>(&k);
+    uint64_t h = 1469598103934665603ull;
+    for (size_t i = 0; i < sizeof(EncodeKey); ++i) h = (h ^ b[i]) * 1099511628211ull;
+    return h;
+}
+
+bool encode_cached(CUtensorMap *map, CUtensorMapDataType dtype, int rank, const void *base, const cuuint64_t *dims,
+                   const cuuint64_t *strides, const cuuint32_t *box, CUtensorMapSwizzle swizzle) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    EncodeKey key;
+    memset(&key, 0, sizeof(key));  // (padding bytes take part in the comparison)
+    key.base = base;
+    key.rank = (uint32_t)rank;
+    key.dtype = (uint32_t)dtype;
+    key.swizzle = (uint32_t)swizzle;
+    for (int i = 0; i < rank; ++i) { key.dims[i] = dims[i]; key.box[i] = box[i]; }
+    for (int i = 0; i + 1 < rank; ++i) key.strides[i] = strides[i];
+    const uint64_t h = key_hash(key);
+    {
+        std::lock_guard<std::mutex> lock(g_cache_mutex);
+        if (!g_cache) g_cache = new CacheSlot[kCacheSlots]();
+        for (int i = 0; i < kCacheProbe; ++i) {
+            const CacheSlot &s = g_cache[(h + i) % kCacheSlots];
+            if (s.used && memcmp(&s.key, &key, sizeof(key)) == 0) { *map = s.map; return true; }
+        }
+    }
+    const cuuint32_t elem_strides[5] = {1, 1, 1, 1, 1};
+    if (fn(map, dtype, rank, const_cast<void *>(base), dims, strides, box, elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE,
+           swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return false;
+    std::lock_guard<std::mutex> lock(g_cache_mutex);
+    int at = (int)(h % kCacheSlots);  // a free slot within the probe window, else the home slot is replaced
+    for (int i = 0; i < kCacheProbe; ++i)
+        if (!g_cache[(h + i) % kCacheSlots].used) { at = (int)((h + i) % kCacheSlots); break; }
+    g_cache[at].key = key;
+    g_cache[at].map = *map;
+    g_cache[at].used = true;
+    return true;
+}
+
 // bf16 operands and MX codes land in the 128-byte-swizzled layout the MMA reads; the FP8 codes of the
 // dequantising kernel are staged unswizzled for its converter warps.
 enum class Operand { kBf16, kCodesForConverter, kCodesForMma };
 
 bool encode(CUtensorMap *map, const void *base, int rank, const cuuint64_t *dims, const cuuint64_t *strides,
             const cuuint32_t *box, Operand kind = Operand::kBf16) {
-    EncodeTiledFn fn = get_encode_fn();
-    if (!fn) return false;
-    const cuuint32_t elem_strides[5] = {1, 1, 1, 1, 1};
-    return fn(map, kind == Operand::kBf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, rank,
-              const_cast<void *>(base), dims, strides, box, elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE,
-              kind == Operand::kCodesForConverter ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B,
-              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    return encode_cached(map, kind == Operand::kBf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8,
+                         rank, base, dims, strides, box,
+                         kind == Operand::kCodesForConverter ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B);
 }
 
 // 2-D bf16 tensor [rows, cols] row-major; box = box_rows x 64 columns, 128-byte swizzle, zero fill.
@@ -130,15 +193,10 @@ bool encode_act_maps(CUtensorMap *maps, const void *act, uint64_t rows, uint64_t
 
 // Scale atoms as a 2-D tensor of 32-bit words: [n_atoms][128 words], box = atoms_per_box whole atoms, unswizzled.
 bool encode_scale_atoms(CUtensorMap *map, const void *atoms, uint64_t n_atoms, uint32_t atoms_per_box) {
-    EncodeTiledFn fn = get_encode_fn();
-    if (!fn) return false;
     const cuuint64_t dims[2] = {kMxSfAtomBytes / 4, n_atoms};
     const cuuint64_t strides[1] = {kMxSfAtomBytes};
     const cuuint32_t box[2] = {kMxSfAtomBytes / 4, atoms_per_box};
-    const cuuint32_t elem_strides[2] = {1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void *>(atoms), dims, strides, box, elem_strides,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    return encode_cached(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, atoms, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE);
 }
 
 int sm_count() {

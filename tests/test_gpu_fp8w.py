@@ -7,7 +7,8 @@ import paper_2602_19128_b200 as moe
 from oracle import moe_oracle
 from paper_2602_19128_b200.inputs import bf16_bits
 from tests.weight_quantizers import make_fp8w_inputs
-from tests.gpu_common import assert_close_out, assert_routing_exact, bf16_to_f64
+from tests.gpu_common import (Guarded, assert_close_out, assert_routing_exact, bf16_to_f64, check_guards, guarded_out,
+                              layer_regions)
 
 pytestmark = pytest.mark.gpu
 
@@ -16,12 +17,13 @@ def run_fp8w(inp):
     T, H = inp["x"].shape
     E, I2, _ = inp["w13_q"].shape
     I, k = I2 // 2, inp["top_k"]
-    ws = moe.alloc_workspace(moe.moe_workspace_bytes(T, H, I, E, k), "cuda")
-    ws.fill_(0xFF)
-    out = torch.full((T, H), float("nan"), dtype=torch.bfloat16, device="cuda")
+    wg = Guarded(moe.moe_workspace_bytes(T, H, I, E, k), "cuda")
+    ws = wg.inner
+    og, out = guarded_out(T, H, "cuda")
     moe.moe_forward_fp8w(inp["x"], inp["router_logits"], inp["w13_q"], inp["w13_scale"], inp["w2_q"], inp["w2_scale"], k,
                          out, ws)
     assert moe.moe_last_status(ws) == moe.MOE_OK
+    check_guards(wg, og, moe.moe_workspace_layout(T, H, I, E, k), layer_regions(T, H, I, E, k), "moe_forward_fp8w")
     return out, moe.workspace_views(ws, T, H, I, E, k)
 
 

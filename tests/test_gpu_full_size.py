@@ -13,9 +13,41 @@ import paper_2602_19128_b200 as moe
 from oracle import moe_oracle
 from paper_2602_19128_b200.inputs import CONFIGS, bf16_bits
 from tests.weight_quantizers import quantize_mxfp8
-from tests.gpu_common import OUT_TOL, assert_close_out, assert_routing_exact, bf16_to_f64, gpu_inputs, run_forward
+from tests.gpu_common import (OUT_TOL, Guarded, assert_close_out, assert_routing_exact, bf16_to_f64, check_guards,
+                              gpu_inputs, guarded_out, mx_regions, run_forward)
 
 pytestmark = pytest.mark.gpu
+
+
+def token_tile_bound(T: int, E: int, k: int) -> int:
+    """The bf16 layer's token-tile bound (the library's rule: the smallest of 32, 64, 128 that holds 1.5 x the mean
+    rows per expert, else 256)."""
+    return next((nt for nt in (32, 64, 128) if 1.5 * T * k / E <= nt), 256)
+
+
+def edge_tokens(off: np.ndarray, s2f: np.ndarray, T: int, E: int, k: int, tile_bound: int) -> np.ndarray:
+    """Tokens the oracle evaluates one by one, chosen from ITS permutation so that they sit where an indexing
+    mistake would show: the first and last row of the heaviest expert, the rows on both sides of that expert's
+    segment, the last row of its first token tile and the first row of the next (when it has several), a token of
+    an expert with exactly one row (when there is one), one routed to the highest-indexed active expert (the
+    largest weight offsets), the first and last token, and six drawn at random.  At most 16."""
+    counts = np.diff(off)
+    rows = []
+    heavy = int(np.argmax(counts))
+    b, c = int(off[heavy]), int(counts[heavy])
+    rows += [b, b + c - 1, max(b - 1, 0), min(b + c, len(s2f) - 1)]
+    n_tiles = -(-c // tile_bound)
+    if n_tiles > 1:
+        per = -(-(-(-c // n_tiles)) // 16) * 16
+        rows += [b + per - 1, b + per]
+    single = np.flatnonzero(counts == 1)
+    if len(single):
+        rows.append(int(off[single[-1]]))
+    last_active = int(np.flatnonzero(counts > 0)[-1])
+    rows.append(int(off[last_active + 1]) - 1)
+    rng = np.random.default_rng(0)
+    tokens = [int(s2f[r]) // k for r in rows] + [0, T - 1] + list(rng.choice(T, size=6, replace=False))
+    return np.unique(np.asarray(tokens)).astype(np.int32)
 
 
 def close_on_device(a: torch.Tensor, b: torch.Tensor, what: str):
@@ -41,9 +73,9 @@ def test_full_size_workload(name):
     assert torch.equal(views["x_perm"].view(torch.int16),
                        inp["x"][views["sorted_to_flat"].long() // k].view(torch.int16))
 
-    # 2. sampled tokens against the oracle (first, last, and a seeded draw; hot and cold experts)
-    rng = np.random.default_rng(0)
-    tokens = np.unique(np.concatenate([[0, T - 1], rng.choice(T, size=6, replace=False)])).astype(np.int32)
+    # 2. sampled tokens against the oracle: tile and segment edges, 64-bit weight offsets, and a seeded draw
+    tokens = edge_tokens(off, s2f, T, E, k, token_tile_bound(T, E, k))
+    assert 8 <= len(tokens) <= 16
     need = sorted({int(e) for t in tokens for e in ids[t]})
     experts = {e: (bf16_bits(inp["w13"][e]), bf16_bits(inp["w2"][e])) for e in need}
     ref = o.forward_sampled(bf16_bits(inp["x"]), logits, experts, I, k, tokens)
@@ -78,10 +110,12 @@ def test_full_size_workload_mxfp8(name):
     sf13, sf2 = moe.moe_mxfp8_pack_scales(w13_s, True), moe.moe_mxfp8_pack_scales(w2_s, False)
 
     def run():
-        ws = moe.alloc_workspace(moe.moe_mxfp8_workspace_bytes(T, H, I, E, k), "cuda")
-        out = torch.full((T, H), float("nan"), dtype=torch.bfloat16, device="cuda")
+        wg = Guarded(moe.moe_mxfp8_workspace_bytes(T, H, I, E, k), "cuda")
+        ws = wg.inner
+        og, out = guarded_out(T, H, "cuda")
         moe.moe_forward_mxfp8(inp["x"], inp["router_logits"], w13_q, sf13, w2_q, sf2, k, out, ws)
         assert moe.moe_last_status(ws) == moe.MOE_OK
+        check_guards(wg, og, moe.moe_mxfp8_workspace_layout(T, H, I, E, k), mx_regions(T, H, I, E, k), f"{name} mxfp8")
         return out, ws
 
     out, ws = run()
@@ -92,8 +126,8 @@ def test_full_size_workload_mxfp8(name):
     off, s2f, f2s = o.permute(ids, E)
     assert_routing_exact(views, ids, w, off, s2f, f2s)
 
-    rng = np.random.default_rng(0)
-    tokens = np.unique(np.concatenate([[0, T - 1], rng.choice(T, size=6, replace=False)])).astype(np.int32)
+    tokens = edge_tokens(off, s2f, T, E, k, int(views["tile_rows"]))
+    assert 8 <= len(tokens) <= 16
     xc, _ = o.mx_quantize(inp["x"][torch.from_numpy(tokens).long().cuda()].float().cpu().numpy())
     for n_i, t in enumerate(tokens):  # every sorted row of a sampled token holds that token's codes
         rows = f2s[t * k:(t + 1) * k]

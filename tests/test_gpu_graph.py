@@ -139,3 +139,91 @@ def test_an_expired_device_wait_is_reported_and_leaves_the_device_usable():
     moe.moe_forward(inp["x"], inp["router_logits"], inp["w13"], inp["w2"], 2, out, ws)
     assert moe.moe_last_status(ws) == moe.MOE_OK
     assert torch.isfinite(out.float()).all()
+
+
+_FRESH = r"""
+import sys, torch
+sys.path.insert(0, {root!r})
+import paper_2602_19128_b200 as moe
+from paper_2602_19128_b200.inputs import make_inputs
+cfg = dict(T={T}, H={H}, I={I}, E={E}, top_k={k}, skew=False)
+inp = make_inputs(cfg, seed={seed}, device="cuda")
+out = torch.empty(({T}, {H}), dtype=torch.bfloat16, device="cuda")
+ws = moe.alloc_workspace(moe.moe_workspace_bytes({T}, {H}, {I}, {E}, {k}), "cuda")
+moe.moe_forward(inp["x"], inp["router_logits"], inp["w13"], inp["w2"], {k}, out, ws)
+assert moe.moe_last_status(ws) == 0
+torch.save(out.cpu(), {path!r})
+"""
+
+
+def test_tensor_map_cache_alternating_weight_sets_and_shapes_match_fresh_processes(tmp_path):
+    """The library caches encoded tensor maps keyed by every argument of the encoding.  One process alternates two
+    weight sets and two shapes, frees a weight set and allocates another where it was, and every result must be
+    bit-identical to the result of a process that has never run anything else (so no entry can be stale)."""
+    import subprocess
+    import sys
+    from pathlib import Path
+    root = str(Path(__file__).resolve().parent.parent)
+    cases = [(dict(T=300, H=256, I=256, E=8, top_k=2, skew=False), 51), (dict(T=300, H=256, I=256, E=8, top_k=2, skew=False), 52),
+             (dict(T=700, H=128, I=192, E=4, top_k=2, skew=False), 53)]
+    fresh = []
+    for i, (c, seed) in enumerate(cases):
+        path = str(tmp_path / f"fresh{i}.pt")
+        src = _FRESH.format(root=root, T=c["T"], H=c["H"], I=c["I"], E=c["E"], k=c["top_k"], seed=seed, path=path)
+        r = subprocess.run([sys.executable, "-c", src], capture_output=True, text=True, timeout=600)
+        assert r.returncode == 0, r.stderr
+        fresh.append(torch.load(path).cuda())
+    inps = [make_inputs(c, seed=s, device="cuda") for c, s in cases]
+    wss = [moe.alloc_workspace(moe.moe_workspace_bytes(c["T"], c["H"], c["I"], c["E"], c["top_k"]), "cuda") for c, _ in cases]
+    for it in range(6):
+        for i in (0, 1, 2, 1, 0):
+            c = cases[i][0]
+            out = torch.empty((c["T"], c["H"]), dtype=torch.bfloat16, device="cuda")
+            moe.moe_forward(inps[i]["x"], inps[i]["router_logits"], inps[i]["w13"], inps[i]["w2"], c["top_k"], out, wss[i])
+            torch.cuda.synchronize()
+            assert torch.equal(out.view(torch.int16), fresh[i].view(torch.int16)), (it, i)
+        if it == 2:  # drop weight set 0 and draw it again: torch's allocator hands back the same addresses
+            ptr = inps[0]["w13"].data_ptr()
+            inps[0] = None
+            inps[0] = make_inputs(cases[0][0], seed=cases[0][1], device="cuda")
+            assert isinstance(ptr, int)
+
+
+def test_two_host_threads_calling_concurrently_with_their_own_workspaces():
+    """The tensor-map cache is the library's only shared mutable state; it is guarded by a mutex, so two host threads
+    may call at the same time (each on its own stream, with its own workspace)."""
+    import threading
+    cfgs = [dict(T=500, H=256, I=256, E=16, top_k=4, skew=True), dict(T=200, H=384, I=128, E=8, top_k=2, skew=False)]
+    inps = [make_inputs(c, seed=60 + i, device="cuda") for i, c in enumerate(cfgs)]
+    refs = []
+    for inp, c in zip(inps, cfgs):
+        ws = moe.alloc_workspace(moe.moe_workspace_bytes(c["T"], c["H"], c["I"], c["E"], c["top_k"]), "cuda")
+        r = torch.empty((c["T"], c["H"]), dtype=torch.bfloat16, device="cuda")
+        moe.moe_forward(inp["x"], inp["router_logits"], inp["w13"], inp["w2"], c["top_k"], r, ws)
+        torch.cuda.synchronize()
+        refs.append(r)
+    errors, outs = [], [None, None]
+
+    def worker(i):
+        try:
+            torch.cuda.set_device(0)
+            c, inp = cfgs[i], inps[i]
+            st = torch.cuda.Stream()
+            ws = moe.alloc_workspace(moe.moe_workspace_bytes(c["T"], c["H"], c["I"], c["E"], c["top_k"]), "cuda")
+            out = torch.empty((c["T"], c["H"]), dtype=torch.bfloat16, device="cuda")
+            for _ in range(200):
+                moe.moe_forward(inp["x"], inp["router_logits"], inp["w13"], inp["w2"], c["top_k"], out, ws, stream=st)
+            st.synchronize()
+            assert moe.moe_last_status(ws, stream=st) == moe.MOE_OK
+            outs[i] = out
+        except Exception as exc:  # surfaced in the main thread
+            errors.append(exc)
+
+    threads = [threading.Thread(target=worker, args=(i,)) for i in range(2)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
+    for out, r in zip(outs, refs):
+        assert torch.equal(out.view(torch.int16), r.view(torch.int16))

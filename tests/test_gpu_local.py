@@ -6,7 +6,8 @@ import torch
 import paper_2602_19128_b200 as moe
 from oracle import moe_oracle
 from paper_2602_19128_b200.inputs import bf16_bits
-from tests.gpu_common import WEIGHT_TOL, assert_close_out, bf16_to_f64, gpu_inputs
+from tests.gpu_common import (WEIGHT_TOL, Guarded, assert_close_out, bf16_to_f64, check_guards, gpu_inputs, guarded_out,
+                              layer_regions)
 
 pytestmark = pytest.mark.gpu
 
@@ -18,11 +19,12 @@ def run_local(inp, lo, n, flags=0):
     w13 = inp["w13"][lo:lo + n].contiguous()
     w2 = inp["w2"][lo:lo + n].contiguous()
     I = w13.shape[1] // 2
-    ws = moe.alloc_workspace(moe.moe_workspace_bytes(T, H, I, E, k), x.device)
-    ws.fill_(0xFF)
-    out = torch.full((T, H), float("nan"), dtype=torch.bfloat16, device=x.device)
+    wg = Guarded(moe.moe_workspace_bytes(T, H, I, E, k), x.device)
+    ws = wg.inner
+    og, out = guarded_out(T, H, x.device)
     moe.moe_forward_local(x, logits, w13, w2, k, lo, out, ws, flags=flags)
     assert moe.moe_last_status(ws) == moe.MOE_OK
+    check_guards(wg, og, moe.moe_workspace_layout(T, H, I, E, k), layer_regions(T, H, I, E, k, n), "moe_forward_local")
     return out, moe.workspace_views(ws, T, H, I, E, k), ws
 
 

@@ -9,7 +9,8 @@ import paper_2602_19128_b200 as moe
 from oracle import moe_oracle
 from paper_2602_19128_b200.inputs import bf16_bits
 from tests.weight_quantizers import make_mxfp8_inputs
-from tests.gpu_common import assert_close_out, assert_routing_exact, bf16_to_f64
+from tests.gpu_common import (Guarded, assert_close_out, assert_routing_exact, bf16_to_f64, check_guards, guarded_out,
+                              mx_regions)
 
 pytestmark = pytest.mark.gpu
 
@@ -42,13 +43,14 @@ def run_mx(inp, local_offset=0):
     I, k = I2 // 2, inp["top_k"]
     w13_sf = moe.moe_mxfp8_pack_scales(inp["w13_s"], gate_up=True)
     w2_sf = moe.moe_mxfp8_pack_scales(inp["w2_s"], gate_up=False)
-    ws = moe.alloc_workspace(moe.moe_mxfp8_workspace_bytes(T, H, I, E, k), "cuda")
-    ws.fill_(0xFF)
-    out = torch.full((T, H), float("nan"), dtype=torch.bfloat16, device="cuda")
+    wg = Guarded(moe.moe_mxfp8_workspace_bytes(T, H, I, E, k), "cuda")
+    ws = wg.inner
+    og, out = guarded_out(T, H, "cuda")
     moe.moe_forward_mxfp8(inp["x"], inp["router_logits"], inp["w13_q"], w13_sf, inp["w2_q"], w2_sf, k, out, ws,
                           local_expert_offset=local_offset)
     status = moe.moe_last_status(ws)
     assert status == moe.MOE_OK, moe.moe_status_string(status)
+    check_guards(wg, og, moe.moe_mxfp8_workspace_layout(T, H, I, E, k), mx_regions(T, H, I, E, k, n_local), "moe_forward_mxfp8")
     return out, moe.mx_workspace_views(ws, T, H, I, E, k)
 
 

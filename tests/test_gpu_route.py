@@ -6,23 +6,28 @@ import torch
 import paper_2602_19128_b200 as moe
 from oracle import moe_oracle
 from paper_2602_19128_b200.inputs import CONFIGS, zipf_bias
-from tests.gpu_common import WEIGHT_TOL
+from tests.gpu_common import WEIGHT_TOL, Guarded
 
 pytestmark = pytest.mark.gpu
 
 
 def run_route(logits: torch.Tensor, k: int):
+    """moe_route with every output array and the workspace between sentinel bands (checked after the call)."""
     T, E = logits.shape
     dev = logits.device
     A = T * k
-    ids = torch.full((T, k), -1, dtype=torch.int32, device=dev)
-    w = torch.full((T, k), float("nan"), dtype=torch.float32, device=dev)
-    off = torch.full((E + 1,), -1, dtype=torch.int32, device=dev)
-    s2f = torch.full((A,), -1, dtype=torch.int32, device=dev)
-    f2s = torch.full((A,), -1, dtype=torch.int32, device=dev)
-    ws = moe.alloc_workspace(moe.moe_route_workspace_bytes(T, E, k), dev)
-    moe.moe_route(logits, k, ids, w, off, s2f, f2s, ws)
-    assert moe.moe_last_status(ws) == moe.MOE_OK
+    guards = [Guarded(n * 4, dev, fill=0xFF) for n in (A, A, E + 1, A, A)]
+    ids, w, off, s2f, f2s = (g.inner[:n * 4].view(dt).view(shape) for g, n, dt, shape in zip(
+        guards, (A, A, E + 1, A, A), (torch.int32, torch.float32, torch.int32, torch.int32, torch.int32),
+        ((T, k), (T, k), (E + 1,), (A,), (A,))))
+    wg = Guarded(moe.moe_route_workspace_bytes(T, E, k), dev)
+    moe.moe_route(logits, k, ids, w, off, s2f, f2s, wg.inner)
+    assert moe.moe_last_status(wg.inner) == moe.MOE_OK
+    for g, name in zip(guards + [wg], ("topk_ids", "topk_weights", "expert_offsets", "sorted_to_flat", "flat_to_sorted",
+                                       "workspace")):
+        g.assert_bands_intact(f"moe_route {name}")
+        if name != "workspace" and g.n > [A, A, E + 1, A, A][guards.index(g)] * 4:   # bytes past the array's end
+            assert bool((g.inner[[A, A, E + 1, A, A][guards.index(g)] * 4:] == 0xFF).all()), name
     return [t.cpu().numpy() for t in (ids, w, off, s2f, f2s)]
 
 
