@@ -19,6 +19,7 @@ workload and metric; it is a deliberately plain program, reported as a baseline.
 from __future__ import annotations
 
 import argparse
+import faulthandler
 import json
 import math
 import os
@@ -82,7 +83,7 @@ class ClockSampler:
     REASON_BITS = {"hw_slowdown": 0x8, "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20, "sw_power_cap": 0x4}
     NAMES = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
 
-    def __init__(self, device: int, period_s: float = 0.005):
+    def __init__(self, device: int, period_s: float = 0.01):
         self.rows, self.proc, self.thread, self.tmp = [], None, None, None
         self.stop_flag = threading.Event()
         uuid = str(torch.cuda.get_device_properties(device).uuid)
@@ -224,24 +225,15 @@ def oracle_sample(cfg_name: str, inp: dict, n_tokens: int, seed: int = 0):
     return o, bf16_bits(inp["x"]), logits, experts, I, k, tokens
 
 
-def token_tile_bound(T: int, E: int, k: int) -> int:
-    """The library's token-tile bound for the bf16 layer: the smallest of 32, 64, 128 holding 1.5 x the mean rows
-    per expert, else 256 (reporting only; mirrors the library's choose_nt_max)."""
-    avg = T * k / E
-    for nt in (32, 64, 128):
-        if 1.5 * avg <= nt:
-            return nt
-    return 256
-
-
 def computed_rows(counts, tile_bound: int, even: bool) -> int:
-    """Rows the GEMMs multiply (MMA N summed over token tiles): an expert's rows are cut into as few tiles as fit
-    under the bound, evenly sized (bf16) or of exactly the bound (MX), and each tile is rounded up to 16 rows."""
+    """Rows the GEMMs multiply (MMA N summed over token tiles): an expert's rows are one tile if they fit under the
+    bound, else as few tiles as fit under min(bound, 256), evenly sized (bf16) or of exactly the bound (MX), and each
+    tile is rounded up to 16 rows."""
     total = 0
     for c in (int(v) for v in counts):
         if c == 0:
             continue
-        n_tiles = -(-c // tile_bound)
+        n_tiles = 1 if c <= tile_bound else -(-c // min(tile_bound, 256))
         rows = -(-(-(-c // n_tiles)) // 16) * 16 if even else tile_bound
         for j in range(n_tiles):
             total += -(-min(rows, c - j * rows) // 16) * 16
@@ -396,9 +388,9 @@ def measure(ctx: Ctx, name: str, inp: dict, steps, warmup: int, with_e2e: bool, 
         elif fp8:
             moe.moe_forward_fp8w(x, logits, w13, w13_scale, w2, w2_scale, k, out, ws, stage_events=events)
         elif events is None:
-            moe.moe_forward_local(x, logits, w13, w2, k, local_offset, out, ws)
+            moe.moe_forward_local(x, logits, w13, w2, k, local_offset, out, ws, flags=args.flags)
         else:
-            moe.moe_forward_staged(x, logits, w13, w2, k, out, ws, events, local_expert_offset=local_offset)
+            moe.moe_forward_staged(x, logits, w13, w2, k, out, ws, events, local_expert_offset=local_offset, flags=args.flags)
     flush_buf = torch.zeros(2 * L2_BYTES // 4, dtype=torch.float32, device=dev) if need_flush else None
 
     def check_status(w=None):
@@ -448,6 +440,8 @@ def measure(ctx: Ctx, name: str, inp: dict, steps, warmup: int, with_e2e: bool, 
     # Per-kernel times: the same steps again, instrumented with an event between the stages
     # (at least 0.15 s of it, so that the clock sampler sees the load even when K is small).
     n_staged = min(max(min(steps, 100), int(150.0 * steps / max(total_ms, 1e-3)) + 1), 2000)
+    if args.few_launches:
+        n_staged = min(steps, 3)
     stage_events = [moe.make_stage_events() for _ in range(n_staged)]
     for s in range(n_staged):
         if need_flush:
@@ -463,12 +457,20 @@ def measure(ctx: Ctx, name: str, inp: dict, steps, warmup: int, with_e2e: bool, 
     # Host time of one call: the calling thread's time over a run of un-synchronised calls (argument checks,
     # tensor-map look-ups, the launches), the queue empty at the start and far from full at the end.
     torch.cuda.synchronize()
-    n_host = int(min(max(steps, 20), 100))
+    n_host = 1 if args.few_launches else int(min(max(steps, 20), 100))
     host_t0 = time.perf_counter()
     for _ in range(n_host):
         forward()
     host_us = (time.perf_counter() - host_t0) / n_host * 1e6
     torch.cuda.synchronize()
+
+    # The GEMM kernels' own clock probes (block 0's SM cycle counter and the global nanosecond timer at its start
+    # and end, left in the status region by the last call): the clock each kernel really ran at.
+    probe = ws[128:192].view(torch.int64).cpu().tolist()
+    probes = []
+    for g in range(2):
+        cyc, ns = probe[4 * g + 1] - probe[4 * g], probe[4 * g + 3] - probe[4 * g + 2]
+        probes.append(dict(cycles=cyc, ns=ns, sm_mhz=1e3 * cyc / ns) if cyc > 0 and ns > 0 else None)
 
     views = moe.mx_workspace_views(ws, T, H, I, E, k) if mx else moe.workspace_views(ws, T, H, I, E, k)
     counts = torch.diff(views["expert_offsets"][:n_local + 1]).cpu().numpy()
@@ -582,11 +584,19 @@ def measure(ctx: Ctx, name: str, inp: dict, steps, warmup: int, with_e2e: bool, 
                         unit="TFLOP/s", frac=g1_tensor["frac_sustained"], frac_sustained=g1_tensor["frac_sustained"],
                         frac_burst=g1_tensor["frac_burst"], frac_nominal=g1_tensor["frac_nominal"],
                         frac_at_clock=g1_tensor["frac_at_clock"], algorithmic_per_launch=g1_flops)
+    def probe_fields(pr, flops):
+        if pr is None or mx or fp8:
+            return dict(kernel_clock_probe=None)
+        return dict(kernel_clock_probe=dict(sm_mhz=round(pr["sm_mhz"], 1), kernel_ms=pr["ns"] * 1e-6,
+                                            frac_of_pipe_cycles=flops / (pr["cycles"] * SM_COUNT * TENSOR_FLOP_PER_CLK_SM),
+                                            how="block 0's cycle counter and the global timer across the kernel's last launch"))
+    roofline.update(probe_fields(probes[0], g1_flops))
     roofline.update(kernel="gate/up GEMM (grouped_gemm_tc*_kernel<swiglu>)", kernel_ms=stage_ms["gemm1_swiglu"],
                     peak_source=f"of {peaks['source']}" + ("" if bound == "hbm" else
                                                            " (sustained: the kernel is timed inside a long step)"),
                     traffic=traffic, traffic_source=traffic_source,
                     down_gemm=dict(kernel="down GEMM (grouped_gemm_tc*_kernel<plain>)", kernel_ms=stage_ms["gemm2"],
+                                   **probe_fields(probes[1], g2_flops),
                                    **({"algorithmic_per_launch": g2_bytes, **g2_hbm} if bound == "hbm" else
                                       {"algorithmic_per_launch": g2_flops, **g2_tensor})))
     step_s = total_ms * 1e-3 / steps
@@ -594,7 +604,7 @@ def measure(ctx: Ctx, name: str, inp: dict, steps, warmup: int, with_e2e: bool, 
     # per-step latencies: from the timed steps when each has its own events, else from the instrumented pass
     per_step_ms = sorted(a.elapsed_time(b) for a, b in step_events) if need_flush else \
         sorted(ev[0].elapsed_time(ev[-1]) for ev in stage_events)
-    tile_bound = int(views["tile_rows"]) if mx else token_tile_bound(T, E, k)
+    tile_bound = int(views["tile_rows"]) if mx else moe.moe_token_tile_rows(T, H, I, E, k, args.flags)
     staged_sum = sum(stage_ms.values())
     non_gemm = stage_ms["route"] + stage_ms["gather"] + stage_ms["combine"]
     layer = dict(stage_ms={n: round(v, 5) for n, v in stage_ms.items()}, n_active_experts=n_active,
@@ -602,6 +612,7 @@ def measure(ctx: Ctx, name: str, inp: dict, steps, warmup: int, with_e2e: bool, 
                  latency_ms_median=statistics.median(per_step_ms), latency_ms_min=per_step_ms[0],
                  latency_source="timed steps" if need_flush else "instrumented pass (events between the stages)",
                  stage_ms_source=f"instrumented pass of {n_staged} steps after the timed ones",
+                 token_tile_bound=tile_bound,
                  padding_efficiency=rows_scheduled / max(1, computed_rows(counts, tile_bound, even=not mx)),
                  rows_per_expert_min=int(counts.min()), rows_per_expert_max=int(counts.max()),
                  weights=hbm_fractions(active_weight_bytes, step_s, peaks),
@@ -663,8 +674,8 @@ def run_ours(args):
                 sweep[name] = dict(error=f"{type(exc).__name__}: {exc}")
             torch.cuda.empty_cache()
     inp = shared if shared is not None else make_inputs(CONFIGS[headline], seed=args.seed + rank, device=ctx.dev)
-    r = measure(ctx, headline, inp, steps=args.steps, warmup=args.warmup, with_e2e=True,
-                with_cpu_baseline=not args.no_cpu_baseline)
+    r = measure(ctx, headline, inp, steps=args.steps, warmup=args.warmup, with_e2e=not args.few_launches,
+                with_cpu_baseline=not args.no_cpu_baseline and not args.few_launches)
     if rank == 0:
         line = dict(metric=METRIC, value=r["value"], unit=UNIT, n_gpus=world, steps=r["steps"], warmup=r["warmup"],
                     ms_per_step=r["ms_per_step"], higher_is_better=True, scaling="weak", vs_baseline=None, dtype=r["dtype"],
@@ -692,13 +703,23 @@ def main():
                          "mxfp8: weights and activations in MX FP8 on the block-scaled MMA (moe_forward_mxfp8)")
     ap.add_argument("--router", choices=["softmax", "grouped"], default="softmax",
                     help="grouped: sigmoid scores, selection bias, 8 groups of which 4 eligible, weights x 2.5 (with --weights mxfp8)")
+    ap.add_argument("--flags", type=int, default=0, help="MOE_FLAG_* bits for the device-resident bf16 steps (A/B timing)")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--warm-seconds", type=float, default=1.0,
                     help="warm-up lasts at least this long (and at least --warmup steps): the settled power state")
     ap.add_argument("--sweep-seconds", type=float, default=0.5, help="timed region of each sweep workload")
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="budget of the CPU-oracle baseline leg")
+    ap.add_argument("--few-launches", action="store_true",
+                    help="for runs under a profiler: six warm-up steps, the K timed steps, at most three instrumented "
+                         "ones, no end-to-end or host-time loops (the numbers of such a run are not benchmark values)")
+    ap.add_argument("--watchdog-seconds", type=float, default=1200.0,
+                    help="dump every thread's Python stack to stderr and exit(1) if the run is not over by then")
     args = ap.parse_args()
+    if args.watchdog_seconds > 0:  # a stuck run ends by itself, with evidence of where it was
+        faulthandler.dump_traceback_later(args.watchdog_seconds, exit=True)
+    if args.few_launches:
+        args.warm_seconds = 0.0
     if args.shape:
         T, H, I, E, k = (int(v) for v in args.shape.split(","))
         args.config = f"custom_{T}x{H}x{I}x{E}x{k}"

@@ -86,6 +86,12 @@ typedef enum {
 /* Let the CTA-pair kernel of the gate/up GEMM use two weight slabs per CTA (512 x N pair tiles) where
  * the shape allows it.  Off by default (slower on the measured workloads); for tests and A/B timing. */
 #define MOE_FLAG_TWO_SLAB_GEMM 4u
+/* Keep token tiles at 256 rows or fewer even where the wide-tile kernel (one pass over a weight slab for an
+ * expert of up to 320 / 384 rows) would be chosen.  For tests and A/B timing. */
+#define MOE_FLAG_NARROW_TILES 8u
+/* Where the wide-tile kernel runs the gate/up GEMM, let it fetch token rows straight from x by row index (TMA
+ * four-row gather) instead of reading the expert-contiguous copy; x_perm is then not written.  Opt-in: for A/B timing. */
+#define MOE_FLAG_GATHER_IN_LOAD 16u
 
 /* Byte offsets of the intermediates inside the workspace of moe_forward (so tests and tools can
  * read them after the stream has been synchronised).  Filled by moe_workspace_layout(). */
@@ -354,6 +360,11 @@ MOE_API int moe_last_status(const void *workspace, void *stream);
  * the same workspace must report MOE_ERR_DEVICE_TIMEOUT and the device must be usable as before.  workspace: at
  * least 2048 bytes, 256-byte aligned (its first 2048 bytes are overwritten). */
 MOE_API int moe_selftest_wait_timeout(void *workspace, size_t workspace_bytes, void *stream);
+
+/* Host-only, pure.  The largest number of token rows one GEMM tile of moe_forward_ex covers for this problem and
+ * these flags (32, 64, 128, 256, 320 or 384; 0 outside the envelope): experts with more rows are cut into evenly
+ * sized tiles.  Reporting only: results never depend on it beyond the fp32 summation order inside a tile. */
+MOE_API int moe_token_tile_rows(int T, int H, int I, int E, int top_k, unsigned flags);
 
 /* Number of kernels moe_forward_ex launches for this problem with these flags (0 when T == 0). */
 MOE_API int moe_forward_launch_count(int T, unsigned flags);

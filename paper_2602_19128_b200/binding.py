@@ -18,12 +18,14 @@ MOE_FLAG_NONE = 0
 MOE_FLAG_VALIDATION_GEMM = 1
 MOE_FLAG_SINGLE_CTA_GEMM = 2
 MOE_FLAG_TWO_SLAB_GEMM = 4
+MOE_FLAG_NARROW_TILES = 8
+MOE_FLAG_GATHER_IN_LOAD = 16
 
 EXPORTED = ["moe_workspace_bytes", "moe_workspace_layout", "moe_route_workspace_bytes", "moe_route", "moe_route_static",
             "moe_forward",
             "moe_forward_ex", "moe_forward_local", "moe_route_grouped", "moe_forward_grouped", "moe_forward_fp8w", "moe_mxfp8_workspace_bytes",
             "moe_mxfp8_workspace_layout", "moe_mxfp8_pack_scales", "moe_mxfp8_quantize_rows", "moe_forward_mxfp8", "moe_forward_mxfp8_host",
-            "moe_forward_staged", "moe_forward_host", "moe_last_status", "moe_selftest_wait_timeout", "moe_forward_launch_count", "moe_status_string"]
+            "moe_forward_staged", "moe_forward_host", "moe_last_status", "moe_selftest_wait_timeout", "moe_forward_launch_count", "moe_token_tile_rows", "moe_status_string"]
 
 
 class MoeError(RuntimeError):
@@ -115,6 +117,8 @@ def lib() -> ctypes.CDLL:
         L.moe_last_status.argtypes = [vp, vp]
         L.moe_forward_launch_count.restype = i
         L.moe_forward_launch_count.argtypes = [i, ctypes.c_uint]
+        L.moe_token_tile_rows.restype = i
+        L.moe_token_tile_rows.argtypes = [i] * 5 + [ctypes.c_uint]
         L.moe_status_string.restype = ctypes.c_char_p
         L.moe_status_string.argtypes = [i]
         _lib = L
@@ -156,6 +160,10 @@ def moe_workspace_layout(T: int, H: int, I: int, E: int, top_k: int) -> Workspac
 
 def moe_forward_launch_count(T: int, flags: int = 0) -> int:
     return int(lib().moe_forward_launch_count(T, flags))
+
+
+def moe_token_tile_rows(T: int, H: int, I: int, E: int, top_k: int, flags: int = 0) -> int:
+    return int(lib().moe_token_tile_rows(T, H, I, E, top_k, flags))
 
 
 def alloc_workspace(nbytes: int, device="cuda") -> torch.Tensor:

@@ -81,6 +81,14 @@ void fill_layout(int T, int H, int I, int E, int k, moe_workspace_layout_t *L) {
     L->total_bytes = off;
 }
 
+// Token-tile bound of the bf16 layer for this problem and these flags: the wide bounds (320 / 384) need the
+// wide-tile kernel for BOTH GEMMs (I a multiple of 128, H of 256) and none of the flags that pin another kernel.
+int layer_token_tile_bound(int T, int H, int I, int E, int k, unsigned flags, bool fp8w) {
+    const bool pinned = fp8w || (flags & (MOE_FLAG_SINGLE_CTA_GEMM | MOE_FLAG_TWO_SLAB_GEMM | MOE_FLAG_NARROW_TILES)) != 0;
+    const bool wide_ok = !pinned && I % 128 == 0 && H % 256 == 0;
+    return choose_nt_max(T, E, k, wide_ok);
+}
+
 int forward_impl(const void *x, const float *logits, const void *w13, const void *w2, int T, int H, int I, int E, int k,
                  void *out, void *workspace, size_t workspace_bytes, cudaStream_t stream, unsigned flags,
                  void *const *stage_events = nullptr, int local_offset = 0, int n_local = -1,
@@ -90,7 +98,9 @@ int forward_impl(const void *x, const float *logits, const void *w13, const void
     if (T < 0 || H <= 0 || I <= 0 || E <= 0 || k <= 0 || k > E) return MOE_ERR_SHAPE;
     if (!envelope_ok(T, H, I, E, k)) return MOE_ERR_UNSUPPORTED;
     if (local_offset < 0 || n_local < 1 || (long long)local_offset + n_local > E) return MOE_ERR_SHAPE;
-    if (flags & ~(MOE_FLAG_VALIDATION_GEMM | MOE_FLAG_SINGLE_CTA_GEMM | MOE_FLAG_TWO_SLAB_GEMM)) return MOE_ERR_UNSUPPORTED;
+    if (flags & ~(MOE_FLAG_VALIDATION_GEMM | MOE_FLAG_SINGLE_CTA_GEMM | MOE_FLAG_TWO_SLAB_GEMM | MOE_FLAG_NARROW_TILES |
+                  MOE_FLAG_GATHER_IN_LOAD))
+        return MOE_ERR_UNSUPPORTED;
     if (fp8w && (I % 128 != 0 || flags != MOE_FLAG_NONE)) return MOE_ERR_UNSUPPORTED;
     if (T == 0) return MOE_OK;
     if (!x || !logits || !w13 || !w2 || !out || !workspace || (fp8w && !w2_scale)) return MOE_ERR_NULL;
@@ -115,7 +125,7 @@ int forward_impl(const void *x, const float *logits, const void *w13, const void
     __nv_bfloat16 *h = reinterpret_cast<__nv_bfloat16 *>(ws + L.h);
     __nv_bfloat16 *y = reinterpret_cast<__nv_bfloat16 *>(ws + L.y);
     const int A = T * k;
-    const int nt_max = choose_nt_max(T, E, k);
+    const int nt_max = layer_token_tile_bound(T, H, I, E, k, flags, fp8w);
 
     auto mark = [&](int i) {
         return !stage_events || cudaEventRecord(static_cast<cudaEvent_t>(stage_events[i]), stream) == cudaSuccess;
@@ -125,7 +135,11 @@ int forward_impl(const void *x, const float *logits, const void *w13, const void
                      stream, 16, router, kStatusBytesForward) != cudaSuccess)
         return MOE_ERR_CUDA;
     if (!mark(1)) return MOE_ERR_CUDA;
-    if (launch_scatter_rows(static_cast<const __nv_bfloat16 *>(x), f2s, T, k, H, x_perm, stream) != cudaSuccess)
+    // Gather-in-load (opt-in): the wide-tile gate/up GEMM fetches token rows from x itself and x_perm is not written.
+    const bool gather_in_load = (flags & MOE_FLAG_GATHER_IN_LOAD) != 0 && (nt_max == 320 || nt_max == 384) &&
+                                !(flags & MOE_FLAG_VALIDATION_GEMM);
+    if (!gather_in_load &&
+        launch_scatter_rows(static_cast<const __nv_bfloat16 *>(x), f2s, T, k, H, x_perm, stream) != cudaSuccess)
         return MOE_ERR_CUDA;
     if (!mark(2)) return MOE_ERR_CUDA;
 
@@ -137,6 +151,12 @@ int forward_impl(const void *x, const float *logits, const void *w13, const void
     GroupedGemmArgs g2 = g1;
     g2.act = h; g2.w = static_cast<const __nv_bfloat16 *>(w2); g2.out = y;
     g2.K = I; g2.n_out = H; g2.w_rows = H; g2.swiglu = false;
+    if (gather_in_load) {
+        g1.gather_x = static_cast<const __nv_bfloat16 *>(x);
+        g1.gather_sorted_to_flat = s2f;
+        g1.gather_T = T;
+        g1.gather_top_k = k;
+    }
 
     if (fp8w) {
         g1.w_scale = w13_scale;
@@ -166,6 +186,7 @@ int forward_impl(const void *x, const float *logits, const void *w13, const void
             g2.handover_per_token_tile = handover_counts_per_token_tile(I);
         }
         auto run = [&](const GroupedGemmArgs &g, bool allow_two_slabs) {
+            if (!single && grouped_gemm_tc_ring_applies(g)) return launch_grouped_gemm_tc_ring(g, stream);
             int slabs = single ? 0 : grouped_gemm_tc_pair_slabs(g);
             if (slabs == 2 && !(dense_tiles && allow_two_slabs)) slabs = grouped_gemm_tc_pair_slabs(g) >= 1 ? 1 : 0;
             if (slabs == 2 || slabs == 1) {
@@ -548,6 +569,11 @@ int moe_last_status(const void *workspace, void *stream) {
     int status[moe::kStatusInts] = {0, 0, 0, 0};
     if (cudaMemcpy(status, workspace, sizeof(status), cudaMemcpyDeviceToHost) != cudaSuccess) return MOE_ERR_CUDA;
     return status[0];
+}
+
+int moe_token_tile_rows(int T, int H, int I, int E, int top_k, unsigned flags) {
+    if (!envelope_ok(T, H, I, E, top_k)) return 0;
+    return layer_token_tile_bound(T, H, I, E, top_k, flags, false);
 }
 
 int moe_forward_launch_count(int T, unsigned flags) {

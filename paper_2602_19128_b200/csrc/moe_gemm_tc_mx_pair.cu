@@ -61,7 +61,7 @@ struct MxPairSmem {
     static constexpr int kTmemSlot = kBars + (2 * STAGES + 4) * 8;
     static constexpr int kAbort = kTmemSlot + 4;
     static constexpr int kBytes = kAbort + 4;
-    static constexpr int kDynamicBytes = kBytes + 1024;
+    static constexpr int kDynamicBytes = kPairDynamicSmemBytes;  // (kBytes + 1024 of it are used)
 };
 
 template <int NT_MAX, int STAGES, bool SWIGLU>
@@ -270,16 +270,13 @@ grouped_gemm_tc_mx_pair_kernel(const __grid_constant__ MxPairMaps maps, const Mx
     if (*abort_flag) {
         for (int i = 0; i < 1000; ++i) __nanosleep(1000);
     }
-    if (warp == 1) {
-        tcgen05_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemColsMx) : "memory");
-    }
+    tmem_release_pair(tmem_base, kTmemColsMx, warp);
 }
 
 template <int NT_MAX, int STAGES, bool SWIGLU>
 int launch_pair_instance(const MxPairMaps &maps, const MxParams &p, int grid, cudaStream_t stream) {
     using L = MxPairSmem<NT_MAX, STAGES>;
-    static_assert(L::kDynamicBytes <= 232448, "ring does not fit in shared memory");
+    static_assert(L::kBytes + 1024 <= L::kDynamicBytes, "ring does not fit in shared memory");
     auto kernel = grouped_gemm_tc_mx_pair_kernel<NT_MAX, STAGES, SWIGLU>;
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) != cudaSuccess)
         return MOE_ERR_CUDA;

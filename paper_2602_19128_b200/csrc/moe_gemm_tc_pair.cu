@@ -53,7 +53,7 @@ struct PairSmem {
     static constexpr int kTmemSlot = kBars + (2 * STAGES + 4) * 8;
     static constexpr int kAbort = kTmemSlot + 4;
     static constexpr int kBytes = kAbort + 4;
-    static constexpr int kDynamicBytes = kBytes + 1024;
+    static constexpr int kDynamicBytes = kPairDynamicSmemBytes;  // (kBytes + 1024 of it are used)
 };
 
 // Drain one accumulator (this warp's 32 TMEM lanes x n_mma columns) to global memory.
@@ -142,6 +142,7 @@ grouped_gemm_tc_pair_kernel(const __grid_constant__ TensorMaps maps, const Kerne
     const bool started = gemm_chain_start(p.handover_role, p.handover, abort_flag, p.status);
     const int total_tiles = started ? p.tile_prefix[p.E] * p.n_feature_tiles : 0;
     const int n_pairs = gridDim.x >> 1, pair = blockIdx.x >> 1;
+    clock_probe_begin(p.status, SWIGLU ? 0 : 1);
 
     // ---------------- TMA producers (both CTAs) ----------------
     // The weight slabs and the token rows of a slot are issued by two different warps: a copy
@@ -283,19 +284,17 @@ grouped_gemm_tc_pair_kernel(const __grid_constant__ TensorMaps maps, const Kerne
     tcgen05_fence_before();
     __syncthreads();
     cluster_sync_all();
+    clock_probe_end(p.status, SWIGLU ? 0 : 1);
     if (*abort_flag) {
         for (int i = 0; i < 1000; ++i) __nanosleep(1000);
     }
-    if (warp == 1) {
-        tcgen05_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
-    }
+    tmem_release_pair(tmem_base, kTmemCols, warp);
 }
 
 template <int NT_MAX, int STAGES, int SLABS, bool SWIGLU>
 int launch_pair_instance(const TensorMaps &maps, const KernelParams &p, int grid, cudaStream_t stream) {
     using L = PairSmem<NT_MAX, STAGES, SLABS>;
-    static_assert(L::kDynamicBytes <= 232448, "ring does not fit in shared memory");
+    static_assert(L::kBytes + 1024 <= L::kDynamicBytes, "ring does not fit in shared memory");
     auto kernel = grouped_gemm_tc_pair_kernel<NT_MAX, STAGES, SLABS, SWIGLU>;
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) != cudaSuccess)
         return MOE_ERR_CUDA;

@@ -25,6 +25,7 @@ constexpr int kStatusBytesRoute = 256;
 constexpr int kStatusBytesForward = 2048;
 constexpr int kHandoverFlagInt = 8;
 constexpr int kReadyTotalInt = 9;       // all experts' counts together
+constexpr int kClockProbeInt = 32;      // 2 x 4 int64 (bytes 128..191): the GEMMs' clock probes (moe_tc_common.cuh)
 constexpr int kReadyCounterInt = 64;    // [kMaxExperts] ints from here
 // What one gate/up tile adds to its expert's counter: each of the 4 epilogue warps of each CTA counts once, and a
 // token tile is covered by I / 64 CTA-tiles of 64 features whichever kernel runs it.
@@ -157,6 +158,11 @@ struct GroupedGemmArgs {
     int handover_role = 0;
     int *handover = nullptr;            // the call's status region (flag and counters at the offsets above)
     int handover_per_token_tile = 0;    // role 2: counts that complete one token tile of an expert
+    // gather-in-load (wide-tile gate/up GEMM): when gather_x is set, `act` is unused and row r of the expert-contiguous
+    // order is row gather_sorted_to_flat[r] / gather_top_k of gather_x [gather_T, K]
+    const __nv_bfloat16 *gather_x = nullptr;
+    const int *gather_sorted_to_flat = nullptr;
+    int gather_T = 0, gather_top_k = 1;
 };
 int launch_grouped_gemm_tc(const GroupedGemmArgs &args, cudaStream_t stream);  // returns a moe_status_t
 
@@ -166,6 +172,11 @@ int launch_grouped_gemm_tc(const GroupedGemmArgs &args, cudaStream_t stream);  /
 // feature count the pair tile does not divide).
 int grouped_gemm_tc_pair_slabs(const GroupedGemmArgs &args);
 int launch_grouped_gemm_tc_pair(const GroupedGemmArgs &args, int slabs, cudaStream_t stream);
+
+// The same GEMM on CTA pairs with wide token tiles (bounds 320 and 384 rows): one pass over a weight slab per
+// expert of up to that many rows, accumulators in a ring of tensor-memory columns (moe_gemm_tc_ring.cu).
+bool grouped_gemm_tc_ring_applies(const GroupedGemmArgs &args);
+int launch_grouped_gemm_tc_ring(const GroupedGemmArgs &args, cudaStream_t stream);
 
 // The one-CTA kernel for FP8 (E4M3) block-scaled weights: args.w holds one code byte per weight and
 // args.w_scale one fp32 scale per 128 x 128 block; converter warps rebuild bf16 operand tiles in shared
@@ -238,7 +249,8 @@ cudaError_t launch_wait_timeout_selftest(int *status, cudaStream_t stream);
 // Same contract on plain CUDA cores (validation only).
 cudaError_t launch_grouped_gemm_validation(const GroupedGemmArgs &args, cudaStream_t stream);
 
-// Token-tile bound chosen from the average rows per expert.
-int choose_nt_max(int T, int E, int k);
+// Token-tile bound chosen from the average rows per expert: 32, 64, 128 or 256, and 320 / 384 (the wide-tile
+// kernel) when experts are expected to hold more than 256 rows.  `wide_ok` = false keeps the bound at 256.
+int choose_nt_max(int T, int E, int k, bool wide_ok = false);
 
 }  // namespace moe

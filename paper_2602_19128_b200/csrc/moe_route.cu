@@ -16,6 +16,7 @@
 #include "moe_internal.cuh"
 
 #include <limits.h>
+#include <math.h>
 
 #include <mutex>
 
@@ -341,11 +342,15 @@ __device__ __forceinline__ void scan_phase(int *chunk_counts, int n_chunks, int 
         counts[e] = e < E ? count : -1;
         tiles_at[e] = 0;
     }
-    // token tiles of this expert: as few as fit under nt_max, evenly sized, rounded up to the row quantum
+    // token tiles of this expert: one tile if it fits under nt_max; otherwise as few as fit under min(nt_max, 256) --
+    // a wide bound (320 / 384) exists to keep an expert in ONE pass over its weights, and consecutive tiles wider than
+    // half of tensor memory cannot overlap their epilogues, so experts that need several tiles get 256-row ones --
+    // evenly sized, rounded up to the row quantum
     // (16 rows, the MMA's N granularity; the MX path passes its tile size, so that every tile is exactly that many rows)
     int n_tiles = 0, rows = 0;
     if (count > 0) {
-        n_tiles = (count + nt_max - 1) / nt_max;
+        const int multi = nt_max > 256 ? 256 : nt_max;
+        n_tiles = count <= nt_max ? 1 : (count + multi - 1) / multi;
         rows = (((count + n_tiles - 1) / n_tiles) + row_quantum - 1) / row_quantum * row_quantum;
     }
     int total_rows, total_tiles;
@@ -570,12 +575,16 @@ combine_kernel(const uint4 *__restrict__ y, const float *__restrict__ topk_w, co
 
 }  // namespace
 
-int choose_nt_max(int T, int E, int k) {
+int choose_nt_max(int T, int E, int k, bool wide_ok) {
     const double avg = (double)T * k / E;
     const int options[3] = {32, 64, 128};
     for (int nt : options)
         if (1.5 * avg <= nt) return nt;
-    return 256;
+    // Between about 160 and 350 rows per expert on average, experts with 257..384 rows are common: a wide bound
+    // keeps each of them in one tile (320 while the mean plus 2.5 standard deviations of a uniform routing fits, else
+    // 384).  With more rows than that nearly every expert needs several tiles anyway, and those are 256-row tiles.
+    if (!wide_ok || avg <= 160.0 || avg > 352.0) return 256;
+    return avg + 2.5 * sqrt(avg) <= 320.0 ? 320 : 384;
 }
 
 cudaError_t launch_route(const float *logits, int T, int E, int k, LocalExperts local, int nt_max, int *topk_ids,

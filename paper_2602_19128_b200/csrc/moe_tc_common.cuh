@@ -35,6 +35,10 @@ struct KernelParams {
     int handover_role;     // hand-over between the two GEMMs of a call (moe_internal.cuh)
     int *handover;
     int handover_per_token_tile;
+    // gather-in-load (wide-tile gate/up GEMM only): token rows are fetched from the layer's input by row index
+    int gather_tokens = 0;
+    const int *sorted_to_flat = nullptr;
+    int top_k = 1;
 };
 
 // ---- PTX wrappers -----------------------------------------------------------------------------
@@ -283,6 +287,29 @@ __device__ __forceinline__ bool handover_wait_expert(int role, int *handover, in
     return ok;
 }
 
+// Clock probe: block 0 of a GEMM grid leaves its SM cycle counter and the global nanosecond timer, at the start of its
+// work and at its end, in the call's status region (kClockProbeInt, 4 x int64 per GEMM: cycles begin / end, ns begin /
+// end).  Their quotient is the clock the SM really ran at during THAT kernel, which a benchmark needs to tell a slow
+// kernel from a power-capped GPU; two stores per block-0 thread-0, nothing else.
+__device__ __forceinline__ void clock_probe_begin(int *status, int which) {
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        long long *slot = reinterpret_cast<long long *>(status + kClockProbeInt) + 4 * which;
+        unsigned long long ns;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ns));
+        slot[0] = clock64();
+        slot[2] = (long long)ns;
+    }
+}
+__device__ __forceinline__ void clock_probe_end(int *status, int which) {
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        long long *slot = reinterpret_cast<long long *>(status + kClockProbeInt) + 4 * which;
+        unsigned long long ns;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ns));
+        slot[1] = clock64();
+        slot[3] = (long long)ns;
+    }
+}
+
 // Static tile assignment: worker w of n_workers takes, in round i, tile i*n_workers + w on even rounds
 // and i*n_workers + (n_workers-1-w) on odd rounds.  With tiles ordered by decreasing cost this
 // back-and-forth deal keeps every worker's total within about 1 % of the mean, without atomics.
@@ -299,7 +326,8 @@ bool encode_weight_map_gate_up(CUtensorMap *map, const void *w13, int E, int I, 
 bool encode_weight_map_2d_fp8(CUtensorMap *map, const void *w, uint64_t rows, uint64_t K);
 bool encode_act_maps_k128(CUtensorMap *maps, const void *act, uint64_t rows, uint64_t K, int row_quantum);
 bool encode_weight_map_gate_up_fp8(CUtensorMap *map, const void *w13, int E, int I, int H);
-bool encode_act_maps(CUtensorMap *maps, const void *act, uint64_t rows, uint64_t K, int row_quantum);
+bool encode_act_maps(CUtensorMap *maps, const void *act, uint64_t rows, uint64_t K, int row_quantum, int count = kNumActMaps);
+bool encode_row_map(CUtensorMap *map, const void *act, uint64_t rows, uint64_t K);
 bool encode_mx_weight_map_2d(CUtensorMap *map, const void *w, uint64_t rows, uint64_t K);
 bool encode_mx_weight_map_gate_up(CUtensorMap *map, const void *w13, int E, int I, int H);
 bool encode_mx_act_maps(CUtensorMap *maps, const void *act, uint64_t rows, uint64_t K, int row_quantum);

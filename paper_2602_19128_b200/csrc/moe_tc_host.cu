@@ -185,11 +185,14 @@ bool encode_act_maps_k128(CUtensorMap *maps, const void *act, uint64_t rows, uin
     return true;
 }
 
-bool encode_act_maps(CUtensorMap *maps, const void *act, uint64_t rows, uint64_t K, int row_quantum) {
-    for (int i = 0; i < kNumActMaps; ++i)
+bool encode_act_maps(CUtensorMap *maps, const void *act, uint64_t rows, uint64_t K, int row_quantum, int count) {
+    for (int i = 0; i < count; ++i)
         if (!encode_2d(&maps[i], act, rows, K, (uint32_t)row_quantum * (uint32_t)(i + 1))) return false;
     return true;
 }
+
+// [rows, K] bf16 with a box of ONE row of 64 columns: the form TMA's four-row gather (tile::gather4) takes.
+bool encode_row_map(CUtensorMap *map, const void *act, uint64_t rows, uint64_t K) { return encode_2d(map, act, rows, K, 1); }
 
 // Scale atoms as a 2-D tensor of 32-bit words: [n_atoms][128 words], box = atoms_per_box whole atoms, unswizzled.
 bool encode_scale_atoms(CUtensorMap *map, const void *atoms, uint64_t n_atoms, uint32_t atoms_per_box) {

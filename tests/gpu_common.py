@@ -88,7 +88,7 @@ def check_guards(ws_guard: Guarded, out_guard: Guarded, layout, used: dict, what
     assert_gaps_untouched(ws_guard.inner, layout, used, what)
 
 
-def run_forward(inp: dict, flags: int = 0, poison: bool = True):
+def run_forward(inp: dict, flags: int = 0, poison: bool = True, x_perm_written: bool = True):
     """moe_forward on device tensors, workspace and result between guard bands.  Returns (out bf16 [T,H] on device,
     workspace views, workspace)."""
     x, logits, w13, w2, k = inp["x"], inp["router_logits"], inp["w13"], inp["w2"], inp["top_k"]
@@ -102,7 +102,10 @@ def run_forward(inp: dict, flags: int = 0, poison: bool = True):
     status = moe.moe_last_status(ws)
     assert status == moe.MOE_OK, moe.moe_status_string(status)
     if poison:
-        check_guards(wg, og, moe.moe_workspace_layout(T, H, I, E, k), layer_regions(T, H, I, E, k), "moe_forward")
+        regions = layer_regions(T, H, I, E, k)
+        if not x_perm_written:  # gather-in-load: the region must stay untouched as a whole
+            regions["x_perm"] = 0
+        check_guards(wg, og, moe.moe_workspace_layout(T, H, I, E, k), regions, "moe_forward")
     else:
         wg.assert_bands_intact("moe_forward workspace")
         og.assert_bands_intact("moe_forward out")

@@ -69,6 +69,19 @@ def test_status_strings_and_launch_count():
     assert moe.moe_forward_launch_count(1024) == 5 and moe.moe_forward_launch_count(1025) == 7
 
 
+def test_token_tile_bound_follows_the_mean_rows_per_expert():
+    assert moe.moe_token_tile_rows(16, 256, 512, 8, 2) == 32            # 4 rows per expert
+    assert moe.moe_token_tile_rows(128, 7168, 2048, 256, 8) == 32
+    assert moe.moe_token_tile_rows(512, 4096, 14336, 8, 2) == 256       # 128 rows per expert: experts fit 256
+    assert moe.moe_token_tile_rows(8192, 7168, 2048, 256, 8) == 320     # 256 on average: one wide tile per expert
+    assert moe.moe_token_tile_rows(4096, 4096, 1536, 128, 8) == 320
+    assert moe.moe_token_tile_rows(8192, 7168, 2048, 208, 8) == 384     # 315 on average
+    assert moe.moe_token_tile_rows(8192, 7168, 2048, 128, 8) == 256     # 512 on average: several tiles per expert anyway
+    assert moe.moe_token_tile_rows(8192, 7168, 2048, 256, 8, binding.MOE_FLAG_NARROW_TILES) == 256
+    assert moe.moe_token_tile_rows(8192, 7040, 2048, 256, 8) == 256     # H not a multiple of 256: no wide-tile kernel
+    assert moe.moe_token_tile_rows(8192, 7168, 2048, 300, 8) == 0       # outside the envelope
+
+
 def test_mx_layout():
     for cfg in [(16, 256, 512, 8, 2), (512, 4096, 14336, 8, 2), (128, 7168, 2048, 256, 8), (8192, 7168, 2048, 256, 8)]:
         n = moe.moe_mxfp8_workspace_bytes(*cfg)

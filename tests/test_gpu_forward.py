@@ -26,6 +26,10 @@ SMALL = [
     (130, 256, 128, 1, 1, False),     # one expert, 130 rows: pair tile with a nearly empty second half
     (700, 256, 256, 2, 1, False),     # ~350 rows per expert: two weight slabs per CTA in the gate/up GEMM
     (600, 512, 512, 2, 2, False),     # 600 rows per expert: three token tiles of 208, two 512-row pair tiles
+    (520, 256, 256, 4, 2, False),     # ~260 rows per expert: wide-tile kernel, one tile of up to 320 rows per expert
+    (900, 256, 128, 8, 2, True),      # skewed, 225 rows on average: bound 320, hot experts cut into 256-row tiles
+    (1200, 512, 384, 8, 2, False),    # 300 rows per expert: bound 384, consecutive tiles overlap in tensor memory
+    (2600, 256, 128, 16, 2, False),   # 325 rows per expert: bound 384 with the three-kernel router
 ]
 
 
@@ -40,8 +44,8 @@ def oracle_everything(case):
 
 
 @pytest.mark.parametrize("flags", [moe.MOE_FLAG_VALIDATION_GEMM, moe.MOE_FLAG_SINGLE_CTA_GEMM,
-                                   moe.MOE_FLAG_TWO_SLAB_GEMM, moe.MOE_FLAG_NONE],
-                         ids=["cuda_core", "tcgen05_single", "tcgen05_two_slab", "tcgen05"])
+                                   moe.MOE_FLAG_TWO_SLAB_GEMM, moe.MOE_FLAG_NARROW_TILES, moe.MOE_FLAG_NONE],
+                         ids=["cuda_core", "tcgen05_single", "tcgen05_two_slab", "tcgen05_narrow", "tcgen05"])
 @pytest.mark.parametrize("T,H,I,E,k,skew", SMALL)
 def test_forward_matches_oracle(T, H, I, E, k, skew, flags):
     inp = gpu_inputs(dict(T=T, H=H, I=I, E=E, top_k=k, skew=skew), seed=0)
@@ -53,6 +57,23 @@ def test_forward_matches_oracle(T, H, I, E, k, skew, flags):
     assert_close_out(bf16_to_f64(views["h"]), h, "h")
     assert_close_out(bf16_to_f64(views["y"]), y, "y")
     assert_close_out(bf16_to_f64(out), ref, "out")
+
+
+@pytest.mark.parametrize("T,H,I,E,k,skew", [(520, 256, 256, 4, 2, False), (900, 256, 128, 8, 2, True),
+                                            (1200, 512, 384, 8, 2, False), (700, 256, 256, 2, 1, False)])
+def test_gather_in_load_matches_oracle(T, H, I, E, k, skew):
+    """The wide-tile gate/up GEMM fetching token rows from x by index (no expert-contiguous copy): h, y and out
+    against the oracle, and bit-identical to the path that reads the copy (same operands, same order)."""
+    assert moe.moe_token_tile_rows(T, H, I, E, k) in (320, 384)
+    inp = gpu_inputs(dict(T=T, H=H, I=I, E=E, top_k=k, skew=skew), seed=0)
+    out, views, _ = run_forward(inp, flags=moe.MOE_FLAG_GATHER_IN_LOAD, x_perm_written=False)
+    ids, w, off, s2f, f2s, h, y, ref = oracle_everything(to_host_case(inp))
+    assert_routing_exact(views, ids, w, off, s2f, f2s)
+    assert_close_out(bf16_to_f64(views["h"]), h, "h")
+    assert_close_out(bf16_to_f64(views["y"]), y, "y")
+    assert_close_out(bf16_to_f64(out), ref, "out")
+    plain, _, _ = run_forward(inp)
+    assert torch.equal(out.view(torch.int16), plain.view(torch.int16))
 
 
 def test_forward_is_deterministic_and_leaves_inputs_alone():

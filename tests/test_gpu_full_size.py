@@ -19,12 +19,6 @@ from tests.gpu_common import (OUT_TOL, Guarded, assert_close_out, assert_routing
 pytestmark = pytest.mark.gpu
 
 
-def token_tile_bound(T: int, E: int, k: int) -> int:
-    """The bf16 layer's token-tile bound (the library's rule: the smallest of 32, 64, 128 that holds 1.5 x the mean
-    rows per expert, else 256)."""
-    return next((nt for nt in (32, 64, 128) if 1.5 * T * k / E <= nt), 256)
-
-
 def edge_tokens(off: np.ndarray, s2f: np.ndarray, T: int, E: int, k: int, tile_bound: int) -> np.ndarray:
     """Tokens the oracle evaluates one by one, chosen from ITS permutation so that they sit where an indexing
     mistake would show: the first and last row of the heaviest expert, the rows on both sides of that expert's
@@ -36,7 +30,7 @@ def edge_tokens(off: np.ndarray, s2f: np.ndarray, T: int, E: int, k: int, tile_b
     heavy = int(np.argmax(counts))
     b, c = int(off[heavy]), int(counts[heavy])
     rows += [b, b + c - 1, max(b - 1, 0), min(b + c, len(s2f) - 1)]
-    n_tiles = -(-c // tile_bound)
+    n_tiles = 1 if c <= tile_bound else -(-c // min(tile_bound, 256))
     if n_tiles > 1:
         per = -(-(-(-c // n_tiles)) // 16) * 16
         rows += [b + per - 1, b + per]
@@ -74,7 +68,7 @@ def test_full_size_workload(name):
                        inp["x"][views["sorted_to_flat"].long() // k].view(torch.int16))
 
     # 2. sampled tokens against the oracle: tile and segment edges, 64-bit weight offsets, and a seeded draw
-    tokens = edge_tokens(off, s2f, T, E, k, token_tile_bound(T, E, k))
+    tokens = edge_tokens(off, s2f, T, E, k, moe.moe_token_tile_rows(T, H, I, E, k))
     assert 8 <= len(tokens) <= 16
     need = sorted({int(e) for t in tokens for e in ids[t]})
     experts = {e: (bf16_bits(inp["w13"][e]), bf16_bits(inp["w2"][e])) for e in need}

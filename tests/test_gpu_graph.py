@@ -227,3 +227,41 @@ def test_two_host_threads_calling_concurrently_with_their_own_workspaces():
     assert not errors, errors
     for out, r in zip(outs, refs):
         assert torch.equal(out.view(torch.int16), r.view(torch.int16))
+
+
+_OVERLAP = r"""
+import sys, torch
+sys.path.insert(0, {root!r})
+import paper_2602_19128_b200 as moe
+from paper_2602_19128_b200.inputs import make_inputs
+cfg = dict(T={T}, H={H}, I={I}, E={E}, top_k={k}, skew=False)
+inp = make_inputs(cfg, seed=70, device="cuda")
+ws = [moe.alloc_workspace(moe.moe_workspace_bytes({T}, {H}, {I}, {E}, {k}), "cuda") for _ in range(2)]
+outs = [torch.empty(({T}, {H}), dtype=torch.bfloat16, device="cuda") for _ in range(3)]
+moe.moe_forward(inp["x"], inp["router_logits"], inp["w13"], inp["w2"], {k}, outs[2], ws[0])
+torch.cuda.synchronize()
+streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+for it in range({groups}):
+    for i in range(20):   # deep queues on both streams: the calls' kernels overlap in every phase combination
+        moe.moe_forward(inp["x"], inp["router_logits"], inp["w13"], inp["w2"], {k}, outs[i % 2], ws[i % 2], stream=streams[i % 2])
+    torch.cuda.synchronize()
+for i in range(2):
+    assert moe.moe_last_status(ws[i], stream=streams[i]) == 0
+    assert torch.equal(outs[i].view(torch.int16), outs[2].view(torch.int16))
+print("overlap ok")
+"""
+
+
+@pytest.mark.parametrize("T,H,I,E,k", [(2048, 512, 256, 256, 8),    # 128-row CTA-pair kernel, three-kernel router
+                                       (2048, 512, 256, 64, 8)])    # wide-tile kernel, three-kernel router
+def test_many_overlapping_calls_on_two_streams_complete(T, H, I, E, k):
+    """Thousands of calls queued twenty deep on two streams, so that every kernel of one call meets every kernel of
+    the other on the SMs.  CTA-pair kernels take a whole SM's shared memory for themselves; before they did, small
+    blocks of the other stream's sort-scatter shared their SMs and, about once per thousand calls, a later pair waited
+    for tensor memory for ever.  Run in a child process with a time limit so that a regression ends as a failure."""
+    import subprocess
+    import sys
+    from pathlib import Path
+    src = _OVERLAP.format(root=str(Path(__file__).resolve().parent.parent), T=T, H=H, I=I, E=E, k=k, groups=150)
+    r = subprocess.run([sys.executable, "-c", src], capture_output=True, text=True, timeout=240)
+    assert r.returncode == 0 and "overlap ok" in r.stdout, r.stderr[-2000:]
