@@ -414,7 +414,7 @@ def measure(ctx: Ctx, name: str, inp: dict, steps, warmup: int, with_e2e: bool, 
         forward()
     n_warm = max(n_warm, 6)
     if steps is None:
-        steps = int(min(max(20, math.ceil(min_timed_s * 1e3 / est_ms)), 2000))
+        steps = args.steps if args.few_launches else int(min(max(20, math.ceil(min_timed_s * 1e3 / est_ms)), 2000))
 
     # ---- device-resident timing ----------------------------------------------------------------
     # The K timed steps run as a user's would: no event between the kernels of a step (an event record between two

@@ -126,16 +126,23 @@ def lib() -> ctypes.CDLL:
 
 
 def _ptr(t):
+    """The address of a contiguous tensor (an int: ctypes converts it for a void* parameter)."""
     if t is None:
         return None
     assert t.is_contiguous(), "tensors must be contiguous"
-    return ctypes.c_void_p(t.data_ptr())
+    return t.data_ptr()
 
 
-def _stream(stream) -> ctypes.c_void_p:
-    if stream is None:
-        stream = torch.cuda.current_stream()
-    return ctypes.c_void_p(stream.cuda_stream)
+_raw_stream = getattr(torch._C, "_cuda_getCurrentRawStream", None)
+
+
+def _stream(stream):
+    """The cudaStream_t to launch on: the given torch stream, else the current stream of the current device."""
+    if stream is not None:
+        return stream.cuda_stream
+    if _raw_stream is not None:
+        return _raw_stream(torch.cuda.current_device())
+    return torch.cuda.current_stream().cuda_stream
 
 
 def moe_status_string(status: int) -> str:

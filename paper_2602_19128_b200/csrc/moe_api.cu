@@ -8,9 +8,12 @@
 namespace moe {
 
 int check_device() {
+    static int verdict[64];  // per device: 0 not asked yet, 1 compute capability 10.x, 2 anything else
     int dev = 0, major = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return MOE_ERR_CUDA;
+    if (dev >= 0 && dev < 64 && verdict[dev]) return verdict[dev] == 1 ? MOE_OK : MOE_ERR_ARCH;
     if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return MOE_ERR_CUDA;
+    if (dev >= 0 && dev < 64) verdict[dev] = major == 10 ? 1 : 2;
     return major == 10 ? MOE_OK : MOE_ERR_ARCH;
 }
 

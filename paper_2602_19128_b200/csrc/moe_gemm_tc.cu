@@ -238,8 +238,7 @@ int launch_instance(const TensorMaps &maps, const KernelParams &p, int grid, cud
     using L = SmemLayout<NT_MAX, STAGES>;
     static_assert(L::kDynamicBytes <= 232448, "ring does not fit in shared memory");
     auto kernel = grouped_gemm_tc_kernel<NT_MAX, STAGES, SWIGLU>;
-    // per device and cheap, so set on every launch rather than cached per process
-    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) != cudaSuccess)
+    if (!set_max_dynamic_smem_once(reinterpret_cast<const void *>(kernel), L::kDynamicBytes))
         return MOE_ERR_CUDA;
     return launch_chained(kernel, grid, kThreads, L::kDynamicBytes, stream, maps, p) == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }

@@ -325,7 +325,7 @@ int launch_fp8_instance(const TensorMaps &maps, const KernelParams &p, int grid,
     using L = Fp8Smem<NT_MAX, STAGES, CONV>;
     static_assert(L::kDynamicBytes <= 232448, "rings do not fit in shared memory");
     auto kernel = grouped_gemm_tc_fp8w_kernel<NT_MAX, STAGES, CONV, SWIGLU>;
-    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) != cudaSuccess)
+    if (!set_max_dynamic_smem_once(reinterpret_cast<const void *>(kernel), L::kDynamicBytes))
         return MOE_ERR_CUDA;
     return launch_chained(kernel, grid, kFp8Threads, L::kDynamicBytes, stream, maps, p) == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }

@@ -249,7 +249,7 @@ int launch_instance(const TensorMaps &maps, const MxParams &p, int grid, cudaStr
     using L = MxSmem<NT_MAX, STAGES>;
     static_assert(L::kDynamicBytes <= 232448, "ring does not fit in shared memory");
     auto kernel = grouped_gemm_tc_mx_kernel<NT_MAX, STAGES, SWIGLU>;
-    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) != cudaSuccess)
+    if (!set_max_dynamic_smem_once(reinterpret_cast<const void *>(kernel), L::kDynamicBytes))
         return MOE_ERR_CUDA;
     return launch_chained(kernel, grid, kThreads, L::kDynamicBytes, stream, maps, p) == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }

@@ -278,7 +278,7 @@ int launch_pair_instance(const MxPairMaps &maps, const MxParams &p, int grid, cu
     using L = MxPairSmem<NT_MAX, STAGES>;
     static_assert(L::kBytes + 1024 <= L::kDynamicBytes, "ring does not fit in shared memory");
     auto kernel = grouped_gemm_tc_mx_pair_kernel<NT_MAX, STAGES, SWIGLU>;
-    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) != cudaSuccess)
+    if (!set_max_dynamic_smem_once(reinterpret_cast<const void *>(kernel), L::kDynamicBytes))
         return MOE_ERR_CUDA;
     return launch_chained(kernel, grid, kPairThreads, L::kDynamicBytes, stream, maps, p) == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }

@@ -296,7 +296,7 @@ int launch_pair_instance(const TensorMaps &maps, const KernelParams &p, int grid
     using L = PairSmem<NT_MAX, STAGES, SLABS>;
     static_assert(L::kBytes + 1024 <= L::kDynamicBytes, "ring does not fit in shared memory");
     auto kernel = grouped_gemm_tc_pair_kernel<NT_MAX, STAGES, SLABS, SWIGLU>;
-    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) != cudaSuccess)
+    if (!set_max_dynamic_smem_once(reinterpret_cast<const void *>(kernel), L::kDynamicBytes))
         return MOE_ERR_CUDA;
     return launch_chained(kernel, grid, kPairThreads, L::kDynamicBytes, stream, maps, p) == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }

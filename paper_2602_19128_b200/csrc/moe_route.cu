@@ -526,51 +526,52 @@ scatter_rows_kernel(const uint4 *__restrict__ x, const int *__restrict__ flat_to
     }
 }
 
-__global__ void __launch_bounds__(256)
+// One thread per 16-byte column of one token: the up to eight rows of a batch are fetched together (eight independent
+// 16-byte loads in flight per thread), then added one rank after the other, so the summation order is fixed.
+constexpr int kCombineThreads = 128, kCombineBatch = 8;
+__global__ void __launch_bounds__(kCombineThreads)
 combine_kernel(const uint4 *__restrict__ y, const float *__restrict__ topk_w, const int *__restrict__ flat_to_sorted,
-               int k, int vec_per_row, uint4 *__restrict__ out) {
+               int k, int vec_per_row, int blocks_per_token, uint4 *__restrict__ out) {
     __shared__ int rows[kMaxTopK];
     __shared__ float weights[kMaxTopK];
     chain_release();
     chain_wait();
-    const int t = blockIdx.x;
+    const int t = blockIdx.x / blocks_per_token;
+    const int i = (blockIdx.x - t * blocks_per_token) * kCombineThreads + threadIdx.x;
     if (threadIdx.x < k) {
         rows[threadIdx.x] = flat_to_sorted[(size_t)t * k + threadIdx.x];
         weights[threadIdx.x] = topk_w[(size_t)t * k + threadIdx.x];
     }
     __syncthreads();
-    for (int i = threadIdx.x; i < vec_per_row; i += 256) {
-        float acc[8];
+    if (i >= vec_per_row) return;
+    float acc[8];
 #pragma unroll
-        for (int c = 0; c < 8; ++c) acc[c] = 0.f;
-        // ascending rank: the summation order is fixed.  Four rows are fetched before the first is used (the
-        // loop is a chain of memory round trips otherwise); the additions still happen one rank after the other.
-        for (int j0 = 0; j0 < k; j0 += 4) {
-            uint4 v[4];
+    for (int c = 0; c < 8; ++c) acc[c] = 0.f;
+    for (int j0 = 0; j0 < k; j0 += kCombineBatch) {
+        uint4 v[kCombineBatch];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const bool live = j0 + u < k && rows[j0 + u] >= 0;  // rank exists and its expert is resident here
-                v[u] = live ? __ldcs(&y[(size_t)rows[j0 + u] * vec_per_row + i]) : make_uint4(0, 0, 0, 0);
-            }
+        for (int u = 0; u < kCombineBatch; ++u) {
+            const bool live = j0 + u < k && rows[j0 + u] >= 0;  // rank exists and its expert is resident here
+            v[u] = live ? __ldcs(&y[(size_t)rows[j0 + u] * vec_per_row + i]) : make_uint4(0, 0, 0, 0);
+        }
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                if (j0 + u >= k || rows[j0 + u] < 0) continue;  // contributes nothing (not even a signed zero)
-                const float wj = weights[j0 + u];
-                const __nv_bfloat162 *h2 = reinterpret_cast<const __nv_bfloat162 *>(&v[u]);
+        for (int u = 0; u < kCombineBatch; ++u) {  // ascending rank
+            if (j0 + u >= k || rows[j0 + u] < 0) continue;  // contributes nothing (not even a signed zero)
+            const float wj = weights[j0 + u];
+            const __nv_bfloat162 *h2 = reinterpret_cast<const __nv_bfloat162 *>(&v[u]);
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    const float2 f = __bfloat1622float2(h2[c]);
-                    acc[2 * c] = fmaf(wj, f.x, acc[2 * c]);
-                    acc[2 * c + 1] = fmaf(wj, f.y, acc[2 * c + 1]);
-                }
+            for (int c = 0; c < 4; ++c) {
+                const float2 f = __bfloat1622float2(h2[c]);
+                acc[2 * c] = fmaf(wj, f.x, acc[2 * c]);
+                acc[2 * c + 1] = fmaf(wj, f.y, acc[2 * c + 1]);
             }
         }
-        uint4 o;
-        __nv_bfloat162 *o2 = reinterpret_cast<__nv_bfloat162 *>(&o);
-#pragma unroll
-        for (int c = 0; c < 4; ++c) o2[c] = __floats2bfloat162_rn(acc[2 * c], acc[2 * c + 1]);
-        out[(size_t)t * vec_per_row + i] = o;
     }
+    uint4 o;
+    __nv_bfloat162 *o2 = reinterpret_cast<__nv_bfloat162 *>(&o);
+#pragma unroll
+    for (int c = 0; c < 4; ++c) o2[c] = __floats2bfloat162_rn(acc[2 * c], acc[2 * c + 1]);
+    out[(size_t)t * vec_per_row + i] = o;
 }
 
 }  // namespace
@@ -629,8 +630,10 @@ cudaError_t launch_scatter_rows(const __nv_bfloat16 *x, const int *flat_to_sorte
 
 cudaError_t launch_combine(const __nv_bfloat16 *y, const float *topk_w, const int *flat_to_sorted, int T, int k,
                            int H, __nv_bfloat16 *out, cudaStream_t stream) {
-    return launch_chained(combine_kernel, T, 256, 0, stream, reinterpret_cast<const uint4 *>(y), topk_w, flat_to_sorted, k,
-                          H / 8, reinterpret_cast<uint4 *>(out));
+    const int vec_per_row = H / 8, blocks_per_token = (vec_per_row + kCombineThreads - 1) / kCombineThreads;
+    return launch_chained(combine_kernel, (unsigned)((long long)T * blocks_per_token), kCombineThreads, 0, stream,
+                          reinterpret_cast<const uint4 *>(y), topk_w, flat_to_sorted, k, vec_per_row, blocks_per_token,
+                          reinterpret_cast<uint4 *>(out));
 }
 
 }  // namespace moe

@@ -332,6 +332,7 @@ bool encode_mx_weight_map_2d(CUtensorMap *map, const void *w, uint64_t rows, uin
 bool encode_mx_weight_map_gate_up(CUtensorMap *map, const void *w13, int E, int I, int H);
 bool encode_mx_act_maps(CUtensorMap *maps, const void *act, uint64_t rows, uint64_t K, int row_quantum);
 int sm_count();
+bool set_max_dynamic_smem_once(const void *kernel, int bytes);
 
 }  // namespace tc
 }  // namespace moe

@@ -51,10 +51,15 @@ constexpr int kCacheSlots = 1024, kCacheProbe = 8;
 std::mutex g_cache_mutex;
 CacheSlot *g_cache = nullptr;  // allocated on first use (host memory), never freed
 
-uint64_t key_hash(const EncodeKey &k) {
-    const unsigned char *b = reinterpret_cast<const unsigned char *>(&k);
-    uint64_t h = 1469598103934665603ull;
-    for (size_t i = 0; i < sizeof(EncodeKey); ++i) h = (h ^ b[i]) * 1099511628211ull;
+static_assert(sizeof(EncodeKey) % 8 == 0, "the key is hashed and compared as 64-bit words");
+uint64_t key_hash(const EncodeKey &k) {  // word-wise multiply-xorshift: a few nanoseconds for the 14 words of a key
+    uint64_t words[sizeof(EncodeKey) / 8];
+    memcpy(words, &k, sizeof(EncodeKey));
+    uint64_t h = 0x9e3779b97f4a7c15ull;
+    for (size_t i = 0; i < sizeof(EncodeKey) / 8; ++i) {
+        h = (h ^ words[i]) * 0xff51afd7ed558ccdull;
+        h ^= h >> 29;
+    }
     return h;
 }
 
@@ -200,6 +205,25 @@ bool encode_scale_atoms(CUtensorMap *map, const void *atoms, uint64_t n_atoms, u
     const cuuint64_t strides[1] = {kMxSfAtomBytes};
     const cuuint32_t box[2] = {kMxSfAtomBytes / 4, atoms_per_box};
     return encode_cached(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, atoms, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE);
+}
+
+// cudaFuncSetAttribute(MaxDynamicSharedMemorySize) once per kernel and device instead of once per launch (it is a
+// driver call on the host path of every forward call otherwise).  A small table under the cache's mutex.
+bool set_max_dynamic_smem_once(const void *kernel, int bytes) {
+    struct Entry { const void *kernel; unsigned long long devices; };
+    static Entry table[64];
+    static int used = 0;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
+    std::lock_guard<std::mutex> lock(g_cache_mutex);
+    Entry *e = nullptr;
+    for (int i = 0; i < used; ++i)
+        if (table[i].kernel == kernel) { e = &table[i]; break; }
+    if (e && ((e->devices >> dev) & 1ull)) return true;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return false;
+    if (!e && used < 64) { e = &table[used++]; e->kernel = kernel; e->devices = 0; }
+    if (e) e->devices |= 1ull << dev;
+    return true;
 }
 
 int sm_count() {
