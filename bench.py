@@ -59,8 +59,12 @@ BOUND = {"tiny": "hbm", "mixtral": "hbm", "dsv3_decode": "hbm", "dsv3_prefill": 
 # entry names the kernel instance and the commit it was captured on; `scale` multiplies a capture of a smaller
 # case of the same per-expert shape up to the units (experts) of a full launch.
 NCU_TRAFFIC = {
-    "mixtral": dict(bytes=1928438528, scale=1, kernel="grouped_gemm_tc_pair_kernel<256,7,1,swiglu>", commit="7375983",
+    "mixtral": dict(bytes=1928651520, scale=1, kernel="grouped_gemm_tc_pair_kernel<256,7,1,swiglu>", commit="b010af5",
                     source="profiles/grouped_gemm_tc_pair_mixtral.md"),
+    "dsv3_prefill": dict(bytes=2055034880, scale=8, kernel="grouped_gemm_tc_ring_kernel<320,6,swiglu>", commit="b010af5",
+                         source="profiles/grouped_gemm_tc_ring_dsv3_prefill.md",
+                         note="captured on T=1024, E=32, top_k=8 (the headline's per-expert shape with an eighth of "
+                              "its experts); traffic grows with the number of experts"),
 }
 
 
