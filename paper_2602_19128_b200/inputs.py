@@ -92,3 +92,48 @@ def bf16_bits(t: torch.Tensor) -> np.ndarray:
 def bits_to_f64(bits: np.ndarray) -> np.ndarray:
     """Widen bf16 bit patterns exactly to float64."""
     return (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+# ---- second workload: one decode step of grouped-query attention over a paged key-value cache -----------------
+# (paper, Table 2 and Sec. 4.6: "GQA Paged Decode", model context Qwen3-30B-A3B: 32 query heads, 4 key-value heads,
+# head dimension 128.)  Seeded stand-ins for the serving traces the paper measured on: a batch of sequences whose
+# cached lengths are drawn uniformly from [len_lo, len_hi], their pages scattered over the physical cache by a random
+# permutation, queries and cache contents N(0,1) rounded to bf16.
+GQA_CONFIGS = {
+    # name: batch, query heads, kv heads, head dim, page size, cached-length range
+    "gqa_tiny": dict(B=3, Hq=8, Hkv=2, D=128, page_size=4, len_lo=1, len_hi=70),
+    "gqa_decode_b64": dict(B=64, Hq=32, Hkv=4, D=128, page_size=16, len_lo=1024, len_hi=8192),
+    "gqa_decode_b1_long": dict(B=1, Hq=32, Hkv=4, D=128, page_size=16, len_lo=65536, len_hi=65536),
+    "gqa_decode_b256": dict(B=256, Hq=32, Hkv=4, D=128, page_size=16, len_lo=256, len_hi=2048),
+}
+
+
+def make_gqa_inputs(cfg, seed: int = 0, device="cpu", spare_pages: int = 7) -> dict:
+    """Draw one paged-decode workload.  ``cfg`` is a name in GQA_CONFIGS or a dict with the same keys (an explicit
+    ``lengths`` list overrides the drawn lengths).  Returns q [B,Hq,D] bf16, k_cache / v_cache [num_pages,P,Hkv,D]
+    bf16, kv_indptr [B+1] / kv_indices / kv_last_page_len [B] int32 (all on ``device``), kv_len (a host list) and
+    sm_scale = D ** -0.5."""
+    if isinstance(cfg, str):
+        cfg = GQA_CONFIGS[cfg]
+    B, Hq, Hkv, D, P = cfg["B"], cfg["Hq"], cfg["Hkv"], cfg["D"], cfg["page_size"]
+    device = torch.device(device)
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(seed)
+    if "lengths" in cfg:
+        lengths = [int(v) for v in cfg["lengths"]]
+    else:
+        lengths = torch.randint(cfg["len_lo"], cfg["len_hi"] + 1, (B,), generator=gen).tolist()
+    pages = [(n + P - 1) // P for n in lengths]
+    num_pages = sum(pages) + spare_pages
+    perm = torch.randperm(num_pages, generator=gen)[:sum(pages)].to(torch.int32)
+    indptr = torch.zeros(B + 1, dtype=torch.int32)
+    indptr[1:] = torch.cumsum(torch.tensor(pages, dtype=torch.int64), 0).to(torch.int32)
+    last = torch.tensor([(n - 1) % P + 1 if n > 0 else 0 for n in lengths], dtype=torch.int32)
+    dgen = torch.Generator(device=device)
+    dgen.manual_seed(seed + 1)
+    q = _normal_bf16((B, Hq, D), 1.0, dgen, device)
+    k_cache = _normal_bf16((num_pages, P, Hkv, D), 1.0, dgen, device)
+    v_cache = _normal_bf16((num_pages, P, Hkv, D), 1.0, dgen, device)
+    return dict(q=q, k_cache=k_cache, v_cache=v_cache, kv_indptr=indptr.to(device), kv_indices=perm.to(device),
+                kv_last_page_len=last.to(device), kv_len=lengths, sm_scale=float(D) ** -0.5, B=B, Hq=Hq, Hkv=Hkv, D=D,
+                page_size=P, num_pages=num_pages)
