@@ -25,7 +25,8 @@ EXPORTED = ["moe_workspace_bytes", "moe_workspace_layout", "moe_route_workspace_
             "moe_forward",
             "moe_forward_ex", "moe_forward_local", "moe_route_grouped", "moe_forward_grouped", "moe_forward_fp8w", "moe_mxfp8_workspace_bytes",
             "moe_mxfp8_workspace_layout", "moe_mxfp8_pack_scales", "moe_mxfp8_quantize_rows", "moe_forward_mxfp8", "moe_forward_mxfp8_host",
-            "moe_forward_staged", "moe_forward_host", "moe_last_status", "moe_selftest_wait_timeout", "moe_forward_launch_count", "moe_token_tile_rows", "moe_status_string"]
+            "moe_forward_staged", "moe_forward_host", "moe_last_status", "moe_selftest_wait_timeout", "moe_forward_launch_count", "moe_token_tile_rows", "moe_status_string",
+            "gqa_decode_workspace_bytes", "gqa_paged_decode", "gqa_decode_split_tokens"]
 
 
 class MoeError(RuntimeError):
@@ -119,6 +120,12 @@ def lib() -> ctypes.CDLL:
         L.moe_forward_launch_count.argtypes = [i, ctypes.c_uint]
         L.moe_token_tile_rows.restype = i
         L.moe_token_tile_rows.argtypes = [i] * 5 + [ctypes.c_uint]
+        L.gqa_decode_workspace_bytes.restype = sz
+        L.gqa_decode_workspace_bytes.argtypes = [i] * 5
+        L.gqa_decode_split_tokens.restype = i
+        L.gqa_decode_split_tokens.argtypes = [i] * 5
+        L.gqa_paged_decode.restype = i
+        L.gqa_paged_decode.argtypes = [vp] * 6 + [i] * 7 + [ctypes.c_float, vp, vp, vp, sz, vp]
         L.moe_status_string.restype = ctypes.c_char_p
         L.moe_status_string.argtypes = [i]
         _lib = L
@@ -437,3 +444,26 @@ def workspace_views(workspace: torch.Tensor, T: int, H: int, I: int, E: int, top
         h=view(L.h, A * I * 2, torch.bfloat16, (A, I)),
         y=view(L.y, A * H * 2, torch.bfloat16, (A, H)),
     )
+
+
+# ---- second workload: paged grouped-query decode attention (include/gqa_decode.h) -------------------------------
+def gqa_decode_workspace_bytes(B: int, Hq: int, Hkv: int, D: int, max_kv_len: int) -> int:
+    return int(lib().gqa_decode_workspace_bytes(B, Hq, Hkv, D, max_kv_len))
+
+
+def gqa_decode_split_tokens(B: int, Hq: int, Hkv: int, D: int, max_kv_len: int) -> int:
+    return int(lib().gqa_decode_split_tokens(B, Hq, Hkv, D, max_kv_len))
+
+
+def gqa_paged_decode(q, k_cache, v_cache, kv_indptr, kv_indices, kv_last_page_len, max_kv_len: int, sm_scale: float, out,
+                     workspace, lse=None, stream=None, check: bool = True) -> int:
+    """One decode step: q [B,Hq,D] bf16, caches [num_pages,page_size,Hkv,D] bf16, int32 page tables, out [B,Hq,D]
+    bf16, lse [B,Hq] f32 or None.  Marshalling only."""
+    B, Hq, D = q.shape
+    num_pages, page_size, Hkv, _ = k_cache.shape
+    st = lib().gqa_paged_decode(_ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(kv_indptr), _ptr(kv_indices),
+                                _ptr(kv_last_page_len), B, Hq, Hkv, D, page_size, num_pages, int(max_kv_len),
+                                float(sm_scale), _ptr(out), _ptr(lse), _ptr(workspace), workspace.numel(), _stream(stream))
+    if check and st != MOE_OK:
+        raise MoeError(st, "gqa_paged_decode")
+    return st

@@ -13,7 +13,7 @@ PKG = Path(__file__).resolve().parent
 ROOT = PKG.parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libmoe_b200.so"
-SOURCES = ["moe_api.cu", "moe_route.cu", "moe_gemm_tc.cu", "moe_gemm_tc_pair.cu", "moe_gemm_tc_ring.cu", "moe_gemm_tc_fp8w.cu", "moe_gemm_tc_mx.cu", "moe_gemm_tc_mx_pair.cu", "moe_mx.cu", "moe_tc_host.cu", "moe_gemm_validation.cu"]
+SOURCES = ["moe_api.cu", "moe_route.cu", "moe_gemm_tc.cu", "moe_gemm_tc_pair.cu", "moe_gemm_tc_ring.cu", "moe_gemm_tc_fp8w.cu", "moe_gemm_tc_mx.cu", "moe_gemm_tc_mx_pair.cu", "moe_mx.cu", "moe_tc_host.cu", "moe_gemm_validation.cu", "gqa_decode.cu"]
 
 
 def _nvcc() -> str:
@@ -26,7 +26,7 @@ def _nvcc() -> str:
 def needs_build() -> bool:
     if not LIB.exists():
         return True
-    deps = [CSRC / s for s in SOURCES] + list(CSRC.glob("*.cuh")) + [ROOT / "include" / "moe.h"]
+    deps = [CSRC / s for s in SOURCES] + list(CSRC.glob("*.cuh")) + [ROOT / "include" / "moe.h", ROOT / "include" / "gqa_decode.h"]
     return any(d.stat().st_mtime > LIB.stat().st_mtime for d in deps)
 
 

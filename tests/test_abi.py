@@ -14,8 +14,8 @@ ROOT = Path(__file__).resolve().parent.parent
 
 
 def declared_symbols():
-    text = (ROOT / "include" / "moe.h").read_text()
-    return sorted(set(re.findall(r"MOE_API[^;(]*?\b(moe_[a-z0-9_]+)\s*\(", text)))
+    text = (ROOT / "include" / "moe.h").read_text() + (ROOT / "include" / "gqa_decode.h").read_text()
+    return sorted(set(re.findall(r"MOE_API[^;(]*?\b((?:moe|gqa)_[a-z0-9_]+)\s*\(", text)))
 
 
 def test_library_builds_loads_and_exports_every_declared_symbol():
@@ -34,7 +34,7 @@ def test_header_stands_alone_in_c_and_cxx(tmp_path, compiler, std, suffix):
     torch header on the include path, and a caller must be able to take the address of every entry point."""
     src = tmp_path / ("use_header" + suffix)
     body = "".join(f"    p[{i}] = (const void *)&{n};\n" for i, n in enumerate(declared_symbols()))
-    src.write_text('#include "moe.h"\n#include "moe.h"\n'  # twice: the include guard holds
+    src.write_text('#include "moe.h"\n#include "gqa_decode.h"\n#include "moe.h"\n#include "gqa_decode.h"\n'  # twice: the include guards hold
                    f"const void *p[{len(declared_symbols())}];\n"
                    "void take_addresses(void) {\n" + body + "}\n")
     r = subprocess.run([compiler, std, "-Wall", "-Wextra", "-Werror", "-I", str(ROOT / "include"),
