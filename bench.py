@@ -37,7 +37,8 @@ import torch
 ROOT = Path(__file__).resolve().parent
 sys.path.insert(0, str(ROOT))
 
-from paper_2602_19128_b200.inputs import CONFIGS, LOCAL_CONFIGS, bf16_bits, make_inputs  # noqa: E402
+from paper_2602_19128_b200.inputs import (CONFIGS, GQA_CONFIGS, LOCAL_CONFIGS, bf16_bits, make_gqa_inputs,  # noqa: E402
+                                          make_inputs)
 from tests.weight_quantizers import quantize_fp8_blocks, quantize_mxfp8  # noqa: E402
 
 CONFIGS = dict(CONFIGS, **LOCAL_CONFIGS)  # the five workloads plus the local-expert-subset shapes
@@ -643,6 +644,73 @@ def measure(ctx: Ctx, name: str, inp: dict, steps, warmup: int, with_e2e: bool, 
                 roofline=roofline, layer=layer, cpu_baseline=cpu_baseline)
 
 
+def measure_gqa(ctx: Ctx, name: str) -> dict:
+    """The second workload (paged grouped-query decode attention, gqa_paged_decode): decode steps per second over a
+    seeded batch of cached sequences, and the cache bytes streamed per second against the HBM roofline (every cached
+    key and value is read once: 2 * Hkv * D * 2 bytes per cached token)."""
+    moe, args, dev, peaks = ctx.moe, ctx.args, ctx.dev, ctx.peaks
+    cfg = GQA_CONFIGS[name]
+    inp = make_gqa_inputs(cfg, seed=args.seed + ctx.rank, device=dev)
+    B, Hq, Hkv, D = inp["B"], inp["Hq"], inp["Hkv"], inp["D"]
+    max_len = max(inp["kv_len"])
+    ws = moe.alloc_workspace(moe.gqa_decode_workspace_bytes(B, Hq, Hkv, D, max_len), dev)
+    out = torch.empty((B, Hq, D), dtype=torch.bfloat16, device=dev)
+    lse = torch.empty((B, Hq), dtype=torch.float32, device=dev)
+    kv_bytes = sum(inp["kv_len"]) * 2 * Hkv * D * 2
+    need_flush = kv_bytes < 2 * L2_BYTES
+    flush_buf = torch.zeros(2 * L2_BYTES // 4, dtype=torch.float32, device=dev) if need_flush else None
+
+    def step():
+        moe.gqa_paged_decode(inp["q"], inp["k_cache"], inp["v_cache"], inp["kv_indptr"], inp["kv_indices"],
+                             inp["kv_last_page_len"], max_len, inp["sm_scale"], out, ws, lse=lse)
+    for _ in range(3):
+        step()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(); step(); e1.record(); e1.synchronize()
+    est_ms = max(e0.elapsed_time(e1), 1e-3)
+    steps = args.steps if args.few_launches else int(min(max(20, math.ceil(300.0 / est_ms)), 2000))
+    for _ in range(3 if args.few_launches else min(steps, 200)):
+        step()
+    pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps if need_flush else 1)]
+    ctx.barrier()
+    sampler = ClockSampler(ctx.local) if ctx.rank == 0 else None
+    if not need_flush:
+        pairs[0][0].record()
+    for s_ in range(steps):
+        if need_flush:
+            flush_l2(flush_buf)
+            pairs[s_][0].record()
+        step()
+        if need_flush:
+            pairs[s_][1].record()
+    if not need_flush:
+        pairs[0][1].record()
+    ctx.barrier()
+    clocks = sampler.stop() if sampler else None
+    ms = max_over_ranks(ctx.dist, sum(a.elapsed_time(b) for a, b in pairs), dev) / steps
+    cpu = None
+    if not args.no_cpu_baseline and not args.few_launches and ctx.world == 1 and sum(inp["kv_len"]) * Hq <= 40_000_000:
+        from oracle import gqa_oracle
+        o = gqa_oracle.get("f64")
+        host = [bf16_bits(inp[n]) for n in ("q", "k_cache", "v_cache")] + [inp[n].cpu().numpy() for n in
+                                                                            ("kv_indptr", "kv_indices", "kv_last_page_len")]
+        t0 = time.perf_counter()
+        o.paged_decode(*host, inp["sm_scale"])
+        wall = time.perf_counter() - t0
+        cpu = dict(value=B / wall, unit="decode tokens/s", cores=o.num_threads, kind="oracle",
+                   sample=f"the whole batch of '{name}' once, double-precision oracle, {wall:.2f} s wall")
+    return dict(metric="gqa_paged_decode_tokens_per_s", value=ctx.world * B / (ms * 1e-3), unit="decode tokens/s",
+                ms_per_step=ms, steps=steps, gpu_launches=steps,
+                config=dict(workload=name, **{k_: cfg[k_] for k_ in ("B", "Hq", "Hkv", "D", "page_size")},
+                            cached_tokens=sum(inp["kv_len"]), kv_len_min=min(inp["kv_len"]), kv_len_max=max_len,
+                            split_tokens=moe.gqa_decode_split_tokens(B, Hq, Hkv, D, max_len),
+                            l2="flushed between steps" if need_flush else "cache larger than L2, no flush"),
+                roofline=dict(bound="hbm", kernel="gqa_paged_decode_kernel", algorithmic_per_launch=kv_bytes, peak=peaks["hbm_gbs"],
+                              frac=kv_bytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], peak_source=f"of {peaks['source']}",
+                              traffic=None, **hbm_fractions(kv_bytes, ms * 1e-3, peaks)),
+                clocks=clocks, cpu_baseline=cpu, dtype="bf16")
+
+
 def sweep_entry(r: dict) -> dict:
     """What the line keeps of a sweep workload."""
     return dict(ms_per_step=r["ms_per_step"], value=r["value"], unit=UNIT, steps=r["steps"], warmup=r["warmup"],
@@ -677,6 +745,15 @@ def run_ours(args):
             except Exception as exc:  # the headline still has to be printed
                 sweep[name] = dict(error=f"{type(exc).__name__}: {exc}")
             torch.cuda.empty_cache()
+    second = None
+    if do_sweep or args.gqa:  # the second workload of the paper (Sec. 4.6), reported beside the layer, never as the headline
+        second = {}
+        for name in ("gqa_decode_b64", "gqa_decode_b256", "gqa_decode_b1_long"):
+            try:
+                second[name] = measure_gqa(ctx, name)
+            except Exception as exc:
+                second[name] = dict(error=f"{type(exc).__name__}: {exc}")
+            torch.cuda.empty_cache()
     inp = shared if shared is not None else make_inputs(CONFIGS[headline], seed=args.seed + rank, device=ctx.dev)
     r = measure(ctx, headline, inp, steps=args.steps, warmup=args.warmup, with_e2e=not args.few_launches,
                 with_cpu_baseline=not args.no_cpu_baseline and not args.few_launches)
@@ -685,7 +762,7 @@ def run_ours(args):
                     ms_per_step=r["ms_per_step"], higher_is_better=True, scaling="weak", vs_baseline=None, dtype=r["dtype"],
                     data="synthetic", config=r["config"], clocks=r["clocks"], e2e=r["e2e"], gpu_launches=r["gpu_launches"],
                     host_us_per_call=r["host_us_per_call"], roofline=r["roofline"], layer=r["layer"],
-                    cpu_baseline=r["cpu_baseline"], sweep=sweep if do_sweep else None)
+                    cpu_baseline=r["cpu_baseline"], sweep=sweep if do_sweep else None, second_workload=second)
         print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
@@ -700,6 +777,7 @@ def main():
     ap.add_argument("--config", choices=list(CONFIGS), default=None,
                     help=f"measure this workload alone (default: headline {HEADLINE} plus a sweep of the other four)")
     ap.add_argument("--sweep", action="store_true", help="with --config: also run the sweep of the other workloads")
+    ap.add_argument("--gqa", action="store_true", help="with --config: also measure the paged grouped-query decode workloads")
     ap.add_argument("--shape", default=None, help="custom T,H,I,E,top_k instead of a named workload (profiling)")
     ap.add_argument("--bound", choices=["hbm", "tensor"], default="hbm", help="with --shape: which roofline to report against")
     ap.add_argument("--weights", choices=["bf16", "fp8", "mxfp8"], default="bf16",

@@ -20,8 +20,10 @@
  * partial result to a temporary buffer, and the block that finds itself last -- a counter -- merges them; keys and
  * values are fetched in chunks while the previous chunk is being used): one block per (sequence chunk, key-value
  * head, batch item) keeps all Hq / Hkv query heads of its key-value head in registers, so every key and value is
- * read from memory once per group, streams its tokens through a three-stage asynchronous copy pipeline, and the last
- * block of each (item, key-value head) merges the partial results.  Results do not depend on which block is last.
+ * read from memory once per group, streams its tokens through a pipeline of TMA copies that follow the page table
+ * (one tile per page for page sizes that are powers of two of at least 8, one 256-byte row copy per token otherwise),
+ * and the last block of each (item, key-value head) merges the partial results.  Results do not depend on which block
+ * is last.
  */
 #ifndef GQA_DECODE_B200_H_
 #define GQA_DECODE_B200_H_
@@ -35,8 +37,8 @@
 extern "C" {
 #endif
 
-/* Host-only, pure.  Bytes of workspace gqa_paged_decode needs (block counters and the partial results of the
- * sequence splits); 0 outside the supported envelope.  max_kv_len: an upper bound of the cached lengths, used to size
+/* Host-only, pure.  Bytes of workspace gqa_paged_decode needs (a status word, block counters and the partial results
+ * of the sequence splits); 0 outside the supported envelope.  max_kv_len: an upper bound of the cached lengths, used to size
  * the split of the sequence (a longer sequence is still computed correctly, by its last block).
  * Envelope: D == 128; Hq a multiple of Hkv with 1 <= Hq / Hkv <= 16; B >= 0; max_kv_len >= 0. */
 MOE_API size_t gqa_decode_workspace_bytes(int B, int Hq, int Hkv, int D, int max_kv_len);
@@ -50,11 +52,15 @@ MOE_API size_t gqa_decode_workspace_bytes(int B, int Hq, int Hkv, int D, int max
  *   sm_scale         the score scale (usually D^-0.5)
  *   out              [B,Hq,D] bf16, out
  *   lse              [B,Hq] f32, out, or NULL
- *   workspace        at least gqa_decode_workspace_bytes(...) bytes, 256-byte aligned; contents undefined afterwards;
- *                    concurrent calls need distinct workspaces
+ *   workspace        at least gqa_decode_workspace_bytes(...) bytes, 256-byte aligned; concurrent calls need distinct
+ *                    workspaces.  Afterwards its first int32 is the call's device status, which
+ *                    moe_last_status(workspace, stream) reads: MOE_OK, or MOE_ERR_DEVICE_TIMEOUT when a block's bounded
+ *                    wait for its copies ran out (out is then incomplete); the rest is undefined
  * Pointers of q, the caches and out must be 16-byte aligned, the int arrays and lse 4-byte aligned.
  * B == 0 succeeds without a launch.  Page numbers and lengths are NOT validated (they live on the device); page
- * numbers outside [0, num_pages) are outside the contract.  Enqueues one memset and one kernel. */
+ * numbers outside [0, num_pages) are outside the contract.  num_pages * page_size must be below 2^31
+ * (MOE_ERR_UNSUPPORTED).  Enqueues one memset and one kernel; returns MOE_ERR_CUDA when a tensor map cannot be encoded
+ * or the launch fails. */
 MOE_API int gqa_paged_decode(const void *q, const void *k_cache, const void *v_cache, const int32_t *kv_indptr,
                              const int32_t *kv_indices, const int32_t *kv_last_page_len, int B, int Hq, int Hkv, int D,
                              int page_size, int num_pages, int max_kv_len, float sm_scale, void *out, float *lse,

@@ -6,9 +6,17 @@
 //   * one block per (sequence split, key-value head, batch item); its 4 warps keep the 16 x 128 query tile of the
 //     group (Hq / Hkv heads, padded to the MMA's 16 rows) in registers, so a key or value byte is fetched from
 //     memory once for all heads of the group (Sec. 4.6 / Table 2: "fusing multiple query heads per KV head");
-//   * tokens arrive in chunks of 64 through a three-stage cp.async pipeline of 16-byte copies that follow the page
-//     table ("vectorized/async paged-KV gather with pipelined global to shared memory prefetch"); two blocks per SM
-//     keep about 128 KiB in flight per SM; rows past the end of the sequence are zero-filled;
+//   * tokens arrive in chunks of 64 through a two-stage pipeline of TMA copies that follow the page table and
+//     complete on the stage's mbarrier ("vectorized/async paged-KV gather with pipelined global to shared memory
+//     prefetch"), three blocks per SM.  Page sizes that are powers of two of at least 8 take the TILED gather: the
+//     cache is a 4-D tensor (dims, key-value head, slot, page) and one `cp.async.bulk.tensor` box brings a page's
+//     slots (up to 64) x 64 dims of one head, 128-byte swizzled, so a chunk costs one lane of warp 0 one page-table
+//     look-up and one instruction per box (16 boxes per chunk at 16-token pages).  Other page sizes take the ROW
+//     gather, one 256-byte `cp.async.bulk` per token row and thread into rows padded to 272 bytes.  What was
+//     measured on the way, B = 64 x 16k tokens: sixteen 16-byte cp.async per thread and chunk, 4.0 TB/s (800
+//     instructions per warp and chunk, instruction-latency bound at 8 warps per SM); the row gather 4.0 TB/s with and
+//     5.2 TB/s without the arithmetic, one 256-byte request per 14 cycles and SM being all the copy engine took; the
+//     tiled gather 5.4 TB/s at 3 stages x 2 blocks and 6.1 TB/s at 2 stages x 3 blocks;
 //   * each warp owns 16 tokens of a chunk: S = Q K^T (mma.sync m16n8k16, bf16 in, fp32 out: the tile is 16 rows, far
 //     too small for a tcgen05 tile, and the kernel is bound by the copy stream), an online softmax in the base-2
 //     domain, O += P V with the probabilities re-used from the accumulator registers;
@@ -16,12 +24,25 @@
 //     workspace, bumps the (item, head) counter, and the block that finds itself last merges the splits and writes
 //     out / lse (Sec. 4.6 "Parallelism over the sequence").  A sequence with one active split skips the round trip.
 // The merge is a fixed-order sum over splits, so results do not depend on which block arrives last.
+// Every wait on a stage's barrier is bounded: a block that gives up records MOE_ERR_DEVICE_TIMEOUT in the
+// workspace's status word (read it with moe_last_status) and leaves without writing a result.
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <math.h>
 #include <stdint.h>
+#include <string.h>
 
 #include "gqa_decode.h"
+
+namespace moe {
+namespace tc {
+// (moe_tc_host.cu) 4-D bf16 tensor map of a paged cache [num_pages, page_size, Hkv, 128]: box = 64 dims x 1 head x
+// box_rows slots x 1 page, 128-byte swizzle; encoded through the driver entry point and cached.
+bool encode_kv_cache_map(CUtensorMap *map, const void *cache, uint64_t num_pages, uint32_t page_size, uint32_t Hkv,
+                         uint32_t box_rows);
+}  // namespace tc
+}  // namespace moe
 
 namespace gqa {
 namespace {
@@ -31,11 +52,20 @@ constexpr int kRows = 16;          // query heads per block: the MMA's M; groups
 constexpr int kChunk = 64;         // tokens per pipeline stage
 constexpr int kWarps = 4;          // each owns 16 tokens of a chunk
 constexpr int kThreads = kWarps * 32;
-constexpr int kStages = 3;
-constexpr int kRowBytes = kD * 2;  // 256 bytes per token and head
-constexpr int kStageBytes = 2 * kChunk * kRowBytes;  // keys, then values: 32 KiB
-constexpr int kSmemBytes = kStages * kStageBytes;    // 96 KiB: two blocks per SM
-constexpr int kMaxSplits = 64;
+constexpr int kStages = 2;         // one chunk in flight while the previous one is used ...
+constexpr int kBlocksPerSm = 3;    // ... in each of three blocks per SM (168 registers per thread, 69 KiB each)
+constexpr int kRowBytes = kD * 2;  // 256 bytes per token and head in the cache
+// Two layouts of a 64-token tile in shared memory, one per gather mode, inside the same 17 KiB:
+//   tiled: two halves of 64 dims, each [64 rows][128 bytes] in TMA's 128-byte swizzle (16 KiB);
+//   rows:  [64 rows][272 bytes], the 16 bytes of padding keeping ldmatrix free of bank conflicts.
+constexpr int kRowPitch = kRowBytes + 16;
+constexpr int kTileBytes = kChunk * kRowPitch;        // 17 KiB, a multiple of 1024 (the swizzle's alignment)
+constexpr int kHalfBytes = kChunk * 128;              // tiled: one half of the dims
+constexpr int kStageBytes = 2 * kTileBytes;           // keys, then values: 34 KiB
+constexpr int kSmemBytes = kStages * kStageBytes + 1024;  // (the base is rounded up to 1024 bytes)
+static_assert(kTileBytes % 1024 == 0, "tiles must keep the swizzle's alignment");
+constexpr int kWaitLimit = 1 << 22;                   // polls of a stage's barrier before the block gives up
+constexpr int kMaxSplits = 128;
 constexpr float kLog2e = 1.4426950408889634f;
 
 struct Params {
@@ -43,23 +73,49 @@ struct Params {
     const int *kv_indptr, *kv_indices, *kv_last_page_len;
     __nv_bfloat16 *out;
     float *lse;
+    int *status;       // the workspace's status word, zeroed before the launch
     int *counters;     // [B * Hkv], zeroed before the launch
     float *part_ml;    // [B * Hkv, n_splits, group, 2]  (max in the base-2 domain, sum)
     float *part_o;     // [B * Hkv, n_splits, group, D]  unnormalised
     int B, Hq, Hkv, group, page_size, split_tokens, n_splits;
+    int box_rows;      // tiled gather: token rows one TMA box brings (min(page_size, 64))
     float scale_log2;  // sm_scale * log2(e)
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
-// 16 bytes global -> shared, or 16 zero bytes when `valid` is false (src-size 0; the source address is not read).
-__device__ __forceinline__ void cp_async_16(uint32_t dst, const void *src, bool valid) {
-    const int n = valid ? 16 : 0;
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(n) : "memory");
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    return done != 0;
+}
+// One bulk copy of `bytes` (a multiple of 16, both addresses 16-byte aligned) that completes on an mbarrier.
+__device__ __forceinline__ void bulk_copy(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
+// One tile of a 4-D tensor map (dims, key-value head, slot, page) that completes on an mbarrier.  c0 * 2 bytes is a
+// multiple of 16 (c0 is 0 or 64).
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map, int c0, int c1, int c2, int c3,
+                                            uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar) : "memory");
+}
 
 __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
@@ -80,13 +136,22 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return *reinterpret_cast<uint32_t *>(&v);
 }
 
-// Byte offset, inside a 64-token tile of 256-byte rows, of 16-byte piece `piece` of token row `row`: the piece index
-// is XOR-ed with the row's low bits so that the eight rows an ldmatrix reads fall into different banks.
-__device__ __forceinline__ uint32_t tile_offset(int row, int piece) { return row * kRowBytes + ((piece ^ (row & 7)) << 4); }
+// Byte offset, inside a 64-token tile, of 16-byte piece `piece` (0..15) of token row `row`.
+template <bool kTiled>
+__device__ __forceinline__ uint32_t tile_offset(int row, int piece) {
+    if (kTiled) return (piece >> 3) * kHalfBytes + row * 128 + (((piece & 7) ^ (row & 7)) << 4);
+    return row * kRowPitch + (piece << 4);
+}
 
-__global__ void __launch_bounds__(kThreads, 2) gqa_paged_decode_kernel(const Params p) {
-    extern __shared__ __align__(128) uint8_t smem[];
-    __shared__ int is_last;
+// kTiled: the page size is a power of two of at least 8, and the gather is one TMA tile per (page, half of the
+// dims, keys or values); otherwise one 256-byte bulk copy per token row.
+template <bool kTiled>
+__global__ void __launch_bounds__(kThreads, kBlocksPerSm)
+gqa_paged_decode_kernel(const Params p, const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map) {
+    extern __shared__ __align__(128) uint8_t smem_raw[];
+    uint8_t *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    __shared__ int is_last, gave_up;
+    __shared__ __align__(8) unsigned long long full_bar[kStages];
     const int split = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int pages = p.kv_indptr[b + 1] - p.kv_indptr[b];
@@ -123,30 +188,71 @@ __global__ void __launch_bounds__(kThreads, 2) gqa_paged_decode_kernel(const Par
         }
     }
 
-    // ---- the copy pipeline: thread i moves pieces i, i + 128, ... (8 of the keys and 8 of the values per chunk) ----
+    // ---- the copy pipeline ----
+    // tiled: lane l of warp 0 brings one TMA box per chunk -- page l / 4 of the chunk, keys or values ((l / 2) % 2),
+    //        half l % 2 of the dims -- and only warp 0 arrives on the stage's barrier;
+    // rows:  thread i brings ONE token row per chunk -- row i % 64 of the keys (i < 64) or of the values -- and every
+    //        thread arrives, with its 256 bytes when its row exists.
     const int *page_list = p.kv_indices + p.kv_indptr[b];
     const size_t token_stride = (size_t)p.Hkv * kD;  // elements between consecutive slots of a page
-    const uint32_t smem_base = smem_u32(smem);
-    auto issue_chunk = [&](int chunk) {
-        if (chunk < n_chunks) {
-            const uint32_t stage = smem_base + (chunk % kStages) * kStageBytes;
-            const int tok0 = begin + chunk * kChunk;
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const int piece_id = tid + j * kThreads, row = piece_id >> 4, piece = piece_id & 15;
-                const int tok = tok0 + row;
-                const bool valid = tok < end;
-                size_t off = 0;
-                if (valid) {
-                    const int page = page_list[tok / p.page_size];
-                    off = ((size_t)page * p.page_size + (tok % p.page_size)) * token_stride + (size_t)kvh * kD + piece * 8;
+    const uint32_t smem_base = smem_u32(smem), bar_base = smem_u32(full_bar);
+    const int my_row = kTiled ? (lane >> 2) * p.box_rows : (tid & (kChunk - 1));  // first row of the box / the row
+    const bool my_values = kTiled ? ((lane >> 1) & 1) : (tid >= kChunk);
+    const __nv_bfloat16 *my_cache = (my_values ? p.v_cache : p.k_cache) + (size_t)kvh * kD;
+    const uint32_t my_dst = (my_values ? (uint32_t)kTileBytes : 0u) +
+                            (kTiled ? (uint32_t)((lane & 1) * kHalfBytes + my_row * 128) : (uint32_t)(my_row * kRowPitch));
+    const bool copier = kTiled ? (warp == 0) : true;
+    const bool has_box = kTiled ? (my_row < kChunk) : true;  // (64 / box_rows pages per chunk)
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) mbar_init(bar_base + s * 8, kTiled ? 32 : kThreads);
+        gave_up = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+    // Where this thread's row (rows: its slot in the cache; tiled: its page) of a chunk lives, -1 past the end of the
+    // split.  The page table is read ONE CHUNK AHEAD of the copy that needs it, so its latency never sits between copies.
+    auto locate = [&](int chunk) -> int {
+        const int tok = begin + chunk * kChunk + my_row;
+        if (!copier || !has_box || chunk >= n_chunks || tok >= end) return -1;
+        const int page = __ldg(&page_list[tok / p.page_size]);
+        return kTiled ? page : page * p.page_size + tok % p.page_size;
+    };
+    int next_loc = locate(0);
+    auto issue_chunk = [&](int chunk) {  // called for chunk 0, 1, 2, ... in order
+        if (copier && chunk < n_chunks) {
+            const int stage = chunk % kStages;
+            const uint32_t dst = smem_base + stage * kStageBytes + my_dst, bar = bar_base + stage * 8;
+            if (kTiled) {
+                if (next_loc >= 0) {
+                    mbar_arrive_expect_tx(bar, p.box_rows * 128);
+                    tma_load_4d(dst, my_values ? &v_map : &k_map, (lane & 1) * 64, kvh,
+                                (begin + chunk * kChunk + my_row) & (p.page_size - 1), next_loc, bar);
+                } else {
+                    mbar_arrive(bar);
                 }
-                const uint32_t dst = stage + tile_offset(row, piece);
-                cp_async_16(dst, p.k_cache + off, valid);
-                cp_async_16(dst + kChunk * kRowBytes, p.v_cache + off, valid);
+            } else if (next_loc >= 0) {
+                mbar_arrive_expect_tx(bar, kRowBytes);
+                bulk_copy(dst, my_cache + (size_t)next_loc * token_stride, kRowBytes, bar);
+            } else {  // a row past the end: zeros, so that a masked probability of 0 meets a finite value
+#pragma unroll
+                for (int i = 0; i < kRowBytes / 16; ++i)
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(dst + i * 16), "r"(0) : "memory");
+                mbar_arrive(bar);
             }
         }
-        cp_async_commit();  // (an empty group keeps the wait counts uniform)
+        next_loc = locate(chunk + 1);
+    };
+    // Bounded wait for a chunk; false once any thread of the block has given up.
+    auto wait_chunk = [&](int chunk) -> bool {
+        const uint32_t bar = bar_base + (chunk % kStages) * 8, parity = (uint32_t)(chunk / kStages) & 1u;
+        for (int i = 0; i < kWaitLimit; ++i) {
+            if (mbar_try_wait(bar, parity)) return true;
+            if (*(volatile int *)&gave_up) return false;
+        }
+        gave_up = 1;
+        if (atomicCAS(p.status, 0, (int)MOE_ERR_DEVICE_TIMEOUT) == 0) { p.status[1] = 12; p.status[2] = blockIdx.x; }
+        return false;
     };
 
     float o_acc[kD / 8][4];  // this warp's 16 x 128 output tile: 16 n-tiles of 8 dims
@@ -157,21 +263,37 @@ __global__ void __launch_bounds__(kThreads, 2) gqa_paged_decode_kernel(const Par
     float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};  // rows lane/4 and lane/4 + 8
 
     for (int c = 0; c < kStages - 1; ++c) issue_chunk(c);
+    bool ok = true;
     for (int chunk = 0; chunk < n_chunks; ++chunk) {
-        cp_async_wait<kStages - 2>();
-        __syncthreads();                      // chunk `chunk` has landed for every thread; stage (chunk-1) is free
+        ok = wait_chunk(chunk);
+        ok = __syncthreads_and(ok);           // chunk `chunk` has landed; every thread is done with chunk - 1's stage
+        if (!ok) break;
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // (that stage is about to be overwritten by copies)
         issue_chunk(chunk + kStages - 1);
-        const uint32_t k_tile = smem_base + (chunk % kStages) * kStageBytes, v_tile = k_tile + kChunk * kRowBytes;
+        const uint32_t k_tile = smem_base + (chunk % kStages) * kStageBytes, v_tile = k_tile + kTileBytes;
         const int row_base = warp * 16;       // this warp's tokens of the chunk
         const int tok_base = begin + chunk * kChunk + row_base;
         if (tok_base < end) {                 // (uniform over the warp)
+            if (kTiled && tok_base + 16 > end) {
+                // A box brings whole pages: value rows past the end of the sequence hold whatever the cache holds there
+                // (and rows of pages that were not fetched, whatever the stage held).  Zero them, so that a masked
+                // probability of 0 meets a finite value.  The rows are this warp's own.
+                const int valid = end - tok_base;  // 1..15
+                for (int i = lane; i < 16 * 16; i += 32) {
+                    const int r = i >> 4;
+                    if (r >= valid)
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};"
+                                     ::"r"(v_tile + tile_offset<true>(row_base + r, i & 15)), "r"(0) : "memory");
+                }
+                __syncwarp();
+            }
             // S = Q K^T for 16 tokens: two n-tiles of 8 tokens, 8 K-steps
             float s[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
             const int m4 = lane >> 3, rr = lane & 7;
 #pragma unroll
             for (int ks = 0; ks < kD / 16; ++ks) {
                 uint32_t kb[4];
-                ldmatrix_x4(kb, k_tile + tile_offset(row_base + ((m4 >> 1) << 3) + rr, 2 * ks + (m4 & 1)));
+                ldmatrix_x4(kb, k_tile + tile_offset<kTiled>(row_base + ((m4 >> 1) << 3) + rr, 2 * ks + (m4 & 1)));
                 mma_bf16(s[0], qa[ks], kb[0], kb[1]);
                 mma_bf16(s[1], qa[ks], kb[2], kb[3]);
             }
@@ -217,23 +339,29 @@ __global__ void __launch_bounds__(kThreads, 2) gqa_paged_decode_kernel(const Par
                 row_sum[r] += __shfl_xor_sync(0xffffffffu, row_sum[r], 2);
                 l_run[r] = l_run[r] * alpha[r] + row_sum[r];
             }
-            // O = O * alpha + P V: 16 n-tiles of 8 dims, two per transposed ldmatrix
+            // O = O * alpha + P V: 16 n-tiles of 8 dims, two per transposed ldmatrix.  Once the running maxima have
+            // settled alpha is exactly 1 for every row, and the 64 multiplications are skipped (same result).
+            if (__any_sync(0xffffffffu, alpha[0] != 1.f || alpha[1] != 1.f)) {
+#pragma unroll
+                for (int n = 0; n < kD / 8; ++n)
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) o_acc[n][i] *= alpha[i >> 1];
+            }
 #pragma unroll
             for (int n = 0; n < kD / 8; n += 2) {
                 uint32_t vb[4];
-                ldmatrix_x4_trans(vb, v_tile + tile_offset(row_base + ((m4 & 1) << 3) + rr, n + (m4 >> 1)));
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    o_acc[n][i] *= alpha[i >> 1];
-                    o_acc[n + 1][i] *= alpha[i >> 1];
-                }
+                ldmatrix_x4_trans(vb, v_tile + tile_offset<kTiled>(row_base + ((m4 & 1) << 3) + rr, n + (m4 >> 1)));
                 mma_bf16(o_acc[n], pa, vb[0], vb[1]);
                 mma_bf16(o_acc[n + 1], pa, vb[2], vb[3]);
             }
         }
     }
-    cp_async_wait<0>();
-    __syncthreads();  // every warp is done with the pipeline's shared memory: it becomes the merge buffer
+    // A block that gave up waits (bounded) for its copies in flight, then leaves without a result: the status word says so.
+    if (!ok) {
+        for (int i = 0; i < 1000; ++i) __nanosleep(1000);
+        return;
+    }
+    __syncthreads();  // every warp is done with the pipeline's shared memory (all copies were waited for): the merge buffer
 
     // ---- merge the four warps: (max, sum, O) per head, in warp order ----
     float *merge_o = reinterpret_cast<float *>(smem);                    // [4 warps][16 rows][128]
@@ -289,18 +417,42 @@ __global__ void __launch_bounds__(kThreads, 2) gqa_paged_decode_kernel(const Par
     __threadfence();
     const float *all_o = p.part_o + bh * p.n_splits * p.group * kD;
     const float *all_ml = p.part_ml + bh * p.n_splits * p.group * 2;
-    for (int i = tid; i < p.group * kD; i += kThreads) {
-        const int g = i / kD, d = i - g * kD;
+    // Scale factors of every (split, head) first, so that the sums below are streams of independent loads.
+    float *head_m = reinterpret_cast<float *>(smem);   // [16]
+    float *head_l = head_m + kRows;                      // [16]
+    float *scale = head_l + kRows;                       // [n_active][group]
+    __syncthreads();                                     // (the warps' merge buffer is free again)
+    if (tid < p.group) {
         float m = -INFINITY;
-        for (int s = 0; s < n_active; ++s) m = fmaxf(m, __ldcg(&all_ml[(s * p.group + g) * 2]));
-        float l = 0.f, o = 0.f;
+        for (int s = 0; s < n_active; ++s) m = fmaxf(m, __ldcg(&all_ml[(s * p.group + tid) * 2]));
+        head_m[tid] = m;
+    }
+    __syncthreads();
+    for (int i = tid; i < n_active * p.group; i += kThreads)
+        scale[i] = exp2f(__ldcg(&all_ml[i * 2]) - head_m[i % p.group]);
+    __syncthreads();
+    if (tid < p.group) {
+        float l = 0.f;
+        for (int s = 0; s < n_active; ++s) l += __ldcg(&all_ml[(s * p.group + tid) * 2 + 1]) * scale[s * p.group + tid];
+        head_l[tid] = l;
+        if (p.lse) p.lse[(size_t)b * p.Hq + head0 + tid] = (head_m[tid] + log2f(l)) * 0.6931471805599453f;
+    }
+    __syncthreads();
+    for (int i = tid; i < p.group * (kD / 4); i += kThreads) {  // one thread per (head, four dims)
+        const int g = i / (kD / 4), d = (i - g * (kD / 4)) * 4;
+        float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 8
         for (int s = 0; s < n_active; ++s) {  // ascending split order: the sum is the same whichever block is last
-            const float f = exp2f(__ldcg(&all_ml[(s * p.group + g) * 2]) - m);
-            l += __ldcg(&all_ml[(s * p.group + g) * 2 + 1]) * f;
-            o += __ldcg(&all_o[(size_t)(s * p.group + g) * kD + d]) * f;
+            const float4 v = __ldcg(reinterpret_cast<const float4 *>(&all_o[(size_t)(s * p.group + g) * kD + d]));
+            const float f = scale[s * p.group + g];
+            o.x += v.x * f; o.y += v.y * f; o.z += v.z * f; o.w += v.w * f;
         }
-        p.out[((size_t)b * p.Hq + head0 + g) * kD + d] = __float2bfloat16_rn(o / l);
-        if (p.lse && d == 0) p.lse[(size_t)b * p.Hq + head0 + g] = (m + log2f(l)) * 0.6931471805599453f;
+        const float l = head_l[g];
+        __nv_bfloat162 lo = __floats2bfloat162_rn(o.x / l, o.y / l), hi = __floats2bfloat162_rn(o.z / l, o.w / l);
+        uint2 packed;
+        packed.x = *reinterpret_cast<uint32_t *>(&lo);
+        packed.y = *reinterpret_cast<uint32_t *>(&hi);
+        *reinterpret_cast<uint2 *>(&p.out[((size_t)b * p.Hq + head0 + g) * kD + d]) = packed;
     }
 }
 
@@ -310,21 +462,28 @@ bool envelope_ok(long long B, int Hq, int Hkv, int D, long long max_kv_len) {
     return B <= 65535 && Hkv <= 65535;  // grid dimensions y and z
 }
 
-// Sequence splits: enough blocks to fill the device a few times over, no split shorter than four chunks.
+// Sequence splits.  Blocks run in waves of 148 SMs x kBlocksPerSm; a block's time is its chunks plus a fixed cost of
+// about six chunks (pipeline fill, the warps' merge), and about six more once the sequence is split at all (partial
+// results written and merged by the last block; a lone split writes the output directly).  The number of splits
+// minimises waves x per-block time in that model, which ranked measured split counts correctly over batches of 1 to
+// 256 and lengths of 2k to 128k; ties go to fewer splits.  No split is shorter than four chunks.
 void choose_split(int B, int Hkv, int max_kv_len, int *split_tokens, int *n_splits) {
-    const long long base = (long long)B * Hkv;
-    long long want = base > 0 ? (4 * 148 * 2 + base - 1) / base : 1;  // about four waves of two blocks per SM
-    const long long most = (max_kv_len + 4 * kChunk - 1) / (4 * kChunk);
-    if (want > most) want = most;
-    if (want > kMaxSplits) want = kMaxSplits;
-    if (want < 1) want = 1;
-    long long st = (max_kv_len + want - 1) / want;
-    st = (st + kChunk - 1) / kChunk * kChunk;
-    if (st < kChunk) st = kChunk;
-    long long n = (max_kv_len + st - 1) / st;
-    if (n < 1) n = 1;
-    *split_tokens = (int)st;
-    *n_splits = (int)n;
+    const long long base = (long long)B * Hkv, slots = 148 * kBlocksPerSm;
+    const long long chunks = max_kv_len > 0 ? ((long long)max_kv_len + kChunk - 1) / kChunk : 1;
+    long long most = (chunks + 3) / 4;
+    if (most > kMaxSplits) most = kMaxSplits;
+    if (most < 1) most = 1;
+    long long best_n = 1, best_cost = -1;
+    for (long long n = 1; n <= most; ++n) {
+        const long long per_block = (chunks + n - 1) / n, n_eff = (chunks + per_block - 1) / per_block;
+        if (n_eff != n) continue;  // (the same split as a smaller n)
+        const long long waves = (base * n + slots - 1) / slots;
+        const long long cost = (waves > 0 ? waves : 1) * (per_block + 6 + (n > 1 ? 6 : 0));
+        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best_n = n; }
+    }
+    const long long per_block = (chunks + best_n - 1) / best_n;
+    *split_tokens = (int)(per_block * kChunk);
+    *n_splits = (int)((chunks + per_block - 1) / per_block);
 }
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -340,7 +499,7 @@ size_t gqa_decode_workspace_bytes(int B, int Hq, int Hkv, int D, int max_kv_len)
     int st, ns;
     choose_split(B, Hkv, max_kv_len, &st, &ns);
     const size_t bh = (size_t)B * Hkv, group = Hq / Hkv;
-    return align_up(bh * sizeof(int), 256) + align_up(bh * ns * group * 2 * sizeof(float), 256) +
+    return 256 + align_up(bh * sizeof(int), 256) + align_up(bh * ns * group * 2 * sizeof(float), 256) +
            align_up(bh * ns * group * kD * sizeof(float), 256) + 256;
 }
 
@@ -359,6 +518,7 @@ int gqa_paged_decode(const void *q, const void *k_cache, const void *v_cache, co
     using namespace gqa;
     if (B < 0 || Hq < 1 || Hkv < 1 || D < 1 || page_size < 1 || num_pages < 0 || max_kv_len < 0) return MOE_ERR_SHAPE;
     if (!envelope_ok(B, Hq, Hkv, D, max_kv_len)) return MOE_ERR_UNSUPPORTED;
+    if ((long long)num_pages * page_size >= (1ll << 31)) return MOE_ERR_UNSUPPORTED;  // slot numbers are 32-bit
     if (B == 0) return MOE_OK;
     if (!q || !k_cache || !v_cache || !kv_indptr || !kv_indices || !kv_last_page_len || !out || !workspace) return MOE_ERR_NULL;
     auto misaligned = [](const void *ptr, size_t a) { return (reinterpret_cast<uintptr_t>(ptr) % a) != 0; };
@@ -387,21 +547,35 @@ int gqa_paged_decode(const void *q, const void *k_cache, const void *v_cache, co
     p.scale_log2 = sm_scale * kLog2e;
     const size_t bh = (size_t)B * Hkv;
     char *ws = static_cast<char *>(workspace);
-    p.counters = reinterpret_cast<int *>(ws);
-    ws += align_up(bh * sizeof(int), 256);
+    p.status = reinterpret_cast<int *>(ws);  // status word first, as in the layer's workspace: moe_last_status reads it
+    p.counters = reinterpret_cast<int *>(ws + 256);
+    ws += 256 + align_up(bh * sizeof(int), 256);
     p.part_ml = reinterpret_cast<float *>(ws);
     ws += align_up(bh * p.n_splits * p.group * 2 * sizeof(float), 256);
     p.part_o = reinterpret_cast<float *>(ws);
 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (cudaMemsetAsync(p.counters, 0, bh * sizeof(int), st) != cudaSuccess) return MOE_ERR_CUDA;
+    if (cudaMemsetAsync(p.status, 0, 256 + bh * sizeof(int), st) != cudaSuccess) return MOE_ERR_CUDA;
     static bool attr_set[64];
     if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-        if (cudaFuncSetAttribute(gqa_paged_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
+        if (cudaFuncSetAttribute(gqa_paged_decode_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess ||
+            cudaFuncSetAttribute(gqa_paged_decode_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
             return MOE_ERR_CUDA;
         attr_set[dev] = true;
     }
-    gqa_paged_decode_kernel<<<dim3(p.n_splits, Hkv, B), kThreads, kSmemBytes, st>>>(p);
+    // Page sizes that are powers of two of at least 8 take the tiled gather: one 4-D tensor map per cache,
+    // (dims, key-value head, slot, page), a box of 64 dims x min(page_size, 64) slots in the 128-byte swizzle.
+    const bool tiled = page_size >= 8 && (page_size & (page_size - 1)) == 0 && num_pages > 0;
+    CUtensorMap k_map, v_map;
+    memset(&k_map, 0, sizeof(k_map));
+    memset(&v_map, 0, sizeof(v_map));
+    p.box_rows = page_size < kChunk ? page_size : kChunk;
+    if (tiled && (!moe::tc::encode_kv_cache_map(&k_map, k_cache, (uint64_t)num_pages, (uint32_t)page_size, (uint32_t)Hkv, (uint32_t)p.box_rows) ||
+                  !moe::tc::encode_kv_cache_map(&v_map, v_cache, (uint64_t)num_pages, (uint32_t)page_size, (uint32_t)Hkv, (uint32_t)p.box_rows)))
+        return MOE_ERR_CUDA;
+    const dim3 grid(p.n_splits, Hkv, B);
+    if (tiled) gqa_paged_decode_kernel<true><<<grid, kThreads, kSmemBytes, st>>>(p, k_map, v_map);
+    else gqa_paged_decode_kernel<false><<<grid, kThreads, kSmemBytes, st>>>(p, k_map, v_map);
     return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
 

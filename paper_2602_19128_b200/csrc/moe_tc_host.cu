@@ -109,6 +109,20 @@ bool encode(CUtensorMap *map, const void *base, int rank, const cuuint64_t *dims
                          kind == Operand::kCodesForConverter ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B);
 }
 
+}  // namespace
+
+// 4-D bf16 tensor map of a paged key-value cache [num_pages, page_size, Hkv, 128] (decode attention): one box is
+// 64 dims x 1 head x box_rows slots x 1 page, in the 128-byte swizzle.
+bool encode_kv_cache_map(CUtensorMap *map, const void *cache, uint64_t num_pages, uint32_t page_size, uint32_t Hkv,
+                         uint32_t box_rows) {
+    const cuuint64_t dims[4] = {128, Hkv, page_size, num_pages};
+    const cuuint64_t strides[3] = {128ull * 2, 128ull * 2 * Hkv, 128ull * 2 * Hkv * page_size};
+    const cuuint32_t box[4] = {64, 1, box_rows, 1};
+    return encode(map, cache, 4, dims, strides, box);
+}
+
+namespace {
+
 // 2-D bf16 tensor [rows, cols] row-major; box = box_rows x 64 columns, 128-byte swizzle, zero fill.
 bool encode_2d(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
     const cuuint64_t dims[2] = {cols, rows};

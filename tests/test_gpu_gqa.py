@@ -66,6 +66,13 @@ CASES = [
     (5, 32, 4, 32, [16, 32, 33, 4096, 257]),          # mixed lengths: some sequences use one split, some many
     (40, 8, 4, 16, [100 + 37 * i for i in range(40)]),  # enough items that every sequence is a single split
     (2, 2, 1, 64, [64, 6000]),                        # groups of two, large pages
+    (3, 32, 4, 8, [7, 1000, 5000]),                   # the smallest page the tiled gather takes: 32 boxes per chunk
+    (2, 32, 4, 128, [100, 7000]),                     # pages larger than a chunk: boxes start inside a page
+    (2, 8, 1, 256, [255, 9000]),
+    (3, 32, 4, 12, [11, 1000, 5000]),                 # page sizes that are no power of two: the row gather
+    (2, 16, 2, 3, [2, 4100]),
+    (2, 32, 4, 24, [24, 6001]),
+    (2, 32, 4, 2, [3000, 1]),
 ]
 
 
@@ -73,6 +80,34 @@ CASES = [
 def test_decode_matches_oracle(B, Hq, Hkv, P, lengths):
     inp = make_gqa_inputs(dict(B=B, Hq=Hq, Hkv=Hkv, D=128, page_size=P, lengths=lengths), seed=B + Hq, device="cuda")
     check(inp)
+
+
+@pytest.mark.parametrize("P", [16, 12, 64, 128])
+def test_slots_past_the_end_of_a_sequence_are_never_used(P):
+    """The cache behind the last token of a sequence, and every page no sequence owns, holds NaN: the tiled gather
+    copies whole pages into shared memory and must still keep those values out of the result."""
+    lengths = [1, P + 1, 5 * P - 1, 3000 + P // 2, 64 * 7 + 5]
+    inp = make_gqa_inputs(dict(B=len(lengths), Hq=32, Hkv=4, D=128, page_size=P, lengths=lengths), seed=P, device="cuda")
+    owned = torch.zeros((inp["num_pages"], P), dtype=torch.bool, device="cuda")
+    indptr, indices = inp["kv_indptr"].tolist(), inp["kv_indices"]
+    for b, n in enumerate(lengths):
+        pages = indices[indptr[b]:indptr[b + 1]].long()
+        flat = torch.zeros(len(pages) * P, dtype=torch.bool, device="cuda")
+        flat[:n] = True
+        owned[pages] = flat.view(len(pages), P)
+    for cache in (inp["k_cache"], inp["v_cache"]):
+        cache[~owned] = float("nan")
+    check(inp)
+
+
+def test_the_workspace_status_word_reports_success():
+    inp = make_gqa_inputs(dict(B=2, Hq=32, Hkv=4, D=128, page_size=16, lengths=[5000, 300]), seed=3, device="cuda")
+    ws = moe.alloc_workspace(moe.gqa_decode_workspace_bytes(2, 32, 4, 128, 5000), "cuda")
+    ws.fill_(0x5A)
+    out = torch.empty((2, 32, 128), dtype=torch.bfloat16, device="cuda")
+    moe.gqa_paged_decode(inp["q"], inp["k_cache"], inp["v_cache"], inp["kv_indptr"], inp["kv_indices"],
+                         inp["kv_last_page_len"], 5000, inp["sm_scale"], out, ws)
+    assert moe.moe_last_status(ws) == 0
 
 
 def test_a_sequence_longer_than_the_hint_is_still_computed_in_full():
