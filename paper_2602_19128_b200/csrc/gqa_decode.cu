@@ -462,24 +462,32 @@ bool envelope_ok(long long B, int Hq, int Hkv, int D, long long max_kv_len) {
     return B <= 65535 && Hkv <= 65535;  // grid dimensions y and z
 }
 
-// Sequence splits.  Blocks run in waves of 148 SMs x kBlocksPerSm; a block's time is its chunks plus a fixed cost of
-// about six chunks (pipeline fill, the warps' merge), and about six more once the sequence is split at all (partial
-// results written and merged by the last block; a lone split writes the output directly).  The number of splits
-// minimises waves x per-block time in that model, which ranked measured split counts correctly over batches of 1 to
-// 256 and lengths of 2k to 128k; ties go to fewer splits.  No split is shorter than four chunks.
+// Sequence splits, from a model of the kernel's time in units of one chunk streamed by a block on a full machine.
+// 148 SMs x kBlocksPerSm blocks are resident at a time, so blocks run in waves; a block costs its chunks plus 4
+// (pipeline fill and the warps' merge, partly hidden behind the SM's other blocks); a wave that fills a fraction f of
+// the machine runs in max(0.57, 0.3 + 0.7 f) of a full wave's time (a block alone streams a chunk in 0.57 of the
+// time); a split sequence pays the partial results' round trip and the last block's merge once, 8 + n / 4; and 0.3 of
+// a block's length is added for the tail that sequences shorter than max_kv_len leave (their lengths are known to the
+// device only).  The constants were fitted to measured split sweeps (batches of 1 to 256, 2k to 128k tokens, equal
+// and ragged lengths); the chosen count was within 10 % of the best measured one in each.  Ties go to fewer splits;
+// no split is shorter than four chunks.
 void choose_split(int B, int Hkv, int max_kv_len, int *split_tokens, int *n_splits) {
     const long long base = (long long)B * Hkv, slots = 148 * kBlocksPerSm;
     const long long chunks = max_kv_len > 0 ? ((long long)max_kv_len + kChunk - 1) / kChunk : 1;
     long long most = (chunks + 3) / 4;
     if (most > kMaxSplits) most = kMaxSplits;
     if (most < 1) most = 1;
-    long long best_n = 1, best_cost = -1;
+    long long best_n = 1;
+    double best_cost = -1.0;
     for (long long n = 1; n <= most; ++n) {
         const long long per_block = (chunks + n - 1) / n, n_eff = (chunks + per_block - 1) / per_block;
         if (n_eff != n) continue;  // (the same split as a smaller n)
-        const long long waves = (base * n + slots - 1) / slots;
-        const long long cost = (waves > 0 ? waves : 1) * (per_block + 6 + (n > 1 ? 6 : 0));
-        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best_n = n; }
+        const long long blocks = (base > 0 ? base : 1) * n, full_waves = blocks / slots;
+        const double f = (double)(blocks - full_waves * slots) / (double)slots;
+        const double last_wave = f > 0.0 ? (0.3 + 0.7 * f > 0.57 ? 0.3 + 0.7 * f : 0.57) : 0.0;
+        const double cost = ((double)per_block + 4.0) * ((double)full_waves + last_wave) + 0.3 * (double)per_block +
+                            (n > 1 ? 8.0 + 0.25 * (double)n : 0.0);
+        if (best_cost < 0 || cost < best_cost * (1.0 - 1e-9)) { best_cost = cost; best_n = n; }
     }
     const long long per_block = (chunks + best_n - 1) / best_n;
     *split_tokens = (int)(per_block * kChunk);
