@@ -689,7 +689,7 @@ def measure_gqa(ctx: Ctx, name: str) -> dict:
     clocks = sampler.stop() if sampler else None
     ms = max_over_ranks(ctx.dist, sum(a.elapsed_time(b) for a, b in pairs), dev) / steps
     cpu = None
-    if not args.no_cpu_baseline and not args.few_launches and ctx.world == 1 and sum(inp["kv_len"]) * Hq <= 40_000_000:
+    if not args.no_cpu_baseline and not args.few_launches and ctx.world == 1 and sum(inp["kv_len"]) * Hq <= 25_000_000:
         from oracle import gqa_oracle
         o = gqa_oracle.get("f64")
         host = [bf16_bits(inp[n]) for n in ("q", "k_cache", "v_cache")] + [inp[n].cpu().numpy() for n in
@@ -748,7 +748,7 @@ def run_ours(args):
     second = None
     if do_sweep or args.gqa:  # the second workload of the paper (Sec. 4.6), reported beside the layer, never as the headline
         second = {}
-        for name in ("gqa_decode_b64", "gqa_decode_b256", "gqa_decode_b1_long"):
+        for name in ("gqa_decode_b64", "gqa_decode_b256", "gqa_decode_b1_long", "gqa_decode_b64_16k"):
             try:
                 second[name] = measure_gqa(ctx, name)
             except Exception as exc:

@@ -105,6 +105,8 @@ GQA_CONFIGS = {
     "gqa_decode_b64": dict(B=64, Hq=32, Hkv=4, D=128, page_size=16, len_lo=1024, len_hi=8192),
     "gqa_decode_b1_long": dict(B=1, Hq=32, Hkv=4, D=128, page_size=16, len_lo=65536, len_hi=65536),
     "gqa_decode_b256": dict(B=256, Hq=32, Hkv=4, D=128, page_size=16, len_lo=256, len_hi=2048),
+    # long enough that launch, pipeline fill and the merge are small beside the stream: the kernel's steady state
+    "gqa_decode_b64_16k": dict(B=64, Hq=32, Hkv=4, D=128, page_size=16, len_lo=16384, len_hi=16384),
 }
 
 

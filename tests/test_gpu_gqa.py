@@ -141,7 +141,7 @@ def test_lse_is_optional_and_arguments_are_checked_before_any_launch():
     assert (o == 0).all()
 
 
-@pytest.mark.parametrize("name", ["gqa_decode_b64", "gqa_decode_b256", "gqa_decode_b1_long"])
+@pytest.mark.parametrize("name", ["gqa_decode_b64", "gqa_decode_b256", "gqa_decode_b1_long", "gqa_decode_b64_16k"])
 def test_full_size_workload(name):
     """The benchmark's workloads in its launch configuration: every element against the oracle."""
     inp = make_gqa_inputs(GQA_CONFIGS[name], seed=0, device="cuda")
