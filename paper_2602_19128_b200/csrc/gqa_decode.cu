@@ -9,14 +9,15 @@
 //   * tokens arrive in chunks of 64 through a two-stage pipeline of TMA copies that follow the page table and
 //     complete on the stage's mbarrier ("vectorized/async paged-KV gather with pipelined global to shared memory
 //     prefetch"), three blocks per SM.  Page sizes that are powers of two of at least 8 take the TILED gather: the
-//     cache is a 4-D tensor (dims, key-value head, slot, page) and one `cp.async.bulk.tensor` box brings a page's
-//     slots (up to 64) x 64 dims of one head, 128-byte swizzled, so a chunk costs one lane of warp 0 one page-table
-//     look-up and one instruction per box (16 boxes per chunk at 16-token pages).  Other page sizes take the ROW
-//     gather, one 256-byte `cp.async.bulk` per token row and thread into rows padded to 272 bytes.  What was
-//     measured on the way, B = 64 x 16k tokens: sixteen 16-byte cp.async per thread and chunk, 4.0 TB/s (800
-//     instructions per warp and chunk, instruction-latency bound at 8 warps per SM); the row gather 4.0 TB/s with and
-//     5.2 TB/s without the arithmetic, one 256-byte request per 14 cycles and SM being all the copy engine took; the
-//     tiled gather 5.4 TB/s at 3 stages x 2 blocks and 6.1 TB/s at 2 stages x 3 blocks;
+//     cache is a 5-D tensor (64 dims, slot, half of the dims, head, page) and one `cp.async.bulk.tensor` box brings a
+//     page's slots (up to 64) of one head as two 128-byte-swizzled blocks, so a chunk of 16-token pages is eight
+//     boxes, dealt out two to each warp (a thread is held 5 to 9 cycles per 128-byte row of a box it issues).
+//     Other page sizes take the ROW gather, one 256-byte `cp.async.bulk` per token row and thread into rows padded
+//     to 272 bytes.  What was measured on the way, B = 64 x 16k tokens: sixteen 16-byte cp.async per thread and
+//     chunk, 4.0 TB/s (800 instructions per warp and chunk, instruction-latency bound at 8 warps per SM); the row
+//     gather 4.0 TB/s with and 5.2 TB/s without the arithmetic, one 256-byte request per 14 cycles and SM being all
+//     the copy engine took; the tiled gather 5.4 TB/s at 3 stages x 2 blocks, 6.1 TB/s at 2 stages x 3 blocks with
+//     one warp issuing, 6.3 TB/s with the boxes dealt out;
 //   * each warp owns 16 tokens of a chunk: S = Q K^T (mma.sync m16n8k16, bf16 in, fp32 out: the tile is 16 rows, far
 //     too small for a tcgen05 tile, and the kernel is bound by the copy stream), an online softmax in the base-2
 //     domain, O += P V with the probabilities re-used from the accumulator registers;
@@ -37,8 +38,9 @@
 
 namespace moe {
 namespace tc {
-// (moe_tc_host.cu) 4-D bf16 tensor map of a paged cache [num_pages, page_size, Hkv, 128]: box = 64 dims x 1 head x
-// box_rows slots x 1 page, 128-byte swizzle; encoded through the driver entry point and cached.
+// (moe_tc_host.cu) 5-D bf16 tensor map of a paged cache [num_pages, page_size, Hkv, 128], dimensions ordered (64
+// dims, slot, half of the dims, head, page): box = 64 dims x box_rows slots x both halves of one head of one page,
+// 128-byte swizzle; encoded through the driver entry point and cached.
 bool encode_kv_cache_map(CUtensorMap *map, const void *cache, uint64_t num_pages, uint32_t page_size, uint32_t Hkv,
                          uint32_t box_rows);
 }  // namespace tc
@@ -56,11 +58,11 @@ constexpr int kStages = 2;         // one chunk in flight while the previous one
 constexpr int kBlocksPerSm = 3;    // ... in each of three blocks per SM (168 registers per thread, 69 KiB each)
 constexpr int kRowBytes = kD * 2;  // 256 bytes per token and head in the cache
 // Two layouts of a 64-token tile in shared memory, one per gather mode, inside the same 17 KiB:
-//   tiled: two halves of 64 dims, each [64 rows][128 bytes] in TMA's 128-byte swizzle (16 KiB);
+//   tiled: one block per TMA box, [64 / box_rows boxes][2 halves of the dims][box_rows rows][128 bytes], each half
+//          block in TMA's 128-byte swizzle (16 KiB);
 //   rows:  [64 rows][272 bytes], the 16 bytes of padding keeping ldmatrix free of bank conflicts.
 constexpr int kRowPitch = kRowBytes + 16;
 constexpr int kTileBytes = kChunk * kRowPitch;        // 17 KiB, a multiple of 1024 (the swizzle's alignment)
-constexpr int kHalfBytes = kChunk * 128;              // tiled: one half of the dims
 constexpr int kStageBytes = 2 * kTileBytes;           // keys, then values: 34 KiB
 constexpr int kSmemBytes = kStages * kStageBytes + 1024;  // (the base is rounded up to 1024 bytes)
 static_assert(kTileBytes % 1024 == 0, "tiles must keep the swizzle's alignment");
@@ -108,13 +110,12 @@ __device__ __forceinline__ void bulk_copy(uint32_t dst, const void *src, uint32_
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
 
-// One tile of a 4-D tensor map (dims, key-value head, slot, page) that completes on an mbarrier.  c0 * 2 bytes is a
-// multiple of 16 (c0 is 0 or 64).
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map, int c0, int c1, int c2, int c3,
-                                            uint32_t bar) {
+// One box of the cache's 5-D tensor map -- coordinates (dim 0, slot, half 0, head, page): the innermost is always 0 --
+// that completes on an mbarrier.
+__device__ __forceinline__ void tma_load_box(uint32_t dst, const CUtensorMap *map, int slot, int head, int page, uint32_t bar) {
     asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
-        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar) : "memory");
+        "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+        ::"r"(dst), "l"(map), "r"(0), "r"(slot), "r"(0), "r"(head), "r"(page), "r"(bar) : "memory");
 }
 
 __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
@@ -137,9 +138,12 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 }
 
 // Byte offset, inside a 64-token tile, of 16-byte piece `piece` (0..15) of token row `row`.
+// `sh` = log2(box_rows) (tiled only).
 template <bool kTiled>
-__device__ __forceinline__ uint32_t tile_offset(int row, int piece) {
-    if (kTiled) return (piece >> 3) * kHalfBytes + row * 128 + (((piece & 7) ^ (row & 7)) << 4);
+__device__ __forceinline__ uint32_t tile_offset(int row, int piece, int sh) {
+    if (kTiled)
+        return ((row >> sh) << (sh + 8)) + ((piece >> 3) << (sh + 7)) + ((row & ((1 << sh) - 1)) << 7) +
+               (((piece & 7) ^ (row & 7)) << 4);
     return row * kRowPitch + (piece << 4);
 }
 
@@ -189,22 +193,27 @@ gqa_paged_decode_kernel(const Params p, const __grid_constant__ CUtensorMap k_ma
     }
 
     // ---- the copy pipeline ----
-    // tiled: lane l of warp 0 brings one TMA box per chunk -- page l / 4 of the chunk, keys or values ((l / 2) % 2),
-    //        half l % 2 of the dims -- and only warp 0 arrives on the stage's barrier;
-    // rows:  thread i brings ONE token row per chunk -- row i % 64 of the keys (i < 64) or of the values -- and every
-    //        thread arrives, with its 256 bytes when its row exists.
+    // tiled: a chunk is 128 / box_rows boxes -- (page of the chunk, keys or values), both halves of the dims in one box
+    //        -- dealt out evenly to the four warps, one per lane: issuing a TMA copy costs its thread 50 to 90 cycles
+    //        whatever its size.  One warp issuing sixteen 2 KiB boxes per chunk of 16-token pages spent 1400 cycles
+    //        per chunk on it against 800 for the arithmetic, with the other warps waiting at the barrier;
+    // rows:  thread i brings ONE token row per chunk -- row i % 64 of the keys (i < 64) or of the values.
+    // Every thread arrives on the stage's barrier once per chunk, with its bytes when it has a copy to make.
     const int *page_list = p.kv_indices + p.kv_indptr[b];
     const size_t token_stride = (size_t)p.Hkv * kD;  // elements between consecutive slots of a page
     const uint32_t smem_base = smem_u32(smem), bar_base = smem_u32(full_bar);
-    const int my_row = kTiled ? (lane >> 2) * p.box_rows : (tid & (kChunk - 1));  // first row of the box / the row
-    const bool my_values = kTiled ? ((lane >> 1) & 1) : (tid >= kChunk);
+    const int sh = 31 - __clz(p.box_rows);                              // (tiled) log2 of the rows of a box
+    const int n_boxes = 2 * kChunk >> sh;                               // 2 (64-row boxes) .. 16 (8-row boxes)
+    const int boxes_per_warp = n_boxes >= kWarps ? n_boxes / kWarps : 1;
+    const int my_box = warp * boxes_per_warp + lane;                    // tiled: page my_box / 2 of the chunk, values?
+    const int my_row = kTiled ? (my_box >> 1) << sh : (tid & (kChunk - 1));  // first row of the box / the row
+    const bool my_values = kTiled ? (my_box & 1) : (tid >= kChunk);
     const __nv_bfloat16 *my_cache = (my_values ? p.v_cache : p.k_cache) + (size_t)kvh * kD;
     const uint32_t my_dst = (my_values ? (uint32_t)kTileBytes : 0u) +
-                            (kTiled ? (uint32_t)((lane & 1) * kHalfBytes + my_row * 128) : (uint32_t)(my_row * kRowPitch));
-    const bool copier = kTiled ? (warp == 0) : true;
-    const bool has_box = kTiled ? (my_row < kChunk) : true;  // (64 / box_rows pages per chunk)
+                            (kTiled ? (uint32_t)(my_row * kRowBytes) : (uint32_t)(my_row * kRowPitch));
+    const bool has_box = kTiled ? (lane < boxes_per_warp && my_box < n_boxes) : true;
     if (tid == 0) {
-        for (int s = 0; s < kStages; ++s) mbar_init(bar_base + s * 8, kTiled ? 32 : kThreads);
+        for (int s = 0; s < kStages; ++s) mbar_init(bar_base + s * 8, kThreads);
         gave_up = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -214,20 +223,20 @@ gqa_paged_decode_kernel(const Params p, const __grid_constant__ CUtensorMap k_ma
     // split.  The page table is read ONE CHUNK AHEAD of the copy that needs it, so its latency never sits between copies.
     auto locate = [&](int chunk) -> int {
         const int tok = begin + chunk * kChunk + my_row;
-        if (!copier || !has_box || chunk >= n_chunks || tok >= end) return -1;
+        if (!has_box || chunk >= n_chunks || tok >= end) return -1;
         const int page = __ldg(&page_list[tok / p.page_size]);
         return kTiled ? page : page * p.page_size + tok % p.page_size;
     };
     int next_loc = locate(0);
     auto issue_chunk = [&](int chunk) {  // called for chunk 0, 1, 2, ... in order
-        if (copier && chunk < n_chunks) {
+        if (chunk < n_chunks) {
             const int stage = chunk % kStages;
             const uint32_t dst = smem_base + stage * kStageBytes + my_dst, bar = bar_base + stage * 8;
             if (kTiled) {
                 if (next_loc >= 0) {
-                    mbar_arrive_expect_tx(bar, p.box_rows * 128);
-                    tma_load_4d(dst, my_values ? &v_map : &k_map, (lane & 1) * 64, kvh,
-                                (begin + chunk * kChunk + my_row) & (p.page_size - 1), next_loc, bar);
+                    mbar_arrive_expect_tx(bar, p.box_rows * kRowBytes);
+                    tma_load_box(dst, my_values ? &v_map : &k_map, (begin + chunk * kChunk + my_row) & (p.page_size - 1), kvh,
+                                 next_loc, bar);
                 } else {
                     mbar_arrive(bar);
                 }
@@ -283,20 +292,42 @@ gqa_paged_decode_kernel(const Params p, const __grid_constant__ CUtensorMap k_ma
                     const int r = i >> 4;
                     if (r >= valid)
                         asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};"
-                                     ::"r"(v_tile + tile_offset<true>(row_base + r, i & 15)), "r"(0) : "memory");
+                                     ::"r"(v_tile + tile_offset<true>(row_base + r, i & 15, sh)), "r"(0) : "memory");
                 }
                 __syncwarp();
             }
-            // S = Q K^T for 16 tokens: two n-tiles of 8 tokens, 8 K-steps
+            // S = Q K^T for 16 tokens: two n-tiles of 8 tokens, 8 K-steps.  A warp is one of one to three on its
+            // scheduler, so the latency of its own chain is what counts: fragments are fetched two steps ahead of the
+            // MMAs that use them, and even and odd K-steps accumulate separately (chains of four instead of eight).
             float s[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+            float s_odd[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
             const int m4 = lane >> 3, rr = lane & 7;
+            const int k_row = row_base + ((m4 >> 1) << 3) + rr, v_row = row_base + ((m4 & 1) << 3) + rr;
+            constexpr int kAhead = 2;
+            uint32_t kb[kAhead + 1][4];
+#pragma unroll
+            for (int ks = 0; ks < kAhead; ++ks) ldmatrix_x4(kb[ks], k_tile + tile_offset<kTiled>(k_row, 2 * ks + (m4 & 1), sh));
 #pragma unroll
             for (int ks = 0; ks < kD / 16; ++ks) {
-                uint32_t kb[4];
-                ldmatrix_x4(kb, k_tile + tile_offset<kTiled>(row_base + ((m4 >> 1) << 3) + rr, 2 * ks + (m4 & 1)));
-                mma_bf16(s[0], qa[ks], kb[0], kb[1]);
-                mma_bf16(s[1], qa[ks], kb[2], kb[3]);
+                if (ks + kAhead < kD / 16)
+                    ldmatrix_x4(kb[(ks + kAhead) % (kAhead + 1)], k_tile + tile_offset<kTiled>(k_row, 2 * (ks + kAhead) + (m4 & 1), sh));
+                const uint32_t(&f)[4] = kb[ks % (kAhead + 1)];
+                if (ks & 1) {
+                    mma_bf16(s_odd[0], qa[ks], f[0], f[1]);
+                    mma_bf16(s_odd[1], qa[ks], f[2], f[3]);
+                } else {
+                    mma_bf16(s[0], qa[ks], f[0], f[1]);
+                    mma_bf16(s[1], qa[ks], f[2], f[3]);
+                }
             }
+            // the first value fragments are on their way while the softmax runs
+            uint32_t vb[kAhead + 1][4];
+#pragma unroll
+            for (int j = 0; j < kAhead; ++j) ldmatrix_x4_trans(vb[j], v_tile + tile_offset<kTiled>(v_row, 2 * j + (m4 >> 1), sh));
+#pragma unroll
+            for (int n = 0; n < 2; ++n)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) s[n][i] += s_odd[n][i];
             // online softmax in the base-2 domain; columns past the end of the sequence are masked
             float row_max[2] = {-INFINITY, -INFINITY};
 #pragma unroll
@@ -348,11 +379,12 @@ gqa_paged_decode_kernel(const Params p, const __grid_constant__ CUtensorMap k_ma
                     for (int i = 0; i < 4; ++i) o_acc[n][i] *= alpha[i >> 1];
             }
 #pragma unroll
-            for (int n = 0; n < kD / 8; n += 2) {
-                uint32_t vb[4];
-                ldmatrix_x4_trans(vb, v_tile + tile_offset<kTiled>(row_base + ((m4 & 1) << 3) + rr, n + (m4 >> 1)));
-                mma_bf16(o_acc[n], pa, vb[0], vb[1]);
-                mma_bf16(o_acc[n + 1], pa, vb[2], vb[3]);
+            for (int j = 0; j < kD / 16; ++j) {  // n-tiles 2j and 2j + 1
+                if (j + kAhead < kD / 16)
+                    ldmatrix_x4_trans(vb[(j + kAhead) % (kAhead + 1)], v_tile + tile_offset<kTiled>(v_row, 2 * (j + kAhead) + (m4 >> 1), sh));
+                const uint32_t(&f)[4] = vb[j % (kAhead + 1)];
+                mma_bf16(o_acc[2 * j], pa, f[0], f[1]);
+                mma_bf16(o_acc[2 * j + 1], pa, f[2], f[3]);
             }
         }
     }
@@ -571,8 +603,8 @@ int gqa_paged_decode(const void *q, const void *k_cache, const void *v_cache, co
             return MOE_ERR_CUDA;
         attr_set[dev] = true;
     }
-    // Page sizes that are powers of two of at least 8 take the tiled gather: one 4-D tensor map per cache,
-    // (dims, key-value head, slot, page), a box of 64 dims x min(page_size, 64) slots in the 128-byte swizzle.
+    // Page sizes that are powers of two of at least 8 take the tiled gather: one 5-D tensor map per cache,
+    // (64 dims, slot, half, head, page), a box of min(page_size, 64) slots x both halves in the 128-byte swizzle.
     const bool tiled = page_size >= 8 && (page_size & (page_size - 1)) == 0 && num_pages > 0;
     CUtensorMap k_map, v_map;
     memset(&k_map, 0, sizeof(k_map));

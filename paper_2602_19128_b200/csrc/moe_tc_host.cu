@@ -111,14 +111,15 @@ bool encode(CUtensorMap *map, const void *base, int rank, const cuuint64_t *dims
 
 }  // namespace
 
-// 4-D bf16 tensor map of a paged key-value cache [num_pages, page_size, Hkv, 128] (decode attention): one box is
-// 64 dims x 1 head x box_rows slots x 1 page, in the 128-byte swizzle.
+// 5-D bf16 tensor map of a paged key-value cache [num_pages, page_size, Hkv, 128] (decode attention), with the
+// dimensions ordered (64 dims, slot, half of the dims, head, page) -- strides need not ascend -- so that one box,
+// 64 dims x box_rows slots x 2 halves of one head of one page, lands as two 128-byte-swizzled blocks of box_rows rows.
 bool encode_kv_cache_map(CUtensorMap *map, const void *cache, uint64_t num_pages, uint32_t page_size, uint32_t Hkv,
                          uint32_t box_rows) {
-    const cuuint64_t dims[4] = {128, Hkv, page_size, num_pages};
-    const cuuint64_t strides[3] = {128ull * 2, 128ull * 2 * Hkv, 128ull * 2 * Hkv * page_size};
-    const cuuint32_t box[4] = {64, 1, box_rows, 1};
-    return encode(map, cache, 4, dims, strides, box);
+    const cuuint64_t dims[5] = {64, page_size, 2, Hkv, num_pages};
+    const cuuint64_t strides[4] = {256ull * Hkv, 128, 256, 256ull * Hkv * page_size};
+    const cuuint32_t box[5] = {64, box_rows, 2, 1, 1};
+    return encode(map, cache, 5, dims, strides, box);
 }
 
 namespace {
