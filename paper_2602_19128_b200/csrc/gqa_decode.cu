@@ -194,9 +194,9 @@ gqa_paged_decode_kernel(const Params p, const __grid_constant__ CUtensorMap k_ma
 
     // ---- the copy pipeline ----
     // tiled: a chunk is 128 / box_rows boxes -- (page of the chunk, keys or values), both halves of the dims in one box
-    //        -- dealt out evenly to the four warps, one per lane: issuing a TMA copy costs its thread 50 to 90 cycles
-    //        whatever its size.  One warp issuing sixteen 2 KiB boxes per chunk of 16-token pages spent 1400 cycles
-    //        per chunk on it against 800 for the arithmetic, with the other warps waiting at the barrier;
+    //        -- dealt out evenly to the four warps, one per lane: a thread that issues a tiled copy is held 5 to 9
+    //        cycles per 128-byte row of the box.  One warp issuing all the boxes of a chunk spent 1400 cycles per chunk
+    //        on it against 800 for the arithmetic, with the other warps waiting at the barrier;
     // rows:  thread i brings ONE token row per chunk -- row i % 64 of the keys (i < 64) or of the values.
     // Every thread arrives on the stage's barrier once per chunk, with its bytes when it has a copy to make.
     const int *page_list = p.kv_indices + p.kv_indptr[b];
