@@ -449,38 +449,57 @@ gqa_paged_decode_kernel(const Params p, const __grid_constant__ CUtensorMap k_ma
     __threadfence();
     const float *all_o = p.part_o + bh * p.n_splits * p.group * kD;
     const float *all_ml = p.part_ml + bh * p.n_splits * p.group * 2;
-    // Scale factors of every (split, head) first, so that the sums below are streams of independent loads.
-    float *head_m = reinterpret_cast<float *>(smem);   // [16]
-    float *head_l = head_m + kRows;                      // [16]
-    float *scale = head_l + kRows;                       // [n_active][group]
-    __syncthreads();                                     // (the warps' merge buffer is free again)
+    // The merge is a chain of round trips to L2 for one block, so every step is laid out for loads in flight: the
+    // (max, sum) pairs of all splits come to shared memory in one sweep, the scale factors are computed from there,
+    // and the sum over the splits runs over all of a thread's outputs at once, eight splits deep.
+    float2 *ml = reinterpret_cast<float2 *>(smem);                       // [n_active][group] (max, sum)
+    float *scale = reinterpret_cast<float *>(ml + kMaxSplits * kRows);   // [n_active][group]
+    float *head_m = scale + kMaxSplits * kRows;                          // [16]
+    float *head_l = head_m + kRows;                                      // [16]
+    __syncthreads();                                                     // (the warps' merge buffer is free again)
+    for (int i = tid; i < n_active * p.group; i += kThreads) ml[i] = __ldcg(reinterpret_cast<const float2 *>(all_ml) + i);
+    __syncthreads();
     if (tid < p.group) {
         float m = -INFINITY;
-        for (int s = 0; s < n_active; ++s) m = fmaxf(m, __ldcg(&all_ml[(s * p.group + tid) * 2]));
+        for (int s = 0; s < n_active; ++s) m = fmaxf(m, ml[s * p.group + tid].x);
         head_m[tid] = m;
     }
     __syncthreads();
-    for (int i = tid; i < n_active * p.group; i += kThreads)
-        scale[i] = exp2f(__ldcg(&all_ml[i * 2]) - head_m[i % p.group]);
+    for (int i = tid; i < n_active * p.group; i += kThreads) scale[i] = exp2f(ml[i].x - head_m[i % p.group]);
     __syncthreads();
     if (tid < p.group) {
         float l = 0.f;
-        for (int s = 0; s < n_active; ++s) l += __ldcg(&all_ml[(s * p.group + tid) * 2 + 1]) * scale[s * p.group + tid];
+        for (int s = 0; s < n_active; ++s) l += ml[s * p.group + tid].y * scale[s * p.group + tid];  // ascending splits
         head_l[tid] = l;
         if (p.lse) p.lse[(size_t)b * p.Hq + head0 + tid] = (head_m[tid] + log2f(l)) * 0.6931471805599453f;
     }
     __syncthreads();
-    for (int i = tid; i < p.group * (kD / 4); i += kThreads) {  // one thread per (head, four dims)
-        const int g = i / (kD / 4), d = (i - g * (kD / 4)) * 4;
-        float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+    // thread t owns (head, four dims) items t, t + 128, ...: at most four (16 heads x 32 groups of four dims)
+    constexpr int kItems = kRows * (kD / 4) / kThreads;
+    const int n_items = p.group * (kD / 4);
+    float4 o[kItems];
+#pragma unroll
+    for (int j = 0; j < kItems; ++j) o[j] = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll 8
-        for (int s = 0; s < n_active; ++s) {  // ascending split order: the sum is the same whichever block is last
-            const float4 v = __ldcg(reinterpret_cast<const float4 *>(&all_o[(size_t)(s * p.group + g) * kD + d]));
-            const float f = scale[s * p.group + g];
-            o.x += v.x * f; o.y += v.y * f; o.z += v.z * f; o.w += v.w * f;
+    for (int s = 0; s < n_active; ++s) {  // ascending split order: the sum is the same whichever block is last
+#pragma unroll
+        for (int j = 0; j < kItems; ++j) {
+            const int i = tid + j * kThreads;
+            if (i < n_items) {
+                const int g = i / (kD / 4), d = (i - g * (kD / 4)) * 4;
+                const float4 v = __ldcg(reinterpret_cast<const float4 *>(&all_o[(size_t)(s * p.group + g) * kD + d]));
+                const float f = scale[s * p.group + g];
+                o[j].x += v.x * f; o[j].y += v.y * f; o[j].z += v.z * f; o[j].w += v.w * f;
+            }
         }
+    }
+#pragma unroll
+    for (int j = 0; j < kItems; ++j) {
+        const int i = tid + j * kThreads;
+        if (i >= n_items) break;
+        const int g = i / (kD / 4), d = (i - g * (kD / 4)) * 4;
         const float l = head_l[g];
-        __nv_bfloat162 lo = __floats2bfloat162_rn(o.x / l, o.y / l), hi = __floats2bfloat162_rn(o.z / l, o.w / l);
+        __nv_bfloat162 lo = __floats2bfloat162_rn(o[j].x / l, o[j].y / l), hi = __floats2bfloat162_rn(o[j].z / l, o[j].w / l);
         uint2 packed;
         packed.x = *reinterpret_cast<uint32_t *>(&lo);
         packed.y = *reinterpret_cast<uint32_t *>(&hi);
