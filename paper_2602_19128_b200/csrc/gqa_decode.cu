@@ -43,7 +43,11 @@ namespace tc {
 // 128-byte swizzle; encoded through the driver entry point and cached.
 bool encode_kv_cache_map(CUtensorMap *map, const void *cache, uint64_t num_pages, uint32_t page_size, uint32_t Hkv,
                          uint32_t box_rows);
+// (moe_tc_host.cu) cudaFuncAttributeMaxDynamicSharedMemorySize, set once per kernel and device, under a mutex.
+bool set_max_dynamic_smem_once(const void *kernel, int bytes);
 }  // namespace tc
+// (moe_api.cu) MOE_OK when the current device has compute capability 10.x (cached per device), else an error code.
+int check_device();
 }  // namespace moe
 
 namespace gqa {
@@ -586,11 +590,8 @@ int gqa_paged_decode(const void *q, const void *k_cache, const void *v_cache, co
         misaligned(workspace, 256))
         return MOE_ERR_ALIGN;
     if (workspace_bytes < gqa_decode_workspace_bytes(B, Hq, Hkv, D, max_kv_len)) return MOE_ERR_WORKSPACE;
-    int dev = 0, major = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
-        return MOE_ERR_CUDA;
-    if (major != 10) return MOE_ERR_ARCH;
+    const int arch = moe::check_device();
+    if (arch != MOE_OK) return arch;
 
     Params p;
     p.q = static_cast<const __nv_bfloat16 *>(q);
@@ -615,13 +616,9 @@ int gqa_paged_decode(const void *q, const void *k_cache, const void *v_cache, co
 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (cudaMemsetAsync(p.status, 0, 256 + bh * sizeof(int), st) != cudaSuccess) return MOE_ERR_CUDA;
-    static bool attr_set[64];
-    if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-        if (cudaFuncSetAttribute(gqa_paged_decode_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess ||
-            cudaFuncSetAttribute(gqa_paged_decode_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
-            return MOE_ERR_CUDA;
-        attr_set[dev] = true;
-    }
+    if (!moe::tc::set_max_dynamic_smem_once(reinterpret_cast<const void *>(gqa_paged_decode_kernel<true>), kSmemBytes) ||
+        !moe::tc::set_max_dynamic_smem_once(reinterpret_cast<const void *>(gqa_paged_decode_kernel<false>), kSmemBytes))
+        return MOE_ERR_CUDA;
     // Page sizes that are powers of two of at least 8 take the tiled gather: one 5-D tensor map per cache,
     // (64 dims, slot, half, head, page), a box of min(page_size, 64) slots x both halves in the 128-byte swizzle.
     const bool tiled = page_size >= 8 && (page_size & (page_size - 1)) == 0 && num_pages > 0;
