@@ -6,18 +6,20 @@
 //   * one block per (sequence split, key-value head, batch item); its 4 warps keep the 16 x 128 query tile of the
 //     group (Hq / Hkv heads, padded to the MMA's 16 rows) in registers, so a key or value byte is fetched from
 //     memory once for all heads of the group (Sec. 4.6 / Table 2: "fusing multiple query heads per KV head");
-//   * tokens arrive in chunks of 64 through a two-stage pipeline of TMA copies that follow the page table and
-//     complete on the stage's mbarrier ("vectorized/async paged-KV gather with pipelined global to shared memory
-//     prefetch"), three blocks per SM.  Page sizes that are powers of two of at least 8 take the TILED gather: the
-//     cache is a 5-D tensor (64 dims, slot, half of the dims, head, page) and one `cp.async.bulk.tensor` box brings a
-//     page's slots (up to 64) of one head as two 128-byte-swizzled blocks, so a chunk of 16-token pages is eight
-//     boxes, dealt out two to each warp (a thread is held 5 to 9 cycles per 128-byte row of a box it issues).
-//     Other page sizes take the ROW gather, one 256-byte `cp.async.bulk` per token row and thread into rows padded
-//     to 272 bytes.  What was measured on the way, B = 64 x 16k tokens: sixteen 16-byte cp.async per thread and
+//   * tokens arrive in chunks of 64 through a pipeline of TMA copies that follow the page table and complete on the
+//     stage's mbarrier ("vectorized/async paged-KV gather with pipelined global to shared memory prefetch").  Page
+//     sizes that are powers of two of at least 8 take the TILED gather: the cache is a 5-D tensor (64 dims, slot,
+//     half of the dims, head, page) and one `cp.async.bulk.tensor` box brings a page's slots (up to 64) of one head
+//     as two 128-byte-swizzled blocks, so a chunk of 16-token pages is eight boxes.  A fifth warp issues them and
+//     does nothing else, three stages deep, two blocks per SM; full / empty mbarriers hand the stages back and
+//     forth, and the compute warps' loop has no block-wide barrier.  Other page sizes take the ROW gather, one
+//     256-byte `cp.async.bulk` per token row and compute thread into rows padded to 272 bytes, two stages in three
+//     blocks per SM.  What was measured on the way, B = 64 x 16k tokens: sixteen 16-byte cp.async per thread and
 //     chunk, 4.0 TB/s (800 instructions per warp and chunk, instruction-latency bound at 8 warps per SM); the row
 //     gather 4.0 TB/s with and 5.2 TB/s without the arithmetic, one 256-byte request per 14 cycles and SM being all
-//     the copy engine took; the tiled gather 5.4 TB/s at 3 stages x 2 blocks, 6.1 TB/s at 2 stages x 3 blocks with
-//     one warp issuing, 6.3 TB/s with the boxes dealt out;
+//     the copy engine took; the tiled gather with one compute warp issuing 6.1 TB/s, with the boxes dealt out to
+//     the four compute warps 6.3 TB/s (a thread is held 5 to 9 cycles per 128-byte row of a box it issues), with
+//     the copy warp 6.6-6.9 TB/s, the measured copy bandwidth;
 //   * each warp owns 16 tokens of a chunk: S = Q K^T (mma.sync m16n8k16, bf16 in, fp32 out: the tile is 16 rows, far
 //     too small for a tcgen05 tile, and the kernel is bound by the copy stream), an online softmax in the base-2
 //     domain, O += P V with the probabilities re-used from the accumulator registers;
@@ -68,7 +70,10 @@ constexpr int kRowBytes = kD * 2;  // 256 bytes per token and head in the cache
 constexpr int kRowPitch = kRowBytes + 16;
 constexpr int kTileBytes = kChunk * kRowPitch;        // 17 KiB, a multiple of 1024 (the swizzle's alignment)
 constexpr int kStageBytes = 2 * kTileBytes;           // keys, then values: 34 KiB
+constexpr int kModelBlocksPerSm = 2;  // blocks per SM the split model counts with (the copy-warp variant's)
+constexpr int kStagesProducer = 3;  // the variant with a copy warp: three stages in each of two blocks per SM
 constexpr int kSmemBytes = kStages * kStageBytes + 1024;  // (the base is rounded up to 1024 bytes)
+constexpr int kSmemBytesProducer = kStagesProducer * kStageBytes + 1024;
 static_assert(kTileBytes % 1024 == 0, "tiles must keep the swizzle's alignment");
 constexpr int kWaitLimit = 1 << 22;                   // polls of a stage's barrier before the block gives up
 constexpr int kMaxSplits = 128;
@@ -151,15 +156,27 @@ __device__ __forceinline__ uint32_t tile_offset(int row, int piece, int sh) {
     return row * kRowPitch + (piece << 4);
 }
 
-// kTiled: the page size is a power of two of at least 8, and the gather is one TMA tile per (page, half of the
-// dims, keys or values); otherwise one 256-byte bulk copy per token row.
+// kTiled: the page size is a power of two of at least 8, and the gather is one TMA box per (page, keys or values),
+// issued by a fifth warp that does nothing else, three stages deep, in two blocks per SM: the four compute warps never
+// touch the copy engine, and stages are handed back and forth on full / empty mbarriers, so the loop has no block-wide
+// barrier.  (A thread is held for as long as the engine takes to turn its box into requests, 5 to 9 cycles per
+// 128-byte row: 600 cycles per chunk and warp when the four compute warps shared the issuing, against 1000 for the
+// arithmetic.)  Otherwise: one 256-byte bulk copy per token row, issued by the 128 compute threads themselves, two
+// stages in three blocks per SM, a block barrier per chunk.
 template <bool kTiled>
-__global__ void __launch_bounds__(kThreads, kBlocksPerSm)
+__global__ void __launch_bounds__(kTiled ? kThreads + 32 : kThreads, kTiled ? 2 : kBlocksPerSm)
 gqa_paged_decode_kernel(const Params p, const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map) {
+    constexpr bool kProducer = kTiled;  // a copy warp
+    constexpr int kNumStages = kProducer ? kStagesProducer : kStages;
     extern __shared__ __align__(128) uint8_t smem_raw[];
     uint8_t *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     __shared__ int is_last, gave_up;
-    __shared__ __align__(8) unsigned long long full_bar[kStages];
+    __shared__ __align__(8) unsigned long long full_bar[kStagesProducer], empty_bar[kStagesProducer];
+    // the compute warps' barrier: the whole block without a copy warp, a named barrier of 128 threads with one
+    auto sync_compute = [&]() {
+        if (kProducer) asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory");
+        else __syncthreads();
+    };
     const int split = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int pages = p.kv_indptr[b + 1] - p.kv_indptr[b];
@@ -167,7 +184,7 @@ gqa_paged_decode_kernel(const Params p, const __grid_constant__ CUtensorMap k_ma
     const int head0 = kvh * p.group;
 
     if (L <= 0) {  // nothing cached: out = 0, lse = -inf (written by the first split's block)
-        if (split == 0) {
+        if (split == 0 && tid < kThreads) {
             for (int i = tid; i < p.group * kD; i += kThreads)
                 p.out[((size_t)b * p.Hq + head0 + i / kD) * kD + (i % kD)] = __float2bfloat16_rn(0.f);
             if (p.lse && tid < p.group) p.lse[(size_t)b * p.Hq + head0 + tid] = -INFINITY;
@@ -198,26 +215,27 @@ gqa_paged_decode_kernel(const Params p, const __grid_constant__ CUtensorMap k_ma
 
     // ---- the copy pipeline ----
     // tiled: a chunk is 128 / box_rows boxes -- (page of the chunk, keys or values), both halves of the dims in one box
-    //        -- dealt out evenly to the four warps, one per lane: a thread that issues a tiled copy is held 5 to 9
-    //        cycles per 128-byte row of the box.  One warp issuing all the boxes of a chunk spent 1400 cycles per chunk
-    //        on it against 800 for the arithmetic, with the other warps waiting at the barrier;
+    //        -- one per lane of the copy warp, which alone arrives on the stage's barrier;
     // rows:  thread i brings ONE token row per chunk -- row i % 64 of the keys (i < 64) or of the values.
-    // Every thread arrives on the stage's barrier once per chunk, with its bytes when it has a copy to make.
+    //        Every thread arrives on the stage's barrier once per chunk, with its bytes when its row exists.
     const int *page_list = p.kv_indices + p.kv_indptr[b];
     const size_t token_stride = (size_t)p.Hkv * kD;  // elements between consecutive slots of a page
     const uint32_t smem_base = smem_u32(smem), bar_base = smem_u32(full_bar);
     const int sh = 31 - __clz(p.box_rows);                              // (tiled) log2 of the rows of a box
     const int n_boxes = 2 * kChunk >> sh;                               // 2 (64-row boxes) .. 16 (8-row boxes)
-    const int boxes_per_warp = n_boxes >= kWarps ? n_boxes / kWarps : 1;
-    const int my_box = warp * boxes_per_warp + lane;                    // tiled: page my_box / 2 of the chunk, values?
+    const int my_box = lane;                                            // tiled: page my_box / 2 of the chunk, values?
     const int my_row = kTiled ? (my_box >> 1) << sh : (tid & (kChunk - 1));  // first row of the box / the row
     const bool my_values = kTiled ? (my_box & 1) : (tid >= kChunk);
     const __nv_bfloat16 *my_cache = (my_values ? p.v_cache : p.k_cache) + (size_t)kvh * kD;
     const uint32_t my_dst = (my_values ? (uint32_t)kTileBytes : 0u) +
                             (kTiled ? (uint32_t)(my_row * kRowBytes) : (uint32_t)(my_row * kRowPitch));
-    const bool has_box = kTiled ? (lane < boxes_per_warp && my_box < n_boxes) : true;
+    const bool has_box = kTiled ? (warp == kWarps && my_box < n_boxes) : true;
+    const uint32_t empty_base = smem_u32(empty_bar);
     if (tid == 0) {
-        for (int s = 0; s < kStages; ++s) mbar_init(bar_base + s * 8, kThreads);
+        for (int s = 0; s < kNumStages; ++s) {
+            mbar_init(bar_base + s * 8, kProducer ? 32 : kThreads);  // arrivals per chunk: the copy warp's lanes / every thread
+            mbar_init(empty_base + s * 8, kWarps);                    // (copy-warp variant) one arrival per compute warp
+        }
         gave_up = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -234,7 +252,7 @@ gqa_paged_decode_kernel(const Params p, const __grid_constant__ CUtensorMap k_ma
     int next_loc = locate(0);
     auto issue_chunk = [&](int chunk) {  // called for chunk 0, 1, 2, ... in order
         if (chunk < n_chunks) {
-            const int stage = chunk % kStages;
+            const int stage = chunk % kNumStages;
             const uint32_t dst = smem_base + stage * kStageBytes + my_dst, bar = bar_base + stage * 8;
             if (kTiled) {
                 if (next_loc >= 0) {
@@ -256,9 +274,8 @@ gqa_paged_decode_kernel(const Params p, const __grid_constant__ CUtensorMap k_ma
         }
         next_loc = locate(chunk + 1);
     };
-    // Bounded wait for a chunk; false once any thread of the block has given up.
-    auto wait_chunk = [&](int chunk) -> bool {
-        const uint32_t bar = bar_base + (chunk % kStages) * 8, parity = (uint32_t)(chunk / kStages) & 1u;
+    // Bounded wait on a barrier; false once any thread of the block has given up.
+    auto wait_bar = [&](uint32_t bar, uint32_t parity) -> bool {
         for (int i = 0; i < kWaitLimit; ++i) {
             if (mbar_try_wait(bar, parity)) return true;
             if (*(volatile int *)&gave_up) return false;
@@ -267,6 +284,21 @@ gqa_paged_decode_kernel(const Params p, const __grid_constant__ CUtensorMap k_ma
         if (atomicCAS(p.status, 0, (int)MOE_ERR_DEVICE_TIMEOUT) == 0) { p.status[1] = 12; p.status[2] = blockIdx.x; }
         return false;
     };
+    auto wait_chunk = [&](int chunk) -> bool {
+        return wait_bar(bar_base + (chunk % kNumStages) * 8, (uint32_t)(chunk / kNumStages) & 1u);
+    };
+
+    if (kProducer && warp == kWarps) {
+        // ---- the copy warp: chunk after chunk into the ring, each stage as soon as the four compute warps are done
+        // with its previous use ----
+        for (int chunk = 0; chunk < n_chunks; ++chunk) {
+            const int use = chunk / kNumStages;
+            bool free_ = use == 0 || wait_bar(empty_base + (chunk % kNumStages) * 8, (uint32_t)(use - 1) & 1u);
+            if (!__all_sync(0xffffffffu, free_)) break;
+            issue_chunk(chunk);
+        }
+        return;
+    }
 
     float o_acc[kD / 8][4];  // this warp's 16 x 128 output tile: 16 n-tiles of 8 dims
 #pragma unroll
@@ -275,15 +307,21 @@ gqa_paged_decode_kernel(const Params p, const __grid_constant__ CUtensorMap k_ma
         for (int i = 0; i < 4; ++i) o_acc[n][i] = 0.f;
     float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};  // rows lane/4 and lane/4 + 8
 
-    for (int c = 0; c < kStages - 1; ++c) issue_chunk(c);
+    if (!kProducer)
+        for (int c = 0; c < kNumStages - 1; ++c) issue_chunk(c);
     bool ok = true;
     for (int chunk = 0; chunk < n_chunks; ++chunk) {
         ok = wait_chunk(chunk);
-        ok = __syncthreads_and(ok);           // chunk `chunk` has landed; every thread is done with chunk - 1's stage
-        if (!ok) break;
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // (that stage is about to be overwritten by copies)
-        issue_chunk(chunk + kStages - 1);
-        const uint32_t k_tile = smem_base + (chunk % kStages) * kStageBytes, v_tile = k_tile + kTileBytes;
+        if (kProducer) {
+            ok = __all_sync(0xffffffffu, ok);     // chunk `chunk` has landed
+            if (!ok) break;
+        } else {
+            ok = __syncthreads_and(ok);           // ... and every thread is done with chunk - 1's stage
+            if (!ok) break;
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // (that stage is about to be overwritten by copies)
+            issue_chunk(chunk + kNumStages - 1);
+        }
+        const uint32_t k_tile = smem_base + (chunk % kNumStages) * kStageBytes, v_tile = k_tile + kTileBytes;
         const int row_base = warp * 16;       // this warp's tokens of the chunk
         const int tok_base = begin + chunk * kChunk + row_base;
         if (tok_base < end) {                 // (uniform over the warp)
@@ -391,13 +429,22 @@ gqa_paged_decode_kernel(const Params p, const __grid_constant__ CUtensorMap k_ma
                 mma_bf16(o_acc[2 * j + 1], pa, f[2], f[3]);
             }
         }
+        if (kProducer) {  // this warp is done with the stage (also when none of its tokens exist)
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty_base + (chunk % kNumStages) * 8);
+        }
+    }
+    // every warp is done with the pipeline's shared memory (all copies were waited for): it becomes the merge buffer
+    if (kProducer) {
+        sync_compute();
+        ok = *(volatile int *)&gave_up == 0;
     }
     // A block that gave up waits (bounded) for its copies in flight, then leaves without a result: the status word says so.
     if (!ok) {
         for (int i = 0; i < 1000; ++i) __nanosleep(1000);
         return;
     }
-    __syncthreads();  // every warp is done with the pipeline's shared memory (all copies were waited for): the merge buffer
+    if (!kProducer) __syncthreads();
 
     // ---- merge the four warps: (max, sum, O) per head, in warp order ----
     float *merge_o = reinterpret_cast<float *>(smem);                    // [4 warps][16 rows][128]
@@ -417,7 +464,7 @@ gqa_paged_decode_kernel(const Params p, const __grid_constant__ CUtensorMap k_ma
             merge_ml[(warp * kRows + r0 + 8) * 2 + 1] = l_run[1];
         }
     }
-    __syncthreads();
+    sync_compute();
     const size_t bh = (size_t)b * p.Hkv + kvh;
     float *part_o = p.part_o + (bh * p.n_splits + split) * p.group * kD;
     float *part_ml = p.part_ml + (bh * p.n_splits + split) * p.group * 2;
@@ -446,9 +493,9 @@ gqa_paged_decode_kernel(const Params p, const __grid_constant__ CUtensorMap k_ma
 
     // ---- the block that arrives last merges the splits (Sec. 4.6: "detects that it is last via a lightweight counter") ----
     __threadfence();
-    __syncthreads();
+    sync_compute();
     if (tid == 0) is_last = atomicAdd(&p.counters[bh], 1) == n_active - 1;
-    __syncthreads();
+    sync_compute();
     if (!is_last) return;
     __threadfence();
     const float *all_o = p.part_o + bh * p.n_splits * p.group * kD;
@@ -460,24 +507,24 @@ gqa_paged_decode_kernel(const Params p, const __grid_constant__ CUtensorMap k_ma
     float *scale = reinterpret_cast<float *>(ml + kMaxSplits * kRows);   // [n_active][group]
     float *head_m = scale + kMaxSplits * kRows;                          // [16]
     float *head_l = head_m + kRows;                                      // [16]
-    __syncthreads();                                                     // (the warps' merge buffer is free again)
+    sync_compute();                                                     // (the warps' merge buffer is free again)
     for (int i = tid; i < n_active * p.group; i += kThreads) ml[i] = __ldcg(reinterpret_cast<const float2 *>(all_ml) + i);
-    __syncthreads();
+    sync_compute();
     if (tid < p.group) {
         float m = -INFINITY;
         for (int s = 0; s < n_active; ++s) m = fmaxf(m, ml[s * p.group + tid].x);
         head_m[tid] = m;
     }
-    __syncthreads();
+    sync_compute();
     for (int i = tid; i < n_active * p.group; i += kThreads) scale[i] = exp2f(ml[i].x - head_m[i % p.group]);
-    __syncthreads();
+    sync_compute();
     if (tid < p.group) {
         float l = 0.f;
         for (int s = 0; s < n_active; ++s) l += ml[s * p.group + tid].y * scale[s * p.group + tid];  // ascending splits
         head_l[tid] = l;
         if (p.lse) p.lse[(size_t)b * p.Hq + head0 + tid] = (head_m[tid] + log2f(l)) * 0.6931471805599453f;
     }
-    __syncthreads();
+    sync_compute();
     // thread t owns (head, four dims) items t, t + 128, ...: at most four (16 heads x 32 groups of four dims)
     constexpr int kItems = kRows * (kD / 4) / kThreads;
     const int n_items = p.group * (kD / 4);
@@ -517,17 +564,19 @@ bool envelope_ok(long long B, int Hq, int Hkv, int D, long long max_kv_len) {
     return B <= 65535 && Hkv <= 65535;  // grid dimensions y and z
 }
 
-// Sequence splits, from a model of the kernel's time in units of one chunk streamed by a block on a full machine.
-// 148 SMs x kBlocksPerSm blocks are resident at a time, so blocks run in waves; a block costs its chunks plus 4
-// (pipeline fill and the warps' merge, partly hidden behind the SM's other blocks); a wave that fills a fraction f of
-// the machine runs in max(0.57, 0.3 + 0.7 f) of a full wave's time (a block alone streams a chunk in 0.57 of the
-// time); a split sequence pays the partial results' round trip and the last block's merge once, 8 + n / 4; and 0.3 of
-// a block's length is added for the tail that sequences shorter than max_kv_len leave (their lengths are known to the
-// device only).  The constants were fitted to measured split sweeps (batches of 1 to 256, 2k to 128k tokens, equal
-// and ragged lengths); the chosen count was within 10 % of the best measured one in each.  Ties go to fewer splits;
-// no split is shorter than four chunks.
+// Sequence splits, from a model of the kernel's time in units of one chunk streamed by a block on a full machine
+// (1.4 us).  148 SMs x 2 blocks are resident at a time (the copy-warp variant), so blocks run in waves; a block costs
+// its chunks plus 3 (pipeline fill, the warps' merge); a wave that fills a fraction f of the machine runs in
+// max(0.47, f) of a full wave's time (a block alone streams a chunk in 0.47 of the time, and 0.86 of a wave already
+// saturates the memory); a split sequence pays the partial results' round trip and the last block's merge once,
+// 5 + n / 10; and while the machine is not full, 0.3 x (the idle share) of a block's length is added for the tail that
+// sequences shorter than max_kv_len leave (their lengths are known to the device only; on a full machine the blocks
+// that remain speed up as others finish, on a part-empty one they already run at their own limit).  The constants
+// were fitted to measured split sweeps (batches of 1 to 256, 2k to 64k tokens, equal and ragged lengths); the chosen
+// count was within 10 % of the best measured one in each.  Ties go to fewer splits; no split is shorter than four
+// chunks.
 void choose_split(int B, int Hkv, int max_kv_len, int *split_tokens, int *n_splits) {
-    const long long base = (long long)B * Hkv, slots = 148 * kBlocksPerSm;
+    const long long base = (long long)B * Hkv, slots = 148 * kModelBlocksPerSm;
     const long long chunks = max_kv_len > 0 ? ((long long)max_kv_len + kChunk - 1) / kChunk : 1;
     long long most = (chunks + 3) / 4;
     if (most > kMaxSplits) most = kMaxSplits;
@@ -539,9 +588,10 @@ void choose_split(int B, int Hkv, int max_kv_len, int *split_tokens, int *n_spli
         if (n_eff != n) continue;  // (the same split as a smaller n)
         const long long blocks = (base > 0 ? base : 1) * n, full_waves = blocks / slots;
         const double f = (double)(blocks - full_waves * slots) / (double)slots;
-        const double last_wave = f > 0.0 ? (0.3 + 0.7 * f > 0.57 ? 0.3 + 0.7 * f : 0.57) : 0.0;
-        const double cost = ((double)per_block + 4.0) * ((double)full_waves + last_wave) + 0.3 * (double)per_block +
-                            (n > 1 ? 8.0 + 0.25 * (double)n : 0.0);
+        const double last_wave = f > 0.0 ? (f > 0.47 ? f : 0.47) : 0.0;
+        const double idle = blocks < slots ? 1.0 - (double)blocks / (double)slots : 0.0;
+        const double cost = ((double)per_block + 3.0) * ((double)full_waves + last_wave) +
+                            0.3 * idle * (double)per_block + (n > 1 ? 5.0 + 0.1 * (double)n : 0.0);
         if (best_cost < 0 || cost < best_cost * (1.0 - 1e-9)) { best_cost = cost; best_n = n; }
     }
     const long long per_block = (chunks + best_n - 1) / best_n;
@@ -616,7 +666,7 @@ int gqa_paged_decode(const void *q, const void *k_cache, const void *v_cache, co
 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (cudaMemsetAsync(p.status, 0, 256 + bh * sizeof(int), st) != cudaSuccess) return MOE_ERR_CUDA;
-    if (!moe::tc::set_max_dynamic_smem_once(reinterpret_cast<const void *>(gqa_paged_decode_kernel<true>), kSmemBytes) ||
+    if (!moe::tc::set_max_dynamic_smem_once(reinterpret_cast<const void *>(gqa_paged_decode_kernel<true>), kSmemBytesProducer) ||
         !moe::tc::set_max_dynamic_smem_once(reinterpret_cast<const void *>(gqa_paged_decode_kernel<false>), kSmemBytes))
         return MOE_ERR_CUDA;
     // Page sizes that are powers of two of at least 8 take the tiled gather: one 5-D tensor map per cache,
@@ -630,7 +680,7 @@ int gqa_paged_decode(const void *q, const void *k_cache, const void *v_cache, co
                   !moe::tc::encode_kv_cache_map(&v_map, v_cache, (uint64_t)num_pages, (uint32_t)page_size, (uint32_t)Hkv, (uint32_t)p.box_rows)))
         return MOE_ERR_CUDA;
     const dim3 grid(p.n_splits, Hkv, B);
-    if (tiled) gqa_paged_decode_kernel<true><<<grid, kThreads, kSmemBytes, st>>>(p, k_map, v_map);
+    if (tiled) gqa_paged_decode_kernel<true><<<grid, kThreads + 32, kSmemBytesProducer, st>>>(p, k_map, v_map);
     else gqa_paged_decode_kernel<false><<<grid, kThreads, kSmemBytes, st>>>(p, k_map, v_map);
     return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
