@@ -13,7 +13,7 @@ PKG = Path(__file__).resolve().parent
 ROOT = PKG.parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libmoe_b200.so"
-SOURCES = ["moe_api.cu", "moe_route.cu", "moe_gemm_tc.cu", "moe_gemm_tc_pair.cu", "moe_gemm_tc_ring.cu", "moe_gemm_tc_fp8w.cu", "moe_gemm_tc_mx.cu", "moe_gemm_tc_mx_pair.cu", "moe_mx.cu", "moe_tc_host.cu", "moe_gemm_validation.cu", "gqa_decode.cu"]
+SOURCES = ["moe_api.cu", "moe_route.cu", "moe_gemm_tc.cu", "moe_gemm_tc_pair.cu", "moe_gemm_tc_ring.cu", "moe_gemm_tc_fp8w.cu", "moe_gemm_tc_mx.cu", "moe_gemm_tc_mx_pair.cu", "moe_gemm_tc_mx_ring.cu", "moe_mx.cu", "moe_tc_host.cu", "moe_gemm_validation.cu", "gqa_decode.cu"]
 
 
 def _nvcc() -> str:

@@ -215,14 +215,17 @@ int forward_impl(const void *x, const float *logits, const void *w13, const void
 // ---- MX FP8 ---------------------------------------------------------------------------------------------
 bool mx_envelope_ok(long long T, int H, int I, int E, int k) { return envelope_ok(T, H, I, E, k) && I % 128 == 0; }
 
-// Token-tile rows of the MX path.  Scale columns sit next to the two accumulators in tensor memory, so the
-// largest tile is 240 rows (2 * 240 + 32 columns); only the CTA-pair kernel has the instances above 128 rows,
-// and its down projection needs H to be a multiple of its 256-row tile.  160-row tiles (a deeper ring) are
-// taken when the mean rows per expert plus 2.5 standard deviations of a uniform routing still fit.
+// Token-tile rows of the MX path.  Scale columns sit next to the accumulators in tensor memory, so the largest tile
+// of the kernel with two fixed accumulators is 240 rows (2 * 240 + 32 columns); only the CTA-pair kernels have the
+// instances above 128 rows, and their down projection needs H to be a multiple of the 256-row pair tile.  Where the
+// bf16 layer takes its wide tiles (160 to 352 rows per expert on average) so does this one: 320 or 384 rows on the
+// accumulator ring, one pass over an expert's weights.  160-row tiles (a deeper ring) are taken when the mean rows per
+// expert plus 2.5 standard deviations of a uniform routing still fit.
 int mx_tile_rows(int T, int H, int E, int k) {
-    const int nt = choose_nt_max(T, E, k);
+    const int nt = choose_nt_max(T, E, k, true);
     if (nt <= 128) return nt;
     if (H % 256 != 0) return 128;
+    if (nt > 256) return nt;
     const double mean = (double)T * k / E;
     return mean + 2.5 * sqrt(mean) <= 160.0 ? 160 : 240;
 }
@@ -322,6 +325,7 @@ int forward_mx_impl(const void *x, const float *logits, const void *w13_q, const
     g1.handover = g2.handover = status;
     g2.handover_per_token_tile = handover_counts_per_token_tile(I);
     auto run = [&](const MxGemmArgs &g) {
+        if (grouped_gemm_tc_mx_ring_applies(g)) return launch_grouped_gemm_tc_mx_ring(g, stream);
         return grouped_gemm_tc_mx_pair_applies(g) ? launch_grouped_gemm_tc_mx_pair(g, stream) : launch_grouped_gemm_tc_mx(g, stream);
     };
     int st = run(g1);

@@ -42,6 +42,7 @@ constexpr int kNumChunks = 32;      // 512 columns of tensor memory
 constexpr int kAccFullBars = 32;    // tiles between the MMA warp and the epilogue: each holds at least one chunk
 constexpr int kTileQueue = 16;      // more entries than ring slots: the producer is at most STAGES tiles ahead
 constexpr int kRingActMaps = 24;    // act[i]: box of 8 * (i + 1) rows, up to 192 rows per CTA (N = 384)
+constexpr int kOutStageBytes = 16 * kTileM * 2;  // one 16-column group of a CTA's 128 output rows, token-major
 
 struct RingMaps {
     CUtensorMap w;
@@ -75,7 +76,8 @@ struct RingSmem {
     static constexpr int kSlotBBytes = (NT_MAX / 2) * kRowBytes;
     static constexpr int kA = 0;
     static constexpr int kB = STAGES * kSlotABytes;
-    static constexpr int kBars = kB + STAGES * kSlotBBytes;  // full[S], empty[S], acc_full[32], acc_empty[32]
+    static constexpr int kOutStage = kB + STAGES * kSlotBBytes;  // down projection: two [16 tokens][128 rows] bf16 tiles
+    static constexpr int kBars = kOutStage + 2 * kOutStageBytes;  // full[S], empty[S], acc_full[32], acc_empty[32]
     static constexpr int kQueue = kBars + (2 * STAGES + kAccFullBars + kNumChunks) * 8;
     static constexpr int kTmemSlot = kQueue + kTileQueue * 4;
     static constexpr int kAbort = kTmemSlot + 4;
@@ -292,7 +294,7 @@ grouped_gemm_tc_ring_kernel(const __grid_constant__ RingMaps maps, const KernelP
         // ---------------- epilogue (both CTAs): own 128 weight rows x all N tokens ----------------
         const int q = warp & 3;  // a warp may only read TMEM lanes 32*(warp%4) .. +31
         const uint32_t lane_base = tmem_base + ((uint32_t)(q * 32) << 16);
-        int seq = 0;
+        int seq = 0, out_flip = 0;
         bool ok = true;
         for (int round = 0; ok; ++round, ++seq) {
             const int tile = tile_of_round(round, pair, n_pairs);
@@ -302,11 +304,11 @@ grouped_gemm_tc_ring_kernel(const __grid_constant__ RingMaps maps, const KernelP
             const Parts parts = split_tile(seq, n_mma);
             ok = pair_wait(bar_acc_full + (seq & (kAccFullBars - 1)) * 8, (uint32_t)(seq / kAccFullBars) & 1u, abort_flag, peer_abort,
                            p.status, kSiteEpilogueTmemFull + kSiteOffset);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
+            if (epilogue_any(!ok)) break;  // the four warps synchronise inside a down-projection tile: they leave together
             tcgen05_fence_after();
             const int lane_feat = SWIGLU ? q * 16 + (lane & 15) : q * 32 + lane;
-            __nv_bfloat16 *dst = p.out + (size_t)t.row0 * p.n_out + t.f * kFeatPerTile + (int)rank * kFeatPerCta + lane_feat;
+            __nv_bfloat16 *dst_rows = p.out + (size_t)t.row0 * p.n_out + t.f * kFeatPerTile + (int)rank * kFeatPerCta;
+            __nv_bfloat16 *dst = dst_rows + lane_feat;
             const size_t row_stride = (size_t)p.n_out;
             // An even tile is drained from its highest 16 columns down, an odd tile from its lowest up: the columns the
             // next tile of this pair is waiting for go back first.
@@ -343,13 +345,22 @@ grouped_gemm_tc_ring_kernel(const __grid_constant__ RingMaps maps, const KernelP
                         out_row += row_stride;
                     }
                 } else {
-                    __nv_bfloat16 *out_a = dst + (size_t)row_a * row_stride, *out_b = dst + (size_t)row_b * row_stride;
+                    // A lane holds one output feature of 16 tokens; stored from here a warp instruction would write
+                    // 32 x 2 bytes of one token.  The four warps transpose the group through shared memory instead and
+                    // each stores four whole 256-byte token rows, 16 bytes per lane.
+                    out_flip ^= 1;  // (across tiles too: two consecutive groups never share a buffer)
+                    uint8_t *stage_buf = base_ptr + L::kOutStage + out_flip * kOutStageBytes;
 #pragma unroll
-                    for (int u = 0; u < 8; ++u) {
-                        if (all_valid || row_a + u < t.n_valid) *out_a = __float2bfloat16_rn(v[u]);
-                        if (all_valid || row_b + u < t.n_valid) *out_b = __float2bfloat16_rn(v[8 + u]);
-                        out_a += row_stride;
-                        out_b += row_stride;
+                    for (int i = 0; i < 16; ++i)
+                        reinterpret_cast<__nv_bfloat16 *>(stage_buf)[i * kTileM + q * 32 + lane] = __float2bfloat16_rn(v[i]);
+                    asm volatile("bar.sync 2, 128;" ::: "memory");  // (two buffers: the next group's writes cannot pass this)
+#pragma unroll
+                    for (int it = 0; it < 2; ++it) {
+                        const int r = q * 4 + it * 2 + (lane >> 4);          // column of the group
+                        const int row = r < 8 ? row_a + r : row_b + r - 8;   // ... and its tile row
+                        const uint4 val = *reinterpret_cast<const uint4 *>(stage_buf + r * (kTileM * 2) + (lane & 15) * 16);
+                        if (row < t.n_valid)
+                            *reinterpret_cast<uint4 *>(dst_rows + (size_t)row * row_stride + (lane & 15) * 8) = val;
                     }
                 }
             }

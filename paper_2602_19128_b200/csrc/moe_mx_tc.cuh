@@ -73,19 +73,6 @@ __device__ __forceinline__ uint32_t instr_desc_mx(int m, int n, int sf) {
            ((uint32_t)sf << 29);
 }
 
-// OR of `flag` over the 128 epilogue threads (named barrier 1), so that they leave their loop together.
-__device__ __forceinline__ bool epilogue_any(bool flag) {
-    uint32_t r;
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t"
-        "setp.ne.u32 q, %1, 0;\n\t"
-        "bar.red.or.pred p, 1, 128, q;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(r)
-        : "r"((uint32_t)flag)
-        : "memory");
-    return r != 0;
-}
 // Barrier of the two epilogue warps (64 threads) that share a block of 32 features.
 __device__ __forceinline__ void pair_sync(int pair) {
     asm volatile("bar.sync %0, 64;" ::"r"(2 + pair) : "memory");

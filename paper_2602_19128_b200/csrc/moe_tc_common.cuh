@@ -177,6 +177,19 @@ __device__ __forceinline__ uint32_t instr_desc_bf16(int m, int n) {
 // were encoded with: 16 rows up to 256 for the one-CTA kernel, 8 rows up to 128 for each CTA of a pair).
 // One copy per ring slot and operand: every TMA copy has a fixed cost in the copy engine that is
 // comparable to moving several KiB, so a token tile is never assembled from smaller boxes.
+// OR of `flag` over the 128 epilogue threads (named barrier 1), so that they leave their loop together.
+__device__ __forceinline__ bool epilogue_any(bool flag) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 q, %1, 0;\n\t"
+        "bar.red.or.pred p, 1, 128, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(r)
+        : "r"((uint32_t)flag)
+        : "memory");
+    return r != 0;
+}
 template <int kQuantum>
 __device__ __forceinline__ const CUtensorMap *act_map(const TensorMaps &maps, int n_rows) {
     return &maps.act[n_rows / kQuantum - 1];

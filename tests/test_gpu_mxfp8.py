@@ -109,10 +109,10 @@ CASES = [
     (128, 384, 128, 256, 8, False),   # decode-like
     (200, 256, 384, 8, 2, False),     # ~50 rows per expert
     (300, 128, 128, 64, 4, True),     # skewed, empty experts, several tiles for the popular ones
-    (700, 256, 256, 4, 2, False),     # ~350 rows per expert: three tiles of up to 128 rows, second atoms
+    (700, 256, 256, 4, 2, False),     # ~350 rows per expert: one wide tile each (bound 384: two MMA parts, three atoms)
     (96, 128, 256, 8, 8, False),
     (513, 128, 128, 2, 1, False),     # ~256 rows per expert; H not a multiple of 256: one-CTA kernel, 128-row tiles
-    (513, 256, 128, 2, 1, False),     # the same on CTA pairs: 240-row tiles (two scale atoms) and a ragged one
+    (513, 256, 128, 2, 1, False),     # the same on CTA pairs: wide tiles, bound 320
     (1000, 512, 384, 4, 2, False),    # ~500 rows per expert: three pair tiles each, several feature tiles
     (130, 256, 256, 4, 2, False),     # 128-row pair tiles (one atom each)
     (300, 256, 128, 16, 4, True),     # the same, skewed: popular experts spill into a second tile
@@ -120,6 +120,10 @@ CASES = [
     (2000, 128, 128, 1, 1, False),    # one expert, sixteen 128-row tiles: gate/up on pairs, down (H % 256 != 0) on one CTA
     (2000, 256, 128, 1, 1, False),    # one expert, nine 240-row tiles on pairs
     (33, 640, 384, 5, 3, False),      # H, I multiples of 128 only; E not a power of two
+    (1200, 512, 384, 8, 2, False),    # ~300 rows per expert, bound 384: tiles of 257..384 rows, several feature tiles
+    (1100, 256, 256, 8, 2, True),     # the same bound, skewed: popular experts take several 384-row tiles, others a few rows
+    (2600, 256, 128, 16, 2, False),   # ~325 rows per expert: consecutive wide tiles overlap in the accumulator ring
+    (1030, 256, 128, 8, 2, False),    # ~257 rows per expert, bound 320: tiles just above and below 256 rows
 ]
 
 
