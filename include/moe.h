@@ -321,7 +321,7 @@ MOE_API int moe_mxfp8_quantize_rows(const void *x, int R, int K, void *codes, vo
  *   stage_events  NULL, or MOE_NUM_STAGE_EVENTS events recorded as by moe_forward_staged
  * Launches the same number of kernels as moe_forward (the scatter into expert-contiguous order also quantises:
  * each token row is read and quantised once and stored to its top_k destinations).  Token tiles are at most
- * 240 rows (128 when H is not a multiple of 256).  Errors as moe_forward; a block of x holding an infinity or NaN makes that token's output NaN. */
+ * 384 rows (128 when H is not a multiple of 256); moe_mxfp8_workspace_layout reports the size in use.  Errors as moe_forward; a block of x holding an infinity or NaN makes that token's output NaN. */
 MOE_API int moe_forward_mxfp8(const void *x, const float *router_logits, const void *w13_q, const void *w13_sf_packed,
                               const void *w2_q, const void *w2_sf_packed, int T, int H, int I, int E, int top_k,
                               const moe_grouped_router_t *router, int local_expert_offset, int num_local_experts,

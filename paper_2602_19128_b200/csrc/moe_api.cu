@@ -218,15 +218,16 @@ bool mx_envelope_ok(long long T, int H, int I, int E, int k) { return envelope_o
 // Token-tile rows of the MX path.  Scale columns sit next to the accumulators in tensor memory, so the largest tile
 // of the kernel with two fixed accumulators is 240 rows (2 * 240 + 32 columns); only the CTA-pair kernels have the
 // instances above 128 rows, and their down projection needs H to be a multiple of the 256-row pair tile.  Where the
-// bf16 layer takes its wide tiles (160 to 352 rows per expert on average) so does this one: 320 or 384 rows on the
-// accumulator ring, one pass over an expert's weights.  160-row tiles (a deeper ring) are taken when the mean rows per
-// expert plus 2.5 standard deviations of a uniform routing still fit.
+// bf16 layer takes its wide tiles (160 to 352 rows per expert on average) so does this one, on the accumulator ring,
+// one pass over an expert's weights: 304 rows while the mean plus 2.5 standard deviations of a uniform routing fits
+// (a 304-row token slot leaves the gate/up kernel room for a sixth ring slot, which the weight-stream-bound calls
+// need), else 384.  160-row tiles (a deeper ring still) are taken when the mean plus 2.5 standard deviations fits.
 int mx_tile_rows(int T, int H, int E, int k) {
     const int nt = choose_nt_max(T, E, k, true);
     if (nt <= 128) return nt;
     if (H % 256 != 0) return 128;
-    if (nt > 256) return nt;
     const double mean = (double)T * k / E;
+    if (nt > 256) return mean + 2.5 * sqrt(mean) <= 304.0 ? 304 : 384;
     return mean + 2.5 * sqrt(mean) <= 160.0 ? 160 : 240;
 }
 

@@ -1,4 +1,4 @@
-// Grouped expert GEMMs in MX FP8 on CTA pairs with WIDE token tiles (up to 320 / 384 rows): the block-scaled MMA of
+// Grouped expert GEMMs in MX FP8 on CTA pairs with WIDE token tiles (up to 304 / 384 rows): the block-scaled MMA of
 // moe_gemm_tc_mx_pair.cu on the accumulator ring of moe_gemm_tc_ring.cu.
 //
 // What is computed: paper Sec. 4.5 "Expert FFN computation" (gate/up with SiLU, then down) on the FP8 workload of
@@ -56,7 +56,7 @@ __device__ __forceinline__ void umma_mx_pair(uint32_t d_tmem, uint64_t a_desc, u
         : "memory");
 }
 
-template <int NT_MAX, int STAGES>
+template <int NT_MAX, int STAGES, bool SWIGLU>
 struct MxRingSmem {
     static constexpr int kAtomsB = (NT_MAX + 127) / 128;
     static constexpr int kSlotBBytes = (NT_MAX / 2) * kMxSlotK;
@@ -66,8 +66,8 @@ struct MxRingSmem {
     static constexpr int kSfA = kB + STAGES * kSlotBBytes;
     static constexpr int kSfB = kSfA + STAGES * kMxSfAtomBytes;
     static constexpr int kAmax = kSfB + STAGES * kSfBBytes;
-    static constexpr int kOutStage = kAmax + 2 * 4 * 16 * 4;  // down projection: two [16 tokens][128 rows] bf16 tiles
-    static constexpr int kBars = kOutStage + 2 * kOutStageBytes;  // full[S], empty[S], acc_full[32], acc_empty[32 (31 used)]
+    static constexpr int kOutStage = kAmax + 2 * 4 * 16 * 4;  // down projection only: two [16 tokens][128 rows] bf16 tiles
+    static constexpr int kBars = kOutStage + (SWIGLU ? 0 : 2 * kOutStageBytes);  // full[S], empty[S], acc_full[32], acc_empty[32 (31 used)]
     static constexpr int kQueue = kBars + (2 * STAGES + kAccFullBars + 32) * 8;
     static constexpr int kTmemSlot = kQueue + kTileQueue * 4;
     static constexpr int kAbort = kTmemSlot + 4;
@@ -97,7 +97,7 @@ __device__ __forceinline__ MxParts split_mx_tile(int seq, int n_cols) {
 template <int NT_MAX, int STAGES, bool SWIGLU>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kMxRingThreads, 1)
 grouped_gemm_tc_mx_ring_kernel(const __grid_constant__ MxRingMaps maps, const MxParams p) {
-    using L = MxRingSmem<NT_MAX, STAGES>;
+    using L = MxRingSmem<NT_MAX, STAGES, SWIGLU>;
     static_assert(NT_MAX % 16 == 0 && NT_MAX <= 384 && NT_MAX > 256, "token-tile bound of the wide-tile kernel");
     static_assert(L::kAtomsB == 3, "three token scale atoms next to the weight scales");
     static_assert(STAGES < kTileQueue, "the tile queue must outlast the ring");
@@ -395,7 +395,7 @@ grouped_gemm_tc_mx_ring_kernel(const __grid_constant__ MxRingMaps maps, const Mx
 
 template <int NT_MAX, int STAGES, bool SWIGLU>
 int launch_mx_ring_instance(const MxRingMaps &maps, const MxParams &p, int grid, cudaStream_t stream) {
-    using L = MxRingSmem<NT_MAX, STAGES>;
+    using L = MxRingSmem<NT_MAX, STAGES, SWIGLU>;
     static_assert(L::kBytes + 1024 <= L::kDynamicBytes, "ring does not fit in shared memory");
     auto kernel = grouped_gemm_tc_mx_ring_kernel<NT_MAX, STAGES, SWIGLU>;
     if (!set_max_dynamic_smem_once(reinterpret_cast<const void *>(kernel), L::kDynamicBytes))
@@ -406,7 +406,7 @@ int launch_mx_ring_instance(const MxRingMaps &maps, const MxParams &p, int grid,
 }  // namespace
 
 bool grouped_gemm_tc_mx_ring_applies(const MxGemmArgs &a) {
-    if (!(a.nt_max == 320 || a.nt_max == 384) || a.K % kMxSlotK != 0 || a.A <= 0) return false;
+    if (!(a.nt_max == 304 || a.nt_max == 384) || a.K % kMxSlotK != 0 || a.A <= 0) return false;
     return a.n_out % (a.swiglu ? kTileM : 2 * kTileM) == 0;
 }
 
@@ -451,9 +451,9 @@ int launch_grouped_gemm_tc_mx_ring(const MxGemmArgs &a, cudaStream_t stream) {
     const int pairs_on_device = sm_count() / 2;
     const int n_pairs = (int)(max_tiles < pairs_on_device ? max_tiles : pairs_on_device);
     const int grid = 2 * (n_pairs > 0 ? n_pairs : 1);
-    if (a.nt_max == 320)
-        return a.swiglu ? launch_mx_ring_instance<320, 5, true>(maps, p, grid, stream)
-                        : launch_mx_ring_instance<320, 5, false>(maps, p, grid, stream);
+    if (a.nt_max == 304)  // (the gate/up kernel has no output staging buffer: room for a sixth ring slot)
+        return a.swiglu ? launch_mx_ring_instance<304, 6, true>(maps, p, grid, stream)
+                        : launch_mx_ring_instance<304, 5, false>(maps, p, grid, stream);
     return a.swiglu ? launch_mx_ring_instance<384, 5, true>(maps, p, grid, stream)
                     : launch_mx_ring_instance<384, 5, false>(maps, p, grid, stream);
 }

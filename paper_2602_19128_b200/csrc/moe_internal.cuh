@@ -228,7 +228,7 @@ int launch_grouped_gemm_tc_mx(const MxGemmArgs &args, cudaStream_t stream);
 // pair tile (128 features of h, 256 output rows of the down projection).
 bool grouped_gemm_tc_mx_pair_applies(const MxGemmArgs &args);
 int launch_grouped_gemm_tc_mx_pair(const MxGemmArgs &args, cudaStream_t stream);
-// The same on CTA pairs with wide token tiles (nt_max 320 or 384: one pass over a weight slab per expert of up to that
+// The same on CTA pairs with wide token tiles (nt_max 304 or 384: one pass over a weight slab per expert of up to that
 // many rows), accumulators handed out in 16-column chunks of tensor memory as in the bf16 wide-tile kernel.
 bool grouped_gemm_tc_mx_ring_applies(const MxGemmArgs &args);
 int launch_grouped_gemm_tc_mx_ring(const MxGemmArgs &args, cudaStream_t stream);

@@ -92,13 +92,15 @@ def test_mx_layout():
         offs = [L.status, L.topk_ids, L.topk_weights, L.expert_offsets, L.sorted_to_flat, L.flat_to_sorted,
                 L.route_scratch, L.x_q, L.x_sf, L.h_q, L.h_sf, L.y, L.staging]
         assert offs == sorted(offs) and all(o % 256 == 0 for o in offs) and offs[-1] < n
-        assert L.tile_rows in (32, 64, 128, 160, 240)
+        assert L.tile_rows in (32, 64, 128, 160, 240, 304, 384)
         atoms_per_tile = (L.tile_rows + 127) // 128
         assert L.sf_atoms == (A // L.tile_rows + E + 1) * atoms_per_tile
         assert L.x_sf - L.x_q >= A * H and L.h_q - L.x_sf >= (H // 128) * L.sf_atoms * 512
         assert L.y - L.h_sf >= (I // 128) * L.sf_atoms * 512
     assert moe.moe_mxfp8_workspace_layout(512, 4096, 14336, 8, 2).tile_rows == 160     # 128 rows per expert on average
-    assert moe.moe_mxfp8_workspace_layout(8192, 7168, 2048, 256, 8).tile_rows == 240   # 256 on average
+    assert moe.moe_mxfp8_workspace_layout(8192, 7168, 2048, 256, 8).tile_rows == 304   # 256 on average: one wide tile per expert
+    assert moe.moe_mxfp8_workspace_layout(8192, 7168, 2048, 208, 8).tile_rows == 384   # 315 on average
+    assert moe.moe_mxfp8_workspace_layout(8192, 7168, 2048, 128, 8).tile_rows == 240   # 512 on average: several tiles anyway
     assert moe.moe_mxfp8_workspace_layout(8192, 7040, 2048, 256, 8).tile_rows == 128   # H not a multiple of 256
     assert moe.moe_mxfp8_workspace_bytes(16, 256, 192, 8, 2) == 0                      # I must be a multiple of 128
 
