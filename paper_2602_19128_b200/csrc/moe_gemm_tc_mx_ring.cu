@@ -333,19 +333,14 @@ grouped_gemm_tc_mx_ring_kernel(const __grid_constant__ MxRingMaps maps, const Mx
                         hv[i] = swiglu(gt, up);
                         mag[i] = __float_as_uint(hv[i]) & 0x7FFFFFFFu;  // magnitudes compare as integers; NaN and inf on top
                     }
-#pragma unroll
-                    for (int off = 8; off >= 1; off >>= 1)
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) mag[i] = max(mag[i], __shfl_xor_sync(0xffffffffu, mag[i], off));
+                    const uint32_t col_max = half_warp_max8(mag, j16);  // of column c0 + hi * 8 + j16 / 2, this warp's 16 features
                     buf ^= 1;
-                    if (j16 == 0) {
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) amax_s[(buf * 4 + q) * 16 + hi * 8 + i] = mag[i];
-                    }
+                    if ((j16 & 1) == 0) amax_s[(buf * 4 + q) * 16 + hi * 8 + (j16 >> 1)] = col_max;
                     pair_sync(q >> 1);
 #pragma unroll
                     for (int i = 0; i < 8; ++i) {
-                        const uint32_t block_mag = max(mag[i], amax_s[(buf * 4 + (q ^ 1)) * 16 + hi * 8 + i]);
+                        const uint32_t block_mag = max(amax_s[(buf * 4 + q) * 16 + hi * 8 + i],
+                                                       amax_s[(buf * 4 + (q ^ 1)) * 16 + hi * 8 + i]);
                         const uint32_t sb = mx_scale_byte(block_mag);
                         const int col = c0 + hi * 8 + i;
                         if (col < t.n_valid) {

@@ -84,6 +84,25 @@ __device__ __forceinline__ uint32_t mx_scale_byte(uint32_t amax_bits) {
     return e > 8u ? e - 8u : 0u;
 }
 
+// Maxima of eight values over the 16 lanes of a half-warp by recursive halving: 8 shuffles instead of the 32 of a
+// butterfly per value.  Afterwards lanes j and j ^ 1 (j = lane % 16) both hold the maximum of value j / 2.
+__device__ __forceinline__ uint32_t half_warp_max8(const uint32_t (&mag)[8], int j) {
+    uint32_t m4[4], m2[2];
+    const bool b8 = (j & 8) != 0, b4 = (j & 4) != 0, b2 = (j & 2) != 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const uint32_t recv = __shfl_xor_sync(0xffffffffu, b8 ? mag[i] : mag[4 + i], 8);
+        m4[i] = max(b8 ? mag[4 + i] : mag[i], recv);
+    }
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        const uint32_t recv = __shfl_xor_sync(0xffffffffu, b4 ? m4[i] : m4[2 + i], 4);
+        m2[i] = max(b4 ? m4[2 + i] : m4[i], recv);
+    }
+    uint32_t m1 = max(b2 ? m2[1] : m2[0], __shfl_xor_sync(0xffffffffu, b2 ? m2[0] : m2[1], 2));
+    return max(m1, __shfl_xor_sync(0xffffffffu, m1, 1));
+}
+
 // Gate/up epilogue of one warp: its 32 TMEM lanes hold, for 16 features, the gate rows (lanes 0..15) and
 // the up rows (lanes 16..31) of n_mma token columns.  Computes h = SiLU(gate) * up, quantises it in
 // blocks of 32 features (this warp's 16 and its partner warp's 16, warps q and q^1), and stores the
@@ -108,19 +127,13 @@ __device__ __forceinline__ void drain_swiglu_mx(uint32_t taddr, int n_mma, int n
             hv[i] = swiglu(g, u);
             mag[i] = __float_as_uint(hv[i]) & 0x7FFFFFFFu;  // magnitudes compare as integers; NaN and inf on top
         }
-#pragma unroll
-        for (int off = 8; off >= 1; off >>= 1)
-#pragma unroll
-            for (int i = 0; i < 8; ++i) mag[i] = max(mag[i], __shfl_xor_sync(0xffffffffu, mag[i], off));
+        const uint32_t col_max = half_warp_max8(mag, j);  // of column c0 + hi * 8 + j / 2 over this warp's 16 features
         buf ^= 1;
-        if (j == 0) {
-#pragma unroll
-            for (int i = 0; i < 8; ++i) amax_s[(buf * 4 + q) * 16 + hi * 8 + i] = mag[i];
-        }
+        if ((j & 1) == 0) amax_s[(buf * 4 + q) * 16 + hi * 8 + (j >> 1)] = col_max;
         pair_sync(q >> 1);
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-            const uint32_t block_mag = max(mag[i], amax_s[(buf * 4 + (q ^ 1)) * 16 + hi * 8 + i]);
+            const uint32_t block_mag = max(amax_s[(buf * 4 + q) * 16 + hi * 8 + i], amax_s[(buf * 4 + (q ^ 1)) * 16 + hi * 8 + i]);
             const uint32_t sb = mx_scale_byte(block_mag);
             const int col = c0 + hi * 8 + i;
             if (col < n_valid) {
