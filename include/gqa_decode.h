@@ -66,6 +66,13 @@ MOE_API int gqa_paged_decode(const void *q, const void *k_cache, const void *v_c
                              int page_size, int num_pages, int max_kv_len, float sm_scale, void *out, float *lse,
                              void *workspace, size_t workspace_bytes, void *stream);
 
+/* Self-test of the device-side error path, as moe_selftest_wait_timeout: every wait of the decode kernel (on the
+ * barriers its copies complete on) is bounded; this call enqueues one warp that waits, with a bound of a few
+ * milliseconds, on a barrier at which nothing arrives.  Afterwards moe_last_status(workspace, stream) must report
+ * MOE_ERR_DEVICE_TIMEOUT and the device must be usable as before.  workspace: at least 256 bytes, 256-byte aligned
+ * (its first 256 bytes are overwritten). */
+MOE_API int gqa_selftest_wait_timeout(void *workspace, size_t workspace_bytes, void *stream);
+
 /* Host-only, pure.  Tokens per sequence split and number of splits the call above uses for these sizes (reporting). */
 MOE_API int gqa_decode_split_tokens(int B, int Hq, int Hkv, int D, int max_kv_len);
 

@@ -26,7 +26,7 @@ EXPORTED = ["moe_workspace_bytes", "moe_workspace_layout", "moe_route_workspace_
             "moe_forward_ex", "moe_forward_local", "moe_route_grouped", "moe_forward_grouped", "moe_forward_fp8w", "moe_mxfp8_workspace_bytes",
             "moe_mxfp8_workspace_layout", "moe_mxfp8_pack_scales", "moe_mxfp8_quantize_rows", "moe_forward_mxfp8", "moe_forward_mxfp8_host",
             "moe_forward_staged", "moe_forward_host", "moe_last_status", "moe_selftest_wait_timeout", "moe_forward_launch_count", "moe_token_tile_rows", "moe_status_string",
-            "gqa_decode_workspace_bytes", "gqa_paged_decode", "gqa_decode_split_tokens"]
+            "gqa_decode_workspace_bytes", "gqa_paged_decode", "gqa_decode_split_tokens", "gqa_selftest_wait_timeout"]
 
 
 class MoeError(RuntimeError):
@@ -124,6 +124,8 @@ def lib() -> ctypes.CDLL:
         L.gqa_decode_workspace_bytes.argtypes = [i] * 5
         L.gqa_decode_split_tokens.restype = i
         L.gqa_decode_split_tokens.argtypes = [i] * 5
+        L.gqa_selftest_wait_timeout.restype = i
+        L.gqa_selftest_wait_timeout.argtypes = [vp, sz, vp]
         L.gqa_paged_decode.restype = i
         L.gqa_paged_decode.argtypes = [vp] * 6 + [i] * 7 + [ctypes.c_float, vp, vp, vp, sz, vp]
         L.moe_status_string.restype = ctypes.c_char_p
@@ -449,6 +451,14 @@ def workspace_views(workspace: torch.Tensor, T: int, H: int, I: int, E: int, top
 # ---- second workload: paged grouped-query decode attention (include/gqa_decode.h) -------------------------------
 def gqa_decode_workspace_bytes(B: int, Hq: int, Hkv: int, D: int, max_kv_len: int) -> int:
     return int(lib().gqa_decode_workspace_bytes(B, Hq, Hkv, D, max_kv_len))
+
+
+def gqa_selftest_wait_timeout(workspace, stream=None) -> int:
+    """Enqueue the decode kernel's bounded-wait self-test; read the outcome with moe_last_status(workspace)."""
+    st = lib().gqa_selftest_wait_timeout(_ptr(workspace), workspace.numel(), _stream(stream))
+    if st != MOE_OK:
+        raise MoeError(st, "gqa_selftest_wait_timeout")
+    return st
 
 
 def gqa_decode_split_tokens(B: int, Hq: int, Hkv: int, D: int, max_kv_len: int) -> int:

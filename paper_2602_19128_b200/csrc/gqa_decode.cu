@@ -146,6 +146,31 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return *reinterpret_cast<uint32_t *>(&v);
 }
 
+// Bounded wait on an mbarrier: false once `limit` polls have passed (the status word then says so: the call's first
+// expired wait records MOE_ERR_DEVICE_TIMEOUT, site 12 and the block) or once another thread of the block has given up.
+__device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, int limit, volatile int *gave_up, int *status) {
+    for (int i = 0; i < limit; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*gave_up) return false;
+    }
+    *gave_up = 1;
+    if (atomicCAS(status, 0, (int)MOE_ERR_DEVICE_TIMEOUT) == 0) { status[1] = 12; status[2] = blockIdx.x; }
+    return false;
+}
+
+// Self-test of that error path: one warp waits, with a small bound, on a barrier at which nothing arrives.
+__global__ void gqa_wait_timeout_selftest_kernel(int *status) {
+    __shared__ __align__(8) unsigned long long bar;
+    __shared__ int gave_up;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        gave_up = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    bounded_wait(smem_u32(&bar), 0, 1 << 14, &gave_up, status);
+}
+
 // Byte offset, inside a 64-token tile, of 16-byte piece `piece` (0..15) of token row `row`.
 // `sh` = log2(box_rows) (tiled only).
 template <bool kTiled>
@@ -274,15 +299,8 @@ gqa_paged_decode_kernel(const Params p, const __grid_constant__ CUtensorMap k_ma
         }
         next_loc = locate(chunk + 1);
     };
-    // Bounded wait on a barrier; false once any thread of the block has given up.
     auto wait_bar = [&](uint32_t bar, uint32_t parity) -> bool {
-        for (int i = 0; i < kWaitLimit; ++i) {
-            if (mbar_try_wait(bar, parity)) return true;
-            if (*(volatile int *)&gave_up) return false;
-        }
-        gave_up = 1;
-        if (atomicCAS(p.status, 0, (int)MOE_ERR_DEVICE_TIMEOUT) == 0) { p.status[1] = 12; p.status[2] = blockIdx.x; }
-        return false;
+        return bounded_wait(bar, parity, kWaitLimit, &gave_up, p.status);
     };
     auto wait_chunk = [&](int chunk) -> bool {
         return wait_bar(bar_base + (chunk % kNumStages) * 8, (uint32_t)(chunk / kNumStages) & 1u);
@@ -614,6 +632,19 @@ size_t gqa_decode_workspace_bytes(int B, int Hq, int Hkv, int D, int max_kv_len)
     const size_t bh = (size_t)B * Hkv, group = Hq / Hkv;
     return 256 + align_up(bh * sizeof(int), 256) + align_up(bh * ns * group * 2 * sizeof(float), 256) +
            align_up(bh * ns * group * kD * sizeof(float), 256) + 256;
+}
+
+int gqa_selftest_wait_timeout(void *workspace, size_t workspace_bytes, void *stream) {
+    using namespace gqa;
+    if (!workspace) return MOE_ERR_NULL;
+    if (reinterpret_cast<uintptr_t>(workspace) % 256 != 0) return MOE_ERR_ALIGN;
+    if (workspace_bytes < 256) return MOE_ERR_WORKSPACE;
+    const int arch = moe::check_device();
+    if (arch != MOE_OK) return arch;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemsetAsync(workspace, 0, 256, st) != cudaSuccess) return MOE_ERR_CUDA;
+    gqa_wait_timeout_selftest_kernel<<<1, 32, 0, st>>>(static_cast<int *>(workspace));
+    return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
 
 int gqa_decode_split_tokens(int B, int Hq, int Hkv, int D, int max_kv_len) {

@@ -110,6 +110,21 @@ def test_the_workspace_status_word_reports_success():
     assert moe.moe_last_status(ws) == 0
 
 
+def test_an_expired_barrier_wait_is_reported_and_leaves_the_device_usable():
+    """Every wait of the kernel is bounded.  The self-test waits a few milliseconds on a barrier at which nothing
+    arrives: it must come back with MOE_ERR_DEVICE_TIMEOUT in the status word, and the next call must work."""
+    inp = make_gqa_inputs(dict(B=2, Hq=32, Hkv=4, D=128, page_size=16, lengths=[5000, 300]), seed=3, device="cuda")
+    ws = moe.alloc_workspace(moe.gqa_decode_workspace_bytes(2, 32, 4, 128, 5000), "cuda")
+    moe.gqa_selftest_wait_timeout(ws)
+    assert moe.moe_last_status(ws) == -7
+    assert ws[:12].view(torch.int32)[1].item() == 12          # the site recorded next to the status
+    check(inp)
+    out = torch.empty((2, 32, 128), dtype=torch.bfloat16, device="cuda")
+    moe.gqa_paged_decode(inp["q"], inp["k_cache"], inp["v_cache"], inp["kv_indptr"], inp["kv_indices"],
+                         inp["kv_last_page_len"], 5000, inp["sm_scale"], out, ws)
+    assert moe.moe_last_status(ws) == 0
+
+
 def test_a_sequence_longer_than_the_hint_is_still_computed_in_full():
     inp = make_gqa_inputs(dict(B=2, Hq=32, Hkv=4, D=128, page_size=16, lengths=[3000, 500]), seed=2, device="cuda")
     check(inp, max_kv_len=1024)     # the last split runs to the end of the sequence
