@@ -280,16 +280,19 @@ typedef struct {
     size_t total_bytes;
     size_t status, topk_ids, topk_weights, expert_offsets, sorted_to_flat, flat_to_sorted, route_scratch; /* as moe_workspace_layout_t */
     size_t x_q;   /* uint8 [A,H]  codes of the token rows in expert-contiguous order */
-    size_t x_sf;  /* scale atoms of x_q: [H/128][sf_atoms][512].  Row i of expert e belongs to token tile
-                     n = expert_offsets[e] / tile_rows + e + i / tile_rows, as its row r = i % tile_rows; a tile owns
-                     ceil(tile_rows / 128) atoms, and the row's scales are in atom n * ceil(tile_rows / 128) + r / 128
-                     at atom row r % 128 */
+    size_t x_sf;  /* scale atoms of x_q: [H/128][sf_atoms][512].  An expert's rows are cut into token tiles of equal
+                     size rows_e (the last may be partial): rows_e = tile_rows for tile_rows <= 256; for the wide
+                     bounds (304, 384) an expert of count <= tile_rows rows is one tile, a larger one
+                     ceil(count / 256) tiles of rows_e = ceil(count / that) rounded up to 16.  Row i of expert e
+                     belongs to token tile n = expert_offsets[e] / min(tile_rows, 256) + e + i / rows_e, as its row
+                     r = i % rows_e; a tile owns ceil(tile_rows / 128) atoms, and the row's scales are in atom
+                     n * ceil(tile_rows / 128) + r / 128 at atom row r % 128 */
     size_t h_q;   /* uint8 [A,I]  codes of h */
     size_t h_sf;  /* scale atoms of h_q: [I/128][sf_atoms][512], same row-to-atom rule */
     size_t y;     /* bf16 [A,H] */
     size_t staging; /* used only by moe_forward_mxfp8_host: device copies of x, logits, out */
     size_t sf_atoms;  /* a count, not an offset: atoms per K-slot in x_sf / h_sf */
-    size_t tile_rows; /* a count: rows per token tile of this problem (32, 64, 128, 160 or 240) */
+    size_t tile_rows; /* a count: the token-tile bound of this problem (32, 64, 128, 160, 240, 304 or 384) */
 } moe_mxfp8_workspace_layout_t;
 
 /* Host-only, pure.  Workspace bytes of moe_forward_mxfp8; 0 outside the envelope (moe_forward's, plus I % 128 == 0). */

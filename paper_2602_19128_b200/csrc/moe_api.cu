@@ -301,13 +301,15 @@ int forward_mx_impl(const void *x, const float *logits, const void *w13_q, const
         return !stage_events || cudaEventRecord(static_cast<cudaEvent_t>(stage_events[i]), stream) == cudaSuccess;
     };
     if (!mark(0)) return MOE_ERR_CUDA;
-    // every token tile exactly nt_max rows (the last of an expert partial): each tile owns one scale atom
+    // Bounds up to 256: every token tile exactly nt_max rows (the last of an expert partial).  Wide bounds: the bf16
+    // schedule's rule (row quantum 16; experts above the bound get evenly sized tiles of at most 256 rows).  Either
+    // way each tile owns its own scale atoms (moe_internal.cuh).
     if (launch_route(logits, T, E, k, LocalExperts{local_offset, n_local}, nt_max, ids, wts, offsets, s2f, f2s, rs, status,
-                     stream, nt_max, router, kStatusBytesForward) != cudaSuccess)
+                     stream, nt_max > 256 ? 16 : nt_max, router, kStatusBytesForward) != cudaSuccess)
         return MOE_ERR_CUDA;
     if (!mark(1)) return MOE_ERR_CUDA;
-    if (launch_mx_scatter_quantize(static_cast<const __nv_bfloat16 *>(x), f2s, ids, offsets, LocalExperts{local_offset, n_local},
-                                   T, k, H, x_q, x_sf, n_atoms, nt_max, stream) != cudaSuccess)
+    if (launch_mx_scatter_quantize(static_cast<const __nv_bfloat16 *>(x), f2s, ids, offsets, rs.tile_rows,
+                                   LocalExperts{local_offset, n_local}, T, k, H, x_q, x_sf, n_atoms, nt_max, stream) != cudaSuccess)
         return MOE_ERR_CUDA;
     if (!mark(2)) return MOE_ERR_CUDA;
 

@@ -293,7 +293,7 @@ int launch_grouped_gemm_tc_mx(const MxGemmArgs &a, cudaStream_t stream) {
     p.w_rows = a.w_rows;
     p.n_feature_tiles = a.n_out / features_per_tile;
     p.n_atoms = a.n_atoms;
-    p.tile_stride = a.nt_max;
+    p.tile_stride = mx_sf_stride(a.nt_max);
     p.atoms_per_tile = 1;
     p.handover_role = a.handover_role;
     p.handover = a.handover;

@@ -320,7 +320,7 @@ int launch_grouped_gemm_tc_mx_pair(const MxGemmArgs &a, cudaStream_t stream) {
     p.w_rows = a.w_rows;
     p.n_feature_tiles = a.n_out / (2 * cta_feat);
     p.n_atoms = a.n_atoms;
-    p.tile_stride = a.nt_max;
+    p.tile_stride = mx_sf_stride(a.nt_max);
     p.atoms_per_tile = atoms_per_tile;
     p.handover_role = a.handover_role;
     p.handover = a.handover;

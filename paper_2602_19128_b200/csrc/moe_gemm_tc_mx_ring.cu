@@ -435,13 +435,13 @@ int launch_grouped_gemm_tc_mx_ring(const MxGemmArgs &a, cudaStream_t stream) {
     p.w_rows = a.w_rows;
     p.n_feature_tiles = a.n_out / (2 * cta_feat);
     p.n_atoms = a.n_atoms;
-    p.tile_stride = a.nt_max;
+    p.tile_stride = mx_sf_stride(a.nt_max);
     p.atoms_per_tile = atoms_per_tile;
     p.handover_role = a.handover_role;
     p.handover = a.handover;
     p.handover_per_token_tile = a.handover_per_token_tile;
 
-    const long long max_token_tiles = (long long)(a.A < a.E ? a.A : a.E) + a.A / a.nt_max;
+    const long long max_token_tiles = (long long)(a.A < a.E ? a.A : a.E) + a.A / 256;  // (experts above the bound: tiles of up to 256 rows)
     const long long max_tiles = max_token_tiles * p.n_feature_tiles;
     const int pairs_on_device = sm_count() / 2;
     const int n_pairs = (int)(max_tiles < pairs_on_device ? max_tiles : pairs_on_device);

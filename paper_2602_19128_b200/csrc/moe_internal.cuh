@@ -190,15 +190,20 @@ int launch_grouped_gemm_tc_fp8w(const GroupedGemmArgs &args, cudaStream_t stream
 // in global memory in that form, one atom per (128-row group, ring slot), so a slot's scales are one
 // bulk copy.
 //   weights     : [E][feature tile][K/128][512]; a gate/up tile's rows are in the tile's interleaved order
-//   activations : [K/128][n_atoms][512], whole atoms per token tile.  The MX schedule cuts every expert's
-//                 rows into tiles of exactly `tile` rows (the token-tile bound: 32, 64, 128, 160 or 240; the last
-//                 may be partial).  Token tile j of expert e is tile number  offsets[e] / tile + e + j  and
-//                 owns ceil(tile / 128) consecutive atoms; its row r sits in atom r / 128 of those, at atom
-//                 row r % 128.  Every tile thus starts a fresh atom, and the MMA reads its token scales from
-//                 the first column of the atom (an odd column offset is a misaligned address for the
-//                 instruction).  n_atoms = (A / tile + E + 1) * ceil(tile / 128) bounds the atom index.
+//   activations : [K/128][n_atoms][512], whole atoms per token tile.  The MX schedule cuts an expert's rows into
+//                 tiles of equal size (the last may be partial): exactly `tile` rows for a token-tile bound of up to
+//                 256 (32, 64, 128, 160 or 240); for the wide bounds (304, 384) an expert of up to `tile` rows is one
+//                 tile, and a larger one is cut into ceil(count / 256) tiles of round16(count / that) <= 256 rows,
+//                 as in the bf16 schedule (two consecutive tiles of more than 248 rows would overlap in the
+//                 accumulator ring).  With stride = min(tile, 256), token tile j of expert e is tile number
+//                 offsets[e] / stride + e + j  (never below the number of tiles before it, so the numbers are
+//                 distinct) and owns ceil(tile / 128) consecutive atoms; its row r sits in atom r / 128 of those,
+//                 at atom row r % 128.  Every tile thus starts a fresh atom, and the MMA reads its token scales
+//                 from the first column of the atom (an odd column offset is a misaligned address for the
+//                 instruction).  n_atoms = (A / stride + E + 1) * ceil(tile / 128) bounds the atom index.
 constexpr int kMxSfAtomBytes = 512;
-static inline int mx_act_sf_atoms(int A, int E, int tile) { return (A / tile + E + 1) * ((tile + 127) / 128); }
+static inline int mx_sf_stride(int tile) { return tile > 256 ? 256 : tile; }
+static inline int mx_act_sf_atoms(int A, int E, int tile) { return (A / mx_sf_stride(tile) + E + 1) * ((tile + 127) / 128); }
 static inline size_t mx_act_sf_bytes(int A, int E, int K, int tile) {
     return (size_t)(K / 128) * mx_act_sf_atoms(A, E, tile) * kMxSfAtomBytes;
 }
@@ -236,8 +241,8 @@ int launch_grouped_gemm_tc_mx_ring(const MxGemmArgs &args, cudaStream_t stream);
 // xq[flat_to_sorted[t*k+j], :] and that row's scale atoms <- MX quantisation of x[t,:], for every assignment with
 // flat_to_sorted >= 0 (token-major: each row is read and quantised once).
 cudaError_t launch_mx_scatter_quantize(const __nv_bfloat16 *x, const int *flat_to_sorted, const int *topk_ids,
-                                       const int *expert_offsets, LocalExperts local, int T, int k, int H, uint8_t *xq,
-                                       uint8_t *x_sf, int n_atoms, int tile, cudaStream_t stream);
+                                       const int *expert_offsets, const int *tile_rows, LocalExperts local, int T, int k,
+                                       int H, uint8_t *xq, uint8_t *x_sf, int n_atoms, int tile, cudaStream_t stream);
 // codes[r,:], scales[r, K/32] (plain row-major) <- MX quantisation of x[r,:].
 cudaError_t launch_mx_quantize_rows(const __nv_bfloat16 *x, int R, int K, uint8_t *codes, uint8_t *scales,
                                     cudaStream_t stream);

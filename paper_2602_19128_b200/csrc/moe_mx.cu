@@ -58,9 +58,9 @@ __device__ __forceinline__ uint2 quantize_8_of_32(const uint4 v, uint32_t &scale
 template <bool kScatter>
 __global__ void __launch_bounds__(256)
 mx_quantize_rows_kernel(const uint4 *__restrict__ x, const int *__restrict__ flat_to_sorted,
-                        const int *__restrict__ topk_ids, const int *__restrict__ expert_offsets, int local_offset,
-                        int n_local, int n_rows, int k, int vec_per_row, int warps_per_row, uint2 *__restrict__ codes,
-                        uint8_t *__restrict__ scales, int n_atoms, int tile) {
+                        const int *__restrict__ topk_ids, const int *__restrict__ expert_offsets,
+                        const int *__restrict__ tile_rows, int local_offset, int n_local, int n_rows, int k, int vec_per_row,
+                        int warps_per_row, uint2 *__restrict__ codes, uint8_t *__restrict__ scales, int n_atoms, int tile) {
     chain_release();
     chain_wait();
     const int lane = threadIdx.x & 31;
@@ -75,8 +75,10 @@ mx_quantize_rows_kernel(const uint4 *__restrict__ x, const int *__restrict__ fla
         if (my_row >= 0) {
             const int e = topk_ids[(size_t)r * k + lane] - local_offset;  // resident, or the row would be -1
             const int begin = expert_offsets[e], i = my_row - begin;
-            const int atoms_per_tile = (tile + 127) / 128, tr = i % tile;  // row tr of token tile i / tile of this expert
-            my_sf_base = (long long)((begin / tile + e + i / tile) * atoms_per_tile + tr / 128) * kMxSfAtomBytes +
+            // row tr of token tile i / rows of this expert, whose tiles all have `rows` rows (the schedule's choice)
+            const int rows = tile_rows[e], stride = tile > 256 ? 256 : tile;
+            const int atoms_per_tile = (tile + 127) / 128, tr = i % rows;
+            my_sf_base = (long long)((begin / stride + e + i / rows) * atoms_per_tile + tr / 128) * kMxSfAtomBytes +
                          mx_atom_byte(tr % 128, 0);
         }
     }
@@ -148,12 +150,12 @@ mx_pack_scales_kernel(const uint32_t *__restrict__ plain, int E, int rows, int s
 }  // namespace
 
 cudaError_t launch_mx_scatter_quantize(const __nv_bfloat16 *x, const int *flat_to_sorted, const int *topk_ids,
-                                       const int *expert_offsets, LocalExperts local, int T, int k, int H, uint8_t *xq,
-                                       uint8_t *x_sf, int n_atoms, int tile, cudaStream_t stream) {
+                                       const int *expert_offsets, const int *tile_rows, LocalExperts local, int T, int k,
+                                       int H, uint8_t *xq, uint8_t *x_sf, int n_atoms, int tile, cudaStream_t stream) {
     const int wpr = mx_quantize_warps_per_row(T, (H / 8 + 31) / 32);
     const long long warps = (long long)T * wpr;
     return launch_chained(mx_quantize_rows_kernel<true>, (unsigned)((warps + 7) / 8), 256, 0, stream,
-                          reinterpret_cast<const uint4 *>(x), flat_to_sorted, topk_ids, expert_offsets, local.offset,
+                          reinterpret_cast<const uint4 *>(x), flat_to_sorted, topk_ids, expert_offsets, tile_rows, local.offset,
                           local.count, T, k, H / 8, wpr, reinterpret_cast<uint2 *>(xq), x_sf, n_atoms, tile);
 }
 
@@ -162,7 +164,7 @@ cudaError_t launch_mx_quantize_rows(const __nv_bfloat16 *x, int R, int K, uint8_
     const int wpr = mx_quantize_warps_per_row(R, (K / 8 + 31) / 32);
     const long long warps = (long long)R * wpr;
     return launch_chained(mx_quantize_rows_kernel<false>, (unsigned)((warps + 7) / 8), 256, 0, stream,
-                          reinterpret_cast<const uint4 *>(x), nullptr, nullptr, nullptr, 0, 0, R, 1, K / 8, wpr,
+                          reinterpret_cast<const uint4 *>(x), nullptr, nullptr, nullptr, nullptr, 0, 0, R, 1, K / 8, wpr,
                           reinterpret_cast<uint2 *>(codes), scales, 0, 1);
 }
 

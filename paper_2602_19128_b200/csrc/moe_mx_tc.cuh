@@ -23,8 +23,8 @@ struct MxParams {
     const int *expert_offsets, *tile_prefix, *tile_order, *tile_rows;
     int *status;
     int E, n_k_blocks, n_out, w_rows, n_feature_tiles, n_atoms;
-    int tile_stride;     // rows of every token tile of the MX schedule (the last of an expert may be partial)
-    int atoms_per_tile;  // ceil(tile_stride / 128)
+    int tile_stride;     // stride of the tile numbering: min(token-tile bound, 256) (moe_internal.cuh)
+    int atoms_per_tile;  // ceil(token-tile bound / 128)
     int handover_role;   // hand-over between the two GEMMs of a call (moe_internal.cuh)
     int *handover;
     int handover_per_token_tile;
@@ -48,7 +48,7 @@ __device__ __forceinline__ MxTile decode_mx_tile(int tile, const MxParams &p) {
     const int local = tile - first * p.n_feature_tiles;
     t.f = local / n_tok_tiles;
     const int j = local - t.f * n_tok_tiles;
-    const int rows = p.tile_rows[t.e];  // == p.tile_stride for every expert of an MX schedule
+    const int rows = p.tile_rows[t.e];  // rows of every tile of this expert (the bound itself for bounds up to 256)
     const int begin = p.expert_offsets[t.e], count = p.expert_offsets[t.e + 1] - begin;
     t.row0 = begin + j * rows;
     t.n_valid = min(rows, count - j * rows);

@@ -346,11 +346,11 @@ __device__ __forceinline__ void scan_phase(int *chunk_counts, int n_chunks, int 
     // a wide bound (320 / 384) exists to keep an expert in ONE pass over its weights, and consecutive tiles wider than
     // half of tensor memory cannot overlap their epilogues, so experts that need several tiles get 256-row ones --
     // evenly sized, rounded up to the row quantum
-    // (16 rows, the MMA's N granularity; the MX path passes its tile size, so that every tile is exactly that many
-    // rows -- its scale atoms are laid out per tile -- and an expert above the bound gets as few such tiles as hold it)
+    // (16 rows, the MMA's N granularity; the MX path with a bound of up to 256 passes its tile size, so that every tile
+    // is exactly that many rows)
     int n_tiles = 0, rows = 0;
     if (count > 0) {
-        const int multi = (nt_max > 256 && row_quantum != nt_max) ? 256 : nt_max;
+        const int multi = nt_max > 256 ? 256 : nt_max;
         n_tiles = count <= nt_max ? 1 : (count + multi - 1) / multi;
         rows = (((count + n_tiles - 1) / n_tiles) + row_quantum - 1) / row_quantum * row_quantum;
     }

@@ -94,7 +94,7 @@ def test_mx_layout():
         assert offs == sorted(offs) and all(o % 256 == 0 for o in offs) and offs[-1] < n
         assert L.tile_rows in (32, 64, 128, 160, 240, 304, 384)
         atoms_per_tile = (L.tile_rows + 127) // 128
-        assert L.sf_atoms == (A // L.tile_rows + E + 1) * atoms_per_tile
+        assert L.sf_atoms == (A // min(L.tile_rows, 256) + E + 1) * atoms_per_tile
         assert L.x_sf - L.x_q >= A * H and L.h_q - L.x_sf >= (H // 128) * L.sf_atoms * 512
         assert L.y - L.h_sf >= (I // 128) * L.sf_atoms * 512
     assert moe.moe_mxfp8_workspace_layout(512, 4096, 14336, 8, 2).tile_rows == 160     # 128 rows per expert on average

@@ -21,16 +21,28 @@ def atom_byte(r, sf):
     return (r % 32) * 16 + (r // 32) * 4 + sf
 
 
+def expert_tile_rows(count: int, tile: int) -> int:
+    """Rows of every token tile of an expert with ``count`` rows (include/moe.h, the MX workspace layout): the bound
+    itself up to 256; for the wide bounds one tile of round16(count) rows, or evenly sized tiles of at most 256."""
+    if tile <= 256:
+        return tile
+    n = 1 if count <= tile else -(-count // 256)
+    return (-(-count // n) + 15) // 16 * 16
+
+
 def unpack_act_scales(atoms: np.ndarray, offsets: np.ndarray, n_blocks: int, tile: int) -> np.ndarray:
     """Scale atoms [K/128, n_atoms, 512] -> plain [rows, K/32] for the rows of every expert segment."""
     E = len(offsets) - 1
     rows = offsets[E]
     plain = np.zeros((rows, n_blocks), np.uint8)
+    apt, stride = (tile + 127) // 128, min(tile, 256)
     for e in range(E):
         begin = offsets[e]
-        for i in range(offsets[e + 1] - begin):
-            apt, r = (tile + 127) // 128, i % tile
-            a = (begin // tile + e + i // tile) * apt + r // 128
+        count = offsets[e + 1] - begin
+        per_tile = expert_tile_rows(int(count), tile) if count else tile
+        for i in range(count):
+            r = i % per_tile
+            a = (begin // stride + e + i // per_tile) * apt + r // 128
             for b in range(n_blocks):
                 plain[begin + i, b] = atoms[b // 4, a, atom_byte(r % 128, b % 4)]
     return plain
@@ -296,11 +308,12 @@ def test_mxfp8_large_batch_codes_and_scale_bytes():
     assert np.array_equal(views["x_q"].cpu().numpy(), xc[tok])
     # scale bytes: vectorised form of unpack_act_scales
     tile = views["tile_rows"]
-    apt = (tile + 127) // 128
+    apt, stride = (tile + 127) // 128, min(tile, 256)
+    per_tile = np.array([expert_tile_rows(int(off[e + 1] - off[e]), tile) if off[e + 1] > off[e] else tile for e in range(E)])
     e_of_row = np.searchsorted(off, np.arange(off[E]), side="right") - 1
     i = np.arange(off[E]) - off[e_of_row]
-    r = i % tile
-    atom = (off[e_of_row] // tile + e_of_row + i // tile) * apt + r // 128
+    r = i % per_tile[e_of_row]
+    atom = (off[e_of_row] // stride + e_of_row + i // per_tile[e_of_row]) * apt + r // 128
     base = (r % 128 % 32) * 16 + (r % 128 // 32) * 4
     atoms = views["x_sf"].cpu().numpy()
     got = np.stack([atoms[b // 4, atom, base + b % 4] for b in range(H // 32)], axis=1)
