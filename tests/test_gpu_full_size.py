@@ -91,8 +91,8 @@ def test_full_size_workload(name):
 
 @pytest.mark.parametrize("name", ["mixtral", "dsv3_decode", "skewed", "dsv3_prefill"])
 def test_full_size_workload_mxfp8(name):
-    """The MX FP8 layer at full size (CTA-pair kernel with 240-row tiles for the large batches, one-CTA kernel
-    for the decode-sized one): routing bit-exact on all tokens, quantised token rows bit-exact on a sample,
+    """The MX FP8 layer at full size (wide-tile CTA-pair kernel for the prefill-sized batches, 160-row pair tiles
+    for the Mixtral shape, one-CTA kernel for the decode-sized one): routing bit-exact on all tokens, quantised token rows bit-exact on a sample,
     the output of sampled tokens against the oracle, and run-to-run determinism."""
     cfg = CONFIGS[name]
     T, H, I, E, k = (cfg[n] for n in ("T", "H", "I", "E", "top_k"))

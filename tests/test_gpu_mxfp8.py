@@ -185,10 +185,12 @@ def test_mxfp8_forward_matches_oracle(T, H, I, E, k, skew):
     assert_close_out(bf16_to_f64(out), ref, "mxfp8 out")
 
 
-def test_mxfp8_local_experts():
-    cfg = dict(T=160, H=256, I=128, E=16, top_k=4, skew=False)
+@pytest.mark.parametrize("cfg,lo,n", [(dict(T=160, H=256, I=128, E=16, top_k=4, skew=False), 4, 8),
+                                      # wide token tiles (bound 384) with resident experts in the middle of the range
+                                      (dict(T=1200, H=256, I=128, E=8, top_k=2, skew=False), 2, 4),
+                                      (dict(T=1100, H=256, I=128, E=8, top_k=2, skew=True), 0, 3)])
+def test_mxfp8_local_experts(cfg, lo, n):
     full = make_mxfp8_inputs(cfg, seed=3, device="cuda")
-    lo, n = 4, 8
     inp = dict(full)
     for key in ("w13_q", "w13_s", "w2_q", "w2_s"):
         inp[key] = full[key][lo:lo + n].contiguous()
