@@ -206,7 +206,7 @@ int forward_impl(const void *x, const float *logits, const void *w13, const void
         if (st != MOE_OK) return st;
     }
     if (!mark(4)) return MOE_ERR_CUDA;
-    if (launch_combine(y, wts, f2s, T, k, H, static_cast<__nv_bfloat16 *>(out), stream) != cudaSuccess)
+    if (launch_combine(y, wts, f2s, T, k, H, static_cast<__nv_bfloat16 *>(out), stream, n_local < E) != cudaSuccess)
         return MOE_ERR_CUDA;
     if (!mark(5)) return MOE_ERR_CUDA;
     return MOE_OK;
@@ -337,7 +337,7 @@ int forward_mx_impl(const void *x, const float *logits, const void *w13_q, const
     st = run(g2);
     if (st != MOE_OK) return st;
     if (!mark(4)) return MOE_ERR_CUDA;
-    if (launch_combine(y, wts, f2s, T, k, H, static_cast<__nv_bfloat16 *>(out), stream) != cudaSuccess)
+    if (launch_combine(y, wts, f2s, T, k, H, static_cast<__nv_bfloat16 *>(out), stream, n_local < E) != cudaSuccess)
         return MOE_ERR_CUDA;
     if (!mark(5)) return MOE_ERR_CUDA;
     return MOE_OK;

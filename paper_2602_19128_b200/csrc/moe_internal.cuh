@@ -131,9 +131,11 @@ cudaError_t launch_route(const float *logits, int T, int E, int k, LocalExperts 
 cudaError_t launch_scatter_rows(const __nv_bfloat16 *x, const int *flat_to_sorted, int T, int k, int H, __nv_bfloat16 *x_perm,
                                 cudaStream_t stream);
 
-// out[t,:] = sum_j topk_w[t,j] * y[flat_to_sorted[t*k+j],:]
+// out[t,:] = sum_j topk_w[t,j] * y[flat_to_sorted[t*k+j],:] over the ranks with a row here (flat_to_sorted >= 0).
+// resident_subset: the call serves a subset of the experts, most ranks have no row: a kernel that takes several
+// tokens per block (same result).
 cudaError_t launch_combine(const __nv_bfloat16 *y, const float *topk_w, const int *flat_to_sorted, int T, int k,
-                           int H, __nv_bfloat16 *out, cudaStream_t stream);
+                           int H, __nv_bfloat16 *out, cudaStream_t stream, bool resident_subset = false);
 
 // Grouped GEMM over expert-contiguous rows, tcgen05 / TMEM / TMA.
 //   swiglu = true : act [A,K=H] x w [E,2I,H]  -> out [A,I]  = SiLU(gate) * up

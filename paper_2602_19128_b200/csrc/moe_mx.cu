@@ -83,6 +83,7 @@ mx_quantize_rows_kernel(const uint4 *__restrict__ x, const int *__restrict__ fla
         }
     }
     (void)n_local;
+    if (kScatter && !__any_sync(0xffffffffu, my_row >= 0)) return;  // none of the token's experts is resident here
     const uint4 *src = x + (size_t)r * vec_per_row;
     constexpr int kInFlight = 4;  // independent 16-byte loads per lane before the first is used
     const int n_segs = (vec_per_row + 31) / 32;

@@ -508,6 +508,7 @@ scatter_rows_kernel(const uint4 *__restrict__ x, const int *__restrict__ flat_to
     const int t = (int)(w / warps_per_token), part = (int)(w % warps_per_token);
     if (t >= T) return;
     const int my_row = lane < k ? flat_to_sorted[(size_t)t * k + lane] : -1;  // lane j holds rank j's destination
+    if (!__any_sync(kFullMask, my_row >= 0)) return;  // none of the token's experts is resident here: nothing to copy
     const uint4 *src = x + (size_t)t * vec_per_row;
     constexpr int kInFlight = 4;  // independent 16-byte loads per lane before the first is used
     const int stride = 32 * warps_per_token;
@@ -575,6 +576,80 @@ combine_kernel(const uint4 *__restrict__ y, const float *__restrict__ topk_w, co
     out[(size_t)t * vec_per_row + i] = o;
 }
 
+// The same sum for a layer with a resident subset of the experts, where most ranks of most tokens have no row here
+// (the paper's 32 of 256: one live rank per token on average).  There the kernel above has one 16-byte load in flight
+// per thread and is bound by the latency of that load (3.1 TB/s alone on the machine, 0.09 ms for 8192 tokens).
+// Here a block takes kSparseTokens consecutive tokens, lists their live (token, rank) pairs in order, and every
+// thread fetches up to kSparseBatch rows at once before it sums them, token after token, rank after rank: the
+// same order of summation, the same result, sixteen loads in flight.
+constexpr int kSparseTokens = 16, kSparseBatch = 16;
+__global__ void __launch_bounds__(kCombineThreads)
+combine_sparse_kernel(const uint4 *__restrict__ y, const float *__restrict__ topk_w, const int *__restrict__ flat_to_sorted,
+                      int T, int k, int vec_per_row, int blocks_per_group, uint4 *__restrict__ out) {
+    __shared__ int live_row[kSparseTokens * kMaxTopK], live_tok[kSparseTokens * kMaxTopK];
+    __shared__ float live_w[kSparseTokens * kMaxTopK];
+    __shared__ int n_live;
+    chain_release();
+    chain_wait();
+    const int group = blockIdx.x / blocks_per_group;
+    const int t0 = group * kSparseTokens, i = (blockIdx.x - group * blocks_per_group) * kCombineThreads + threadIdx.x;
+    const int n_tok = min(kSparseTokens, T - t0);
+    if (threadIdx.x < 32) {  // warp 0 compacts the live pairs, in (token, rank) order
+        int count = 0;
+        for (int e0 = 0; e0 < n_tok * k; e0 += 32) {
+            const int e = e0 + threadIdx.x;
+            const int row = e < n_tok * k ? flat_to_sorted[(size_t)t0 * k + e] : -1;
+            const unsigned mask = __ballot_sync(kFullMask, row >= 0);
+            if (row >= 0) {
+                const int at = count + __popc(mask & ((1u << threadIdx.x) - 1u));
+                live_row[at] = row;
+                live_tok[at] = e / k;
+                live_w[at] = topk_w[(size_t)t0 * k + e];
+            }
+            count += __popc(mask);
+        }
+        if (threadIdx.x == 0) n_live = count;
+    }
+    __syncthreads();
+    if (i >= vec_per_row) return;
+    const int L = n_live;
+    float acc[8];
+#pragma unroll
+    for (int c = 0; c < 8; ++c) acc[c] = 0.f;
+    int cur = 0;  // the token whose sum is in acc
+    auto flush = [&]() {
+        uint4 o;
+        __nv_bfloat162 *o2 = reinterpret_cast<__nv_bfloat162 *>(&o);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) o2[c] = __floats2bfloat162_rn(acc[2 * c], acc[2 * c + 1]);
+        out[(size_t)(t0 + cur) * vec_per_row + i] = o;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) acc[c] = 0.f;
+        ++cur;
+    };
+    for (int base = 0; base < L; base += kSparseBatch) {
+        uint4 v[kSparseBatch];
+#pragma unroll
+        for (int u = 0; u < kSparseBatch; ++u)
+            v[u] = base + u < L ? __ldcs(&y[(size_t)live_row[base + u] * vec_per_row + i]) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+        for (int u = 0; u < kSparseBatch; ++u) {
+            if (base + u >= L) break;  // (uniform over the block)
+            const int tok = live_tok[base + u];
+            while (cur < tok) flush();
+            const float wj = live_w[base + u];
+            const __nv_bfloat162 *h2 = reinterpret_cast<const __nv_bfloat162 *>(&v[u]);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const float2 f = __bfloat1622float2(h2[c]);
+                acc[2 * c] = fmaf(wj, f.x, acc[2 * c]);
+                acc[2 * c + 1] = fmaf(wj, f.y, acc[2 * c + 1]);
+            }
+        }
+    }
+    while (cur < n_tok) flush();
+}
+
 }  // namespace
 
 int choose_nt_max(int T, int E, int k, bool wide_ok) {
@@ -630,8 +705,14 @@ cudaError_t launch_scatter_rows(const __nv_bfloat16 *x, const int *flat_to_sorte
 }
 
 cudaError_t launch_combine(const __nv_bfloat16 *y, const float *topk_w, const int *flat_to_sorted, int T, int k,
-                           int H, __nv_bfloat16 *out, cudaStream_t stream) {
+                           int H, __nv_bfloat16 *out, cudaStream_t stream, bool resident_subset) {
     const int vec_per_row = H / 8, blocks_per_token = (vec_per_row + kCombineThreads - 1) / kCombineThreads;
+    if (resident_subset) {
+        const long long groups = ((long long)T + kSparseTokens - 1) / kSparseTokens;
+        return launch_chained(combine_sparse_kernel, (unsigned)(groups * blocks_per_token), kCombineThreads, 0, stream,
+                              reinterpret_cast<const uint4 *>(y), topk_w, flat_to_sorted, T, k, vec_per_row, blocks_per_token,
+                              reinterpret_cast<uint4 *>(out));
+    }
     return launch_chained(combine_kernel, (unsigned)((long long)T * blocks_per_token), kCombineThreads, 0, stream,
                           reinterpret_cast<const uint4 *>(y), topk_w, flat_to_sorted, k, vec_per_row, blocks_per_token,
                           reinterpret_cast<uint4 *>(out));
