@@ -265,3 +265,42 @@ def test_many_overlapping_calls_on_two_streams_complete(T, H, I, E, k):
     src = _OVERLAP.format(root=str(Path(__file__).resolve().parent.parent), T=T, H=H, I=I, E=E, k=k, groups=150)
     r = subprocess.run([sys.executable, "-c", src], capture_output=True, text=True, timeout=240)
     assert r.returncode == 0 and "overlap ok" in r.stdout, r.stderr[-2000:]
+
+
+_OVERLAP_MX = r"""
+import sys, torch
+sys.path.insert(0, {root!r})
+import paper_2602_19128_b200 as moe
+from tests.weight_quantizers import make_mxfp8_inputs
+cfg = dict(T={T}, H={H}, I={I}, E={E}, top_k={k}, skew=False)
+inp = make_mxfp8_inputs(cfg, seed=71, device="cuda")
+sf13, sf2 = moe.moe_mxfp8_pack_scales(inp["w13_s"], True), moe.moe_mxfp8_pack_scales(inp["w2_s"], False)
+ws = [moe.alloc_workspace(moe.moe_mxfp8_workspace_bytes({T}, {H}, {I}, {E}, {k}), "cuda") for _ in range(2)]
+outs = [torch.empty(({T}, {H}), dtype=torch.bfloat16, device="cuda") for _ in range(3)]
+def call(o, w, stream=None):
+    moe.moe_forward_mxfp8(inp["x"], inp["router_logits"], inp["w13_q"], sf13, inp["w2_q"], sf2, {k}, o, w, stream=stream)
+call(outs[2], ws[0])
+torch.cuda.synchronize()
+streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+for it in range({groups}):
+    for i in range(20):
+        call(outs[i % 2], ws[i % 2], streams[i % 2])
+    torch.cuda.synchronize()
+for i in range(2):
+    assert moe.moe_last_status(ws[i], stream=streams[i]) == 0
+    assert torch.equal(outs[i].view(torch.int16), outs[2].view(torch.int16))
+print("overlap ok")
+"""
+
+
+def test_many_overlapping_mxfp8_calls_on_two_streams_complete():
+    """The same stress for the MX FP8 layer on its wide-tile kernel (304-row bound), which also takes a whole SM's
+    shared memory: a child process with a time limit."""
+    import subprocess
+    import sys
+    from pathlib import Path
+    T, H, I, E, k = 2048, 512, 256, 64, 8
+    assert moe.moe_mxfp8_workspace_layout(T, H, I, E, k).tile_rows == 304
+    src = _OVERLAP_MX.format(root=str(Path(__file__).resolve().parent.parent), T=T, H=H, I=I, E=E, k=k, groups=100)
+    r = subprocess.run([sys.executable, "-c", src], capture_output=True, text=True, timeout=240)
+    assert r.returncode == 0 and "overlap ok" in r.stdout, r.stderr[-2000:]
